@@ -1,0 +1,206 @@
+/*
+ * cachescout.h -- C ABI of the B200 (sm_100a) hot path of an agent-aware KV-cache layer:
+ * the batched cache-management step (online agent-transition model, per-block reuse score,
+ * eviction-victim and prefetch-candidate selection) and the paged-KV block mover that
+ * carries the decisions out between a paged GPU pool and a pinned host tier.
+ *
+ * General rules
+ *  - Every function returns an int: CS_OK (0) or a negative CS_E* code.  Nothing throws,
+ *    aborts or prints.
+ *  - Calls ENQUEUE work on the given CUDA stream and return; outputs are valid once that
+ *    stream has been synchronised.  Only cs_get_status() synchronises.
+ *  - "dev" pointers are caller-owned device memory, "pinned" pointers caller-owned
+ *    page-locked host memory that the device can address (cudaHostAlloc /
+ *    cudaHostRegister; with unified addressing the host pointer is used as is).  The
+ *    library never allocates or frees device or pinned memory; it owns only the small
+ *    host-side cs_ctx.  All scratch lives in the workspace the caller hands to cs_create().
+ *  - Every array pointer must be 16-byte aligned (the kernels use 128-bit accesses);
+ *    a violation is CS_EINVAL before anything is launched.
+ *  - All calls on one cs_ctx except the three mover calls share workspace scratch: issue
+ *    them on one stream (or order them with events).  The mover calls touch no workspace
+ *    scratch besides the status word and may run on a side stream concurrently.
+ *  - Bad ids inside device arrays (agent >= n_agents, chain >= n_chains, slot >= n_slots)
+ *    are detected in the kernels: the entry is skipped and a bit is set in the device
+ *    status word (read with cs_get_status()).  Kernels never trap or spin unboundedly.
+ */
+#ifndef CACHESCOUT_H
+#define CACHESCOUT_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct cs_ctx cs_ctx;
+typedef struct CUstream_st *cs_stream_t;   /* the same type as cudaStream_t */
+
+/* ---- return codes ---------------------------------------------------------------- */
+#define CS_OK 0
+#define CS_EINVAL (-1)          /* bad argument (NULL, misaligned, inconsistent sizes) */
+#define CS_ECAPACITY (-2)       /* n_blocks or k beyond what the workspace was sized for */
+#define CS_ENOTIMPL (-3)
+#define CS_ECUDA (-4)           /* a CUDA runtime call failed; see cs_last_cuda_error() */
+#define CS_EDEVICE_STATUS (-5)  /* cs_get_status(): the device status word was non-zero */
+#define CS_ENOMEM (-6)          /* host allocation of the context failed */
+
+/* ---- device status word bits (cs_get_status) ---------------------------------------- */
+#define CS_ST_BAD_AGENT 1u      /* an event or index entry named an agent >= n_agents */
+#define CS_ST_BAD_CHAIN 2u      /* an event named a chain >= n_chains */
+#define CS_ST_BAD_SLOT 4u       /* a mover list entry named a slot >= n_slots */
+#define CS_ST_BAD_SOURCE 8u     /* a BFS source >= n_agents */
+
+/* ---- sentinels ---------------------------------------------------------------------------- */
+#define CS_AGENT_NONE 0xFFFFu      /* "no current agent yet" (the initial state of Algorithm 1) */
+#define CS_ID_NONE 0xFFFFFFFFu     /* padding of id lists; skipped by the mover */
+#define CS_HOP_NONE 0xFFFFu        /* unreachable in the execution graph */
+
+/* ---- block-index flag bits ------------------------------------------------------------------ */
+#define CS_FLAG_VALID 1u
+#define CS_FLAG_PINNED 2u
+#define CS_FLAG_TIER_HOST 4u
+#define CS_FLAG_OTHER_COPY 8u      /* the block's contents also exist on the other tier */
+
+#define CS_EV_WARMUP 1u            /* event flag: warmup request, excluded from learning (Sec. 4) */
+
+#define CS_LAYER_MAJOR 0u
+#define CS_BLOCK_MAJOR 1u
+
+#define CS_MAX_AGENTS 1024u
+
+/* Constants of the method (Algorithm 1 state; Eq. 3, 7, 8, 9, 11).  The paper names them
+ * without values; the defaults used by the tests are eps 0.01, tau 0.05, e_max 4,
+ * lambda 0.01 per scheduler step, delta 0.01, r_min 0.3. */
+typedef struct cs_params {
+    uint32_t n_agents;      /* A: 1 .. CS_MAX_AGENTS; Eq. 3's sum runs over all A slots */
+    uint32_t n_chains;      /* independent "current agent" registers; 1 = the paper's single a_t */
+    uint32_t max_blocks;    /* largest n_blocks / k any select call will use */
+    uint32_t block_tokens;  /* |b| of a full block (1..255), used when n_tokens is NULL */
+    uint32_t e_max;         /* E_max of Eq. 8, >= 1 */
+    float eps;              /* smoothing constant of Eq. 3, > 0 */
+    float tau;              /* confidence threshold of Eq. 7 */
+    float lambda;           /* recency decay rate of Eq. 9, >= 0 */
+    float delta;            /* floor of Eq. 9, > 0 */
+    float r_min;            /* prefetch gate of Eq. 11 */
+} cs_params;
+
+/* Structure-of-arrays metadata of the cached blocks (all dev, each [n_blocks] unless
+ * noted).  Entry i describes block id i. */
+typedef struct cs_block_index {
+    uint32_t n_blocks;
+    const uint16_t *agent;          /* owning agent (agentOf[] of Algorithm 1) */
+    const uint16_t *depth;          /* position of the block in its prompt */
+    const uint8_t *ref_count;       /* in use by running requests when > 0 */
+    const uint8_t *flags;           /* CS_FLAG_* */
+    const uint32_t *last_access;    /* scheduler step of the last touch (lastAccess[]) */
+    const uint8_t *n_tokens;        /* tokens cached per block, or NULL = block_tokens */
+    const uint16_t *anchor_blocks;  /* [n_agents] length of each agent's fixed context in
+                                       blocks, or NULL = no depth restriction on prefetch */
+} cs_block_index;
+
+/* A paged KV pool.  One chunk = block_tokens*n_kv_heads*head_dim*elem_bytes bytes holds one
+ * layer, one of K/V, one block ([token][head][dim] inside).  Byte offset of the chunk of
+ * layer l, plane p (0 = K, 1 = V), slot s:
+ *   CS_LAYER_MAJOR: ((l*2 + p)*n_slots + s) * chunk_bytes
+ *   CS_BLOCK_MAJOR: ((s*n_layers + l)*2 + p) * chunk_bytes
+ * base is dev or pinned; chunk_bytes must be a multiple of 16. */
+typedef struct cs_kv_pool {
+    void *base;
+    uint32_t n_slots, layout, n_layers, n_kv_heads, head_dim, block_tokens, elem_bytes;
+} cs_kv_pool;
+
+/* ---- life cycle -------------------------------------------------------------------------------- */
+
+/* Bytes of device workspace cs_create() needs for these parameters (host call, no CUDA). */
+int cs_workspace_bytes(const cs_params *p, size_t *dev_bytes);
+
+/* Creates a context on the current device over caller-owned `dev_workspace` (256-byte
+ * aligned, >= cs_workspace_bytes()).  Enqueues the initialisation on `init_stream`: zero
+ * counts, no current agent, the uniform Eq. 3 matrix, the recency table of Eq. 9.
+ * The workspace must outlive the context; cs_destroy() frees only the host struct. */
+int cs_create(const cs_params *p, void *dev_workspace, size_t bytes, cs_stream_t init_stream,
+              cs_ctx **out);
+int cs_destroy(cs_ctx *ctx);
+
+/* ---- cache-management step ----------------------------------------------------------------------- */
+
+/* Transition Learner (Sec. 3.2; Algorithm 1, ObserveTouch).  For the events in order, per
+ * chain c: if a current agent exists and differs from the event's agent, C[cur][agent] += 1;
+ * then cur[c] = agent.  Events with CS_EV_WARMUP are ignored.  After the batch the call
+ * refreshes everything derived from the counts: the smoothed matrix of Eq. 3, each row's
+ * arg-max (Eq. 5 / Eq. 10, lowest index among equal maxima), the predictability R of Eq. 2
+ * with the gate of Eq. 11, the threshold graph of Eq. 7, and -- from the agent of the last
+ * non-warmup event -- the BFS hop table and the survival scores of Eq. 8.
+ * chain, agent, evflags: dev [n_events]; evflags may be NULL.  n_events may be 0 (refresh only). */
+int cs_observe_invocations(cs_ctx *ctx, const uint32_t *chain, const uint16_t *agent,
+                           const uint8_t *evflags, uint32_t n_events, cs_stream_t stream);
+
+/* ScoreBlock of Algorithm 1 / Eq. 9 for every index entry:
+ *   score = (p~(agent) + delta) * (exp(-lambda * age) + delta) * |b|,  age = now - last_access
+ * (0 when last_access > now).  fp32, each product rounded once.  sources == NULL uses the
+ * survival table cached by the last cs_observe_invocations(); otherwise a BFS from the given
+ * agents (dev [n_sources]) is run first and used for this call only.
+ * scores_out: dev [n_blocks]; entries whose agent is out of range get 0. */
+int cs_score_blocks(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, const uint16_t *sources,
+                    uint32_t n_sources, float *scores_out, cs_stream_t stream);
+
+/* Evict of Algorithm 1, k times over: the k eligible entries with the lowest
+ * (score, last_access, id), in ascending order.  Eligible: VALID, not PINNED, ref_count 0,
+ * TIER_HOST bit == tier (0 GPU, 1 host).  ids_out: dev [k], padded with CS_ID_NONE;
+ * n_out: dev, = min(k, number eligible).  k <= max_blocks. */
+int cs_select_victims(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, uint32_t tier, uint32_t k,
+                      uint32_t *ids_out, uint32_t *n_out, cs_stream_t stream);
+
+/* BetweenStep of Algorithm 1 with Eq. 10-11, at block level: empty unless R >= r_min and a
+ * current agent exists.  a* = arg-max row of the current agent.  Eligible: VALID, not
+ * PINNED, ref_count 0, on the host tier, no copy on the GPU tier, and depth <
+ * anchor_blocks[agent] when that table is given.  Order: blocks of a* first, then score
+ * descending, last_access descending, id ascending.  Outputs as for cs_select_victims(). */
+int cs_select_prefetch(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, uint32_t k,
+                       uint32_t *ids_out, uint32_t *n_out, cs_stream_t stream);
+
+/* ---- block mover (the paper reuses the serving engine's offload path, Sec. 4; these calls
+ *      are that path written for B200) ------------------------------------------------------------ */
+
+/* For i < n (n = min(n_max, *n_dev) when n_dev != NULL, else n_max), every layer and both
+ * planes: copy the chunk of src slot src_slots[i] to dst slot dst_slots[i].  Entries with
+ * CS_ID_NONE on either side are skipped.  src_slots / dst_slots / n_dev: dev.  The two pools
+ * must agree in everything but base, n_slots and layout.  Destination slots must be distinct;
+ * when src and dst are the same pool the two slot sets must be disjoint (not checked). */
+int cs_offload_blocks(cs_ctx *ctx, const cs_kv_pool *gpu, const cs_kv_pool *host, const uint32_t *src_slots,
+                      const uint32_t *dst_slots, uint32_t n_max, const uint32_t *n_dev, cs_stream_t side);
+int cs_prefetch_blocks(cs_ctx *ctx, const cs_kv_pool *host, const cs_kv_pool *gpu, const uint32_t *src_slots,
+                       const uint32_t *dst_slots, uint32_t n_max, const uint32_t *n_dev, cs_stream_t side);
+int cs_compact_blocks(cs_ctx *ctx, const cs_kv_pool *src, const cs_kv_pool *dst, const uint32_t *src_slots,
+                      const uint32_t *dst_slots, uint32_t n_max, const uint32_t *n_dev, cs_stream_t stream);
+
+/* ---- inspection ------------------------------------------------------------------------------------ */
+
+/* Copies the learner / scorer state into caller dev buffers (any may be NULL):
+ * C [A*A] counts, P [A*A] Eq. 3, amax [A], hops [A] (CS_HOP_NONE = unreachable), fsurv [A]
+ * (= p~ + delta), R [1], cur [n_chains], last_agent [1]. */
+int cs_get_model(cs_ctx *ctx, uint32_t *C_out, float *P_out, uint16_t *amax_out, uint16_t *hops_out,
+                 float *fsurv_out, float *R_out, uint16_t *cur_out, uint16_t *last_agent_out,
+                 cs_stream_t stream);
+
+/* Synchronises `stream`, returns the device status word in *device_status and clears it.
+ * Returns CS_EDEVICE_STATUS when it was non-zero. */
+int cs_get_status(cs_ctx *ctx, uint32_t *device_status, cs_stream_t stream);
+
+/* Number of kernels this context has launched so far (host counter). */
+int cs_launch_count(cs_ctx *ctx, uint64_t *n_launches);
+
+/* Grid sizes of the mover (0 keeps the default): CTAs used for transfers that cross the
+ * host link, and for device-to-device moves. */
+int cs_set_mover_ctas(cs_ctx *ctx, uint32_t host_link_ctas, uint32_t d2d_ctas);
+
+/* cudaError_t of the last failing CUDA call on this context (0 if none). */
+int cs_last_cuda_error(cs_ctx *ctx);
+const char *cs_strerror(int code);
+int cs_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CACHESCOUT_H */

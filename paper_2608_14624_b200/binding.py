@@ -1,0 +1,354 @@
+"""Thin Python binding of libcachescout (argument marshalling only).
+
+Every ``cs_*`` function below calls the C function of the same name declared in
+``include/cachescout.h``; all arithmetic runs in the CUDA kernels.  PyTorch is used for
+device memory, pinned memory and streams only.  There is no CPU fallback: if the shared
+library is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass, field
+from typing import Optional
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "libcachescout.so")
+
+CS_OK = 0
+CS_EINVAL, CS_ECAPACITY, CS_ENOTIMPL, CS_ECUDA, CS_EDEVICE_STATUS, CS_ENOMEM = -1, -2, -3, -4, -5, -6
+CS_ST_BAD_AGENT, CS_ST_BAD_CHAIN, CS_ST_BAD_SLOT, CS_ST_BAD_SOURCE = 1, 2, 4, 8
+CS_AGENT_NONE, CS_ID_NONE, CS_HOP_NONE = 0xFFFF, 0xFFFFFFFF, 0xFFFF
+CS_FLAG_VALID, CS_FLAG_PINNED, CS_FLAG_TIER_HOST, CS_FLAG_OTHER_COPY = 1, 2, 4, 8
+CS_EV_WARMUP = 1
+CS_LAYER_MAJOR, CS_BLOCK_MAJOR = 0, 1
+
+# every symbol include/cachescout.h declares
+EXPORTS = ("cs_workspace_bytes", "cs_create", "cs_destroy", "cs_observe_invocations", "cs_score_blocks",
+           "cs_select_victims", "cs_select_prefetch", "cs_offload_blocks", "cs_prefetch_blocks",
+           "cs_compact_blocks", "cs_get_model", "cs_get_status", "cs_launch_count", "cs_set_mover_ctas",
+           "cs_last_cuda_error", "cs_strerror", "cs_version")
+
+
+class cs_params(C.Structure):
+    _fields_ = [("n_agents", C.c_uint32), ("n_chains", C.c_uint32), ("max_blocks", C.c_uint32),
+                ("block_tokens", C.c_uint32), ("e_max", C.c_uint32), ("eps", C.c_float), ("tau", C.c_float),
+                ("lambda_", C.c_float), ("delta", C.c_float), ("r_min", C.c_float)]
+
+
+class cs_block_index(C.Structure):
+    _fields_ = [("n_blocks", C.c_uint32), ("agent", C.c_void_p), ("depth", C.c_void_p), ("ref_count", C.c_void_p),
+                ("flags", C.c_void_p), ("last_access", C.c_void_p), ("n_tokens", C.c_void_p),
+                ("anchor_blocks", C.c_void_p)]
+
+
+class cs_kv_pool(C.Structure):
+    _fields_ = [("base", C.c_void_p), ("n_slots", C.c_uint32), ("layout", C.c_uint32), ("n_layers", C.c_uint32),
+                ("n_kv_heads", C.c_uint32), ("head_dim", C.c_uint32), ("block_tokens", C.c_uint32),
+                ("elem_bytes", C.c_uint32)]
+
+
+class CacheScoutError(RuntimeError):
+    def __init__(self, code: int, where: str, extra: str = ""):
+        self.code = code
+        msg = "%s: %s (%d)%s" % (where, lib().cs_strerror(code).decode(), code, extra)
+        super().__init__(msg)
+
+
+_lib = None
+
+
+def lib():
+    """Loads libcachescout.so (building is the job of ``build.build_library``); never falls back."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError("libcachescout.so is missing: build it with "
+                               "`python -m paper_2608_14624_b200.build` (there is no CPU fallback)")
+        L = C.CDLL(LIB_PATH)
+        L.cs_strerror.restype = C.c_char_p
+        L.cs_strerror.argtypes = [C.c_int]
+        vp, u32 = C.c_void_p, C.c_uint32
+        L.cs_workspace_bytes.argtypes = [C.POINTER(cs_params), C.POINTER(C.c_size_t)]
+        L.cs_create.argtypes = [C.POINTER(cs_params), vp, C.c_size_t, vp, C.POINTER(vp)]
+        L.cs_destroy.argtypes = [vp]
+        L.cs_observe_invocations.argtypes = [vp, vp, vp, vp, u32, vp]
+        L.cs_score_blocks.argtypes = [vp, C.POINTER(cs_block_index), u32, vp, u32, vp, vp]
+        L.cs_select_victims.argtypes = [vp, C.POINTER(cs_block_index), u32, u32, u32, vp, vp, vp]
+        L.cs_select_prefetch.argtypes = [vp, C.POINTER(cs_block_index), u32, u32, vp, vp, vp]
+        for name in ("cs_offload_blocks", "cs_prefetch_blocks", "cs_compact_blocks"):
+            getattr(L, name).argtypes = [vp, C.POINTER(cs_kv_pool), C.POINTER(cs_kv_pool), vp, vp, u32, vp, vp]
+        L.cs_get_model.argtypes = [vp] * 10
+        L.cs_get_status.argtypes = [vp, C.POINTER(u32), vp]
+        L.cs_launch_count.argtypes = [vp, C.POINTER(C.c_uint64)]
+        L.cs_set_mover_ctas.argtypes = [vp, u32, u32]
+        L.cs_last_cuda_error.argtypes = [vp]
+        _lib = L
+    return _lib
+
+
+def _ptr(t) -> Optional[int]:
+    """Device (or pinned host) address of a tensor, None for None, ints pass through."""
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    return t.data_ptr()
+
+
+def _stream(s) -> Optional[int]:
+    if s is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream
+    if isinstance(s, int):
+        return s
+    return s.cuda_stream
+
+
+def _chk(code: int, where: str, ctx=None):
+    if code != CS_OK:
+        extra = ""
+        if code == CS_ECUDA and ctx:
+            extra = " [cudaError %d]" % lib().cs_last_cuda_error(ctx)
+        raise CacheScoutError(code, where, extra)
+
+
+# ---- the C-ABI, one Python function per exported call -----------------------------------------------
+def cs_workspace_bytes(params: cs_params) -> int:
+    n = C.c_size_t(0)
+    _chk(lib().cs_workspace_bytes(C.byref(params), C.byref(n)), "cs_workspace_bytes")
+    return int(n.value)
+
+
+def cs_create(params: cs_params, workspace, stream=None) -> int:
+    ctx = C.c_void_p()
+    _chk(lib().cs_create(C.byref(params), _ptr(workspace), workspace.numel() * workspace.element_size(),
+                         _stream(stream), C.byref(ctx)), "cs_create")
+    return ctx.value
+
+
+def cs_destroy(ctx: int):
+    _chk(lib().cs_destroy(ctx), "cs_destroy")
+
+
+def cs_observe_invocations(ctx, chain, agent, evflags, n_events: int, stream=None):
+    _chk(lib().cs_observe_invocations(ctx, _ptr(chain), _ptr(agent), _ptr(evflags), n_events, _stream(stream)),
+         "cs_observe_invocations", ctx)
+
+
+def cs_score_blocks(ctx, idx: cs_block_index, now: int, sources, n_sources: int, scores_out, stream=None):
+    _chk(lib().cs_score_blocks(ctx, C.byref(idx), now, _ptr(sources), n_sources, _ptr(scores_out), _stream(stream)),
+         "cs_score_blocks", ctx)
+
+
+def cs_select_victims(ctx, idx: cs_block_index, now: int, tier: int, k: int, ids_out, n_out, stream=None):
+    _chk(lib().cs_select_victims(ctx, C.byref(idx), now, tier, k, _ptr(ids_out), _ptr(n_out), _stream(stream)),
+         "cs_select_victims", ctx)
+
+
+def cs_select_prefetch(ctx, idx: cs_block_index, now: int, k: int, ids_out, n_out, stream=None):
+    _chk(lib().cs_select_prefetch(ctx, C.byref(idx), now, k, _ptr(ids_out), _ptr(n_out), _stream(stream)),
+         "cs_select_prefetch", ctx)
+
+
+def cs_offload_blocks(ctx, gpu: cs_kv_pool, host: cs_kv_pool, src_slots, dst_slots, n_max: int, n_dev=None, stream=None):
+    _chk(lib().cs_offload_blocks(ctx, C.byref(gpu), C.byref(host), _ptr(src_slots), _ptr(dst_slots), n_max,
+                                 _ptr(n_dev), _stream(stream)), "cs_offload_blocks", ctx)
+
+
+def cs_prefetch_blocks(ctx, host: cs_kv_pool, gpu: cs_kv_pool, src_slots, dst_slots, n_max: int, n_dev=None, stream=None):
+    _chk(lib().cs_prefetch_blocks(ctx, C.byref(host), C.byref(gpu), _ptr(src_slots), _ptr(dst_slots), n_max,
+                                  _ptr(n_dev), _stream(stream)), "cs_prefetch_blocks", ctx)
+
+
+def cs_compact_blocks(ctx, src: cs_kv_pool, dst: cs_kv_pool, src_slots, dst_slots, n_max: int, n_dev=None, stream=None):
+    _chk(lib().cs_compact_blocks(ctx, C.byref(src), C.byref(dst), _ptr(src_slots), _ptr(dst_slots), n_max,
+                                 _ptr(n_dev), _stream(stream)), "cs_compact_blocks", ctx)
+
+
+def cs_get_model(ctx, C_out=None, P_out=None, amax_out=None, hops_out=None, fsurv_out=None, R_out=None,
+                 cur_out=None, last_agent_out=None, stream=None):
+    _chk(lib().cs_get_model(ctx, _ptr(C_out), _ptr(P_out), _ptr(amax_out), _ptr(hops_out), _ptr(fsurv_out),
+                            _ptr(R_out), _ptr(cur_out), _ptr(last_agent_out), _stream(stream)), "cs_get_model", ctx)
+
+
+def cs_get_status(ctx, stream=None, raise_on_set: bool = False) -> int:
+    st = C.c_uint32(0)
+    code = lib().cs_get_status(ctx, C.byref(st), _stream(stream))
+    if code not in (CS_OK, CS_EDEVICE_STATUS) or (raise_on_set and code != CS_OK):
+        _chk(code, "cs_get_status", ctx)
+    return int(st.value)
+
+
+def cs_launch_count(ctx) -> int:
+    n = C.c_uint64(0)
+    _chk(lib().cs_launch_count(ctx, C.byref(n)), "cs_launch_count")
+    return int(n.value)
+
+
+def cs_set_mover_ctas(ctx, host_link_ctas: int, d2d_ctas: int):
+    _chk(lib().cs_set_mover_ctas(ctx, host_link_ctas, d2d_ctas), "cs_set_mover_ctas")
+
+
+def cs_version() -> int:
+    return int(lib().cs_version())
+
+
+# ---- small holders that keep tensors alive next to the structs that point into them ---------------------
+def make_params(n_agents: int, n_chains: int = 1, max_blocks: int = 1, block_tokens: int = 16, e_max: int = 4,
+                eps: float = 0.01, tau: float = 0.05, lam: float = 0.01, delta: float = 0.01,
+                r_min: float = 0.3) -> cs_params:
+    return cs_params(n_agents, n_chains, max_blocks, block_tokens, e_max, eps, tau, lam, delta, r_min)
+
+
+@dataclass
+class DeviceIndex:
+    """SoA block metadata on the device (torch tensors) plus the struct the C calls take."""
+    agent: object
+    depth: object
+    ref_count: object
+    flags: object
+    last_access: object
+    n_tokens: object = None
+    anchor_blocks: object = None
+
+    @classmethod
+    def from_host(cls, idx, device="cuda:0"):
+        import torch
+        up = lambda a: None if a is None else torch.from_numpy(a).to(device)
+        return cls(up(idx.agent), up(idx.depth), up(idx.ref_count), up(idx.flags), up(idx.last_access),
+                   up(idx.n_tokens), up(idx.anchor_blocks))
+
+    @property
+    def n(self) -> int:
+        return int(self.agent.numel())
+
+    def struct(self) -> cs_block_index:
+        return cs_block_index(self.n, _ptr(self.agent), _ptr(self.depth), _ptr(self.ref_count), _ptr(self.flags),
+                              _ptr(self.last_access), _ptr(self.n_tokens), _ptr(self.anchor_blocks))
+
+
+@dataclass
+class KVPool:
+    """A paged KV pool: flat tensor (device, or pinned host) + geometry."""
+    buf: object
+    n_slots: int
+    layout: int
+    n_layers: int
+    n_kv_heads: int = 8
+    head_dim: int = 128
+    block_tokens: int = 16
+    elem_bytes: int = 2
+
+    @property
+    def chunk_bytes(self) -> int:
+        return self.block_tokens * self.n_kv_heads * self.head_dim * self.elem_bytes
+
+    @property
+    def block_bytes(self) -> int:
+        return self.n_layers * 2 * self.chunk_bytes
+
+    def struct(self) -> cs_kv_pool:
+        assert self.buf.numel() * self.buf.element_size() >= self.n_slots * self.block_bytes
+        return cs_kv_pool(_ptr(self.buf), self.n_slots, self.layout, self.n_layers, self.n_kv_heads, self.head_dim,
+                          self.block_tokens, self.elem_bytes)
+
+
+class CacheScout:
+    """One context: owns the torch workspace tensor and forwards to the cs_* calls."""
+
+    def __init__(self, params: cs_params, device="cuda:0", stream=None):
+        import torch
+        if not torch.cuda.is_available():
+            raise RuntimeError("CacheScout needs a CUDA device (sm_100a); there is no CPU fallback")
+        self.params = params
+        self.device = torch.device(device)
+        with torch.cuda.device(self.device):
+            self.workspace = torch.empty(cs_workspace_bytes(params) + 256, dtype=torch.uint8, device=self.device)
+            self.ctx = cs_create(params, self.workspace, stream)
+
+    def close(self):
+        if getattr(self, "ctx", None):
+            cs_destroy(self.ctx)
+            self.ctx = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- calls ---------------------------------------------------------------------------------------
+    def observe_invocations(self, chain, agent, evflags=None, n_events=None, stream=None):
+        n = int(agent.numel()) if n_events is None and agent is not None else int(n_events or 0)
+        cs_observe_invocations(self.ctx, chain, agent, evflags, n, stream)
+
+    def score_blocks(self, idx: DeviceIndex, now: int, sources=None, out=None, stream=None):
+        import torch
+        if out is None:
+            out = torch.empty(idx.n, dtype=torch.float32, device=self.device)
+        cs_score_blocks(self.ctx, idx.struct(), now, sources, 0 if sources is None else int(sources.numel()), out, stream)
+        return out
+
+    def select_victims(self, idx: DeviceIndex, now: int, tier: int, k: int, ids_out=None, n_out=None, stream=None):
+        import torch
+        if ids_out is None:
+            ids_out = torch.empty(max(k, 4), dtype=torch.int32, device=self.device)
+        if n_out is None:
+            n_out = torch.empty(1, dtype=torch.int32, device=self.device)
+        cs_select_victims(self.ctx, idx.struct(), now, tier, k, ids_out, n_out, stream)
+        return ids_out, n_out
+
+    def select_prefetch(self, idx: DeviceIndex, now: int, k: int, ids_out=None, n_out=None, stream=None):
+        import torch
+        if ids_out is None:
+            ids_out = torch.empty(max(k, 4), dtype=torch.int32, device=self.device)
+        if n_out is None:
+            n_out = torch.empty(1, dtype=torch.int32, device=self.device)
+        cs_select_prefetch(self.ctx, idx.struct(), now, k, ids_out, n_out, stream)
+        return ids_out, n_out
+
+    def offload_blocks(self, gpu: KVPool, host: KVPool, src_slots, dst_slots, n_max=None, n_dev=None, stream=None):
+        cs_offload_blocks(self.ctx, gpu.struct(), host.struct(), src_slots, dst_slots,
+                          int(src_slots.numel()) if n_max is None else n_max, n_dev, stream)
+
+    def prefetch_blocks(self, host: KVPool, gpu: KVPool, src_slots, dst_slots, n_max=None, n_dev=None, stream=None):
+        cs_prefetch_blocks(self.ctx, host.struct(), gpu.struct(), src_slots, dst_slots,
+                           int(src_slots.numel()) if n_max is None else n_max, n_dev, stream)
+
+    def compact_blocks(self, src: KVPool, dst: KVPool, src_slots, dst_slots, n_max=None, n_dev=None, stream=None):
+        cs_compact_blocks(self.ctx, src.struct(), dst.struct(), src_slots, dst_slots,
+                          int(src_slots.numel()) if n_max is None else n_max, n_dev, stream)
+
+    def get_model(self, stream=None) -> dict:
+        """Copies of the learner / scorer state as host NumPy arrays (synchronises)."""
+        import torch
+        A, nc = self.params.n_agents, self.params.n_chains
+        dev = self.device
+        out = dict(C=torch.empty(A * A, dtype=torch.int32, device=dev), P=torch.empty(A * A, dtype=torch.float32, device=dev),
+                   amax=torch.empty(A + 8, dtype=torch.int16, device=dev), hops=torch.empty(A + 8, dtype=torch.int16, device=dev),
+                   fsurv=torch.empty(A, dtype=torch.float32, device=dev), R=torch.empty(1, dtype=torch.float32, device=dev),
+                   cur=torch.empty(nc + 8, dtype=torch.int16, device=dev), last_agent=torch.empty(8, dtype=torch.int16, device=dev))
+        cs_get_model(self.ctx, out["C"], out["P"], out["amax"], out["hops"], out["fsurv"], out["R"], out["cur"],
+                     out["last_agent"], stream)
+        torch.cuda.synchronize(dev)
+        import numpy as np
+        res = {}
+        res["C"] = out["C"].cpu().numpy().view(np.uint32).reshape(A, A)
+        res["P"] = out["P"].cpu().numpy().reshape(A, A)
+        res["amax"] = out["amax"].cpu().numpy().view(np.uint16)[:A]
+        res["hops"] = out["hops"].cpu().numpy().view(np.uint16)[:A]
+        res["fsurv"] = out["fsurv"].cpu().numpy()
+        res["R"] = float(out["R"].item())
+        res["cur"] = out["cur"].cpu().numpy().view(np.uint16)[:nc]
+        res["last_agent"] = int(out["last_agent"].cpu().numpy().view(np.uint16)[0])
+        return res
+
+    def get_status(self, stream=None) -> int:
+        return cs_get_status(self.ctx, stream)
+
+    def launch_count(self) -> int:
+        return cs_launch_count(self.ctx)
+
+    def set_mover_ctas(self, host_link_ctas: int = 0, d2d_ctas: int = 0):
+        cs_set_mover_ctas(self.ctx, host_link_ctas, d2d_ctas)

@@ -1,0 +1,306 @@
+// C-ABI entry points: argument validation, workspace layout, context life cycle.
+// All device work is in cs_model.cu, cs_select.cu and cs_mover.cu.
+#include <math.h>
+#include <new>
+#include <string.h>
+
+#include "cs_common.cuh"
+
+static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+static inline bool aligned16(const void *p) { return (((uintptr_t)p) & 15u) == 0; }
+
+int cs_validate_params(const cs_params *p)
+{
+    if (!p) return CS_EINVAL;
+    if (p->n_agents < 1 || p->n_agents > CS_MAX_AGENTS) return CS_EINVAL;
+    if (p->n_chains < 1 || p->n_chains > (1u << 24)) return CS_EINVAL;
+    if (p->max_blocks < 1) return CS_EINVAL;
+    if (p->block_tokens < 1 || p->block_tokens > 255) return CS_EINVAL;
+    if (p->e_max < 1 || p->e_max > 0xFFFEu) return CS_EINVAL;
+    if (!(p->eps > 0.0f) || !isfinite(p->eps)) return CS_EINVAL;       // Eq. 3 is 0/0 on a cold row otherwise
+    if (!isfinite(p->tau)) return CS_EINVAL;
+    if (!(p->lambda >= 0.0f) || !isfinite(p->lambda)) return CS_EINVAL;
+    if (!(p->delta > 0.0f) || !isfinite(p->delta)) return CS_EINVAL;    // the floor keeps both factors positive
+    if (!isfinite(p->r_min)) return CS_EINVAL;
+    return CS_OK;
+}
+
+// exp(-lambda*age) <= delta * 2^-26 cannot change f32(exp(..) + delta): from that age on the
+// recency factor is the constant f32(delta)-rounded value, so only younger ages need a table.
+void cs_recency_table_shape(const cs_params *p, uint32_t *gtab_len, uint32_t *age_sat)
+{
+    double sat;
+    if (p->lambda > 0.0f) sat = ceil((26.0 * log(2.0) - log((double)p->delta)) / (double)p->lambda) + 1.0;
+    else sat = 1.0;                                   // lambda = 0: the factor is constant from age 0
+    if (sat < 1.0) sat = 1.0;
+    if (sat > 4294967295.0) sat = 4294967295.0;
+    *age_sat = (uint32_t)sat;
+    *gtab_len = *age_sat < CS_GTAB_MAX ? *age_sat : CS_GTAB_MAX;
+}
+
+size_t cs_layout_workspace(const cs_params *p, uint32_t gtab_len, void *base, cs_workspace *ws)
+{
+    const size_t A = p->n_agents, W = (A + 31) / 32, N = p->max_blocks;
+    size_t off = 0;
+    char *b = (char *)base;
+#define TAKE(field, type, count)                                  \
+    do {                                                          \
+        if (ws) ws->field = (type *)(b + off);                    \
+        off = align_up(off + sizeof(type) * (size_t)(count), 256); \
+    } while (0)
+    TAKE(sc, cs_scalars, 1);
+    TAKE(C, uint32_t, A * A);
+    TAKE(rowsum, uint32_t, A);
+    TAKE(cur, uint16_t, p->n_chains);
+    TAKE(P, float, A * A);
+    TAKE(amax, uint16_t, A);
+    TAKE(rowH, double, A);
+    TAKE(adj, uint32_t, A * W);
+    TAKE(hops, uint16_t, A);
+    TAKE(fsurv, float, A);
+    TAKE(hops_tmp, uint16_t, A);
+    TAKE(fsurv_tmp, float, A);
+    TAKE(gtab, float, gtab_len);
+    TAKE(hist, uint32_t, CS_HIST_BINS);
+    TAKE(cand_km, unsigned long long, N);
+    TAKE(cand_id, uint32_t, N);
+    TAKE(cand_bkt, uint32_t, N);
+    TAKE(cand_slot, uint32_t, N);
+    TAKE(sort_km, unsigned long long, N);
+    TAKE(sort_id, uint32_t, N);
+    TAKE(spl_km, unsigned long long, CS_MAX_SPLITTERS + 1);
+    TAKE(spl_id, uint32_t, CS_MAX_SPLITTERS + 1);
+    TAKE(bcount, uint32_t, CS_MAX_SPLITTERS + 1);
+    TAKE(boff, uint32_t, CS_MAX_SPLITTERS + 2);
+#undef TAKE
+    return off;
+}
+
+extern "C" {
+
+int cs_version(void) { return 100; }
+
+const char *cs_strerror(int code)
+{
+    switch (code) {
+    case CS_OK: return "ok";
+    case CS_EINVAL: return "invalid argument";
+    case CS_ECAPACITY: return "size beyond the capacity the workspace was created for";
+    case CS_ENOTIMPL: return "not implemented";
+    case CS_ECUDA: return "CUDA runtime error";
+    case CS_EDEVICE_STATUS: return "device status word set (bad ids skipped)";
+    case CS_ENOMEM: return "out of host memory";
+    default: return "unknown error";
+    }
+}
+
+int cs_workspace_bytes(const cs_params *p, size_t *dev_bytes)
+{
+    int rc = cs_validate_params(p);
+    if (rc != CS_OK) return rc;
+    if (!dev_bytes) return CS_EINVAL;
+    uint32_t gl, as;
+    cs_recency_table_shape(p, &gl, &as);
+    *dev_bytes = cs_layout_workspace(p, gl, nullptr, nullptr);
+    return CS_OK;
+}
+
+int cs_create(const cs_params *p, void *dev_workspace, size_t bytes, cs_stream_t init_stream, cs_ctx **out)
+{
+    int rc = cs_validate_params(p);
+    if (rc != CS_OK) return rc;
+    if (!out || !dev_workspace || (((uintptr_t)dev_workspace) & 255u)) return CS_EINVAL;
+    uint32_t gl, as;
+    cs_recency_table_shape(p, &gl, &as);
+    size_t need = cs_layout_workspace(p, gl, nullptr, nullptr);
+    if (bytes < need) return CS_ECAPACITY;
+    cs_ctx *ctx = new (std::nothrow) cs_ctx;
+    if (!ctx) return CS_ENOMEM;
+    memset(ctx, 0, sizeof(*ctx));
+    ctx->p = *p;
+    ctx->gtab_len = gl;
+    ctx->age_sat = as;
+    ctx->W = (p->n_agents + 31) / 32;
+    ctx->ws_bytes = cs_layout_workspace(p, gl, dev_workspace, &ctx->ws);
+    cudaError_t e = cudaGetDevice(&ctx->device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, ctx->device);
+    if (e != cudaSuccess) { delete ctx; return CS_ECUDA; }
+    ctx->host_link_ctas = 0;
+    ctx->d2d_ctas = 0;
+    rc = cs_launch_init(ctx, (cudaStream_t)init_stream);
+    if (rc != CS_OK) { delete ctx; return rc; }
+    *out = ctx;
+    return CS_OK;
+}
+
+int cs_destroy(cs_ctx *ctx)
+{
+    if (!ctx) return CS_EINVAL;
+    delete ctx;
+    return CS_OK;
+}
+
+int cs_observe_invocations(cs_ctx *ctx, const uint32_t *chain, const uint16_t *agent, const uint8_t *evflags,
+                           uint32_t n_events, cs_stream_t stream)
+{
+    if (!ctx) return CS_EINVAL;
+    if (n_events && (!chain || !agent)) return CS_EINVAL;
+    if (!aligned16(chain) || !aligned16(agent) || !aligned16(evflags)) return CS_EINVAL;
+    return cs_launch_observe(ctx, chain, agent, evflags, n_events, (cudaStream_t)stream);
+}
+
+static int check_index(const cs_ctx *ctx, const cs_block_index *idx)
+{
+    if (!idx) return CS_EINVAL;
+    if (idx->n_blocks > ctx->p.max_blocks) return CS_ECAPACITY;
+    if (idx->n_blocks == 0) return CS_OK;
+    if (!idx->agent || !idx->depth || !idx->ref_count || !idx->flags || !idx->last_access) return CS_EINVAL;
+    if (!aligned16(idx->agent) || !aligned16(idx->depth) || !aligned16(idx->ref_count) ||
+        !aligned16(idx->flags) || !aligned16(idx->last_access) || !aligned16(idx->n_tokens) ||
+        !aligned16(idx->anchor_blocks))
+        return CS_EINVAL;
+    return CS_OK;
+}
+
+int cs_score_blocks(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, const uint16_t *sources,
+                    uint32_t n_sources, float *scores_out, cs_stream_t stream)
+{
+    if (!ctx) return CS_EINVAL;
+    int rc = check_index(ctx, idx);
+    if (rc != CS_OK) return rc;
+    if (idx->n_blocks && (!scores_out || !aligned16(scores_out))) return CS_EINVAL;
+    if (sources && !aligned16(sources)) return CS_EINVAL;
+    const float *fsurv = ctx->ws.fsurv;
+    if (sources) {
+        rc = cs_launch_survival(ctx, sources, n_sources, (cudaStream_t)stream);
+        if (rc != CS_OK) return rc;
+        fsurv = ctx->ws.fsurv_tmp;
+    }
+    if (idx->n_blocks == 0) return CS_OK;
+    return cs_launch_score(ctx, idx, now, fsurv, scores_out, (cudaStream_t)stream);
+}
+
+static int select_common(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, int prefetch, uint32_t tier,
+                         uint32_t k, uint32_t *ids_out, uint32_t *n_out, cs_stream_t stream)
+{
+    if (!ctx) return CS_EINVAL;
+    int rc = check_index(ctx, idx);
+    if (rc != CS_OK) return rc;
+    if (k > ctx->p.max_blocks) return CS_ECAPACITY;
+    if (!n_out || (((uintptr_t)n_out) & 3u)) return CS_EINVAL;
+    if (k && (!ids_out || !aligned16(ids_out))) return CS_EINVAL;
+    if (tier > 1) return CS_EINVAL;
+    return cs_launch_select(ctx, idx, now, prefetch, tier, k, ids_out, n_out, (cudaStream_t)stream);
+}
+
+int cs_select_victims(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, uint32_t tier, uint32_t k,
+                      uint32_t *ids_out, uint32_t *n_out, cs_stream_t stream)
+{
+    return select_common(ctx, idx, now, 0, tier, k, ids_out, n_out, stream);
+}
+
+int cs_select_prefetch(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, uint32_t k, uint32_t *ids_out,
+                       uint32_t *n_out, cs_stream_t stream)
+{
+    return select_common(ctx, idx, now, 1, 1, k, ids_out, n_out, stream);
+}
+
+static int check_pools(const cs_kv_pool *a, const cs_kv_pool *b)
+{
+    if (!a || !b || !a->base || !b->base) return CS_EINVAL;
+    if (!aligned16(a->base) || !aligned16(b->base)) return CS_EINVAL;
+    if (a->layout > 1 || b->layout > 1) return CS_EINVAL;
+    if (a->n_layers != b->n_layers || a->n_kv_heads != b->n_kv_heads || a->head_dim != b->head_dim ||
+        a->block_tokens != b->block_tokens || a->elem_bytes != b->elem_bytes)
+        return CS_EINVAL;
+    if (a->n_layers == 0 || a->n_slots == 0 || b->n_slots == 0) return CS_EINVAL;
+    unsigned long long chunk = (unsigned long long)a->block_tokens * a->n_kv_heads * a->head_dim * a->elem_bytes;
+    if (chunk == 0 || (chunk & 15u) || chunk > (1ull << 30)) return CS_EINVAL;
+    return CS_OK;
+}
+
+static int mover_common(cs_ctx *ctx, const cs_kv_pool *src, const cs_kv_pool *dst, const uint32_t *src_slots,
+                        const uint32_t *dst_slots, uint32_t n_max, const uint32_t *n_dev, int host_link,
+                        cs_stream_t s)
+{
+    if (!ctx) return CS_EINVAL;
+    int rc = check_pools(src, dst);
+    if (rc != CS_OK) return rc;
+    if (n_max == 0) return CS_OK;
+    if (!src_slots || !dst_slots || (((uintptr_t)src_slots) & 3u) || (((uintptr_t)dst_slots) & 3u)) return CS_EINVAL;
+    if (n_dev && (((uintptr_t)n_dev) & 3u)) return CS_EINVAL;
+    return cs_launch_mover(ctx, src, dst, src_slots, dst_slots, n_max, n_dev, host_link, (cudaStream_t)s);
+}
+
+int cs_offload_blocks(cs_ctx *ctx, const cs_kv_pool *gpu, const cs_kv_pool *host, const uint32_t *src_slots,
+                      const uint32_t *dst_slots, uint32_t n_max, const uint32_t *n_dev, cs_stream_t side)
+{
+    return mover_common(ctx, gpu, host, src_slots, dst_slots, n_max, n_dev, 1, side);
+}
+
+int cs_prefetch_blocks(cs_ctx *ctx, const cs_kv_pool *host, const cs_kv_pool *gpu, const uint32_t *src_slots,
+                       const uint32_t *dst_slots, uint32_t n_max, const uint32_t *n_dev, cs_stream_t side)
+{
+    return mover_common(ctx, host, gpu, src_slots, dst_slots, n_max, n_dev, 1, side);
+}
+
+int cs_compact_blocks(cs_ctx *ctx, const cs_kv_pool *src, const cs_kv_pool *dst, const uint32_t *src_slots,
+                      const uint32_t *dst_slots, uint32_t n_max, const uint32_t *n_dev, cs_stream_t stream)
+{
+    return mover_common(ctx, src, dst, src_slots, dst_slots, n_max, n_dev, 0, stream);
+}
+
+int cs_get_model(cs_ctx *ctx, uint32_t *C_out, float *P_out, uint16_t *amax_out, uint16_t *hops_out,
+                 float *fsurv_out, float *R_out, uint16_t *cur_out, uint16_t *last_agent_out, cs_stream_t stream)
+{
+    if (!ctx) return CS_EINVAL;
+    const size_t A = ctx->p.n_agents;
+    cudaStream_t s = (cudaStream_t)stream;
+    cudaError_t e = cudaSuccess;
+#define COPY(dst, src, bytes) \
+    if (e == cudaSuccess && (dst)) e = cudaMemcpyAsync((dst), (src), (bytes), cudaMemcpyDeviceToDevice, s)
+    COPY(C_out, ctx->ws.C, A * A * sizeof(uint32_t));
+    COPY(P_out, ctx->ws.P, A * A * sizeof(float));
+    COPY(amax_out, ctx->ws.amax, A * sizeof(uint16_t));
+    COPY(hops_out, ctx->ws.hops, A * sizeof(uint16_t));
+    COPY(fsurv_out, ctx->ws.fsurv, A * sizeof(float));
+    COPY(R_out, &ctx->ws.sc->R, sizeof(float));
+    COPY(cur_out, ctx->ws.cur, ctx->p.n_chains * sizeof(uint16_t));
+    COPY(last_agent_out, &ctx->ws.sc->last_agent, sizeof(uint16_t));   // little endian: low half of the u32
+#undef COPY
+    if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; return CS_ECUDA; }
+    return CS_OK;
+}
+
+int cs_get_status(cs_ctx *ctx, uint32_t *device_status, cs_stream_t stream)
+{
+    if (!ctx || !device_status) return CS_EINVAL;
+    cudaStream_t s = (cudaStream_t)stream;
+    uint32_t st = 0;
+    cudaError_t e = cudaMemcpyAsync(&st, &ctx->ws.sc->status, sizeof(st), cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e == cudaSuccess && st) e = cudaMemsetAsync(&ctx->ws.sc->status, 0, sizeof(st), s);
+    if (e == cudaSuccess && st) e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; return CS_ECUDA; }
+    *device_status = st;
+    return st ? CS_EDEVICE_STATUS : CS_OK;
+}
+
+int cs_launch_count(cs_ctx *ctx, uint64_t *n)
+{
+    if (!ctx || !n) return CS_EINVAL;
+    *n = ctx->n_launches;
+    return CS_OK;
+}
+
+int cs_set_mover_ctas(cs_ctx *ctx, uint32_t host_link_ctas, uint32_t d2d_ctas)
+{
+    if (!ctx) return CS_EINVAL;
+    ctx->host_link_ctas = host_link_ctas;
+    ctx->d2d_ctas = d2d_ctas;
+    return CS_OK;
+}
+
+int cs_last_cuda_error(cs_ctx *ctx) { return ctx ? ctx->last_cuda_error : 0; }
+
+} // extern "C"

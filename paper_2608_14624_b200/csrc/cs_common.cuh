@@ -1,0 +1,109 @@
+// Internal declarations shared by the translation units of libcachescout (sm_100a only).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "cachescout.h"
+
+#if defined(__CUDA_ARCH__) && (__CUDA_ARCH__ < 1000)
+#error "libcachescout is written for sm_100a (B200) only"
+#endif
+
+#define CS_HIST_BINS 4096u        // first radix digit of the select: top 12 bits of the primary key
+#define CS_MAX_SPLITTERS 255u     // bucket sort of the candidates: up to 256 buckets
+#define CS_SAMPLE 1024u           // candidates sampled to choose the splitters
+#define CS_GTAB_MAX 4096u          // largest recency table kept in shared memory (ages below saturation)
+
+// Scalars the kernels share, one 256-byte line in the workspace.
+struct cs_scalars {
+    uint32_t status;        // CS_ST_* bits
+    uint32_t last_agent;    // agent of the last non-warmup event, CS_AGENT_NONE initially
+    float R;                // Eq. 2
+    uint32_t gate;          // Eq. 11: R >= r_min
+    uint32_t n_transitions; // sum of all counts
+    uint32_t ticket[6];     // "last CTA done" counters, one per kernel that has an epilogue
+    // select state, rewritten by every select call
+    uint32_t sel_b0;        // threshold bin of the first digit
+    uint32_t sel_n_elig;    // eligible entries
+    uint32_t sel_c;         // candidates collected (first digit <= b0)
+    uint32_t sel_n_spl;     // splitters in use
+    uint32_t sel_b_last;    // last bucket that holds one of the k winners
+    uint32_t sel_p_end;     // end position of that bucket
+    uint32_t sel_n_out;     // min(k, eligible)
+};
+
+// Device pointers into the caller's workspace.
+struct cs_workspace {
+    cs_scalars *sc;
+    uint32_t *C;          // [A*A] transition counts
+    uint32_t *rowsum;     // [A]
+    uint16_t *cur;        // [n_chains]
+    float *P;             // [A*A] Eq. 3
+    uint16_t *amax;       // [A]
+    double *rowH;         // [A] sum_j P_ij ln P_ij
+    uint32_t *adj;        // [A*W] Eq. 7 adjacency, one bit per edge, W = ceil(A/32)
+    uint16_t *hops;       // [A]
+    float *fsurv;         // [A] p~ + delta for the cached source
+    uint16_t *hops_tmp;   // [A] same, for cs_score_blocks() with explicit sources
+    float *fsurv_tmp;     // [A]
+    float *gtab;          // [gtab_len] exp(-lambda*age)+delta for age < gtab_len
+    uint32_t *hist;       // [CS_HIST_BINS]
+    unsigned long long *cand_km;    // [max_blocks] (primary<<32 | secondary) of each candidate
+    uint32_t *cand_id;    // [max_blocks]
+    uint32_t *cand_bkt;   // [max_blocks]
+    uint32_t *cand_slot;  // [max_blocks]
+    unsigned long long *sort_km;    // [max_blocks] candidates grouped by bucket
+    uint32_t *sort_id;    // [max_blocks]
+    unsigned long long *spl_km;     // [CS_MAX_SPLITTERS+1]
+    uint32_t *spl_id;     // [CS_MAX_SPLITTERS+1]
+    uint32_t *bcount;     // [CS_MAX_SPLITTERS+1]
+    uint32_t *boff;       // [CS_MAX_SPLITTERS+2]
+};
+
+struct cs_ctx {
+    cs_params p;
+    cs_workspace ws;
+    size_t ws_bytes;
+    uint32_t W;            // adjacency words per row
+    uint32_t gtab_len;     // ages [0, gtab_len) come from the table
+    uint32_t age_sat;      // ages >= age_sat all give g_sat
+    int device;
+    int sm_count;
+    uint32_t host_link_ctas, d2d_ctas;
+    uint64_t n_launches;
+    int last_cuda_error;
+};
+
+// ---- workspace layout (host) -------------------------------------------------------------------
+size_t cs_layout_workspace(const cs_params *p, uint32_t gtab_len, void *base, cs_workspace *ws);
+int cs_validate_params(const cs_params *p);
+void cs_recency_table_shape(const cs_params *p, uint32_t *gtab_len, uint32_t *age_sat);
+
+// ---- launchers implemented in the kernel files ---------------------------------------------------
+int cs_launch_init(cs_ctx *ctx, cudaStream_t s);
+int cs_launch_observe(cs_ctx *ctx, const uint32_t *chain, const uint16_t *agent, const uint8_t *evflags,
+                      uint32_t n_events, cudaStream_t s);
+int cs_launch_survival(cs_ctx *ctx, const uint16_t *sources, uint32_t n_sources, cudaStream_t s);
+int cs_launch_score(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, const float *fsurv,
+                    float *scores_out, cudaStream_t s);
+int cs_launch_select(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, int prefetch, uint32_t tier,
+                     uint32_t k, uint32_t *ids_out, uint32_t *n_out, cudaStream_t s);
+int cs_launch_mover(cs_ctx *ctx, const cs_kv_pool *src, const cs_kv_pool *dst, const uint32_t *src_slots,
+                    const uint32_t *dst_slots, uint32_t n_max, const uint32_t *n_dev, int crosses_host_link,
+                    cudaStream_t s);
+
+static inline int cs_check_launch(cs_ctx *ctx)
+{
+    cudaError_t e = cudaGetLastError();
+    ctx->n_launches++;
+    if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; return CS_ECUDA; }
+    return CS_OK;
+}
+
+#ifdef __CUDACC__
+// Recency factor of Eq. 9 as every kernel computes it: fp64 exp and add, rounded once to fp32.
+__device__ __forceinline__ float cs_recency(float lambda, float delta, uint32_t age)
+{
+    return (float)(exp(-(double)lambda * (double)age) + (double)delta);
+}
+#endif

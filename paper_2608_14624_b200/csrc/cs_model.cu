@@ -1,0 +1,300 @@
+// Transition Learner and Survival Scorer state: transition counting (Algorithm 1,
+// ObserveTouch), Eq. 3 normalisation with row arg-max (Eq. 5 / Eq. 10), predictability
+// (Eq. 2) and gate (Eq. 11), threshold graph (Eq. 7), BFS hop table and survival scores
+// (Eq. 8).  The model is tiny (A <= 1024), so these kernels are latency-bound: the design
+// goal is few launches and no host round trip, not bandwidth.
+#include "cs_common.cuh"
+
+#define OBS_THREADS 1024
+#define ROW_THREADS 256
+
+// ---------------------------------------------------------------------------------------------
+// Initial state of Algorithm 1: zero counts, no current agent; plus the recency table.
+// ---------------------------------------------------------------------------------------------
+__global__ void cs_init_kernel(cs_workspace ws, uint32_t A, uint32_t n_chains, uint32_t gtab_len, float lambda,
+                               float delta)
+{
+    const uint32_t tid = blockIdx.x * blockDim.x + threadIdx.x, nth = gridDim.x * blockDim.x;
+    for (uint32_t i = tid; i < A * A; i += nth) ws.C[i] = 0;
+    for (uint32_t i = tid; i < A; i += nth) ws.rowsum[i] = 0;
+    for (uint32_t i = tid; i < n_chains; i += nth) ws.cur[i] = CS_AGENT_NONE;
+    for (uint32_t i = tid; i < CS_HIST_BINS; i += nth) ws.hist[i] = 0;
+    for (uint32_t i = tid; i <= CS_MAX_SPLITTERS; i += nth) ws.bcount[i] = 0;
+    for (uint32_t i = tid; i < gtab_len; i += nth) ws.gtab[i] = cs_recency(lambda, delta, i);
+    if (tid == 0) {
+        cs_scalars z;
+        memset(&z, 0, sizeof(z));
+        z.last_agent = CS_AGENT_NONE;
+        *ws.sc = z;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Transition counting over one batch of events, one CTA.  The update is sequential per chain
+// (each event's predecessor is the previous non-warmup event of the same chain, in this batch
+// or carried in cur[]), but the counter increments commute, so every event is handled by its
+// own thread: it looks its predecessor up in the shared-memory copy of the batch and adds 1
+// atomically.  Integer adds make the result independent of the order the atomics land in.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(OBS_THREADS)
+cs_observe_kernel(cs_workspace ws, uint32_t A, uint32_t n_chains, const uint32_t *__restrict__ chain,
+                  const uint16_t *__restrict__ agent, const uint8_t *__restrict__ evflags, uint32_t n_events)
+{
+    __shared__ uint32_t s_chain[OBS_THREADS];
+    __shared__ uint16_t s_agent[OBS_THREADS];     // CS_AGENT_NONE marks an event that is skipped
+    __shared__ int s_last;
+    const int tid = threadIdx.x;
+    for (uint32_t base = 0; base < n_events; base += OBS_THREADS) {
+        const uint32_t e = base + tid;
+        uint32_t c = 0, a = CS_AGENT_NONE;
+        if (tid == 0) s_last = -1;
+        if (e < n_events) {
+            c = chain[e];
+            a = agent[e];
+            const bool warm = evflags && (evflags[e] & CS_EV_WARMUP);
+            uint32_t bad = 0;
+            if (!warm && a >= A) bad |= CS_ST_BAD_AGENT;
+            if (!warm && c >= n_chains) bad |= CS_ST_BAD_CHAIN;
+            if (bad) atomicOr(&ws.sc->status, bad);
+            if (warm || bad) a = CS_AGENT_NONE;
+        }
+        s_chain[tid] = c;
+        s_agent[tid] = (uint16_t)a;
+        __syncthreads();
+        const bool live = a != CS_AGENT_NONE;
+        uint32_t prev = CS_AGENT_NONE;
+        bool last_of_chain = live;
+        if (live) {
+            int j = tid - 1;
+            for (; j >= 0; --j)
+                if (s_chain[j] == c && s_agent[j] != CS_AGENT_NONE) { prev = s_agent[j]; break; }
+            if (j < 0) prev = ws.cur[c];
+            const int lim = min((int)OBS_THREADS, (int)(n_events - base));
+            for (int q = tid + 1; q < lim; ++q)
+                if (s_chain[q] == c && s_agent[q] != CS_AGENT_NONE) { last_of_chain = false; break; }
+            atomicMax(&s_last, tid);
+        }
+        __syncthreads();                       // every read of cur[] above precedes the writes below
+        if (live) {
+            if (prev != CS_AGENT_NONE && prev != a) {
+                atomicAdd(&ws.C[prev * A + a], 1u);
+                atomicAdd(&ws.rowsum[prev], 1u);
+                atomicAdd(&ws.sc->n_transitions, 1u);
+            }
+            if (last_of_chain) ws.cur[c] = (uint16_t)a;
+            if (s_last == tid) ws.sc->last_agent = a;
+        }
+        __syncthreads();
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// BFS over the bit-matrix graph from a set of source bits, then Eq. 8.  Runs inside one CTA;
+// thread w < W owns word w of the frontier / visited sets.  Level-synchronous: the next
+// frontier is the OR of the adjacency rows of the current one, minus what was visited.
+// ---------------------------------------------------------------------------------------------
+__device__ void cs_bfs_survival(const uint32_t *__restrict__ adj, uint32_t A, uint32_t W, uint32_t *s_front,
+                                uint32_t *s_visit, uint16_t *hops, float *fsurv, uint32_t e_max, float delta)
+{
+    // on entry s_front[] holds the source bits (already synchronised by the caller)
+    const uint32_t tid = threadIdx.x;
+    for (uint32_t a = tid; a < A; a += blockDim.x)
+        hops[a] = ((s_front[a >> 5] >> (a & 31)) & 1u) ? 0 : CS_HOP_NONE;
+    if (tid < W) s_visit[tid] = s_front[tid];
+    __syncthreads();
+    for (uint32_t level = 1; level <= A; ++level) {
+        uint32_t acc = 0;
+        if (tid < W) {
+            for (uint32_t fw = 0; fw < W; ++fw) {
+                uint32_t bits = s_front[fw];
+                while (bits) {
+                    const uint32_t i = fw * 32 + (__ffs(bits) - 1);
+                    bits &= bits - 1;
+                    acc |= __ldcg(&adj[i * W + tid]);
+                }
+            }
+            acc &= ~s_visit[tid];
+        }
+        const int any = __syncthreads_or(acc != 0);      // also orders the reads of s_front before its rewrite
+        if (!any) break;
+        if (tid < W) {
+            s_front[tid] = acc;
+            s_visit[tid] |= acc;
+            uint32_t bits = acc;
+            while (bits) {
+                const uint32_t b = tid * 32 + (__ffs(bits) - 1);
+                bits &= bits - 1;
+                if (b < A) hops[b] = (uint16_t)level;
+            }
+        }
+        __syncthreads();
+    }
+    __syncthreads();
+    for (uint32_t a = tid; a < A; a += blockDim.x) {
+        const uint32_t h = hops[a];
+        const uint32_t m = h < e_max ? h : e_max;          // CS_HOP_NONE > e_max by construction
+        const double ptilde = 1.0 - (double)m / (double)e_max;
+        fsurv[a] = (float)(ptilde + (double)delta);
+    }
+}
+
+// Deterministic block reductions (fixed tree, so results do not depend on scheduling).
+template <typename T>
+__device__ T cs_block_sum(T v, T *s_red)
+{
+    const uint32_t tid = threadIdx.x;
+    __syncthreads();
+    s_red[tid] = v;
+    __syncthreads();
+    for (uint32_t s = blockDim.x >> 1; s > 0; s >>= 1) {
+        if (tid < s) s_red[tid] += s_red[tid + s];
+        __syncthreads();
+    }
+    T r = s_red[0];
+    __syncthreads();
+    return r;
+}
+
+// ---------------------------------------------------------------------------------------------
+// One CTA per row i: Eq. 3 in canonical fp32 (one rounding per operation, no FMA), the row's
+// arg-max, its adjacency bits (Eq. 7) and its entropy term.  The last CTA to finish then
+// computes Eq. 2 / Eq. 11 over all rows and refreshes the cached BFS / Eq. 8 tables.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(ROW_THREADS)
+cs_normalise_kernel(cs_workspace ws, uint32_t A, uint32_t W, float eps, float tau, float r_min, uint32_t e_max,
+                    float delta)
+{
+    __shared__ double s_red[ROW_THREADS];
+    __shared__ float s_bestv[ROW_THREADS];
+    __shared__ uint32_t s_besti[ROW_THREADS];
+    __shared__ uint32_t s_front[32], s_visit[32];
+    __shared__ bool s_is_last;
+    const uint32_t tid = threadIdx.x;
+
+    for (uint32_t i = blockIdx.x; i < A; i += gridDim.x) {
+        const uint32_t n_i = ws.rowsum[i];
+        const float den = __fadd_rn((float)n_i, __fmul_rn((float)A, eps));
+        float bestv = -1.0f;
+        uint32_t besti = 0xFFFFFFFFu;
+        double h = 0.0;
+        for (uint32_t j0 = 0; j0 < A; j0 += ROW_THREADS) {       // A is padded to whole warps for the ballot
+            const uint32_t j = j0 + tid;
+            bool edge = false;
+            if (j < A) {
+                const float p = __fdiv_rn(__fadd_rn((float)ws.C[i * A + j], eps), den);
+                ws.P[i * A + j] = p;
+                if (p > bestv) { bestv = p; besti = j; }         // strict: the lowest j among equals stays
+                const double pd = (double)p;
+                h += pd * log(pd);
+                edge = p >= tau;
+            }
+            const uint32_t bits = __ballot_sync(0xFFFFFFFFu, edge);
+            if ((tid & 31) == 0 && (j >> 5) < W) ws.adj[i * W + (j >> 5)] = bits;
+        }
+        // arg-max: max value, then min index
+        s_bestv[tid] = bestv;
+        s_besti[tid] = besti;
+        __syncthreads();
+        for (uint32_t s = ROW_THREADS >> 1; s > 0; s >>= 1) {
+            if (tid < s) {
+                const float v = s_bestv[tid + s];
+                const uint32_t x = s_besti[tid + s];
+                if (v > s_bestv[tid] || (v == s_bestv[tid] && x < s_besti[tid])) { s_bestv[tid] = v; s_besti[tid] = x; }
+            }
+            __syncthreads();
+        }
+        if (tid == 0) ws.amax[i] = (uint16_t)s_besti[0];
+        const double hsum = cs_block_sum<double>(h, s_red);
+        if (tid == 0) ws.rowH[i] = hsum;
+    }
+
+    // ---- last CTA done: global quantities ---------------------------------------------------------
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+        const uint32_t t = atomicAdd(&ws.sc->ticket[0], 1u);
+        s_is_last = (t == gridDim.x - 1);
+    }
+    __syncthreads();
+    if (!s_is_last) return;
+    __threadfence();
+
+    const uint32_t N = __ldcg(&ws.sc->n_transitions);
+    double Hc = 0.0, Hm = 0.0;
+    if (N > 0) {
+        const double invN = 1.0 / (double)N;
+        for (uint32_t i = tid; i < A; i += ROW_THREADS) Hc -= ((double)__ldcg(&ws.rowsum[i]) * invN) * __ldcg(&ws.rowH[i]);
+        for (uint32_t j = tid; j < A; j += ROW_THREADS) {
+            double q = 0.0;
+            for (uint32_t i = 0; i < A; ++i) {
+                const uint32_t n_i = __ldcg(&ws.rowsum[i]);
+                if (n_i) q += ((double)n_i * invN) * (double)__ldcg(&ws.P[i * A + j]);
+            }
+            if (q > 0.0) Hm -= q * log(q);
+        }
+    }
+    Hc = cs_block_sum<double>(Hc, s_red);
+    Hm = cs_block_sum<double>(Hm, s_red);
+    const uint32_t la = __ldcg(&ws.sc->last_agent);
+    if (tid == 0) {
+        double R = 0.0;
+        if (N > 0 && Hm > 0.0) R = 1.0 - Hc / Hm;
+        const float Rf = (float)R;
+        ws.sc->R = Rf;
+        ws.sc->gate = (Rf >= r_min) ? 1u : 0u;
+        ws.sc->ticket[0] = 0;
+    }
+    if (tid < 32) s_front[tid] = (la < A && (la >> 5) == tid) ? (1u << (la & 31)) : 0u;
+    __syncthreads();
+    cs_bfs_survival(ws.adj, A, W, s_front, s_visit, ws.hops, ws.fsurv, e_max, delta);
+}
+
+// BFS + Eq. 8 from explicit sources into the temporary tables (cs_score_blocks with sources).
+__global__ void __launch_bounds__(ROW_THREADS)
+cs_survival_kernel(cs_workspace ws, uint32_t A, uint32_t W, const uint16_t *__restrict__ sources, uint32_t n_sources,
+                   uint32_t e_max, float delta)
+{
+    __shared__ uint32_t s_front[32], s_visit[32];
+    const uint32_t tid = threadIdx.x;
+    if (tid < 32) s_front[tid] = 0;
+    __syncthreads();
+    for (uint32_t s = tid; s < n_sources; s += ROW_THREADS) {
+        const uint32_t a = sources[s];
+        if (a < A) atomicOr(&s_front[a >> 5], 1u << (a & 31));
+        else atomicOr(&ws.sc->status, CS_ST_BAD_SOURCE);
+    }
+    __syncthreads();
+    cs_bfs_survival(ws.adj, A, W, s_front, s_visit, ws.hops_tmp, ws.fsurv_tmp, e_max, delta);
+}
+
+// ---------------------------------------------------------------------------------------------
+int cs_launch_init(cs_ctx *ctx, cudaStream_t s)
+{
+    const cs_params &p = ctx->p;
+    cs_init_kernel<<<64, 256, 0, s>>>(ctx->ws, p.n_agents, p.n_chains, ctx->gtab_len, p.lambda, p.delta);
+    int rc = cs_check_launch(ctx);
+    if (rc != CS_OK) return rc;
+    return cs_launch_observe(ctx, nullptr, nullptr, nullptr, 0, s);
+}
+
+int cs_launch_observe(cs_ctx *ctx, const uint32_t *chain, const uint16_t *agent, const uint8_t *evflags,
+                      uint32_t n_events, cudaStream_t s)
+{
+    const cs_params &p = ctx->p;
+    if (n_events) {
+        cs_observe_kernel<<<1, OBS_THREADS, 0, s>>>(ctx->ws, p.n_agents, p.n_chains, chain, agent, evflags, n_events);
+        int rc = cs_check_launch(ctx);
+        if (rc != CS_OK) return rc;
+    }
+    const uint32_t grid = p.n_agents < 2u * (uint32_t)ctx->sm_count ? p.n_agents : 2u * (uint32_t)ctx->sm_count;
+    cs_normalise_kernel<<<grid, ROW_THREADS, 0, s>>>(ctx->ws, p.n_agents, ctx->W, p.eps, p.tau, p.r_min, p.e_max,
+                                                      p.delta);
+    return cs_check_launch(ctx);
+}
+
+int cs_launch_survival(cs_ctx *ctx, const uint16_t *sources, uint32_t n_sources, cudaStream_t s)
+{
+    const cs_params &p = ctx->p;
+    cs_survival_kernel<<<1, ROW_THREADS, 0, s>>>(ctx->ws, p.n_agents, ctx->W, sources, n_sources, p.e_max, p.delta);
+    return cs_check_launch(ctx);
+}

@@ -1,0 +1,595 @@
+// Block scoring (Eq. 9 / ScoreBlock of Algorithm 1) and exact, ordered top-k selection of
+// eviction victims (Evict of Algorithm 1) and prefetch candidates (BetweenStep, Eq. 10-11).
+//
+// Every kernel that walks the block index reads the SoA metadata with 128-bit loads, 16
+// entries per thread and iteration, and never materialises the score in the select path.
+// A positive fp32 score orders like its bit pattern, so each eligible entry has a 96-bit
+// integer key (primary, secondary, id) and "the k best in order" is "the k smallest keys in
+// ascending order":
+//   victims : primary = score bits,                      secondary = last_access
+//   prefetch: primary = (not a*)<<31 | ~score bits[30:0], secondary = ~last_access
+//
+// Selection in five launches, none of which waits on another CTA:
+//   1 histogram : 4096-bin histogram of the top 12 primary bits; the last CTA to finish finds
+//                 the threshold bin b0 (first bin whose running count reaches k).
+//   2 collect   : every eligible entry whose bin <= b0 is appended to the candidate buffer
+//                 (c >= min(k, eligible) keys); the last CTA samples <= 1024 candidates,
+//                 sorts them in shared memory and publishes <= 255 splitters.
+//   3 bucket    : each candidate finds its bucket by binary search over the splitters and
+//                 takes a slot in it; the last CTA prefix-sums the bucket sizes and finds the
+//                 last bucket that can hold one of the k winners.
+//   4 scatter   : candidates of the needed buckets are grouped by bucket.
+//   5 rank      : each grouped candidate counts the smaller keys of its bucket; bucket offset
+//                 + that count is its exact rank, i.e. its position in the output list.
+// Keys are unique (the id is part of the key), so ranks are a permutation and the output does
+// not depend on the order in which atomics were served.
+#include "cs_common.cuh"
+
+#define SEL_THREADS 512
+#define GRP 16                    // index entries per thread and iteration (one 128-bit load of bytes)
+
+struct SelArgs {
+    const uint16_t *agent;
+    const uint16_t *depth;
+    const uint8_t *ref;
+    const uint8_t *flags;
+    const uint32_t *la;
+    const uint8_t *ntok;
+    const uint16_t *anchor;
+    const float *fsurv;
+    uint32_t n, now, A, block_tokens, gtab_len, age_sat;
+    float lambda, delta;
+    uint32_t tier, k;
+};
+
+// Per-CTA copies of the small tables every entry looks up.
+struct Tables {
+    float *fsurv;       // [A]
+    float *gtab;        // [gtab_len]
+    uint16_t *anchor;   // [A] or unused
+    float g_sat;
+    uint32_t a_star;
+};
+
+__device__ __forceinline__ void load_tables(const SelArgs &a, const cs_workspace &ws, float *smem, Tables &T,
+                                            bool want_anchor)
+{
+    T.fsurv = smem;
+    T.gtab = smem + a.A;
+    T.anchor = (uint16_t *)(smem + a.A + a.gtab_len);
+    for (uint32_t i = threadIdx.x; i < a.A; i += blockDim.x) T.fsurv[i] = a.fsurv[i];
+    for (uint32_t i = threadIdx.x; i < a.gtab_len; i += blockDim.x) T.gtab[i] = ws.gtab[i];
+    if (want_anchor)
+        for (uint32_t i = threadIdx.x; i < a.A; i += blockDim.x) T.anchor[i] = a.anchor[i];
+    T.g_sat = cs_recency(a.lambda, a.delta, a.age_sat);
+    const uint32_t la = ws.sc->last_agent;
+    T.a_star = (la < a.A) ? ws.amax[la] : 0xFFFFFFFFu;
+}
+
+__device__ __forceinline__ float score_of(const SelArgs &a, const Tables &T, uint32_t agent, uint32_t la,
+                                          uint32_t tok)
+{
+    const uint32_t age = la <= a.now ? a.now - la : 0u;
+    float g;
+    if (age < a.gtab_len) g = T.gtab[age];
+    else if (age >= a.age_sat) g = T.g_sat;
+    else g = cs_recency(a.lambda, a.delta, age);
+    return __fmul_rn(__fmul_rn(T.fsurv[agent], g), (float)tok);      // two roundings, never an FMA
+}
+
+// Eligibility and key of one entry.  PF = prefetch-candidate rules, else eviction-victim rules.
+template <bool PF>
+__device__ __forceinline__ bool entry_key(const SelArgs &a, const Tables &T, uint32_t *status, uint32_t agent,
+                                          uint32_t depth, uint32_t ref, uint32_t flags, uint32_t la, uint32_t tok,
+                                          uint32_t &primary, uint32_t &secondary)
+{
+    if (!(flags & CS_FLAG_VALID) || (flags & CS_FLAG_PINNED) || ref != 0) return false;
+    if (PF) {
+        if (!(flags & CS_FLAG_TIER_HOST) || (flags & CS_FLAG_OTHER_COPY)) return false;
+    } else {
+        if (((flags >> 2) & 1u) != a.tier) return false;
+    }
+    if (agent >= a.A) { atomicOr(status, CS_ST_BAD_AGENT); return false; }
+    if (PF && a.anchor && !(depth < T.anchor[agent])) return false;
+    const uint32_t bits = __float_as_uint(score_of(a, T, agent, la, tok));
+    if (PF) {
+        primary = ((agent == T.a_star) ? 0u : 0x80000000u) | (~bits & 0x7FFFFFFFu);
+        secondary = ~la;
+    } else {
+        primary = bits;
+        secondary = la;
+    }
+    return true;
+}
+
+// One group of 16 consecutive entries in registers.
+struct Group {
+    uint4 ag0, ag1, dp0, dp1, rf, fl, la0, la1, la2, la3, tk;
+};
+
+template <bool PF>
+__device__ __forceinline__ void load_group(const SelArgs &a, uint32_t g, Group &G)
+{
+    G.ag0 = __ldg((const uint4 *)a.agent + 2 * g);
+    G.ag1 = __ldg((const uint4 *)a.agent + 2 * g + 1);
+    G.rf = __ldg((const uint4 *)a.ref + g);
+    G.fl = __ldg((const uint4 *)a.flags + g);
+    G.la0 = __ldg((const uint4 *)a.la + 4 * g);
+    G.la1 = __ldg((const uint4 *)a.la + 4 * g + 1);
+    G.la2 = __ldg((const uint4 *)a.la + 4 * g + 2);
+    G.la3 = __ldg((const uint4 *)a.la + 4 * g + 3);
+    if (a.ntok) G.tk = __ldg((const uint4 *)a.ntok + g);
+    if (PF && a.anchor) {
+        G.dp0 = __ldg((const uint4 *)a.depth + 2 * g);
+        G.dp1 = __ldg((const uint4 *)a.depth + 2 * g + 1);
+    }
+}
+
+__device__ __forceinline__ uint32_t u4_word(const uint4 &v, int w)
+{
+    return w == 0 ? v.x : (w == 1 ? v.y : (w == 2 ? v.z : v.w));
+}
+__device__ __forceinline__ uint32_t grp_u16(const uint4 &lo, const uint4 &hi, int j)   // j in [0,16)
+{
+    const uint32_t w = u4_word(j < 8 ? lo : hi, (j & 7) >> 1);
+    return (w >> ((j & 1) * 16)) & 0xFFFFu;
+}
+__device__ __forceinline__ uint32_t grp_u8(const uint4 &v, int j)
+{
+    return (u4_word(v, j >> 2) >> ((j & 3) * 8)) & 0xFFu;
+}
+__device__ __forceinline__ uint32_t grp_u32(const Group &G, int j)
+{
+    const uint4 &v = j < 4 ? G.la0 : (j < 8 ? G.la1 : (j < 12 ? G.la2 : G.la3));
+    return u4_word(v, j & 3);
+}
+
+// Calls f(id, primary, secondary) for every eligible entry this thread owns: whole groups
+// grid-strided, then the ragged tail (n % 16 entries) one entry per thread.
+template <bool PF, typename F>
+__device__ __forceinline__ void for_each_eligible(const SelArgs &a, const Tables &T, uint32_t *status, F f)
+{
+    const uint32_t gtid = blockIdx.x * blockDim.x + threadIdx.x, nth = gridDim.x * blockDim.x;
+    const uint32_t n_groups = a.n / GRP;
+    for (uint32_t g = gtid; g < n_groups; g += nth) {
+        Group G;
+        load_group<PF>(a, g, G);
+#pragma unroll
+        for (int j = 0; j < GRP; ++j) {
+            uint32_t pr, se;
+            const uint32_t tok = a.ntok ? grp_u8(G.tk, j) : a.block_tokens;
+            const uint32_t dp = (PF && a.anchor) ? grp_u16(G.dp0, G.dp1, j) : 0u;
+            if (entry_key<PF>(a, T, status, grp_u16(G.ag0, G.ag1, j), dp, grp_u8(G.rf, j), grp_u8(G.fl, j),
+                              grp_u32(G, j), tok, pr, se))
+                f(g * GRP + j, pr, se);
+        }
+    }
+    const uint32_t t0 = n_groups * GRP;
+    if (gtid < a.n - t0) {
+        const uint32_t i = t0 + gtid;
+        uint32_t pr, se;
+        const uint32_t tok = a.ntok ? a.ntok[i] : a.block_tokens;
+        if (entry_key<PF>(a, T, status, a.agent[i], a.depth[i], a.ref[i], a.flags[i], a.la[i], tok, pr, se))
+            f(i, pr, se);
+    }
+}
+
+// The prefetch list is empty unless the gate of Eq. 11 is open and a current agent exists.
+__device__ __forceinline__ bool prefetch_enabled(const cs_workspace &ws, uint32_t A)
+{
+    return ws.sc->gate != 0 && ws.sc->last_agent < A;
+}
+
+__device__ __forceinline__ bool last_cta_done(uint32_t *ticket, bool *s_flag)
+{
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) *s_flag = (atomicAdd(ticket, 1u) == gridDim.x - 1);
+    __syncthreads();
+    const bool last = *s_flag;
+    if (last) __threadfence();
+    return last;
+}
+
+// ---------------------------------------------------------------------------------------------
+// ScoreBlock for every entry (cs_score_blocks).
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(SEL_THREADS) cs_score_kernel(SelArgs a, cs_workspace ws, float *__restrict__ out)
+{
+    extern __shared__ float smem[];
+    Tables T;
+    load_tables(a, ws, smem, T, false);
+    __syncthreads();
+    const uint32_t gtid = blockIdx.x * blockDim.x + threadIdx.x, nth = gridDim.x * blockDim.x;
+    const uint32_t n_groups = a.n / GRP;
+    for (uint32_t g = gtid; g < n_groups; g += nth) {
+        Group G;
+        load_group<false>(a, g, G);
+        float s[GRP];
+#pragma unroll
+        for (int j = 0; j < GRP; ++j) {
+            const uint32_t ag = grp_u16(G.ag0, G.ag1, j);
+            const uint32_t tok = a.ntok ? grp_u8(G.tk, j) : a.block_tokens;
+            if (ag < a.A) s[j] = score_of(a, T, ag, grp_u32(G, j), tok);
+            else { s[j] = 0.0f; atomicOr(&ws.sc->status, CS_ST_BAD_AGENT); }
+        }
+        float4 *o = (float4 *)out + 4 * g;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) __stcs(o + q, make_float4(s[4 * q], s[4 * q + 1], s[4 * q + 2], s[4 * q + 3]));
+    }
+    const uint32_t t0 = n_groups * GRP;
+    if (gtid < a.n - t0) {
+        const uint32_t i = t0 + gtid;
+        const uint32_t ag = a.agent[i];
+        const uint32_t tok = a.ntok ? a.ntok[i] : a.block_tokens;
+        if (ag < a.A) out[i] = score_of(a, T, ag, a.la[i], tok);
+        else { out[i] = 0.0f; atomicOr(&ws.sc->status, CS_ST_BAD_AGENT); }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// 1 histogram
+// ---------------------------------------------------------------------------------------------
+template <bool PF>
+__global__ void __launch_bounds__(SEL_THREADS) cs_sel_hist_kernel(SelArgs a, cs_workspace ws)
+{
+    extern __shared__ float smem[];
+    __shared__ uint32_t s_hist[CS_HIST_BINS];
+    __shared__ uint32_t s_part[SEL_THREADS];
+    __shared__ bool s_flag;
+    Tables T;
+    load_tables(a, ws, smem, T, PF && a.anchor);
+    for (uint32_t i = threadIdx.x; i < CS_HIST_BINS; i += blockDim.x) s_hist[i] = 0;
+    __syncthreads();
+    if (!PF || prefetch_enabled(ws, a.A)) {
+        uint32_t run_bin = 0xFFFFFFFFu, run_cnt = 0;          // adjacent entries often share a bin
+        for_each_eligible<PF>(a, T, &ws.sc->status, [&](uint32_t, uint32_t pr, uint32_t) {
+            const uint32_t bin = pr >> 20;
+            if (bin == run_bin) { ++run_cnt; return; }
+            if (run_cnt) atomicAdd(&s_hist[run_bin], run_cnt);
+            run_bin = bin;
+            run_cnt = 1;
+        });
+        if (run_cnt) atomicAdd(&s_hist[run_bin], run_cnt);
+    }
+    __syncthreads();
+    for (uint32_t i = threadIdx.x; i < CS_HIST_BINS; i += blockDim.x) {
+        const uint32_t v = s_hist[i];
+        if (v) atomicAdd(&ws.hist[i], v);
+    }
+    if (!last_cta_done(&ws.sc->ticket[1], &s_flag)) return;
+
+    // ---- last CTA: threshold bin = first bin whose inclusive running count reaches k ------------
+    constexpr uint32_t PER = CS_HIST_BINS / SEL_THREADS;
+    uint32_t loc[PER], sum = 0;
+#pragma unroll
+    for (uint32_t q = 0; q < PER; ++q) {
+        loc[q] = __ldcg(&ws.hist[threadIdx.x * PER + q]);
+        ws.hist[threadIdx.x * PER + q] = 0;                 // ready for the next call
+        sum += loc[q];
+    }
+    s_part[threadIdx.x] = sum;
+    __syncthreads();
+    for (uint32_t d = 1; d < SEL_THREADS; d <<= 1) {         // inclusive scan
+        const uint32_t v = threadIdx.x >= d ? s_part[threadIdx.x - d] : 0;
+        __syncthreads();
+        s_part[threadIdx.x] += v;
+        __syncthreads();
+    }
+    const uint32_t total = s_part[SEL_THREADS - 1];
+    const uint32_t before = s_part[threadIdx.x] - sum;
+    if (total < a.k || a.k == 0) {
+        if (threadIdx.x == 0) ws.sc->sel_b0 = (a.k == 0) ? 0xFFFFFFFFu : CS_HIST_BINS - 1;   // k = 0: collect nothing
+    } else if (before < a.k && a.k <= before + sum) {
+        uint32_t run = before;
+#pragma unroll
+        for (uint32_t q = 0; q < PER; ++q) {
+            run += loc[q];
+            if (run >= a.k) { ws.sc->sel_b0 = threadIdx.x * PER + q; break; }
+        }
+    }
+    if (threadIdx.x == 0) {
+        ws.sc->sel_n_elig = total;
+        ws.sc->sel_n_out = total < a.k ? total : a.k;
+        ws.sc->sel_c = 0;
+        ws.sc->ticket[1] = 0;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// 2 collect (+ splitters)
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ bool key_less(unsigned long long km_a, uint32_t id_a, unsigned long long km_b,
+                                         uint32_t id_b)
+{
+    return km_a < km_b || (km_a == km_b && id_a < id_b);
+}
+
+template <bool PF>
+__global__ void __launch_bounds__(SEL_THREADS) cs_sel_collect_kernel(SelArgs a, cs_workspace ws)
+{
+    extern __shared__ float smem[];
+    __shared__ unsigned long long s_km[CS_SAMPLE];
+    __shared__ uint32_t s_id[CS_SAMPLE];
+    __shared__ bool s_flag;
+    Tables T;
+    load_tables(a, ws, smem, T, PF && a.anchor);
+    __syncthreads();
+    const uint32_t b0 = ws.sc->sel_b0;
+    const uint32_t lane = threadIdx.x & 31;
+    if (b0 != 0xFFFFFFFFu && (!PF || prefetch_enabled(ws, a.A))) {
+        // Whole groups: count this thread's candidates, reserve a range with one atomic per warp,
+        // then write.  The loop bound is rounded up so that whole warps stay in the shuffles.
+        const uint32_t gtid = blockIdx.x * blockDim.x + threadIdx.x, nth = gridDim.x * blockDim.x;
+        const uint32_t n_groups = a.n / GRP;
+        const uint32_t n_iter = (n_groups + nth - 1) / nth;
+        for (uint32_t it = 0; it < n_iter; ++it) {
+            const uint32_t g = it * nth + gtid;
+            uint32_t pr[GRP], mask = 0;
+            Group G;
+            if (g < n_groups) {
+                load_group<PF>(a, g, G);
+#pragma unroll
+                for (int j = 0; j < GRP; ++j) {
+                    uint32_t se;
+                    const uint32_t tok = a.ntok ? grp_u8(G.tk, j) : a.block_tokens;
+                    const uint32_t dp = (PF && a.anchor) ? grp_u16(G.dp0, G.dp1, j) : 0u;
+                    if (entry_key<PF>(a, T, &ws.sc->status, grp_u16(G.ag0, G.ag1, j), dp, grp_u8(G.rf, j),
+                                      grp_u8(G.fl, j), grp_u32(G, j), tok, pr[j], se) &&
+                        (pr[j] >> 20) <= b0)
+                        mask |= 1u << j;
+                }
+            }
+            const uint32_t cnt = __popc(mask);
+            uint32_t incl = cnt;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+                if (lane >= d) incl += v;
+            }
+            uint32_t base = 0;
+            if (lane == 31 && incl) base = atomicAdd(&ws.sc->sel_c, incl);
+            base = __shfl_sync(0xFFFFFFFFu, base, 31);
+            uint32_t pos = base + incl - cnt;
+#pragma unroll
+            for (int j = 0; j < GRP; ++j) {
+                if (mask & (1u << j)) {
+                    const uint32_t la = grp_u32(G, j);
+                    ws.cand_km[pos] = ((unsigned long long)pr[j] << 32) | (PF ? ~la : la);
+                    ws.cand_id[pos] = g * GRP + j;
+                    ++pos;
+                }
+            }
+        }
+        const uint32_t t0 = n_groups * GRP;
+        if (gtid < a.n - t0) {
+            const uint32_t i = t0 + gtid;
+            uint32_t p, se;
+            const uint32_t tok = a.ntok ? a.ntok[i] : a.block_tokens;
+            if (entry_key<PF>(a, T, &ws.sc->status, a.agent[i], a.depth[i], a.ref[i], a.flags[i], a.la[i], tok, p, se) &&
+                (p >> 20) <= b0) {
+                const uint32_t pos = atomicAdd(&ws.sc->sel_c, 1u);
+                ws.cand_km[pos] = ((unsigned long long)p << 32) | se;
+                ws.cand_id[pos] = i;
+            }
+        }
+    }
+    if (!last_cta_done(&ws.sc->ticket[2], &s_flag)) return;
+
+    // ---- last CTA: sample, sort the sample (bitonic, shared memory), publish splitters -----------
+    const uint32_t c = __ldcg(&ws.sc->sel_c);
+    const uint32_t n_samp = c < CS_SAMPLE ? c : CS_SAMPLE;
+    for (uint32_t i = threadIdx.x; i < CS_SAMPLE; i += blockDim.x) {
+        if (i < n_samp) {
+            const uint32_t pos = (uint32_t)(((unsigned long long)i * c) / n_samp);
+            s_km[i] = __ldcg(&ws.cand_km[pos]);
+            s_id[i] = __ldcg(&ws.cand_id[pos]);
+        } else {
+            s_km[i] = ~0ull;
+            s_id[i] = 0xFFFFFFFFu;
+        }
+    }
+    __syncthreads();
+    for (uint32_t size = 2; size <= CS_SAMPLE; size <<= 1) {
+        for (uint32_t stride = size >> 1; stride > 0; stride >>= 1) {
+            for (uint32_t t = threadIdx.x; t < CS_SAMPLE / 2; t += blockDim.x) {
+                const uint32_t lo = 2 * t - (t & (stride - 1));
+                const uint32_t hi = lo + stride;
+                const bool up = (lo & size) == 0;
+                const unsigned long long ka = s_km[lo], kb = s_km[hi];
+                const uint32_t ia = s_id[lo], ib = s_id[hi];
+                if (key_less(kb, ib, ka, ia) == up) {
+                    s_km[lo] = kb; s_id[lo] = ib;
+                    s_km[hi] = ka; s_id[hi] = ia;
+                }
+            }
+            __syncthreads();
+        }
+    }
+    uint32_t n_spl = c / 64;
+    if (n_spl > CS_MAX_SPLITTERS) n_spl = CS_MAX_SPLITTERS;
+    for (uint32_t j = threadIdx.x; j <= CS_MAX_SPLITTERS; j += blockDim.x) {
+        if (j < n_spl) {
+            const uint32_t q = (uint32_t)(((unsigned long long)(j + 1) * n_samp) / (n_spl + 1));
+            ws.spl_km[j] = s_km[q];
+            ws.spl_id[j] = s_id[q];
+        }
+        ws.bcount[j] = 0;
+    }
+    if (threadIdx.x == 0) {
+        ws.sc->sel_n_spl = n_spl;
+        ws.sc->ticket[2] = 0;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// 3 bucket (+ offsets)
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) cs_sel_bucket_kernel(cs_workspace ws)
+{
+    __shared__ unsigned long long s_km[CS_MAX_SPLITTERS + 1];
+    __shared__ uint32_t s_id[CS_MAX_SPLITTERS + 1];
+    __shared__ uint32_t s_scan[CS_MAX_SPLITTERS + 1];
+    __shared__ bool s_flag;
+    const uint32_t c = ws.sc->sel_c, n_spl = ws.sc->sel_n_spl;
+    for (uint32_t j = threadIdx.x; j < n_spl; j += blockDim.x) { s_km[j] = ws.spl_km[j]; s_id[j] = ws.spl_id[j]; }
+    __syncthreads();
+    for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < c; i += gridDim.x * blockDim.x) {
+        const unsigned long long km = ws.cand_km[i];
+        const uint32_t id = ws.cand_id[i];
+        uint32_t lo = 0, hi = n_spl;                         // bucket = number of splitters <= key
+        while (lo < hi) {
+            const uint32_t mid = (lo + hi) >> 1;
+            if (key_less(km, id, s_km[mid], s_id[mid])) hi = mid;
+            else lo = mid + 1;
+        }
+        ws.cand_bkt[i] = lo;
+        ws.cand_slot[i] = atomicAdd(&ws.bcount[lo], 1u);
+    }
+    if (!last_cta_done(&ws.sc->ticket[3], &s_flag)) return;
+
+    // ---- last CTA: exclusive prefix sum of the bucket sizes; last bucket needed ----------------------
+    const uint32_t t = threadIdx.x;                          // blockDim.x == 256 == buckets
+    const uint32_t mine = (t <= n_spl) ? __ldcg(&ws.bcount[t]) : 0u;
+    s_scan[t] = mine;
+    __syncthreads();
+    for (uint32_t d = 1; d < 256; d <<= 1) {
+        const uint32_t v = t >= d ? s_scan[t - d] : 0;
+        __syncthreads();
+        s_scan[t] += v;
+        __syncthreads();
+    }
+    const uint32_t excl = s_scan[t] - mine;
+    ws.boff[t] = excl;
+    if (t == 255) ws.boff[256] = s_scan[255];
+    const uint32_t n_out = ws.sc->sel_n_out;
+    if (n_out == 0) {
+        if (t == 0) { ws.sc->sel_b_last = 0; ws.sc->sel_p_end = 0; }
+    } else if (mine && excl <= n_out - 1 && n_out - 1 < excl + mine) {
+        ws.sc->sel_b_last = t;
+        ws.sc->sel_p_end = excl + mine;
+    }
+    if (t == 0) ws.sc->ticket[3] = 0;
+}
+
+// ---------------------------------------------------------------------------------------------
+// 4 scatter
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) cs_sel_scatter_kernel(cs_workspace ws)
+{
+    __shared__ uint32_t s_off[CS_MAX_SPLITTERS + 1];
+    const uint32_t c = ws.sc->sel_c, b_last = ws.sc->sel_b_last;
+    if (ws.sc->sel_p_end == 0) return;
+    s_off[threadIdx.x] = ws.boff[threadIdx.x];
+    __syncthreads();
+    for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < c; i += gridDim.x * blockDim.x) {
+        const uint32_t b = ws.cand_bkt[i];
+        if (b > b_last) continue;
+        const uint32_t pos = s_off[b] + ws.cand_slot[i];
+        ws.sort_km[pos] = ws.cand_km[i];
+        ws.sort_id[pos] = ws.cand_id[i];
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// 5 rank and emit
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+cs_sel_rank_kernel(cs_workspace ws, uint32_t k, uint32_t *__restrict__ ids_out, uint32_t *__restrict__ n_out_dev)
+{
+    __shared__ uint32_t s_off[CS_MAX_SPLITTERS + 2];
+    const uint32_t p_end = ws.sc->sel_p_end, n_out = ws.sc->sel_n_out, n_b = ws.sc->sel_n_spl + 1;
+    const uint32_t gtid = blockIdx.x * blockDim.x + threadIdx.x, nth = gridDim.x * blockDim.x;
+    for (uint32_t i = n_out + gtid; i < k; i += nth) ids_out[i] = CS_ID_NONE;
+    if (gtid == 0) *n_out_dev = n_out;
+    if (p_end == 0) return;
+    s_off[threadIdx.x] = ws.boff[threadIdx.x];
+    if (threadIdx.x == 0) s_off[256] = ws.boff[256];
+    __syncthreads();
+    for (uint32_t p = gtid; p < p_end; p += nth) {
+        uint32_t lo = 0, hi = n_b;                            // bucket of position p: last b with off[b] <= p
+        while (hi - lo > 1) {
+            const uint32_t mid = (lo + hi) >> 1;
+            if (s_off[mid] <= p) lo = mid;
+            else hi = mid;
+        }
+        const uint32_t beg = s_off[lo], end = s_off[lo + 1];
+        const unsigned long long km = ws.sort_km[p];
+        const uint32_t id = ws.sort_id[p];
+        uint32_t rank = 0;
+        for (uint32_t q = beg; q < end; ++q) rank += key_less(ws.sort_km[q], ws.sort_id[q], km, id) ? 1u : 0u;
+        if (beg + rank < n_out) ids_out[beg + rank] = id;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+static void fill_args(const cs_ctx *ctx, const cs_block_index *idx, uint32_t now, const float *fsurv, SelArgs &a)
+{
+    a.agent = idx->agent;
+    a.depth = idx->depth;
+    a.ref = idx->ref_count;
+    a.flags = idx->flags;
+    a.la = idx->last_access;
+    a.ntok = idx->n_tokens;
+    a.anchor = idx->anchor_blocks;
+    a.fsurv = fsurv;
+    a.n = idx->n_blocks;
+    a.now = now;
+    a.A = ctx->p.n_agents;
+    a.block_tokens = ctx->p.block_tokens;
+    a.gtab_len = ctx->gtab_len;
+    a.age_sat = ctx->age_sat;
+    a.lambda = ctx->p.lambda;
+    a.delta = ctx->p.delta;
+    a.tier = 0;
+    a.k = 0;
+}
+
+static uint32_t scan_grid(const cs_ctx *ctx, uint32_t n, uint32_t per_cta)
+{
+    uint32_t g = (n + per_cta - 1) / per_cta;
+    const uint32_t cap = 2u * (uint32_t)ctx->sm_count;
+    if (g > cap) g = cap;
+    return g ? g : 1u;
+}
+
+static size_t table_smem(const cs_ctx *ctx)
+{
+    return (size_t)(ctx->p.n_agents + ctx->gtab_len) * sizeof(float) + (size_t)ctx->p.n_agents * sizeof(uint16_t) + 16;
+}
+
+int cs_launch_score(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, const float *fsurv, float *scores_out,
+                    cudaStream_t s)
+{
+    SelArgs a;
+    fill_args(ctx, idx, now, fsurv, a);
+    a.anchor = nullptr;
+    const uint32_t grid = scan_grid(ctx, idx->n_blocks, SEL_THREADS * GRP);
+    cs_score_kernel<<<grid, SEL_THREADS, table_smem(ctx), s>>>(a, ctx->ws, scores_out);
+    return cs_check_launch(ctx);
+}
+
+int cs_launch_select(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, int prefetch, uint32_t tier, uint32_t k,
+                     uint32_t *ids_out, uint32_t *n_out, cudaStream_t s)
+{
+    SelArgs a;
+    fill_args(ctx, idx, now, ctx->ws.fsurv, a);
+    a.tier = tier;
+    a.k = k;
+    const uint32_t grid = scan_grid(ctx, idx->n_blocks, SEL_THREADS * GRP);
+    const uint32_t grid_c = scan_grid(ctx, idx->n_blocks, 256);
+    const size_t sm = table_smem(ctx);
+    int rc;
+    if (prefetch) cs_sel_hist_kernel<true><<<grid, SEL_THREADS, sm, s>>>(a, ctx->ws);
+    else cs_sel_hist_kernel<false><<<grid, SEL_THREADS, sm, s>>>(a, ctx->ws);
+    if ((rc = cs_check_launch(ctx)) != CS_OK) return rc;
+    if (prefetch) cs_sel_collect_kernel<true><<<grid, SEL_THREADS, sm, s>>>(a, ctx->ws);
+    else cs_sel_collect_kernel<false><<<grid, SEL_THREADS, sm, s>>>(a, ctx->ws);
+    if ((rc = cs_check_launch(ctx)) != CS_OK) return rc;
+    cs_sel_bucket_kernel<<<grid_c, 256, 0, s>>>(ctx->ws);
+    if ((rc = cs_check_launch(ctx)) != CS_OK) return rc;
+    cs_sel_scatter_kernel<<<grid_c, 256, 0, s>>>(ctx->ws);
+    if ((rc = cs_check_launch(ctx)) != CS_OK) return rc;
+    cs_sel_rank_kernel<<<grid_c, 256, 0, s>>>(ctx->ws, k, ids_out, n_out);
+    return cs_check_launch(ctx);
+}

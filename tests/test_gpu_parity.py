@@ -1,0 +1,350 @@
+"""GPU parity: the CUDA path (through the C ABI) against the CPU oracle, element by element,
+on the same seeded inputs.  Counts, tables, lists and copied bytes are compared bit-exactly;
+fp32 scores within 1e-6 relative of the fp64 oracle."""
+import numpy as np
+import pytest
+
+torch = pytest.importorskip("torch")
+
+from oracle import cs_oracle as orc
+from paper_2608_14624_b200 import binding as cs
+from paper_2608_14624_b200 import synth
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+
+DEV = "cuda:0"
+
+
+def dev(a):
+    return None if a is None else torch.from_numpy(np.ascontiguousarray(a)).to(DEV)
+
+
+def make_ctx(cfg, max_blocks, **kw):
+    p = cs.make_params(n_agents=cfg.n_agents, n_chains=cfg.n_chains, max_blocks=max_blocks,
+                       block_tokens=cfg.block_tokens, **kw)
+    return cs.CacheScout(p, DEV), orc.Oracle(H.oracle_params(p))
+
+
+def feed_trace(c, o, tr, steps=None, check_every=0):
+    n_steps = len(tr.step_off) - 1 if steps is None else steps
+    for s in range(n_steps):
+        lo, hi = int(tr.step_off[s]), int(tr.step_off[s + 1])
+        c.observe_invocations(dev(tr.chain[lo:hi]), dev(tr.agent[lo:hi]), dev(tr.evflags[lo:hi]))
+        o.observe(tr.chain[lo:hi], tr.agent[lo:hi], tr.evflags[lo:hi])
+        if check_every and s % check_every == 0:
+            H.compare_model(c, o)
+
+
+# ---- learner + scorer state ---------------------------------------------------------------------------
+@pytest.mark.parametrize("name,n_inv,chain_mode", [
+    ("tiny", 200, "session"), ("llama8b", 3000, "session"), ("llama8b", 3000, "single"),
+    ("llama70b", 4000, "session"), ("meta1m", 6400, "session")])
+def test_model_parity_stepwise(name, n_inv, chain_mode):
+    cfg = synth.CONFIGS[name]
+    if chain_mode == "single":                      # the paper's single current-agent register
+        cfg = synth.shrink(cfg, n_chains=1)
+    tr = synth.make_trace(cfg, n_invocations=n_inv, warmup_frac=0.05)
+    c, o = make_ctx(cfg, 64)
+    H.compare_model(c, o)                           # initial state: uniform matrix, no current agent
+    n_steps = len(tr.step_off) - 1
+    feed_trace(c, o, tr, check_every=max(1, n_steps // 25))
+    H.compare_model(c, o)
+    assert c.get_status() == 0
+
+
+def test_model_big_batches_and_bad_ids():
+    cfg = synth.shrink(synth.CONFIGS["llama70b"], n_chains=7)
+    tr = synth.make_trace(cfg, n_invocations=5000, warmup_frac=0.1)
+    c, o = make_ctx(cfg, 64)
+    agent = tr.agent.copy()
+    chain = tr.chain.copy()
+    agent[100] = cfg.n_agents + 3                   # skipped, status bit set
+    chain[2500] = 7
+    for lo, hi in ((0, 1), (1, 2400), (2400, 5000)):   # batches above the 1024-event shared-memory tile
+        c.observe_invocations(dev(chain[lo:hi]), dev(agent[lo:hi]), dev(tr.evflags[lo:hi]))
+        o.observe(chain[lo:hi], agent[lo:hi], tr.evflags[lo:hi])
+    H.compare_model(c, o)
+    assert c.get_status() == (cs.CS_ST_BAD_AGENT | cs.CS_ST_BAD_CHAIN)
+    assert c.get_status() == 0                      # cleared by the read
+    c.observe_invocations(None, None, None, n_events=0)     # refresh only
+    H.compare_model(c, o)
+
+
+def test_worked_examples_on_gpu(golden):
+    for fixture, A in (("worked_example_a.txt", 3), ("worked_example_b.txt", 4)):
+        g = golden(fixture)
+        trace = np.array(g["trace"][0], np.uint16)
+        p = cs.make_params(n_agents=A, max_blocks=16)
+        c = cs.CacheScout(p, DEV)
+        c.observe_invocations(dev(np.zeros(len(trace), np.uint32)), dev(trace), None)
+        m = c.get_model()
+        assert abs(m["R"] - g["R"][0][0]) < 1e-5
+        assert m["hops"].tolist() == [int(x) for x in g["E"][0]]
+        assert np.allclose(m["fsurv"], np.array(g["ptilde"][0]) + 0.01, rtol=1e-6)
+
+
+# ---- scores ----------------------------------------------------------------------------------------------
+def warm_state(cfg, n_inv, max_blocks, **kw):
+    tr = synth.make_trace(cfg, n_invocations=n_inv)
+    c, o = make_ctx(cfg, max_blocks, **kw)
+    c.observe_invocations(dev(tr.chain), dev(tr.agent), dev(tr.evflags))
+    o.observe(tr.chain, tr.agent, tr.evflags)
+    return c, o
+
+
+@pytest.mark.parametrize("name,n", [("tiny", 2560), ("tiny", 37), ("llama8b", 80000), ("llama70b", 52000 + 5)])
+@pytest.mark.parametrize("with_tokens", [True, False])
+def test_score_parity(name, n, with_tokens):
+    cfg = synth.CONFIGS[name]
+    c, o = warm_state(cfg, 500, n)
+    idx = synth.make_block_index(cfg, n=n, with_tokens=with_tokens)
+    idx.last_access[::97] = 100_000 + 5             # in the future: age clamps to 0
+    idx.last_access[1::89] = 3                      # far beyond saturation
+    d = cs.DeviceIndex.from_host(idx, DEV)
+    s = c.score_blocks(d, 100_000).cpu().numpy()
+    s64, s32 = o.scores(idx, 100_000)
+    assert np.all(np.abs(s - s64) <= H.REL_TOL * s64)
+    assert np.array_equal(s, s32)
+    # explicit sources (multi-source BFS), used for that call only
+    src = np.array([0, cfg.n_agents - 1], np.uint16)
+    s_b = c.score_blocks(d, 100_000, sources=dev(np.concatenate([src, np.zeros(6, np.uint16)]))[:2]).cpu().numpy()
+    o.survival(src)
+    s64b, s32b = o.scores(idx, 100_000)
+    o.survival()
+    assert np.array_equal(s_b, s32b) and np.all(np.abs(s_b - s64b) <= H.REL_TOL * s64b)
+    assert np.array_equal(c.score_blocks(d, 100_000).cpu().numpy(), s32)    # cached table untouched
+    assert c.get_status() == 0
+
+
+def test_score_slow_decay_uses_direct_path():
+    """A decay rate so small that the recency table does not cover all unsaturated ages."""
+    cfg = synth.CONFIGS["tiny"]
+    c, o = warm_state(cfg, 200, 4096, lam=0.0007)
+    idx = synth.make_block_index(cfg, n=4096)
+    d = cs.DeviceIndex.from_host(idx, DEV)
+    s = c.score_blocks(d, 100_000).cpu().numpy()
+    s64, s32 = o.scores(idx, 100_000)
+    assert np.all(np.abs(s - s64) <= H.REL_TOL * s64)
+    assert np.mean(s == s32) > 0.999                # device exp vs libm exp may differ in the last fp64 bit
+
+
+# ---- selections ---------------------------------------------------------------------------------------------
+def run_selects(c, o, idx, now, ks, tiers=(0, 1)):
+    d = cs.DeviceIndex.from_host(idx, DEV)
+    s64, s32 = o.scores(idx, now)
+    tolerated = 0
+    for k in ks:
+        for tier in tiers:
+            ids, n_out = c.select_victims(d, now, tier, k)
+            ids2, n_out2 = c.select_victims(d, now, tier, k)           # determinism: identical on a second run
+            g_ids, g_n = ids.cpu().numpy().view(np.uint32)[:k], int(n_out.item())
+            assert np.array_equal(g_ids, ids2.cpu().numpy().view(np.uint32)[:k]) and g_n == int(n_out2.item())
+            o_ids, o_n = o.select_victims(idx, now, tier, k, s32)
+            tolerated += H.assert_list_matches(g_ids, g_n, o_ids, o_n, s64)
+            sel = g_ids[:g_n].astype(np.int64)
+            assert not np.any(idx.flags[sel] & synth.FLAG_PINNED) and np.all(idx.ref_count[sel] == 0)
+        ids, n_out = c.select_prefetch(d, now, k)
+        g_ids, g_n = ids.cpu().numpy().view(np.uint32)[:k], int(n_out.item())
+        o_ids, o_n = o.select_prefetch(idx, now, k, s32)
+        tolerated += H.assert_list_matches(g_ids, g_n, o_ids, o_n, s64)
+    assert c.get_status() == 0
+    return tolerated
+
+
+@pytest.mark.parametrize("name,n,ks", [
+    ("tiny", 2560, (1, 32, 64, 700, 2560)),
+    ("tiny", 0, (4,)), ("tiny", 5, (1, 8)), ("tiny", 16, (3,)), ("tiny", 1029, (32, 1029)),
+    ("llama8b", 80000, (256, 384, 5000)),
+    ("llama70b", 52000, (256, 384)),
+])
+def test_select_parity(name, n, ks):
+    cfg = synth.CONFIGS[name]
+    c, o = warm_state(cfg, 1000, max(n, max(ks)), r_min=0.02)
+    H.reject_fragile(o)
+    assert o.gate
+    idx = synth.make_block_index(cfg, n=n)
+    assert run_selects(c, o, idx, 100_000, ks) == 0
+
+
+def test_select_massive_ties_and_lru_case():
+    """tau > 1 removes every edge: survival is flat and eviction must be exact LRU (Sec. 3.3),
+    with most keys tied in score so that last_access and id decide."""
+    cfg = synth.CONFIGS["llama8b"]
+    c, o = warm_state(cfg, 1000, 40000, tau=1.5)
+    idx = synth.make_block_index(cfg, n=40000, with_tokens=False)
+    idx.last_access[:] = 100_000 - 3000 - (np.arange(40000) % 211) * 5        # all ages saturated
+    assert run_selects(c, o, idx, 100_000, (1, 300, 4000, 40000)) == 0
+    ids, n_out = c.select_victims(cs.DeviceIndex.from_host(idx, DEV), 100_000, 0, 300)
+    sel = ids.cpu().numpy().view(np.uint32)[:int(n_out.item())].astype(np.int64)
+    la = int(o.last_agent[0])
+    rest = sel[idx.agent[sel] != la]                 # the current agent keeps its survival bonus
+    assert np.all(np.diff(idx.last_access[rest].astype(np.int64)) >= 0)
+
+
+def test_select_gate_closed_and_cold_start():
+    cfg = synth.CONFIGS["tiny"]
+    idx = synth.make_block_index(cfg, n=2560)
+    c, o = warm_state(cfg, 200, 2560, r_min=5.0)     # gate can never open
+    assert run_selects(c, o, idx, 100_000, (64,)) == 0
+    c2, o2 = make_ctx(cfg, 2560, r_min=-1.0)          # gate open but no current agent yet
+    assert run_selects(c2, o2, idx, 100_000, (64,)) == 0
+
+
+def test_select_without_optional_tables_and_capacity_errors():
+    cfg = synth.CONFIGS["llama70b"]
+    c, o = warm_state(cfg, 2000, 9000, r_min=0.02)
+    idx = synth.make_block_index(cfg, n=9000, with_tokens=False, with_anchor=False)
+    assert run_selects(c, o, idx, 100_000, (100,)) == 0
+    d = cs.DeviceIndex.from_host(idx, DEV)
+    with pytest.raises(cs.CacheScoutError) as e:
+        c.select_victims(d, 1, 0, 9001)
+    assert e.value.code == cs.CS_ECAPACITY
+    big = cs.DeviceIndex.from_host(synth.make_block_index(cfg, n=9016), DEV)
+    with pytest.raises(cs.CacheScoutError) as e:
+        c.select_victims(big, 1, 0, 4)
+    assert e.value.code == cs.CS_ECAPACITY
+    off = cs.DeviceIndex(d.agent[1:], d.depth, d.ref_count, d.flags, d.last_access)      # misaligned pointer
+    with pytest.raises(cs.CacheScoutError) as e:
+        c.select_victims(off, 1, 0, 4)
+    assert e.value.code == cs.CS_EINVAL
+
+
+def test_metadata_scale_first_calls():
+    """1,000,000-entry index, 256 agents, k = 10,000 victims / 2,000 prefetch candidates, state
+    evolving between calls (the launch configuration the benchmark times)."""
+    cfg = synth.CONFIGS["meta1m"]
+    N = 1_000_000
+    tr = synth.make_trace(cfg, n_invocations=64 * 40)
+    c, o = make_ctx(cfg, N, r_min=0.02)
+    idx = synth.make_block_index(cfg, n=N, tier="random")
+    rng = synth.rng_for(cfg, 9)
+    now0 = 100_000
+    for call in range(6):
+        lo, hi = int(tr.step_off[call * 4]), int(tr.step_off[call * 4 + 4])
+        c.observe_invocations(dev(tr.chain[lo:hi]), dev(tr.agent[lo:hi]), None)
+        o.observe(tr.chain[lo:hi], tr.agent[lo:hi])
+        now = now0 + call
+        d = cs.DeviceIndex.from_host(idx, DEV)
+        s64, s32 = o.scores(idx, now)
+        v_ids, v_n = c.select_victims(d, now, 0, cfg.k_victims)
+        p_ids, p_n = c.select_prefetch(d, now, cfg.k_prefetch)
+        ov, ovn = o.select_victims(idx, now, 0, cfg.k_victims, s32)
+        op, opn = o.select_prefetch(idx, now, cfg.k_prefetch, s32)
+        H.assert_list_matches(v_ids.cpu().numpy().view(np.uint32)[:cfg.k_victims], int(v_n.item()), ov, ovn, s64)
+        H.assert_list_matches(p_ids.cpu().numpy().view(np.uint32)[:cfg.k_prefetch], int(p_n.item()), op, opn, s64)
+        synth.mutate_index(idx, rng, now, ov, op, int(o.last_agent[0]), cfg.n_agents)
+    H.compare_model(c, o)
+    assert c.get_status() == 0
+
+
+# ---- mover -----------------------------------------------------------------------------------------------------
+def pinned_zeros(nbytes):
+    return torch.zeros(nbytes, dtype=torch.uint8).pin_memory()
+
+
+@pytest.mark.parametrize("gpu_layout", [synth.LAYER_MAJOR, synth.BLOCK_MAJOR])
+@pytest.mark.parametrize("host_layout", [synth.BLOCK_MAJOR, synth.LAYER_MAJOR])
+def test_mover_offload_prefetch_compact(gpu_layout, host_layout):
+    cfg = synth.CONFIGS["tiny"]
+    L, chunk, G, Hs = cfg.n_layers, cfg.chunk_bytes, 96, 160
+    rng = synth.rng_for(cfg, 5)
+    c, _ = make_ctx(cfg, 64)
+    gpu_np = synth.kv_pool_u16(G, L, chunk, rng).view(np.uint8)
+    gpu = cs.KVPool(dev(gpu_np), G, gpu_layout, L)
+    host_t = pinned_zeros(Hs * L * 2 * chunk)
+    host = cs.KVPool(host_t, Hs, host_layout, L)
+    host_np = np.zeros(Hs * L * 2 * chunk, np.uint8)
+
+    n = 41
+    src, dst = synth.mover_batch(n, G, Hs, rng)
+    src[5] = orc.ID_NONE                                       # sentinel: skipped
+    side = torch.cuda.Stream(device=DEV)
+    n_dev = dev(np.array([37, 0, 0, 0], np.uint32))            # device-resident count below n_max
+    side.wait_stream(torch.cuda.current_stream())
+    c.offload_blocks(gpu, host, dev(src), dev(dst), n_dev=n_dev, stream=side)
+    side.synchronize()
+    orc.move_blocks(gpu_np, gpu_layout, G, host_np, host_layout, Hs, L, chunk, src[:37], dst[:37])
+    assert np.array_equal(host_t.numpy(), host_np)
+
+    # prefetch the same blocks back into other GPU slots, byte-for-byte
+    back = rng.choice(G, size=37, replace=False).astype(np.uint32)
+    c.prefetch_blocks(host, gpu, dev(dst[:37]), dev(back), stream=side)
+    side.synchronize()
+    want = gpu_np.copy()
+    orc.move_blocks(host_np, host_layout, Hs, want, gpu_layout, G, L, chunk, dst[:37], back)
+    got = gpu.buf.cpu().numpy()
+    assert np.array_equal(got, want)
+    ok = src[:37] != orc.ID_NONE
+    assert np.array_equal(H.pool_view(got, gpu_layout, G, L, chunk)[back[ok]],
+                          H.pool_view(gpu_np, gpu_layout, G, L, chunk)[src[:37][ok]])
+
+    # device-to-device compaction into a packed staging pool of the other layout
+    stage = cs.KVPool(torch.zeros(n * L * 2 * chunk, dtype=torch.uint8, device=DEV), n, 1 - gpu_layout, L)
+    s2, d2 = synth.mover_batch(n, G, n, rng, packed_dst=True)
+    c.compact_blocks(gpu, stage, dev(s2), dev(d2))
+    torch.cuda.synchronize()
+    want_s = np.zeros(n * L * 2 * chunk, np.uint8)
+    orc.move_blocks(got, gpu_layout, G, want_s, 1 - gpu_layout, n, L, chunk, s2, d2)
+    assert np.array_equal(stage.buf.cpu().numpy(), want_s)
+    assert c.get_status() == 0
+
+    # an out-of-range slot is skipped and reported, nothing else is touched
+    bad_src = src.copy()
+    bad_src[0] = G
+    before = host_t.numpy().copy()
+    c.offload_blocks(gpu, host, dev(bad_src[:1]), dev(dst[:1]), stream=side)
+    side.synchronize()
+    assert c.get_status() == cs.CS_ST_BAD_SLOT
+    assert np.array_equal(host_t.numpy(), before)
+
+
+def test_mover_small_chunks_and_geometry_errors():
+    """Chunks that are not a whole number of 16 KiB pieces, and a one-block batch."""
+    cfg = synth.CONFIGS["tiny"]
+    c, _ = make_ctx(cfg, 64)
+    rng = synth.rng_for(cfg, 6)
+    for heads, hd, tok in ((3, 40, 16), (8, 128, 16), (1, 8, 1), (5, 128, 9)):
+        chunk = tok * heads * hd * 2
+        L, G = 3, 17
+        src_np = synth.kv_pool_u16(G, L, chunk, rng).view(np.uint8)
+        a = cs.KVPool(dev(src_np), G, 0, L, heads, hd, tok)
+        b = cs.KVPool(torch.zeros(G * L * 2 * chunk, dtype=torch.uint8, device=DEV), G, 1, L, heads, hd, tok)
+        s, d = synth.mover_batch(1 if heads == 1 else 9, G, G, rng)
+        c.compact_blocks(a, b, dev(s), dev(d))
+        want = np.zeros_like(src_np)
+        orc.move_blocks(src_np, 0, G, want, 1, G, L, chunk, s, d)
+        assert np.array_equal(b.buf.cpu().numpy(), want)
+    bad = cs.KVPool(b.buf, G, 1, L + 1, heads, hd, tok)
+    with pytest.raises(cs.CacheScoutError) as e:
+        cs.cs_compact_blocks(c.ctx, a.struct(), cs.cs_kv_pool(bad.buf.data_ptr(), G, 1, L + 1, heads, hd, tok, 2),
+                             dev(s), dev(d), 1)
+    assert e.value.code == cs.CS_EINVAL
+    odd = cs.cs_kv_pool(a.buf.data_ptr(), G, 0, L, 1, 3, 1, 2)          # 6-byte chunks: not 16-byte multiples
+    with pytest.raises(cs.CacheScoutError):
+        cs.cs_compact_blocks(c.ctx, odd, odd, dev(s), dev(d), 1)
+
+
+def test_offload_straight_from_select_output():
+    """The victim list and its device-resident count drive the mover without a host round trip."""
+    cfg = synth.CONFIGS["tiny"]
+    L, chunk, G, Hs = cfg.n_layers, cfg.chunk_bytes, cfg.gpu_blocks, 64
+    c, o = warm_state(cfg, 200, cfg.n_index)
+    idx = synth.make_block_index(cfg)                            # ids [0,512) GPU tier, rest host tier
+    d = cs.DeviceIndex.from_host(idx, DEV)
+    rng = synth.rng_for(cfg, 7)
+    gpu_np = synth.kv_pool_u16(G, L, chunk, rng).view(np.uint8)
+    gpu = cs.KVPool(dev(gpu_np), G, synth.LAYER_MAJOR, L)
+    host_t = pinned_zeros(Hs * L * 2 * chunk)
+    host = cs.KVPool(host_t, Hs, synth.BLOCK_MAJOR, L)
+    k = cfg.k_victims
+    ids, n_out = c.select_victims(d, 100_000, 0, k)
+    dst = dev(np.arange(k, dtype=np.uint32))
+    c.offload_blocks(gpu, host, ids, dst, n_max=k, n_dev=n_out)
+    torch.cuda.synchronize()
+    o_ids, o_n = o.select_victims(idx, 100_000, 0, k)
+    want = np.zeros(Hs * L * 2 * chunk, np.uint8)
+    orc.move_blocks(gpu_np, synth.LAYER_MAJOR, G, want, synth.BLOCK_MAJOR, Hs, L, chunk, o_ids[:o_n], np.arange(o_n))
+    assert np.array_equal(host_t.numpy(), want)
+    assert c.get_status() == 0
+    assert c.launch_count() > 0
