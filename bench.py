@@ -1,0 +1,660 @@
+#!/usr/bin/env python
+"""Benchmark of the agent-aware KV-cache hot path on B200.
+
+One "step" is one scheduler step of the Llama-3-8B-shaped configuration (32 layers x 8 KV
+heads x 128, bf16, 16-token blocks of 2 MiB; GPU pool 20,000 blocks, host tier 60,000, 12
+agents): observe the step's agent invocations, select 256 GPU-tier victims, 256 host-tier
+victims (their slots receive the offloaded blocks) and 384 prefetch candidates, compact the
+victims into a packed device staging pool, offload them to the pinned host tier and prefetch
+the candidates into free GPU slots.  Transfers run on two side streams and overlap the next
+step's selection.  value = KV bytes moved across the host link per second over the K steps.
+
+    python bench.py --gpus 1 --steps 20 --warmup 3
+    python bench.py --impl reference          # the CPU oracle on the host cores, same metric
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+METRIC = "KV block offload/prefetch GB/s vs host-link peak; blocks scored+selected/sec"
+GIB = 1 << 30
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--host-slots", type=int, default=0, help="host-tier slots backed by pinned memory (0 = auto)")
+    ap.add_argument("--no-extras", action="store_true", help="skip the mover sweep and the metadata-scale section")
+    ap.add_argument("--quick", action="store_true", help="small pools (debugging only; not a valid bench line)")
+    ap.add_argument("--workload", default="step", choices=["step", "mover", "select"],
+                    help="'mover'/'select' run one small case of that kernel family only (profiling)")
+    return ap.parse_args()
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+def mem_available_bytes():
+    with open("/proc/meminfo") as f:
+        for line in f:
+            if line.startswith("MemAvailable:"):
+                return int(line.split()[1]) * 1024
+    return 0
+
+
+# ---- clocks sampled during the timed region -----------------------------------------------------------
+class ClockSampler:
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+
+    def start(self):
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), "--query-gpu=" + self.Q,
+                                       "--format=csv,noheader,nounits", "-lms", "100"],
+                                      stdout=self.f, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.p = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.p.kill()
+        self.f.flush()
+        self.f.seek(0)
+        sm, mx, reasons = [], [], set()
+        for line in self.f.read().splitlines():
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 9:
+                continue
+            try:
+                sm.append(float(parts[1]))
+                mx.append(float(parts[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), parts[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        self.f.close()
+        os.unlink(self.f.name)
+        if sm:
+            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+# ---- the workload ---------------------------------------------------------------------------------------
+class StepWorkload:
+    """Config-1 state on one GPU: pools, index, trace, context, ring of id buffers."""
+    RING = 3
+
+    def __init__(self, args, device, n_replicas):
+        import torch
+        from paper_2608_14624_b200 import binding as cs
+        from paper_2608_14624_b200 import build, synth
+        build.build_library()
+        self.torch, self.cs, self.synth = torch, cs, synth
+        self.dev = device
+        cfg = synth.CONFIGS["llama8b"]
+        if args.quick:
+            cfg = synth.shrink(cfg, gpu_blocks=2048, host_blocks=6144)
+        self.cfg = cfg
+        G, Hs, L = cfg.gpu_blocks, cfg.host_blocks, cfg.n_layers
+        bb = cfg.block_bytes
+        # host tier: back as many of the 60,000 slots as the box's memory safely allows
+        # (torch's pinned allocator rounds sizes up to a power of two, so only powers of two are asked for)
+        want = args.host_slots or 16384
+        budget = int(0.40 * mem_available_bytes() / max(1, n_replicas))
+        fit = max(1, min(want, Hs, budget // bb))
+        self.host_backed = 1 << (int(fit).bit_length() - 1)
+        if args.quick:
+            self.host_backed = min(self.host_backed, 1024)
+        t0 = time.time()
+        self.host_buf = torch.empty(self.host_backed * bb, dtype=torch.uint8, pin_memory=True)
+        self.t_pin = time.time() - t0
+        self.gpu_buf = torch.empty(G * bb // 2, dtype=torch.bfloat16, device=device)
+        step_elems = 1 << 28
+        for lo in range(0, self.gpu_buf.numel(), step_elems):           # N(0,1) bf16 KV values, seeded
+            g = torch.Generator(device=device)
+            g.manual_seed(cfg.seed + lo // step_elems)
+            self.gpu_buf[lo:lo + step_elems].normal_(generator=g)
+        self.k_v, self.k_p = cfg.k_victims, cfg.k_prefetch
+        self.stage_buf = torch.empty(self.k_v * bb, dtype=torch.uint8, device=device)
+        self.gpu_pool = cs.KVPool(self.gpu_buf, G, cs.CS_LAYER_MAJOR, L)
+        self.host_pool = cs.KVPool(self.host_buf, self.host_backed, cs.CS_BLOCK_MAJOR, L, first_id=G)
+        self.stage_pool = cs.KVPool(self.stage_buf, self.k_v, cs.CS_BLOCK_MAJOR, L)
+
+        # index: ids [0, G) GPU tier, [G, G+Hs) host tier; host entries without backing are not VALID
+        idx = synth.make_block_index(cfg)
+        if self.host_backed < Hs:
+            idx.flags[G + self.host_backed:] &= np.uint8(~synth.FLAG_VALID & 0xFF)
+        self.idx_host = idx
+        self.N = idx.n
+        self.didx = cs.DeviceIndex.from_host(idx, device)
+        self.la_i32 = self.didx.last_access.view(torch.int32)
+        self.pin_idx = {k: torch.from_numpy(getattr(idx, k)).pin_memory()
+                        for k in ("agent", "depth", "ref_count", "flags", "last_access", "n_tokens")}
+        self.meta_bytes = sum(int(t.numel() * t.element_size()) for t in self.pin_idx.values())
+
+        # trace, events of step s padded to 16 per step so slices are cheap
+        self.tr = synth.make_trace(cfg)
+        self.n_steps = len(self.tr.step_off) - 1
+        self.ev_chain = torch.from_numpy(self.tr.chain).pin_memory()
+        self.ev_agent = torch.from_numpy(self.tr.agent).pin_memory()
+        self.ev_flags = torch.from_numpy(self.tr.evflags).pin_memory()
+        self.d_chain, self.d_agent, self.d_flags = (t.to(device) for t in (self.ev_chain, self.ev_agent, self.ev_flags))
+        self.e2e_chain = torch.empty(64, dtype=self.ev_chain.dtype, device=device)
+        self.e2e_agent = torch.empty(64, dtype=self.ev_agent.dtype, device=device)
+        self.e2e_flags = torch.empty(64, dtype=self.ev_flags.dtype, device=device)
+
+        p = cs.make_params(n_agents=cfg.n_agents, n_chains=cfg.n_chains, max_blocks=self.N,
+                           block_tokens=cfg.block_tokens, r_min=0.02)
+        self.params = p
+        self.c = cs.CacheScout(p, device)
+        # ring of list buffers: dst[b][:k_v] receives the GPU victims of step s (b = s % RING) and, one
+        # step later, serves with the reserve tail as the free GPU slots the prefetch fills
+        reserve = torch.arange(G - (self.k_p - self.k_v), G, dtype=torch.int32, device=device)
+        self.dst = []
+        for _ in range(self.RING):
+            t = torch.empty(self.k_p, dtype=torch.int32, device=device)
+            t[:self.k_v] = torch.arange(0, self.k_v, dtype=torch.int32, device=device)
+            t[self.k_v:] = reserve
+            self.dst.append(t)
+        mk = lambda n: [torch.zeros(max(n, 4), dtype=torch.int32, device=device) for _ in range(self.RING)]
+        self.hv, self.pf = mk(self.k_v), mk(self.k_p)
+        self.vn, self.hn, self.pn = mk(1), mk(1), mk(1)
+        self.packed = torch.arange(self.k_v, dtype=torch.int32, device=device)
+        self.res_pin = torch.zeros(self.k_v * 2 + self.k_p + 16, dtype=torch.int32).pin_memory()
+        self.main = torch.cuda.current_stream(device)
+        self.side_o = torch.cuda.Stream(device=device)
+        self.side_p = torch.cuda.Stream(device=device)
+        self.done_o = [None] * self.RING
+        self.done_p = [None] * self.RING
+        self.now0 = 100_000
+        self.bytes_per_step = (self.k_v + self.k_p) * bb
+        self.timers = {"select": [], "compact": [], "offload": [], "prefetch": [], "observe": []}
+        # warm the learner so that the prefetch gate has something to work with
+        self.c.observe_invocations(self.d_chain[:2000], self.d_agent[:2000], self.d_flags[:2000])
+        torch.cuda.synchronize(device)
+
+    def step(self, s, e2e=False, timed=False):
+        torch, c = self.torch, self.c
+        b, prev = s % self.RING, (s - 1) % self.RING
+        main = self.main
+        # ring slot b is rewritten now: the transfers that read it (step s - RING) must be over
+        if self.done_o[b] is not None:
+            main.wait_event(self.done_o[b])
+            main.wait_event(self.done_p[b])
+        now = self.now0 + s
+        st = (600 + s) % (self.n_steps - 1)
+        lo, hi = int(self.tr.step_off[st]), int(self.tr.step_off[st + 1])
+        n_ev = hi - lo
+        ev = (lambda: torch.cuda.Event(enable_timing=True)) if timed else (lambda: None)
+        t = [ev() for _ in range(10)]
+        rec = lambda e, stream: e.record(stream) if e is not None else None
+        if e2e:      # this step's inputs come from pinned host memory
+            self.e2e_chain[:n_ev].copy_(self.ev_chain[lo:hi], non_blocking=True)
+            self.e2e_agent[:n_ev].copy_(self.ev_agent[lo:hi], non_blocking=True)
+            self.e2e_flags[:n_ev].copy_(self.ev_flags[lo:hi], non_blocking=True)
+            for k, src in self.pin_idx.items():
+                getattr(self.didx, k).copy_(src, non_blocking=True)
+            chain, agent, flags = self.e2e_chain, self.e2e_agent, self.e2e_flags
+        else:
+            chain, agent, flags = self.d_chain[lo:hi], self.d_agent[lo:hi], self.d_flags[lo:hi]
+        rec(t[0], main)
+        c.observe_invocations(chain, agent, flags, n_events=n_ev)
+        rec(t[1], main)
+        vict = self.dst[b][:self.k_v]
+        c.select_victims(self.didx, now, 0, self.k_v, vict, self.vn[b])
+        c.select_victims(self.didx, now, 1, self.k_v, self.hv[b], self.hn[b])
+        c.select_prefetch(self.didx, now, self.k_p, self.pf[b], self.pn[b])
+        rec(t[2], main)
+        c.compact_blocks(self.gpu_pool, self.stage_pool, vict, self.packed, n_max=self.k_v, n_dev=self.vn[b])
+        rec(t[3], main)
+        ready = torch.cuda.Event()
+        ready.record(main)
+        # offload on side stream 1: GPU victims -> the slots of the host-tier victims
+        self.side_o.wait_event(ready)
+        rec(t[4], self.side_o)
+        c.offload_blocks(self.gpu_pool, self.host_pool, vict, self.hv[b], n_max=self.k_v, n_dev=self.vn[b],
+                         stream=self.side_o)
+        rec(t[5], self.side_o)
+        self.done_o[b] = torch.cuda.Event()
+        self.done_o[b].record(self.side_o)
+        # prefetch on side stream 2 into the slots freed one step earlier (their offload must be over)
+        self.side_p.wait_event(ready)
+        if self.done_o[prev] is not None:
+            self.side_p.wait_event(self.done_o[prev])
+        rec(t[6], self.side_p)
+        c.prefetch_blocks(self.host_pool, self.gpu_pool, self.pf[b], self.dst[prev], n_max=self.k_p, n_dev=self.pn[b],
+                          stream=self.side_p)
+        rec(t[7], self.side_p)
+        self.done_p[b] = torch.cuda.Event()
+        self.done_p[b].record(self.side_p)
+        # engine bookkeeping (plumbing, not the method): refilled victim slots are touched now, prefetched
+        # host entries now have a GPU copy
+        vi = vict.long().clamp_(min=0)
+        self.la_i32[vi] = now
+        pi = self.pf[b][:self.k_p].long().clamp_(min=0)
+        self.didx.flags[pi] |= self.cs.CS_FLAG_OTHER_COPY
+        if e2e:      # the step's result goes back to the host
+            r = self.res_pin
+            r[:self.k_v].copy_(vict, non_blocking=True)
+            r[self.k_v:2 * self.k_v].copy_(self.hv[b][:self.k_v], non_blocking=True)
+            r[2 * self.k_v:2 * self.k_v + self.k_p].copy_(self.pf[b][:self.k_p], non_blocking=True)
+            r[-16:-15].copy_(self.vn[b][:1], non_blocking=True)
+            r[-15:-14].copy_(self.hn[b][:1], non_blocking=True)
+            r[-14:-13].copy_(self.pn[b][:1], non_blocking=True)
+            main.synchronize()
+        if timed:
+            self._pending = getattr(self, "_pending", [])
+            self._pending.append(t)
+
+    def drain(self):
+        self.main.wait_stream(self.side_o)
+        self.main.wait_stream(self.side_p)
+
+    def collect_timers(self):
+        for t in getattr(self, "_pending", []):
+            self.timers["observe"].append(t[0].elapsed_time(t[1]))
+            self.timers["select"].append(t[1].elapsed_time(t[2]))
+            self.timers["compact"].append(t[2].elapsed_time(t[3]))
+            self.timers["offload"].append(t[4].elapsed_time(t[5]))
+            self.timers["prefetch"].append(t[6].elapsed_time(t[7]))
+        self._pending = []
+
+    def e2e_bytes(self):
+        ev = 8 * 7          # <= 8 events x (4 + 2 + 1) bytes
+        h2d = self.meta_bytes + ev + self.k_p * self.cfg.block_bytes
+        d2h = (2 * self.k_v + self.k_p + 3) * 4 + self.k_v * self.cfg.block_bytes
+        return h2d, d2h
+
+
+def host_link_peak(torch, device, n_bytes=GIB, reps=10):
+    """Pinned cudaMemcpyAsync of one contiguous buffer, each direction alone and both at once."""
+    h = torch.empty(n_bytes, dtype=torch.uint8, pin_memory=True)
+    h2 = torch.empty(n_bytes, dtype=torch.uint8, pin_memory=True)
+    d = torch.empty(n_bytes, dtype=torch.uint8, device=device)
+    d2 = torch.empty(n_bytes, dtype=torch.uint8, device=device)
+    s1, s2 = torch.cuda.Stream(device=device), torch.cuda.Stream(device=device)
+    out = {}
+    for name in ("d2h", "h2d", "bidir"):
+        best = 0.0
+        for _ in range(reps):
+            torch.cuda.synchronize(device)
+            e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+            e0.record(s1)
+            s2.wait_event(e0)
+            if name in ("d2h", "bidir"):
+                with torch.cuda.stream(s1):
+                    h.copy_(d, non_blocking=True)
+            if name in ("h2d", "bidir"):
+                with torch.cuda.stream(s2):
+                    d2.copy_(h2, non_blocking=True)
+            e2.record(s2)
+            s1.wait_event(e2)
+            e1.record(s1)
+            torch.cuda.synchronize(device)
+            ms = e0.elapsed_time(e1)
+            moved = n_bytes * (2 if name == "bidir" else 1)
+            best = max(best, moved / ms / 1e6)
+        out[name] = best
+    del h, h2, d, d2
+    return out
+
+
+def time_call(torch, stream, fn, reps, warm=1):
+    for _ in range(warm):
+        fn()
+    stream.synchronize()
+    ts = []
+    for _ in range(reps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        fn()
+        e1.record(stream)
+        stream.synchronize()
+        ts.append(e0.elapsed_time(e1))
+    return float(np.median(ts)), float(min(ts))
+
+
+def mover_sweep(w, hbm_peak, link):
+    """Batches of 1..4096 uniformly random scattered blocks: offload, prefetch, device-to-device,
+    GPU pool addressed layer-major and block-major (same memory, two address formulas)."""
+    torch, cs, synth, c = w.torch, w.cs, w.synth, w.c
+    cfg, dev = w.cfg, w.dev
+    rng = synth.rng_for(cfg, 11)
+    G, L, bb = cfg.gpu_blocks, cfg.n_layers, cfg.block_bytes
+    rows = []
+    side = w.side_o
+    up = lambda a: torch.from_numpy(a.view(np.int32)).to(dev)
+    for n in (1, 8, 64, 512, 4096):
+        if n > w.host_backed or 2 * n > G:
+            continue
+        src, dst_h = synth.mover_batch(n, G - n, w.host_backed, rng)
+        dst_h = dst_h + G                                                   # host pool ids start at G
+        d_src, d_dst_h = up(src.astype(np.uint32)), up(dst_h.astype(np.uint32))
+        d_back = up((G - n + np.arange(n)).astype(np.uint32))              # disjoint from every src
+        reps = 5 if n <= 512 else 3
+        for lay_name, lay in (("layer_major", cs.CS_LAYER_MAJOR), ("block_major", cs.CS_BLOCK_MAJOR)):
+            gp = cs.KVPool(w.gpu_buf, G, lay, L)
+            med_o, best_o = time_call(torch, side, lambda: c.offload_blocks(gp, w.host_pool, d_src, d_dst_h, stream=side), reps)
+            med_p, best_p = time_call(torch, side, lambda: c.prefetch_blocks(w.host_pool, gp, d_dst_h, d_back, stream=side), reps)
+            med_c, best_c = time_call(torch, side, lambda: c.compact_blocks(gp, gp, d_src, d_back, stream=side), reps)
+            gb = n * bb / 1e9
+            rows.append({"blocks": n, "gpu_layout": lay_name,
+                         "offload_GBps": gb / (med_o / 1e3), "offload_frac_of_link": gb / (med_o / 1e3) / link["d2h"],
+                         "prefetch_GBps": gb / (med_p / 1e3), "prefetch_frac_of_link": gb / (med_p / 1e3) / link["h2d"],
+                         "d2d_GBps_rw": 2 * gb / (med_c / 1e3), "d2d_frac_of_hbm": 2 * gb / (med_c / 1e3) / hbm_peak,
+                         "offload_ms": med_o, "prefetch_ms": med_p, "d2d_ms": med_c})
+    return rows
+
+
+def metadata_scale(torch, cs, synth, dev, hbm_peak, calls=200):
+    """1,000,000-entry index, 256 agents: observe 64 events + select 10,000 victims + 2,000 prefetch
+    candidates per call; the first `calls` calls are timed with CUDA events on the stream."""
+    cfg = synth.CONFIGS["meta1m"]
+    N = 1_000_000
+    idx = synth.make_block_index(cfg, n=N, tier="random")
+    d = cs.DeviceIndex.from_host(idx, dev)
+    tr = synth.make_trace(cfg, n_invocations=64 * (calls + 40))
+    p = cs.make_params(n_agents=cfg.n_agents, n_chains=cfg.n_chains, max_blocks=N, block_tokens=cfg.block_tokens, r_min=0.02)
+    c = cs.CacheScout(p, dev)
+    ch, ag = torch.from_numpy(tr.chain).to(dev), torch.from_numpy(tr.agent).to(dev)
+    c.observe_invocations(ch[:64 * 30], ag[:64 * 30], None)
+    v = torch.empty(cfg.k_victims, dtype=torch.int32, device=dev)
+    pf = torch.empty(cfg.k_prefetch, dtype=torch.int32, device=dev)
+    vn, pn = torch.zeros(4, dtype=torch.int32, device=dev), torch.zeros(4, dtype=torch.int32, device=dev)
+    la = d.last_access.view(torch.int32)
+    stream = torch.cuda.current_stream(dev)
+    evs = []
+    l0 = c.launch_count()
+    for call in range(calls + 5):
+        now = 100_000 + call
+        lo = 64 * (30 + call)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        c.observe_invocations(ch[lo:lo + 64], ag[lo:lo + 64], None)
+        c.select_victims(d, now, 0, cfg.k_victims, v, vn)
+        c.select_prefetch(d, now, cfg.k_prefetch, pf, pn)
+        e1.record(stream)
+        la[v.long().clamp_(min=0)] = now                      # untimed bookkeeping: victims refilled
+        d.flags[pf.long().clamp_(min=0)] &= 0xFB              # prefetched entries leave the host tier
+        if call >= 5:
+            evs.append((e0, e1))
+    torch.cuda.synchronize(dev)
+    launches = (c.launch_count() - l0) / (calls + 5)
+    ms = np.array([a.elapsed_time(b) for a, b in evs])
+    per_call = float(np.median(ms)) * 1e-3
+    algo_bytes = 2 * N * 11 + (cfg.k_victims + cfg.k_prefetch) * 4          # two selects each read 11 B per entry
+    return {"workload": "metadata-scale: 1,000,000-entry index, 256 agents, k=10000 victims + 2000 prefetch per call",
+            "calls_timed": calls, "us_per_call_median": per_call * 1e6, "us_per_call_min": float(ms.min()) * 1e3,
+            "blocks_scored_selected_per_s": 2 * N / per_call,
+            "algorithmic_GBps": algo_bytes / per_call / 1e9, "frac_of_hbm_peak": algo_bytes / per_call / 1e9 / hbm_peak,
+            "kernel_launches_per_call": launches, "n_out": [int(vn[0].item()), int(pn[0].item())]}
+
+
+# ---- the oracle on the host cores (cpu_baseline and --impl reference) ----------------------------------------
+class OracleStep:
+    """The same scheduler step computed by the CPU oracle.  Bounded sample: the selections run over
+    the full 80,000-entry index, the mover copies the same 256 + 384 blocks of 2 MiB but between two
+    2,048-slot stand-in pools in host memory (ids taken modulo 2,048), single thread."""
+
+    def __init__(self):
+        from oracle import cs_oracle as orc
+        from paper_2608_14624_b200 import synth
+        self.orc, self.synth = orc, synth
+        cfg = synth.CONFIGS["llama8b"]
+        self.cfg = cfg
+        self.o = orc.Oracle(orc.Params(n_agents=cfg.n_agents, n_chains=cfg.n_chains, block_tokens=cfg.block_tokens, r_min=0.02))
+        self.tr = synth.make_trace(cfg)
+        self.o.observe(self.tr.chain[:2000], self.tr.agent[:2000], self.tr.evflags[:2000])
+        self.idx = synth.make_block_index(cfg)
+        self.S = 2048
+        rng = synth.rng_for(cfg, 21)
+        self.a = synth.kv_pool_u16(self.S, cfg.n_layers, cfg.chunk_bytes, rng).view(np.uint8)
+        self.b = np.zeros_like(self.a)
+        self.bytes_per_step = (cfg.k_victims + cfg.k_prefetch) * cfg.block_bytes
+
+    def step(self, s):
+        cfg, o, idx = self.cfg, self.o, self.idx
+        now = 100_000 + s
+        st = (250 + s) % (len(self.tr.step_off) - 2)
+        lo, hi = int(self.tr.step_off[st]), int(self.tr.step_off[st + 1])
+        o.observe(self.tr.chain[lo:hi], self.tr.agent[lo:hi], self.tr.evflags[lo:hi])
+        _, s32 = o.scores(idx, now)
+        v, vn = o.select_victims(idx, now, 0, cfg.k_victims, s32)
+        h, hn = o.select_victims(idx, now, 1, cfg.k_victims, s32)
+        p, pn = o.select_prefetch(idx, now, cfg.k_prefetch, s32)
+        L, ch, S = cfg.n_layers, cfg.chunk_bytes, self.S
+        m = lambda x, n: (x[:n] % S).astype(np.uint32)
+        self.orc.move_blocks(self.a, 0, S, self.b, 1, S, L, ch, m(v, vn), m(h, vn))                       # offload
+        self.orc.move_blocks(self.b, 1, S, self.a, 0, S, L, ch, m(p, pn), np.arange(pn, dtype=np.uint32) % S)  # prefetch
+        idx.last_access[v[:vn].astype(np.int64)] = now
+        return vn + pn
+
+
+def run_reference(args):
+    """--impl reference: the oracle, as it stands, timed on the host cores (rank 0 only)."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    ow = OracleStep()
+    for s in range(args.warmup):
+        ow.step(s)
+    t0 = time.perf_counter()
+    for s in range(args.steps):
+        ow.step(args.warmup + s)
+    dt = time.perf_counter() - t0
+    gbps = ow.bytes_per_step * args.steps / dt / 1e9
+    sample = ("full 80,000-entry index for observe/score/select; mover copies the step's 256+384 blocks of 2 MiB "
+              "between two 2,048-slot host stand-in pools (ids modulo 2,048)")
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": gbps, "unit": "GB/s", "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "u8", "data": "synthetic",
+        "config": {"workload": "llama8b-kv step (config 1): observe + 3 selects over 80,000 entries + offload 256 / prefetch 384 blocks of 2 MiB",
+                   "sample": sample},
+        "cpu_baseline": {"value": gbps, "unit": "GB/s", "cores": 1, "kind": "oracle", "sample": sample,
+                         "blocks_scored_selected_per_s": 3 * ow.idx.n * args.steps / dt},
+        "e2e": {"value": gbps, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+# ---- main ------------------------------------------------------------------------------------------------------
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+    import torch
+    import torch.distributed as dist
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=device)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(device)
+
+    hbm_peak, peak_kind = measured_peaks()
+    w = StepWorkload(args, device, world)
+    cs, synth = w.cs, w.synth
+    if args.workload != "step":          # small single-family runs for profiling
+        if args.workload == "mover":
+            n = 512
+            rng = synth.rng_for(w.cfg, 11)
+            src, _ = synth.mover_batch(n, w.cfg.gpu_blocks - n, n, rng)
+            d_src = torch.from_numpy(src.view(np.int32)).to(device)
+            d_back = torch.arange(w.cfg.gpu_blocks - n, w.cfg.gpu_blocks, dtype=torch.int32, device=device)
+            for _ in range(max(1, args.steps)):
+                w.c.compact_blocks(w.gpu_pool, w.gpu_pool, d_src, d_back)
+        else:
+            for s in range(max(1, args.steps)):
+                w.c.select_victims(w.didx, w.now0 + s, 0, w.k_v, w.dst[0][:w.k_v], w.vn[0])
+                w.c.select_prefetch(w.didx, w.now0 + s, w.k_p, w.pf[0], w.pn[0])
+        torch.cuda.synchronize(device)
+        print(json.dumps({"workload": args.workload, "launches": w.c.launch_count()}))
+        return
+
+    link = host_link_peak(torch, device) if rank == 0 else None
+
+    # ---- device-resident inputs: the headline value ------------------------------------------------------
+    for s in range(args.warmup):
+        w.step(s)
+    w.drain()
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    l0 = w.c.launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(w.main)
+    for s in range(args.steps):
+        w.step(args.warmup + s, timed=True)
+    w.drain()
+    e1.record(w.main)
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    launches = w.c.launch_count() - l0
+    ms = torch.tensor([e0.elapsed_time(e1)], device=device)
+    if world > 1:
+        dist.all_reduce(ms, op=dist.ReduceOp.MAX)
+    total_ms = float(ms.item())
+    w.collect_timers()
+    status = w.c.get_status()
+    n_out = [int(w.vn[(args.warmup + args.steps - 1) % w.RING][0].item()),
+             int(w.hn[(args.warmup + args.steps - 1) % w.RING][0].item()),
+             int(w.pn[(args.warmup + args.steps - 1) % w.RING][0].item())]
+
+    # ---- end to end: inputs from pinned host memory, results read back, every step ---------------------------
+    base = args.warmup + args.steps
+    for s in range(2):
+        w.step(base + s, e2e=True)
+    w.drain()
+    barrier()
+    f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    f0.record(w.main)
+    for s in range(args.steps):
+        w.step(base + 2 + s, e2e=True)
+    w.drain()
+    f1.record(w.main)
+    barrier()
+    ms2 = torch.tensor([f0.elapsed_time(f1)], device=device)
+    if world > 1:
+        dist.all_reduce(ms2, op=dist.ReduceOp.MAX)
+    e2e_ms = float(ms2.item())
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    value = world * w.bytes_per_step * args.steps / (total_ms / 1e3) / 1e9
+    e2e_value = world * w.bytes_per_step * args.steps / (e2e_ms / 1e3) / 1e9
+    bb = w.cfg.block_bytes
+    med = lambda k: float(np.median(w.timers[k])) if w.timers[k] else None
+    t_c, t_o, t_p, t_s, t_ob = med("compact"), med("offload"), med("prefetch"), med("select"), med("observe")
+    d2d_gbps = 2 * w.k_v * bb / (t_c / 1e3) / 1e9
+    off_gbps = w.k_v * bb / (t_o / 1e3) / 1e9
+    pre_gbps = w.k_p * bb / (t_p / 1e3) / 1e9
+    sel_bytes = 3 * w.N * 11 + (2 * w.k_v + w.k_p) * 4
+    h2d, d2h = w.e2e_bytes()
+    traffic = None
+    tpath = os.path.join(ROOT, "profiles", "ncu_traffic.json")
+    if os.path.exists(tpath):
+        with open(tpath) as f:
+            traffic = json.load(f).get("cs_mover_kernel_d2d_256_blocks_bytes")
+
+    out = {
+        "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "u8", "data": "synthetic",
+        "config": {"workload": "llama8b-kv step (config 1): 32 layers x 8 KV heads x 128 bf16, 2 MiB blocks; GPU pool %d blocks "
+                               "layer-major, host tier %d blocks (%d backed by pinned memory); 12 agents; per step: observe <= 8 "
+                               "invocations, select 256 GPU victims + 256 host victims + 384 prefetch candidates over %d "
+                               "entries, compact 256, offload 256, prefetch 384 blocks" % (
+                                   w.cfg.gpu_blocks, w.cfg.host_blocks, w.host_backed, w.N),
+                   "l2_policy": "inputs larger than L2: every step moves 1.75 GiB of scattered blocks; index 0.9 MB is L2-resident by design",
+                   "replicas": "replicas only (no data-path collective)", "pin_seconds": round(w.t_pin, 2), "quick": bool(args.quick)},
+        "blocks_scored_selected_per_s": world * 3 * w.N / (t_s / 1e3),
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+        "roofline": {"kernel": "cs_mover_kernel (device-to-device compaction of the 256 victims, inside the step)", "bound": "hbm",
+                     "achieved": d2d_gbps, "peak": hbm_peak, "unit": "GB/s", "frac": d2d_gbps / hbm_peak, "traffic": traffic,
+                     "peak_kind": "of %s" % peak_kind, "algorithmic_bytes_per_launch": 2 * w.k_v * bb, "ms_per_launch": t_c},
+        "host_link": {"peak_d2h_GBps": link["d2h"], "peak_h2d_GBps": link["h2d"], "peak_bidir_GBps": link["bidir"],
+                      "how": "pinned cudaMemcpyAsync of 1 GiB, best of 10, same run",
+                      "offload_GBps": off_gbps, "offload_frac": off_gbps / link["d2h"], "offload_ms": t_o,
+                      "prefetch_GBps": pre_gbps, "prefetch_frac": pre_gbps / link["h2d"], "prefetch_ms": t_p,
+                      "step_frac_of_bidir": value / world / link["bidir"],
+                      "note": "offload and prefetch of a step overlap (full duplex); per-direction times are measured while the other direction is busy"},
+        "select": {"ms_three_selects": t_s, "ms_observe": t_ob, "algorithmic_bytes": sel_bytes,
+                   "achieved_GBps": sel_bytes / (t_s / 1e3) / 1e9, "frac_of_hbm_peak": sel_bytes / (t_s / 1e3) / 1e9 / hbm_peak,
+                   "n_out_last_step": n_out, "device_status": status},
+        "e2e": {"value": e2e_value, "unit": "GB/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "ms_per_step": e2e_ms / args.steps,
+                "includes": "per step: H2D of the step's events and of the 80,000-entry index from pinned memory, D2H of the three id lists and counts, host sync on the result"},
+    }
+    if not args.no_extras and world == 1:
+        out["mover_sweep"] = mover_sweep(w, hbm_peak, link)
+        del w
+        torch.cuda.empty_cache()
+        out["metadata_scale"] = metadata_scale(torch, cs, synth, device, hbm_peak)
+    # the oracle, as it stands, on this machine's host cores
+    ow = OracleStep()
+    ow.step(0)
+    t0 = time.perf_counter()
+    n_or = 0
+    while time.perf_counter() - t0 < 10.0 and n_or < 40:
+        ow.step(1 + n_or)
+        n_or += 1
+    dt = time.perf_counter() - t0
+    out["cpu_baseline"] = {"value": ow.bytes_per_step * n_or / dt / 1e9, "unit": "GB/s", "cores": 1, "kind": "oracle",
+                           "sample": "%d oracle steps: selections over the full 80,000-entry index, mover copies 256+384 blocks of 2 MiB "
+                                     "between two 2,048-slot host stand-in pools (ids modulo 2,048)" % n_or,
+                           "blocks_scored_selected_per_s": 3 * ow.idx.n * n_or / dt, "ms_per_step": dt / n_or * 1e3}
+    print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -14,8 +14,9 @@
  *    cudaHostRegister; with unified addressing the host pointer is used as is).  The
  *    library never allocates or frees device or pinned memory; it owns only the small
  *    host-side cs_ctx.  All scratch lives in the workspace the caller hands to cs_create().
- *  - Every array pointer must be 16-byte aligned (the kernels use 128-bit accesses);
- *    a violation is CS_EINVAL before anything is launched.
+ *  - Block-index arrays, score / id output arrays and pool bases must be 16-byte aligned (the
+ *    kernels use 128-bit accesses); event arrays, slot lists and counts need only their natural
+ *    alignment.  A violation is CS_EINVAL before anything is launched.
  *  - All calls on one cs_ctx except the three mover calls share workspace scratch: issue
  *    them on one stream (or order them with events).  The mover calls touch no workspace
  *    scratch besides the status word and may run on a side stream concurrently.
@@ -104,10 +105,15 @@ typedef struct cs_block_index {
  * layer l, plane p (0 = K, 1 = V), slot s:
  *   CS_LAYER_MAJOR: ((l*2 + p)*n_slots + s) * chunk_bytes
  *   CS_BLOCK_MAJOR: ((s*n_layers + l)*2 + p) * chunk_bytes
- * base is dev or pinned; chunk_bytes must be a multiple of 16. */
+ * base is dev or pinned; chunk_bytes must be a multiple of 16.
+ * Slot lists given to the mover hold block ids of the index; the pool's slot is
+ * id - first_id (first_id = 0 when ids are slot numbers).  This lets the lists the select
+ * calls emit drive the mover directly when the index numbers the GPU tier [0, G) and the host
+ * tier [G, G + H).  Ids outside [first_id, first_id + n_slots) are out of range. */
 typedef struct cs_kv_pool {
     void *base;
     uint32_t n_slots, layout, n_layers, n_kv_heads, head_dim, block_tokens, elem_bytes;
+    uint32_t first_id;
 } cs_kv_pool;
 
 /* ---- life cycle -------------------------------------------------------------------------------- */

@@ -45,7 +45,7 @@ class cs_block_index(C.Structure):
 class cs_kv_pool(C.Structure):
     _fields_ = [("base", C.c_void_p), ("n_slots", C.c_uint32), ("layout", C.c_uint32), ("n_layers", C.c_uint32),
                 ("n_kv_heads", C.c_uint32), ("head_dim", C.c_uint32), ("block_tokens", C.c_uint32),
-                ("elem_bytes", C.c_uint32)]
+                ("elem_bytes", C.c_uint32), ("first_id", C.c_uint32)]
 
 
 class CacheScoutError(RuntimeError):
@@ -239,6 +239,7 @@ class KVPool:
     head_dim: int = 128
     block_tokens: int = 16
     elem_bytes: int = 2
+    first_id: int = 0
 
     @property
     def chunk_bytes(self) -> int:
@@ -251,7 +252,7 @@ class KVPool:
     def struct(self) -> cs_kv_pool:
         assert self.buf.numel() * self.buf.element_size() >= self.n_slots * self.block_bytes
         return cs_kv_pool(_ptr(self.buf), self.n_slots, self.layout, self.n_layers, self.n_kv_heads, self.head_dim,
-                          self.block_tokens, self.elem_bytes)
+                          self.block_tokens, self.elem_bytes, self.first_id)
 
 
 class CacheScout:

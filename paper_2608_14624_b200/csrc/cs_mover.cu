@@ -18,7 +18,7 @@
 struct MoverArgs {
     const char *src;
     char *dst;
-    uint32_t src_total, dst_total, src_layout, dst_layout, L, pieces;
+    uint32_t src_total, dst_total, src_layout, dst_layout, L, pieces, src_first, dst_first;
     unsigned long long chunk;
     const uint32_t *src_slots, *dst_slots, *n_dev;
     uint32_t n_max;
@@ -42,8 +42,10 @@ __global__ void __launch_bounds__(MV_THREADS) cs_mover_kernel(MoverArgs a)
         const uint32_t i = (uint32_t)(w / per_block);
         const uint32_t r = (uint32_t)(w - (unsigned long long)i * per_block);
         const uint32_t lp = r / a.pieces, piece = r - lp * a.pieces;
-        const uint32_t s = __ldg(a.src_slots + i), d = __ldg(a.dst_slots + i);
+        uint32_t s = __ldg(a.src_slots + i), d = __ldg(a.dst_slots + i);
         if (s == CS_ID_NONE || d == CS_ID_NONE) continue;
+        s -= a.src_first;                                   // ids below first_id wrap and fail the range check
+        d -= a.dst_first;
         if (s >= a.src_total || d >= a.dst_total) {
             if (threadIdx.x == 0 && r == 0) atomicOr(a.status, CS_ST_BAD_SLOT);
             continue;
@@ -76,6 +78,8 @@ int cs_launch_mover(cs_ctx *ctx, const cs_kv_pool *src, const cs_kv_pool *dst, c
     a.dst = (char *)dst->base;
     a.src_total = src->n_slots;
     a.dst_total = dst->n_slots;
+    a.src_first = src->first_id;
+    a.dst_first = dst->first_id;
     a.src_layout = src->layout;
     a.dst_layout = dst->layout;
     a.L = src->n_layers;

@@ -317,10 +317,10 @@ def test_mover_small_chunks_and_geometry_errors():
         assert np.array_equal(b.buf.cpu().numpy(), want)
     bad = cs.KVPool(b.buf, G, 1, L + 1, heads, hd, tok)
     with pytest.raises(cs.CacheScoutError) as e:
-        cs.cs_compact_blocks(c.ctx, a.struct(), cs.cs_kv_pool(bad.buf.data_ptr(), G, 1, L + 1, heads, hd, tok, 2),
+        cs.cs_compact_blocks(c.ctx, a.struct(), cs.cs_kv_pool(bad.buf.data_ptr(), G, 1, L + 1, heads, hd, tok, 2, 0),
                              dev(s), dev(d), 1)
     assert e.value.code == cs.CS_EINVAL
-    odd = cs.cs_kv_pool(a.buf.data_ptr(), G, 0, L, 1, 3, 1, 2)          # 6-byte chunks: not 16-byte multiples
+    odd = cs.cs_kv_pool(a.buf.data_ptr(), G, 0, L, 1, 3, 1, 2, 0)          # 6-byte chunks: not 16-byte multiples
     with pytest.raises(cs.CacheScoutError):
         cs.cs_compact_blocks(c.ctx, odd, odd, dev(s), dev(d), 1)
 
