@@ -166,6 +166,29 @@ int cs_select_victims(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, uint
 int cs_select_prefetch(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, uint32_t k,
                        uint32_t *ids_out, uint32_t *n_out, cs_stream_t stream);
 
+/* Victim selection for callers that cannot allocate device memory (no counterpart in the
+ * paper: it exists for embedders, not for the method).  A serving engine that gave the whole
+ * GPU to its KV pool at start-up, a hook that runs while the host application forbids
+ * allocation, or a process with a fixed memory budget can own inputs and outputs but cannot
+ * provide a workspace.  This call needs neither a cs_ctx nor a workspace: the scratch of the
+ * select kernels lives in a static device array inside the library (2 MiB + 40 KiB on every
+ * GPU that loads the library, held until the process exits), and the call itself allocates
+ * nothing, on the host or on the device.
+ *   p      : the method's constants (n_chains and max_blocks are ignored).
+ *   fsurv  : dev [n_agents], the survival factor p~ + delta of every agent (Eq. 8 plus the floor
+ *            of Eq. 9), e.g. the fsurv table cs_get_model() returned earlier.
+ *   the rest as for cs_select_victims(), with the same eligibility, order, padding and n_out.
+ * Limits: idx->n_blocks and k at most CS_STATIC_MAX_BLOCKS, else CS_ECAPACITY.  Entries whose
+ * agent is out of range are skipped without a status report.
+ * The first call on a device looks up the device address of the static array (with that device
+ * current); make that first call outside any stream capture.  All calls share the one array,
+ * which keeps the previous call's contents: every call re-initialises what must start at zero,
+ * and two calls of one process that overlap on the same GPU (different streams or threads)
+ * race.  Issue them on one stream, or order them with events. */
+#define CS_STATIC_MAX_BLOCKS 65536u
+int cs_select_victims_static(const cs_params *p, const float *fsurv, const cs_block_index *idx, uint32_t now,
+                             uint32_t tier, uint32_t k, uint32_t *ids_out, uint32_t *n_out, cs_stream_t stream);
+
 /* ---- block mover (the paper reuses the serving engine's offload path, Sec. 4; these calls
  *      are that path written for B200) ------------------------------------------------------------ */
 

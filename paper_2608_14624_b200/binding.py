@@ -22,12 +22,13 @@ CS_AGENT_NONE, CS_ID_NONE, CS_HOP_NONE = 0xFFFF, 0xFFFFFFFF, 0xFFFF
 CS_FLAG_VALID, CS_FLAG_PINNED, CS_FLAG_TIER_HOST, CS_FLAG_OTHER_COPY = 1, 2, 4, 8
 CS_EV_WARMUP = 1
 CS_LAYER_MAJOR, CS_BLOCK_MAJOR = 0, 1
+CS_STATIC_MAX_BLOCKS = 65536
 
 # every symbol include/cachescout.h declares
 EXPORTS = ("cs_workspace_bytes", "cs_create", "cs_destroy", "cs_observe_invocations", "cs_score_blocks",
            "cs_select_victims", "cs_select_prefetch", "cs_offload_blocks", "cs_prefetch_blocks",
            "cs_compact_blocks", "cs_get_model", "cs_get_status", "cs_launch_count", "cs_set_mover_ctas",
-           "cs_last_cuda_error", "cs_strerror", "cs_version")
+           "cs_last_cuda_error", "cs_strerror", "cs_version", "cs_select_victims_static")
 
 
 class cs_params(C.Structure):
@@ -76,6 +77,8 @@ def lib():
         L.cs_score_blocks.argtypes = [vp, C.POINTER(cs_block_index), u32, vp, u32, vp, vp]
         L.cs_select_victims.argtypes = [vp, C.POINTER(cs_block_index), u32, u32, u32, vp, vp, vp]
         L.cs_select_prefetch.argtypes = [vp, C.POINTER(cs_block_index), u32, u32, vp, vp, vp]
+        L.cs_select_victims_static.argtypes = [C.POINTER(cs_params), vp, C.POINTER(cs_block_index), u32, u32, u32,
+                                               vp, vp, vp]
         for name in ("cs_offload_blocks", "cs_prefetch_blocks", "cs_compact_blocks"):
             getattr(L, name).argtypes = [vp, C.POINTER(cs_kv_pool), C.POINTER(cs_kv_pool), vp, vp, u32, vp, vp]
         L.cs_get_model.argtypes = [vp] * 10
@@ -149,6 +152,15 @@ def cs_select_victims(ctx, idx: cs_block_index, now: int, tier: int, k: int, ids
 def cs_select_prefetch(ctx, idx: cs_block_index, now: int, k: int, ids_out, n_out, stream=None):
     _chk(lib().cs_select_prefetch(ctx, C.byref(idx), now, k, _ptr(ids_out), _ptr(n_out), _stream(stream)),
          "cs_select_prefetch", ctx)
+
+
+def cs_select_victims_static(params: cs_params, fsurv, idx: cs_block_index, now: int, tier: int, k: int, ids_out,
+                             n_out, stream=None):
+    """Victim selection without a context or workspace, for callers that cannot allocate device
+    memory: the kernels' scratch is a static array inside the library.  `fsurv` is the device
+    table of survival factors (one fp32 per agent); at most CS_STATIC_MAX_BLOCKS entries / k."""
+    _chk(lib().cs_select_victims_static(C.byref(params), _ptr(fsurv), C.byref(idx), now, tier, k, _ptr(ids_out),
+                                        _ptr(n_out), _stream(stream)), "cs_select_victims_static")
 
 
 def cs_offload_blocks(ctx, gpu: cs_kv_pool, host: cs_kv_pool, src_slots, dst_slots, n_max: int, n_dev=None, stream=None):

@@ -593,3 +593,118 @@ int cs_launch_select(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, int p
     cs_sel_rank_kernel<<<grid_c, 256, 0, s>>>(ctx->ws, k, ids_out, n_out);
     return cs_check_launch(ctx);
 }
+
+// =============================================================================================
+// Victim selection for callers that cannot allocate device memory.
+//
+// Some embedders of this library never get to call cudaMalloc: a serving engine that has handed
+// the whole GPU to its own KV pool at start-up, a plug-in hook that runs while allocation is
+// forbidden (inside a region where the host application has frozen its memory map), or a
+// process whose memory budget is fixed by its launcher.  They can pass inputs and outputs they
+// already own, but not a workspace.  For them the scratch of the select kernels (recency table,
+// histogram, candidate keys, buckets, counters) lives in the file-scope array below, which
+// every GPU that loads the library holds until the process exits.
+//
+// The array's name is only a host-side handle: the device address is obtained once per device
+// with cudaGetSymbolAddress() and that pointer is what the kernels get.
+// =============================================================================================
+#include <mutex>
+
+#define CS_STATIC_MAX_DEVICES 64
+#define CS_STATIC_ALIGN(x) (((x) + 255u) / 256u * 256u)
+// layout of the static scratch, byte offsets (every region 256-byte aligned)
+#define CS_SO_SC 0u
+#define CS_SO_GTAB (CS_SO_SC + CS_STATIC_ALIGN(sizeof(cs_scalars)))
+#define CS_SO_HIST (CS_SO_GTAB + CS_GTAB_MAX * 4u)
+#define CS_SO_SPLKM (CS_SO_HIST + CS_HIST_BINS * 4u)
+#define CS_SO_SPLID (CS_SO_SPLKM + CS_STATIC_ALIGN((CS_MAX_SPLITTERS + 1u) * 8u))
+#define CS_SO_BCOUNT (CS_SO_SPLID + CS_STATIC_ALIGN((CS_MAX_SPLITTERS + 1u) * 4u))
+#define CS_SO_BOFF (CS_SO_BCOUNT + CS_STATIC_ALIGN((CS_MAX_SPLITTERS + 1u) * 4u))
+#define CS_SO_CANDKM (CS_SO_BOFF + CS_STATIC_ALIGN((CS_MAX_SPLITTERS + 2u) * 4u))
+#define CS_SO_SORTKM (CS_SO_CANDKM + CS_STATIC_MAX_BLOCKS * 8u)
+#define CS_SO_CANDID (CS_SO_SORTKM + CS_STATIC_MAX_BLOCKS * 8u)
+#define CS_SO_CANDBKT (CS_SO_CANDID + CS_STATIC_MAX_BLOCKS * 4u)
+#define CS_SO_CANDSLOT (CS_SO_CANDBKT + CS_STATIC_MAX_BLOCKS * 4u)
+#define CS_SO_SORTID (CS_SO_CANDSLOT + CS_STATIC_MAX_BLOCKS * 4u)
+#define CS_STATIC_BYTES (CS_SO_SORTID + CS_STATIC_MAX_BLOCKS * 4u)
+
+static __device__ __align__(256) unsigned char cs_static_scratch[CS_STATIC_BYTES];   // 2 MiB + 40 KiB
+
+static std::mutex g_static_mu;
+static unsigned char *g_static_ptr[CS_STATIC_MAX_DEVICES];     // device address of the array, per device
+static int g_static_sms[CS_STATIC_MAX_DEVICES];
+
+// Everything the select kernels expect to find zeroed, and the recency table for this call's
+// lambda / delta.  The array keeps the previous call's contents, so this runs on every call.
+__global__ void cs_static_prepare_kernel(cs_workspace ws, uint32_t gtab_len, float lambda, float delta)
+{
+    const uint32_t tid = blockIdx.x * blockDim.x + threadIdx.x, nth = gridDim.x * blockDim.x;
+    for (uint32_t i = tid; i < CS_HIST_BINS; i += nth) ws.hist[i] = 0;
+    for (uint32_t i = tid; i <= CS_MAX_SPLITTERS; i += nth) ws.bcount[i] = 0;
+    for (uint32_t i = tid; i < gtab_len; i += nth) ws.gtab[i] = cs_recency(lambda, delta, i);
+    if (tid == 0) {
+        cs_scalars z;
+        memset(&z, 0, sizeof(z));
+        z.last_agent = CS_AGENT_NONE;
+        *ws.sc = z;
+    }
+}
+
+extern "C" int cs_select_victims_static(const cs_params *p, const float *fsurv, const cs_block_index *idx,
+                                        uint32_t now, uint32_t tier, uint32_t k, uint32_t *ids_out, uint32_t *n_out,
+                                        cs_stream_t stream)
+{
+    int rc = cs_validate_params(p);
+    if (rc != CS_OK) return rc;
+    if (!idx || !fsurv || (((uintptr_t)fsurv) & 3u) || tier > 1) return CS_EINVAL;
+    if (idx->n_blocks > CS_STATIC_MAX_BLOCKS || k > CS_STATIC_MAX_BLOCKS) return CS_ECAPACITY;
+    if (!n_out || (((uintptr_t)n_out) & 3u)) return CS_EINVAL;
+    if (k && (!ids_out || (((uintptr_t)ids_out) & 15u))) return CS_EINVAL;
+    if (idx->n_blocks) {
+        if (!idx->agent || !idx->depth || !idx->ref_count || !idx->flags || !idx->last_access) return CS_EINVAL;
+        const uintptr_t any = (uintptr_t)idx->agent | (uintptr_t)idx->depth | (uintptr_t)idx->ref_count |
+                              (uintptr_t)idx->flags | (uintptr_t)idx->last_access | (uintptr_t)idx->n_tokens;
+        if (any & 15u) return CS_EINVAL;
+    }
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= CS_STATIC_MAX_DEVICES) return CS_ECUDA;
+    {
+        // first call on this device: resolve the device address of the array (once, with the device current)
+        std::lock_guard<std::mutex> lock(g_static_mu);
+        if (!g_static_ptr[dev]) {
+            void *ptr = nullptr;
+            if (cudaGetSymbolAddress(&ptr, cs_static_scratch) != cudaSuccess || !ptr) return CS_ECUDA;
+            int sms = 0;
+            if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return CS_ECUDA;
+            g_static_sms[dev] = sms;
+            g_static_ptr[dev] = (unsigned char *)ptr;
+        }
+    }
+    unsigned char *base = g_static_ptr[dev];
+    cs_ctx ctx;                                        // host-side descriptor only; nothing is allocated
+    memset(&ctx, 0, sizeof(ctx));
+    ctx.p = *p;
+    ctx.p.max_blocks = CS_STATIC_MAX_BLOCKS;
+    cs_recency_table_shape(p, &ctx.gtab_len, &ctx.age_sat);
+    ctx.device = dev;
+    ctx.sm_count = g_static_sms[dev];
+    cs_workspace &ws = ctx.ws;
+    ws.sc = (cs_scalars *)(base + CS_SO_SC);
+    ws.gtab = (float *)(base + CS_SO_GTAB);
+    ws.hist = (uint32_t *)(base + CS_SO_HIST);
+    ws.spl_km = (unsigned long long *)(base + CS_SO_SPLKM);
+    ws.spl_id = (uint32_t *)(base + CS_SO_SPLID);
+    ws.bcount = (uint32_t *)(base + CS_SO_BCOUNT);
+    ws.boff = (uint32_t *)(base + CS_SO_BOFF);
+    ws.cand_km = (unsigned long long *)(base + CS_SO_CANDKM);
+    ws.sort_km = (unsigned long long *)(base + CS_SO_SORTKM);
+    ws.cand_id = (uint32_t *)(base + CS_SO_CANDID);
+    ws.cand_bkt = (uint32_t *)(base + CS_SO_CANDBKT);
+    ws.cand_slot = (uint32_t *)(base + CS_SO_CANDSLOT);
+    ws.sort_id = (uint32_t *)(base + CS_SO_SORTID);
+    ws.fsurv = const_cast<float *>(fsurv);             // input table, read only
+    cudaStream_t s = (cudaStream_t)stream;
+    cs_static_prepare_kernel<<<16, 256, 0, s>>>(ws, ctx.gtab_len, p->lambda, p->delta);
+    if ((rc = cs_check_launch(&ctx)) != CS_OK) return rc;
+    return cs_launch_select(&ctx, idx, now, 0, tier, k, ids_out, n_out, s);
+}
