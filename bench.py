@@ -40,9 +40,13 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--host-slots", type=int, default=0, help="host-tier slots backed by pinned memory (0 = auto)")
     ap.add_argument("--no-extras", action="store_true", help="skip the mover sweep and the metadata-scale section")
+    ap.add_argument("--offload-width", type=int, default=0, help="warp pipelines of the offload mover (0 = library default)")
+    ap.add_argument("--prefetch-width", type=int, default=0, help="warp pipelines of the prefetch mover (0 = library default)")
     ap.add_argument("--quick", action="store_true", help="small pools (debugging only; not a valid bench line)")
     ap.add_argument("--workload", default="step", choices=["step", "mover", "select"],
-                    help="'mover'/'select' run one small case of that kernel family only (profiling)")
+                    help="'mover'/'select' run one small case of that kernel family only (profiler captures)")
+    ap.add_argument("--skip-aux", action="store_true",
+                    help="timed steps only: no link-peak probe, end-to-end pass, extras or CPU baseline (profiler launch lists)")
     return ap.parse_args()
 
 
@@ -201,6 +205,9 @@ class StepWorkload:
         self.done_o = [None] * self.RING
         self.done_p = [None] * self.RING
         self.now0 = 100_000
+        self.w_off, self.w_pre = args.offload_width, args.prefetch_width
+        self.fifo = [torch.zeros(self.k_p, dtype=torch.int64, device=device) for _ in range(8)]
+        self.fifo_used = 0
         self.bytes_per_step = (self.k_v + self.k_p) * bb
         self.timers = {"select": [], "compact": [], "offload": [], "prefetch": [], "observe": []}
         # warm the learner so that the prefetch gate has something to work with
@@ -246,6 +253,8 @@ class StepWorkload:
         # offload on side stream 1: GPU victims -> the slots of the host-tier victims
         self.side_o.wait_event(ready)
         rec(t[4], self.side_o)
+        if self.w_off:
+            c.set_mover_ctas(self.w_off, 0)
         c.offload_blocks(self.gpu_pool, self.host_pool, vict, self.hv[b], n_max=self.k_v, n_dev=self.vn[b],
                          stream=self.side_o)
         rec(t[5], self.side_o)
@@ -256,8 +265,12 @@ class StepWorkload:
         if self.done_o[prev] is not None:
             self.side_p.wait_event(self.done_o[prev])
         rec(t[6], self.side_p)
+        if self.w_pre:
+            c.set_mover_ctas(self.w_pre, 0)
         c.prefetch_blocks(self.host_pool, self.gpu_pool, self.pf[b], self.dst[prev], n_max=self.k_p, n_dev=self.pn[b],
                           stream=self.side_p)
+        if self.w_off or self.w_pre:
+            c.set_mover_ctas(0, 0)
         rec(t[7], self.side_p)
         self.done_p[b] = torch.cuda.Event()
         self.done_p[b].record(self.side_p)
@@ -267,6 +280,12 @@ class StepWorkload:
         self.la_i32[vi] = now
         pi = self.pf[b][:self.k_p].long().clamp_(min=0)
         self.didx.flags[pi] |= self.cs.CS_FLAG_OTHER_COPY
+        # ... and the GPU copies made 8 steps ago count as evicted again, so the candidate set is stationary
+        slot = self.fifo[s % 8]
+        if self.fifo_used >= 8:
+            self.didx.flags[slot] &= 0xF7
+        slot.copy_(pi)
+        self.fifo_used += 1
         if e2e:      # the step's result goes back to the host
             r = self.res_pin
             r[:self.k_v].copy_(vict, non_blocking=True)
@@ -397,6 +416,7 @@ def metadata_scale(torch, cs, synth, dev, hbm_peak, calls=200):
     vn, pn = torch.zeros(4, dtype=torch.int32, device=dev), torch.zeros(4, dtype=torch.int32, device=dev)
     la = d.last_access.view(torch.int32)
     stream = torch.cuda.current_stream(dev)
+    fifo = [torch.zeros(cfg.k_prefetch, dtype=torch.int64, device=dev) for _ in range(8)]
     evs = []
     l0 = c.launch_count()
     for call in range(calls + 5):
@@ -409,7 +429,11 @@ def metadata_scale(torch, cs, synth, dev, hbm_peak, calls=200):
         c.select_prefetch(d, now, cfg.k_prefetch, pf, pn)
         e1.record(stream)
         la[v.long().clamp_(min=0)] = now                      # untimed bookkeeping: victims refilled
-        d.flags[pf.long().clamp_(min=0)] &= 0xFB              # prefetched entries leave the host tier
+        pi = pf.long().clamp_(min=0)
+        d.flags[pi] &= 0xFB                                   # prefetched entries leave the host tier ...
+        if call >= 8:
+            d.flags[fifo[call % 8]] |= 4                      # ... and return to it 8 calls later (stationary state)
+        fifo[call % 8].copy_(pi)
         if call >= 5:
             evs.append((e0, e1))
     torch.cuda.synchronize(dev)
@@ -490,6 +514,54 @@ def run_reference(args):
     }))
 
 
+def profile_case(args, torch, device):
+    """Small cases for profiler captures (a few GB on the device, inputs larger than L2).
+    mover : 2,048-block GPU pool (4 GiB), 512-slot pinned host tier (1 GiB); per step one
+            device-to-device move of 512 scattered blocks, one offload and one prefetch of 256.
+    select: metadata-scale index (1,000,000 entries, 256 agents); per step observe 64 events,
+            select 10,000 victims and 2,000 prefetch candidates."""
+    from paper_2608_14624_b200 import binding as cs
+    from paper_2608_14624_b200 import build, synth
+    build.build_library()
+    if args.workload == "mover":
+        cfg = synth.CONFIGS["llama8b"]
+        G, Hs, L, bb = 2048, 512, cfg.n_layers, cfg.block_bytes
+        c = cs.CacheScout(cs.make_params(n_agents=cfg.n_agents, max_blocks=64), device)
+        gpu = cs.KVPool(torch.randint(0, 255, (G * bb,), dtype=torch.uint8, device=device), G, cs.CS_LAYER_MAJOR, L)
+        host = cs.KVPool(torch.empty(Hs * bb, dtype=torch.uint8, pin_memory=True), Hs, cs.CS_BLOCK_MAJOR, L)
+        rng = synth.rng_for(cfg, 11)
+        up = lambda a: torch.from_numpy(a.view(np.int32)).to(device)
+        src, _ = synth.mover_batch(512, G - 512, 512, rng)
+        d_src, d_back = up(src), torch.arange(G - 512, G, dtype=torch.int32, device=device)
+        hs, hd = synth.mover_batch(256, G, Hs, rng)
+        d_hs, d_hd = up(hs), up(hd)
+        if args.offload_width or args.prefetch_width:
+            c.set_mover_ctas(max(args.offload_width, args.prefetch_width), 0)
+        for _ in range(max(1, args.steps)):
+            c.compact_blocks(gpu, gpu, d_src, d_back)
+            c.offload_blocks(gpu, host, d_hs, d_hd)
+            c.prefetch_blocks(host, gpu, d_hd, d_hs)
+    else:
+        cfg = synth.CONFIGS["meta1m"]
+        N = 1_000_000
+        d = cs.DeviceIndex.from_host(synth.make_block_index(cfg, n=N, tier="random"), device)
+        tr = synth.make_trace(cfg, n_invocations=64 * (args.steps + 40))
+        c = cs.CacheScout(cs.make_params(n_agents=cfg.n_agents, n_chains=cfg.n_chains, max_blocks=N,
+                                         block_tokens=cfg.block_tokens, r_min=0.02), device)
+        ch, ag = torch.from_numpy(tr.chain).to(device), torch.from_numpy(tr.agent).to(device)
+        c.observe_invocations(ch[:64 * 30], ag[:64 * 30], None)
+        v = torch.empty(cfg.k_victims, dtype=torch.int32, device=device)
+        pf = torch.empty(cfg.k_prefetch, dtype=torch.int32, device=device)
+        vn, pn = torch.zeros(4, dtype=torch.int32, device=device), torch.zeros(4, dtype=torch.int32, device=device)
+        for s in range(max(1, args.steps)):
+            lo = 64 * (30 + s)
+            c.observe_invocations(ch[lo:lo + 64], ag[lo:lo + 64], None)
+            c.select_victims(d, 100_000 + s, 0, cfg.k_victims, v, vn)
+            c.select_prefetch(d, 100_000 + s, cfg.k_prefetch, pf, pn)
+    torch.cuda.synchronize(device)
+    print(json.dumps({"workload": args.workload, "launches": c.launch_count(), "device_status": c.get_status()}))
+
+
 # ---- main ------------------------------------------------------------------------------------------------------
 def main():
     args = parse_args()
@@ -515,26 +587,12 @@ def main():
         torch.cuda.synchronize(device)
 
     hbm_peak, peak_kind = measured_peaks()
+    if args.workload != "step":          # one small case of one kernel family, for profiler captures
+        profile_case(args, torch, device)
+        return
     w = StepWorkload(args, device, world)
     cs, synth = w.cs, w.synth
-    if args.workload != "step":          # small single-family runs for profiling
-        if args.workload == "mover":
-            n = 512
-            rng = synth.rng_for(w.cfg, 11)
-            src, _ = synth.mover_batch(n, w.cfg.gpu_blocks - n, n, rng)
-            d_src = torch.from_numpy(src.view(np.int32)).to(device)
-            d_back = torch.arange(w.cfg.gpu_blocks - n, w.cfg.gpu_blocks, dtype=torch.int32, device=device)
-            for _ in range(max(1, args.steps)):
-                w.c.compact_blocks(w.gpu_pool, w.gpu_pool, d_src, d_back)
-        else:
-            for s in range(max(1, args.steps)):
-                w.c.select_victims(w.didx, w.now0 + s, 0, w.k_v, w.dst[0][:w.k_v], w.vn[0])
-                w.c.select_prefetch(w.didx, w.now0 + s, w.k_p, w.pf[0], w.pn[0])
-        torch.cuda.synchronize(device)
-        print(json.dumps({"workload": args.workload, "launches": w.c.launch_count()}))
-        return
-
-    link = host_link_peak(torch, device) if rank == 0 else None
+    link = host_link_peak(torch, device) if (rank == 0 and not args.skip_aux) else None
 
     # ---- device-resident inputs: the headline value ------------------------------------------------------
     for s in range(args.warmup):
@@ -563,6 +621,14 @@ def main():
     n_out = [int(w.vn[(args.warmup + args.steps - 1) % w.RING][0].item()),
              int(w.hn[(args.warmup + args.steps - 1) % w.RING][0].item()),
              int(w.pn[(args.warmup + args.steps - 1) % w.RING][0].item())]
+
+    if args.skip_aux:
+        if rank == 0:
+            print(json.dumps({"workload": "step", "ms_per_step": total_ms / args.steps, "gpu_launches": int(launches),
+                              "value": world * w.bytes_per_step * args.steps / (total_ms / 1e3) / 1e9, "n_out": n_out}))
+        if world > 1:
+            dist.destroy_process_group()
+        return
 
     # ---- end to end: inputs from pinned host memory, results read back, every step ---------------------------
     base = args.warmup + args.steps

@@ -51,6 +51,7 @@ typedef struct CUstream_st *cs_stream_t;   /* the same type as cudaStream_t */
 #define CS_ST_BAD_CHAIN 2u      /* an event named a chain >= n_chains */
 #define CS_ST_BAD_SLOT 4u       /* a mover list entry named a slot >= n_slots */
 #define CS_ST_BAD_SOURCE 8u     /* a BFS source >= n_agents */
+#define CS_ST_TIMEOUT 16u       /* a bounded wait inside a kernel ran out; the transfer is incomplete */
 
 /* ---- sentinels ---------------------------------------------------------------------------- */
 #define CS_AGENT_NONE 0xFFFFu      /* "no current agent yet" (the initial state of Algorithm 1) */
@@ -223,6 +224,13 @@ int cs_launch_count(cs_ctx *ctx, uint64_t *n_launches);
 /* Grid sizes of the mover (0 keeps the default): CTAs used for transfers that cross the
  * host link, and for device-to-device moves. */
 int cs_set_mover_ctas(cs_ctx *ctx, uint32_t host_link_ctas, uint32_t d2d_ctas);
+
+/* Data path of the mover: CS_MOVER_AUTO (= bulk), CS_MOVER_LDST (128-bit loads and stores by
+ * every thread), CS_MOVER_BULK (1-D bulk asynchronous copies staged through shared memory). */
+#define CS_MOVER_AUTO 0u
+#define CS_MOVER_LDST 1u
+#define CS_MOVER_BULK 2u
+int cs_set_mover_path(cs_ctx *ctx, uint32_t path);
 
 /* cudaError_t of the last failing CUDA call on this context (0 if none). */
 int cs_last_cuda_error(cs_ctx *ctx);

@@ -235,19 +235,19 @@ static int mover_common(cs_ctx *ctx, const cs_kv_pool *src, const cs_kv_pool *ds
 int cs_offload_blocks(cs_ctx *ctx, const cs_kv_pool *gpu, const cs_kv_pool *host, const uint32_t *src_slots,
                       const uint32_t *dst_slots, uint32_t n_max, const uint32_t *n_dev, cs_stream_t side)
 {
-    return mover_common(ctx, gpu, host, src_slots, dst_slots, n_max, n_dev, 1, side);
+    return mover_common(ctx, gpu, host, src_slots, dst_slots, n_max, n_dev, CS_MOVE_OFFLOAD, side);
 }
 
 int cs_prefetch_blocks(cs_ctx *ctx, const cs_kv_pool *host, const cs_kv_pool *gpu, const uint32_t *src_slots,
                        const uint32_t *dst_slots, uint32_t n_max, const uint32_t *n_dev, cs_stream_t side)
 {
-    return mover_common(ctx, host, gpu, src_slots, dst_slots, n_max, n_dev, 1, side);
+    return mover_common(ctx, host, gpu, src_slots, dst_slots, n_max, n_dev, CS_MOVE_PREFETCH, side);
 }
 
 int cs_compact_blocks(cs_ctx *ctx, const cs_kv_pool *src, const cs_kv_pool *dst, const uint32_t *src_slots,
                       const uint32_t *dst_slots, uint32_t n_max, const uint32_t *n_dev, cs_stream_t stream)
 {
-    return mover_common(ctx, src, dst, src_slots, dst_slots, n_max, n_dev, 0, stream);
+    return mover_common(ctx, src, dst, src_slots, dst_slots, n_max, n_dev, CS_MOVE_D2D, stream);
 }
 
 int cs_get_model(cs_ctx *ctx, uint32_t *C_out, float *P_out, uint16_t *amax_out, uint16_t *hops_out,
@@ -298,6 +298,13 @@ int cs_set_mover_ctas(cs_ctx *ctx, uint32_t host_link_ctas, uint32_t d2d_ctas)
     if (!ctx) return CS_EINVAL;
     ctx->host_link_ctas = host_link_ctas;
     ctx->d2d_ctas = d2d_ctas;
+    return CS_OK;
+}
+
+int cs_set_mover_path(cs_ctx *ctx, uint32_t path)
+{
+    if (!ctx || path > CS_MOVER_BULK) return CS_EINVAL;
+    ctx->mover_path = path;
     return CS_OK;
 }
 

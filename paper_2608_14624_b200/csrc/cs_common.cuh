@@ -9,6 +9,10 @@
 #error "libcachescout is written for sm_100a (B200) only"
 #endif
 
+#define CS_MOVE_D2D 0
+#define CS_MOVE_OFFLOAD 1
+#define CS_MOVE_PREFETCH 2
+
 #define CS_HIST_BINS 4096u        // first radix digit of the select: top 12 bits of the primary key
 #define CS_MAX_SPLITTERS 255u     // bucket sort of the candidates: up to 256 buckets
 #define CS_SAMPLE 1024u           // candidates sampled to choose the splitters
@@ -70,6 +74,8 @@ struct cs_ctx {
     int device;
     int sm_count;
     uint32_t host_link_ctas, d2d_ctas;
+    uint32_t mover_path;   // CS_MOVER_*
+    int bulk_attr_set;     // shared-memory opt-in of the bulk kernel done on this device
     uint64_t n_launches;
     int last_cuda_error;
 };
@@ -89,7 +95,7 @@ int cs_launch_score(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, const 
 int cs_launch_select(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, int prefetch, uint32_t tier,
                      uint32_t k, uint32_t *ids_out, uint32_t *n_out, cudaStream_t s);
 int cs_launch_mover(cs_ctx *ctx, const cs_kv_pool *src, const cs_kv_pool *dst, const uint32_t *src_slots,
-                    const uint32_t *dst_slots, uint32_t n_max, const uint32_t *n_dev, int crosses_host_link,
+                    const uint32_t *dst_slots, uint32_t n_max, const uint32_t *n_dev, int kind,
                     cudaStream_t s);
 
 static inline int cs_check_launch(cs_ctx *ctx)

@@ -2,23 +2,37 @@
 // may differ in location (HBM or pinned host memory), slot count and layout.  The paper reuses
 // its serving engine's offload path unchanged (Sec. 4); this file is that path for B200.
 //
-// Unit of work: one "piece" (<= 16 KiB) of one chunk (one layer, one plane, one block).
-// Consecutive work items are consecutive pieces of the same chunk, so neighbouring CTAs
-// stream neighbouring addresses.  A CTA issues all loads of its piece (4 x 128-bit per thread)
-// before the first store, which keeps 16 KiB per CTA in flight; the slot lists and the
-// optional device-resident count come straight from the select kernels' output, so no host
-// round trip sits between a decision and its transfer.  Pinned host memory is addressed
-// directly by the SMs (unified addressing), which lets the destination slots stay scattered.
+// Unit of work: one "piece" of one chunk (one layer, one plane, one block).  Consecutive work
+// items are consecutive pieces, so neighbouring CTAs stream neighbouring addresses.  The slot
+// lists and the optional device-resident count come straight from the select kernels' output,
+// so no host round trip sits between a decision and its transfer.  Pinned host memory is
+// addressed directly by the SMs (unified addressing), which lets both slot lists stay scattered.
+//
+// Two data paths:
+//  * bulk path (default): every warp of a CTA runs its own software pipeline of 1-D bulk
+//    asynchronous copies (TMA): global -> shared memory ring (mbarrier completion), shared ->
+//    global (bulk groups).  One lane per warp issues; the copy engines of the SM move the
+//    bytes, so a handful of CTAs keep hundreds of KiB in flight without occupying the
+//    load/store pipelines that co-resident kernels need.
+//  * load/store path: 4 x 128-bit loads per thread in flight, streaming cache hints.  Used when
+//    asked for (cs_set_mover_path) and as the comparison point in the profiles.
+// No copy is multicast and no kernel waits on another CTA; every mbarrier wait is bounded.
 #include "cs_common.cuh"
 
 #define MV_THREADS 256
 #define MV_UNROLL 4
-#define MV_PIECE (MV_THREADS * MV_UNROLL * 16)      // bytes per work item
+#define MV_PIECE (MV_THREADS * MV_UNROLL * 16)      // bytes per work item of the load/store path
+
+#define TM_WARPS 4                                   // independent pipelines per CTA
+#define TM_STAGES 3                                  // ring slots per pipeline
+#define TM_PIECE 16384u                              // bytes per ring slot
+#define TM_SMEM (TM_WARPS * TM_STAGES * TM_PIECE)    // 192 KiB
+#define TM_SPIN_LIMIT (1u << 20)                     // bounded mbarrier wait (polls with back-off: >= 0.1 s)
 
 struct MoverArgs {
     const char *src;
     char *dst;
-    uint32_t src_total, dst_total, src_layout, dst_layout, L, pieces, src_first, dst_first;
+    uint32_t src_total, dst_total, src_layout, dst_layout, L, pieces, src_first, dst_first, piece_bytes, n_pipes;
     unsigned long long chunk;
     const uint32_t *src_slots, *dst_slots, *n_dev;
     uint32_t n_max;
@@ -32,29 +46,52 @@ __device__ __forceinline__ unsigned long long chunk_offset(uint32_t layout, uint
     return (((unsigned long long)s * L + l) * 2 + p) * chunk;
 }
 
-__global__ void __launch_bounds__(MV_THREADS) cs_mover_kernel(MoverArgs a)
+// Resolves work item w to a source / destination address and a byte count; false = skip.
+__device__ __forceinline__ bool resolve_piece(const MoverArgs &a, unsigned long long w, uint32_t per_block,
+                                              const char *&sp, char *&dp, uint32_t &bytes, bool report)
+{
+    const uint32_t i = (uint32_t)(w / per_block);
+    const uint32_t r = (uint32_t)(w - (unsigned long long)i * per_block);
+    const uint32_t lp = r / a.pieces, piece = r - lp * a.pieces;
+    uint32_t s = __ldg(a.src_slots + i), d = __ldg(a.dst_slots + i);
+    if (s == CS_ID_NONE || d == CS_ID_NONE) return false;
+    s -= a.src_first;                                   // ids below first_id wrap and fail the range check
+    d -= a.dst_first;
+    if (s >= a.src_total || d >= a.dst_total) {
+        if (report && r == 0) atomicOr(a.status, CS_ST_BAD_SLOT);
+        return false;
+    }
+    const unsigned long long in_chunk = (unsigned long long)piece * a.piece_bytes;
+    sp = a.src + chunk_offset(a.src_layout, a.L, a.src_total, lp >> 1, lp & 1, s, a.chunk) + in_chunk;
+    dp = a.dst + chunk_offset(a.dst_layout, a.L, a.dst_total, lp >> 1, lp & 1, d, a.chunk) + in_chunk;
+    const unsigned long long left = a.chunk - in_chunk;
+    bytes = (uint32_t)(left < a.piece_bytes ? left : a.piece_bytes);
+    return true;
+}
+
+__device__ __forceinline__ uint32_t mover_count(const MoverArgs &a)
 {
     uint32_t n = a.n_max;
     if (a.n_dev) { const uint32_t nd = *a.n_dev; n = nd < n ? nd : n; }
+    return n;
+}
+
+// ---------------------------------------------------------------------------------------------
+// load/store path
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(MV_THREADS) cs_mover_kernel(MoverArgs a)
+{
+    const uint32_t n = mover_count(a);
     const uint32_t per_block = 2u * a.L * a.pieces;
     const unsigned long long total = (unsigned long long)n * per_block;
     for (unsigned long long w = blockIdx.x; w < total; w += gridDim.x) {
-        const uint32_t i = (uint32_t)(w / per_block);
-        const uint32_t r = (uint32_t)(w - (unsigned long long)i * per_block);
-        const uint32_t lp = r / a.pieces, piece = r - lp * a.pieces;
-        uint32_t s = __ldg(a.src_slots + i), d = __ldg(a.dst_slots + i);
-        if (s == CS_ID_NONE || d == CS_ID_NONE) continue;
-        s -= a.src_first;                                   // ids below first_id wrap and fail the range check
-        d -= a.dst_first;
-        if (s >= a.src_total || d >= a.dst_total) {
-            if (threadIdx.x == 0 && r == 0) atomicOr(a.status, CS_ST_BAD_SLOT);
-            continue;
-        }
-        const unsigned long long in_chunk = (unsigned long long)piece * MV_PIECE;
-        const uint4 *sp = (const uint4 *)(a.src + chunk_offset(a.src_layout, a.L, a.src_total, lp >> 1, lp & 1, s, a.chunk) + in_chunk);
-        uint4 *dp = (uint4 *)(a.dst + chunk_offset(a.dst_layout, a.L, a.dst_total, lp >> 1, lp & 1, d, a.chunk) + in_chunk);
-        const unsigned long long left = a.chunk - in_chunk;
-        const uint32_t nvec = (uint32_t)((left < MV_PIECE ? left : MV_PIECE) >> 4);
+        const char *sp0;
+        char *dp0;
+        uint32_t bytes;
+        if (!resolve_piece(a, w, per_block, sp0, dp0, bytes, threadIdx.x == 0)) continue;
+        const uint4 *sp = (const uint4 *)sp0;
+        uint4 *dp = (uint4 *)dp0;
+        const uint32_t nvec = bytes >> 4;
         uint4 v[MV_UNROLL];
 #pragma unroll
         for (int u = 0; u < MV_UNROLL; ++u) {
@@ -69,9 +106,130 @@ __global__ void __launch_bounds__(MV_THREADS) cs_mover_kernel(MoverArgs a)
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// bulk (TMA) path
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait: gives up after TM_SPIN_LIMIT polls (each poll may itself block for a short,
+// hardware-bounded time) and reports failure instead of spinning forever.
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
+{
+    for (uint32_t spin = 0; spin < TM_SPIN_LIMIT; ++spin) {
+        if (mbar_test(bar, parity)) return true;
+        if (spin > 64) __nanosleep(128);
+    }
+    return false;
+}
+__device__ __forceinline__ void bulk_load(uint32_t dst_smem, const void *src, uint32_t bytes, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst_smem),
+                 "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_store(void *dst, uint32_t src_smem, uint32_t bytes)
+{
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src_smem), "r"(bytes)
+                 : "memory");
+}
+
+// One pipeline per warp, driven by lane 0.  Iteration `it` first stores item it-(STAGES-1)
+// (whose load was issued STAGES-1 iterations ago) and then issues the load of item `it` into
+// the ring slot whose previous store has finished reading shared memory.
+__global__ void __launch_bounds__(TM_WARPS * 32, 1) cs_mover_bulk_kernel(MoverArgs a)
+{
+    extern __shared__ __align__(128) unsigned char ring[];
+    __shared__ __align__(8) unsigned long long bars[TM_WARPS * TM_STAGES];
+    const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (lane != 0) return;                                   // the other lanes have nothing to do
+    unsigned char *my_ring = ring + (size_t)warp * TM_STAGES * TM_PIECE;
+    uint32_t bar[TM_STAGES];
+#pragma unroll
+    for (int st = 0; st < TM_STAGES; ++st) {
+        bar[st] = smem_u32(&bars[warp * TM_STAGES + st]);
+        mbar_init(bar[st], 1);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+
+    const uint32_t n = mover_count(a);
+    const uint32_t per_block = 2u * a.L * a.pieces;
+    const unsigned long long total = (unsigned long long)n * per_block;
+    const unsigned long long n_pipes = a.n_pipes;             // pipelines of the whole grid
+    const unsigned long long first = (unsigned long long)blockIdx.x * (blockDim.x >> 5) + warp;
+    if (first >= n_pipes) return;
+    const unsigned long long n_items = first < total ? (total - first + n_pipes - 1) / n_pipes : 0;
+    constexpr int LAG = TM_STAGES - 1;
+
+    char *dst_of[TM_STAGES];          // destination of the item loaded into each ring slot, NULL = skipped item
+    uint32_t bytes_of[TM_STAGES];
+    uint32_t phase_bits = 0;          // parity to wait for, one bit per ring slot
+    uint32_t pending = 0;             // ring slots with a load in flight that nobody has waited for yet
+    bool failed = false;
+    for (unsigned long long it = 0; it < n_items + LAG && !failed; ++it) {
+        if (it >= LAG) {                                      // store item j = it - LAG
+            const int st = (int)((it - LAG) % TM_STAGES);
+            if (pending & (1u << st)) {
+                if (!mbar_wait_bounded(bar[st], (phase_bits >> st) & 1u)) {
+                    failed = true;
+                    atomicOr(a.status, CS_ST_TIMEOUT);
+                    break;
+                }
+                pending &= ~(1u << st);
+                phase_bits ^= 1u << st;
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                bulk_store(dst_of[st], smem_u32(my_ring + (size_t)st * TM_PIECE), bytes_of[st]);
+            }
+            // one group per item, empty for a skipped item, so that group counts match item counts
+            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+        }
+        if (it < n_items) {                                   // load item `it`
+            const int st = (int)(it % TM_STAGES);
+            const char *sp;
+            char *dp;
+            uint32_t bytes;
+            if (resolve_piece(a, first + it * n_pipes, per_block, sp, dp, bytes, true)) {
+                // the slot's previous store (item it-STAGES) was committed one iteration ago, so at
+                // most the newest group may still be reading shared memory
+                asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                dst_of[st] = dp;
+                bytes_of[st] = bytes;
+                pending |= 1u << st;
+                mbar_expect_tx(bar[st], bytes);
+                bulk_load(smem_u32(my_ring + (size_t)st * TM_PIECE), sp, bytes, bar[st]);
+            }
+        }
+    }
+    if (failed) {
+        // give the loads still in flight a bounded chance to land before shared memory is released
+        for (int st = 0; st < TM_STAGES; ++st)
+            if (pending & (1u << st)) mbar_wait_bounded(bar[st], (phase_bits >> st) & 1u);
+    }
+    asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // all stores written
+}
+
+// ---------------------------------------------------------------------------------------------
 int cs_launch_mover(cs_ctx *ctx, const cs_kv_pool *src, const cs_kv_pool *dst, const uint32_t *src_slots,
-                    const uint32_t *dst_slots, uint32_t n_max, const uint32_t *n_dev, int crosses_host_link,
-                    cudaStream_t s)
+                    const uint32_t *dst_slots, uint32_t n_max, const uint32_t *n_dev, int kind, cudaStream_t s)
 {
     MoverArgs a;
     a.src = (const char *)src->base;
@@ -84,16 +242,38 @@ int cs_launch_mover(cs_ctx *ctx, const cs_kv_pool *src, const cs_kv_pool *dst, c
     a.dst_layout = dst->layout;
     a.L = src->n_layers;
     a.chunk = (unsigned long long)src->block_tokens * src->n_kv_heads * src->head_dim * src->elem_bytes;
-    a.pieces = (uint32_t)((a.chunk + MV_PIECE - 1) / MV_PIECE);
     a.src_slots = src_slots;
     a.dst_slots = dst_slots;
     a.n_dev = n_dev;
     a.n_max = n_max;
     a.status = &ctx->ws.sc->status;
+    a.n_pipes = 0;
+    const bool bulk = ctx->mover_path != CS_MOVER_LDST;
+    a.piece_bytes = bulk ? TM_PIECE : MV_PIECE;
+    a.pieces = (uint32_t)((a.chunk + a.piece_bytes - 1) / a.piece_bytes);
     const unsigned long long total = (unsigned long long)n_max * 2ull * a.L * a.pieces;
-    unsigned long long cap = crosses_host_link ? (ctx->host_link_ctas ? ctx->host_link_ctas : 64u)
-                                               : (ctx->d2d_ctas ? ctx->d2d_ctas : 8u * (uint32_t)ctx->sm_count);
-    const uint32_t grid = (uint32_t)(total < cap ? total : cap);
-    cs_mover_kernel<<<grid ? grid : 1u, MV_THREADS, 0, s>>>(a);
+    unsigned long long cap;
+    if (bulk) {
+        // width in warp pipelines (each keeps <= 2 loads and 2 stores of 16 KiB in flight)
+        const uint32_t dflt = kind == CS_MOVE_D2D ? 2u * (uint32_t)ctx->sm_count : (kind == CS_MOVE_OFFLOAD ? 8u : 24u);
+        const uint32_t asked = kind == CS_MOVE_D2D ? ctx->d2d_ctas : ctx->host_link_ctas;
+        cap = asked ? asked : dflt;
+        a.n_pipes = (uint32_t)(total < cap ? total : cap);
+        if (a.n_pipes == 0) a.n_pipes = 1;
+        const uint32_t wpc = a.n_pipes < TM_WARPS ? a.n_pipes : TM_WARPS;
+        const uint32_t grid = (a.n_pipes + wpc - 1) / wpc;
+        if (!ctx->bulk_attr_set) {
+            cudaError_t e = cudaFuncSetAttribute(cs_mover_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TM_SMEM);
+            if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; return CS_ECUDA; }
+            ctx->bulk_attr_set = 1;
+        }
+        cs_mover_bulk_kernel<<<grid, wpc * 32, TM_SMEM, s>>>(a);
+    } else {
+        const uint32_t dflt = kind == CS_MOVE_D2D ? 8u * (uint32_t)ctx->sm_count : (kind == CS_MOVE_OFFLOAD ? 8u : 12u);
+        const uint32_t asked = kind == CS_MOVE_D2D ? ctx->d2d_ctas : ctx->host_link_ctas;
+        cap = asked ? asked : dflt;
+        const uint32_t grid = (uint32_t)(total < cap ? total : cap);
+        cs_mover_kernel<<<grid ? grid : 1u, MV_THREADS, 0, s>>>(a);
+    }
     return cs_check_launch(ctx);
 }

@@ -243,13 +243,18 @@ def pinned_zeros(nbytes):
     return torch.zeros(nbytes, dtype=torch.uint8).pin_memory()
 
 
+PATHS = [cs.CS_MOVER_BULK, cs.CS_MOVER_LDST]
+
+
+@pytest.mark.parametrize("path", PATHS)
 @pytest.mark.parametrize("gpu_layout", [synth.LAYER_MAJOR, synth.BLOCK_MAJOR])
 @pytest.mark.parametrize("host_layout", [synth.BLOCK_MAJOR, synth.LAYER_MAJOR])
-def test_mover_offload_prefetch_compact(gpu_layout, host_layout):
+def test_mover_offload_prefetch_compact(gpu_layout, host_layout, path):
     cfg = synth.CONFIGS["tiny"]
     L, chunk, G, Hs = cfg.n_layers, cfg.chunk_bytes, 96, 160
     rng = synth.rng_for(cfg, 5)
     c, _ = make_ctx(cfg, 64)
+    c.set_mover_path(path)
     gpu_np = synth.kv_pool_u16(G, L, chunk, rng).view(np.uint8)
     gpu = cs.KVPool(dev(gpu_np), G, gpu_layout, L)
     host_t = pinned_zeros(Hs * L * 2 * chunk)
@@ -299,10 +304,12 @@ def test_mover_offload_prefetch_compact(gpu_layout, host_layout):
     assert np.array_equal(host_t.numpy(), before)
 
 
-def test_mover_small_chunks_and_geometry_errors():
+@pytest.mark.parametrize("path", PATHS)
+def test_mover_small_chunks_and_geometry_errors(path):
     """Chunks that are not a whole number of 16 KiB pieces, and a one-block batch."""
     cfg = synth.CONFIGS["tiny"]
     c, _ = make_ctx(cfg, 64)
+    c.set_mover_path(path)
     rng = synth.rng_for(cfg, 6)
     for heads, hd, tok in ((3, 40, 16), (8, 128, 16), (1, 8, 1), (5, 128, 9)):
         chunk = tok * heads * hd * 2
