@@ -232,6 +232,15 @@ int cs_set_mover_ctas(cs_ctx *ctx, uint32_t host_link_ctas, uint32_t d2d_ctas);
 #define CS_MOVER_BULK 2u
 int cs_set_mover_path(cs_ctx *ctx, uint32_t path);
 
+/* Implementation of the two select calls: CS_SELECT_AUTO (= the single-launch cluster kernel up
+ * to 262,144 index entries, the multi-launch path above), CS_SELECT_CLUSTER, CS_SELECT_MULTI
+ * (histogram / collect / bucket / scatter / rank as five grid-wide launches).  Both give the
+ * same lists. */
+#define CS_SELECT_AUTO 0u
+#define CS_SELECT_CLUSTER 1u
+#define CS_SELECT_MULTI 2u
+int cs_set_select_path(cs_ctx *ctx, uint32_t path);
+
 /* cudaError_t of the last failing CUDA call on this context (0 if none). */
 int cs_last_cuda_error(cs_ctx *ctx);
 const char *cs_strerror(int code);

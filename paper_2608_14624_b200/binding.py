@@ -25,12 +25,13 @@ CS_LAYER_MAJOR, CS_BLOCK_MAJOR = 0, 1
 CS_STATIC_MAX_BLOCKS = 65536
 CS_MOVER_AUTO, CS_MOVER_LDST, CS_MOVER_BULK = 0, 1, 2
 CS_ST_TIMEOUT = 16
+CS_SELECT_AUTO, CS_SELECT_CLUSTER, CS_SELECT_MULTI = 0, 1, 2
 
 # every symbol include/cachescout.h declares
 EXPORTS = ("cs_workspace_bytes", "cs_create", "cs_destroy", "cs_observe_invocations", "cs_score_blocks",
            "cs_select_victims", "cs_select_prefetch", "cs_offload_blocks", "cs_prefetch_blocks",
            "cs_compact_blocks", "cs_get_model", "cs_get_status", "cs_launch_count", "cs_set_mover_ctas",
-           "cs_last_cuda_error", "cs_strerror", "cs_version", "cs_select_victims_static", "cs_set_mover_path")
+           "cs_last_cuda_error", "cs_strerror", "cs_version", "cs_select_victims_static", "cs_set_mover_path", "cs_set_select_path")
 
 
 class cs_params(C.Structure):
@@ -89,6 +90,7 @@ def lib():
         L.cs_set_mover_ctas.argtypes = [vp, u32, u32]
         L.cs_last_cuda_error.argtypes = [vp]
         L.cs_set_mover_path.argtypes = [vp, u32]
+        L.cs_set_select_path.argtypes = [vp, u32]
         _lib = L
     return _lib
 
@@ -163,7 +165,7 @@ def cs_select_victims_static(params: cs_params, fsurv, idx: cs_block_index, now:
     memory: the kernels' scratch is a static array inside the library.  `fsurv` is the device
     table of survival factors (one fp32 per agent); at most CS_STATIC_MAX_BLOCKS entries / k."""
     _chk(lib().cs_select_victims_static(C.byref(params), _ptr(fsurv), C.byref(idx), now, tier, k, _ptr(ids_out),
-                                        _ptr(n_out), _stream(stream)), "cs_select_victims_static", "cs_set_mover_path")
+                                        _ptr(n_out), _stream(stream)), "cs_select_victims_static")
 
 
 def cs_offload_blocks(ctx, gpu: cs_kv_pool, host: cs_kv_pool, src_slots, dst_slots, n_max: int, n_dev=None, stream=None):
@@ -207,6 +209,10 @@ def cs_set_mover_ctas(ctx, host_link_ctas: int, d2d_ctas: int):
 
 def cs_set_mover_path(ctx, path: int):
     _chk(lib().cs_set_mover_path(ctx, path), "cs_set_mover_path")
+
+
+def cs_set_select_path(ctx, path: int):
+    _chk(lib().cs_set_select_path(ctx, path), "cs_set_select_path")
 
 
 def cs_version() -> int:
@@ -369,6 +375,9 @@ class CacheScout:
 
     def launch_count(self) -> int:
         return cs_launch_count(self.ctx)
+
+    def set_select_path(self, path: int):
+        cs_set_select_path(self.ctx, path)
 
     def set_mover_path(self, path: int):
         cs_set_mover_path(self.ctx, path)

@@ -55,6 +55,7 @@ size_t cs_layout_workspace(const cs_params *p, uint32_t gtab_len, void *base, cs
     TAKE(P, float, A * A);
     TAKE(amax, uint16_t, A);
     TAKE(rowH, double, A);
+    TAKE(qfix, unsigned long long, A);
     TAKE(adj, uint32_t, A * W);
     TAKE(hops, uint16_t, A);
     TAKE(fsurv, float, A);
@@ -305,6 +306,13 @@ int cs_set_mover_path(cs_ctx *ctx, uint32_t path)
 {
     if (!ctx || path > CS_MOVER_BULK) return CS_EINVAL;
     ctx->mover_path = path;
+    return CS_OK;
+}
+
+int cs_set_select_path(cs_ctx *ctx, uint32_t path)
+{
+    if (!ctx || path > CS_SELECT_MULTI) return CS_EINVAL;
+    ctx->select_path = path;
     return CS_OK;
 }
 

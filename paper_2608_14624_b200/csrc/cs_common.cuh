@@ -9,6 +9,8 @@
 #error "libcachescout is written for sm_100a (B200) only"
 #endif
 
+#define CS_SELECT_CLUSTER_MAX_BLOCKS (1u << 18)   // above this the index is scanned by the whole grid instead
+
 #define CS_MOVE_D2D 0
 #define CS_MOVE_OFFLOAD 1
 #define CS_MOVE_PREFETCH 2
@@ -34,6 +36,8 @@ struct cs_scalars {
     uint32_t sel_b_last;    // last bucket that holds one of the k winners
     uint32_t sel_p_end;     // end position of that bucket
     uint32_t sel_n_out;     // min(k, eligible)
+    uint32_t pad_;
+    unsigned long long t_phase[8];   // globaltimer stamps of the last cluster select (phase boundaries, ns)
 };
 
 // Device pointers into the caller's workspace.
@@ -45,6 +49,7 @@ struct cs_workspace {
     float *P;             // [A*A] Eq. 3
     uint16_t *amax;       // [A]
     double *rowH;         // [A] sum_j P_ij ln P_ij
+    unsigned long long *qfix;   // [A] column sums of Eq. 2 in 2^-60 fixed point, zero between refreshes
     uint32_t *adj;        // [A*W] Eq. 7 adjacency, one bit per edge, W = ceil(A/32)
     uint16_t *hops;       // [A]
     float *fsurv;         // [A] p~ + delta for the cached source
@@ -75,6 +80,8 @@ struct cs_ctx {
     int sm_count;
     uint32_t host_link_ctas, d2d_ctas;
     uint32_t mover_path;   // CS_MOVER_*
+    uint32_t select_path;  // CS_SELECT_*
+    int cluster_max_v, cluster_max_pf;   // largest usable cluster of the single-launch select (0 = not probed, -1 = none)
     int bulk_attr_set;     // shared-memory opt-in of the bulk kernel done on this device
     uint64_t n_launches;
     int last_cuda_error;
@@ -94,6 +101,8 @@ int cs_launch_score(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, const 
                     float *scores_out, cudaStream_t s);
 int cs_launch_select(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, int prefetch, uint32_t tier,
                      uint32_t k, uint32_t *ids_out, uint32_t *n_out, cudaStream_t s);
+int cs_launch_select_cluster(cs_ctx *ctx, const void *sel_args, int prefetch, uint32_t *ids_out, uint32_t *n_out,
+                             cudaStream_t s);
 int cs_launch_mover(cs_ctx *ctx, const cs_kv_pool *src, const cs_kv_pool *dst, const uint32_t *src_slots,
                     const uint32_t *dst_slots, uint32_t n_max, const uint32_t *n_dev, int kind,
                     cudaStream_t s);

@@ -16,7 +16,7 @@ __global__ void cs_init_kernel(cs_workspace ws, uint32_t A, uint32_t n_chains, u
 {
     const uint32_t tid = blockIdx.x * blockDim.x + threadIdx.x, nth = gridDim.x * blockDim.x;
     for (uint32_t i = tid; i < A * A; i += nth) ws.C[i] = 0;
-    for (uint32_t i = tid; i < A; i += nth) ws.rowsum[i] = 0;
+    for (uint32_t i = tid; i < A; i += nth) { ws.rowsum[i] = 0; ws.qfix[i] = 0; }
     for (uint32_t i = tid; i < n_chains; i += nth) ws.cur[i] = CS_AGENT_NONE;
     for (uint32_t i = tid; i < CS_HIST_BINS; i += nth) ws.hist[i] = 0;
     for (uint32_t i = tid; i <= CS_MAX_SPLITTERS; i += nth) ws.bcount[i] = 0;
@@ -89,45 +89,46 @@ cs_observe_kernel(cs_workspace ws, uint32_t A, uint32_t n_chains, const uint32_t
 }
 
 // ---------------------------------------------------------------------------------------------
-// BFS over the bit-matrix graph from a set of source bits, then Eq. 8.  Runs inside one CTA;
-// thread w < W owns word w of the frontier / visited sets.  Level-synchronous: the next
-// frontier is the OR of the adjacency rows of the current one, minus what was visited.
+// BFS over the bit-matrix graph from a set of source bits, then Eq. 8.  Runs inside one CTA.
+// Level-synchronous: every thread owns a few nodes; a node of the current frontier ORs its
+// adjacency row into the next frontier (shared-memory atomics), so one level costs one round
+// trip to the adjacency matrix whatever the frontier size.  Thread w < W then retires word w.
+// s_front / s_visit / s_next: 32 words each.
 // ---------------------------------------------------------------------------------------------
 __device__ void cs_bfs_survival(const uint32_t *__restrict__ adj, uint32_t A, uint32_t W, uint32_t *s_front,
-                                uint32_t *s_visit, uint16_t *hops, float *fsurv, uint32_t e_max, float delta)
+                                uint32_t *s_visit, uint32_t *s_next, uint16_t *hops, float *fsurv, uint32_t e_max,
+                                float delta)
 {
     // on entry s_front[] holds the source bits (already synchronised by the caller)
     const uint32_t tid = threadIdx.x;
     for (uint32_t a = tid; a < A; a += blockDim.x)
         hops[a] = ((s_front[a >> 5] >> (a & 31)) & 1u) ? 0 : CS_HOP_NONE;
-    if (tid < W) s_visit[tid] = s_front[tid];
+    if (tid < W) { s_visit[tid] = s_front[tid]; s_next[tid] = 0; }
     __syncthreads();
     for (uint32_t level = 1; level <= A; ++level) {
-        uint32_t acc = 0;
-        if (tid < W) {
-            for (uint32_t fw = 0; fw < W; ++fw) {
-                uint32_t bits = s_front[fw];
-                while (bits) {
-                    const uint32_t i = fw * 32 + (__ffs(bits) - 1);
-                    bits &= bits - 1;
-                    acc |= __ldcg(&adj[i * W + tid]);
+        for (uint32_t node = tid; node < A; node += blockDim.x) {
+            if ((s_front[node >> 5] >> (node & 31)) & 1u) {
+                for (uint32_t w = 0; w < W; ++w) {
+                    const uint32_t v = __ldcg(&adj[node * W + w]);
+                    if (v) atomicOr(&s_next[w], v);
                 }
             }
-            acc &= ~s_visit[tid];
         }
-        const int any = __syncthreads_or(acc != 0);      // also orders the reads of s_front before its rewrite
-        if (!any) break;
+        __syncthreads();
+        uint32_t acc = 0;
         if (tid < W) {
+            acc = s_next[tid] & ~s_visit[tid];
+            s_next[tid] = 0;
             s_front[tid] = acc;
             s_visit[tid] |= acc;
             uint32_t bits = acc;
             while (bits) {
-                const uint32_t b = tid * 32 + (__ffs(bits) - 1);
+                const uint32_t b2 = tid * 32 + (__ffs(bits) - 1);
                 bits &= bits - 1;
-                if (b < A) hops[b] = (uint16_t)level;
+                if (b2 < A) hops[b2] = (uint16_t)level;
             }
         }
-        __syncthreads();
+        if (!__syncthreads_or(acc != 0)) break;
     }
     __syncthreads();
     for (uint32_t a = tid; a < A; a += blockDim.x) {
@@ -167,12 +168,18 @@ cs_normalise_kernel(cs_workspace ws, uint32_t A, uint32_t W, float eps, float ta
     __shared__ double s_red[ROW_THREADS];
     __shared__ float s_bestv[ROW_THREADS];
     __shared__ uint32_t s_besti[ROW_THREADS];
-    __shared__ uint32_t s_front[32], s_visit[32];
+    __shared__ uint32_t s_front[32], s_visit[32], s_next[32];
     __shared__ bool s_is_last;
     const uint32_t tid = threadIdx.x;
 
+    // Column sums q_j = sum_i pi_i P_ij of Eq. 2 are accumulated by the row CTAs in 2^-60 fixed
+    // point with integer atomics: integer addition commutes, so the sum is bit-identical from run
+    // to run whatever order the CTAs finish in (a float atomic would not be).
+    const uint32_t n_total = ws.sc->n_transitions;
+    const double inv_total = n_total ? 1.0 / (double)n_total : 0.0;
     for (uint32_t i = blockIdx.x; i < A; i += gridDim.x) {
         const uint32_t n_i = ws.rowsum[i];
+        const double pi_fix = (double)n_i * inv_total * 1152921504606846976.0;      // pi_i * 2^60
         const float den = __fadd_rn((float)n_i, __fmul_rn((float)A, eps));
         float bestv = -1.0f;
         uint32_t besti = 0xFFFFFFFFu;
@@ -187,6 +194,7 @@ cs_normalise_kernel(cs_workspace ws, uint32_t A, uint32_t W, float eps, float ta
                 const double pd = (double)p;
                 h += pd * log(pd);
                 edge = p >= tau;
+                if (n_i) atomicAdd(&ws.qfix[j], (unsigned long long)__double2ll_rn(pi_fix * pd));
             }
             const uint32_t bits = __ballot_sync(0xFFFFFFFFu, edge);
             if ((tid & 31) == 0 && (j >> 5) < W) ws.adj[i * W + (j >> 5)] = bits;
@@ -225,14 +233,11 @@ cs_normalise_kernel(cs_workspace ws, uint32_t A, uint32_t W, float eps, float ta
         const double invN = 1.0 / (double)N;
         for (uint32_t i = tid; i < A; i += ROW_THREADS) Hc -= ((double)__ldcg(&ws.rowsum[i]) * invN) * __ldcg(&ws.rowH[i]);
         for (uint32_t j = tid; j < A; j += ROW_THREADS) {
-            double q = 0.0;
-            for (uint32_t i = 0; i < A; ++i) {
-                const uint32_t n_i = __ldcg(&ws.rowsum[i]);
-                if (n_i) q += ((double)n_i * invN) * (double)__ldcg(&ws.P[i * A + j]);
-            }
+            const double q = (double)__ldcg(&ws.qfix[j]) * (1.0 / 1152921504606846976.0);
             if (q > 0.0) Hm -= q * log(q);
         }
     }
+    for (uint32_t j = tid; j < A; j += ROW_THREADS) ws.qfix[j] = 0;      // ready for the next refresh
     Hc = cs_block_sum<double>(Hc, s_red);
     Hm = cs_block_sum<double>(Hm, s_red);
     const uint32_t la = __ldcg(&ws.sc->last_agent);
@@ -246,7 +251,7 @@ cs_normalise_kernel(cs_workspace ws, uint32_t A, uint32_t W, float eps, float ta
     }
     if (tid < 32) s_front[tid] = (la < A && (la >> 5) == tid) ? (1u << (la & 31)) : 0u;
     __syncthreads();
-    cs_bfs_survival(ws.adj, A, W, s_front, s_visit, ws.hops, ws.fsurv, e_max, delta);
+    cs_bfs_survival(ws.adj, A, W, s_front, s_visit, s_next, ws.hops, ws.fsurv, e_max, delta);
 }
 
 // BFS + Eq. 8 from explicit sources into the temporary tables (cs_score_blocks with sources).
@@ -254,7 +259,7 @@ __global__ void __launch_bounds__(ROW_THREADS)
 cs_survival_kernel(cs_workspace ws, uint32_t A, uint32_t W, const uint16_t *__restrict__ sources, uint32_t n_sources,
                    uint32_t e_max, float delta)
 {
-    __shared__ uint32_t s_front[32], s_visit[32];
+    __shared__ uint32_t s_front[32], s_visit[32], s_next[32];
     const uint32_t tid = threadIdx.x;
     if (tid < 32) s_front[tid] = 0;
     __syncthreads();
@@ -264,7 +269,7 @@ cs_survival_kernel(cs_workspace ws, uint32_t A, uint32_t W, const uint16_t *__re
         else atomicOr(&ws.sc->status, CS_ST_BAD_SOURCE);
     }
     __syncthreads();
-    cs_bfs_survival(ws.adj, A, W, s_front, s_visit, ws.hops_tmp, ws.fsurv_tmp, e_max, delta);
+    cs_bfs_survival(ws.adj, A, W, s_front, s_visit, s_next, ws.hops_tmp, ws.fsurv_tmp, e_max, delta);
 }
 
 // ---------------------------------------------------------------------------------------------

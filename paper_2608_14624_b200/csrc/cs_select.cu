@@ -25,171 +25,7 @@
 // not depend on the order in which atomics were served.
 #include "cs_common.cuh"
 
-#define SEL_THREADS 512
-#define GRP 16                    // index entries per thread and iteration (one 128-bit load of bytes)
-
-struct SelArgs {
-    const uint16_t *agent;
-    const uint16_t *depth;
-    const uint8_t *ref;
-    const uint8_t *flags;
-    const uint32_t *la;
-    const uint8_t *ntok;
-    const uint16_t *anchor;
-    const float *fsurv;
-    uint32_t n, now, A, block_tokens, gtab_len, age_sat;
-    float lambda, delta;
-    uint32_t tier, k;
-};
-
-// Per-CTA copies of the small tables every entry looks up.
-struct Tables {
-    float *fsurv;       // [A]
-    float *gtab;        // [gtab_len]
-    uint16_t *anchor;   // [A] or unused
-    float g_sat;
-    uint32_t a_star;
-};
-
-__device__ __forceinline__ void load_tables(const SelArgs &a, const cs_workspace &ws, float *smem, Tables &T,
-                                            bool want_anchor)
-{
-    T.fsurv = smem;
-    T.gtab = smem + a.A;
-    T.anchor = (uint16_t *)(smem + a.A + a.gtab_len);
-    for (uint32_t i = threadIdx.x; i < a.A; i += blockDim.x) T.fsurv[i] = a.fsurv[i];
-    for (uint32_t i = threadIdx.x; i < a.gtab_len; i += blockDim.x) T.gtab[i] = ws.gtab[i];
-    if (want_anchor)
-        for (uint32_t i = threadIdx.x; i < a.A; i += blockDim.x) T.anchor[i] = a.anchor[i];
-    T.g_sat = cs_recency(a.lambda, a.delta, a.age_sat);
-    const uint32_t la = ws.sc->last_agent;
-    T.a_star = (la < a.A) ? ws.amax[la] : 0xFFFFFFFFu;
-}
-
-__device__ __forceinline__ float score_of(const SelArgs &a, const Tables &T, uint32_t agent, uint32_t la,
-                                          uint32_t tok)
-{
-    const uint32_t age = la <= a.now ? a.now - la : 0u;
-    float g;
-    if (age < a.gtab_len) g = T.gtab[age];
-    else if (age >= a.age_sat) g = T.g_sat;
-    else g = cs_recency(a.lambda, a.delta, age);
-    return __fmul_rn(__fmul_rn(T.fsurv[agent], g), (float)tok);      // two roundings, never an FMA
-}
-
-// Eligibility and key of one entry.  PF = prefetch-candidate rules, else eviction-victim rules.
-template <bool PF>
-__device__ __forceinline__ bool entry_key(const SelArgs &a, const Tables &T, uint32_t *status, uint32_t agent,
-                                          uint32_t depth, uint32_t ref, uint32_t flags, uint32_t la, uint32_t tok,
-                                          uint32_t &primary, uint32_t &secondary)
-{
-    if (!(flags & CS_FLAG_VALID) || (flags & CS_FLAG_PINNED) || ref != 0) return false;
-    if (PF) {
-        if (!(flags & CS_FLAG_TIER_HOST) || (flags & CS_FLAG_OTHER_COPY)) return false;
-    } else {
-        if (((flags >> 2) & 1u) != a.tier) return false;
-    }
-    if (agent >= a.A) { atomicOr(status, CS_ST_BAD_AGENT); return false; }
-    if (PF && a.anchor && !(depth < T.anchor[agent])) return false;
-    const uint32_t bits = __float_as_uint(score_of(a, T, agent, la, tok));
-    if (PF) {
-        primary = ((agent == T.a_star) ? 0u : 0x80000000u) | (~bits & 0x7FFFFFFFu);
-        secondary = ~la;
-    } else {
-        primary = bits;
-        secondary = la;
-    }
-    return true;
-}
-
-// One group of 16 consecutive entries in registers.
-struct Group {
-    uint4 ag0, ag1, dp0, dp1, rf, fl, la0, la1, la2, la3, tk;
-};
-
-template <bool PF>
-__device__ __forceinline__ void load_group(const SelArgs &a, uint32_t g, Group &G)
-{
-    G.ag0 = __ldg((const uint4 *)a.agent + 2 * g);
-    G.ag1 = __ldg((const uint4 *)a.agent + 2 * g + 1);
-    G.rf = __ldg((const uint4 *)a.ref + g);
-    G.fl = __ldg((const uint4 *)a.flags + g);
-    G.la0 = __ldg((const uint4 *)a.la + 4 * g);
-    G.la1 = __ldg((const uint4 *)a.la + 4 * g + 1);
-    G.la2 = __ldg((const uint4 *)a.la + 4 * g + 2);
-    G.la3 = __ldg((const uint4 *)a.la + 4 * g + 3);
-    if (a.ntok) G.tk = __ldg((const uint4 *)a.ntok + g);
-    if (PF && a.anchor) {
-        G.dp0 = __ldg((const uint4 *)a.depth + 2 * g);
-        G.dp1 = __ldg((const uint4 *)a.depth + 2 * g + 1);
-    }
-}
-
-__device__ __forceinline__ uint32_t u4_word(const uint4 &v, int w)
-{
-    return w == 0 ? v.x : (w == 1 ? v.y : (w == 2 ? v.z : v.w));
-}
-__device__ __forceinline__ uint32_t grp_u16(const uint4 &lo, const uint4 &hi, int j)   // j in [0,16)
-{
-    const uint32_t w = u4_word(j < 8 ? lo : hi, (j & 7) >> 1);
-    return (w >> ((j & 1) * 16)) & 0xFFFFu;
-}
-__device__ __forceinline__ uint32_t grp_u8(const uint4 &v, int j)
-{
-    return (u4_word(v, j >> 2) >> ((j & 3) * 8)) & 0xFFu;
-}
-__device__ __forceinline__ uint32_t grp_u32(const Group &G, int j)
-{
-    const uint4 &v = j < 4 ? G.la0 : (j < 8 ? G.la1 : (j < 12 ? G.la2 : G.la3));
-    return u4_word(v, j & 3);
-}
-
-// Calls f(id, primary, secondary) for every eligible entry this thread owns: whole groups
-// grid-strided, then the ragged tail (n % 16 entries) one entry per thread.
-template <bool PF, typename F>
-__device__ __forceinline__ void for_each_eligible(const SelArgs &a, const Tables &T, uint32_t *status, F f)
-{
-    const uint32_t gtid = blockIdx.x * blockDim.x + threadIdx.x, nth = gridDim.x * blockDim.x;
-    const uint32_t n_groups = a.n / GRP;
-    for (uint32_t g = gtid; g < n_groups; g += nth) {
-        Group G;
-        load_group<PF>(a, g, G);
-#pragma unroll
-        for (int j = 0; j < GRP; ++j) {
-            uint32_t pr, se;
-            const uint32_t tok = a.ntok ? grp_u8(G.tk, j) : a.block_tokens;
-            const uint32_t dp = (PF && a.anchor) ? grp_u16(G.dp0, G.dp1, j) : 0u;
-            if (entry_key<PF>(a, T, status, grp_u16(G.ag0, G.ag1, j), dp, grp_u8(G.rf, j), grp_u8(G.fl, j),
-                              grp_u32(G, j), tok, pr, se))
-                f(g * GRP + j, pr, se);
-        }
-    }
-    const uint32_t t0 = n_groups * GRP;
-    if (gtid < a.n - t0) {
-        const uint32_t i = t0 + gtid;
-        uint32_t pr, se;
-        const uint32_t tok = a.ntok ? a.ntok[i] : a.block_tokens;
-        if (entry_key<PF>(a, T, status, a.agent[i], a.depth[i], a.ref[i], a.flags[i], a.la[i], tok, pr, se))
-            f(i, pr, se);
-    }
-}
-
-// The prefetch list is empty unless the gate of Eq. 11 is open and a current agent exists.
-__device__ __forceinline__ bool prefetch_enabled(const cs_workspace &ws, uint32_t A)
-{
-    return ws.sc->gate != 0 && ws.sc->last_agent < A;
-}
-
-__device__ __forceinline__ bool last_cta_done(uint32_t *ticket, bool *s_flag)
-{
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) *s_flag = (atomicAdd(ticket, 1u) == gridDim.x - 1);
-    __syncthreads();
-    const bool last = *s_flag;
-    if (last) __threadfence();
-    return last;
-}
+#include "cs_select_common.cuh"
 
 // ---------------------------------------------------------------------------------------------
 // ScoreBlock for every entry (cs_score_blocks).
@@ -299,12 +135,6 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_hist_kernel(SelArgs a, cs_
 // ---------------------------------------------------------------------------------------------
 // 2 collect (+ splitters)
 // ---------------------------------------------------------------------------------------------
-__device__ __forceinline__ bool key_less(unsigned long long km_a, uint32_t id_a, unsigned long long km_b,
-                                         uint32_t id_b)
-{
-    return km_a < km_b || (km_a == km_b && id_a < id_b);
-}
-
 template <bool PF>
 __global__ void __launch_bounds__(SEL_THREADS) cs_sel_collect_kernel(SelArgs a, cs_workspace ws)
 {
@@ -431,20 +261,49 @@ __global__ void __launch_bounds__(256) cs_sel_bucket_kernel(cs_workspace ws)
     __shared__ uint32_t s_id[CS_MAX_SPLITTERS + 1];
     __shared__ uint32_t s_scan[CS_MAX_SPLITTERS + 1];
     __shared__ bool s_flag;
+    __shared__ uint32_t s_cnt[CS_MAX_SPLITTERS + 1], s_base[CS_MAX_SPLITTERS + 1];
+    constexpr int ITEMS = 4;                                  // candidates per thread and reservation round
     const uint32_t c = ws.sc->sel_c, n_spl = ws.sc->sel_n_spl;
     for (uint32_t j = threadIdx.x; j < n_spl; j += blockDim.x) { s_km[j] = ws.spl_km[j]; s_id[j] = ws.spl_id[j]; }
+    s_cnt[threadIdx.x] = 0;
     __syncthreads();
-    for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < c; i += gridDim.x * blockDim.x) {
-        const unsigned long long km = ws.cand_km[i];
-        const uint32_t id = ws.cand_id[i];
-        uint32_t lo = 0, hi = n_spl;                         // bucket = number of splitters <= key
-        while (lo < hi) {
-            const uint32_t mid = (lo + hi) >> 1;
-            if (key_less(km, id, s_km[mid], s_id[mid])) hi = mid;
-            else lo = mid + 1;
+    // Per round a CTA takes 1024 candidates: each finds its bucket and a CTA-local slot (shared-memory
+    // atomics), then one global atomic per non-empty bucket reserves the CTA's range in that bucket.
+    for (uint32_t base = blockIdx.x * (256 * ITEMS); base < c; base += gridDim.x * (256 * ITEMS)) {
+        uint32_t bkt[ITEMS], loc[ITEMS];
+#pragma unroll
+        for (int u = 0; u < ITEMS; ++u) {
+            const uint32_t i = base + u * 256 + threadIdx.x;
+            bkt[u] = 0xFFFFFFFFu;
+            if (i < c) {
+                const unsigned long long km = ws.cand_km[i];
+                const uint32_t id = ws.cand_id[i];
+                uint32_t lo = 0, hi = n_spl;                 // bucket = number of splitters <= key
+                while (lo < hi) {
+                    const uint32_t mid = (lo + hi) >> 1;
+                    if (key_less(km, id, s_km[mid], s_id[mid])) hi = mid;
+                    else lo = mid + 1;
+                }
+                bkt[u] = lo;
+                loc[u] = atomicAdd(&s_cnt[lo], 1u);
+            }
         }
-        ws.cand_bkt[i] = lo;
-        ws.cand_slot[i] = atomicAdd(&ws.bcount[lo], 1u);
+        __syncthreads();
+        {
+            const uint32_t n_b = s_cnt[threadIdx.x];
+            if (n_b) s_base[threadIdx.x] = atomicAdd(&ws.bcount[threadIdx.x], n_b);
+            s_cnt[threadIdx.x] = 0;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int u = 0; u < ITEMS; ++u) {
+            const uint32_t i = base + u * 256 + threadIdx.x;
+            if (bkt[u] != 0xFFFFFFFFu) {
+                ws.cand_bkt[i] = bkt[u];
+                ws.cand_slot[i] = s_base[bkt[u]] + loc[u];
+            }
+        }
+        __syncthreads();
     }
     if (!last_cta_done(&ws.sc->ticket[3], &s_flag)) return;
 
@@ -494,31 +353,58 @@ __global__ void __launch_bounds__(256) cs_sel_scatter_kernel(cs_workspace ws)
 // ---------------------------------------------------------------------------------------------
 // 5 rank and emit
 // ---------------------------------------------------------------------------------------------
+#define RANK_TILE 2048u
+// Each needed bucket is ordered by one CTA: a bitonic sort of the bucket in a shared-memory tile
+// (O(m log^2 m), so an unlucky large bucket costs little more than an average one), after which
+// position i of the bucket is position offset + i of the output list.
 __global__ void __launch_bounds__(256)
 cs_sel_rank_kernel(cs_workspace ws, uint32_t k, uint32_t *__restrict__ ids_out, uint32_t *__restrict__ n_out_dev)
 {
-    __shared__ uint32_t s_off[CS_MAX_SPLITTERS + 2];
-    const uint32_t p_end = ws.sc->sel_p_end, n_out = ws.sc->sel_n_out, n_b = ws.sc->sel_n_spl + 1;
+    __shared__ unsigned long long t_km[RANK_TILE];
+    __shared__ uint32_t t_id[RANK_TILE];
+    const uint32_t p_end = ws.sc->sel_p_end, n_out = ws.sc->sel_n_out, b_last = ws.sc->sel_b_last;
     const uint32_t gtid = blockIdx.x * blockDim.x + threadIdx.x, nth = gridDim.x * blockDim.x;
     for (uint32_t i = n_out + gtid; i < k; i += nth) ids_out[i] = CS_ID_NONE;
     if (gtid == 0) *n_out_dev = n_out;
     if (p_end == 0) return;
-    s_off[threadIdx.x] = ws.boff[threadIdx.x];
-    if (threadIdx.x == 0) s_off[256] = ws.boff[256];
-    __syncthreads();
-    for (uint32_t p = gtid; p < p_end; p += nth) {
-        uint32_t lo = 0, hi = n_b;                            // bucket of position p: last b with off[b] <= p
-        while (hi - lo > 1) {
-            const uint32_t mid = (lo + hi) >> 1;
-            if (s_off[mid] <= p) lo = mid;
-            else hi = mid;
+    for (uint32_t b = blockIdx.x; b <= b_last; b += gridDim.x) {
+        const uint32_t beg = ws.boff[b], end = ws.boff[b + 1], m = end - beg;
+        __syncthreads();
+        if (m <= RANK_TILE) {
+            uint32_t P = 2;
+            while (P < m) P <<= 1;
+            for (uint32_t i = threadIdx.x; i < P; i += blockDim.x) {
+                t_km[i] = i < m ? ws.sort_km[beg + i] : ~0ull;
+                t_id[i] = i < m ? ws.sort_id[beg + i] : 0xFFFFFFFFu;
+            }
+            __syncthreads();
+            for (uint32_t size = 2; size <= P; size <<= 1) {
+                for (uint32_t stride = size >> 1; stride > 0; stride >>= 1) {
+                    for (uint32_t t = threadIdx.x; t < P / 2; t += blockDim.x) {
+                        const uint32_t lo = 2 * t - (t & (stride - 1));
+                        const uint32_t hi = lo + stride;
+                        const bool up = (lo & size) == 0;
+                        const unsigned long long ka = t_km[lo], kb = t_km[hi];
+                        const uint32_t ia = t_id[lo], ib = t_id[hi];
+                        if (key_less(kb, ib, ka, ia) == up) {
+                            t_km[lo] = kb; t_id[lo] = ib;
+                            t_km[hi] = ka; t_id[hi] = ia;
+                        }
+                    }
+                    __syncthreads();
+                }
+            }
+            for (uint32_t i = threadIdx.x; i < m; i += blockDim.x)
+                if (beg + i < n_out) ids_out[beg + i] = t_id[i];
+        } else {                                              // larger than the tile: rank straight from global memory
+            for (uint32_t i = threadIdx.x; i < m; i += blockDim.x) {
+                const unsigned long long km = ws.sort_km[beg + i];
+                const uint32_t id = ws.sort_id[beg + i];
+                uint32_t rank = 0;
+                for (uint32_t q = beg; q < end; ++q) rank += key_less(ws.sort_km[q], ws.sort_id[q], km, id) ? 1u : 0u;
+                if (beg + rank < n_out) ids_out[beg + rank] = id;
+            }
         }
-        const uint32_t beg = s_off[lo], end = s_off[lo + 1];
-        const unsigned long long km = ws.sort_km[p];
-        const uint32_t id = ws.sort_id[p];
-        uint32_t rank = 0;
-        for (uint32_t q = beg; q < end; ++q) rank += key_less(ws.sort_km[q], ws.sort_id[q], km, id) ? 1u : 0u;
-        if (beg + rank < n_out) ids_out[beg + rank] = id;
     }
 }
 
@@ -576,6 +462,10 @@ int cs_launch_select(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, int p
     fill_args(ctx, idx, now, ctx->ws.fsurv, a);
     a.tier = tier;
     a.k = k;
+    if (ctx->select_path != CS_SELECT_MULTI && idx->n_blocks <= CS_SELECT_CLUSTER_MAX_BLOCKS) {
+        const int rc1 = cs_launch_select_cluster(ctx, &a, prefetch, ids_out, n_out, s);
+        if (rc1 != CS_ENOTIMPL) return rc1;          // no usable cluster on this device: fall through
+    }
     const uint32_t grid = scan_grid(ctx, idx->n_blocks, SEL_THREADS * GRP);
     const uint32_t grid_c = scan_grid(ctx, idx->n_blocks, 256);
     const size_t sm = table_smem(ctx);
@@ -590,7 +480,7 @@ int cs_launch_select(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, int p
     if ((rc = cs_check_launch(ctx)) != CS_OK) return rc;
     cs_sel_scatter_kernel<<<grid_c, 256, 0, s>>>(ctx->ws);
     if ((rc = cs_check_launch(ctx)) != CS_OK) return rc;
-    cs_sel_rank_kernel<<<grid_c, 256, 0, s>>>(ctx->ws, k, ids_out, n_out);
+    cs_sel_rank_kernel<<<CS_MAX_SPLITTERS + 1, 256, 0, s>>>(ctx->ws, k, ids_out, n_out);
     return cs_check_launch(ctx);
 }
 

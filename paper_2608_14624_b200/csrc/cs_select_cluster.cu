@@ -1,0 +1,426 @@
+// Single-launch select: the whole top-k (histogram -> threshold -> collect -> order) inside ONE
+// thread-block cluster, for index sizes where a handful of SMs can stream the metadata in a few
+// microseconds (every configuration of this library's workloads).  Compared with the
+// five-launch path (cs_select.cu) it replaces four kernel boundaries by hardware cluster
+// barriers, reduces the per-CTA histograms through distributed shared memory instead of global
+// atomics, loads the small tables once, and occupies at most 16 SMs, which leaves the rest of
+// the GPU to the serving kernels.  Same key, same eligibility rules, same exact ordered output.
+//
+// Phases (cluster.sync() between them; no spin-waits of our own):
+//   1 every CTA scans its slice of the index and builds a 4096-bin histogram of the top 12
+//     primary-key bits in its shared memory;
+//   2 CTA r sums bins [r*B/CL, (r+1)*B/CL) over all CTAs through DSMEM and writes the sums into
+//     every CTA's copy of the total histogram; each CTA then finds the threshold bin b0;
+//   3 every CTA re-scans its slice (L2-resident) and appends the entries with bin <= b0 to the
+//     candidate buffer (c >= min(k, eligible) keys);
+//   4 c <= 4096: CTA 0 sorts the candidates in shared memory (bitonic) and emits the list;
+//     otherwise a sample sort across the cluster: CTA 0 sorts a 1024-key sample and publishes
+//     <= 255 splitters; all CTAs bucket their candidates; offsets by prefix sum; scatter into
+//     bucket order; each needed bucket is sorted in a shared-memory tile.
+#include <cooperative_groups.h>
+
+#include "cs_select_common.cuh"
+
+namespace cg = cooperative_groups;
+
+#define CSEL_THREADS 512
+#define CSEL_SORT_MAX 4096u       // keys one CTA orders in shared memory
+#define CSEL_MAX_CLUSTER 16
+
+struct ClusterSmem {
+    float *tables;
+    uint32_t *hist;                 // [4096] this CTA's histogram
+    uint32_t *tot;                  // [4096] cluster-wide histogram (same in every CTA after phase 2)
+    unsigned long long *km;         // [CSEL_SORT_MAX]
+    uint32_t *id;                   // [CSEL_SORT_MAX]
+    uint32_t *part;                 // [CSEL_THREADS] scan scratch
+    uint32_t *misc;                 // [8]
+};
+
+__host__ __device__ inline size_t csel_table_bytes(uint32_t A, uint32_t gtab_len)
+{
+    return (((size_t)(A + gtab_len) * 4 + (size_t)A * 2) + 15) / 16 * 16;
+}
+static size_t csel_smem_bytes(uint32_t A, uint32_t gtab_len)
+{
+    return csel_table_bytes(A, gtab_len) + 2 * CS_HIST_BINS * 4 + CSEL_SORT_MAX * 12 + CSEL_THREADS * 4 + 64;
+}
+
+__device__ __forceinline__ void csel_carve(unsigned char *base, uint32_t A, uint32_t gtab_len, ClusterSmem &S)
+{
+    S.tables = (float *)base;
+    S.hist = (uint32_t *)(base + csel_table_bytes(A, gtab_len));
+    S.tot = S.hist + CS_HIST_BINS;
+    S.km = (unsigned long long *)(S.tot + CS_HIST_BINS);
+    S.id = (uint32_t *)(S.km + CSEL_SORT_MAX);
+    S.part = S.id + CSEL_SORT_MAX;
+    S.misc = S.part + CSEL_THREADS;
+}
+
+// Exclusive prefix sum of one value per thread over the CTA (CSEL_THREADS threads); also returns the total.
+__device__ __forceinline__ uint32_t csel_block_scan(uint32_t v, uint32_t *s_part, uint32_t &total)
+{
+    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint32_t incl = v;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+        if (lane >= d) incl += t;
+    }
+    __syncthreads();
+    if (lane == 31) s_part[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+        uint32_t w = lane < (CSEL_THREADS / 32) ? s_part[lane] : 0;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, w, d);
+            if (lane >= d) w += t;
+        }
+        s_part[32 + lane] = w;                         // inclusive warp totals
+    }
+    __syncthreads();
+    total = s_part[32 + CSEL_THREADS / 32 - 1];
+    const uint32_t before = warp ? s_part[32 + warp - 1] : 0;
+    return before + incl - v;
+}
+
+// In-place bitonic sort of P (power of two) keys in shared memory, ascending by (km, id).
+__device__ __forceinline__ void csel_bitonic(unsigned long long *km, uint32_t *id, uint32_t P)
+{
+    for (uint32_t size = 2; size <= P; size <<= 1) {
+        for (uint32_t stride = size >> 1; stride > 0; stride >>= 1) {
+            for (uint32_t t = threadIdx.x; t < P / 2; t += blockDim.x) {
+                const uint32_t lo = 2 * t - (t & (stride - 1));
+                const uint32_t hi = lo + stride;
+                const bool up = (lo & size) == 0;
+                const unsigned long long ka = km[lo], kb = km[hi];
+                const uint32_t ia = id[lo], ib = id[hi];
+                if (key_less(kb, ib, ka, ia) == up) {
+                    km[lo] = kb; id[lo] = ib;
+                    km[hi] = ka; id[hi] = ia;
+                }
+            }
+            __syncthreads();
+        }
+    }
+}
+
+__device__ __forceinline__ void csel_stamp(const cs_workspace &ws, uint32_t rank, int slot)
+{
+    if (rank == 0 && threadIdx.x == 0) {
+        unsigned long long t;
+        asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+        ws.sc->t_phase[slot] = t;
+    }
+}
+
+template <bool PF>
+__global__ void __launch_bounds__(CSEL_THREADS, 1)
+cs_select_cluster_kernel(SelArgs a, cs_workspace ws, uint32_t *__restrict__ ids_out, uint32_t *__restrict__ n_out_dev)
+{
+    extern __shared__ __align__(16) unsigned char dsm[];
+    cg::cluster_group cluster = cg::this_cluster();
+    const uint32_t CL = cluster.num_blocks(), rank = cluster.block_rank();
+    const uint32_t tid = threadIdx.x, lane = tid & 31;
+    ClusterSmem S;
+    csel_carve(dsm, a.A, a.gtab_len, S);
+    Tables T;
+    load_tables(a, ws, S.tables, T, PF && a.anchor);
+    for (uint32_t i = tid; i < CS_HIST_BINS; i += CSEL_THREADS) S.hist[i] = 0;
+    if (rank == 0 && tid == 0) ws.sc->sel_c = 0;
+    if (tid == 0) S.misc[1] = 0;
+    __syncthreads();
+    const bool enabled = !PF || prefetch_enabled(ws, a.A);
+    csel_stamp(ws, rank, 0);
+    const uint32_t n_groups = a.n / GRP;
+    const uint32_t cthreads = CL * CSEL_THREADS, ctid = rank * CSEL_THREADS + tid;   // cluster-wide thread id
+    const uint32_t t0 = n_groups * GRP;                                             // start of the ragged tail
+
+    // ---- phase 1: histogram of this CTA's slice ------------------------------------------------
+    if (enabled) {
+        uint32_t run_bin = 0xFFFFFFFFu, run_cnt = 0;          // adjacent entries often share a bin
+        auto add = [&](uint32_t pr) {
+            const uint32_t bin = pr >> 20;
+            if (bin == run_bin) { ++run_cnt; return; }
+            if (run_cnt) atomicAdd(&S.hist[run_bin], run_cnt);
+            run_bin = bin;
+            run_cnt = 1;
+        };
+        for (uint32_t g = ctid; g < n_groups; g += cthreads) {
+            Group G;
+            load_group<PF>(a, g, G);
+#pragma unroll
+            for (int j = 0; j < GRP; ++j) {
+                uint32_t pr, se;
+                const uint32_t tok = a.ntok ? grp_u8(G.tk, j) : a.block_tokens;
+                const uint32_t dp = (PF && a.anchor) ? grp_u16(G.dp0, G.dp1, j) : 0u;
+                if (entry_key<PF>(a, T, &ws.sc->status, grp_u16(G.ag0, G.ag1, j), dp, grp_u8(G.rf, j), grp_u8(G.fl, j),
+                                  grp_u32(G, j), tok, pr, se))
+                    add(pr);
+            }
+        }
+        if (ctid < a.n - t0) {
+            const uint32_t i = t0 + ctid;
+            uint32_t pr, se;
+            const uint32_t tok = a.ntok ? a.ntok[i] : a.block_tokens;
+            if (entry_key<PF>(a, T, &ws.sc->status, a.agent[i], a.depth[i], a.ref[i], a.flags[i], a.la[i], tok, pr, se))
+                add(pr);
+        }
+        if (run_cnt) atomicAdd(&S.hist[run_bin], run_cnt);
+    }
+    __threadfence();
+    cluster.sync();
+    csel_stamp(ws, rank, 1);
+
+    // ---- phase 2: reduce the histograms through DSMEM, broadcast, find the threshold bin ---------------
+    {
+        const uint32_t per = CS_HIST_BINS / CL;                     // CL is a power of two <= 16
+        for (uint32_t b = tid; b < per; b += CSEL_THREADS) {
+            const uint32_t bin = rank * per + b;
+            uint32_t sum = 0;
+            for (uint32_t q = 0; q < CL; ++q) sum += cluster.map_shared_rank(S.hist, q)[bin];
+            for (uint32_t q = 0; q < CL; ++q) cluster.map_shared_rank(S.tot, q)[bin] = sum;
+        }
+    }
+    cluster.sync();
+    constexpr uint32_t PER = CS_HIST_BINS / CSEL_THREADS;
+    uint32_t loc[PER], sum = 0;
+#pragma unroll
+    for (uint32_t q = 0; q < PER; ++q) { loc[q] = S.tot[tid * PER + q]; sum += loc[q]; }
+    uint32_t n_elig;
+    const uint32_t before = csel_block_scan(sum, S.part, n_elig);
+    if (tid == 0) S.misc[0] = (a.k == 0) ? 0xFFFFFFFFu : CS_HIST_BINS - 1;      // k = 0: nothing; k > eligible: everything
+    __syncthreads();
+    if (a.k && n_elig >= a.k && before < a.k && a.k <= before + sum) {
+        uint32_t run = before;
+#pragma unroll
+        for (uint32_t q = 0; q < PER; ++q) {
+            run += loc[q];
+            if (run >= a.k) { S.misc[0] = tid * PER + q; break; }
+        }
+    }
+    __syncthreads();
+    const uint32_t b0 = S.misc[0];
+    const uint32_t n_out = n_elig < a.k ? n_elig : a.k;
+    // the tail of the list is known now: pad it while the candidates are being collected
+    for (uint32_t i = n_out + ctid; i < a.k; i += cthreads) ids_out[i] = CS_ID_NONE;
+    if (ctid == 0) *n_out_dev = n_out;
+
+    csel_stamp(ws, rank, 2);
+    // ---- phase 3: collect the candidates (bin <= b0) ------------------------------------------------------
+    if (enabled && b0 != 0xFFFFFFFFu) {
+        const uint32_t n_iter = (n_groups + cthreads - 1) / cthreads;
+        for (uint32_t it = 0; it < n_iter; ++it) {
+            const uint32_t g = it * cthreads + ctid;
+            uint32_t pr[GRP], mask = 0;
+            Group G;
+            if (g < n_groups) {
+                load_group<PF>(a, g, G);
+#pragma unroll
+                for (int j = 0; j < GRP; ++j) {
+                    uint32_t se;
+                    const uint32_t tok = a.ntok ? grp_u8(G.tk, j) : a.block_tokens;
+                    const uint32_t dp = (PF && a.anchor) ? grp_u16(G.dp0, G.dp1, j) : 0u;
+                    if (entry_key<PF>(a, T, &ws.sc->status, grp_u16(G.ag0, G.ag1, j), dp, grp_u8(G.rf, j),
+                                      grp_u8(G.fl, j), grp_u32(G, j), tok, pr[j], se) &&
+                        (pr[j] >> 20) <= b0)
+                        mask |= 1u << j;
+                }
+            }
+            const uint32_t cnt = __popc(mask);
+            uint32_t incl = cnt;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+                if (lane >= d) incl += v;
+            }
+            uint32_t base = 0;
+            if (lane == 31 && incl) base = atomicAdd(&ws.sc->sel_c, incl);
+            base = __shfl_sync(0xFFFFFFFFu, base, 31);
+            uint32_t pos = base + incl - cnt;
+#pragma unroll
+            for (int j = 0; j < GRP; ++j) {
+                if (mask & (1u << j)) {
+                    const uint32_t la = grp_u32(G, j);
+                    ws.cand_km[pos] = ((unsigned long long)pr[j] << 32) | (PF ? ~la : la);
+                    ws.cand_id[pos] = g * GRP + j;
+                    ++pos;
+                }
+            }
+        }
+        if (ctid < a.n - t0) {
+            const uint32_t i = t0 + ctid;
+            uint32_t p, se;
+            const uint32_t tok = a.ntok ? a.ntok[i] : a.block_tokens;
+            if (entry_key<PF>(a, T, &ws.sc->status, a.agent[i], a.depth[i], a.ref[i], a.flags[i], a.la[i], tok, p, se) &&
+                (p >> 20) <= b0) {
+                const uint32_t pos = atomicAdd(&ws.sc->sel_c, 1u);
+                ws.cand_km[pos] = ((unsigned long long)p << 32) | se;
+                ws.cand_id[pos] = i;
+            }
+        }
+    }
+    __threadfence();
+    cluster.sync();
+    const uint32_t c = __ldcg(&ws.sc->sel_c);
+    csel_stamp(ws, rank, 3);
+
+    // ---- phase 4, small: CTA 0 sorts everything in shared memory ---------------------------------------------
+    if (c <= CSEL_SORT_MAX) {
+        if (rank != 0 || c == 0) return;
+        uint32_t P = 32;
+        while (P < c) P <<= 1;
+        for (uint32_t i = tid; i < P; i += CSEL_THREADS) {
+            S.km[i] = i < c ? __ldcg(&ws.cand_km[i]) : ~0ull;
+            S.id[i] = i < c ? __ldcg(&ws.cand_id[i]) : 0xFFFFFFFFu;
+        }
+        __syncthreads();
+        csel_bitonic(S.km, S.id, P);
+        for (uint32_t i = tid; i < n_out; i += CSEL_THREADS) ids_out[i] = S.id[i];
+        csel_stamp(ws, rank, 4);
+        return;
+    }
+
+    // ---- phase 4, large: sample sort across the cluster ---------------------------------------------------------
+    if (rank == 0) {
+        for (uint32_t i = tid; i < CS_SAMPLE; i += CSEL_THREADS) {
+            const uint32_t pos = (uint32_t)(((unsigned long long)i * c) / CS_SAMPLE);
+            S.km[i] = __ldcg(&ws.cand_km[pos]);
+            S.id[i] = __ldcg(&ws.cand_id[pos]);
+        }
+        __syncthreads();
+        csel_bitonic(S.km, S.id, CS_SAMPLE);
+        for (uint32_t j = tid; j <= CS_MAX_SPLITTERS; j += CSEL_THREADS) {
+            if (j < CS_MAX_SPLITTERS) {
+                const uint32_t q = (uint32_t)(((unsigned long long)(j + 1) * CS_SAMPLE) / (CS_MAX_SPLITTERS + 1));
+                ws.spl_km[j] = S.km[q];
+                ws.spl_id[j] = S.id[q];
+            }
+            ws.bcount[j] = 0;
+        }
+    }
+    __threadfence();
+    cluster.sync();
+    csel_stamp(ws, rank, 4);
+    // bucket: number of splitters <= key; slot by a global counter per bucket
+    unsigned long long *spl_km = S.km;               // shared-memory copy of the splitters
+    uint32_t *spl_id = S.id;
+    __syncthreads();
+    for (uint32_t j = tid; j < CS_MAX_SPLITTERS; j += CSEL_THREADS) { spl_km[j] = __ldcg(&ws.spl_km[j]); spl_id[j] = __ldcg(&ws.spl_id[j]); }
+    __syncthreads();
+    for (uint32_t i = ctid; i < c; i += cthreads) {
+        const unsigned long long km = __ldcg(&ws.cand_km[i]);
+        const uint32_t id = __ldcg(&ws.cand_id[i]);
+        uint32_t lo = 0, hi = CS_MAX_SPLITTERS;
+        while (lo < hi) {
+            const uint32_t mid = (lo + hi) >> 1;
+            if (key_less(km, id, spl_km[mid], spl_id[mid])) hi = mid;
+            else lo = mid + 1;
+        }
+        ws.cand_bkt[i] = lo;
+        ws.cand_slot[i] = atomicAdd(&ws.bcount[lo], 1u);
+    }
+    __threadfence();
+    cluster.sync();
+    csel_stamp(ws, rank, 5);
+    // offsets (every CTA computes the same prefix sum), then scatter the needed buckets into bucket order
+    uint32_t *s_off = S.hist;                        // reuse: [CS_MAX_SPLITTERS + 2]
+    {
+        const uint32_t mine = tid <= CS_MAX_SPLITTERS ? __ldcg(&ws.bcount[tid]) : 0u;
+        uint32_t total;
+        const uint32_t excl = csel_block_scan(mine, S.part, total);
+        if (tid <= CS_MAX_SPLITTERS) s_off[tid] = excl;
+        if (tid == CS_MAX_SPLITTERS) s_off[CS_MAX_SPLITTERS + 1] = excl + mine;
+        if (mine && excl <= n_out - 1 && n_out - 1 < excl + mine) S.misc[1] = tid;     // last needed bucket (n_out > 0 here)
+        __syncthreads();
+    }
+    const uint32_t b_last = S.misc[1];
+    for (uint32_t i = ctid; i < c; i += cthreads) {
+        const uint32_t b = __ldcg(&ws.cand_bkt[i]);
+        if (b > b_last) continue;
+        const uint32_t pos = s_off[b] + __ldcg(&ws.cand_slot[i]);
+        ws.sort_km[pos] = __ldcg(&ws.cand_km[i]);
+        ws.sort_id[pos] = __ldcg(&ws.cand_id[i]);
+    }
+    __threadfence();
+    cluster.sync();
+    csel_stamp(ws, rank, 6);
+    // rank: buckets round-robin over the CTAs; a bucket is ranked from a shared-memory tile
+    for (uint32_t b = rank; b <= b_last; b += CL) {
+        const uint32_t beg = s_off[b], end = s_off[b + 1], m = end - beg;
+        __syncthreads();
+        if (m <= CSEL_SORT_MAX) {
+            uint32_t P = 2;
+            while (P < m) P <<= 1;
+            for (uint32_t i = tid; i < P; i += CSEL_THREADS) {
+                S.km[i] = i < m ? __ldcg(&ws.sort_km[beg + i]) : ~0ull;
+                S.id[i] = i < m ? __ldcg(&ws.sort_id[beg + i]) : 0xFFFFFFFFu;
+            }
+            __syncthreads();
+            csel_bitonic(S.km, S.id, P);
+            for (uint32_t i = tid; i < m; i += CSEL_THREADS)
+                if (beg + i < n_out) ids_out[beg + i] = S.id[i];
+        } else {                                     // a bucket larger than the tile: rank straight from global memory
+            for (uint32_t i = tid; i < m; i += CSEL_THREADS) {
+                const unsigned long long km = __ldcg(&ws.sort_km[beg + i]);
+                const uint32_t id = __ldcg(&ws.sort_id[beg + i]);
+                uint32_t r = 0;
+                for (uint32_t q = beg; q < end; ++q) r += key_less(__ldcg(&ws.sort_km[q]), __ldcg(&ws.sort_id[q]), km, id) ? 1u : 0u;
+                if (beg + r < n_out) ids_out[beg + r] = id;
+            }
+        }
+    }
+    csel_stamp(ws, rank, 7);
+}
+
+// ---------------------------------------------------------------------------------------------
+template <bool PF>
+static int launch_cluster(cs_ctx *ctx, const SelArgs &a, uint32_t *ids_out, uint32_t *n_out, cudaStream_t s)
+{
+    auto kernel = cs_select_cluster_kernel<PF>;
+    const size_t smem = csel_smem_bytes(a.A, a.gtab_len);
+    int &max_cl = PF ? ctx->cluster_max_pf : ctx->cluster_max_v;
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.blockDim = dim3(CSEL_THREADS);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (max_cl == 0) {           // first use on this context: shared-memory opt-in, largest cluster that fits
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+        if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; (void)cudaGetLastError(); max_cl = -1; return CS_ENOTIMPL; }
+        max_cl = -1;
+        for (int cl = CSEL_MAX_CLUSTER; cl >= 1; cl >>= 1) {
+            cfg.gridDim = dim3(cl);
+            attr[0].val.clusterDim.x = cl;
+            int n_clusters = 0;
+            e = cudaOccupancyMaxActiveClusters(&n_clusters, kernel, &cfg);
+            if (e == cudaSuccess && n_clusters >= 1) { max_cl = cl; break; }
+            (void)cudaGetLastError();
+        }
+    }
+    if (max_cl < 1) return CS_ENOTIMPL;
+    // smallest power-of-two cluster that gives every 16-entry group its own thread, at most max_cl
+    const uint32_t n_groups = a.n / GRP;
+    int cl = 1;
+    while (cl < max_cl && (uint32_t)cl * CSEL_THREADS < n_groups) cl <<= 1;
+    cfg.gridDim = dim3(cl);
+    attr[0].val.clusterDim.x = cl;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, a, ctx->ws, ids_out, n_out);
+    ctx->n_launches++;
+    if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; return CS_ECUDA; }
+    return CS_OK;
+}
+
+int cs_launch_select_cluster(cs_ctx *ctx, const void *sel_args, int prefetch, uint32_t *ids_out, uint32_t *n_out,
+                             cudaStream_t s)
+{
+    const SelArgs &a = *(const SelArgs *)sel_args;
+    return prefetch ? launch_cluster<true>(ctx, a, ids_out, n_out, s) : launch_cluster<false>(ctx, a, ids_out, n_out, s);
+}

@@ -1,0 +1,178 @@
+// Device helpers shared by the select kernels: the per-entry eligibility rules and 96-bit key
+// (Algorithm 1, Evict / BetweenStep; Eq. 9), 128-bit loads of the SoA block index, small tables.
+#pragma once
+#include "cs_common.cuh"
+
+#define SEL_THREADS 512
+#define GRP 16                    // index entries per thread and iteration (one 128-bit load of bytes)
+
+struct SelArgs {
+    const uint16_t *agent;
+    const uint16_t *depth;
+    const uint8_t *ref;
+    const uint8_t *flags;
+    const uint32_t *la;
+    const uint8_t *ntok;
+    const uint16_t *anchor;
+    const float *fsurv;
+    uint32_t n, now, A, block_tokens, gtab_len, age_sat;
+    float lambda, delta;
+    uint32_t tier, k;
+};
+
+// Per-CTA copies of the small tables every entry looks up.
+struct Tables {
+    float *fsurv;       // [A]
+    float *gtab;        // [gtab_len]
+    uint16_t *anchor;   // [A] or unused
+    float g_sat;
+    uint32_t a_star;
+};
+
+__device__ __forceinline__ void load_tables(const SelArgs &a, const cs_workspace &ws, float *smem, Tables &T,
+                                            bool want_anchor)
+{
+    T.fsurv = smem;
+    T.gtab = smem + a.A;
+    T.anchor = (uint16_t *)(smem + a.A + a.gtab_len);
+    for (uint32_t i = threadIdx.x; i < a.A; i += blockDim.x) T.fsurv[i] = a.fsurv[i];
+    for (uint32_t i = threadIdx.x; i < a.gtab_len; i += blockDim.x) T.gtab[i] = ws.gtab[i];
+    if (want_anchor)
+        for (uint32_t i = threadIdx.x; i < a.A; i += blockDim.x) T.anchor[i] = a.anchor[i];
+    T.g_sat = cs_recency(a.lambda, a.delta, a.age_sat);
+    const uint32_t la = ws.sc->last_agent;
+    T.a_star = (la < a.A) ? ws.amax[la] : 0xFFFFFFFFu;
+}
+
+__device__ __forceinline__ float score_of(const SelArgs &a, const Tables &T, uint32_t agent, uint32_t la,
+                                          uint32_t tok)
+{
+    const uint32_t age = la <= a.now ? a.now - la : 0u;
+    float g;
+    if (age < a.gtab_len) g = T.gtab[age];
+    else if (age >= a.age_sat) g = T.g_sat;
+    else g = cs_recency(a.lambda, a.delta, age);
+    return __fmul_rn(__fmul_rn(T.fsurv[agent], g), (float)tok);      // two roundings, never an FMA
+}
+
+// Eligibility and key of one entry.  PF = prefetch-candidate rules, else eviction-victim rules.
+template <bool PF>
+__device__ __forceinline__ bool entry_key(const SelArgs &a, const Tables &T, uint32_t *status, uint32_t agent,
+                                          uint32_t depth, uint32_t ref, uint32_t flags, uint32_t la, uint32_t tok,
+                                          uint32_t &primary, uint32_t &secondary)
+{
+    if (!(flags & CS_FLAG_VALID) || (flags & CS_FLAG_PINNED) || ref != 0) return false;
+    if (PF) {
+        if (!(flags & CS_FLAG_TIER_HOST) || (flags & CS_FLAG_OTHER_COPY)) return false;
+    } else {
+        if (((flags >> 2) & 1u) != a.tier) return false;
+    }
+    if (agent >= a.A) { atomicOr(status, CS_ST_BAD_AGENT); return false; }
+    if (PF && a.anchor && !(depth < T.anchor[agent])) return false;
+    const uint32_t bits = __float_as_uint(score_of(a, T, agent, la, tok));
+    if (PF) {
+        primary = ((agent == T.a_star) ? 0u : 0x80000000u) | (~bits & 0x7FFFFFFFu);
+        secondary = ~la;
+    } else {
+        primary = bits;
+        secondary = la;
+    }
+    return true;
+}
+
+// One group of 16 consecutive entries in registers.
+struct Group {
+    uint4 ag0, ag1, dp0, dp1, rf, fl, la0, la1, la2, la3, tk;
+};
+
+template <bool PF>
+__device__ __forceinline__ void load_group(const SelArgs &a, uint32_t g, Group &G)
+{
+    G.ag0 = __ldg((const uint4 *)a.agent + 2 * g);
+    G.ag1 = __ldg((const uint4 *)a.agent + 2 * g + 1);
+    G.rf = __ldg((const uint4 *)a.ref + g);
+    G.fl = __ldg((const uint4 *)a.flags + g);
+    G.la0 = __ldg((const uint4 *)a.la + 4 * g);
+    G.la1 = __ldg((const uint4 *)a.la + 4 * g + 1);
+    G.la2 = __ldg((const uint4 *)a.la + 4 * g + 2);
+    G.la3 = __ldg((const uint4 *)a.la + 4 * g + 3);
+    if (a.ntok) G.tk = __ldg((const uint4 *)a.ntok + g);
+    if (PF && a.anchor) {
+        G.dp0 = __ldg((const uint4 *)a.depth + 2 * g);
+        G.dp1 = __ldg((const uint4 *)a.depth + 2 * g + 1);
+    }
+}
+
+__device__ __forceinline__ uint32_t u4_word(const uint4 &v, int w)
+{
+    return w == 0 ? v.x : (w == 1 ? v.y : (w == 2 ? v.z : v.w));
+}
+__device__ __forceinline__ uint32_t grp_u16(const uint4 &lo, const uint4 &hi, int j)   // j in [0,16)
+{
+    const uint32_t w = u4_word(j < 8 ? lo : hi, (j & 7) >> 1);
+    return (w >> ((j & 1) * 16)) & 0xFFFFu;
+}
+__device__ __forceinline__ uint32_t grp_u8(const uint4 &v, int j)
+{
+    return (u4_word(v, j >> 2) >> ((j & 3) * 8)) & 0xFFu;
+}
+__device__ __forceinline__ uint32_t grp_u32(const Group &G, int j)
+{
+    const uint4 &v = j < 4 ? G.la0 : (j < 8 ? G.la1 : (j < 12 ? G.la2 : G.la3));
+    return u4_word(v, j & 3);
+}
+
+// Calls f(id, primary, secondary) for every eligible entry this thread owns: whole groups
+// grid-strided, then the ragged tail (n % 16 entries) one entry per thread.
+template <bool PF, typename F>
+__device__ __forceinline__ void for_each_eligible(const SelArgs &a, const Tables &T, uint32_t *status, F f)
+{
+    const uint32_t gtid = blockIdx.x * blockDim.x + threadIdx.x, nth = gridDim.x * blockDim.x;
+    const uint32_t n_groups = a.n / GRP;
+    for (uint32_t g = gtid; g < n_groups; g += nth) {
+        Group G;
+        load_group<PF>(a, g, G);
+#pragma unroll
+        for (int j = 0; j < GRP; ++j) {
+            uint32_t pr, se;
+            const uint32_t tok = a.ntok ? grp_u8(G.tk, j) : a.block_tokens;
+            const uint32_t dp = (PF && a.anchor) ? grp_u16(G.dp0, G.dp1, j) : 0u;
+            if (entry_key<PF>(a, T, status, grp_u16(G.ag0, G.ag1, j), dp, grp_u8(G.rf, j), grp_u8(G.fl, j),
+                              grp_u32(G, j), tok, pr, se))
+                f(g * GRP + j, pr, se);
+        }
+    }
+    const uint32_t t0 = n_groups * GRP;
+    if (gtid < a.n - t0) {
+        const uint32_t i = t0 + gtid;
+        uint32_t pr, se;
+        const uint32_t tok = a.ntok ? a.ntok[i] : a.block_tokens;
+        if (entry_key<PF>(a, T, status, a.agent[i], a.depth[i], a.ref[i], a.flags[i], a.la[i], tok, pr, se))
+            f(i, pr, se);
+    }
+}
+
+// The prefetch list is empty unless the gate of Eq. 11 is open and a current agent exists.
+__device__ __forceinline__ bool prefetch_enabled(const cs_workspace &ws, uint32_t A)
+{
+    return ws.sc->gate != 0 && ws.sc->last_agent < A;
+}
+
+__device__ __forceinline__ bool last_cta_done(uint32_t *ticket, bool *s_flag)
+{
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) *s_flag = (atomicAdd(ticket, 1u) == gridDim.x - 1);
+    __syncthreads();
+    const bool last = *s_flag;
+    if (last) __threadfence();
+    return last;
+}
+
+__device__ __forceinline__ bool key_less(unsigned long long km_a, uint32_t id_a, unsigned long long km_b,
+                                         uint32_t id_b)
+{
+    return km_a < km_b || (km_a == km_b && id_a < id_b);
+}
+
+

@@ -134,7 +134,8 @@ def run_selects(c, o, idx, now, ks, tiers=(0, 1)):
     d = cs.DeviceIndex.from_host(idx, DEV)
     s64, s32 = o.scores(idx, now)
     tolerated = 0
-    for k in ks:
+    for path, k in [(p_, k_) for p_ in (cs.CS_SELECT_CLUSTER, cs.CS_SELECT_MULTI) for k_ in ks]:
+        c.set_select_path(path)
         for tier in tiers:
             ids, n_out = c.select_victims(d, now, tier, k)
             ids2, n_out2 = c.select_victims(d, now, tier, k)           # determinism: identical on a second run
