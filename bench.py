@@ -162,6 +162,7 @@ class StepWorkload:
         idx = synth.make_block_index(cfg)
         if self.host_backed < Hs:
             idx.flags[G + self.host_backed:] &= np.uint8(~synth.FLAG_VALID & 0xFF)
+        idx.flags[G - cfg.k_prefetch:G] &= np.uint8(~synth.FLAG_VALID & 0xFF)      # initially free GPU slots
         self.idx_host = idx
         self.N = idx.n
         self.didx = cs.DeviceIndex.from_host(idx, device)
@@ -187,13 +188,9 @@ class StepWorkload:
         self.c = cs.CacheScout(p, device)
         # ring of list buffers: dst[b][:k_v] receives the GPU victims of step s (b = s % RING) and, one
         # step later, serves with the reserve tail as the free GPU slots the prefetch fills
-        reserve = torch.arange(G - (self.k_p - self.k_v), G, dtype=torch.int32, device=device)
-        self.dst = []
-        for _ in range(self.RING):
-            t = torch.empty(self.k_p, dtype=torch.int32, device=device)
-            t[:self.k_v] = torch.arange(0, self.k_v, dtype=torch.int32, device=device)
-            t[self.k_v:] = reserve
-            self.dst.append(t)
+        # (the last k_p GPU slots start out free -- not VALID in the index -- so the first prefetch has a target)
+        free0 = torch.arange(G - self.k_p, G, dtype=torch.int32, device=device)
+        self.dst = [free0.clone() for _ in range(self.RING)]
         mk = lambda n: [torch.zeros(max(n, 4), dtype=torch.int32, device=device) for _ in range(self.RING)]
         self.hv, self.pf = mk(self.k_v), mk(self.k_p)
         self.vn, self.hn, self.pn = mk(1), mk(1), mk(1)
@@ -562,6 +559,22 @@ def profile_case(args, torch, device):
     print(json.dumps({"workload": args.workload, "launches": c.launch_count(), "device_status": c.get_status()}))
 
 
+def reduce_max_ms(local_ms: float, world: int, device) -> float:
+    """Job time = the slowest rank's device time (all-reduce MAX; identity for one rank)."""
+    if world <= 1:
+        return float(local_ms)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([float(local_ms)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_value(world: int, bytes_per_step_per_rank: int, steps: int, job_ms: float) -> float:
+    """Whole-job GB/s of independent replicas: every rank moves the same bytes per step."""
+    return world * bytes_per_step_per_rank * steps / (job_ms / 1e3) / 1e9
+
+
 # ---- main ------------------------------------------------------------------------------------------------------
 def main():
     args = parse_args()
@@ -612,10 +625,7 @@ def main():
     barrier()
     clocks = sampler.stop() if rank == 0 else None
     launches = w.c.launch_count() - l0
-    ms = torch.tensor([e0.elapsed_time(e1)], device=device)
-    if world > 1:
-        dist.all_reduce(ms, op=dist.ReduceOp.MAX)
-    total_ms = float(ms.item())
+    total_ms = reduce_max_ms(e0.elapsed_time(e1), world, device)
     w.collect_timers()
     status = w.c.get_status()
     n_out = [int(w.vn[(args.warmup + args.steps - 1) % w.RING][0].item()),
@@ -625,7 +635,7 @@ def main():
     if args.skip_aux:
         if rank == 0:
             print(json.dumps({"workload": "step", "ms_per_step": total_ms / args.steps, "gpu_launches": int(launches),
-                              "value": world * w.bytes_per_step * args.steps / (total_ms / 1e3) / 1e9, "n_out": n_out}))
+                              "value": job_value(world, w.bytes_per_step, args.steps, total_ms), "n_out": n_out}))
         if world > 1:
             dist.destroy_process_group()
         return
@@ -643,18 +653,15 @@ def main():
     w.drain()
     f1.record(w.main)
     barrier()
-    ms2 = torch.tensor([f0.elapsed_time(f1)], device=device)
-    if world > 1:
-        dist.all_reduce(ms2, op=dist.ReduceOp.MAX)
-    e2e_ms = float(ms2.item())
+    e2e_ms = reduce_max_ms(f0.elapsed_time(f1), world, device)
 
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
 
-    value = world * w.bytes_per_step * args.steps / (total_ms / 1e3) / 1e9
-    e2e_value = world * w.bytes_per_step * args.steps / (e2e_ms / 1e3) / 1e9
+    value = job_value(world, w.bytes_per_step, args.steps, total_ms)
+    e2e_value = job_value(world, w.bytes_per_step, args.steps, e2e_ms)
     bb = w.cfg.block_bytes
     med = lambda k: float(np.median(w.timers[k])) if w.timers[k] else None
     t_c, t_o, t_p, t_s, t_ob = med("compact"), med("offload"), med("prefetch"), med("select"), med("observe")
