@@ -43,7 +43,7 @@ def parse_args():
     ap.add_argument("--offload-width", type=int, default=0, help="warp pipelines of the offload mover (0 = library default)")
     ap.add_argument("--prefetch-width", type=int, default=0, help="warp pipelines of the prefetch mover (0 = library default)")
     ap.add_argument("--quick", action="store_true", help="small pools (debugging only; not a valid bench line)")
-    ap.add_argument("--workload", default="step", choices=["step", "mover", "select"],
+    ap.add_argument("--workload", default="step", choices=["step", "mover", "select", "select80k"],
                     help="'mover'/'select' run one small case of that kernel family only (profiler captures)")
     ap.add_argument("--skip-aux", action="store_true",
                     help="timed steps only: no link-peak probe, end-to-end pass, extras or CPU baseline (profiler launch lists)")
@@ -516,7 +516,9 @@ def profile_case(args, torch, device):
     mover : 2,048-block GPU pool (4 GiB), 512-slot pinned host tier (1 GiB); per step one
             device-to-device move of 512 scattered blocks, one offload and one prefetch of 256.
     select: metadata-scale index (1,000,000 entries, 256 agents); per step observe 64 events,
-            select 10,000 victims and 2,000 prefetch candidates."""
+            select 10,000 victims and 2,000 prefetch candidates (multi-launch select path).
+    select80k: the 80,000-entry index of the Llama-8B configuration, 256 victims / 384 prefetch
+            candidates (single-launch cluster select path)."""
     from paper_2608_14624_b200 import binding as cs
     from paper_2608_14624_b200 import build, synth
     build.build_library()
@@ -539,9 +541,10 @@ def profile_case(args, torch, device):
             c.offload_blocks(gpu, host, d_hs, d_hd)
             c.prefetch_blocks(host, gpu, d_hd, d_hs)
     else:
-        cfg = synth.CONFIGS["meta1m"]
-        N = 1_000_000
-        d = cs.DeviceIndex.from_host(synth.make_block_index(cfg, n=N, tier="random"), device)
+        big = args.workload == "select"
+        cfg = synth.CONFIGS["meta1m" if big else "llama8b"]
+        N = 1_000_000 if big else cfg.n_index
+        d = cs.DeviceIndex.from_host(synth.make_block_index(cfg, n=N, tier="random" if big else "range"), device)
         tr = synth.make_trace(cfg, n_invocations=64 * (args.steps + 40))
         c = cs.CacheScout(cs.make_params(n_agents=cfg.n_agents, n_chains=cfg.n_chains, max_blocks=N,
                                          block_tokens=cfg.block_tokens, r_min=0.02), device)
@@ -690,7 +693,7 @@ def main():
         "blocks_scored_selected_per_s": world * 3 * w.N / (t_s / 1e3),
         "gpu_launches": int(launches),
         "clocks": clocks,
-        "roofline": {"kernel": "cs_mover_kernel (device-to-device compaction of the 256 victims, inside the step)", "bound": "hbm",
+        "roofline": {"kernel": "cs_mover_bulk_kernel (device-to-device compaction of the 256 victims, inside the step, while offload and prefetch run on the side streams)", "bound": "hbm",
                      "achieved": d2d_gbps, "peak": hbm_peak, "unit": "GB/s", "frac": d2d_gbps / hbm_peak, "traffic": traffic,
                      "peak_kind": "of %s" % peak_kind, "algorithmic_bytes_per_launch": 2 * w.k_v * bb, "ms_per_launch": t_c},
         "host_link": {"peak_d2h_GBps": link["d2h"], "peak_h2d_GBps": link["h2d"], "peak_bidir_GBps": link["bidir"],
