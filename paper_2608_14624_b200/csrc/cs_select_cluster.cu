@@ -150,13 +150,14 @@ cs_select_cluster_kernel(SelArgs a, cs_workspace ws, uint32_t *__restrict__ ids_
         for (uint32_t g = ctid; g < n_groups; g += cthreads) {
             Group G;
             load_group<PF>(a, g, G);
+            const uint32_t em = group_elig<PF>(a, G);
 #pragma unroll
             for (int j = 0; j < GRP; ++j) {
+                if (!((em >> j) & 1u)) continue;
                 uint32_t pr, se;
                 const uint32_t tok = a.ntok ? grp_u8(G.tk, j) : a.block_tokens;
                 const uint32_t dp = (PF && a.anchor) ? grp_u16(G.dp0, G.dp1, j) : 0u;
-                if (entry_key<PF>(a, T, &ws.sc->status, grp_u16(G.ag0, G.ag1, j), dp, grp_u8(G.rf, j), grp_u8(G.fl, j),
-                                  grp_u32(G, j), tok, pr, se))
+                if (entry_key_rest<PF>(a, T, &ws.sc->status, grp_u16(G.ag0, G.ag1, j), dp, grp_u32(G, j), tok, pr, se))
                     add(pr);
             }
         }
@@ -213,21 +214,25 @@ cs_select_cluster_kernel(SelArgs a, cs_workspace ws, uint32_t *__restrict__ ids_
         const uint32_t n_iter = (n_groups + cthreads - 1) / cthreads;
         for (uint32_t it = 0; it < n_iter; ++it) {
             const uint32_t g = it * cthreads + ctid;
-            uint32_t pr[GRP], mask = 0;
+            uint32_t mask = 0;               // keys are recomputed for the (few) candidates instead of kept in registers
             Group G;
             if (g < n_groups) {
                 load_group<PF>(a, g, G);
+                const uint32_t em = group_elig<PF>(a, G);
 #pragma unroll
                 for (int j = 0; j < GRP; ++j) {
+                    if (!((em >> j) & 1u)) continue;
                     uint32_t se;
                     const uint32_t tok = a.ntok ? grp_u8(G.tk, j) : a.block_tokens;
                     const uint32_t dp = (PF && a.anchor) ? grp_u16(G.dp0, G.dp1, j) : 0u;
-                    if (entry_key<PF>(a, T, &ws.sc->status, grp_u16(G.ag0, G.ag1, j), dp, grp_u8(G.rf, j),
-                                      grp_u8(G.fl, j), grp_u32(G, j), tok, pr[j], se) &&
-                        (pr[j] >> 20) <= b0)
+                    uint32_t prj;
+                    if (entry_key_rest<PF>(a, T, &ws.sc->status, grp_u16(G.ag0, G.ag1, j), dp, grp_u32(G, j), tok,
+                                           prj, se) &&
+                        (prj >> 20) <= b0)
                         mask |= 1u << j;
                 }
             }
+            if (!__any_sync(0xFFFFFFFFu, mask != 0)) continue;      // most warps hold no candidate at all
             const uint32_t cnt = __popc(mask);
             uint32_t incl = cnt;
 #pragma unroll
@@ -242,8 +247,11 @@ cs_select_cluster_kernel(SelArgs a, cs_workspace ws, uint32_t *__restrict__ ids_
 #pragma unroll
             for (int j = 0; j < GRP; ++j) {
                 if (mask & (1u << j)) {
-                    const uint32_t la = grp_u32(G, j);
-                    ws.cand_km[pos] = ((unsigned long long)pr[j] << 32) | (PF ? ~la : la);
+                    uint32_t prj, se;
+                    const uint32_t tok = a.ntok ? grp_u8(G.tk, j) : a.block_tokens;
+                    const uint32_t dp = (PF && a.anchor) ? grp_u16(G.dp0, G.dp1, j) : 0u;
+                    entry_key_rest<PF>(a, T, &ws.sc->status, grp_u16(G.ag0, G.ag1, j), dp, grp_u32(G, j), tok, prj, se);
+                    ws.cand_km[pos] = ((unsigned long long)prj << 32) | se;
                     ws.cand_id[pos] = g * GRP + j;
                     ++pos;
                 }

@@ -55,18 +55,13 @@ __device__ __forceinline__ float score_of(const SelArgs &a, const Tables &T, uin
     return __fmul_rn(__fmul_rn(T.fsurv[agent], g), (float)tok);      // two roundings, never an FMA
 }
 
-// Eligibility and key of one entry.  PF = prefetch-candidate rules, else eviction-victim rules.
+// Key of an entry already known to pass the flag / ref_count rules: the agent range check, the
+// anchor-depth rule of the prefetch list, and the 96-bit key.
 template <bool PF>
-__device__ __forceinline__ bool entry_key(const SelArgs &a, const Tables &T, uint32_t *status, uint32_t agent,
-                                          uint32_t depth, uint32_t ref, uint32_t flags, uint32_t la, uint32_t tok,
-                                          uint32_t &primary, uint32_t &secondary)
+__device__ __forceinline__ bool entry_key_rest(const SelArgs &a, const Tables &T, uint32_t *status, uint32_t agent,
+                                               uint32_t depth, uint32_t la, uint32_t tok, uint32_t &primary,
+                                               uint32_t &secondary)
 {
-    if (!(flags & CS_FLAG_VALID) || (flags & CS_FLAG_PINNED) || ref != 0) return false;
-    if (PF) {
-        if (!(flags & CS_FLAG_TIER_HOST) || (flags & CS_FLAG_OTHER_COPY)) return false;
-    } else {
-        if (((flags >> 2) & 1u) != a.tier) return false;
-    }
     if (agent >= a.A) { atomicOr(status, CS_ST_BAD_AGENT); return false; }
     if (PF && a.anchor && !(depth < T.anchor[agent])) return false;
     const uint32_t bits = __float_as_uint(score_of(a, T, agent, la, tok));
@@ -80,18 +75,35 @@ __device__ __forceinline__ bool entry_key(const SelArgs &a, const Tables &T, uin
     return true;
 }
 
+// Eligibility and key of one entry.  PF = prefetch-candidate rules, else eviction-victim rules.
+template <bool PF>
+__device__ __forceinline__ bool entry_key(const SelArgs &a, const Tables &T, uint32_t *status, uint32_t agent,
+                                          uint32_t depth, uint32_t ref, uint32_t flags, uint32_t la, uint32_t tok,
+                                          uint32_t &primary, uint32_t &secondary)
+{
+    if (!(flags & CS_FLAG_VALID) || (flags & CS_FLAG_PINNED) || ref != 0) return false;
+    if (PF) {
+        if (!(flags & CS_FLAG_TIER_HOST) || (flags & CS_FLAG_OTHER_COPY)) return false;
+    } else {
+        if (((flags >> 2) & 1u) != a.tier) return false;
+    }
+    return entry_key_rest<PF>(a, T, status, agent, depth, la, tok, primary, secondary);
+}
+
 // One group of 16 consecutive entries in registers.
 struct Group {
     uint4 ag0, ag1, dp0, dp1, rf, fl, la0, la1, la2, la3, tk;
 };
 
-template <bool PF>
+template <bool PF, bool FLAGS = true>
 __device__ __forceinline__ void load_group(const SelArgs &a, uint32_t g, Group &G)
 {
     G.ag0 = __ldg((const uint4 *)a.agent + 2 * g);
     G.ag1 = __ldg((const uint4 *)a.agent + 2 * g + 1);
-    G.rf = __ldg((const uint4 *)a.ref + g);
-    G.fl = __ldg((const uint4 *)a.flags + g);
+    if (FLAGS) {
+        G.rf = __ldg((const uint4 *)a.ref + g);
+        G.fl = __ldg((const uint4 *)a.flags + g);
+    }
     G.la0 = __ldg((const uint4 *)a.la + 4 * g);
     G.la1 = __ldg((const uint4 *)a.la + 4 * g + 1);
     G.la2 = __ldg((const uint4 *)a.la + 4 * g + 2);
@@ -122,6 +134,24 @@ __device__ __forceinline__ uint32_t grp_u32(const Group &G, int j)
     return u4_word(v, j & 3);
 }
 
+// Flag / ref_count rules for the 16 entries of a group at once, four entries per 32-bit word
+// (byte-wise SIMD compares): bit j of the result is set when entry j is VALID, not PINNED, on the
+// requested tier (prefetch: on the host tier without a GPU copy) and unreferenced.
+template <bool PF>
+__device__ __forceinline__ uint32_t group_elig(const SelArgs &a, const Group &G)
+{
+    const uint32_t fmask = PF ? 0x0F0F0F0Fu : 0x07070707u;
+    const uint32_t fpat = PF ? 0x05050505u : (0x01010101u * (CS_FLAG_VALID | (a.tier << 2)));
+    uint32_t out = 0;
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {
+        const uint32_t ok = __vcmpeq4(u4_word(G.fl, w) & fmask, fpat) & __vcmpeq4(u4_word(G.rf, w), 0u);
+        const uint32_t t = (ok >> 7) & 0x01010101u;                    // one bit per byte
+        out |= (((t * 0x01020408u) >> 24) & 0xFu) << (4 * w);           // gather bytes' bits into a nibble
+    }
+    return out;
+}
+
 // Calls f(id, primary, secondary) for every eligible entry this thread owns: whole groups
 // grid-strided, then the ragged tail (n % 16 entries) one entry per thread.
 template <bool PF, typename F>
@@ -132,13 +162,14 @@ __device__ __forceinline__ void for_each_eligible(const SelArgs &a, const Tables
     for (uint32_t g = gtid; g < n_groups; g += nth) {
         Group G;
         load_group<PF>(a, g, G);
+        const uint32_t em = group_elig<PF>(a, G);
 #pragma unroll
         for (int j = 0; j < GRP; ++j) {
+            if (!((em >> j) & 1u)) continue;
             uint32_t pr, se;
             const uint32_t tok = a.ntok ? grp_u8(G.tk, j) : a.block_tokens;
             const uint32_t dp = (PF && a.anchor) ? grp_u16(G.dp0, G.dp1, j) : 0u;
-            if (entry_key<PF>(a, T, status, grp_u16(G.ag0, G.ag1, j), dp, grp_u8(G.rf, j), grp_u8(G.fl, j),
-                              grp_u32(G, j), tok, pr, se))
+            if (entry_key_rest<PF>(a, T, status, grp_u16(G.ag0, G.ag1, j), dp, grp_u32(G, j), tok, pr, se))
                 f(g * GRP + j, pr, se);
         }
     }
