@@ -305,3 +305,38 @@ uint32_t orc_move_blocks(const uint8_t *src, uint32_t src_layout, uint32_t src_s
     }
     return bad;
 }
+
+/* ------------------------------------------------------------------------------------
+ * Eq. 6: exact survival probability p_surv(a; a0, K) = Pr(exists k in [1, K]: A_{t+k} = a |
+ * A_t = a0) under the first-order chain with matrix P.  Written out from the definition: make
+ * a absorbing-and-removed (zero column a: mass that reaches a leaves the vector), push the unit
+ * mass at a0 through K steps, and what is left never visited a:
+ *     v_0 = e_{a0};  v_{t+1}[j] = sum_i v_t[i] P[i][j]  (j != a),  v_{t+1}[a] = 0;
+ *     p_surv(a) = 1 - sum_j v_K[j].
+ * The paper calls this prohibitively expensive for its runtime and approximates it with the
+ * hop-distance proxy of Eq. 8; here it is the alternative scorer.  a0 >= A gives all zeros.
+ * ------------------------------------------------------------------------------------ */
+void orc_exact_survival(uint32_t A, const double *P64, uint32_t a0, uint32_t K, double *psurv /*[A]*/)
+{
+    double *v = (double *)malloc((size_t)A * sizeof(double));
+    double *w = (double *)malloc((size_t)A * sizeof(double));
+    for (uint32_t a = 0; a < A; ++a) {
+        if (a0 >= A) { psurv[a] = 0.0; continue; }
+        for (uint32_t j = 0; j < A; ++j) v[j] = 0.0;
+        v[a0] = 1.0;
+        for (uint32_t t = 0; t < K; ++t) {
+            for (uint32_t j = 0; j < A; ++j) {
+                double s = 0.0;
+                if (j != a)
+                    for (uint32_t i = 0; i < A; ++i) s += v[i] * P64[(size_t)i * A + j];
+                w[j] = s;
+            }
+            double *tmp = v; v = w; w = tmp;
+        }
+        double left = 0.0;
+        for (uint32_t j = 0; j < A; ++j) left += v[j];
+        psurv[a] = 1.0 - left;
+    }
+    free(v);
+    free(w);
+}

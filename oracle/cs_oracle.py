@@ -120,6 +120,14 @@ class Oracle:
         L.orc_survival(C.c_uint32(A), _p(self.E), C.c_uint32(self.p.e_max),
                        C.c_float(self.p.delta), _p(self.ptilde), _p(self.fsurv32))
 
+    def exact_survival(self, K: int, a0: Optional[int] = None) -> np.ndarray:
+        """Eq. 6 for every agent, from the current agent (or `a0`) over K steps; fp64."""
+        A = self.p.n_agents
+        a0 = int(self.last_agent[0]) if a0 is None else int(a0)
+        out = np.zeros(A, np.float64)
+        lib().orc_exact_survival(C.c_uint32(A), _p(self.P64), C.c_uint32(a0), C.c_uint32(K), _p(out))
+        return out
+
     @property
     def gate(self) -> bool:
         """Eq. 11, decided on the fp32 value of R like the kernels do."""

@@ -438,3 +438,46 @@ def test_offload_then_prefetch_roundtrip_is_bytewise_identity():
         assert np.array_equal(v(back)[g_ids], v(gpu)[g_ids])
     bad = orc.move_blocks(gpu, 0, G, host, 1, H, L, chunk, np.array([G], np.uint32), np.array([0], np.uint32))
     assert bad == 1
+
+
+# ---- Eq. 6: exact survival probability --------------------------------------------------------------
+def brute_survival(Pm, a0, K):
+    """Enumerate every path of K steps from a0 and add up the probability of those that visit a."""
+    A = Pm.shape[0]
+    out = np.zeros(A)
+    for path in itertools.product(range(A), repeat=K):
+        pr, cur = 1.0, a0
+        for nxt in path:
+            pr *= Pm[cur, nxt]
+            cur = nxt
+        for a in set(path):
+            out[a] += pr
+    return out
+
+
+@pytest.mark.parametrize("seed", range(4))
+def test_exact_survival_vs_path_enumeration(seed):
+    rng = np.random.default_rng(40 + seed)
+    A, K = 4, 4
+    o = orc.Oracle(P(n_agents=A))
+    o.C[:] = rng.integers(0, 9, (A, A))
+    np.fill_diagonal(o.C, 0)
+    o.refresh()
+    for a0 in range(A):
+        got = o.exact_survival(K, a0)
+        assert np.allclose(got, brute_survival(o.P64, a0, K), rtol=1e-12, atol=1e-15)
+        assert np.allclose(o.exact_survival(1, a0), o.P64[a0], rtol=1e-13)         # one step: the row itself
+        assert np.all(np.diff([o.exact_survival(k, a0) for k in range(0, 6)], axis=0) >= -1e-15)   # grows with K
+    assert np.all(o.exact_survival(0, 0) == 0.0)
+    assert np.all(o.exact_survival(3, orc.AGENT_NONE) == 0.0)                      # no current agent yet
+
+
+def test_exact_survival_on_a_deterministic_cycle():
+    """Pipeline topology: agent at distance d is reached within K steps iff d <= K (Sec. 2.2)."""
+    o = run_trace(list(range(5)) * 30, 5, eps=1e-9)
+    for K in (1, 2, 4, 5):
+        got = o.exact_survival(K)                       # current agent is 4; distances: 0->1, 1->2, ... 4->5
+        want = np.array([1.0 if ((a - 4) % 5 or 5) <= K else 0.0 for a in range(5)])
+        assert np.allclose(got, want, atol=1e-6)
+    # the hop-distance proxy of Eq. 8 orders the agents the same way on this chain
+    assert np.array_equal(np.argsort(-o.exact_survival(3), kind="stable")[:3], np.argsort(o.E, kind="stable")[1:4])
