@@ -445,6 +445,33 @@ def metadata_scale(torch, cs, synth, dev, hbm_peak, calls=200):
             "kernel_launches_per_call": launches, "n_out": [int(vn[0].item()), int(pn[0].item())]}
 
 
+def exact_survival_section(torch, cs, synth, dev):
+    """Eq. 6 as an alternative scorer: time of one table (CUDA events) and how far the victim list it
+    gives is from the list of the hop-distance proxy of Eq. 8 (context for the approximation)."""
+    rows = []
+    for name, n_idx, k, K in (("llama8b", 80_000, 256, 4), ("llama70b", 52_000, 256, 4), ("meta1m", 1_000_000, 10_000, 4)):
+        cfg = synth.CONFIGS[name]
+        tr = synth.make_trace(cfg, n_invocations=6000)
+        c = cs.CacheScout(cs.make_params(n_agents=cfg.n_agents, n_chains=cfg.n_chains, max_blocks=n_idx,
+                                         block_tokens=cfg.block_tokens, r_min=0.02), dev)
+        c.observe_invocations(torch.from_numpy(tr.chain).to(dev), torch.from_numpy(tr.agent).to(dev), None)
+        stream = torch.cuda.current_stream(dev)
+        A = cfg.n_agents
+        ps = torch.empty(A, dtype=torch.float32, device=dev)
+        fs = torch.empty(A, dtype=torch.float32, device=dev)
+        med, best = time_call(torch, stream, lambda: cs.cs_exact_survival(c.ctx, cs.CS_AGENT_NONE, K, ps, fs), 20, warm=3)
+        d = cs.DeviceIndex.from_host(synth.make_block_index(cfg, n=n_idx, tier="random" if name == "meta1m" else "range"), dev)
+        v_proxy, _ = c.select_victims(d, 100_000, 0, k)
+        c.use_survival_table(fs)
+        v_exact, _ = c.select_victims(d, 100_000, 0, k)
+        c.use_survival_table(None)
+        common = len(set(v_proxy[:k].tolist()) & set(v_exact[:k].tolist()))
+        rows.append({"config": name, "agents": A, "steps_K": K, "us_per_table_median": med * 1e3, "us_min": best * 1e3,
+                     "fp64_GFLOPs": 2.0 * A ** 3 * K / (med / 1e3) / 1e9,
+                     "victims_shared_with_hop_proxy": common / k})
+    return rows
+
+
 # ---- the oracle on the host cores (cpu_baseline and --impl reference) ----------------------------------------
 class OracleStep:
     """The same scheduler step computed by the CPU oracle.  Bounded sample: the selections run over
@@ -714,6 +741,7 @@ def main():
         del w
         torch.cuda.empty_cache()
         out["metadata_scale"] = metadata_scale(torch, cs, synth, device, hbm_peak)
+        out["exact_survival"] = exact_survival_section(torch, cs, synth, device)
     # the oracle, as it stands, on this machine's host cores
     ow = OracleStep()
     ow.step(0)

@@ -232,6 +232,22 @@ int cs_set_mover_ctas(cs_ctx *ctx, uint32_t host_link_ctas, uint32_t d2d_ctas);
 #define CS_MOVER_BULK 2u
 int cs_set_mover_path(cs_ctx *ctx, uint32_t path);
 
+/* ---- exact survival probability (the quantity Eq. 8 approximates) ---------------------------------- */
+
+/* Eq. 6 for every agent a: p_surv(a; a0, K) = Pr(a is invoked within the next K dispatches | the
+ * current agent is a0), computed exactly from the matrix of Eq. 3 by pushing the unit mass at a0
+ * through K steps of the chain with state a removed.  a0 = CS_AGENT_NONE uses the current agent
+ * (agent of the last observed event; all zeros while there is none).  n_steps = K <= 4096.
+ * psurv_out: dev [n_agents] p_surv; fsurv_out: dev [n_agents] p_surv + delta, the first factor of
+ * Eq. 9 (either may be NULL).  fp64 accumulation, fp32 results.  Cost n_agents^3 * K multiply-adds. */
+int cs_exact_survival(cs_ctx *ctx, uint32_t a0, uint32_t n_steps, float *psurv_out, float *fsurv_out,
+                      cs_stream_t stream);
+
+/* Makes cs_score_blocks (without explicit sources), cs_select_victims and cs_select_prefetch use
+ * the caller's survival table (dev [n_agents], e.g. fsurv_out above, which must stay alive) in place
+ * of the hop-distance table of Eq. 8; NULL restores the default.  Host-side switch, no launch. */
+int cs_use_survival_table(cs_ctx *ctx, const float *fsurv);
+
 /* Implementation of the two select calls: CS_SELECT_AUTO (= the single-launch cluster kernel up
  * to 262,144 index entries, the multi-launch path above), CS_SELECT_CLUSTER, CS_SELECT_MULTI
  * (histogram / collect / bucket / scatter / rank as five grid-wide launches).  Both give the

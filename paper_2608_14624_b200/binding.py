@@ -31,7 +31,8 @@ CS_SELECT_AUTO, CS_SELECT_CLUSTER, CS_SELECT_MULTI = 0, 1, 2
 EXPORTS = ("cs_workspace_bytes", "cs_create", "cs_destroy", "cs_observe_invocations", "cs_score_blocks",
            "cs_select_victims", "cs_select_prefetch", "cs_offload_blocks", "cs_prefetch_blocks",
            "cs_compact_blocks", "cs_get_model", "cs_get_status", "cs_launch_count", "cs_set_mover_ctas",
-           "cs_last_cuda_error", "cs_strerror", "cs_version", "cs_select_victims_static", "cs_set_mover_path", "cs_set_select_path")
+           "cs_last_cuda_error", "cs_strerror", "cs_version", "cs_select_victims_static", "cs_set_mover_path", "cs_set_select_path",
+           "cs_exact_survival", "cs_use_survival_table")
 
 
 class cs_params(C.Structure):
@@ -91,6 +92,8 @@ def lib():
         L.cs_last_cuda_error.argtypes = [vp]
         L.cs_set_mover_path.argtypes = [vp, u32]
         L.cs_set_select_path.argtypes = [vp, u32]
+        L.cs_exact_survival.argtypes = [vp, u32, u32, vp, vp, vp]
+        L.cs_use_survival_table.argtypes = [vp, vp]
         _lib = L
     return _lib
 
@@ -209,6 +212,15 @@ def cs_set_mover_ctas(ctx, host_link_ctas: int, d2d_ctas: int):
 
 def cs_set_mover_path(ctx, path: int):
     _chk(lib().cs_set_mover_path(ctx, path), "cs_set_mover_path")
+
+
+def cs_exact_survival(ctx, a0: int, n_steps: int, psurv_out, fsurv_out, stream=None):
+    _chk(lib().cs_exact_survival(ctx, a0, n_steps, _ptr(psurv_out), _ptr(fsurv_out), _stream(stream)),
+         "cs_exact_survival", ctx)
+
+
+def cs_use_survival_table(ctx, fsurv):
+    _chk(lib().cs_use_survival_table(ctx, _ptr(fsurv)), "cs_use_survival_table", ctx)
 
 
 def cs_set_select_path(ctx, path: int):
@@ -375,6 +387,19 @@ class CacheScout:
 
     def launch_count(self) -> int:
         return cs_launch_count(self.ctx)
+
+    def exact_survival(self, n_steps: int, a0: int = CS_AGENT_NONE, stream=None):
+        """Eq. 6 for every agent: returns (p_surv, p_surv + delta) as device tensors."""
+        import torch
+        A = self.params.n_agents
+        ps = torch.empty(A, dtype=torch.float32, device=self.device)
+        fs = torch.empty(A, dtype=torch.float32, device=self.device)
+        cs_exact_survival(self.ctx, a0, n_steps, ps, fs, stream)
+        return ps, fs
+
+    def use_survival_table(self, fsurv):
+        self._fsurv_keepalive = fsurv
+        cs_use_survival_table(self.ctx, fsurv)
 
     def set_select_path(self, path: int):
         cs_set_select_path(self.ctx, path)

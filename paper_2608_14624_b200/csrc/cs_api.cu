@@ -171,7 +171,7 @@ int cs_score_blocks(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, const 
     if (rc != CS_OK) return rc;
     if (idx->n_blocks && (!scores_out || !aligned16(scores_out))) return CS_EINVAL;
     if (sources && !aligned16(sources)) return CS_EINVAL;
-    const float *fsurv = ctx->ws.fsurv;
+    const float *fsurv = ctx->fsurv_override ? ctx->fsurv_override : ctx->ws.fsurv;
     if (sources) {
         rc = cs_launch_survival(ctx, sources, n_sources, (cudaStream_t)stream);
         if (rc != CS_OK) return rc;
@@ -306,6 +306,23 @@ int cs_set_mover_path(cs_ctx *ctx, uint32_t path)
 {
     if (!ctx || path > CS_MOVER_BULK) return CS_EINVAL;
     ctx->mover_path = path;
+    return CS_OK;
+}
+
+int cs_exact_survival(cs_ctx *ctx, uint32_t a0, uint32_t n_steps, float *psurv_out, float *fsurv_out, cs_stream_t stream)
+{
+    if (!ctx) return CS_EINVAL;
+    if (a0 != CS_AGENT_NONE && a0 >= ctx->p.n_agents) return CS_EINVAL;
+    if (n_steps > 4096) return CS_EINVAL;
+    if ((((uintptr_t)psurv_out) & 3u) || (((uintptr_t)fsurv_out) & 3u)) return CS_EINVAL;
+    if (!psurv_out && !fsurv_out) return CS_OK;
+    return cs_launch_exact_survival(ctx, a0, n_steps, psurv_out, fsurv_out, (cudaStream_t)stream);
+}
+
+int cs_use_survival_table(cs_ctx *ctx, const float *fsurv)
+{
+    if (!ctx || (((uintptr_t)fsurv) & 3u)) return CS_EINVAL;
+    ctx->fsurv_override = fsurv;
     return CS_OK;
 }
 

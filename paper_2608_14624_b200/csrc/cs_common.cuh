@@ -81,6 +81,7 @@ struct cs_ctx {
     uint32_t host_link_ctas, d2d_ctas;
     uint32_t mover_path;   // CS_MOVER_*
     uint32_t select_path;  // CS_SELECT_*
+    const float *fsurv_override;   // caller's survival table for score / select, NULL = the BFS table of Eq. 8
     int cluster_max_v, cluster_max_pf;   // largest usable cluster of the single-launch select (0 = not probed, -1 = none)
     int bulk_attr_set;     // shared-memory opt-in of the bulk kernel done on this device
     uint64_t n_launches;
@@ -97,6 +98,7 @@ int cs_launch_init(cs_ctx *ctx, cudaStream_t s);
 int cs_launch_observe(cs_ctx *ctx, const uint32_t *chain, const uint16_t *agent, const uint8_t *evflags,
                       uint32_t n_events, cudaStream_t s);
 int cs_launch_survival(cs_ctx *ctx, const uint16_t *sources, uint32_t n_sources, cudaStream_t s);
+int cs_launch_exact_survival(cs_ctx *ctx, uint32_t a0, uint32_t K, float *psurv_out, float *fsurv_out, cudaStream_t s);
 int cs_launch_score(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, const float *fsurv,
                     float *scores_out, cudaStream_t s);
 int cs_launch_select(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, int prefetch, uint32_t tier,

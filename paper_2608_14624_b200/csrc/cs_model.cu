@@ -273,6 +273,63 @@ cs_survival_kernel(cs_workspace ws, uint32_t A, uint32_t W, const uint16_t *__re
 }
 
 // ---------------------------------------------------------------------------------------------
+// Exact survival probability of Eq. 6 for every agent: one CTA per target agent a.  The unit
+// mass at the current agent a0 is pushed through K steps of the chain with column a removed
+// (mass that reaches a leaves the vector); what is left after K steps never visited a:
+//     v_0 = e_{a0};  v_{t+1}[j] = sum_i v_t[i] P[i][j] (j != a), v_{t+1}[a] = 0;
+//     p = sum_t sum_i v_t[i] P[i][a]  (= 1 - sum_j v_K[j]).
+// fp64 accumulation over the canonical fp32 matrix, terms added in index order.  The paper
+// treats this as too expensive for its per-request runtime and uses the hop proxy of Eq. 8;
+// here it is an alternative scorer (A^3 K multiply-adds, off the critical path).
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(ROW_THREADS)
+cs_exact_survival_kernel(cs_workspace ws, uint32_t A, uint32_t a0_arg, uint32_t K, float delta,
+                         float *__restrict__ psurv_out, float *__restrict__ fsurv_out)
+{
+    extern __shared__ double s_vec[];                 // v[A], w[A]
+    double *v = s_vec, *w = s_vec + A;
+    const uint32_t tid = threadIdx.x;
+    const uint32_t a0 = a0_arg == CS_AGENT_NONE ? ws.sc->last_agent : a0_arg;
+    for (uint32_t a = blockIdx.x; a < A; a += gridDim.x) {
+        // The probability is accumulated as the mass absorbed at a step by step (no 1 - x
+        // cancellation, so small probabilities keep full relative accuracy); the thread that owns
+        // column a does the adding.
+        double hit = 0.0;
+        if (a0 < A) {
+            __syncthreads();
+            for (uint32_t j = tid; j < A; j += ROW_THREADS) v[j] = (j == a0) ? 1.0 : 0.0;
+            __syncthreads();
+            for (uint32_t t = 0; t < K; ++t) {
+                for (uint32_t j = tid; j < A; j += ROW_THREADS) {
+                    double s = 0.0;
+                    for (uint32_t i = 0; i < A; ++i) {
+                        const double vi = v[i];
+                        if (vi != 0.0) s = __dadd_rn(s, __dmul_rn(vi, (double)ws.P[i * A + j]));
+                    }
+                    if (j == a) { hit += s; s = 0.0; }
+                    w[j] = s;
+                }
+                __syncthreads();
+                double *tmp = v; v = w; w = tmp;
+            }
+        }
+        if (tid == (a % ROW_THREADS)) {
+            if (psurv_out) psurv_out[a] = (float)hit;
+            if (fsurv_out) fsurv_out[a] = (float)(hit + (double)delta);
+        }
+    }
+}
+
+int cs_launch_exact_survival(cs_ctx *ctx, uint32_t a0, uint32_t K, float *psurv_out, float *fsurv_out, cudaStream_t s)
+{
+    const cs_params &p = ctx->p;
+    const uint32_t grid = p.n_agents < 4u * (uint32_t)ctx->sm_count ? p.n_agents : 4u * (uint32_t)ctx->sm_count;
+    cs_exact_survival_kernel<<<grid, ROW_THREADS, 2 * p.n_agents * sizeof(double), s>>>(ctx->ws, p.n_agents, a0, K,
+                                                                                         p.delta, psurv_out, fsurv_out);
+    return cs_check_launch(ctx);
+}
+
+// ---------------------------------------------------------------------------------------------
 int cs_launch_init(cs_ctx *ctx, cudaStream_t s)
 {
     const cs_params &p = ctx->p;

@@ -466,7 +466,7 @@ int cs_launch_select(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, int p
                      uint32_t *ids_out, uint32_t *n_out, cudaStream_t s)
 {
     SelArgs a;
-    fill_args(ctx, idx, now, ctx->ws.fsurv, a);
+    fill_args(ctx, idx, now, ctx->fsurv_override ? ctx->fsurv_override : ctx->ws.fsurv, a);
     a.tier = tier;
     a.k = k;
     if (ctx->select_path != CS_SELECT_MULTI && idx->n_blocks <= CS_SELECT_CLUSTER_MAX_BLOCKS) {

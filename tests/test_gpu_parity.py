@@ -356,3 +356,38 @@ def test_offload_straight_from_select_output():
     assert np.array_equal(host_t.numpy(), want)
     assert c.get_status() == 0
     assert c.launch_count() > 0
+
+
+# ---- exact survival probability (Eq. 6) as an alternative scorer -----------------------------------------
+@pytest.mark.parametrize("name,K", [("tiny", 4), ("llama8b", 3), ("llama70b", 5), ("meta1m", 4)])
+def test_exact_survival_parity_and_select(name, K):
+    cfg = synth.CONFIGS[name]
+    n = 20000
+    c, o = warm_state(cfg, 3000, n, r_min=0.02)
+    ps, fs = c.exact_survival(K)
+    want = o.exact_survival(K)
+    got = ps.cpu().numpy().astype(np.float64)
+    assert np.all(np.abs(got - want) <= H.REL_TOL * np.maximum(want, 1e-3)), np.abs(got - want).max()
+    assert np.all(np.abs(fs.cpu().numpy() - (want + float(np.float32(0.01)))) <= 2e-7 * (want + 0.01) + 1e-9)
+    assert abs(float(want.sum()) - float(got.sum())) < 1e-4 and np.all(got >= 0) and np.all(got <= 1 + 1e-6)
+    # explicit start agent, K = 1 is the row of the transition matrix
+    ps1, _ = c.exact_survival(1, a0=2)
+    assert np.allclose(ps1.cpu().numpy(), o.P64[2], rtol=1e-6, atol=1e-9)
+    # selections driven by the exact table: same kernels, other first factor of Eq. 9
+    idx = synth.make_block_index(cfg, n=n)
+    d = cs.DeviceIndex.from_host(idx, DEV)
+    c.use_survival_table(fs)
+    o.ptilde = want.copy()
+    o.fsurv32 = (want + float(np.float32(o.p.delta))).astype(np.float32)
+    s64, s32 = o.scores(idx, 100_000)
+    s = c.score_blocks(d, 100_000).cpu().numpy()
+    assert np.all(np.abs(s - s64) <= H.REL_TOL * s64)
+    for k in (64, 2000):
+        ids, n_out = c.select_victims(d, 100_000, 0, k)
+        o_ids, o_n = o.select_victims(idx, 100_000, 0, k, s32)
+        H.assert_list_matches(ids.cpu().numpy().view(np.uint32)[:k], int(n_out.item()), o_ids, o_n, s64)
+    c.use_survival_table(None)                           # back to the hop-distance table of Eq. 8
+    o.survival()
+    _, s32b = o.scores(idx, 100_000)
+    assert np.array_equal(c.score_blocks(d, 100_000).cpu().numpy(), s32b)
+    assert c.get_status() == 0
