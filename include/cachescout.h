@@ -85,6 +85,9 @@ typedef struct cs_params {
     float lambda;           /* recency decay rate of Eq. 9, >= 0 */
     float delta;            /* floor of Eq. 9, > 0 */
     float r_min;            /* prefetch gate of Eq. 11 */
+    uint32_t prefer_other_copy; /* 0: victims ordered by (score, last_access, id).  1: among equal scores,
+                                   blocks whose contents already exist on the other tier go first (no
+                                   offload needed, Sec. 4): (score, has no copy, last_access, id) */
 } cs_params;
 
 /* Structure-of-arrays metadata of the cached blocks (all dev, each [n_blocks] unless

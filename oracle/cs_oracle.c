@@ -197,12 +197,13 @@ void orc_scores(uint32_t n, uint32_t A, const uint16_t *agent, const uint32_t *l
  * first k.  Keys use the bit pattern of the (positive) fp32 score, so equal scores are
  * exactly the equal floats.
  * ------------------------------------------------------------------------------------ */
-typedef struct { uint32_t primary, secondary, id; } orc_key;
+typedef struct { uint32_t primary, tiebreak, secondary, id; } orc_key;
 
 static int key_cmp(const void *x, const void *y)
 {
     const orc_key *a = (const orc_key *)x, *b = (const orc_key *)y;
     if (a->primary != b->primary) return a->primary < b->primary ? -1 : 1;
+    if (a->tiebreak != b->tiebreak) return a->tiebreak < b->tiebreak ? -1 : 1;
     if (a->secondary != b->secondary) return a->secondary < b->secondary ? -1 : 1;
     if (a->id != b->id) return a->id < b->id ? -1 : 1;
     return 0;
@@ -212,10 +213,14 @@ static uint32_t f32_bits(float f) { uint32_t u; memcpy(&u, &f, 4); return u; }
 
 /* Algorithm 1, Evict: arg-min of ScoreBlock over the evictable set, k times over: the k
  * lowest (score, last_access, id) among VALID, not PINNED, ref_count 0, on tier `tier`
- * (0 GPU, 1 host), agent < A.  ids_out padded with ORC_ID_NONE; returns n_out. */
+ * (0 GPU, 1 host), agent < A.  ids_out padded with ORC_ID_NONE; returns n_out.
+ * prefer_copy != 0 adds the preference of Sec. 4 for blocks whose contents already exist on the
+ * other tier (no offload needed): among equal scores those go first, i.e. the order becomes
+ * (score, has no copy, last_access, id). */
 uint32_t orc_select_victims(uint32_t n, uint32_t A, const uint16_t *agent, const uint8_t *ref_count,
                             const uint8_t *flags, const uint32_t *last_access,
-                            const float *score32, uint32_t tier, uint32_t k, uint32_t *ids_out)
+                            const float *score32, uint32_t tier, uint32_t k, int prefer_copy,
+                            uint32_t *ids_out)
 {
     orc_key *keys = (orc_key *)malloc(((size_t)n + 1) * sizeof(orc_key));
     uint32_t m = 0;
@@ -225,6 +230,7 @@ uint32_t orc_select_victims(uint32_t n, uint32_t A, const uint16_t *agent, const
         if (((f & FLAG_TIER_HOST) ? 1u : 0u) != tier) continue;
         if (agent[b] >= A) continue;
         keys[m].primary = f32_bits(score32[b]);
+        keys[m].tiebreak = (prefer_copy && !(f & FLAG_OTHER_COPY)) ? 1u : 0u;
         keys[m].secondary = last_access[b];
         keys[m].id = b;
         ++m;
@@ -261,6 +267,7 @@ uint32_t orc_select_prefetch(uint32_t n, uint32_t A, const uint16_t *agent, cons
         if (anchor_blocks && !(depth[b] < anchor_blocks[a])) continue;
         /* descending score / last_access as ascending complemented words; a* class first */
         keys[m].primary = ((a == a_star) ? 0u : 0x80000000u) | (~f32_bits(score32[b]) & 0x7FFFFFFFu);
+        keys[m].tiebreak = 0u;
         keys[m].secondary = ~last_access[b];
         keys[m].id = b;
         ++m;

@@ -65,6 +65,7 @@ class Params:
     lam: float = 0.01
     delta: float = 0.01
     r_min: float = 0.3
+    prefer_other_copy: int = 0
 
 
 class Oracle:
@@ -150,7 +151,8 @@ class Oracle:
         ids = np.empty(k, np.uint32)
         n_out = lib().orc_select_victims(
             C.c_uint32(idx.n), C.c_uint32(self.p.n_agents), _p(idx.agent), _p(idx.ref_count),
-            _p(idx.flags), _p(idx.last_access), _p(score32), C.c_uint32(tier), C.c_uint32(k), _p(ids))
+            _p(idx.flags), _p(idx.last_access), _p(score32), C.c_uint32(tier), C.c_uint32(k),
+            C.c_int(int(self.p.prefer_other_copy)), _p(ids))
         return ids, int(n_out)
 
     def select_prefetch(self, idx, now: int, k: int, score32=None):

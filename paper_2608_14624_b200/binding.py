@@ -38,7 +38,8 @@ EXPORTS = ("cs_workspace_bytes", "cs_create", "cs_destroy", "cs_observe_invocati
 class cs_params(C.Structure):
     _fields_ = [("n_agents", C.c_uint32), ("n_chains", C.c_uint32), ("max_blocks", C.c_uint32),
                 ("block_tokens", C.c_uint32), ("e_max", C.c_uint32), ("eps", C.c_float), ("tau", C.c_float),
-                ("lambda_", C.c_float), ("delta", C.c_float), ("r_min", C.c_float)]
+                ("lambda_", C.c_float), ("delta", C.c_float), ("r_min", C.c_float),
+                ("prefer_other_copy", C.c_uint32)]
 
 
 class cs_block_index(C.Structure):
@@ -234,8 +235,9 @@ def cs_version() -> int:
 # ---- small holders that keep tensors alive next to the structs that point into them ---------------------
 def make_params(n_agents: int, n_chains: int = 1, max_blocks: int = 1, block_tokens: int = 16, e_max: int = 4,
                 eps: float = 0.01, tau: float = 0.05, lam: float = 0.01, delta: float = 0.01,
-                r_min: float = 0.3) -> cs_params:
-    return cs_params(n_agents, n_chains, max_blocks, block_tokens, e_max, eps, tau, lam, delta, r_min)
+                r_min: float = 0.3, prefer_other_copy: int = 0) -> cs_params:
+    return cs_params(n_agents, n_chains, max_blocks, block_tokens, e_max, eps, tau, lam, delta, r_min,
+                     prefer_other_copy)
 
 
 @dataclass

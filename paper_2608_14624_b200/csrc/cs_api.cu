@@ -22,6 +22,7 @@ int cs_validate_params(const cs_params *p)
     if (!(p->lambda >= 0.0f) || !isfinite(p->lambda)) return CS_EINVAL;
     if (!(p->delta > 0.0f) || !isfinite(p->delta)) return CS_EINVAL;    // the floor keeps both factors positive
     if (!isfinite(p->r_min)) return CS_EINVAL;
+    if (p->prefer_other_copy > 1) return CS_EINVAL;
     return CS_OK;
 }
 

@@ -167,7 +167,7 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_collect_kernel(SelArgs a, 
                     const uint32_t tok = a.ntok ? grp_u8(G.tk, j) : a.block_tokens;
                     const uint32_t dp = (PF && a.anchor) ? grp_u16(G.dp0, G.dp1, j) : 0u;
                     uint32_t prj;
-                    if (entry_key_rest<PF>(a, T, &ws.sc->status, grp_u16(G.ag0, G.ag1, j), dp, grp_u32(G, j), tok,
+                    if (entry_key_rest<PF>(a, T, &ws.sc->status, grp_u16(G.ag0, G.ag1, j), dp, grp_u8(G.fl, j), grp_u32(G, j), tok,
                                            prj, se) &&
                         (prj >> 20) <= b0)
                         mask |= 1u << j;
@@ -191,7 +191,7 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_collect_kernel(SelArgs a, 
                     uint32_t prj, se;
                     const uint32_t tok = a.ntok ? grp_u8(G.tk, j) : a.block_tokens;
                     const uint32_t dp = (PF && a.anchor) ? grp_u16(G.dp0, G.dp1, j) : 0u;
-                    entry_key_rest<PF>(a, T, &ws.sc->status, grp_u16(G.ag0, G.ag1, j), dp, grp_u32(G, j), tok, prj, se);
+                    entry_key_rest<PF>(a, T, &ws.sc->status, grp_u16(G.ag0, G.ag1, j), dp, grp_u8(G.fl, j), grp_u32(G, j), tok, prj, se);
                     ws.cand_km[pos] = ((unsigned long long)prj << 32) | se;
                     ws.cand_id[pos] = g * GRP + j;
                     ++pos;
@@ -436,6 +436,7 @@ static void fill_args(const cs_ctx *ctx, const cs_block_index *idx, uint32_t now
     a.delta = ctx->p.delta;
     a.tier = 0;
     a.k = 0;
+    a.prefer_copy = ctx->p.prefer_other_copy ? 1u : 0u;
 }
 
 static uint32_t scan_grid(const cs_ctx *ctx, uint32_t n, uint32_t per_cta)

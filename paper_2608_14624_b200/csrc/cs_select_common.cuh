@@ -17,7 +17,7 @@ struct SelArgs {
     const float *fsurv;
     uint32_t n, now, A, block_tokens, gtab_len, age_sat;
     float lambda, delta;
-    uint32_t tier, k;
+    uint32_t tier, k, prefer_copy;
 };
 
 // Per-CTA copies of the small tables every entry looks up.
@@ -59,8 +59,8 @@ __device__ __forceinline__ float score_of(const SelArgs &a, const Tables &T, uin
 // anchor-depth rule of the prefetch list, and the 96-bit key.
 template <bool PF>
 __device__ __forceinline__ bool entry_key_rest(const SelArgs &a, const Tables &T, uint32_t *status, uint32_t agent,
-                                               uint32_t depth, uint32_t la, uint32_t tok, uint32_t &primary,
-                                               uint32_t &secondary)
+                                               uint32_t depth, uint32_t flags, uint32_t la, uint32_t tok,
+                                               uint32_t &primary, uint32_t &secondary)
 {
     if (agent >= a.A) { atomicOr(status, CS_ST_BAD_AGENT); return false; }
     if (PF && a.anchor && !(depth < T.anchor[agent])) return false;
@@ -69,7 +69,9 @@ __device__ __forceinline__ bool entry_key_rest(const SelArgs &a, const Tables &T
         primary = ((agent == T.a_star) ? 0u : 0x80000000u) | (~bits & 0x7FFFFFFFu);
         secondary = ~la;
     } else {
-        primary = bits;
+        // Optional preference (Sec. 4) for victims whose contents already exist on the other tier:
+        // one extra key bit right below the score (a positive float leaves bit 31 free).
+        primary = a.prefer_copy ? ((bits << 1) | ((flags & CS_FLAG_OTHER_COPY) ? 0u : 1u)) : bits;
         secondary = la;
     }
     return true;
@@ -87,7 +89,7 @@ __device__ __forceinline__ bool entry_key(const SelArgs &a, const Tables &T, uin
     } else {
         if (((flags >> 2) & 1u) != a.tier) return false;
     }
-    return entry_key_rest<PF>(a, T, status, agent, depth, la, tok, primary, secondary);
+    return entry_key_rest<PF>(a, T, status, agent, depth, flags, la, tok, primary, secondary);
 }
 
 // One group of 16 consecutive entries in registers.
@@ -169,7 +171,7 @@ __device__ __forceinline__ void for_each_eligible(const SelArgs &a, const Tables
             uint32_t pr, se;
             const uint32_t tok = a.ntok ? grp_u8(G.tk, j) : a.block_tokens;
             const uint32_t dp = (PF && a.anchor) ? grp_u16(G.dp0, G.dp1, j) : 0u;
-            if (entry_key_rest<PF>(a, T, status, grp_u16(G.ag0, G.ag1, j), dp, grp_u32(G, j), tok, pr, se))
+            if (entry_key_rest<PF>(a, T, status, grp_u16(G.ag0, G.ag1, j), dp, grp_u8(G.fl, j), grp_u32(G, j), tok, pr, se))
                 f(g * GRP + j, pr, se);
         }
     }

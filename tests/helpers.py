@@ -12,7 +12,8 @@ R_FRAGILE = 1e-4        # inputs whose R lies this close to r_min are rejected a
 def oracle_params(p) -> orc.Params:
     """cs_params (ctypes) -> oracle Params."""
     return orc.Params(n_agents=p.n_agents, n_chains=p.n_chains, block_tokens=p.block_tokens, e_max=p.e_max,
-                      eps=p.eps, tau=p.tau, lam=p.lambda_, delta=p.delta, r_min=p.r_min)
+                      eps=p.eps, tau=p.tau, lam=p.lambda_, delta=p.delta, r_min=p.r_min,
+                      prefer_other_copy=p.prefer_other_copy)
 
 
 def compare_model(cs, o: orc.Oracle):

@@ -391,3 +391,15 @@ def test_exact_survival_parity_and_select(name, K):
     _, s32b = o.scores(idx, 100_000)
     assert np.array_equal(c.score_blocks(d, 100_000).cpu().numpy(), s32b)
     assert c.get_status() == 0
+
+
+def test_select_with_other_tier_copy_preference():
+    """cs_params.prefer_other_copy = 1: (score, has no copy, last_access, id), both select paths."""
+    cfg = synth.CONFIGS["llama8b"]
+    c, o = warm_state(cfg, 1000, 40000, r_min=0.02, prefer_other_copy=1)
+    idx = synth.make_block_index(cfg, n=40000, with_tokens=False)
+    idx.last_access[:] = 100_000 - (np.arange(40000) % 37)                 # many equal scores
+    assert run_selects(c, o, idx, 100_000, (64, 3000)) == 0
+    c2, o2 = warm_state(synth.CONFIGS["meta1m"], 2000, 300_000, r_min=0.02, prefer_other_copy=1)
+    idx2 = synth.make_block_index(synth.CONFIGS["meta1m"], n=300_000, tier="random")     # above the cluster limit
+    assert run_selects(c2, o2, idx2, 100_000, (10_000,), tiers=(0,)) == 0

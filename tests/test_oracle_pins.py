@@ -481,3 +481,28 @@ def test_exact_survival_on_a_deterministic_cycle():
         assert np.allclose(got, want, atol=1e-6)
     # the hop-distance proxy of Eq. 8 orders the agents the same way on this chain
     assert np.array_equal(np.argsort(-o.exact_survival(3), kind="stable")[:3], np.argsort(o.E, kind="stable")[1:4])
+
+
+def test_preference_for_blocks_with_a_copy_on_the_other_tier():
+    """Sec. 4: among equally scored victims, those whose contents already exist on the other tier
+    go first (they need no offload); the score still dominates."""
+    for seed in range(4):
+        cfg, o, idx = small_state(seed)
+        o.p.prefer_other_copy = 1
+        _, s32 = o.scores(idx, 3000)
+        for tier in (0, 1):
+            ids, n_out = o.select_victims(idx, 3000, tier, 40)
+            rows = []
+            for b in range(idx.n):
+                f = int(idx.flags[b])
+                if not f & 1 or f & 2 or idx.ref_count[b] != 0 or ((f >> 2) & 1) != tier:
+                    continue
+                rows.append((float(s32[b]), 0 if f & 8 else 1, int(idx.last_access[b]), b))
+            rows.sort()
+            assert ids[:n_out].tolist() == [r[3] for r in rows[:40]]
+    o = run_trace([0, 1], 2, prefer_other_copy=1)
+    # equal scores need equal ages: blocks 0 and 1 tie, block 1 has a copy and goes first
+    idx = make_idx([0, 0], [90, 90], flags=[1, 1 | 8])
+    assert o.select_victims(idx, 100, 0, 2)[0].tolist() == [1, 0]
+    o.p.prefer_other_copy = 0
+    assert o.select_victims(idx, 100, 0, 2)[0].tolist() == [0, 1]
