@@ -403,3 +403,36 @@ def test_select_with_other_tier_copy_preference():
     c2, o2 = warm_state(synth.CONFIGS["meta1m"], 2000, 300_000, r_min=0.02, prefer_other_copy=1)
     idx2 = synth.make_block_index(synth.CONFIGS["meta1m"], n=300_000, tier="random")     # above the cluster limit
     assert run_selects(c2, o2, idx2, 100_000, (10_000,), tiers=(0,)) == 0
+
+
+# ---- corners of the parameter space -----------------------------------------------------------------------
+@pytest.mark.parametrize("kw", [
+    dict(lam=0.0), dict(e_max=1), dict(tau=0.0), dict(tau=1.5), dict(delta=0.5, eps=1.0),
+    dict(lam=3.0, delta=1e-4), dict(e_max=37, tau=0.2), dict(block_tokens=255), dict(lam=1e-5)])
+def test_parameter_corners(kw):
+    cfg = synth.shrink(synth.CONFIGS["llama70b"], block_tokens=kw.pop("block_tokens", 16))
+    c, o = warm_state(cfg, 2000, 5000, r_min=0.02, **kw)
+    H.compare_model(c, o)
+    idx = synth.make_block_index(cfg, n=5000)
+    idx.last_access[::3] = 100_000 - np.arange(len(idx.last_access[::3])) % 9000    # ages across the whole table range
+    d = cs.DeviceIndex.from_host(idx, DEV)
+    s = c.score_blocks(d, 100_000).cpu().numpy()
+    s64, s32 = o.scores(idx, 100_000)
+    assert np.all(np.abs(s - s64) <= H.REL_TOL * s64)
+    run_selects(c, o, idx, 100_000, (100,))
+
+
+def test_maximum_agent_count():
+    """1,024 agents: 32-word adjacency rows, 4 MiB transition matrix, rows that span several warps."""
+    cfg = synth.shrink(synth.CONFIGS["meta1m"], n_agents=1024, sessions=64, n_chains=64, events_per_step=(8, 8))
+    tr = synth.make_trace(cfg, n_invocations=30000)
+    c, o = make_ctx(cfg, 20000, r_min=0.02, tau=0.1)
+    for lo in range(0, 30000, 7000):
+        c.observe_invocations(dev(tr.chain[lo:lo + 7000]), dev(tr.agent[lo:lo + 7000]), None)
+        o.observe(tr.chain[lo:lo + 7000], tr.agent[lo:lo + 7000])
+        H.compare_model(c, o)
+    idx = synth.make_block_index(cfg, n=20000)
+    assert run_selects(c, o, idx, 100_000, (500,)) == 0
+    ps, _ = c.exact_survival(3)
+    want = o.exact_survival(3)
+    assert np.all(np.abs(ps.cpu().numpy() - want) <= H.REL_TOL * np.maximum(want, 1e-3))
