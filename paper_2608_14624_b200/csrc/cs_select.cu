@@ -37,10 +37,10 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_score_kernel(SelArgs a, cs_wor
     load_tables(a, ws, smem, T, false);
     __syncthreads();
     const uint32_t gtid = blockIdx.x * blockDim.x + threadIdx.x, nth = gridDim.x * blockDim.x;
-    const uint32_t n_groups = a.n / GRP;
-    for (uint32_t g = gtid; g < n_groups; g += nth) {
+    const uint32_t lane = threadIdx.x & 31, n_tiles = a.n / TILE;
+    for (uint32_t t = gtid >> 5; t < n_tiles; t += nth >> 5) {
         Group G;
-        load_group<false, false>(a, g, G);                  // the score needs agent, last_access and size only
+        load_group<false, false>(a, t, lane, G);            // the score needs agent, last_access and size only
         float s[GRP];
 #pragma unroll
         for (int j = 0; j < GRP; ++j) {
@@ -49,11 +49,11 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_score_kernel(SelArgs a, cs_wor
             if (ag < a.A) s[j] = score_of(a, T, ag, grp_u32(G, j), tok);
             else { s[j] = 0.0f; atomicOr(&ws.sc->status, CS_ST_BAD_AGENT); }
         }
-        float4 *o = (float4 *)out + 4 * g;
+        float4 *o = (float4 *)out + t * 128u + lane;         // quad q of this lane: coalesced 512 B per warp store
 #pragma unroll
-        for (int q = 0; q < 4; ++q) __stcs(o + q, make_float4(s[4 * q], s[4 * q + 1], s[4 * q + 2], s[4 * q + 3]));
+        for (int q = 0; q < 4; ++q) __stcs(o + 32 * q, make_float4(s[4 * q], s[4 * q + 1], s[4 * q + 2], s[4 * q + 3]));
     }
-    const uint32_t t0 = n_groups * GRP;
+    const uint32_t t0 = n_tiles * TILE;
     if (gtid < a.n - t0) {
         const uint32_t i = t0 + gtid;
         const uint32_t ag = a.agent[i];
@@ -151,14 +151,14 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_collect_kernel(SelArgs a, 
         // Whole groups: count this thread's candidates, reserve a range with one atomic per warp,
         // then write.  The loop bound is rounded up so that whole warps stay in the shuffles.
         const uint32_t gtid = blockIdx.x * blockDim.x + threadIdx.x, nth = gridDim.x * blockDim.x;
-        const uint32_t n_groups = a.n / GRP;
-        const uint32_t n_iter = (n_groups + nth - 1) / nth;
+        const uint32_t n_tiles = a.n / TILE, n_warps = nth >> 5;
+        const uint32_t n_iter = (n_tiles + n_warps - 1) / n_warps;
         for (uint32_t it = 0; it < n_iter; ++it) {
-            const uint32_t g = it * nth + gtid;
+            const uint32_t t = it * n_warps + (gtid >> 5);
             uint32_t mask = 0;               // keys are recomputed for the (few) candidates instead of kept in registers
             Group G;
-            if (g < n_groups) {
-                load_group<PF>(a, g, G);
+            if (t < n_tiles) {
+                load_group<PF>(a, t, lane, G);
                 const uint32_t em = group_elig<PF>(a, G);
 #pragma unroll
                 for (int j = 0; j < GRP; ++j) {
@@ -193,12 +193,12 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_collect_kernel(SelArgs a, 
                     const uint32_t dp = (PF && a.anchor) ? grp_u16(G.dp0, G.dp1, j) : 0u;
                     entry_key_rest<PF>(a, T, &ws.sc->status, grp_u16(G.ag0, G.ag1, j), dp, grp_u8(G.fl, j), grp_u32(G, j), tok, prj, se);
                     ws.cand_km[pos] = ((unsigned long long)prj << 32) | se;
-                    ws.cand_id[pos] = g * GRP + j;
+                    ws.cand_id[pos] = grp_id(t, lane, j);
                     ++pos;
                 }
             }
         }
-        const uint32_t t0 = n_groups * GRP;
+        const uint32_t t0 = n_tiles * TILE;
         if (gtid < a.n - t0) {
             const uint32_t i = t0 + gtid;
             uint32_t p, se;

@@ -133,9 +133,9 @@ cs_select_cluster_kernel(SelArgs a, cs_workspace ws, uint32_t *__restrict__ ids_
     __syncthreads();
     const bool enabled = !PF || prefetch_enabled(ws, a.A);
     csel_stamp(ws, rank, 0);
-    const uint32_t n_groups = a.n / GRP;
+    const uint32_t n_tiles = a.n / TILE;
     const uint32_t cthreads = CL * CSEL_THREADS, ctid = rank * CSEL_THREADS + tid;   // cluster-wide thread id
-    const uint32_t t0 = n_groups * GRP;                                             // start of the ragged tail
+    const uint32_t t0 = n_tiles * TILE;                                              // start of the ragged tail
 
     // ---- phase 1: histogram of this CTA's slice ------------------------------------------------
     if (enabled) {
@@ -147,9 +147,9 @@ cs_select_cluster_kernel(SelArgs a, cs_workspace ws, uint32_t *__restrict__ ids_
             run_bin = bin;
             run_cnt = 1;
         };
-        for (uint32_t g = ctid; g < n_groups; g += cthreads) {
+        for (uint32_t t = ctid >> 5; t < n_tiles; t += cthreads >> 5) {
             Group G;
-            load_group<PF>(a, g, G);
+            load_group<PF>(a, t, lane, G);
             const uint32_t em = group_elig<PF>(a, G);
 #pragma unroll
             for (int j = 0; j < GRP; ++j) {
@@ -211,13 +211,14 @@ cs_select_cluster_kernel(SelArgs a, cs_workspace ws, uint32_t *__restrict__ ids_
     csel_stamp(ws, rank, 2);
     // ---- phase 3: collect the candidates (bin <= b0) ------------------------------------------------------
     if (enabled && b0 != 0xFFFFFFFFu) {
-        const uint32_t n_iter = (n_groups + cthreads - 1) / cthreads;
+        const uint32_t n_warps = cthreads >> 5;
+        const uint32_t n_iter = (n_tiles + n_warps - 1) / n_warps;
         for (uint32_t it = 0; it < n_iter; ++it) {
-            const uint32_t g = it * cthreads + ctid;
+            const uint32_t t = it * n_warps + (ctid >> 5);
             uint32_t mask = 0;               // keys are recomputed for the (few) candidates instead of kept in registers
             Group G;
-            if (g < n_groups) {
-                load_group<PF>(a, g, G);
+            if (t < n_tiles) {
+                load_group<PF>(a, t, lane, G);
                 const uint32_t em = group_elig<PF>(a, G);
 #pragma unroll
                 for (int j = 0; j < GRP; ++j) {
@@ -252,7 +253,7 @@ cs_select_cluster_kernel(SelArgs a, cs_workspace ws, uint32_t *__restrict__ ids_
                     const uint32_t dp = (PF && a.anchor) ? grp_u16(G.dp0, G.dp1, j) : 0u;
                     entry_key_rest<PF>(a, T, &ws.sc->status, grp_u16(G.ag0, G.ag1, j), dp, grp_u8(G.fl, j), grp_u32(G, j), tok, prj, se);
                     ws.cand_km[pos] = ((unsigned long long)prj << 32) | se;
-                    ws.cand_id[pos] = g * GRP + j;
+                    ws.cand_id[pos] = grp_id(t, lane, j);
                     ++pos;
                 }
             }
@@ -415,7 +416,7 @@ static int launch_cluster(cs_ctx *ctx, const SelArgs &a, uint32_t *ids_out, uint
     }
     if (max_cl < 1) return CS_ENOTIMPL;
     // smallest power-of-two cluster that gives every 16-entry group its own thread, at most max_cl
-    const uint32_t n_groups = a.n / GRP;
+    const uint32_t n_groups = a.n / GRP;                 // 16 entries per thread and pass
     int cl = 1;
     while (cl < max_cl && (uint32_t)cl * CSEL_THREADS < n_groups) cl <<= 1;
     cfg.gridDim = dim3(cl);

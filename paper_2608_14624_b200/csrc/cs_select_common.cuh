@@ -4,7 +4,7 @@
 #include "cs_common.cuh"
 
 #define SEL_THREADS 512
-#define GRP 16                    // index entries per thread and iteration (one 128-bit load of bytes)
+#define GRP 16                    // index entries per thread and iteration
 
 struct SelArgs {
     const uint16_t *agent;
@@ -92,28 +92,48 @@ __device__ __forceinline__ bool entry_key(const SelArgs &a, const Tables &T, uin
     return entry_key_rest<PF>(a, T, status, agent, depth, flags, la, tok, primary, secondary);
 }
 
-// One group of 16 consecutive entries in registers.
+// The index is walked in warp tiles of 512 entries.  In step q (0..3) lane L owns the four
+// consecutive entries tile*512 + q*128 + 4L .. +3, so every load instruction of a warp covers one
+// contiguous, fully used span: 512 B of last_access (128-bit loads), 256 B of agent / depth
+// (64-bit), 128 B of flags / ref_count / n_tokens (32-bit).  A thread's 16 entries are numbered
+// j = 4q + r locally; Group keeps them in the order the accessors below expect.
+#define TILE 512u
 struct Group {
     uint4 ag0, ag1, dp0, dp1, rf, fl, la0, la1, la2, la3, tk;
 };
 
-template <bool PF, bool FLAGS = true>
-__device__ __forceinline__ void load_group(const SelArgs &a, uint32_t g, Group &G)
+__device__ __forceinline__ uint32_t grp_id(uint32_t tile, uint32_t lane, int j)
 {
-    G.ag0 = __ldg((const uint4 *)a.agent + 2 * g);
-    G.ag1 = __ldg((const uint4 *)a.agent + 2 * g + 1);
+    return tile * TILE + (uint32_t)(j >> 2) * 128u + 4u * lane + (uint32_t)(j & 3);
+}
+
+template <bool PF, bool FLAGS = true>
+__device__ __forceinline__ void load_group(const SelArgs &a, uint32_t tile, uint32_t lane, Group &G)
+{
+    const uint32_t q0 = tile * 128u + lane;            // index of this lane's first quad, in units of 4 entries
+    const uint4 *la = (const uint4 *)a.la + q0;
+    G.la0 = __ldg(la);
+    G.la1 = __ldg(la + 32);
+    G.la2 = __ldg(la + 64);
+    G.la3 = __ldg(la + 96);
+    const uint2 *ag = (const uint2 *)a.agent + q0;
+    const uint2 g0 = __ldg(ag), g1 = __ldg(ag + 32), g2 = __ldg(ag + 64), g3 = __ldg(ag + 96);
+    G.ag0 = make_uint4(g0.x, g0.y, g1.x, g1.y);
+    G.ag1 = make_uint4(g2.x, g2.y, g3.x, g3.y);
     if (FLAGS) {
-        G.rf = __ldg((const uint4 *)a.ref + g);
-        G.fl = __ldg((const uint4 *)a.flags + g);
+        const uint32_t *rf = (const uint32_t *)a.ref + q0, *fl = (const uint32_t *)a.flags + q0;
+        G.rf = make_uint4(__ldg(rf), __ldg(rf + 32), __ldg(rf + 64), __ldg(rf + 96));
+        G.fl = make_uint4(__ldg(fl), __ldg(fl + 32), __ldg(fl + 64), __ldg(fl + 96));
     }
-    G.la0 = __ldg((const uint4 *)a.la + 4 * g);
-    G.la1 = __ldg((const uint4 *)a.la + 4 * g + 1);
-    G.la2 = __ldg((const uint4 *)a.la + 4 * g + 2);
-    G.la3 = __ldg((const uint4 *)a.la + 4 * g + 3);
-    if (a.ntok) G.tk = __ldg((const uint4 *)a.ntok + g);
+    if (a.ntok) {
+        const uint32_t *tk = (const uint32_t *)a.ntok + q0;
+        G.tk = make_uint4(__ldg(tk), __ldg(tk + 32), __ldg(tk + 64), __ldg(tk + 96));
+    }
     if (PF && a.anchor) {
-        G.dp0 = __ldg((const uint4 *)a.depth + 2 * g);
-        G.dp1 = __ldg((const uint4 *)a.depth + 2 * g + 1);
+        const uint2 *dp = (const uint2 *)a.depth + q0;
+        const uint2 d0 = __ldg(dp), d1 = __ldg(dp + 32), d2 = __ldg(dp + 64), d3 = __ldg(dp + 96);
+        G.dp0 = make_uint4(d0.x, d0.y, d1.x, d1.y);
+        G.dp1 = make_uint4(d2.x, d2.y, d3.x, d3.y);
     }
 }
 
@@ -154,16 +174,16 @@ __device__ __forceinline__ uint32_t group_elig(const SelArgs &a, const Group &G)
     return out;
 }
 
-// Calls f(id, primary, secondary) for every eligible entry this thread owns: whole groups
-// grid-strided, then the ragged tail (n % 16 entries) one entry per thread.
+// Calls f(id, primary, secondary) for every eligible entry this thread owns: whole warp tiles
+// grid-strided, then the ragged tail (n % 512 entries) one entry per thread.
 template <bool PF, typename F>
 __device__ __forceinline__ void for_each_eligible(const SelArgs &a, const Tables &T, uint32_t *status, F f)
 {
     const uint32_t gtid = blockIdx.x * blockDim.x + threadIdx.x, nth = gridDim.x * blockDim.x;
-    const uint32_t n_groups = a.n / GRP;
-    for (uint32_t g = gtid; g < n_groups; g += nth) {
+    const uint32_t lane = threadIdx.x & 31, n_tiles = a.n / TILE;
+    for (uint32_t t = gtid >> 5; t < n_tiles; t += nth >> 5) {
         Group G;
-        load_group<PF>(a, g, G);
+        load_group<PF>(a, t, lane, G);
         const uint32_t em = group_elig<PF>(a, G);
 #pragma unroll
         for (int j = 0; j < GRP; ++j) {
@@ -172,10 +192,10 @@ __device__ __forceinline__ void for_each_eligible(const SelArgs &a, const Tables
             const uint32_t tok = a.ntok ? grp_u8(G.tk, j) : a.block_tokens;
             const uint32_t dp = (PF && a.anchor) ? grp_u16(G.dp0, G.dp1, j) : 0u;
             if (entry_key_rest<PF>(a, T, status, grp_u16(G.ag0, G.ag1, j), dp, grp_u8(G.fl, j), grp_u32(G, j), tok, pr, se))
-                f(g * GRP + j, pr, se);
+                f(grp_id(t, lane, j), pr, se);
         }
     }
-    const uint32_t t0 = n_groups * GRP;
+    const uint32_t t0 = n_tiles * TILE;
     if (gtid < a.n - t0) {
         const uint32_t i = t0 + gtid;
         uint32_t pr, se;
