@@ -445,6 +445,33 @@ def metadata_scale(torch, cs, synth, dev, hbm_peak, calls=200):
             "kernel_launches_per_call": launches, "n_out": [int(vn[0].item()), int(pn[0].item())]}
 
 
+def hbm_regime_section(torch, cs, synth, dev, hbm_peak, n_entries=64_000_000):
+    """Score and select over an index far larger than L2 (64,000,000 entries = 704 MB of metadata), where
+    the scans are bound by memory or instruction issue instead of launch latency: the regime in which a
+    fraction of the HBM roofline is meaningful for these kernels."""
+    cfg = synth.CONFIGS["meta1m"]
+    idx = synth.make_block_index(cfg, n=n_entries, tier="random")
+    d = cs.DeviceIndex.from_host(idx, dev)
+    del idx
+    tr = synth.make_trace(cfg, n_invocations=4000)
+    c = cs.CacheScout(cs.make_params(n_agents=cfg.n_agents, n_chains=cfg.n_chains, max_blocks=n_entries,
+                                     block_tokens=cfg.block_tokens, r_min=0.02), dev)
+    c.observe_invocations(torch.from_numpy(tr.chain).to(dev), torch.from_numpy(tr.agent).to(dev), None)
+    k = cfg.k_victims
+    v = torch.empty(k, dtype=torch.int32, device=dev)
+    vn = torch.zeros(4, dtype=torch.int32, device=dev)
+    sc = torch.empty(n_entries, dtype=torch.float32, device=dev)
+    stream = torch.cuda.current_stream(dev)
+    t_score, _ = time_call(torch, stream, lambda: c.score_blocks(d, 100_000, out=sc), 5, warm=2)
+    t_sel, _ = time_call(torch, stream, lambda: c.select_victims(d, 100_000, 0, k, v, vn), 5, warm=2)
+    score_bytes = n_entries * (2 + 4 + 1 + 4)             # agent, last_access, n_tokens in; fp32 score out
+    sel_bytes = 2 * n_entries * 9 + 4 * k                 # two scans of agent, ref_count, flags, last_access, n_tokens
+    return {"entries": n_entries, "k": k,
+            "score_ms": t_score, "score_GBps": score_bytes / t_score / 1e6, "score_frac_of_hbm_peak": score_bytes / t_score / 1e6 / hbm_peak,
+            "select_ms": t_sel, "select_GBps": sel_bytes / t_sel / 1e6, "select_frac_of_hbm_peak": sel_bytes / t_sel / 1e6 / hbm_peak,
+            "blocks_scored_selected_per_s": n_entries / (t_sel / 1e3), "n_out": int(vn[0].item())}
+
+
 def exact_survival_section(torch, cs, synth, dev):
     """Eq. 6 as an alternative scorer: time of one table (CUDA events) and how far the victim list it
     gives is from the list of the hop-distance proxy of Eq. 8 (context for the approximation)."""
@@ -742,6 +769,7 @@ def main():
         torch.cuda.empty_cache()
         out["metadata_scale"] = metadata_scale(torch, cs, synth, device, hbm_peak)
         out["exact_survival"] = exact_survival_section(torch, cs, synth, device)
+        out["hbm_regime"] = hbm_regime_section(torch, cs, synth, device, hbm_peak)
     # the oracle, as it stands, on this machine's host cores
     ow = OracleStep()
     ow.step(0)

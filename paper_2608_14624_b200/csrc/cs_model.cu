@@ -282,40 +282,70 @@ cs_survival_kernel(cs_workspace ws, uint32_t A, uint32_t W, const uint16_t *__re
 // treats this as too expensive for its per-request runtime and uses the hop proxy of Eq. 8;
 // here it is an alternative scorer (A^3 K multiply-adds, off the critical path).
 // ---------------------------------------------------------------------------------------------
+#define XS_MAX_TARGETS 8
 __global__ void __launch_bounds__(ROW_THREADS)
-cs_exact_survival_kernel(cs_workspace ws, uint32_t A, uint32_t a0_arg, uint32_t K, float delta,
+cs_exact_survival_kernel(cs_workspace ws, uint32_t A, uint32_t a0_arg, uint32_t K, uint32_t n_tgt, float delta,
                          float *__restrict__ psurv_out, float *__restrict__ fsurv_out)
 {
-    extern __shared__ double s_vec[];                 // v[A], w[A]
-    double *v = s_vec, *w = s_vec + A;
+    // A CTA advances n_tgt target agents together, so that every element of the matrix it reads
+    // feeds n_tgt accumulators (the matrix is the only sizeable traffic: A^2 floats per step).
+    extern __shared__ double s_vec[];                 // v[n_tgt][A], w[n_tgt][A]
+    double *v = s_vec, *w = s_vec + (size_t)n_tgt * A;
     const uint32_t tid = threadIdx.x;
     const uint32_t a0 = a0_arg == CS_AGENT_NONE ? ws.sc->last_agent : a0_arg;
-    for (uint32_t a = blockIdx.x; a < A; a += gridDim.x) {
-        // The probability is accumulated as the mass absorbed at a step by step (no 1 - x
-        // cancellation, so small probabilities keep full relative accuracy); the thread that owns
-        // column a does the adding.
-        double hit = 0.0;
-        if (a0 < A) {
+    for (uint32_t base = blockIdx.x * n_tgt; base < A; base += gridDim.x * n_tgt) {
+        // The probability is accumulated as the mass absorbed at the target step by step (no 1 - x
+        // cancellation, so small probabilities keep full relative accuracy).  Column (base + m) of
+        // target m is owned by one thread, which does the adding for that target.
+        double hit[XS_MAX_TARGETS];
+#pragma unroll
+        for (int m = 0; m < XS_MAX_TARGETS; ++m) hit[m] = 0.0;
+        if (a0 < A && K > 0) {
             __syncthreads();
-            for (uint32_t j = tid; j < A; j += ROW_THREADS) v[j] = (j == a0) ? 1.0 : 0.0;
-            __syncthreads();
-            for (uint32_t t = 0; t < K; ++t) {
-                for (uint32_t j = tid; j < A; j += ROW_THREADS) {
-                    double s = 0.0;
-                    for (uint32_t i = 0; i < A; ++i) {
-                        const double vi = v[i];
-                        if (vi != 0.0) s = __dadd_rn(s, __dmul_rn(vi, (double)ws.P[i * A + j]));
+            // step 1: every target starts from the unit mass at a0, i.e. from row a0 of the matrix
+            for (uint32_t j = tid; j < A; j += ROW_THREADS) {
+                const double p = (double)ws.P[a0 * A + j];
+#pragma unroll
+                for (int m = 0; m < XS_MAX_TARGETS; ++m) {
+                    if ((uint32_t)m < n_tgt) {
+                        const bool own = (j == base + m);
+                        if (own) hit[m] += p;
+                        v[(size_t)m * A + j] = own ? 0.0 : p;
                     }
-                    if (j == a) { hit += s; s = 0.0; }
-                    w[j] = s;
+                }
+            }
+            __syncthreads();
+            for (uint32_t t = 1; t < K; ++t) {
+                for (uint32_t j = tid; j < A; j += ROW_THREADS) {
+                    double s[XS_MAX_TARGETS];
+#pragma unroll
+                    for (int m = 0; m < XS_MAX_TARGETS; ++m) s[m] = 0.0;
+                    for (uint32_t i = 0; i < A; ++i) {
+                        const double p = (double)ws.P[i * A + j];
+#pragma unroll
+                        for (int m = 0; m < XS_MAX_TARGETS; ++m)
+                            if ((uint32_t)m < n_tgt) s[m] = fma(v[(size_t)m * A + i], p, s[m]);
+                    }
+#pragma unroll
+                    for (int m = 0; m < XS_MAX_TARGETS; ++m) {
+                        if ((uint32_t)m < n_tgt) {
+                            const bool own = (j == base + m);
+                            if (own) hit[m] += s[m];
+                            w[(size_t)m * A + j] = own ? 0.0 : s[m];
+                        }
+                    }
                 }
                 __syncthreads();
                 double *tmp = v; v = w; w = tmp;
             }
         }
-        if (tid == (a % ROW_THREADS)) {
-            if (psurv_out) psurv_out[a] = (float)hit;
-            if (fsurv_out) fsurv_out[a] = (float)(hit + (double)delta);
+#pragma unroll
+        for (int m = 0; m < XS_MAX_TARGETS; ++m) {
+            const uint32_t a = base + m;
+            if ((uint32_t)m < n_tgt && a < A && tid == (a % ROW_THREADS)) {
+                if (psurv_out) psurv_out[a] = (float)hit[m];
+                if (fsurv_out) fsurv_out[a] = (float)(hit[m] + (double)delta);
+            }
         }
     }
 }
@@ -323,9 +353,12 @@ cs_exact_survival_kernel(cs_workspace ws, uint32_t A, uint32_t a0_arg, uint32_t 
 int cs_launch_exact_survival(cs_ctx *ctx, uint32_t a0, uint32_t K, float *psurv_out, float *fsurv_out, cudaStream_t s)
 {
     const cs_params &p = ctx->p;
-    const uint32_t grid = p.n_agents < 4u * (uint32_t)ctx->sm_count ? p.n_agents : 4u * (uint32_t)ctx->sm_count;
-    cs_exact_survival_kernel<<<grid, ROW_THREADS, 2 * p.n_agents * sizeof(double), s>>>(ctx->ws, p.n_agents, a0, K,
-                                                                                         p.delta, psurv_out, fsurv_out);
+    uint32_t n_tgt = 2048u / p.n_agents;               // 2 * n_tgt * A doubles of shared memory <= 32 KiB
+    if (n_tgt > XS_MAX_TARGETS) n_tgt = XS_MAX_TARGETS;
+    if (n_tgt < 1) n_tgt = 1;
+    const uint32_t grid = (p.n_agents + n_tgt - 1) / n_tgt;
+    cs_exact_survival_kernel<<<grid, ROW_THREADS, 2 * (size_t)n_tgt * p.n_agents * sizeof(double), s>>>(
+        ctx->ws, p.n_agents, a0, K, n_tgt, p.delta, psurv_out, fsurv_out);
     return cs_check_launch(ctx);
 }
 
