@@ -13,7 +13,7 @@ from dataclasses import dataclass, field
 from typing import Optional
 
 HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(HERE, "libcachescout.so")
+LIB_PATH = os.environ.get("CACHESCOUT_LIB") or os.path.join(HERE, "libcachescout.so")   # override: another build of the same ABI
 
 CS_OK = 0
 CS_EINVAL, CS_ECAPACITY, CS_ENOTIMPL, CS_ECUDA, CS_EDEVICE_STATUS, CS_ENOMEM = -1, -2, -3, -4, -5, -6

@@ -23,9 +23,15 @@
 #define MV_UNROLL 4
 #define MV_PIECE (MV_THREADS * MV_UNROLL * 16)      // bytes per work item of the load/store path
 
+#ifndef TM_WARPS
 #define TM_WARPS 4                                   // independent pipelines per CTA
+#endif
+#ifndef TM_STAGES
 #define TM_STAGES 3                                  // ring slots per pipeline
+#endif
+#ifndef TM_PIECE
 #define TM_PIECE 16384u                              // bytes per ring slot
+#endif
 #define TM_SMEM (TM_WARPS * TM_STAGES * TM_PIECE)    // 192 KiB
 #define TM_SPIN_LIMIT (1u << 20)                     // bounded mbarrier wait (polls with back-off: >= 0.1 s)
 

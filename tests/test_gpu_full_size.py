@@ -129,7 +129,7 @@ def test_mover_70b_block_geometry():
         assert c.get_status() == cs.CS_ST_BAD_SLOT
 
 
-@pytest.mark.parametrize("chain_mode", ["session", "single"])
+@pytest.mark.parametrize("chain_mode", ["session", "single", "llama70b-shape"])
 def test_closed_loop_teacher_forced_tiny(chain_mode):
     """Tiny configuration end to end: 4 agents, 200 invocations, 512-block GPU pool, 2,048-slot host
     tier, 32 victims / 64 prefetch candidates per step.  Every step both sides get the same state;
@@ -137,6 +137,9 @@ def test_closed_loop_teacher_forced_tiny(chain_mode):
     cfg = synth.CONFIGS["tiny"]
     if chain_mode == "session":
         cfg = synth.shrink(cfg, sessions=4, n_chains=4, events_per_step=(1, 3))
+    elif chain_mode == "llama70b-shape":          # 30 agents, sparse workflow matrix, 5 MiB blocks; pools cut to fit the oracle
+        cfg = synth.shrink(synth.CONFIGS["llama70b"], gpu_blocks=64, host_blocks=128, invocations=240, sessions=16,
+                           n_chains=16, k_victims=8, k_prefetch=12)
     G, Hs, L, chunk = cfg.gpu_blocks, cfg.host_blocks, cfg.n_layers, cfg.chunk_bytes
     p = cs.make_params(n_agents=cfg.n_agents, n_chains=cfg.n_chains, max_blocks=cfg.n_index,
                        block_tokens=cfg.block_tokens, r_min=0.05)
