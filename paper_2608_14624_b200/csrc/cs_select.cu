@@ -227,22 +227,7 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_collect_kernel(SelArgs a, 
         }
     }
     __syncthreads();
-    for (uint32_t size = 2; size <= CS_SAMPLE; size <<= 1) {
-        for (uint32_t stride = size >> 1; stride > 0; stride >>= 1) {
-            for (uint32_t t = threadIdx.x; t < CS_SAMPLE / 2; t += blockDim.x) {
-                const uint32_t lo = 2 * t - (t & (stride - 1));
-                const uint32_t hi = lo + stride;
-                const bool up = (lo & size) == 0;
-                const unsigned long long ka = s_km[lo], kb = s_km[hi];
-                const uint32_t ia = s_id[lo], ib = s_id[hi];
-                if (key_less(kb, ib, ka, ia) == up) {
-                    s_km[lo] = kb; s_id[lo] = ib;
-                    s_km[hi] = ka; s_id[hi] = ia;
-                }
-            }
-            __syncthreads();
-        }
-    }
+    bitonic_sort_fast(s_km, s_id, CS_SAMPLE);            // 512 threads, two keys each
     uint32_t n_spl = c / 64;
     if (n_spl > CS_MAX_SPLITTERS) n_spl = CS_MAX_SPLITTERS;
     for (uint32_t j = threadIdx.x; j <= CS_MAX_SPLITTERS; j += blockDim.x) {
@@ -378,27 +363,31 @@ cs_sel_rank_kernel(cs_workspace ws, uint32_t k, uint32_t *__restrict__ ids_out, 
         const uint32_t beg = ws.boff[b], end = ws.boff[b + 1], m = end - beg;
         __syncthreads();
         if (m <= RANK_TILE) {
-            uint32_t P = 2;
+            uint32_t P = 64;
             while (P < m) P <<= 1;
             for (uint32_t i = threadIdx.x; i < P; i += blockDim.x) {
                 t_km[i] = i < m ? ws.sort_km[beg + i] : ~0ull;
                 t_id[i] = i < m ? ws.sort_id[beg + i] : 0xFFFFFFFFu;
             }
             __syncthreads();
-            for (uint32_t size = 2; size <= P; size <<= 1) {
-                for (uint32_t stride = size >> 1; stride > 0; stride >>= 1) {
-                    for (uint32_t t = threadIdx.x; t < P / 2; t += blockDim.x) {
-                        const uint32_t lo = 2 * t - (t & (stride - 1));
-                        const uint32_t hi = lo + stride;
-                        const bool up = (lo & size) == 0;
-                        const unsigned long long ka = t_km[lo], kb = t_km[hi];
-                        const uint32_t ia = t_id[lo], ib = t_id[hi];
-                        if (key_less(kb, ib, ka, ia) == up) {
-                            t_km[lo] = kb; t_id[lo] = ib;
-                            t_km[hi] = ka; t_id[hi] = ia;
+            if (P <= 2 * blockDim.x) {
+                bitonic_sort_fast(t_km, t_id, P);
+            } else {
+                for (uint32_t size = 2; size <= P; size <<= 1) {
+                    for (uint32_t stride = size >> 1; stride > 0; stride >>= 1) {
+                        for (uint32_t t = threadIdx.x; t < P / 2; t += blockDim.x) {
+                            const uint32_t lo = 2 * t - (t & (stride - 1));
+                            const uint32_t hi = lo + stride;
+                            const bool up = (lo & size) == 0;
+                            const unsigned long long ka = t_km[lo], kb = t_km[hi];
+                            const uint32_t ia = t_id[lo], ib = t_id[hi];
+                            if (key_less(kb, ib, ka, ia) == up) {
+                                t_km[lo] = kb; t_id[lo] = ib;
+                                t_km[hi] = ka; t_id[hi] = ia;
+                            }
                         }
+                        __syncthreads();
                     }
-                    __syncthreads();
                 }
             }
             for (uint32_t i = threadIdx.x; i < m; i += blockDim.x)

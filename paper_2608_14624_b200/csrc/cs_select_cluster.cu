@@ -88,6 +88,7 @@ __device__ __forceinline__ uint32_t csel_block_scan(uint32_t v, uint32_t *s_part
 // In-place bitonic sort of P (power of two) keys in shared memory, ascending by (km, id).
 __device__ __forceinline__ void csel_bitonic(unsigned long long *km, uint32_t *id, uint32_t P)
 {
+    if (P >= 64 && P <= 2 * CSEL_THREADS) { bitonic_sort_fast(km, id, P); return; }
     for (uint32_t size = 2; size <= P; size <<= 1) {
         for (uint32_t stride = size >> 1; stride > 0; stride >>= 1) {
             for (uint32_t t = threadIdx.x; t < P / 2; t += blockDim.x) {
@@ -278,7 +279,7 @@ cs_select_cluster_kernel(SelArgs a, cs_workspace ws, uint32_t *__restrict__ ids_
     // ---- phase 4, small: CTA 0 sorts everything in shared memory ---------------------------------------------
     if (c <= CSEL_SORT_MAX) {
         if (rank != 0 || c == 0) return;
-        uint32_t P = 32;
+        uint32_t P = 64;
         while (P < c) P <<= 1;
         for (uint32_t i = tid; i < P; i += CSEL_THREADS) {
             S.km[i] = i < c ? __ldcg(&ws.cand_km[i]) : ~0ull;
@@ -360,7 +361,7 @@ cs_select_cluster_kernel(SelArgs a, cs_workspace ws, uint32_t *__restrict__ ids_
         const uint32_t beg = s_off[b], end = s_off[b + 1], m = end - beg;
         __syncthreads();
         if (m <= CSEL_SORT_MAX) {
-            uint32_t P = 2;
+            uint32_t P = 64;
             while (P < m) P <<= 1;
             for (uint32_t i = tid; i < P; i += CSEL_THREADS) {
                 S.km[i] = i < m ? __ldcg(&ws.sort_km[beg + i]) : ~0ull;

@@ -229,3 +229,61 @@ __device__ __forceinline__ bool key_less(unsigned long long km_a, uint32_t id_a,
 }
 
 
+
+// ---------------------------------------------------------------------------------------------
+// Bitonic sort of P keys (power of two, 64 <= P <= 2 * blockDim.x) held in shared memory,
+// ascending by (km, id).  Each thread keeps two neighbouring elements in registers; compare-
+// exchange steps whose partner lies in the same warp (element distance <= 32) use shuffles and
+// no barrier, only the longer distances go through shared memory.  Called by the whole CTA.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void cx_keep(unsigned long long &k, uint32_t &i, unsigned long long pk, uint32_t pi,
+                                        bool keep_min)
+{
+    const bool partner_less = key_less(pk, pi, k, i);
+    if (partner_less == keep_min) { k = pk; i = pi; }
+}
+
+__device__ __forceinline__ void bitonic_sort_fast(unsigned long long *km, uint32_t *id, uint32_t P)
+{
+    const uint32_t t = threadIdx.x;
+    const bool act = t < P / 2;                           // whole warps, because P >= 64
+    unsigned long long k0 = 0, k1 = 0;
+    uint32_t i0 = 0, i1 = 0;
+    if (act) { k0 = km[2 * t]; k1 = km[2 * t + 1]; i0 = id[2 * t]; i1 = id[2 * t + 1]; }
+    for (uint32_t size = 2; size <= P; size <<= 1) {
+        const bool up = ((2 * t) & size) == 0;            // both of this thread's elements share the direction
+        uint32_t stride = size >> 1;
+        if (stride >= 64) {                               // partners in other warps: through shared memory
+            if (act) { km[2 * t] = k0; km[2 * t + 1] = k1; id[2 * t] = i0; id[2 * t + 1] = i1; }
+            __syncthreads();
+            for (; stride >= 64; stride >>= 1) {
+                if (act) {
+                    const uint32_t lo = 2 * t - (t & (stride - 1)), hi = lo + stride;
+                    const bool up2 = (lo & size) == 0;
+                    const unsigned long long ka = km[lo], kb = km[hi];
+                    const uint32_t ia = id[lo], ib = id[hi];
+                    if (key_less(kb, ib, ka, ia) == up2) { km[lo] = kb; id[lo] = ib; km[hi] = ka; id[hi] = ia; }
+                }
+                __syncthreads();
+            }
+            if (act) { k0 = km[2 * t]; k1 = km[2 * t + 1]; i0 = id[2 * t]; i1 = id[2 * t + 1]; }
+        }
+        if (act) {
+            for (; stride >= 2; stride >>= 1) {           // partner thread t ^ (stride / 2), same warp
+                const uint32_t d = stride >> 1;
+                const unsigned long long pk0 = __shfl_xor_sync(0xFFFFFFFFu, k0, d), pk1 = __shfl_xor_sync(0xFFFFFFFFu, k1, d);
+                const uint32_t pi0 = __shfl_xor_sync(0xFFFFFFFFu, i0, d), pi1 = __shfl_xor_sync(0xFFFFFFFFu, i1, d);
+                const bool keep_min = ((t & d) == 0) == up;
+                cx_keep(k0, i0, pk0, pi0, keep_min);
+                cx_keep(k1, i1, pk1, pi1, keep_min);
+            }
+            if (key_less(k1, i1, k0, i0) == up) {         // distance 1: this thread's own pair
+                const unsigned long long tk = k0; k0 = k1; k1 = tk;
+                const uint32_t ti = i0; i0 = i1; i1 = ti;
+            }
+        }
+    }
+    __syncthreads();
+    if (act) { km[2 * t] = k0; km[2 * t + 1] = k1; id[2 * t] = i0; id[2 * t + 1] = i1; }
+    __syncthreads();
+}
