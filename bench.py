@@ -219,6 +219,9 @@ class StepWorkload:
         if self.done_o[b] is not None:
             main.wait_event(self.done_o[b])
             main.wait_event(self.done_p[b])
+        nxt = (s + 1) % self.RING                 # prefetch of step s-2 reads dst[b] as its destination list
+        if self.done_p[nxt] is not None:
+            main.wait_event(self.done_p[nxt])
         now = self.now0 + s
         st = (600 + s) % (self.n_steps - 1)
         lo, hi = int(self.tr.step_off[st]), int(self.tr.step_off[st + 1])
