@@ -217,6 +217,15 @@ int cs_get_model(cs_ctx *ctx, uint32_t *C_out, float *P_out, uint16_t *amax_out,
                  float *fsurv_out, float *R_out, uint16_t *cur_out, uint16_t *last_agent_out,
                  cs_stream_t stream);
 
+/* Checkpoint / resume.  The learner's state is the counts, the per-chain current agents and the last
+ * agent; cs_get_model() exports them (C_out, cur_out, last_agent_out) and this call restores them into
+ * a context created with the same n_agents / n_chains, then refreshes everything derived from the
+ * counts exactly as cs_observe_invocations() does.  C_in: dev [A*A] (the diagonal is ignored: self
+ * transitions are never counted); cur_in: dev [n_chains] or NULL (= no current agent on any chain);
+ * last_agent: CS_AGENT_NONE or an agent id. */
+int cs_import_state(cs_ctx *ctx, const uint32_t *C_in, const uint16_t *cur_in, uint32_t last_agent,
+                    cs_stream_t stream);
+
 /* Synchronises `stream`, returns the device status word in *device_status and clears it.
  * Returns CS_EDEVICE_STATUS when it was non-zero. */
 int cs_get_status(cs_ctx *ctx, uint32_t *device_status, cs_stream_t stream);
@@ -224,8 +233,10 @@ int cs_get_status(cs_ctx *ctx, uint32_t *device_status, cs_stream_t stream);
 /* Number of kernels this context has launched so far (host counter). */
 int cs_launch_count(cs_ctx *ctx, uint64_t *n_launches);
 
-/* Grid sizes of the mover (0 keeps the default): CTAs used for transfers that cross the
- * host link, and for device-to-device moves. */
+/* Width of the mover (0 keeps the default): for transfers that cross the host link and for
+ * device-to-device moves.  Unit: warp pipelines on the bulk path (each keeps up to two loads and two
+ * stores of 16 KiB in flight; defaults 8 offload / 24 prefetch / 2 per SM device-to-device), CTAs of
+ * 256 threads on the load/store path.  Narrow host-link transfers disturb other kernels less. */
 int cs_set_mover_ctas(cs_ctx *ctx, uint32_t host_link_ctas, uint32_t d2d_ctas);
 
 /* Data path of the mover: CS_MOVER_AUTO (= bulk), CS_MOVER_LDST (128-bit loads and stores by

@@ -32,7 +32,7 @@ EXPORTS = ("cs_workspace_bytes", "cs_create", "cs_destroy", "cs_observe_invocati
            "cs_select_victims", "cs_select_prefetch", "cs_offload_blocks", "cs_prefetch_blocks",
            "cs_compact_blocks", "cs_get_model", "cs_get_status", "cs_launch_count", "cs_set_mover_ctas",
            "cs_last_cuda_error", "cs_strerror", "cs_version", "cs_select_victims_static", "cs_set_mover_path", "cs_set_select_path",
-           "cs_exact_survival", "cs_use_survival_table")
+           "cs_exact_survival", "cs_use_survival_table", "cs_import_state")
 
 
 class cs_params(C.Structure):
@@ -95,6 +95,7 @@ def lib():
         L.cs_set_select_path.argtypes = [vp, u32]
         L.cs_exact_survival.argtypes = [vp, u32, u32, vp, vp, vp]
         L.cs_use_survival_table.argtypes = [vp, vp]
+        L.cs_import_state.argtypes = [vp, vp, vp, u32, vp]
         _lib = L
     return _lib
 
@@ -218,6 +219,10 @@ def cs_set_mover_path(ctx, path: int):
 def cs_exact_survival(ctx, a0: int, n_steps: int, psurv_out, fsurv_out, stream=None):
     _chk(lib().cs_exact_survival(ctx, a0, n_steps, _ptr(psurv_out), _ptr(fsurv_out), _stream(stream)),
          "cs_exact_survival", ctx)
+
+
+def cs_import_state(ctx, C_in, cur_in, last_agent: int, stream=None):
+    _chk(lib().cs_import_state(ctx, _ptr(C_in), _ptr(cur_in), last_agent, _stream(stream)), "cs_import_state", ctx)
 
 
 def cs_use_survival_table(ctx, fsurv):
@@ -398,6 +403,10 @@ class CacheScout:
         fs = torch.empty(A, dtype=torch.float32, device=self.device)
         cs_exact_survival(self.ctx, a0, n_steps, ps, fs, stream)
         return ps, fs
+
+    def import_state(self, C, cur, last_agent: int, stream=None):
+        """Restores the learner state exported by get_model() (device tensors: counts [A*A] u32, cur [n_chains] u16)."""
+        cs_import_state(self.ctx, C, cur, int(last_agent), stream)
 
     def use_survival_table(self, fsurv):
         self._fsurv_keepalive = fsurv

@@ -274,6 +274,12 @@ int cs_get_model(cs_ctx *ctx, uint32_t *C_out, float *P_out, uint16_t *amax_out,
     return CS_OK;
 }
 
+int cs_import_state(cs_ctx *ctx, const uint32_t *C_in, const uint16_t *cur_in, uint32_t last_agent, cs_stream_t stream)
+{
+    if (!ctx || !C_in || (((uintptr_t)C_in) & 3u) || (((uintptr_t)cur_in) & 1u)) return CS_EINVAL;
+    return cs_launch_import(ctx, C_in, cur_in, last_agent, (cudaStream_t)stream);
+}
+
 int cs_get_status(cs_ctx *ctx, uint32_t *device_status, cs_stream_t stream)
 {
     if (!ctx || !device_status) return CS_EINVAL;

@@ -97,6 +97,7 @@ void cs_recency_table_shape(const cs_params *p, uint32_t *gtab_len, uint32_t *ag
 int cs_launch_init(cs_ctx *ctx, cudaStream_t s);
 int cs_launch_observe(cs_ctx *ctx, const uint32_t *chain, const uint16_t *agent, const uint8_t *evflags,
                       uint32_t n_events, cudaStream_t s);
+int cs_launch_import(cs_ctx *ctx, const uint32_t *C_in, const uint16_t *cur_in, uint32_t last_agent, cudaStream_t s);
 int cs_launch_survival(cs_ctx *ctx, const uint16_t *sources, uint32_t n_sources, cudaStream_t s);
 int cs_launch_exact_survival(cs_ctx *ctx, uint32_t a0, uint32_t K, float *psurv_out, float *fsurv_out, cudaStream_t s);
 int cs_launch_score(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, const float *fsurv,

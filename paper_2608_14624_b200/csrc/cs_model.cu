@@ -363,6 +363,51 @@ int cs_launch_exact_survival(cs_ctx *ctx, uint32_t a0, uint32_t K, float *psurv_
 }
 
 // ---------------------------------------------------------------------------------------------
+// Restores learner state saved with cs_get_model(): counts, per-chain current agents, last agent.
+// Row sums and the transition total are recomputed from the counts (one CTA per row; integer
+// atomics, so the total does not depend on arrival order).
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(ROW_THREADS)
+cs_import_kernel(cs_workspace ws, uint32_t A, uint32_t n_chains, const uint32_t *__restrict__ C_in,
+                 const uint16_t *__restrict__ cur_in, uint32_t last_agent)
+{
+    __shared__ uint32_t s_red[ROW_THREADS];
+    const uint32_t tid = threadIdx.x;
+    if (blockIdx.x == 0) {
+        if (tid == 0) { ws.sc->last_agent = last_agent < A ? last_agent : CS_AGENT_NONE; }
+        for (uint32_t c = tid; c < n_chains; c += ROW_THREADS) {
+            const uint32_t a = cur_in ? cur_in[c] : CS_AGENT_NONE;
+            ws.cur[c] = (uint16_t)(a < A ? a : CS_AGENT_NONE);
+        }
+    }
+    for (uint32_t i = blockIdx.x; i < A; i += gridDim.x) {
+        uint32_t part = 0;
+        for (uint32_t j = tid; j < A; j += ROW_THREADS) {
+            const uint32_t v = (i == j) ? 0u : C_in[i * A + j];      // a self transition is never counted
+            ws.C[i * A + j] = v;
+            part += v;
+        }
+        const uint32_t n_i = cs_block_sum<uint32_t>(part, s_red);
+        if (tid == 0) {
+            ws.rowsum[i] = n_i;
+            atomicAdd(&ws.sc->n_transitions, n_i);
+        }
+    }
+}
+
+int cs_launch_import(cs_ctx *ctx, const uint32_t *C_in, const uint16_t *cur_in, uint32_t last_agent, cudaStream_t s)
+{
+    const cs_params &p = ctx->p;
+    cudaError_t e = cudaMemsetAsync(&ctx->ws.sc->n_transitions, 0, sizeof(uint32_t), s);
+    if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; return CS_ECUDA; }
+    const uint32_t grid = p.n_agents < 2u * (uint32_t)ctx->sm_count ? p.n_agents : 2u * (uint32_t)ctx->sm_count;
+    cs_import_kernel<<<grid, ROW_THREADS, 0, s>>>(ctx->ws, p.n_agents, p.n_chains, C_in, cur_in, last_agent);
+    int rc = cs_check_launch(ctx);
+    if (rc != CS_OK) return rc;
+    return cs_launch_observe(ctx, nullptr, nullptr, nullptr, 0, s);      // refresh everything derived from the counts
+}
+
+// ---------------------------------------------------------------------------------------------
 int cs_launch_init(cs_ctx *ctx, cudaStream_t s)
 {
     const cs_params &p = ctx->p;

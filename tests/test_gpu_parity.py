@@ -436,3 +436,23 @@ def test_maximum_agent_count():
     ps, _ = c.exact_survival(3)
     want = o.exact_survival(3)
     assert np.all(np.abs(ps.cpu().numpy() - want) <= H.REL_TOL * np.maximum(want, 1e-3))
+
+
+def test_checkpoint_and_resume_of_the_learner():
+    cfg = synth.CONFIGS["llama70b"]
+    tr = synth.make_trace(cfg, n_invocations=4000, warmup_frac=0.05)
+    c1, o = make_ctx(cfg, 64)
+    c1.observe_invocations(dev(tr.chain[:2500]), dev(tr.agent[:2500]), dev(tr.evflags[:2500]))
+    o.observe(tr.chain[:2500], tr.agent[:2500], tr.evflags[:2500])
+    m = c1.get_model()
+    c2, _ = make_ctx(cfg, 64)
+    c2.import_state(dev(m["C"].astype(np.uint32).ravel()), dev(m["cur"]), m["last_agent"])
+    H.compare_model(c2, o)                                     # restored state = the oracle's after the same events
+    for c in (c1, c2):
+        c.observe_invocations(dev(tr.chain[2500:]), dev(tr.agent[2500:]), dev(tr.evflags[2500:]))
+    o.observe(tr.chain[2500:], tr.agent[2500:], tr.evflags[2500:])
+    H.compare_model(c1, o)
+    H.compare_model(c2, o)
+    c3, o3 = make_ctx(cfg, 64)
+    c3.import_state(dev(np.zeros(cfg.n_agents ** 2, np.uint32)), None, cs.CS_AGENT_NONE)
+    H.compare_model(c3, o3)                                    # importing nothing is the initial state
