@@ -11,6 +11,8 @@
 
 #define CS_SELECT_CLUSTER_MAX_BLOCKS (1u << 18)   // above this the index is scanned by the whole grid instead
 
+#define CS_AGE_LIMIT_MIN_BLOCKS (1u << 21)        // index size from which the collect pass builds age limits
+
 #define CS_MOVE_D2D 0
 #define CS_MOVE_OFFLOAD 1
 #define CS_MOVE_PREFETCH 2
@@ -36,7 +38,7 @@ struct cs_scalars {
     uint32_t sel_b_last;    // last bucket that holds one of the k winners
     uint32_t sel_p_end;     // end position of that bucket
     uint32_t sel_n_out;     // min(k, eligible)
-    uint32_t pad_;
+    uint32_t gtab_monotone; // the recency table covers every unsaturated age and never increases with age
     unsigned long long t_phase[8];   // globaltimer stamps of the last cluster select (phase boundaries, ns)
 };
 
@@ -84,6 +86,7 @@ struct cs_ctx {
     const float *fsurv_override;   // caller's survival table for score / select, NULL = the BFS table of Eq. 8
     int cluster_max_v, cluster_max_pf;   // largest usable cluster of the single-launch select (0 = not probed, -1 = none)
     int bulk_attr_set;     // shared-memory opt-in of the bulk kernel done on this device
+    int collect_attr_set;  // same for the collect kernel with age limits
     uint64_t n_launches;
     int last_cuda_error;
 };

@@ -29,6 +29,22 @@ __global__ void cs_init_kernel(cs_workspace ws, uint32_t A, uint32_t n_chains, u
     }
 }
 
+// The recency factor must not increase with age for the select's age-limit prefilter to be exact.
+// exp() is monotone mathematically; this checks the table that was actually produced.
+__global__ void cs_gtab_check_kernel(cs_workspace ws, uint32_t gtab_len, uint32_t age_sat, float lambda, float delta)
+{
+    __shared__ int s_bad;
+    if (threadIdx.x == 0) s_bad = (gtab_len != age_sat) ? 1 : 0;
+    __syncthreads();
+    const float g_sat = cs_recency(lambda, delta, age_sat);
+    for (uint32_t i = threadIdx.x; i < gtab_len; i += blockDim.x) {
+        const float next = (i + 1 < gtab_len) ? ws.gtab[i + 1] : g_sat;
+        if (next > ws.gtab[i]) s_bad = 1;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) ws.sc->gtab_monotone = s_bad ? 0u : 1u;
+}
+
 // ---------------------------------------------------------------------------------------------
 // Transition counting over one batch of events, one CTA.  The update is sequential per chain
 // (each event's predecessor is the previous non-warmup event of the same chain, in this batch
@@ -414,6 +430,8 @@ int cs_launch_init(cs_ctx *ctx, cudaStream_t s)
     cs_init_kernel<<<64, 256, 0, s>>>(ctx->ws, p.n_agents, p.n_chains, ctx->gtab_len, p.lambda, p.delta);
     int rc = cs_check_launch(ctx);
     if (rc != CS_OK) return rc;
+    cs_gtab_check_kernel<<<1, 256, 0, s>>>(ctx->ws, ctx->gtab_len, ctx->age_sat, p.lambda, p.delta);
+    if ((rc = cs_check_launch(ctx)) != CS_OK) return rc;
     return cs_launch_observe(ctx, nullptr, nullptr, nullptr, 0, s);
 }
 

@@ -135,6 +135,46 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_hist_kernel(SelArgs a, cs_
 // ---------------------------------------------------------------------------------------------
 // 2 collect (+ splitters)
 // ---------------------------------------------------------------------------------------------
+// Age limits.  For a fixed agent and block size the score never increases with age (the recency
+// table is checked to be monotone, IEEE multiplication is), so "first digit <= b0" is an interval
+// of ages: victims  age >= lim (low scores are old blocks), prefetch  age + 1 <= lim (high scores
+// are young blocks).  One limit per (agent, size) found by binary search lets the scan of a large
+// index decide with one table look-up per entry; the full key is computed for candidates only.
+#define AGE_LIM_MAX 8192u
+#define AGE_CLAMP 0xFFFFFFFEu
+
+template <bool PF>
+__device__ __forceinline__ uint32_t age_limit_of(const SelArgs &a, const Tables &T, uint32_t agent, uint32_t tok,
+                                                 uint32_t b0)
+{
+    const uint32_t n_age = a.age_sat;                        // ages >= age_sat all score like age_sat
+    if (!PF) {
+        // candidate <=> score bits < lim_bits, i.e. (bits [<< 1 | copy bit]) >> 20 <= b0
+        const unsigned long long lim_bits = (unsigned long long)(b0 + 1u) << (a.prefer_copy ? 19 : 20);
+        uint32_t lo = 0, hi = n_age + 1;                      // first age with bits < lim_bits; n_age + 1 = none
+        while (lo < hi) {
+            const uint32_t mid = (lo + hi) >> 1;
+            const unsigned long long bits = __float_as_uint(score_from_age(a, T, agent, mid, tok));
+            if (bits < lim_bits) hi = mid;
+            else lo = mid + 1;
+        }
+        return lo > n_age ? 0xFFFFFFFFu : lo;                 // 0xFFFFFFFF: no age qualifies (ages are clamped below it)
+    } else {
+        const bool star = agent == T.a_star;
+        if (!star && b0 < 2048u) return 0u;                   // the whole non-a* class lies above the threshold bin
+        if (star && b0 >= 2048u) return 0xFFFFFFFFu;          // every a* entry is a candidate
+        const uint32_t x = star ? b0 : b0 - 2048u;            // (~bits & 0x7FFFFFFF) >> 20 <= x  <=>  bits >= lim_bits
+        const uint32_t lim_bits = (0x7FFu - x) << 20;
+        uint32_t lo = 0, hi = n_age + 1;                      // first age with bits < lim_bits
+        while (lo < hi) {
+            const uint32_t mid = (lo + hi) >> 1;
+            if (__float_as_uint(score_from_age(a, T, agent, mid, tok)) < lim_bits) hi = mid;
+            else lo = mid + 1;
+        }
+        return lo > n_age ? 0xFFFFFFFFu : lo;                 // candidate <=> age + 1 <= lo  (lo = 0: none)
+    }
+}
+
 template <bool PF>
 __global__ void __launch_bounds__(SEL_THREADS) cs_sel_collect_kernel(SelArgs a, cs_workspace ws)
 {
@@ -147,6 +187,16 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_collect_kernel(SelArgs a, 
     __syncthreads();
     const uint32_t b0 = ws.sc->sel_b0;
     const uint32_t lane = threadIdx.x & 31;
+    const uint32_t n_cls = a.ntok ? a.block_tokens : 1u;     // size classes: tok = 1 .. block_tokens (or the constant)
+    const bool limits = a.use_age_limits && ws.sc->gtab_monotone && b0 != 0xFFFFFFFFu;
+    uint32_t *s_lim = (uint32_t *)(smem + a.A + a.gtab_len) + (a.A + 1) / 2;      // after the tables (and the anchor table)
+    if (limits) {
+        for (uint32_t e = threadIdx.x; e < a.A * n_cls; e += blockDim.x) {
+            const uint32_t agent = e / n_cls, tok = a.ntok ? (e - agent * n_cls) + 1u : a.block_tokens;
+            s_lim[e] = age_limit_of<PF>(a, T, agent, tok, b0);
+        }
+        __syncthreads();
+    }
     if (b0 != 0xFFFFFFFFu && (!PF || prefetch_enabled(ws, a.A))) {
         // Whole groups: count this thread's candidates, reserve a range with one atomic per warp,
         // then write.  The loop bound is rounded up so that whole warps stay in the shuffles.
@@ -166,9 +216,19 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_collect_kernel(SelArgs a, 
                     uint32_t se;
                     const uint32_t tok = a.ntok ? grp_u8(G.tk, j) : a.block_tokens;
                     const uint32_t dp = (PF && a.anchor) ? grp_u16(G.dp0, G.dp1, j) : 0u;
+                    const uint32_t ag = grp_u16(G.ag0, G.ag1, j);
+                    if (limits && ag < a.A && tok - 1u < n_cls) {
+                        // prefilter: one look-up; exact, so the key is only needed when the entry is written
+                        const uint32_t la = grp_u32(G, j);
+                        uint32_t age = la <= a.now ? a.now - la : 0u;
+                        age = age < AGE_CLAMP ? age : AGE_CLAMP;
+                        const uint32_t lim = s_lim[ag * n_cls + (a.ntok ? tok - 1u : 0u)];
+                        const bool in = PF ? (age + 1u <= lim) : (age >= lim);
+                        if (in && !(PF && a.anchor && !(dp < T.anchor[ag]))) mask |= 1u << j;
+                        continue;
+                    }
                     uint32_t prj;
-                    if (entry_key_rest<PF>(a, T, &ws.sc->status, grp_u16(G.ag0, G.ag1, j), dp, grp_u8(G.fl, j), grp_u32(G, j), tok,
-                                           prj, se) &&
+                    if (entry_key_rest<PF>(a, T, &ws.sc->status, ag, dp, grp_u8(G.fl, j), grp_u32(G, j), tok, prj, se) &&
                         (prj >> 20) <= b0)
                         mask |= 1u << j;
                 }
@@ -191,9 +251,12 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_collect_kernel(SelArgs a, 
                     uint32_t prj, se;
                     const uint32_t tok = a.ntok ? grp_u8(G.tk, j) : a.block_tokens;
                     const uint32_t dp = (PF && a.anchor) ? grp_u16(G.dp0, G.dp1, j) : 0u;
-                    entry_key_rest<PF>(a, T, &ws.sc->status, grp_u16(G.ag0, G.ag1, j), dp, grp_u8(G.fl, j), grp_u32(G, j), tok, prj, se);
-                    ws.cand_km[pos] = ((unsigned long long)prj << 32) | se;
-                    ws.cand_id[pos] = grp_id(t, lane, j);
+                    const bool ok = entry_key_rest<PF>(a, T, &ws.sc->status, grp_u16(G.ag0, G.ag1, j), dp, grp_u8(G.fl, j),
+                                                       grp_u32(G, j), tok, prj, se) && (prj >> 20) <= b0;
+                    // (a slot was reserved from the prefilter's verdict; should the exact key ever disagree,
+                    //  the slot gets a key that sorts behind every real candidate and is never emitted)
+                    ws.cand_km[pos] = ok ? (((unsigned long long)prj << 32) | se) : ~0ull;
+                    ws.cand_id[pos] = ok ? grp_id(t, lane, j) : CS_ID_NONE;
                     ++pos;
                 }
             }
@@ -426,12 +489,13 @@ static void fill_args(const cs_ctx *ctx, const cs_block_index *idx, uint32_t now
     a.tier = 0;
     a.k = 0;
     a.prefer_copy = ctx->p.prefer_other_copy ? 1u : 0u;
+    a.use_age_limits = 0;
 }
 
-static uint32_t scan_grid(const cs_ctx *ctx, uint32_t n, uint32_t per_cta)
+static uint32_t scan_grid(const cs_ctx *ctx, uint32_t n, uint32_t per_cta, uint32_t ctas_per_sm = 2)
 {
     uint32_t g = (n + per_cta - 1) / per_cta;
-    const uint32_t cap = 2u * (uint32_t)ctx->sm_count;
+    const uint32_t cap = ctas_per_sm * (uint32_t)ctx->sm_count;
     if (g > cap) g = cap;
     return g ? g : 1u;
 }
@@ -467,11 +531,26 @@ int cs_launch_select(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, int p
     const uint32_t grid_c = scan_grid(ctx, idx->n_blocks, 256);
     const size_t sm = table_smem(ctx);
     int rc;
-    if (prefetch) cs_sel_hist_kernel<true><<<grid, SEL_THREADS, sm, s>>>(a, ctx->ws);
-    else cs_sel_hist_kernel<false><<<grid, SEL_THREADS, sm, s>>>(a, ctx->ws);
+    const uint32_t grid_h = grid;
+    if (prefetch) cs_sel_hist_kernel<true><<<grid_h, SEL_THREADS, sm, s>>>(a, ctx->ws);
+    else cs_sel_hist_kernel<false><<<grid_h, SEL_THREADS, sm, s>>>(a, ctx->ws);
     if ((rc = cs_check_launch(ctx)) != CS_OK) return rc;
-    if (prefetch) cs_sel_collect_kernel<true><<<grid, SEL_THREADS, sm, s>>>(a, ctx->ws);
-    else cs_sel_collect_kernel<false><<<grid, SEL_THREADS, sm, s>>>(a, ctx->ws);
+    // large indexes: the collect pass prefilters by age limits (one look-up per entry instead of the full key)
+    const uint32_t n_cls = idx->n_tokens ? ctx->p.block_tokens : 1u;
+    size_t sm_collect = sm;
+    if (idx->n_blocks >= CS_AGE_LIMIT_MIN_BLOCKS && (size_t)ctx->p.n_agents * n_cls <= AGE_LIM_MAX) {
+        a.use_age_limits = 1;
+        sm_collect += (size_t)ctx->p.n_agents * n_cls * sizeof(uint32_t);
+        if (!ctx->collect_attr_set) {
+            cudaError_t e = cudaFuncSetAttribute(cs_sel_collect_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
+            if (e == cudaSuccess)
+                e = cudaFuncSetAttribute(cs_sel_collect_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
+            if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; return CS_ECUDA; }
+            ctx->collect_attr_set = 1;
+        }
+    }
+    if (prefetch) cs_sel_collect_kernel<true><<<grid, SEL_THREADS, sm_collect, s>>>(a, ctx->ws);
+    else cs_sel_collect_kernel<false><<<grid, SEL_THREADS, sm_collect, s>>>(a, ctx->ws);
     if ((rc = cs_check_launch(ctx)) != CS_OK) return rc;
     cs_sel_bucket_kernel<<<grid_c, 256, 0, s>>>(ctx->ws);
     if ((rc = cs_check_launch(ctx)) != CS_OK) return rc;

@@ -18,6 +18,7 @@ struct SelArgs {
     uint32_t n, now, A, block_tokens, gtab_len, age_sat;
     float lambda, delta;
     uint32_t tier, k, prefer_copy;
+    uint32_t use_age_limits;      // collect pass may prefilter by per-(agent, size) age limits (large indexes)
 };
 
 // Per-CTA copies of the small tables every entry looks up.
@@ -42,6 +43,16 @@ __device__ __forceinline__ void load_tables(const SelArgs &a, const cs_workspace
     T.g_sat = cs_recency(a.lambda, a.delta, a.age_sat);
     const uint32_t la = ws.sc->last_agent;
     T.a_star = (la < a.A) ? ws.amax[la] : 0xFFFFFFFFu;
+}
+
+__device__ __forceinline__ float score_from_age(const SelArgs &a, const Tables &T, uint32_t agent, uint32_t age,
+                                                uint32_t tok)
+{
+    float g;
+    if (age < a.gtab_len) g = T.gtab[age];
+    else if (age >= a.age_sat) g = T.g_sat;
+    else g = cs_recency(a.lambda, a.delta, age);
+    return __fmul_rn(__fmul_rn(T.fsurv[agent], g), (float)tok);      // two roundings, never an FMA
 }
 
 __device__ __forceinline__ float score_of(const SelArgs &a, const Tables &T, uint32_t agent, uint32_t la,

@@ -456,3 +456,27 @@ def test_checkpoint_and_resume_of_the_learner():
     c3, o3 = make_ctx(cfg, 64)
     c3.import_state(dev(np.zeros(cfg.n_agents ** 2, np.uint32)), None, cs.CS_AGENT_NONE)
     H.compare_model(c3, o3)                                    # importing nothing is the initial state
+
+
+@pytest.mark.parametrize("with_tokens,prefer", [(True, 0), (False, 0), (True, 1)])
+def test_select_large_index_uses_age_limits(with_tokens, prefer):
+    """Above 2^21 entries the collect pass decides by per-(agent, size) age limits; the lists must
+    still equal the full sort, including sizes outside the table (0 and > block_tokens)."""
+    cfg = synth.CONFIGS["meta1m"]
+    n = (1 << 21) + 100_037
+    c, o = warm_state(cfg, 3000, n, r_min=0.02, prefer_other_copy=prefer)
+    idx = synth.make_block_index(cfg, n=n, tier="random", with_tokens=with_tokens)
+    if with_tokens:
+        idx.n_tokens[::1001] = 0
+        idx.n_tokens[7::1003] = 200
+    d = cs.DeviceIndex.from_host(idx, DEV)
+    s64, s32 = o.scores(idx, 100_000)
+    for k, tier in ((10_000, 0), (333, 1)):
+        ids, n_out = c.select_victims(d, 100_000, tier, k)
+        o_ids, o_n = o.select_victims(idx, 100_000, tier, k, s32)
+        assert H.assert_list_matches(ids.cpu().numpy().view(np.uint32)[:k], int(n_out.item()), o_ids, o_n, s64) == 0
+    ids, n_out = c.select_prefetch(d, 100_000, 2000)
+    o_ids, o_n = o.select_prefetch(idx, 100_000, 2000, s32)
+    assert o_n == 2000
+    assert H.assert_list_matches(ids.cpu().numpy().view(np.uint32)[:2000], int(n_out.item()), o_ids, o_n, s64) == 0
+    assert c.get_status() == 0
