@@ -1,15 +1,18 @@
 // Block scoring (Eq. 9 / ScoreBlock of Algorithm 1) and exact, ordered top-k selection of
 // eviction victims (Evict of Algorithm 1) and prefetch candidates (BetweenStep, Eq. 10-11).
 //
-// Every kernel that walks the block index reads the SoA metadata with 128-bit loads, 16
-// entries per thread and iteration, and never materialises the score in the select path.
+// Every kernel that walks the block index reads the SoA metadata in 512-entry warp tiles
+// (contiguous 128-, 64- and 32-bit loads; 16 entries per thread and iteration) and the select
+// path never materialises the score.
 // A positive fp32 score orders like its bit pattern, so each eligible entry has a 96-bit
 // integer key (primary, secondary, id) and "the k best in order" is "the k smallest keys in
 // ascending order":
 //   victims : primary = score bits,                      secondary = last_access
 //   prefetch: primary = (not a*)<<31 | ~score bits[30:0], secondary = ~last_access
 //
-// Selection in five launches, none of which waits on another CTA:
+// This file holds the multi-launch path, used for indexes above 262,144 entries (smaller ones take
+// the single-launch cluster kernel of cs_select_cluster.cu).  Five launches, none of which waits
+// on another CTA:
 //   1 histogram : 4096-bin histogram of the top 12 primary bits; the last CTA to finish finds
 //                 the threshold bin b0 (first bin whose running count reaches k).
 //   2 collect   : every eligible entry whose bin <= b0 is appended to the candidate buffer
@@ -19,10 +22,10 @@
 //                 takes a slot in it; the last CTA prefix-sums the bucket sizes and finds the
 //                 last bucket that can hold one of the k winners.
 //   4 scatter   : candidates of the needed buckets are grouped by bucket.
-//   5 rank      : each grouped candidate counts the smaller keys of its bucket; bucket offset
-//                 + that count is its exact rank, i.e. its position in the output list.
-// Keys are unique (the id is part of the key), so ranks are a permutation and the output does
-// not depend on the order in which atomics were served.
+//   5 rank      : every needed bucket is sorted by one CTA in a shared-memory tile; bucket offset
+//                 + position in the bucket is the position in the output list.
+// Keys are unique (the id is part of the key), so the order is total and the output does not
+// depend on the order in which atomics were served.
 #include "cs_common.cuh"
 
 #include "cs_select_common.cuh"
