@@ -602,6 +602,7 @@ static __device__ __align__(256) unsigned char cs_static_scratch[CS_STATIC_BYTES
 static std::mutex g_static_mu;
 static unsigned char *g_static_ptr[CS_STATIC_MAX_DEVICES];     // device address of the array, per device
 static int g_static_sms[CS_STATIC_MAX_DEVICES];
+static int g_static_cluster[CS_STATIC_MAX_DEVICES];   // largest usable select cluster on the device (0 = not probed yet)
 
 // Everything the select kernels expect to find zeroed, and the recency table for this call's
 // lambda / delta.  The array keeps the previous call's contents, so this runs on every call.
@@ -657,6 +658,7 @@ extern "C" int cs_select_victims_static(const cs_params *p, const float *fsurv, 
     cs_recency_table_shape(p, &ctx.gtab_len, &ctx.age_sat);
     ctx.device = dev;
     ctx.sm_count = g_static_sms[dev];
+    ctx.cluster_max_v = g_static_cluster[dev];         // probed once per device, not once per call
     cs_workspace &ws = ctx.ws;
     ws.sc = (cs_scalars *)(base + CS_SO_SC);
     ws.gtab = (float *)(base + CS_SO_GTAB);
@@ -675,5 +677,7 @@ extern "C" int cs_select_victims_static(const cs_params *p, const float *fsurv, 
     cudaStream_t s = (cudaStream_t)stream;
     cs_static_prepare_kernel<<<16, 256, 0, s>>>(ws, ctx.gtab_len, p->lambda, p->delta);
     if ((rc = cs_check_launch(&ctx)) != CS_OK) return rc;
-    return cs_launch_select(&ctx, idx, now, 0, tier, k, ids_out, n_out, s);
+    rc = cs_launch_select(&ctx, idx, now, 0, tier, k, ids_out, n_out, s);
+    g_static_cluster[dev] = ctx.cluster_max_v;
+    return rc;
 }

@@ -108,7 +108,7 @@ def test_score_parity(name, n, with_tokens):
     assert np.array_equal(s, s32)
     # explicit sources (multi-source BFS), used for that call only
     src = np.array([0, cfg.n_agents - 1], np.uint16)
-    s_b = c.score_blocks(d, 100_000, sources=dev(np.concatenate([src, np.zeros(6, np.uint16)]))[:2]).cpu().numpy()
+    s_b = c.score_blocks(d, 100_000, sources=dev(src)).cpu().numpy()
     o.survival(src)
     s64b, s32b = o.scores(idx, 100_000)
     o.survival()
