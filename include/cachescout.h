@@ -271,6 +271,12 @@ int cs_use_survival_table(cs_ctx *ctx, const float *fsurv);
 #define CS_SELECT_MULTI 2u
 int cs_set_select_path(cs_ctx *ctx, uint32_t path);
 
+/* The multi-launch select remembers the threshold bin each kind of call (GPU victims, host victims,
+ * prefetch) ended with, and the next call of that kind collects candidates up to that bin while it
+ * builds its histogram; when the new threshold is not above the remembered one the index is read
+ * once instead of twice.  The result never depends on it.  enabled = 0 turns the speculation off. */
+int cs_set_select_speculation(cs_ctx *ctx, uint32_t enabled);
+
 /* cudaError_t of the last failing CUDA call on this context (0 if none). */
 int cs_last_cuda_error(cs_ctx *ctx);
 const char *cs_strerror(int code);

@@ -32,7 +32,7 @@ EXPORTS = ("cs_workspace_bytes", "cs_create", "cs_destroy", "cs_observe_invocati
            "cs_select_victims", "cs_select_prefetch", "cs_offload_blocks", "cs_prefetch_blocks",
            "cs_compact_blocks", "cs_get_model", "cs_get_status", "cs_launch_count", "cs_set_mover_ctas",
            "cs_last_cuda_error", "cs_strerror", "cs_version", "cs_select_victims_static", "cs_set_mover_path", "cs_set_select_path",
-           "cs_exact_survival", "cs_use_survival_table", "cs_import_state")
+           "cs_exact_survival", "cs_use_survival_table", "cs_import_state", "cs_set_select_speculation")
 
 
 class cs_params(C.Structure):
@@ -93,6 +93,7 @@ def lib():
         L.cs_last_cuda_error.argtypes = [vp]
         L.cs_set_mover_path.argtypes = [vp, u32]
         L.cs_set_select_path.argtypes = [vp, u32]
+        L.cs_set_select_speculation.argtypes = [vp, u32]
         L.cs_exact_survival.argtypes = [vp, u32, u32, vp, vp, vp]
         L.cs_use_survival_table.argtypes = [vp, vp]
         L.cs_import_state.argtypes = [vp, vp, vp, u32, vp]
@@ -227,6 +228,10 @@ def cs_import_state(ctx, C_in, cur_in, last_agent: int, stream=None):
 
 def cs_use_survival_table(ctx, fsurv):
     _chk(lib().cs_use_survival_table(ctx, _ptr(fsurv)), "cs_use_survival_table", ctx)
+
+
+def cs_set_select_speculation(ctx, enabled: bool):
+    _chk(lib().cs_set_select_speculation(ctx, 1 if enabled else 0), "cs_set_select_speculation")
 
 
 def cs_set_select_path(ctx, path: int):
@@ -411,6 +416,9 @@ class CacheScout:
     def use_survival_table(self, fsurv):
         self._fsurv_keepalive = fsurv
         cs_use_survival_table(self.ctx, fsurv)
+
+    def set_select_speculation(self, enabled: bool):
+        cs_set_select_speculation(self.ctx, enabled)
 
     def set_select_path(self, path: int):
         cs_set_select_path(self.ctx, path)

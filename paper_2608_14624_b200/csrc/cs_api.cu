@@ -340,6 +340,13 @@ int cs_set_select_path(cs_ctx *ctx, uint32_t path)
     return CS_OK;
 }
 
+int cs_set_select_speculation(cs_ctx *ctx, uint32_t enabled)
+{
+    if (!ctx) return CS_EINVAL;
+    ctx->no_speculation = enabled ? 0u : 1u;
+    return CS_OK;
+}
+
 int cs_last_cuda_error(cs_ctx *ctx) { return ctx ? ctx->last_cuda_error : 0; }
 
 } // extern "C"

@@ -39,6 +39,10 @@ struct cs_scalars {
     uint32_t sel_p_end;     // end position of that bucket
     uint32_t sel_n_out;     // min(k, eligible)
     uint32_t gtab_monotone; // the recency table covers every unsaturated age and never increases with age
+    uint32_t sel_hint[4];   // threshold bin of the previous select (GPU victims, host victims, prefetch); ~0 = none;
+                            // slot 3 is never written: calls that must not speculate read it
+    uint32_t sel_c_spec;    // candidates appended speculatively by the histogram pass; 0 between calls
+    uint32_t sel_spec;      // 1: the speculative candidates cover the k winners, the collect pass is skipped
     unsigned long long t_phase[8];   // globaltimer stamps of the last cluster select (phase boundaries, ns)
 };
 
@@ -83,6 +87,7 @@ struct cs_ctx {
     uint32_t host_link_ctas, d2d_ctas;
     uint32_t mover_path;   // CS_MOVER_*
     uint32_t select_path;  // CS_SELECT_*
+    uint32_t no_speculation;       // 1: the histogram pass never collects ahead of the threshold
     const float *fsurv_override;   // caller's survival table for score / select, NULL = the BFS table of Eq. 8
     int cluster_max_v, cluster_max_pf;   // largest usable cluster of the single-launch select (0 = not probed, -1 = none)
     int bulk_attr_set;     // shared-memory opt-in of the bulk kernel done on this device

@@ -25,6 +25,7 @@ __global__ void cs_init_kernel(cs_workspace ws, uint32_t A, uint32_t n_chains, u
         cs_scalars z;
         memset(&z, 0, sizeof(z));
         z.last_agent = CS_AGENT_NONE;
+        z.sel_hint[0] = z.sel_hint[1] = z.sel_hint[2] = z.sel_hint[3] = 0xFFFFFFFFu;
         *ws.sc = z;
     }
 }

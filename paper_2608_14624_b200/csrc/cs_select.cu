@@ -67,28 +67,131 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_score_kernel(SelArgs a, cs_wor
 }
 
 // ---------------------------------------------------------------------------------------------
-// 1 histogram
+// Sample sort set-up, run by one CTA once every candidate is in the buffer: sort <= 1024 sampled
+// keys in shared memory, publish <= 255 splitters, clear the bucket counters.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void publish_splitters(const cs_workspace &ws, unsigned long long *s_km, uint32_t *s_id,
+                                                  uint32_t c)
+{
+    const uint32_t n_samp = c < CS_SAMPLE ? c : CS_SAMPLE;
+    for (uint32_t i = threadIdx.x; i < CS_SAMPLE; i += blockDim.x) {
+        if (i < n_samp) {
+            const uint32_t pos = (uint32_t)(((unsigned long long)i * c) / n_samp);
+            s_km[i] = __ldcg(&ws.cand_km[pos]);
+            s_id[i] = __ldcg(&ws.cand_id[pos]);
+        } else {
+            s_km[i] = ~0ull;
+            s_id[i] = 0xFFFFFFFFu;
+        }
+    }
+    __syncthreads();
+    bitonic_sort_fast(s_km, s_id, CS_SAMPLE);            // 512 threads, two keys each
+    uint32_t n_spl = c / 64;
+    if (n_spl > CS_MAX_SPLITTERS) n_spl = CS_MAX_SPLITTERS;
+    for (uint32_t j = threadIdx.x; j <= CS_MAX_SPLITTERS; j += blockDim.x) {
+        if (j < n_spl) {
+            const uint32_t q = (uint32_t)(((unsigned long long)(j + 1) * n_samp) / (n_spl + 1));
+            ws.spl_km[j] = s_km[q];
+            ws.spl_id[j] = s_id[q];
+        }
+        ws.bcount[j] = 0;
+    }
+    if (threadIdx.x == 0) ws.sc->sel_n_spl = n_spl;
+}
+
+// ---------------------------------------------------------------------------------------------
+// 1 histogram (+ speculative collect)
+//
+// The threshold bin moves little from one call to the next, so the pass that builds the histogram
+// also appends, speculatively, every entry at or below the bin the previous call of the same kind
+// ended with.  The last CTA finds the true threshold from the exact histogram; if it is not above
+// the remembered one, the candidates are already complete and the collect pass has nothing to do.
+// Otherwise the speculative candidates are dropped and the collect pass runs as usual.  Either
+// way the result is exact: the remembered bin only decides how many times the index is read.
 // ---------------------------------------------------------------------------------------------
 template <bool PF>
 __global__ void __launch_bounds__(SEL_THREADS) cs_sel_hist_kernel(SelArgs a, cs_workspace ws)
 {
     extern __shared__ float smem[];
-    __shared__ uint32_t s_hist[CS_HIST_BINS];
+    __shared__ __align__(16) uint32_t s_hist[CS_HIST_BINS];
     __shared__ uint32_t s_part[SEL_THREADS];
+    __shared__ uint32_t s_b0;
     __shared__ bool s_flag;
     Tables T;
     load_tables(a, ws, smem, T, PF && a.anchor);
     for (uint32_t i = threadIdx.x; i < CS_HIST_BINS; i += blockDim.x) s_hist[i] = 0;
     __syncthreads();
+    const uint32_t hint = ws.sc->sel_hint[a.hint_slot];     // ~0: nothing remembered, no speculation
+    const uint32_t lane = threadIdx.x & 31;
     if (!PF || prefetch_enabled(ws, a.A)) {
-        uint32_t run_bin = 0xFFFFFFFFu, run_cnt = 0;          // adjacent entries often share a bin
-        for_each_eligible<PF>(a, T, &ws.sc->status, [&](uint32_t, uint32_t pr, uint32_t) {
-            const uint32_t bin = pr >> 20;
+        const uint32_t gtid = blockIdx.x * blockDim.x + threadIdx.x, nth = gridDim.x * blockDim.x;
+        const uint32_t n_tiles = a.n / TILE, n_warps = nth >> 5;
+        const uint32_t n_iter = (n_tiles + n_warps - 1) / n_warps;     // whole warps stay in the shuffles
+        uint32_t run_bin = 0xFFFFFFFFu, run_cnt = 0;                    // adjacent entries often share a bin
+        auto add = [&](uint32_t bin) {
             if (bin == run_bin) { ++run_cnt; return; }
             if (run_cnt) atomicAdd(&s_hist[run_bin], run_cnt);
             run_bin = bin;
             run_cnt = 1;
-        });
+        };
+        for (uint32_t it = 0; it < n_iter; ++it) {
+            const uint32_t t = it * n_warps + (gtid >> 5);
+            uint32_t mask = 0;
+            Group G;
+            if (t < n_tiles) {
+                load_group<PF>(a, t, lane, G);
+                const uint32_t em = group_elig<PF>(a, G);
+#pragma unroll
+                for (int j = 0; j < GRP; ++j) {
+                    if (!((em >> j) & 1u)) continue;
+                    uint32_t pr, se;
+                    const uint32_t tok = a.ntok ? grp_u8(G.tk, j) : a.block_tokens;
+                    const uint32_t dp = (PF && a.anchor) ? grp_u16(G.dp0, G.dp1, j) : 0u;
+                    if (entry_key_rest<PF>(a, T, &ws.sc->status, grp_u16(G.ag0, G.ag1, j), dp, grp_u8(G.fl, j), grp_u32(G, j), tok, pr, se)) {
+                        add(pr >> 20);
+                        if (hint != 0xFFFFFFFFu && (pr >> 20) <= hint) mask |= 1u << j;
+                    }
+                }
+            }
+            if (hint == 0xFFFFFFFFu || !__any_sync(0xFFFFFFFFu, mask != 0)) continue;
+            const uint32_t cnt = __popc(mask);
+            uint32_t incl = cnt;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+                if (lane >= d) incl += v;
+            }
+            uint32_t base = 0;
+            if (lane == 31 && incl) base = atomicAdd(&ws.sc->sel_c_spec, incl);
+            base = __shfl_sync(0xFFFFFFFFu, base, 31);
+            uint32_t pos = base + incl - cnt;
+#pragma unroll
+            for (int j = 0; j < GRP; ++j) {
+                if (mask & (1u << j)) {                       // the key again, for the few that are written
+                    uint32_t pr, se;
+                    const uint32_t tok = a.ntok ? grp_u8(G.tk, j) : a.block_tokens;
+                    const uint32_t dp = (PF && a.anchor) ? grp_u16(G.dp0, G.dp1, j) : 0u;
+                    entry_key_rest<PF>(a, T, &ws.sc->status, grp_u16(G.ag0, G.ag1, j), dp, grp_u8(G.fl, j), grp_u32(G, j), tok, pr, se);
+                    ws.cand_km[pos] = ((unsigned long long)pr << 32) | se;
+                    ws.cand_id[pos] = grp_id(t, lane, j);
+                    ++pos;
+                }
+            }
+        }
+        const uint32_t t0 = n_tiles * TILE;
+        if (gtid < a.n - t0) {
+            const uint32_t i = t0 + gtid;
+            uint32_t pr, se;
+            const uint32_t tok = a.ntok ? a.ntok[i] : a.block_tokens;
+            if (entry_key<PF>(a, T, &ws.sc->status, a.agent[i], a.depth[i], a.ref[i], a.flags[i], a.la[i], tok, pr, se)) {
+                add(pr >> 20);
+                if (hint != 0xFFFFFFFFu && (pr >> 20) <= hint) {
+                    const uint32_t pos = atomicAdd(&ws.sc->sel_c_spec, 1u);
+                    ws.cand_km[pos] = ((unsigned long long)pr << 32) | se;
+                    ws.cand_id[pos] = i;
+                }
+            }
+        }
         if (run_cnt) atomicAdd(&s_hist[run_bin], run_cnt);
     }
     __syncthreads();
@@ -108,6 +211,7 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_hist_kernel(SelArgs a, cs_
         sum += loc[q];
     }
     s_part[threadIdx.x] = sum;
+    if (threadIdx.x == 0) s_b0 = (a.k == 0) ? 0xFFFFFFFFu : CS_HIST_BINS - 1;   // k = 0: nothing; k > eligible: everything
     __syncthreads();
     for (uint32_t d = 1; d < SEL_THREADS; d <<= 1) {         // inclusive scan
         const uint32_t v = threadIdx.x >= d ? s_part[threadIdx.x - d] : 0;
@@ -117,20 +221,28 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_hist_kernel(SelArgs a, cs_
     }
     const uint32_t total = s_part[SEL_THREADS - 1];
     const uint32_t before = s_part[threadIdx.x] - sum;
-    if (total < a.k || a.k == 0) {
-        if (threadIdx.x == 0) ws.sc->sel_b0 = (a.k == 0) ? 0xFFFFFFFFu : CS_HIST_BINS - 1;   // k = 0: collect nothing
-    } else if (before < a.k && a.k <= before + sum) {
+    if (a.k && total >= a.k && before < a.k && a.k <= before + sum) {
         uint32_t run = before;
 #pragma unroll
         for (uint32_t q = 0; q < PER; ++q) {
             run += loc[q];
-            if (run >= a.k) { ws.sc->sel_b0 = threadIdx.x * PER + q; break; }
+            if (run >= a.k) { s_b0 = threadIdx.x * PER + q; break; }
         }
     }
+    __syncthreads();
+    const uint32_t b0 = s_b0;
+    const bool spec_ok = hint != 0xFFFFFFFFu && b0 != 0xFFFFFFFFu && b0 <= hint;
+    const uint32_t c_spec = __ldcg(&ws.sc->sel_c_spec);
+    if (spec_ok)                                             // the shared histogram is free now: it holds the sample
+        publish_splitters(ws, (unsigned long long *)s_hist, s_hist + 2 * CS_SAMPLE, c_spec);
     if (threadIdx.x == 0) {
+        ws.sc->sel_b0 = b0;
         ws.sc->sel_n_elig = total;
         ws.sc->sel_n_out = total < a.k ? total : a.k;
-        ws.sc->sel_c = 0;
+        ws.sc->sel_c = spec_ok ? c_spec : 0;
+        ws.sc->sel_c_spec = 0;
+        ws.sc->sel_spec = spec_ok ? 1u : 0u;
+        if (a.hint_slot < 3) ws.sc->sel_hint[a.hint_slot] = (a.k && total >= a.k) ? b0 : 0xFFFFFFFFu;
         ws.sc->ticket[1] = 0;
     }
 }
@@ -185,6 +297,7 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_collect_kernel(SelArgs a, 
     __shared__ unsigned long long s_km[CS_SAMPLE];
     __shared__ uint32_t s_id[CS_SAMPLE];
     __shared__ bool s_flag;
+    if (ws.sc->sel_spec) return;          // the histogram pass already collected the candidates
     Tables T;
     load_tables(a, ws, smem, T, PF && a.anchor);
     __syncthreads();
@@ -280,34 +393,8 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_collect_kernel(SelArgs a, 
     if (!last_cta_done(&ws.sc->ticket[2], &s_flag)) return;
 
     // ---- last CTA: sample, sort the sample (bitonic, shared memory), publish splitters -----------
-    const uint32_t c = __ldcg(&ws.sc->sel_c);
-    const uint32_t n_samp = c < CS_SAMPLE ? c : CS_SAMPLE;
-    for (uint32_t i = threadIdx.x; i < CS_SAMPLE; i += blockDim.x) {
-        if (i < n_samp) {
-            const uint32_t pos = (uint32_t)(((unsigned long long)i * c) / n_samp);
-            s_km[i] = __ldcg(&ws.cand_km[pos]);
-            s_id[i] = __ldcg(&ws.cand_id[pos]);
-        } else {
-            s_km[i] = ~0ull;
-            s_id[i] = 0xFFFFFFFFu;
-        }
-    }
-    __syncthreads();
-    bitonic_sort_fast(s_km, s_id, CS_SAMPLE);            // 512 threads, two keys each
-    uint32_t n_spl = c / 64;
-    if (n_spl > CS_MAX_SPLITTERS) n_spl = CS_MAX_SPLITTERS;
-    for (uint32_t j = threadIdx.x; j <= CS_MAX_SPLITTERS; j += blockDim.x) {
-        if (j < n_spl) {
-            const uint32_t q = (uint32_t)(((unsigned long long)(j + 1) * n_samp) / (n_spl + 1));
-            ws.spl_km[j] = s_km[q];
-            ws.spl_id[j] = s_id[q];
-        }
-        ws.bcount[j] = 0;
-    }
-    if (threadIdx.x == 0) {
-        ws.sc->sel_n_spl = n_spl;
-        ws.sc->ticket[2] = 0;
-    }
+    publish_splitters(ws, s_km, s_id, __ldcg(&ws.sc->sel_c));
+    if (threadIdx.x == 0) ws.sc->ticket[2] = 0;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -493,6 +580,7 @@ static void fill_args(const cs_ctx *ctx, const cs_block_index *idx, uint32_t now
     a.k = 0;
     a.prefer_copy = ctx->p.prefer_other_copy ? 1u : 0u;
     a.use_age_limits = 0;
+    a.hint_slot = 0;
 }
 
 static uint32_t scan_grid(const cs_ctx *ctx, uint32_t n, uint32_t per_cta, uint32_t ctas_per_sm = 2)
@@ -526,6 +614,7 @@ int cs_launch_select(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, int p
     fill_args(ctx, idx, now, ctx->fsurv_override ? ctx->fsurv_override : ctx->ws.fsurv, a);
     a.tier = tier;
     a.k = k;
+    a.hint_slot = ctx->no_speculation ? 3u : (prefetch ? 2u : tier);
     if (ctx->select_path != CS_SELECT_MULTI && idx->n_blocks <= CS_SELECT_CLUSTER_MAX_BLOCKS) {
         const int rc1 = cs_launch_select_cluster(ctx, &a, prefetch, ids_out, n_out, s);
         if (rc1 != CS_ENOTIMPL) return rc1;          // no usable cluster on this device: fall through
@@ -616,6 +705,7 @@ __global__ void cs_static_prepare_kernel(cs_workspace ws, uint32_t gtab_len, flo
         cs_scalars z;
         memset(&z, 0, sizeof(z));
         z.last_agent = CS_AGENT_NONE;
+        z.sel_hint[0] = z.sel_hint[1] = z.sel_hint[2] = z.sel_hint[3] = 0xFFFFFFFFu;
         *ws.sc = z;
     }
 }

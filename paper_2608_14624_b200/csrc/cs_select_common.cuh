@@ -19,6 +19,7 @@ struct SelArgs {
     float lambda, delta;
     uint32_t tier, k, prefer_copy;
     uint32_t use_age_limits;      // collect pass may prefilter by per-(agent, size) age limits (large indexes)
+    uint32_t hint_slot;           // which remembered threshold bin this call may speculate on
 };
 
 // Per-CTA copies of the small tables every entry looks up.

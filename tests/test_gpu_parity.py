@@ -134,8 +134,9 @@ def run_selects(c, o, idx, now, ks, tiers=(0, 1)):
     d = cs.DeviceIndex.from_host(idx, DEV)
     s64, s32 = o.scores(idx, now)
     tolerated = 0
-    for path, k in [(p_, k_) for p_ in (cs.CS_SELECT_CLUSTER, cs.CS_SELECT_MULTI) for k_ in ks]:
-        c.set_select_path(path)
+    for path, k in [(p_, k_) for p_ in (cs.CS_SELECT_CLUSTER, cs.CS_SELECT_MULTI, -1) for k_ in ks]:
+        c.set_select_path(cs.CS_SELECT_MULTI if path == -1 else path)
+        c.set_select_speculation(path != -1)          # -1: multi-launch path without the remembered threshold
         for tier in tiers:
             ids, n_out = c.select_victims(d, now, tier, k)
             ids2, n_out2 = c.select_victims(d, now, tier, k)           # determinism: identical on a second run
