@@ -43,6 +43,8 @@ struct cs_scalars {
                             // slot 3 is never written: calls that must not speculate read it
     uint32_t sel_c_spec;    // candidates appended speculatively by the histogram pass; 0 between calls
     uint32_t sel_spec;      // 1: the speculative candidates cover the k winners, the collect pass is skipped
+    uint32_t sel_cc[2];     // candidate counters of the cluster kernel: a call uses one and clears the other for
+                            // the next call, so that the counter is zero on entry without a barrier
     unsigned long long t_phase[8];   // globaltimer stamps of the last cluster select (phase boundaries, ns)
 };
 
@@ -87,6 +89,7 @@ struct cs_ctx {
     uint32_t host_link_ctas, d2d_ctas;
     uint32_t mover_path;   // CS_MOVER_*
     uint32_t select_path;  // CS_SELECT_*
+    uint32_t cluster_slot;         // which of the two candidate counters the next cluster select uses
     uint32_t no_speculation;       // 1: the histogram pass never collects ahead of the threshold
     const float *fsurv_override;   // caller's survival table for score / select, NULL = the BFS table of Eq. 8
     int cluster_max_v, cluster_max_pf;   // largest usable cluster of the single-launch select (0 = not probed, -1 = none)

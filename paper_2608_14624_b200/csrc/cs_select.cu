@@ -581,6 +581,7 @@ static void fill_args(const cs_ctx *ctx, const cs_block_index *idx, uint32_t now
     a.prefer_copy = ctx->p.prefer_other_copy ? 1u : 0u;
     a.use_age_limits = 0;
     a.hint_slot = 0;
+    a.c_slot = 0;
 }
 
 static uint32_t scan_grid(const cs_ctx *ctx, uint32_t n, uint32_t per_cta, uint32_t ctas_per_sm = 2)

@@ -129,7 +129,8 @@ cs_select_cluster_kernel(SelArgs a, cs_workspace ws, uint32_t *__restrict__ ids_
     Tables T;
     load_tables(a, ws, S.tables, T, PF && a.anchor);
     for (uint32_t i = tid; i < CS_HIST_BINS; i += CSEL_THREADS) S.hist[i] = 0;
-    if (rank == 0 && tid == 0) ws.sc->sel_c = 0;
+    uint32_t *cand_count = &ws.sc->sel_cc[a.c_slot];          // zero on entry: the previous call cleared it
+    if (rank == 0 && tid == 0) ws.sc->sel_cc[a.c_slot ^ 1u] = 0;
     if (tid == 0) S.misc[1] = 0;
     __syncthreads();
     const bool enabled = !PF || prefetch_enabled(ws, a.A);
@@ -138,37 +139,83 @@ cs_select_cluster_kernel(SelArgs a, cs_workspace ws, uint32_t *__restrict__ ids_
     const uint32_t cthreads = CL * CSEL_THREADS, ctid = rank * CSEL_THREADS + tid;   // cluster-wide thread id
     const uint32_t t0 = n_tiles * TILE;                                              // start of the ragged tail
 
-    // ---- phase 1: histogram of this CTA's slice ------------------------------------------------
-    if (enabled) {
-        uint32_t run_bin = 0xFFFFFFFFu, run_cnt = 0;          // adjacent entries often share a bin
-        auto add = [&](uint32_t pr) {
-            const uint32_t bin = pr >> 20;
-            if (bin == run_bin) { ++run_cnt; return; }
-            if (run_cnt) atomicAdd(&S.hist[run_bin], run_cnt);
-            run_bin = bin;
-            run_cnt = 1;
-        };
-        for (uint32_t t = ctid >> 5; t < n_tiles; t += cthreads >> 5) {
+    // One routine serves both scans: per warp tile it computes the keys of the eligible entries, feeds
+    // the histogram (first scan) and appends the entries whose first digit is <= `limit` to the
+    // candidate buffer (warp-aggregated reservation, keys recomputed for the few that are written).
+    uint32_t run_bin = 0xFFFFFFFFu, run_cnt = 0;              // adjacent entries often share a bin
+    auto hist_add = [&](uint32_t pr) {
+        const uint32_t bin = pr >> 20;
+        if (bin == run_bin) { ++run_cnt; return; }
+        if (run_cnt) atomicAdd(&S.hist[run_bin], run_cnt);
+        run_bin = bin;
+        run_cnt = 1;
+    };
+    auto scan = [&](bool do_hist, bool do_collect, uint32_t limit) {
+        const uint32_t n_warps = cthreads >> 5;
+        const uint32_t n_iter = (n_tiles + n_warps - 1) / n_warps;       // whole warps stay in the shuffles
+        for (uint32_t it = 0; it < n_iter; ++it) {
+            const uint32_t t = it * n_warps + (ctid >> 5);
+            uint32_t mask = 0;
             Group G;
-            load_group<PF>(a, t, lane, G);
-            const uint32_t em = group_elig<PF>(a, G);
+            if (t < n_tiles) {
+                load_group<PF>(a, t, lane, G);
+                const uint32_t em = group_elig<PF>(a, G);
+#pragma unroll
+                for (int j = 0; j < GRP; ++j) {
+                    if (!((em >> j) & 1u)) continue;
+                    uint32_t pr, se;
+                    const uint32_t tok = a.ntok ? grp_u8(G.tk, j) : a.block_tokens;
+                    const uint32_t dp = (PF && a.anchor) ? grp_u16(G.dp0, G.dp1, j) : 0u;
+                    if (entry_key_rest<PF>(a, T, &ws.sc->status, grp_u16(G.ag0, G.ag1, j), dp, grp_u8(G.fl, j), grp_u32(G, j), tok, pr, se)) {
+                        if (do_hist) hist_add(pr);
+                        if (do_collect && (pr >> 20) <= limit) mask |= 1u << j;
+                    }
+                }
+            }
+            if (!do_collect || !__any_sync(0xFFFFFFFFu, mask != 0)) continue;      // most warps hold no candidate at all
+            const uint32_t cnt = __popc(mask);
+            uint32_t incl = cnt;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+                if (lane >= d) incl += v;
+            }
+            uint32_t base = 0;
+            if (lane == 31 && incl) base = atomicAdd(cand_count, incl);
+            base = __shfl_sync(0xFFFFFFFFu, base, 31);
+            uint32_t pos = base + incl - cnt;
 #pragma unroll
             for (int j = 0; j < GRP; ++j) {
-                if (!((em >> j) & 1u)) continue;
-                uint32_t pr, se;
-                const uint32_t tok = a.ntok ? grp_u8(G.tk, j) : a.block_tokens;
-                const uint32_t dp = (PF && a.anchor) ? grp_u16(G.dp0, G.dp1, j) : 0u;
-                if (entry_key_rest<PF>(a, T, &ws.sc->status, grp_u16(G.ag0, G.ag1, j), dp, grp_u8(G.fl, j), grp_u32(G, j), tok, pr, se))
-                    add(pr);
+                if (mask & (1u << j)) {
+                    uint32_t prj, se;
+                    const uint32_t tok = a.ntok ? grp_u8(G.tk, j) : a.block_tokens;
+                    const uint32_t dp = (PF && a.anchor) ? grp_u16(G.dp0, G.dp1, j) : 0u;
+                    entry_key_rest<PF>(a, T, &ws.sc->status, grp_u16(G.ag0, G.ag1, j), dp, grp_u8(G.fl, j), grp_u32(G, j), tok, prj, se);
+                    ws.cand_km[pos] = ((unsigned long long)prj << 32) | se;
+                    ws.cand_id[pos] = grp_id(t, lane, j);
+                    ++pos;
+                }
             }
         }
-        if (ctid < a.n - t0) {
+        if (ctid < a.n - t0) {                                 // ragged tail, one entry per thread
             const uint32_t i = t0 + ctid;
-            uint32_t pr, se;
+            uint32_t p, se;
             const uint32_t tok = a.ntok ? a.ntok[i] : a.block_tokens;
-            if (entry_key<PF>(a, T, &ws.sc->status, a.agent[i], a.depth[i], a.ref[i], a.flags[i], a.la[i], tok, pr, se))
-                add(pr);
+            if (entry_key<PF>(a, T, &ws.sc->status, a.agent[i], a.depth[i], a.ref[i], a.flags[i], a.la[i], tok, p, se)) {
+                if (do_hist) hist_add(p);
+                if (do_collect && (p >> 20) <= limit) {
+                    const uint32_t pos = atomicAdd(cand_count, 1u);
+                    ws.cand_km[pos] = ((unsigned long long)p << 32) | se;
+                    ws.cand_id[pos] = i;
+                }
+            }
         }
+    };
+
+    // ---- phase 1: histogram of this CTA's slice, and candidates up to the remembered threshold bin -----
+    const uint32_t hint = ws.sc->sel_hint[a.hint_slot];       // ~0: nothing remembered
+    if (enabled) {
+        scan(true, hint != 0xFFFFFFFFu, hint);
         if (run_cnt) atomicAdd(&S.hist[run_bin], run_cnt);
     }
     __threadfence();
@@ -210,70 +257,21 @@ cs_select_cluster_kernel(SelArgs a, cs_workspace ws, uint32_t *__restrict__ ids_
     if (ctid == 0) *n_out_dev = n_out;
 
     csel_stamp(ws, rank, 2);
-    // ---- phase 3: collect the candidates (bin <= b0) ------------------------------------------------------
-    if (enabled && b0 != 0xFFFFFFFFu) {
-        const uint32_t n_warps = cthreads >> 5;
-        const uint32_t n_iter = (n_tiles + n_warps - 1) / n_warps;
-        for (uint32_t it = 0; it < n_iter; ++it) {
-            const uint32_t t = it * n_warps + (ctid >> 5);
-            uint32_t mask = 0;               // keys are recomputed for the (few) candidates instead of kept in registers
-            Group G;
-            if (t < n_tiles) {
-                load_group<PF>(a, t, lane, G);
-                const uint32_t em = group_elig<PF>(a, G);
-#pragma unroll
-                for (int j = 0; j < GRP; ++j) {
-                    if (!((em >> j) & 1u)) continue;
-                    uint32_t se;
-                    const uint32_t tok = a.ntok ? grp_u8(G.tk, j) : a.block_tokens;
-                    const uint32_t dp = (PF && a.anchor) ? grp_u16(G.dp0, G.dp1, j) : 0u;
-                    uint32_t prj;
-                    if (entry_key_rest<PF>(a, T, &ws.sc->status, grp_u16(G.ag0, G.ag1, j), dp, grp_u8(G.fl, j), grp_u32(G, j), tok,
-                                           prj, se) &&
-                        (prj >> 20) <= b0)
-                        mask |= 1u << j;
-                }
-            }
-            if (!__any_sync(0xFFFFFFFFu, mask != 0)) continue;      // most warps hold no candidate at all
-            const uint32_t cnt = __popc(mask);
-            uint32_t incl = cnt;
-#pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, incl, d);
-                if (lane >= d) incl += v;
-            }
-            uint32_t base = 0;
-            if (lane == 31 && incl) base = atomicAdd(&ws.sc->sel_c, incl);
-            base = __shfl_sync(0xFFFFFFFFu, base, 31);
-            uint32_t pos = base + incl - cnt;
-#pragma unroll
-            for (int j = 0; j < GRP; ++j) {
-                if (mask & (1u << j)) {
-                    uint32_t prj, se;
-                    const uint32_t tok = a.ntok ? grp_u8(G.tk, j) : a.block_tokens;
-                    const uint32_t dp = (PF && a.anchor) ? grp_u16(G.dp0, G.dp1, j) : 0u;
-                    entry_key_rest<PF>(a, T, &ws.sc->status, grp_u16(G.ag0, G.ag1, j), dp, grp_u8(G.fl, j), grp_u32(G, j), tok, prj, se);
-                    ws.cand_km[pos] = ((unsigned long long)prj << 32) | se;
-                    ws.cand_id[pos] = grp_id(t, lane, j);
-                    ++pos;
-                }
-            }
+    // ---- phase 3: collect the candidates (bin <= b0), unless the first scan already has them ----------------
+    const bool spec_ok = hint != 0xFFFFFFFFu && b0 != 0xFFFFFFFFu && b0 <= hint;     // same verdict in every CTA
+    if (rank == 0 && tid == 0 && a.hint_slot < 3) ws.sc->sel_hint[a.hint_slot] = (a.k && n_elig >= a.k) ? b0 : 0xFFFFFFFFu;
+    if (!spec_ok) {
+        if (hint != 0xFFFFFFFFu) {                            // drop what the first scan appended
+            if (rank == 0 && tid == 0) *cand_count = 0;
+            __threadfence();
+            cluster.sync();
         }
-        if (ctid < a.n - t0) {
-            const uint32_t i = t0 + ctid;
-            uint32_t p, se;
-            const uint32_t tok = a.ntok ? a.ntok[i] : a.block_tokens;
-            if (entry_key<PF>(a, T, &ws.sc->status, a.agent[i], a.depth[i], a.ref[i], a.flags[i], a.la[i], tok, p, se) &&
-                (p >> 20) <= b0) {
-                const uint32_t pos = atomicAdd(&ws.sc->sel_c, 1u);
-                ws.cand_km[pos] = ((unsigned long long)p << 32) | se;
-                ws.cand_id[pos] = i;
-            }
-        }
+        if (enabled && b0 != 0xFFFFFFFFu) scan(false, true, b0);
+        __threadfence();
+        cluster.sync();
     }
-    __threadfence();
-    cluster.sync();
-    const uint32_t c = __ldcg(&ws.sc->sel_c);
+    const uint32_t c = __ldcg(cand_count);
+    if (rank == 0 && tid == 0) ws.sc->sel_c = c;              // for inspection only
     csel_stamp(ws, rank, 3);
 
     // ---- phase 4, small: CTA 0 sorts everything in shared memory ---------------------------------------------
@@ -422,7 +420,10 @@ static int launch_cluster(cs_ctx *ctx, const SelArgs &a, uint32_t *ids_out, uint
     while (cl < max_cl && (uint32_t)cl * CSEL_THREADS < n_groups) cl <<= 1;
     cfg.gridDim = dim3(cl);
     attr[0].val.clusterDim.x = cl;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, a, ctx->ws, ids_out, n_out);
+    SelArgs args = a;
+    args.c_slot = ctx->cluster_slot;
+    ctx->cluster_slot ^= 1u;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, args, ctx->ws, ids_out, n_out);
     ctx->n_launches++;
     if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; return CS_ECUDA; }
     return CS_OK;

@@ -20,6 +20,7 @@ struct SelArgs {
     uint32_t tier, k, prefer_copy;
     uint32_t use_age_limits;      // collect pass may prefilter by per-(agent, size) age limits (large indexes)
     uint32_t hint_slot;           // which remembered threshold bin this call may speculate on
+    uint32_t c_slot;              // candidate counter of the cluster kernel for this call
 };
 
 // Per-CTA copies of the small tables every entry looks up.
