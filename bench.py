@@ -6,7 +6,8 @@ heads x 128, bf16, 16-token blocks of 2 MiB; GPU pool 20,000 blocks, host tier 6
 agents): observe the step's agent invocations, select 256 GPU-tier victims, 256 host-tier
 victims (their slots receive the offloaded blocks) and 384 prefetch candidates, compact the
 victims into a packed device staging pool, offload them to the pinned host tier and prefetch
-the candidates into free GPU slots.  Transfers run on two side streams and overlap the next
+the candidates into free GPU slots.  The two transfers run as one fused launch on a side
+stream (or, with --transfers split, as two launches on two side streams) and overlap the next
 step's selection.  value = KV bytes moved across the host link per second over the K steps.
 
     python bench.py --gpus 1 --steps 20 --warmup 3
@@ -42,6 +43,9 @@ def parse_args():
     ap.add_argument("--no-extras", action="store_true", help="skip the mover sweep and the metadata-scale section")
     ap.add_argument("--offload-width", type=int, default=0, help="warp pipelines of the offload mover (0 = library default)")
     ap.add_argument("--prefetch-width", type=int, default=0, help="warp pipelines of the prefetch mover (0 = library default)")
+    ap.add_argument("--transfers", default="exchange", choices=["exchange", "split"],
+                    help="offload and prefetch of a step as one fused launch (exchange) or as two launches on two streams (split)")
+    ap.add_argument("--exchange-width", type=int, default=0, help="warp pipelines of the fused transfer (0 = library default)")
     ap.add_argument("--quick", action="store_true", help="small pools (debugging only; not a valid bench line)")
     ap.add_argument("--workload", default="step", choices=["step", "mover", "select", "select80k"],
                     help="'mover'/'select' run one small case of that kernel family only (profiler captures)")
@@ -203,6 +207,7 @@ class StepWorkload:
         self.done_p = [None] * self.RING
         self.now0 = 100_000
         self.w_off, self.w_pre = args.offload_width, args.prefetch_width
+        self.fused, self.w_ex = args.transfers == "exchange", args.exchange_width
         self.fifo = [torch.zeros(self.k_p, dtype=torch.int64, device=device) for _ in range(8)]
         self.fifo_used = 0
         self.bytes_per_step = (self.k_v + self.k_p) * bb
@@ -250,30 +255,48 @@ class StepWorkload:
         rec(t[3], main)
         ready = torch.cuda.Event()
         ready.record(main)
-        # offload on side stream 1: GPU victims -> the slots of the host-tier victims
-        self.side_o.wait_event(ready)
-        rec(t[4], self.side_o)
-        if self.w_off:
-            c.set_mover_ctas(self.w_off, 0)
-        c.offload_blocks(self.gpu_pool, self.host_pool, vict, self.hv[b], n_max=self.k_v, n_dev=self.vn[b],
-                         stream=self.side_o)
-        rec(t[5], self.side_o)
-        self.done_o[b] = torch.cuda.Event()
-        self.done_o[b].record(self.side_o)
-        # prefetch on side stream 2 into the slots freed one step earlier (their offload must be over)
-        self.side_p.wait_event(ready)
-        if self.done_o[prev] is not None:
-            self.side_p.wait_event(self.done_o[prev])
-        rec(t[6], self.side_p)
-        if self.w_pre:
-            c.set_mover_ctas(self.w_pre, 0)
-        c.prefetch_blocks(self.host_pool, self.gpu_pool, self.pf[b], self.dst[prev], n_max=self.k_p, n_dev=self.pn[b],
-                          stream=self.side_p)
-        if self.w_off or self.w_pre:
-            c.set_mover_ctas(0, 0)
-        rec(t[7], self.side_p)
-        self.done_p[b] = torch.cuda.Event()
-        self.done_p[b].record(self.side_p)
+        if self.fused:
+            # one launch on side stream 1: GPU victims -> the slots of the host-tier victims, and the prefetch
+            # candidates -> the slots freed one step earlier (their offload ran in the previous launch of this stream)
+            self.side_o.wait_event(ready)
+            rec(t[4], self.side_o)
+            if self.w_ex:
+                c.set_mover_ctas(self.w_ex, 0)
+            c.exchange_blocks(self.gpu_pool, self.host_pool, vict, self.hv[b], self.pf[b], self.dst[prev],
+                              n_off_max=self.k_v, n_off_dev=self.vn[b], n_pre_max=self.k_p, n_pre_dev=self.pn[b],
+                              stream=self.side_o)
+            if self.w_ex:
+                c.set_mover_ctas(0, 0)
+            rec(t[5], self.side_o)
+            self.done_o[b] = torch.cuda.Event()
+            self.done_o[b].record(self.side_o)
+            self.done_p[b] = self.done_o[b]
+            t[6], t[7] = t[4], t[5]
+        else:
+            # offload on side stream 1: GPU victims -> the slots of the host-tier victims
+            self.side_o.wait_event(ready)
+            rec(t[4], self.side_o)
+            if self.w_off:
+                c.set_mover_ctas(self.w_off, 0)
+            c.offload_blocks(self.gpu_pool, self.host_pool, vict, self.hv[b], n_max=self.k_v, n_dev=self.vn[b],
+                             stream=self.side_o)
+            rec(t[5], self.side_o)
+            self.done_o[b] = torch.cuda.Event()
+            self.done_o[b].record(self.side_o)
+            # prefetch on side stream 2 into the slots freed one step earlier (their offload must be over)
+            self.side_p.wait_event(ready)
+            if self.done_o[prev] is not None:
+                self.side_p.wait_event(self.done_o[prev])
+            rec(t[6], self.side_p)
+            if self.w_pre:
+                c.set_mover_ctas(self.w_pre, 0)
+            c.prefetch_blocks(self.host_pool, self.gpu_pool, self.pf[b], self.dst[prev], n_max=self.k_p, n_dev=self.pn[b],
+                              stream=self.side_p)
+            if self.w_off or self.w_pre:
+                c.set_mover_ctas(0, 0)
+            rec(t[7], self.side_p)
+            self.done_p[b] = torch.cuda.Event()
+            self.done_p[b].record(self.side_p)
         # engine bookkeeping (plumbing, not the method): refilled victim slots are touched now, prefetched
         # host entries now have a GPU copy
         vi = vict.long().clamp_(min=0)
@@ -320,14 +343,16 @@ class StepWorkload:
 
 
 def host_link_peak(torch, device, n_bytes=GIB, reps=10):
-    """Pinned cudaMemcpyAsync of one contiguous buffer, each direction alone and both at once."""
+    """Pinned cudaMemcpyAsync of one contiguous buffer, each direction alone, both at once, and both at once in
+    the step's proportions (2 bytes out for every 3 bytes in: 256 blocks offloaded, 384 prefetched)."""
     h = torch.empty(n_bytes, dtype=torch.uint8, pin_memory=True)
     h2 = torch.empty(n_bytes, dtype=torch.uint8, pin_memory=True)
     d = torch.empty(n_bytes, dtype=torch.uint8, device=device)
     d2 = torch.empty(n_bytes, dtype=torch.uint8, device=device)
     s1, s2 = torch.cuda.Stream(device=device), torch.cuda.Stream(device=device)
     out = {}
-    for name in ("d2h", "h2d", "bidir"):
+    n_out = (n_bytes * 2 // 3) & ~4095
+    for name in ("d2h", "h2d", "bidir", "bidir_step_mix"):
         best = 0.0
         for _ in range(reps):
             torch.cuda.synchronize(device)
@@ -337,7 +362,10 @@ def host_link_peak(torch, device, n_bytes=GIB, reps=10):
             if name in ("d2h", "bidir"):
                 with torch.cuda.stream(s1):
                     h.copy_(d, non_blocking=True)
-            if name in ("h2d", "bidir"):
+            if name == "bidir_step_mix":
+                with torch.cuda.stream(s1):
+                    h[:n_out].copy_(d[:n_out], non_blocking=True)
+            if name in ("h2d", "bidir", "bidir_step_mix"):
                 with torch.cuda.stream(s2):
                     d2.copy_(h2, non_blocking=True)
             e2.record(s2)
@@ -345,7 +373,7 @@ def host_link_peak(torch, device, n_bytes=GIB, reps=10):
             e1.record(s1)
             torch.cuda.synchronize(device)
             ms = e0.elapsed_time(e1)
-            moved = n_bytes * (2 if name == "bidir" else 1)
+            moved = {"bidir": 2 * n_bytes, "bidir_step_mix": n_bytes + n_out}.get(name, n_bytes)
             best = max(best, moved / ms / 1e6)
         out[name] = best
     del h, h2, d, d2
@@ -757,11 +785,17 @@ def main():
                      "achieved": d2d_gbps, "peak": hbm_peak, "unit": "GB/s", "frac": d2d_gbps / hbm_peak, "traffic": traffic,
                      "peak_kind": "of %s" % peak_kind, "algorithmic_bytes_per_launch": 2 * w.k_v * bb, "ms_per_launch": t_c},
         "host_link": {"peak_d2h_GBps": link["d2h"], "peak_h2d_GBps": link["h2d"], "peak_bidir_GBps": link["bidir"],
-                      "how": "pinned cudaMemcpyAsync of 1 GiB, best of 10, same run",
+                      "peak_bidir_step_mix_GBps": link["bidir_step_mix"],
+                      "how": "pinned cudaMemcpyAsync of 1 GiB, best of 10, same run; step_mix = 2/3 GiB out while 1 GiB comes in, "
+                             "the proportions of a step, whose inbound direction is the longer one",
                       "offload_GBps": off_gbps, "offload_frac": off_gbps / link["d2h"], "offload_ms": t_o,
                       "prefetch_GBps": pre_gbps, "prefetch_frac": pre_gbps / link["h2d"], "prefetch_ms": t_p,
                       "step_frac_of_bidir": value / world / link["bidir"],
-                      "note": "offload and prefetch of a step overlap (full duplex); per-direction times are measured while the other direction is busy"},
+                      "step_frac_of_bidir_step_mix": value / world / link["bidir_step_mix"],
+                      "transfers": args.transfers,
+                      "note": ("offload and prefetch of a step run as one fused launch (cs_exchange_blocks): both per-direction times "
+                               "are that launch's duration" if w.fused else
+                               "offload and prefetch of a step overlap (full duplex); per-direction times are measured while the other direction is busy")},
         "select": {"ms_three_selects": t_s, "ms_observe": t_ob, "algorithmic_bytes": sel_bytes,
                    "achieved_GBps": sel_bytes / (t_s / 1e3) / 1e9, "frac_of_hbm_peak": sel_bytes / (t_s / 1e3) / 1e9 / hbm_peak,
                    "n_out_last_step": n_out, "device_status": status},

@@ -208,6 +208,22 @@ int cs_prefetch_blocks(cs_ctx *ctx, const cs_kv_pool *host, const cs_kv_pool *gp
 int cs_compact_blocks(cs_ctx *ctx, const cs_kv_pool *src, const cs_kv_pool *dst, const uint32_t *src_slots,
                       const uint32_t *dst_slots, uint32_t n_max, const uint32_t *n_dev, cs_stream_t stream);
 
+/* Offload and prefetch of one step in a single launch (the paper runs its evictions and prefetches
+ * through the serving engine's offload path side by side, Sec. 4; the fused launch is this library's
+ * way of keeping the two directions of the host link in step).  Equivalent to
+ *   cs_offload_blocks(ctx, gpu, host, off_gpu_slots, off_host_slots, n_off_max, n_off_dev, side) and
+ *   cs_prefetch_blocks(ctx, host, gpu, pre_host_slots, pre_gpu_slots, n_pre_max, n_pre_dev, side)
+ * when no slot is written by one transfer and read or written by the other (not checked; otherwise the
+ * order of the conflicting copies is unspecified).  Every copy pipeline walks its share of both lists
+ * interleaved in proportion to their lengths, so both transfers finish together.  All slot lists and
+ * counts: dev, as for the calls above; either list may be empty (n_*_max == 0 with NULL pointers).
+ * Always takes the bulk path; its width is the host-link width of cs_set_mover_ctas() (default 32 warp
+ * pipelines). */
+int cs_exchange_blocks(cs_ctx *ctx, const cs_kv_pool *gpu, const cs_kv_pool *host, const uint32_t *off_gpu_slots,
+                       const uint32_t *off_host_slots, uint32_t n_off_max, const uint32_t *n_off_dev,
+                       const uint32_t *pre_host_slots, const uint32_t *pre_gpu_slots, uint32_t n_pre_max,
+                       const uint32_t *n_pre_dev, cs_stream_t side);
+
 /* ---- inspection ------------------------------------------------------------------------------------ */
 
 /* Copies the learner / scorer state into caller dev buffers (any may be NULL):

@@ -32,7 +32,7 @@ EXPORTS = ("cs_workspace_bytes", "cs_create", "cs_destroy", "cs_observe_invocati
            "cs_select_victims", "cs_select_prefetch", "cs_offload_blocks", "cs_prefetch_blocks",
            "cs_compact_blocks", "cs_get_model", "cs_get_status", "cs_launch_count", "cs_set_mover_ctas",
            "cs_last_cuda_error", "cs_strerror", "cs_version", "cs_select_victims_static", "cs_set_mover_path", "cs_set_select_path",
-           "cs_exact_survival", "cs_use_survival_table", "cs_import_state", "cs_set_select_speculation")
+           "cs_exact_survival", "cs_use_survival_table", "cs_import_state", "cs_set_select_speculation", "cs_exchange_blocks")
 
 
 class cs_params(C.Structure):
@@ -86,6 +86,8 @@ def lib():
                                                vp, vp, vp]
         for name in ("cs_offload_blocks", "cs_prefetch_blocks", "cs_compact_blocks"):
             getattr(L, name).argtypes = [vp, C.POINTER(cs_kv_pool), C.POINTER(cs_kv_pool), vp, vp, u32, vp, vp]
+        L.cs_exchange_blocks.argtypes = [vp, C.POINTER(cs_kv_pool), C.POINTER(cs_kv_pool), vp, vp, u32, vp, vp, vp, u32,
+                                         vp, vp]
         L.cs_get_model.argtypes = [vp] * 10
         L.cs_get_status.argtypes = [vp, C.POINTER(u32), vp]
         L.cs_launch_count.argtypes = [vp, C.POINTER(C.c_uint64)]
@@ -182,6 +184,13 @@ def cs_offload_blocks(ctx, gpu: cs_kv_pool, host: cs_kv_pool, src_slots, dst_slo
 def cs_prefetch_blocks(ctx, host: cs_kv_pool, gpu: cs_kv_pool, src_slots, dst_slots, n_max: int, n_dev=None, stream=None):
     _chk(lib().cs_prefetch_blocks(ctx, C.byref(host), C.byref(gpu), _ptr(src_slots), _ptr(dst_slots), n_max,
                                   _ptr(n_dev), _stream(stream)), "cs_prefetch_blocks", ctx)
+
+
+def cs_exchange_blocks(ctx, gpu: cs_kv_pool, host: cs_kv_pool, off_gpu_slots, off_host_slots, n_off_max: int, n_off_dev,
+                       pre_host_slots, pre_gpu_slots, n_pre_max: int, n_pre_dev, stream=None):
+    _chk(lib().cs_exchange_blocks(ctx, C.byref(gpu), C.byref(host), _ptr(off_gpu_slots), _ptr(off_host_slots), n_off_max,
+                                  _ptr(n_off_dev), _ptr(pre_host_slots), _ptr(pre_gpu_slots), n_pre_max,
+                                  _ptr(n_pre_dev), _stream(stream)), "cs_exchange_blocks", ctx)
 
 
 def cs_compact_blocks(ctx, src: cs_kv_pool, dst: cs_kv_pool, src_slots, dst_slots, n_max: int, n_dev=None, stream=None):
@@ -365,6 +374,16 @@ class CacheScout:
     def prefetch_blocks(self, host: KVPool, gpu: KVPool, src_slots, dst_slots, n_max=None, n_dev=None, stream=None):
         cs_prefetch_blocks(self.ctx, host.struct(), gpu.struct(), src_slots, dst_slots,
                            int(src_slots.numel()) if n_max is None else n_max, n_dev, stream)
+
+    def exchange_blocks(self, gpu: KVPool, host: KVPool, off_gpu_slots, off_host_slots, pre_host_slots, pre_gpu_slots,
+                        n_off_max=None, n_off_dev=None, n_pre_max=None, n_pre_dev=None, stream=None):
+        """Offload and prefetch of one step in a single launch; either pair of lists may be None."""
+        if n_off_max is None:
+            n_off_max = 0 if off_gpu_slots is None else int(off_gpu_slots.numel())
+        if n_pre_max is None:
+            n_pre_max = 0 if pre_host_slots is None else int(pre_host_slots.numel())
+        cs_exchange_blocks(self.ctx, gpu.struct(), host.struct(), off_gpu_slots, off_host_slots, n_off_max, n_off_dev,
+                           pre_host_slots, pre_gpu_slots, n_pre_max, n_pre_dev, stream)
 
     def compact_blocks(self, src: KVPool, dst: KVPool, src_slots, dst_slots, n_max=None, n_dev=None, stream=None):
         cs_compact_blocks(self.ctx, src.struct(), dst.struct(), src_slots, dst_slots,

@@ -252,6 +252,25 @@ int cs_compact_blocks(cs_ctx *ctx, const cs_kv_pool *src, const cs_kv_pool *dst,
     return mover_common(ctx, src, dst, src_slots, dst_slots, n_max, n_dev, CS_MOVE_D2D, stream);
 }
 
+int cs_exchange_blocks(cs_ctx *ctx, const cs_kv_pool *gpu, const cs_kv_pool *host, const uint32_t *off_gpu_slots,
+                       const uint32_t *off_host_slots, uint32_t n_off_max, const uint32_t *n_off_dev,
+                       const uint32_t *pre_host_slots, const uint32_t *pre_gpu_slots, uint32_t n_pre_max,
+                       const uint32_t *n_pre_dev, cs_stream_t side)
+{
+    if (!ctx) return CS_EINVAL;
+    int rc = check_pools(gpu, host);
+    if (rc != CS_OK) return rc;
+    if (n_off_max == 0 && n_pre_max == 0) return CS_OK;
+    const uint32_t *lists[4] = {off_gpu_slots, off_host_slots, pre_host_slots, pre_gpu_slots};
+    for (int i = 0; i < 4; ++i) {
+        const uint32_t n = i < 2 ? n_off_max : n_pre_max;
+        if (n && (!lists[i] || (((uintptr_t)lists[i]) & 3u))) return CS_EINVAL;
+    }
+    if ((n_off_dev && (((uintptr_t)n_off_dev) & 3u)) || (n_pre_dev && (((uintptr_t)n_pre_dev) & 3u))) return CS_EINVAL;
+    return cs_launch_exchange(ctx, gpu, host, off_gpu_slots, off_host_slots, n_off_max, n_off_dev, pre_host_slots,
+                              pre_gpu_slots, n_pre_max, n_pre_dev, (cudaStream_t)side);
+}
+
 int cs_get_model(cs_ctx *ctx, uint32_t *C_out, float *P_out, uint16_t *amax_out, uint16_t *hops_out,
                  float *fsurv_out, float *R_out, uint16_t *cur_out, uint16_t *last_agent_out, cs_stream_t stream)
 {

@@ -121,6 +121,11 @@ int cs_launch_mover(cs_ctx *ctx, const cs_kv_pool *src, const cs_kv_pool *dst, c
                     const uint32_t *dst_slots, uint32_t n_max, const uint32_t *n_dev, int kind,
                     cudaStream_t s);
 
+int cs_launch_exchange(cs_ctx *ctx, const cs_kv_pool *gpu, const cs_kv_pool *host, const uint32_t *off_gpu_slots,
+                       const uint32_t *off_host_slots, uint32_t n_off_max, const uint32_t *n_off_dev,
+                       const uint32_t *pre_host_slots, const uint32_t *pre_gpu_slots, uint32_t n_pre_max,
+                       const uint32_t *n_pre_dev, cudaStream_t s);
+
 static inline int cs_check_launch(cs_ctx *ctx)
 {
     cudaError_t e = cudaGetLastError();

@@ -33,6 +33,7 @@
 #define TM_PIECE 16384u                              // bytes per ring slot
 #endif
 #define TM_SMEM (TM_WARPS * TM_STAGES * TM_PIECE)    // 192 KiB
+#define CS_EXCHANGE_PIPES 32u                         // default width of the two-way transfer, in warp pipelines
 #define TM_SPIN_LIMIT (1u << 20)                     // bounded mbarrier wait (polls with back-off: >= 0.1 s)
 
 struct MoverArgs {
@@ -161,32 +162,14 @@ __device__ __forceinline__ void bulk_store(void *dst, uint32_t src_smem, uint32_
 
 // One pipeline per warp, driven by lane 0.  Iteration `it` first stores item it-(STAGES-1)
 // (whose load was issued STAGES-1 iterations ago) and then issues the load of item `it` into
-// the ring slot whose previous store has finished reading shared memory.
-__global__ void __launch_bounds__(TM_WARPS * 32, 1) cs_mover_bulk_kernel(MoverArgs a)
+// the ring slot whose previous store has finished reading shared memory.  `item(it, sp, dp, bytes)`
+// resolves the pipeline's it-th item; false = nothing to copy.
+template <class Item>
+__device__ __forceinline__ void bulk_pipeline(unsigned char *my_ring, const uint32_t (&bar)[TM_STAGES],
+                                              unsigned long long n_items, uint32_t *status, Item item)
 {
-    extern __shared__ __align__(128) unsigned char ring[];
-    __shared__ __align__(8) unsigned long long bars[TM_WARPS * TM_STAGES];
-    const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    if (lane != 0) return;                                   // the other lanes have nothing to do
-    unsigned char *my_ring = ring + (size_t)warp * TM_STAGES * TM_PIECE;
-    uint32_t bar[TM_STAGES];
-#pragma unroll
-    for (int st = 0; st < TM_STAGES; ++st) {
-        bar[st] = smem_u32(&bars[warp * TM_STAGES + st]);
-        mbar_init(bar[st], 1);
-    }
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-
-    const uint32_t n = mover_count(a);
-    const uint32_t per_block = 2u * a.L * a.pieces;
-    const unsigned long long total = (unsigned long long)n * per_block;
-    const unsigned long long n_pipes = a.n_pipes;             // pipelines of the whole grid
-    const unsigned long long first = (unsigned long long)blockIdx.x * (blockDim.x >> 5) + warp;
-    if (first >= n_pipes) return;
-    const unsigned long long n_items = first < total ? (total - first + n_pipes - 1) / n_pipes : 0;
     constexpr int LAG = TM_STAGES - 1;
-
-    char *dst_of[TM_STAGES];          // destination of the item loaded into each ring slot, NULL = skipped item
+    char *dst_of[TM_STAGES];          // destination of the item loaded into each ring slot
     uint32_t bytes_of[TM_STAGES];
     uint32_t phase_bits = 0;          // parity to wait for, one bit per ring slot
     uint32_t pending = 0;             // ring slots with a load in flight that nobody has waited for yet
@@ -197,7 +180,7 @@ __global__ void __launch_bounds__(TM_WARPS * 32, 1) cs_mover_bulk_kernel(MoverAr
             if (pending & (1u << st)) {
                 if (!mbar_wait_bounded(bar[st], (phase_bits >> st) & 1u)) {
                     failed = true;
-                    atomicOr(a.status, CS_ST_TIMEOUT);
+                    atomicOr(status, CS_ST_TIMEOUT);
                     break;
                 }
                 pending &= ~(1u << st);
@@ -213,7 +196,7 @@ __global__ void __launch_bounds__(TM_WARPS * 32, 1) cs_mover_bulk_kernel(MoverAr
             const char *sp;
             char *dp;
             uint32_t bytes;
-            if (resolve_piece(a, first + it * n_pipes, per_block, sp, dp, bytes, true)) {
+            if (item(it, sp, dp, bytes)) {
                 // the slot's previous store (item it-STAGES) was committed one iteration ago, so at
                 // most the newest group may still be reading shared memory
                 asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
@@ -233,11 +216,80 @@ __global__ void __launch_bounds__(TM_WARPS * 32, 1) cs_mover_bulk_kernel(MoverAr
     asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // all stores written
 }
 
-// ---------------------------------------------------------------------------------------------
-int cs_launch_mover(cs_ctx *ctx, const cs_kv_pool *src, const cs_kv_pool *dst, const uint32_t *src_slots,
-                    const uint32_t *dst_slots, uint32_t n_max, const uint32_t *n_dev, int kind, cudaStream_t s)
+// Per-warp set-up shared by the bulk kernels: ring slice and barriers.  Returns false for the
+// lanes and warps that have nothing to do.
+__device__ __forceinline__ bool bulk_setup(unsigned char *ring, unsigned long long *bars, uint32_t n_pipes,
+                                           unsigned char *&my_ring, uint32_t (&bar)[TM_STAGES],
+                                           unsigned long long &first)
 {
-    MoverArgs a;
+    const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (lane != 0) return false;                             // the other lanes have nothing to do
+    my_ring = ring + (size_t)warp * TM_STAGES * TM_PIECE;
+#pragma unroll
+    for (int st = 0; st < TM_STAGES; ++st) {
+        bar[st] = smem_u32(&bars[warp * TM_STAGES + st]);
+        mbar_init(bar[st], 1);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    first = (unsigned long long)blockIdx.x * (blockDim.x >> 5) + warp;
+    return first < n_pipes;
+}
+
+__device__ __forceinline__ unsigned long long items_of_pipe(unsigned long long total, unsigned long long first,
+                                                            unsigned long long n_pipes)
+{
+    return first < total ? (total - first + n_pipes - 1) / n_pipes : 0;
+}
+
+// One transfer: pipeline `first` of n_pipes takes the pieces first, first + n_pipes, ...
+__global__ void __launch_bounds__(TM_WARPS * 32, 1) cs_mover_bulk_kernel(MoverArgs a)
+{
+    extern __shared__ __align__(128) unsigned char ring[];
+    __shared__ __align__(8) unsigned long long bars[TM_WARPS * TM_STAGES];
+    unsigned char *my_ring;
+    uint32_t bar[TM_STAGES];
+    unsigned long long first;
+    if (!bulk_setup(ring, bars, a.n_pipes, my_ring, bar, first)) return;
+    const uint32_t per_block = 2u * a.L * a.pieces;
+    const unsigned long long total = (unsigned long long)mover_count(a) * per_block;
+    const unsigned long long n_pipes = a.n_pipes;
+    bulk_pipeline(my_ring, bar, items_of_pipe(total, first, n_pipes), a.status,
+                  [&](unsigned long long it, const char *&sp, char *&dp, uint32_t &bytes) {
+                      return resolve_piece(a, first + it * n_pipes, per_block, sp, dp, bytes, true);
+                  });
+}
+
+// Two transfers in opposite directions over the host link in one launch.  Every pipeline takes its
+// share of both piece lists and walks them interleaved in proportion to their lengths, so the two
+// directions advance in lock step and finish together whatever the link's arbitration between reads
+// and writes would otherwise give each of them.
+__global__ void __launch_bounds__(TM_WARPS * 32, 1) cs_exchange_bulk_kernel(MoverArgs off, MoverArgs pre)
+{
+    extern __shared__ __align__(128) unsigned char ring[];
+    __shared__ __align__(8) unsigned long long bars[TM_WARPS * TM_STAGES];
+    unsigned char *my_ring;
+    uint32_t bar[TM_STAGES];
+    unsigned long long first;
+    if (!bulk_setup(ring, bars, off.n_pipes, my_ring, bar, first)) return;
+    const uint32_t per_block = 2u * off.L * off.pieces;
+    const unsigned long long n_pipes = off.n_pipes;
+    const unsigned long long n_o = items_of_pipe((unsigned long long)mover_count(off) * per_block, first, n_pipes);
+    const unsigned long long n_p = items_of_pipe((unsigned long long)mover_count(pre) * per_block, first, n_pipes);
+    const unsigned long long n_items = n_o + n_p;
+    bulk_pipeline(my_ring, bar, n_items, off.status,
+                  [&](unsigned long long it, const char *&sp, char *&dp, uint32_t &bytes) {
+                      // offload pieces among the first `it` items: floor(it * n_o / n_items)
+                      const unsigned long long before = it * n_o / n_items, after = (it + 1) * n_o / n_items;
+                      if (after != before) return resolve_piece(off, first + before * n_pipes, per_block, sp, dp, bytes, true);
+                      return resolve_piece(pre, first + (it - before) * n_pipes, per_block, sp, dp, bytes, true);
+                  });
+}
+
+// ---------------------------------------------------------------------------------------------
+static void fill_mover_args(cs_ctx *ctx, MoverArgs &a, const cs_kv_pool *src, const cs_kv_pool *dst,
+                            const uint32_t *src_slots, const uint32_t *dst_slots, uint32_t n_max, const uint32_t *n_dev,
+                            uint32_t piece_bytes)
+{
     a.src = (const char *)src->base;
     a.dst = (char *)dst->base;
     a.src_total = src->n_slots;
@@ -254,9 +306,27 @@ int cs_launch_mover(cs_ctx *ctx, const cs_kv_pool *src, const cs_kv_pool *dst, c
     a.n_max = n_max;
     a.status = &ctx->ws.sc->status;
     a.n_pipes = 0;
+    a.piece_bytes = piece_bytes;
+    a.pieces = (uint32_t)((a.chunk + piece_bytes - 1) / piece_bytes);
+}
+
+static int bulk_opt_in(cs_ctx *ctx)
+{
+    if (ctx->bulk_attr_set) return CS_OK;
+    cudaError_t e = cudaFuncSetAttribute(cs_mover_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TM_SMEM);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(cs_exchange_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TM_SMEM);
+    if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; return CS_ECUDA; }
+    ctx->bulk_attr_set = 1;
+    return CS_OK;
+}
+
+int cs_launch_mover(cs_ctx *ctx, const cs_kv_pool *src, const cs_kv_pool *dst, const uint32_t *src_slots,
+                    const uint32_t *dst_slots, uint32_t n_max, const uint32_t *n_dev, int kind, cudaStream_t s)
+{
     const bool bulk = ctx->mover_path != CS_MOVER_LDST;
-    a.piece_bytes = bulk ? TM_PIECE : MV_PIECE;
-    a.pieces = (uint32_t)((a.chunk + a.piece_bytes - 1) / a.piece_bytes);
+    MoverArgs a;
+    fill_mover_args(ctx, a, src, dst, src_slots, dst_slots, n_max, n_dev, bulk ? TM_PIECE : MV_PIECE);
     const unsigned long long total = (unsigned long long)n_max * 2ull * a.L * a.pieces;
     unsigned long long cap;
     if (bulk) {
@@ -268,11 +338,8 @@ int cs_launch_mover(cs_ctx *ctx, const cs_kv_pool *src, const cs_kv_pool *dst, c
         if (a.n_pipes == 0) a.n_pipes = 1;
         const uint32_t wpc = a.n_pipes < TM_WARPS ? a.n_pipes : TM_WARPS;
         const uint32_t grid = (a.n_pipes + wpc - 1) / wpc;
-        if (!ctx->bulk_attr_set) {
-            cudaError_t e = cudaFuncSetAttribute(cs_mover_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TM_SMEM);
-            if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; return CS_ECUDA; }
-            ctx->bulk_attr_set = 1;
-        }
+        const int rc = bulk_opt_in(ctx);
+        if (rc != CS_OK) return rc;
         cs_mover_bulk_kernel<<<grid, wpc * 32, TM_SMEM, s>>>(a);
     } else {
         const uint32_t dflt = kind == CS_MOVE_D2D ? 8u * (uint32_t)ctx->sm_count : (kind == CS_MOVE_OFFLOAD ? 8u : 12u);
@@ -281,5 +348,27 @@ int cs_launch_mover(cs_ctx *ctx, const cs_kv_pool *src, const cs_kv_pool *dst, c
         const uint32_t grid = (uint32_t)(total < cap ? total : cap);
         cs_mover_kernel<<<grid ? grid : 1u, MV_THREADS, 0, s>>>(a);
     }
+    return cs_check_launch(ctx);
+}
+
+// Offload and prefetch of one step as a single launch (bulk path only).
+int cs_launch_exchange(cs_ctx *ctx, const cs_kv_pool *gpu, const cs_kv_pool *host, const uint32_t *off_gpu_slots,
+                       const uint32_t *off_host_slots, uint32_t n_off_max, const uint32_t *n_off_dev,
+                       const uint32_t *pre_host_slots, const uint32_t *pre_gpu_slots, uint32_t n_pre_max,
+                       const uint32_t *n_pre_dev, cudaStream_t s)
+{
+    MoverArgs off, pre;
+    fill_mover_args(ctx, off, gpu, host, off_gpu_slots, off_host_slots, n_off_max, n_off_dev, TM_PIECE);
+    fill_mover_args(ctx, pre, host, gpu, pre_host_slots, pre_gpu_slots, n_pre_max, n_pre_dev, TM_PIECE);
+    const unsigned long long total = ((unsigned long long)n_off_max + n_pre_max) * 2ull * off.L * off.pieces;
+    const unsigned long long cap = ctx->host_link_ctas ? ctx->host_link_ctas : CS_EXCHANGE_PIPES;
+    uint32_t n_pipes = (uint32_t)(total < cap ? total : cap);
+    if (n_pipes == 0) n_pipes = 1;
+    off.n_pipes = pre.n_pipes = n_pipes;
+    const uint32_t wpc = n_pipes < TM_WARPS ? n_pipes : TM_WARPS;
+    const uint32_t grid = (n_pipes + wpc - 1) / wpc;
+    const int rc = bulk_opt_in(ctx);
+    if (rc != CS_OK) return rc;
+    cs_exchange_bulk_kernel<<<grid, wpc * 32, TM_SMEM, s>>>(off, pre);
     return cs_check_launch(ctx);
 }

@@ -31,12 +31,14 @@ def block_bytes_from_pool(buf_u8, layout, n_slots, L, chunk, slot):
     return buf_u8.view(n_slots, L, 2, chunk)[slot].cpu().numpy()
 
 
-def test_bench_step_at_full_size_matches_oracle():
+@pytest.mark.parametrize("transfers", ["exchange", "split"])
+def test_bench_step_at_full_size_matches_oracle(transfers):
     import bench
     free = torch.cuda.mem_get_info()[0]
     if free < 60 * (1 << 30) or bench.mem_available_bytes() < 60 * (1 << 30):
         pytest.skip("needs 60 GiB of free device and host memory")
-    args = argparse.Namespace(quick=False, host_slots=8192, offload_width=0, prefetch_width=0)
+    args = argparse.Namespace(quick=False, host_slots=8192, offload_width=0, prefetch_width=0, transfers=transfers,
+                              exchange_width=0)
     w = bench.StepWorkload(args, torch.device(DEV), 1)
     cfg, G, L, chunk = w.cfg, w.cfg.gpu_blocks, w.cfg.n_layers, w.cfg.chunk_bytes
     o = orc.Oracle(H.oracle_params(w.params))

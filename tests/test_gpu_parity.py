@@ -334,6 +334,48 @@ def test_mover_small_chunks_and_geometry_errors(path):
         cs.cs_compact_blocks(c.ctx, odd, odd, dev(s), dev(d), 1)
 
 
+@pytest.mark.parametrize("gpu_layout,host_layout", [(0, 1), (1, 0)])
+@pytest.mark.parametrize("n_off,n_pre,width", [(41, 67, 0), (50, 0, 3), (0, 33, 0), (1, 1, 64), (37, 5, 7)])
+def test_exchange_matches_offload_then_prefetch(gpu_layout, host_layout, n_off, n_pre, width):
+    """Both directions in one launch: byte-exact against the oracle's two transfers on disjoint slots,
+    for uneven list lengths, empty lists, device-resident counts and sentinels."""
+    cfg = synth.CONFIGS["tiny"]
+    L, chunk, G, Hs = cfg.n_layers, cfg.chunk_bytes, 160, 200
+    rng = synth.rng_for(cfg, 15)
+    c, _ = make_ctx(cfg, 64)
+    c.set_mover_ctas(width, 0)
+    gpu_np = synth.kv_pool_u16(G, L, chunk, rng).view(np.uint8)
+    host_np = synth.kv_pool_u16(Hs, L, chunk, rng).view(np.uint8)
+    gpu = cs.KVPool(dev(gpu_np), G, gpu_layout, L)
+    host_t = pinned_zeros(Hs * L * 2 * chunk)
+    host_t.numpy()[:] = host_np
+    host = cs.KVPool(host_t, Hs, host_layout, L)
+    g_perm = rng.permutation(G).astype(np.uint32)              # disjoint GPU slots: sources then destinations
+    h_perm = rng.permutation(Hs).astype(np.uint32)
+    off_src, pre_dst = g_perm[:n_off].copy(), g_perm[n_off:n_off + n_pre].copy()
+    off_dst, pre_src = h_perm[:n_off].copy(), h_perm[n_off:n_off + n_pre].copy()
+    m_off, m_pre = n_off, n_pre
+    if n_off > 8:
+        off_src[3] = orc.ID_NONE                                # skipped
+        m_off = n_off - 4                                       # device-resident count below n_max
+    if n_pre > 8:
+        pre_dst[2] = orc.ID_NONE
+        m_pre = n_pre - 1
+    side = torch.cuda.Stream(device=DEV)
+    side.wait_stream(torch.cuda.current_stream())
+    c.exchange_blocks(gpu, host, dev(off_src) if n_off else None, dev(off_dst) if n_off else None,
+                      dev(pre_src) if n_pre else None, dev(pre_dst) if n_pre else None,
+                      n_off_dev=dev(np.array([m_off], np.uint32)) if n_off else None,
+                      n_pre_dev=dev(np.array([m_pre], np.uint32)) if n_pre else None, stream=side)
+    side.synchronize()
+    want_h, want_g = host_np.copy(), gpu_np.copy()
+    orc.move_blocks(gpu_np, gpu_layout, G, want_h, host_layout, Hs, L, chunk, off_src[:m_off], off_dst[:m_off])
+    orc.move_blocks(host_np, host_layout, Hs, want_g, gpu_layout, G, L, chunk, pre_src[:m_pre], pre_dst[:m_pre])
+    assert np.array_equal(host_t.numpy(), want_h)
+    assert np.array_equal(gpu.buf.cpu().numpy(), want_g)
+    assert c.get_status() == 0
+
+
 def test_offload_straight_from_select_output():
     """The victim list and its device-resident count drive the mover without a host round trip."""
     cfg = synth.CONFIGS["tiny"]
