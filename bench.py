@@ -219,6 +219,7 @@ class StepWorkload:
     def step(self, s, e2e=False, timed=False):
         torch, c = self.torch, self.c
         b, prev = s % self.RING, (s - 1) % self.RING
+        self.last_s = s
         main = self.main
         # ring slot b is rewritten now: the transfers that read it (step s - RING) must be over
         if self.done_o[b] is not None:
@@ -340,6 +341,132 @@ class StepWorkload:
         h2d = self.meta_bytes + ev + self.k_p * self.cfg.block_bytes
         d2h = (2 * self.k_v + self.k_p + 3) * 4 + self.k_v * self.cfg.block_bytes
         return h2d, d2h
+
+
+def fused_step_section(w, steps=10):
+    """The whole step as ONE library call (cs_step): issued afresh every step, and captured once into a CUDA
+    graph that reads the clock and the event count from device memory and is replayed; then the interference
+    between the two-way transfer on the side stream and synthetic serving kernels on the main stream (a
+    bandwidth-bound copy standing in for decode, a bf16 GEMM standing in for prefill; both are torch's
+    kernels, they are the disturbed party, not the product).  Steps run back to back without overlap
+    (the side stream rejoins the main stream every step, as a graph capture requires)."""
+    torch, c, dev = w.torch, w.c, w.dev
+    main, side = torch.cuda.Stream(device=dev), w.side_o          # a graph cannot be captured on the default stream
+    kv, kp, bb = w.k_v, w.k_p, w.cfg.block_bytes
+    i32 = lambda n, fill=0: torch.full((max(n, 4),), fill, dtype=torch.int32, device=dev)
+    gv, gh, gp = i32(kv), i32(kv), i32(kp)
+    gvn, ghn, gpn, now_d, nev_d = i32(1), i32(1), i32(1), i32(1), i32(1)
+    free_d = w.dst[w.last_s % w.RING].clone()                  # slots freed by the last step of the main run + reserve tail
+    free_last = free_d.clone()                                 # the destination list the latest step used
+    cap = 16
+    ev_c = torch.zeros(cap, dtype=w.d_chain.dtype, device=dev)
+    ev_a = torch.zeros(cap, dtype=w.d_agent.dtype, device=dev)
+    ev_f = torch.zeros(cap, dtype=w.d_flags.dtype, device=dev)
+    fifo = [torch.zeros(kp, dtype=torch.int64, device=dev) for _ in range(8)]
+    state = {"s": w.last_s + 1, "n": 0}
+
+    def issue(by_value, now=0, n_ev=cap):
+        c.step(w.didx, now, ev_c, ev_a, ev_f, n_ev, kv, kp, gv, gvn, gh, ghn, gp, gpn, w.gpu_pool, w.host_pool, free_d,
+               stage=w.stage_pool, stage_slots=w.packed, now_dev=None if by_value else now_d,
+               n_events_dev=None if by_value else nev_d, main=main, side=side, join_main=True)
+
+    def one_step(graph):
+        s = state["s"]
+        now = w.now0 + s
+        st = (600 + s) % (w.n_steps - 1)
+        lo, hi = int(w.tr.step_off[st]), int(w.tr.step_off[st + 1])
+        n_ev = hi - lo
+        ev_c[:n_ev].copy_(w.d_chain[lo:hi]); ev_a[:n_ev].copy_(w.d_agent[lo:hi]); ev_f[:n_ev].copy_(w.d_flags[lo:hi])
+        now_d.fill_(now); nev_d.fill_(n_ev)
+        if graph is None:
+            issue(True, now, n_ev)
+        else:
+            graph.replay()
+        # engine bookkeeping, as in the main run
+        vi = gv[:kv].long().clamp_(min=0)
+        w.la_i32[vi] = now
+        pi = gp[:kp].long().clamp_(min=0)
+        w.didx.flags[pi] |= w.cs.CS_FLAG_OTHER_COPY
+        if state["n"] >= 8:
+            w.didx.flags[fifo[state["n"] % 8]] &= 0xF7
+        fifo[state["n"] % 8].copy_(pi)
+        free_last.copy_(free_d)
+        free_d[:kv].copy_(gv[:kv])
+        state["s"] += 1
+        state["n"] += 1
+
+    def timed(graph, k):
+        with torch.cuda.stream(main):
+            for _ in range(3):
+                one_step(graph)
+            main.synchronize()
+            l0 = c.launch_count()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(main)
+            for _ in range(k):
+                one_step(graph)
+            e1.record(main)
+            main.synchronize()
+        return e0.elapsed_time(e1) / k, (c.launch_count() - l0) / k
+
+    w.drain()
+    torch.cuda.synchronize(dev)
+    with torch.cuda.stream(main):                               # buffers made above belong to this stream from here on
+        pass
+    ms_call, launches_call = timed(None, steps)
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=main, capture_error_mode="relaxed"):
+        issue(False)
+    ms_graph, _ = timed(g, steps)
+    out = {"what": "cs_step: observe + 3 selects + conflict filter + compaction + two-way transfer as one call; steps back to back, no overlap between steps",
+           "ms_per_step_call": ms_call, "GBps_call": w.bytes_per_step / ms_call / 1e6, "kernel_launches_per_step": launches_call,
+           "ms_per_step_graph_replay": ms_graph, "GBps_graph_replay": w.bytes_per_step / ms_graph / 1e6,
+           "n_out_last_step": [int(gvn[0].item()), int(ghn[0].item()), int(gpn[0].item())], "device_status": c.get_status()}
+
+    # ---- interference with synthetic serving kernels ------------------------------------------------------
+    x = torch.empty(1 << 30, dtype=torch.float32, device=dev).normal_()
+    y = torch.empty_like(x)
+    a = torch.randn(8192, 8192, dtype=torch.bfloat16, device=dev)
+    b = torch.randn(8192, 8192, dtype=torch.bfloat16, device=dev)
+    o = torch.empty(8192, 8192, dtype=torch.bfloat16, device=dev)
+    loads = {"hbm_copy_8GiB_x16": (lambda: y.copy_(x), 16), "bf16_gemm_8192_x24": (lambda: torch.matmul(a, b, out=o), 24)}
+
+    def transfer():
+        c.exchange_blocks(w.gpu_pool, w.host_pool, gv, gh, gp, free_last, n_off_max=kv, n_off_dev=gvn, n_pre_max=kp,
+                          n_pre_dev=gpn, stream=side)
+
+    def run(load, with_transfer, with_load=True):
+        fn, reps = load
+        ts = []
+        for _ in range(3):
+            torch.cuda.synchronize(dev)
+            m0, m1, s0, s1 = (torch.cuda.Event(enable_timing=True) for _ in range(4))
+            m0.record(main)
+            side.wait_event(m0)
+            if with_transfer:
+                s0.record(side)
+                transfer()
+                s1.record(side)
+            with torch.cuda.stream(main):
+                if with_load:
+                    for _ in range(reps):
+                        fn()
+            m1.record(main)
+            torch.cuda.synchronize(dev)
+            ts.append((m0.elapsed_time(m1), s0.elapsed_time(s1) if with_transfer else 0.0))
+        return min(t[0] for t in ts), min(t[1] for t in ts)
+
+    _, x_alone = run(loads["hbm_copy_8GiB_x16"], True, with_load=False)
+    inter = {"transfer_alone_ms": x_alone}
+    for name, load in loads.items():
+        run(load, False)
+        alone, _ = run(load, False)
+        both, x_both = run(load, True)
+        inter[name] = {"serving_alone_ms": alone, "serving_with_transfer_ms": both, "serving_slowdown": both / alone,
+                       "transfer_with_serving_ms": x_both, "transfer_slowdown": x_both / x_alone}
+    out["interference"] = inter
+    del x, y, a, b, o
+    return out
 
 
 def host_link_peak(torch, device, n_bytes=GIB, reps=10):
@@ -468,12 +595,33 @@ def metadata_scale(torch, cs, synth, dev, hbm_peak, calls=200):
     launches = (c.launch_count() - l0) / (calls + 5)
     ms = np.array([a.elapsed_time(b) for a, b in evs])
     per_call = float(np.median(ms)) * 1e-3
+    # the same call captured once into a CUDA graph and replayed (same events and clock every time: timing only)
+    cap = torch.cuda.Stream(device=dev)
+    cap.wait_stream(stream)
+    g = torch.cuda.CUDAGraph()
+    lo = 64 * 30
+    with torch.cuda.graph(g, stream=cap, capture_error_mode="relaxed"):
+        c.observe_invocations(ch[lo:lo + 64], ag[lo:lo + 64], None, stream=cap)
+        c.select_victims(d, 100_000, 0, cfg.k_victims, v, vn, stream=cap)
+        c.select_prefetch(d, 100_000, cfg.k_prefetch, pf, pn, stream=cap)
+    gms = []
+    with torch.cuda.stream(cap):
+        for call in range(calls + 5):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(cap)
+            g.replay()
+            e1.record(cap)
+            if call >= 5:
+                gms.append((e0, e1))
+    cap.synchronize()
+    graph_us = float(np.median([a.elapsed_time(b) for a, b in gms])) * 1e3
     algo_bytes = N * (9 + 11) + (cfg.k_victims + cfg.k_prefetch) * 4        # one scan per select when the remembered
     #                                                                        threshold holds: 9 B (victims) + 11 B (prefetch) per entry
     return {"workload": "metadata-scale: 1,000,000-entry index, 256 agents, k=10000 victims + 2000 prefetch per call",
             "calls_timed": calls, "us_per_call_median": per_call * 1e6, "us_per_call_min": float(ms.min()) * 1e3,
             "blocks_scored_selected_per_s": 2 * N / per_call,
             "algorithmic_GBps": algo_bytes / per_call / 1e9, "frac_of_hbm_peak": algo_bytes / per_call / 1e9 / hbm_peak,
+            "us_per_call_graph_replay": graph_us,
             "kernel_launches_per_call": launches, "n_out": [int(vn[0].item()), int(pn[0].item())]}
 
 
@@ -602,7 +750,8 @@ def run_reference(args):
 def profile_case(args, torch, device):
     """Small cases for profiler captures (a few GB on the device, inputs larger than L2).
     mover : 2,048-block GPU pool (4 GiB), 512-slot pinned host tier (1 GiB); per step one
-            device-to-device move of 512 scattered blocks, one offload and one prefetch of 256.
+            device-to-device move of 512 scattered blocks, one offload and one prefetch of 256, and
+            one fused two-way transfer of 170 blocks out and 256 in.
     select: metadata-scale index (1,000,000 entries, 256 agents); per step observe 64 events,
             select 10,000 victims and 2,000 prefetch candidates (multi-launch select path).
     select80k: the 80,000-entry index of the Llama-8B configuration, 256 victims / 384 prefetch
@@ -622,12 +771,16 @@ def profile_case(args, torch, device):
         d_src, d_back = up(src), torch.arange(G - 512, G, dtype=torch.int32, device=device)
         hs, hd = synth.mover_batch(256, G, Hs, rng)
         d_hs, d_hd = up(hs), up(hd)
+        h_perm = rng.permutation(Hs).astype(np.uint32)
+        x_off_src, x_off_dst = up(src[:170].copy()), up(h_perm[:170].copy())
+        x_pre_src, x_pre_dst = up(h_perm[170:426].copy()), torch.arange(G - 512, G - 256, dtype=torch.int32, device=device)
         if args.offload_width or args.prefetch_width:
             c.set_mover_ctas(max(args.offload_width, args.prefetch_width), 0)
         for _ in range(max(1, args.steps)):
             c.compact_blocks(gpu, gpu, d_src, d_back)
             c.offload_blocks(gpu, host, d_hs, d_hd)
             c.prefetch_blocks(host, gpu, d_hd, d_hs)
+            c.exchange_blocks(gpu, host, x_off_src, x_off_dst, x_pre_src, x_pre_dst)
     else:
         big = args.workload == "select"
         cfg = synth.CONFIGS["meta1m" if big else "llama8b"]
@@ -804,6 +957,7 @@ def main():
                 "includes": "per step: H2D of the step's events and of the 80,000-entry index from pinned memory, D2H of the three id lists and counts, host sync on the result"},
     }
     if not args.no_extras and world == 1:
+        out["fused_step"] = fused_step_section(w)
         out["mover_sweep"] = mover_sweep(w, hbm_peak, link)
         del w
         torch.cuda.empty_cache()

@@ -224,6 +224,51 @@ int cs_exchange_blocks(cs_ctx *ctx, const cs_kv_pool *gpu, const cs_kv_pool *hos
                        const uint32_t *pre_host_slots, const uint32_t *pre_gpu_slots, uint32_t n_pre_max,
                        const uint32_t *n_pre_dev, cs_stream_t side);
 
+/* ---- one whole step as one call ------------------------------------------------------------------------ */
+
+/* The calls of one scheduler step in their order (Algorithm 1: ObserveTouch for the step's invocations,
+ * Evict for both tiers, BetweenStep's prefetch ranking) followed by the transfers that carry the decisions
+ * out, with every list and count staying on the device:
+ *   main: cs_observe_invocations(chain, agent, evflags, n_events)
+ *         cs_select_victims(idx, now, tier 0, k_victims) -> gpu_victims, n_gpu_victims
+ *         cs_select_victims(idx, now, tier 1, k_victims) -> host_victims, n_host_victims
+ *         cs_select_prefetch(idx, now, k_prefetch)       -> prefetch_ids, n_prefetch
+ *         every prefetch candidate whose host slot is one of this step's offload destinations is replaced
+ *         by CS_ID_NONE in prefetch_ids (it would be read while it is overwritten); n_prefetch still counts it
+ *         cs_compact_blocks(gpu -> stage, gpu_victims -> stage_slots)            (skipped when stage == NULL)
+ *   side: cs_exchange_blocks(gpu, host; gpu_victims -> host_victims, count min(n_gpu_victims, n_max);
+ *                            prefetch_ids -> free_gpu_slots)                     (after the calls above)
+ * The number of blocks offloaded is *n_gpu_victims; when the host tier yields fewer victims than that, the
+ * surplus entries of host_victims hold CS_ID_NONE and those blocks are skipped.  side may equal main; when
+ * it differs, main does not wait for the transfers unless join_main != 0 (needed when the call is captured
+ * into a CUDA graph from main: the side stream must rejoin before the capture ends).
+ * now_dev / n_events_dev (dev, optional): when not NULL the clock and the event count (at most n_events) are
+ * read from device memory when the kernels run, not when the call is made, so that a captured graph can be
+ * replayed for later steps after the caller has updated those words and the event buffers.
+ * All pointers in the struct: dev, except idx / gpu / host / stage (host structs).  The fork and join use two
+ * CUDA events the context owns (host objects made by cs_create, released by cs_destroy).  Before capturing
+ * the call into a graph, run each kind of call it contains once outside capture: the first launch of a
+ * kernel family sets its shared-memory attributes and probes the cluster size. */
+typedef struct cs_step_io {
+    const uint32_t *chain;
+    const uint16_t *agent;
+    const uint8_t *evflags;
+    uint32_t n_events;
+    const uint32_t *n_events_dev;
+    const cs_block_index *idx;
+    uint32_t now;
+    const uint32_t *now_dev;
+    uint32_t k_victims, k_prefetch;
+    uint32_t *gpu_victims, *n_gpu_victims;
+    uint32_t *host_victims, *n_host_victims;
+    uint32_t *prefetch_ids, *n_prefetch;
+    const cs_kv_pool *gpu, *host, *stage;
+    const uint32_t *stage_slots;       /* [k_victims] destination slots in the staging pool */
+    const uint32_t *free_gpu_slots;    /* [k_prefetch] GPU slots that receive the prefetched blocks */
+    uint32_t join_main;
+} cs_step_io;
+int cs_step(cs_ctx *ctx, const cs_step_io *io, cs_stream_t main, cs_stream_t side);
+
 /* ---- inspection ------------------------------------------------------------------------------------ */
 
 /* Copies the learner / scorer state into caller dev buffers (any may be NULL):

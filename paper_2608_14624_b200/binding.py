@@ -32,7 +32,7 @@ EXPORTS = ("cs_workspace_bytes", "cs_create", "cs_destroy", "cs_observe_invocati
            "cs_select_victims", "cs_select_prefetch", "cs_offload_blocks", "cs_prefetch_blocks",
            "cs_compact_blocks", "cs_get_model", "cs_get_status", "cs_launch_count", "cs_set_mover_ctas",
            "cs_last_cuda_error", "cs_strerror", "cs_version", "cs_select_victims_static", "cs_set_mover_path", "cs_set_select_path",
-           "cs_exact_survival", "cs_use_survival_table", "cs_import_state", "cs_set_select_speculation", "cs_exchange_blocks")
+           "cs_exact_survival", "cs_use_survival_table", "cs_import_state", "cs_set_select_speculation", "cs_exchange_blocks", "cs_step")
 
 
 class cs_params(C.Structure):
@@ -52,6 +52,16 @@ class cs_kv_pool(C.Structure):
     _fields_ = [("base", C.c_void_p), ("n_slots", C.c_uint32), ("layout", C.c_uint32), ("n_layers", C.c_uint32),
                 ("n_kv_heads", C.c_uint32), ("head_dim", C.c_uint32), ("block_tokens", C.c_uint32),
                 ("elem_bytes", C.c_uint32), ("first_id", C.c_uint32)]
+
+
+class cs_step_io(C.Structure):
+    _fields_ = [("chain", C.c_void_p), ("agent", C.c_void_p), ("evflags", C.c_void_p), ("n_events", C.c_uint32),
+                ("n_events_dev", C.c_void_p), ("idx", C.POINTER(cs_block_index)), ("now", C.c_uint32),
+                ("now_dev", C.c_void_p), ("k_victims", C.c_uint32), ("k_prefetch", C.c_uint32),
+                ("gpu_victims", C.c_void_p), ("n_gpu_victims", C.c_void_p), ("host_victims", C.c_void_p),
+                ("n_host_victims", C.c_void_p), ("prefetch_ids", C.c_void_p), ("n_prefetch", C.c_void_p),
+                ("gpu", C.POINTER(cs_kv_pool)), ("host", C.POINTER(cs_kv_pool)), ("stage", C.POINTER(cs_kv_pool)),
+                ("stage_slots", C.c_void_p), ("free_gpu_slots", C.c_void_p), ("join_main", C.c_uint32)]
 
 
 class CacheScoutError(RuntimeError):
@@ -88,6 +98,7 @@ def lib():
             getattr(L, name).argtypes = [vp, C.POINTER(cs_kv_pool), C.POINTER(cs_kv_pool), vp, vp, u32, vp, vp]
         L.cs_exchange_blocks.argtypes = [vp, C.POINTER(cs_kv_pool), C.POINTER(cs_kv_pool), vp, vp, u32, vp, vp, vp, u32,
                                          vp, vp]
+        L.cs_step.argtypes = [vp, C.POINTER(cs_step_io), vp, vp]
         L.cs_get_model.argtypes = [vp] * 10
         L.cs_get_status.argtypes = [vp, C.POINTER(u32), vp]
         L.cs_launch_count.argtypes = [vp, C.POINTER(C.c_uint64)]
@@ -191,6 +202,10 @@ def cs_exchange_blocks(ctx, gpu: cs_kv_pool, host: cs_kv_pool, off_gpu_slots, of
     _chk(lib().cs_exchange_blocks(ctx, C.byref(gpu), C.byref(host), _ptr(off_gpu_slots), _ptr(off_host_slots), n_off_max,
                                   _ptr(n_off_dev), _ptr(pre_host_slots), _ptr(pre_gpu_slots), n_pre_max,
                                   _ptr(n_pre_dev), _stream(stream)), "cs_exchange_blocks", ctx)
+
+
+def cs_step(ctx, io: cs_step_io, main=None, side=None):
+    _chk(lib().cs_step(ctx, C.byref(io), _stream(main), _stream(side)), "cs_step", ctx)
 
 
 def cs_compact_blocks(ctx, src: cs_kv_pool, dst: cs_kv_pool, src_slots, dst_slots, n_max: int, n_dev=None, stream=None):
@@ -384,6 +399,20 @@ class CacheScout:
             n_pre_max = 0 if pre_host_slots is None else int(pre_host_slots.numel())
         cs_exchange_blocks(self.ctx, gpu.struct(), host.struct(), off_gpu_slots, off_host_slots, n_off_max, n_off_dev,
                            pre_host_slots, pre_gpu_slots, n_pre_max, n_pre_dev, stream)
+
+    def step(self, idx: "DeviceIndex", now: int, chain, agent, evflags, n_events: int, k_victims: int, k_prefetch: int,
+             gpu_victims, n_gpu_victims, host_victims, n_host_victims, prefetch_ids, n_prefetch,
+             gpu: KVPool, host: KVPool, free_gpu_slots, stage: Optional[KVPool] = None, stage_slots=None,
+             now_dev=None, n_events_dev=None, main=None, side=None, join_main: bool = False):
+        """One whole step (observe, three selects, compaction, two-way transfer) as one call."""
+        i_s, g_s, h_s = idx.struct(), gpu.struct(), host.struct()
+        st_s = stage.struct() if stage is not None else None
+        io = cs_step_io(_ptr(chain), _ptr(agent), _ptr(evflags), n_events, _ptr(n_events_dev), C.pointer(i_s), now,
+                        _ptr(now_dev), k_victims, k_prefetch, _ptr(gpu_victims), _ptr(n_gpu_victims),
+                        _ptr(host_victims), _ptr(n_host_victims), _ptr(prefetch_ids), _ptr(n_prefetch),
+                        C.pointer(g_s), C.pointer(h_s), C.pointer(st_s) if st_s is not None else None,
+                        _ptr(stage_slots), _ptr(free_gpu_slots), 1 if join_main else 0)
+        cs_step(self.ctx, io, main, side)
 
     def compact_blocks(self, src: KVPool, dst: KVPool, src_slots, dst_slots, n_max=None, n_dev=None, stream=None):
         cs_compact_blocks(self.ctx, src.struct(), dst.struct(), src_slots, dst_slots,

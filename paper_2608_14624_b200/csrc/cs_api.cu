@@ -78,6 +78,32 @@ size_t cs_layout_workspace(const cs_params *p, uint32_t gtab_len, void *base, cs
     return off;
 }
 
+// cs_step(): a prefetch candidate whose host slot receives an offloaded block in the same step must not be
+// read while it is being overwritten; its entry in the prefetch list becomes CS_ID_NONE (the mover skips it).
+// One thread per candidate; the offload destinations pass through shared memory in chunks.
+#define STEP_FILTER_THREADS 256
+__global__ void __launch_bounds__(STEP_FILTER_THREADS)
+cs_step_filter_kernel(uint32_t *__restrict__ prefetch_ids, const uint32_t *__restrict__ n_prefetch, uint32_t k_prefetch,
+                      const uint32_t *__restrict__ host_victims, const uint32_t *__restrict__ n_gpu_victims,
+                      uint32_t k_victims)
+{
+    __shared__ uint32_t s_dst[STEP_FILTER_THREADS];
+    const uint32_t n_pf = min(k_prefetch, *n_prefetch), n_off = min(k_victims, *n_gpu_victims);
+    const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    const uint32_t mine = i < n_pf ? prefetch_ids[i] : CS_ID_NONE;
+    bool hit = false;
+    for (uint32_t base = 0; base < n_off; base += STEP_FILTER_THREADS) {
+        __syncthreads();
+        s_dst[threadIdx.x] = base + threadIdx.x < n_off ? host_victims[base + threadIdx.x] : CS_ID_NONE;
+        __syncthreads();
+        if (mine != CS_ID_NONE) {
+            const uint32_t lim = min((uint32_t)STEP_FILTER_THREADS, n_off - base);
+            for (uint32_t q = 0; q < lim; ++q) hit |= s_dst[q] == mine;
+        }
+    }
+    if (hit) prefetch_ids[i] = CS_ID_NONE;
+}
+
 extern "C" {
 
 int cs_version(void) { return 100; }
@@ -129,8 +155,12 @@ int cs_create(const cs_params *p, void *dev_workspace, size_t bytes, cs_stream_t
     if (e != cudaSuccess) { delete ctx; return CS_ECUDA; }
     ctx->host_link_ctas = 0;
     ctx->d2d_ctas = 0;
+    // fork / join events of cs_step(): host objects, created here so that the call itself creates nothing
+    e = cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_join, cudaEventDisableTiming);
+    if (e != cudaSuccess) { cs_destroy(ctx); return CS_ECUDA; }
     rc = cs_launch_init(ctx, (cudaStream_t)init_stream);
-    if (rc != CS_OK) { delete ctx; return rc; }
+    if (rc != CS_OK) { cs_destroy(ctx); return rc; }
     *out = ctx;
     return CS_OK;
 }
@@ -138,6 +168,8 @@ int cs_create(const cs_params *p, void *dev_workspace, size_t bytes, cs_stream_t
 int cs_destroy(cs_ctx *ctx)
 {
     if (!ctx) return CS_EINVAL;
+    if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
+    if (ctx->ev_join) cudaEventDestroy(ctx->ev_join);
     delete ctx;
     return CS_OK;
 }
@@ -269,6 +301,50 @@ int cs_exchange_blocks(cs_ctx *ctx, const cs_kv_pool *gpu, const cs_kv_pool *hos
     if ((n_off_dev && (((uintptr_t)n_off_dev) & 3u)) || (n_pre_dev && (((uintptr_t)n_pre_dev) & 3u))) return CS_EINVAL;
     return cs_launch_exchange(ctx, gpu, host, off_gpu_slots, off_host_slots, n_off_max, n_off_dev, pre_host_slots,
                               pre_gpu_slots, n_pre_max, n_pre_dev, (cudaStream_t)side);
+}
+
+int cs_step(cs_ctx *ctx, const cs_step_io *io, cs_stream_t main_, cs_stream_t side_)
+{
+    if (!ctx || !io || !io->idx || !io->gpu || !io->host) return CS_EINVAL;
+    if ((io->now_dev && (((uintptr_t)io->now_dev) & 3u)) || (io->n_events_dev && (((uintptr_t)io->n_events_dev) & 3u)))
+        return CS_EINVAL;
+    if (io->stage && !io->stage_slots) return CS_EINVAL;
+    cudaStream_t main = (cudaStream_t)main_, side = (cudaStream_t)side_;
+    const bool forked = side != main;
+    ctx->step_now_dev = io->now_dev;
+    ctx->step_n_events_dev = io->n_events_dev;
+    int rc = cs_observe_invocations(ctx, io->chain, io->agent, io->evflags, io->n_events, main_);
+    if (rc == CS_OK) rc = cs_select_victims(ctx, io->idx, io->now, 0, io->k_victims, io->gpu_victims, io->n_gpu_victims, main_);
+    if (rc == CS_OK) rc = cs_select_victims(ctx, io->idx, io->now, 1, io->k_victims, io->host_victims, io->n_host_victims, main_);
+    if (rc == CS_OK) rc = cs_select_prefetch(ctx, io->idx, io->now, io->k_prefetch, io->prefetch_ids, io->n_prefetch, main_);
+    ctx->step_now_dev = nullptr;
+    ctx->step_n_events_dev = nullptr;
+    if (rc != CS_OK) return rc;
+    if (io->k_prefetch && io->k_victims) {
+        const uint32_t grid = (io->k_prefetch + STEP_FILTER_THREADS - 1) / STEP_FILTER_THREADS;
+        cs_step_filter_kernel<<<grid, STEP_FILTER_THREADS, 0, main>>>(io->prefetch_ids, io->n_prefetch, io->k_prefetch,
+                                                                      io->host_victims, io->n_gpu_victims, io->k_victims);
+        if ((rc = cs_check_launch(ctx)) != CS_OK) return rc;
+    }
+    if (io->stage) {
+        rc = cs_compact_blocks(ctx, io->gpu, io->stage, io->gpu_victims, io->stage_slots, io->k_victims, io->n_gpu_victims, main_);
+        if (rc != CS_OK) return rc;
+    }
+    cudaError_t e = cudaSuccess;
+    if (forked) {
+        e = cudaEventRecord(ctx->ev_fork, main);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(side, ctx->ev_fork, 0);
+        if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; return CS_ECUDA; }
+    }
+    rc = cs_exchange_blocks(ctx, io->gpu, io->host, io->gpu_victims, io->host_victims, io->k_victims, io->n_gpu_victims,
+                            io->prefetch_ids, io->free_gpu_slots, io->k_prefetch, io->n_prefetch, side_);
+    if (rc != CS_OK) return rc;
+    if (forked && io->join_main) {
+        e = cudaEventRecord(ctx->ev_join, side);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(main, ctx->ev_join, 0);
+        if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; return CS_ECUDA; }
+    }
+    return CS_OK;
 }
 
 int cs_get_model(cs_ctx *ctx, uint32_t *C_out, float *P_out, uint16_t *amax_out, uint16_t *hops_out,

@@ -20,6 +20,7 @@
 #define CS_HIST_BINS 4096u        // first radix digit of the select: top 12 bits of the primary key
 #define CS_MAX_SPLITTERS 255u     // bucket sort of the candidates: up to 256 buckets
 #define CS_SAMPLE 1024u           // candidates sampled to choose the splitters
+#define CS_SPEC_MARGIN_CALLS 16u    // after a missed speculation: calls that collect one bin beyond the last threshold
 #define CS_GTAB_MAX 4096u          // largest recency table kept in shared memory (ages below saturation)
 
 // Scalars the kernels share, one 256-byte line in the workspace.
@@ -39,12 +40,17 @@ struct cs_scalars {
     uint32_t sel_p_end;     // end position of that bucket
     uint32_t sel_n_out;     // min(k, eligible)
     uint32_t gtab_monotone; // the recency table covers every unsaturated age and never increases with age
-    uint32_t sel_hint[4];   // threshold bin of the previous select (GPU victims, host victims, prefetch); ~0 = none;
+    uint32_t sel_hint[4];   // bin up to which the next select of each kind (GPU victims, host victims, prefetch)
+                            // collects ahead: the previous threshold bin, plus one while sel_margin > 0; ~0 = none;
                             // slot 3 is never written: calls that must not speculate read it
+    uint32_t sel_margin[4]; // per kind: calls left during which the next call collects one bin beyond the remembered
+                            // threshold (set after a miss: that kind's threshold is moving upwards or jitters)
     uint32_t sel_c_spec;    // candidates appended speculatively by the histogram pass; 0 between calls
     uint32_t sel_spec;      // 1: the speculative candidates cover the k winners, the collect pass is skipped
     uint32_t sel_cc[2];     // candidate counters of the cluster kernel: a call uses one and clears the other for
                             // the next call, so that the counter is zero on entry without a barrier
+    uint32_t sel_toggle;    // which of the two the next cluster select uses; flipped by every call on the device, so
+                            // that a captured sequence of calls stays consistent when it is replayed
     unsigned long long t_phase[8];   // globaltimer stamps of the last cluster select (phase boundaries, ns)
 };
 
@@ -89,12 +95,14 @@ struct cs_ctx {
     uint32_t host_link_ctas, d2d_ctas;
     uint32_t mover_path;   // CS_MOVER_*
     uint32_t select_path;  // CS_SELECT_*
-    uint32_t cluster_slot;         // which of the two candidate counters the next cluster select uses
     uint32_t no_speculation;       // 1: the histogram pass never collects ahead of the threshold
     const float *fsurv_override;   // caller's survival table for score / select, NULL = the BFS table of Eq. 8
     int cluster_max_v, cluster_max_pf;   // largest usable cluster of the single-launch select (0 = not probed, -1 = none)
     int bulk_attr_set;     // shared-memory opt-in of the bulk kernel done on this device
     int collect_attr_set;  // same for the collect kernel with age limits
+    const uint32_t *step_now_dev;        // set only while cs_step() issues its calls: device-resident clock / event count
+    const uint32_t *step_n_events_dev;
+    cudaEvent_t ev_fork, ev_join;        // cs_step(): main -> side and side -> main, created on first use
     uint64_t n_launches;
     int last_cuda_error;
 };

@@ -55,8 +55,10 @@ __global__ void cs_gtab_check_kernel(cs_workspace ws, uint32_t gtab_len, uint32_
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(OBS_THREADS)
 cs_observe_kernel(cs_workspace ws, uint32_t A, uint32_t n_chains, const uint32_t *__restrict__ chain,
-                  const uint16_t *__restrict__ agent, const uint8_t *__restrict__ evflags, uint32_t n_events)
+                  const uint16_t *__restrict__ agent, const uint8_t *__restrict__ evflags, uint32_t n_events,
+                  const uint32_t *__restrict__ n_events_dev)
 {
+    if (n_events_dev) n_events = min(n_events, *n_events_dev);     // device-resident count (graph replay)
     __shared__ uint32_t s_chain[OBS_THREADS];
     __shared__ uint16_t s_agent[OBS_THREADS];     // CS_AGENT_NONE marks an event that is skipped
     __shared__ int s_last;
@@ -441,7 +443,8 @@ int cs_launch_observe(cs_ctx *ctx, const uint32_t *chain, const uint16_t *agent,
 {
     const cs_params &p = ctx->p;
     if (n_events) {
-        cs_observe_kernel<<<1, OBS_THREADS, 0, s>>>(ctx->ws, p.n_agents, p.n_chains, chain, agent, evflags, n_events);
+        cs_observe_kernel<<<1, OBS_THREADS, 0, s>>>(ctx->ws, p.n_agents, p.n_chains, chain, agent, evflags, n_events,
+                                                ctx->step_n_events_dev);
         int rc = cs_check_launch(ctx);
         if (rc != CS_OK) return rc;
     }

@@ -36,6 +36,7 @@
 __global__ void __launch_bounds__(SEL_THREADS) cs_score_kernel(SelArgs a, cs_workspace ws, float *__restrict__ out)
 {
     extern __shared__ float smem[];
+    resolve_now(a);
     Tables T;
     load_tables(a, ws, smem, T, false);
     __syncthreads();
@@ -117,6 +118,7 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_hist_kernel(SelArgs a, cs_
     __shared__ uint32_t s_part[SEL_THREADS];
     __shared__ uint32_t s_b0;
     __shared__ bool s_flag;
+    resolve_now(a);
     Tables T;
     load_tables(a, ws, smem, T, PF && a.anchor);
     for (uint32_t i = threadIdx.x; i < CS_HIST_BINS; i += blockDim.x) s_hist[i] = 0;
@@ -242,7 +244,7 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_hist_kernel(SelArgs a, cs_
         ws.sc->sel_c = spec_ok ? c_spec : 0;
         ws.sc->sel_c_spec = 0;
         ws.sc->sel_spec = spec_ok ? 1u : 0u;
-        if (a.hint_slot < 3) ws.sc->sel_hint[a.hint_slot] = (a.k && total >= a.k) ? b0 : 0xFFFFFFFFu;
+        remember_threshold(ws.sc, a.hint_slot, a.k && total >= a.k, b0, hint != 0xFFFFFFFFu, spec_ok);
         ws.sc->ticket[1] = 0;
     }
 }
@@ -298,6 +300,7 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_collect_kernel(SelArgs a, 
     __shared__ uint32_t s_id[CS_SAMPLE];
     __shared__ bool s_flag;
     if (ws.sc->sel_spec) return;          // the histogram pass already collected the candidates
+    resolve_now(a);
     Tables T;
     load_tables(a, ws, smem, T, PF && a.anchor);
     __syncthreads();
@@ -581,7 +584,7 @@ static void fill_args(const cs_ctx *ctx, const cs_block_index *idx, uint32_t now
     a.prefer_copy = ctx->p.prefer_other_copy ? 1u : 0u;
     a.use_age_limits = 0;
     a.hint_slot = 0;
-    a.c_slot = 0;
+    a.now_dev = ctx->step_now_dev;
 }
 
 static uint32_t scan_grid(const cs_ctx *ctx, uint32_t n, uint32_t per_cta, uint32_t ctas_per_sm = 2)

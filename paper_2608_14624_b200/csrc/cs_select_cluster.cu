@@ -121,6 +121,7 @@ __global__ void __launch_bounds__(CSEL_THREADS, 1)
 cs_select_cluster_kernel(SelArgs a, cs_workspace ws, uint32_t *__restrict__ ids_out, uint32_t *__restrict__ n_out_dev)
 {
     extern __shared__ __align__(16) unsigned char dsm[];
+    resolve_now(a);
     cg::cluster_group cluster = cg::this_cluster();
     const uint32_t CL = cluster.num_blocks(), rank = cluster.block_rank();
     const uint32_t tid = threadIdx.x, lane = tid & 31;
@@ -129,8 +130,9 @@ cs_select_cluster_kernel(SelArgs a, cs_workspace ws, uint32_t *__restrict__ ids_
     Tables T;
     load_tables(a, ws, S.tables, T, PF && a.anchor);
     for (uint32_t i = tid; i < CS_HIST_BINS; i += CSEL_THREADS) S.hist[i] = 0;
-    uint32_t *cand_count = &ws.sc->sel_cc[a.c_slot];          // zero on entry: the previous call cleared it
-    if (rank == 0 && tid == 0) ws.sc->sel_cc[a.c_slot ^ 1u] = 0;
+    const uint32_t c_slot = *(volatile uint32_t *)&ws.sc->sel_toggle & 1u;   // read here, before any CTA can flip it (first cluster barrier)
+    uint32_t *cand_count = &ws.sc->sel_cc[c_slot];            // zero on entry: the previous call cleared it
+    if (rank == 0 && tid == 0) ws.sc->sel_cc[c_slot ^ 1u] = 0;
     if (tid == 0) S.misc[1] = 0;
     __syncthreads();
     const bool enabled = !PF || prefetch_enabled(ws, a.A);
@@ -233,6 +235,7 @@ cs_select_cluster_kernel(SelArgs a, cs_workspace ws, uint32_t *__restrict__ ids_
         }
     }
     cluster.sync();
+    if (rank == 0 && tid == 0) ws.sc->sel_toggle = c_slot ^ 1u;      // every CTA has read it: the next call takes the other counter
     constexpr uint32_t PER = CS_HIST_BINS / CSEL_THREADS;
     uint32_t loc[PER], sum = 0;
 #pragma unroll
@@ -259,7 +262,7 @@ cs_select_cluster_kernel(SelArgs a, cs_workspace ws, uint32_t *__restrict__ ids_
     csel_stamp(ws, rank, 2);
     // ---- phase 3: collect the candidates (bin <= b0), unless the first scan already has them ----------------
     const bool spec_ok = hint != 0xFFFFFFFFu && b0 != 0xFFFFFFFFu && b0 <= hint;     // same verdict in every CTA
-    if (rank == 0 && tid == 0 && a.hint_slot < 3) ws.sc->sel_hint[a.hint_slot] = (a.k && n_elig >= a.k) ? b0 : 0xFFFFFFFFu;
+    if (rank == 0 && tid == 0) remember_threshold(ws.sc, a.hint_slot, a.k && n_elig >= a.k, b0, hint != 0xFFFFFFFFu, spec_ok);
     if (!spec_ok) {
         if (hint != 0xFFFFFFFFu) {                            // drop what the first scan appended
             if (rank == 0 && tid == 0) *cand_count = 0;
@@ -420,10 +423,7 @@ static int launch_cluster(cs_ctx *ctx, const SelArgs &a, uint32_t *ids_out, uint
     while (cl < max_cl && (uint32_t)cl * CSEL_THREADS < n_groups) cl <<= 1;
     cfg.gridDim = dim3(cl);
     attr[0].val.clusterDim.x = cl;
-    SelArgs args = a;
-    args.c_slot = ctx->cluster_slot;
-    ctx->cluster_slot ^= 1u;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, args, ctx->ws, ids_out, n_out);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, a, ctx->ws, ids_out, n_out);
     ctx->n_launches++;
     if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; return CS_ECUDA; }
     return CS_OK;

@@ -20,8 +20,30 @@ struct SelArgs {
     uint32_t tier, k, prefer_copy;
     uint32_t use_age_limits;      // collect pass may prefilter by per-(agent, size) age limits (large indexes)
     uint32_t hint_slot;           // which remembered threshold bin this call may speculate on
-    uint32_t c_slot;              // candidate counter of the cluster kernel for this call
+    const uint32_t *now_dev;      // when set, the clock is read from device memory at execution time (graph replay)
 };
+
+// What the next call of this kind may collect ahead of its own threshold.  The threshold bin of
+// consecutive calls moves little; where it moves upwards or jitters (a miss), one extra bin is allowed
+// for the next CS_SPEC_MARGIN_CALLS calls.  Only the amount of work depends on this, never the result.
+__device__ __forceinline__ void remember_threshold(cs_scalars *sc, uint32_t slot, bool valid, uint32_t b0, bool had_hint,
+                                                   bool spec_ok)
+{
+    if (slot >= 3) return;
+    if (!valid) { sc->sel_hint[slot] = 0xFFFFFFFFu; return; }
+    uint32_t m = sc->sel_margin[slot];
+    if (had_hint && !spec_ok) m = CS_SPEC_MARGIN_CALLS;
+    else if (m) --m;
+    sc->sel_margin[slot] = m;
+    const uint32_t lim = b0 + (m ? 1u : 0u);
+    sc->sel_hint[slot] = lim < CS_HIST_BINS ? lim : CS_HIST_BINS - 1;
+}
+
+// The clock of a call: by value, or from device memory when the caller asked for that.
+__device__ __forceinline__ void resolve_now(SelArgs &a)
+{
+    if (a.now_dev) a.now = __ldg(a.now_dev);
+}
 
 // Per-CTA copies of the small tables every entry looks up.
 struct Tables {
