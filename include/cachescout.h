@@ -307,6 +307,17 @@ int cs_set_mover_ctas(cs_ctx *ctx, uint32_t host_link_ctas, uint32_t d2d_ctas);
 #define CS_MOVER_BULK 2u
 int cs_set_mover_path(cs_ctx *ctx, uint32_t path);
 
+/* Sources of the cached hop table (Eq. 8).  The paper's runtime serves one request at a time and starts
+ * the BFS at that request's current agent (Sec. 3.3); CS_SOURCES_LAST_AGENT is that.  With many sessions
+ * in flight, CS_SOURCES_ALL_CHAINS starts it at the current agent of EVERY chain that has one (all live
+ * sessions): E[a] is then the hop distance from the nearest of them, and blocks of any agent that some live
+ * session is about to reach are protected.  Prefetch ranking keeps using the successor of the last invoked
+ * agent (Eq. 10).  The call refreshes the cached tables on `stream`; later cs_observe_invocations() calls
+ * keep the mode. */
+#define CS_SOURCES_LAST_AGENT 0u
+#define CS_SOURCES_ALL_CHAINS 1u
+int cs_set_survival_sources(cs_ctx *ctx, uint32_t mode, cs_stream_t stream);
+
 /* ---- exact survival probability (the quantity Eq. 8 approximates) ---------------------------------- */
 
 /* Eq. 6 for every agent a: p_surv(a; a0, K) = Pr(a is invoked within the next K dispatches | the

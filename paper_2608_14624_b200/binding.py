@@ -32,7 +32,7 @@ EXPORTS = ("cs_workspace_bytes", "cs_create", "cs_destroy", "cs_observe_invocati
            "cs_select_victims", "cs_select_prefetch", "cs_offload_blocks", "cs_prefetch_blocks",
            "cs_compact_blocks", "cs_get_model", "cs_get_status", "cs_launch_count", "cs_set_mover_ctas",
            "cs_last_cuda_error", "cs_strerror", "cs_version", "cs_select_victims_static", "cs_set_mover_path", "cs_set_select_path",
-           "cs_exact_survival", "cs_use_survival_table", "cs_import_state", "cs_set_select_speculation", "cs_exchange_blocks", "cs_step")
+           "cs_exact_survival", "cs_use_survival_table", "cs_import_state", "cs_set_select_speculation", "cs_exchange_blocks", "cs_step", "cs_set_survival_sources")
 
 
 class cs_params(C.Structure):
@@ -98,6 +98,7 @@ def lib():
             getattr(L, name).argtypes = [vp, C.POINTER(cs_kv_pool), C.POINTER(cs_kv_pool), vp, vp, u32, vp, vp]
         L.cs_exchange_blocks.argtypes = [vp, C.POINTER(cs_kv_pool), C.POINTER(cs_kv_pool), vp, vp, u32, vp, vp, vp, u32,
                                          vp, vp]
+        L.cs_set_survival_sources.argtypes = [vp, u32, vp]
         L.cs_step.argtypes = [vp, C.POINTER(cs_step_io), vp, vp]
         L.cs_get_model.argtypes = [vp] * 10
         L.cs_get_status.argtypes = [vp, C.POINTER(u32), vp]
@@ -202,6 +203,13 @@ def cs_exchange_blocks(ctx, gpu: cs_kv_pool, host: cs_kv_pool, off_gpu_slots, of
     _chk(lib().cs_exchange_blocks(ctx, C.byref(gpu), C.byref(host), _ptr(off_gpu_slots), _ptr(off_host_slots), n_off_max,
                                   _ptr(n_off_dev), _ptr(pre_host_slots), _ptr(pre_gpu_slots), n_pre_max,
                                   _ptr(n_pre_dev), _stream(stream)), "cs_exchange_blocks", ctx)
+
+
+CS_SOURCES_LAST_AGENT, CS_SOURCES_ALL_CHAINS = 0, 1
+
+
+def cs_set_survival_sources(ctx, mode: int, stream=None):
+    _chk(lib().cs_set_survival_sources(ctx, mode, _stream(stream)), "cs_set_survival_sources", ctx)
 
 
 def cs_step(ctx, io: cs_step_io, main=None, side=None):
@@ -464,6 +472,9 @@ class CacheScout:
     def use_survival_table(self, fsurv):
         self._fsurv_keepalive = fsurv
         cs_use_survival_table(self.ctx, fsurv)
+
+    def set_survival_sources(self, mode: int, stream=None):
+        cs_set_survival_sources(self.ctx, mode, stream)
 
     def set_select_speculation(self, enabled: bool):
         cs_set_select_speculation(self.ctx, enabled)

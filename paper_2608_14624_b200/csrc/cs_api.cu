@@ -404,6 +404,13 @@ int cs_set_mover_ctas(cs_ctx *ctx, uint32_t host_link_ctas, uint32_t d2d_ctas)
     return CS_OK;
 }
 
+int cs_set_survival_sources(cs_ctx *ctx, uint32_t mode, cs_stream_t stream)
+{
+    if (!ctx || mode > CS_SOURCES_ALL_CHAINS) return CS_EINVAL;
+    ctx->source_mode = mode;
+    return cs_launch_observe(ctx, nullptr, nullptr, nullptr, 0, (cudaStream_t)stream);   // refresh the cached tables
+}
+
 int cs_set_mover_path(cs_ctx *ctx, uint32_t path)
 {
     if (!ctx || path > CS_MOVER_BULK) return CS_EINVAL;

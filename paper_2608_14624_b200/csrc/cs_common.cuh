@@ -96,6 +96,7 @@ struct cs_ctx {
     uint32_t mover_path;   // CS_MOVER_*
     uint32_t select_path;  // CS_SELECT_*
     uint32_t no_speculation;       // 1: the histogram pass never collects ahead of the threshold
+    uint32_t source_mode;          // CS_SOURCES_*: where the cached BFS of Eq. 8 starts
     const float *fsurv_override;   // caller's survival table for score / select, NULL = the BFS table of Eq. 8
     int cluster_max_v, cluster_max_pf;   // largest usable cluster of the single-launch select (0 = not probed, -1 = none)
     int bulk_attr_set;     // shared-memory opt-in of the bulk kernel done on this device

@@ -182,7 +182,7 @@ __device__ T cs_block_sum(T v, T *s_red)
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(ROW_THREADS)
 cs_normalise_kernel(cs_workspace ws, uint32_t A, uint32_t W, float eps, float tau, float r_min, uint32_t e_max,
-                    float delta)
+                    float delta, uint32_t all_chains, uint32_t n_chains)
 {
     __shared__ double s_red[ROW_THREADS];
     __shared__ float s_bestv[ROW_THREADS];
@@ -268,7 +268,17 @@ cs_normalise_kernel(cs_workspace ws, uint32_t A, uint32_t W, float eps, float ta
         ws.sc->gate = (Rf >= r_min) ? 1u : 0u;
         ws.sc->ticket[0] = 0;
     }
-    if (tid < 32) s_front[tid] = (la < A && (la >> 5) == tid) ? (1u << (la & 31)) : 0u;
+    if (all_chains) {
+        // sources: the current agent of every chain that has one (all live sessions)
+        if (tid < 32) s_front[tid] = 0;
+        __syncthreads();
+        for (uint32_t ch = tid; ch < n_chains; ch += ROW_THREADS) {
+            const uint32_t a = __ldcg(&ws.cur[ch]);
+            if (a < A) atomicOr(&s_front[a >> 5], 1u << (a & 31));
+        }
+    } else if (tid < 32) {
+        s_front[tid] = (la < A && (la >> 5) == tid) ? (1u << (la & 31)) : 0u;
+    }
     __syncthreads();
     cs_bfs_survival(ws.adj, A, W, s_front, s_visit, s_next, ws.hops, ws.fsurv, e_max, delta);
 }
@@ -450,7 +460,8 @@ int cs_launch_observe(cs_ctx *ctx, const uint32_t *chain, const uint16_t *agent,
     }
     const uint32_t grid = p.n_agents < 2u * (uint32_t)ctx->sm_count ? p.n_agents : 2u * (uint32_t)ctx->sm_count;
     cs_normalise_kernel<<<grid, ROW_THREADS, 0, s>>>(ctx->ws, p.n_agents, ctx->W, p.eps, p.tau, p.r_min, p.e_max,
-                                                      p.delta);
+                                                      p.delta, ctx->source_mode == CS_SOURCES_ALL_CHAINS ? 1u : 0u,
+                                                      p.n_chains);
     return cs_check_launch(ctx);
 }
 

@@ -523,3 +523,41 @@ def test_select_large_index_uses_age_limits(with_tokens, prefer):
     assert o_n == 2000
     assert H.assert_list_matches(ids.cpu().numpy().view(np.uint32)[:2000], int(n_out.item()), o_ids, o_n, s64) == 0
     assert c.get_status() == 0
+
+
+# ---- hop table from every live session's current agent ----------------------------------------------------
+@pytest.mark.parametrize("name,n_inv", [("tiny", 60), ("llama8b", 400), ("meta1m", 3000)])
+def test_survival_from_all_chains(name, n_inv):
+    """CS_SOURCES_ALL_CHAINS: the cached BFS starts at the current agent of every chain; the oracle runs its
+    multi-source BFS (pinned by brute force) from the same set, and the selects follow the new table."""
+    cfg = synth.CONFIGS[name]
+    if name == "tiny":
+        cfg = synth.shrink(cfg, sessions=4, n_chains=4)
+    n = 20000
+    c, o = warm_state(cfg, n_inv, n, r_min=0.02)
+    c.set_survival_sources(cs.CS_SOURCES_ALL_CHAINS)
+    srcs = np.unique(o.cur[o.cur != orc.AGENT_NONE])
+    assert len(srcs) >= 2, "needs several live chains"
+    o.survival(sources=srcs)
+    H.compare_model(c, o)
+    assert np.all(o.E[srcs] == 0)
+    # the mode persists across observe calls
+    tr = synth.make_trace(cfg, n_invocations=n_inv + 40)
+    lo = len(tr.agent) - 40
+    c.observe_invocations(dev(tr.chain[lo:]), dev(tr.agent[lo:]), dev(tr.evflags[lo:]))
+    o.observe(tr.chain[lo:], tr.agent[lo:], tr.evflags[lo:])
+    o.survival(sources=np.unique(o.cur[o.cur != orc.AGENT_NONE]))
+    H.compare_model(c, o)
+    idx = synth.make_block_index(cfg, n=n, tier="random")
+    d = cs.DeviceIndex.from_host(idx, DEV)
+    s64, s32 = o.scores(idx, 100_000)
+    assert np.array_equal(c.score_blocks(d, 100_000).cpu().numpy(), s32)
+    k = 300
+    ids, n_out = c.select_victims(d, 100_000, 0, k)
+    o_ids, o_n = o.select_victims(idx, 100_000, 0, k, s32)
+    assert H.assert_list_matches(ids.cpu().numpy().view(np.uint32)[:k], int(n_out[0].item()), o_ids, o_n, s64) == 0
+    # back to the single source
+    c.set_survival_sources(cs.CS_SOURCES_LAST_AGENT)
+    o.survival()
+    H.compare_model(c, o)
+    assert c.get_status() == 0
