@@ -45,6 +45,8 @@ def parse_args():
     ap.add_argument("--prefetch-width", type=int, default=0, help="warp pipelines of the prefetch mover (0 = library default)")
     ap.add_argument("--transfers", default="exchange", choices=["exchange", "split"],
                     help="offload and prefetch of a step as one fused launch (exchange) or as two launches on two streams (split)")
+    ap.add_argument("--selects", default="fused", choices=["fused", "separate"],
+                    help="the three selects of a step as one launch (cs_select_step) or as three calls")
     ap.add_argument("--exchange-width", type=int, default=0, help="warp pipelines of the fused transfer (0 = library default)")
     ap.add_argument("--quick", action="store_true", help="small pools (debugging only; not a valid bench line)")
     ap.add_argument("--workload", default="step", choices=["step", "mover", "select", "select80k"],
@@ -208,6 +210,7 @@ class StepWorkload:
         self.now0 = 100_000
         self.w_off, self.w_pre = args.offload_width, args.prefetch_width
         self.fused, self.w_ex = args.transfers == "exchange", args.exchange_width
+        self.fused_selects = getattr(args, "selects", "fused") == "fused"
         self.fifo = [torch.zeros(self.k_p, dtype=torch.int64, device=device) for _ in range(8)]
         self.fifo_used = 0
         self.bytes_per_step = (self.k_v + self.k_p) * bb
@@ -248,9 +251,12 @@ class StepWorkload:
         c.observe_invocations(chain, agent, flags, n_events=n_ev)
         rec(t[1], main)
         vict = self.dst[b][:self.k_v]
-        c.select_victims(self.didx, now, 0, self.k_v, vict, self.vn[b])
-        c.select_victims(self.didx, now, 1, self.k_v, self.hv[b], self.hn[b])
-        c.select_prefetch(self.didx, now, self.k_p, self.pf[b], self.pn[b])
+        if self.fused_selects:         # one launch: three thread-block clusters side by side
+            c.select_step(self.didx, now, self.k_v, self.k_p, vict, self.vn[b], self.hv[b], self.hn[b], self.pf[b], self.pn[b])
+        else:
+            c.select_victims(self.didx, now, 0, self.k_v, vict, self.vn[b])
+            c.select_victims(self.didx, now, 1, self.k_v, self.hv[b], self.hn[b])
+            c.select_prefetch(self.didx, now, self.k_p, self.pf[b], self.pn[b])
         rec(t[2], main)
         c.compact_blocks(self.gpu_pool, self.stage_pool, vict, self.packed, n_max=self.k_v, n_dev=self.vn[b])
         rec(t[3], main)
@@ -949,7 +955,7 @@ def main():
                       "note": ("offload and prefetch of a step run as one fused launch (cs_exchange_blocks): both per-direction times "
                                "are that launch's duration" if w.fused else
                                "offload and prefetch of a step overlap (full duplex); per-direction times are measured while the other direction is busy")},
-        "select": {"ms_three_selects": t_s, "ms_observe": t_ob, "algorithmic_bytes": sel_bytes,
+        "select": {"how": "cs_select_step: one launch of three 16-CTA clusters" if w.fused_selects else "three calls", "ms_three_selects": t_s, "ms_observe": t_ob, "algorithmic_bytes": sel_bytes,
                    "achieved_GBps": sel_bytes / (t_s / 1e3) / 1e9, "frac_of_hbm_peak": sel_bytes / (t_s / 1e3) / 1e9 / hbm_peak,
                    "n_out_last_step": n_out, "device_status": status},
         "e2e": {"value": e2e_value, "unit": "GB/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,

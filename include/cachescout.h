@@ -224,15 +224,23 @@ int cs_exchange_blocks(cs_ctx *ctx, const cs_kv_pool *gpu, const cs_kv_pool *hos
                        const uint32_t *pre_host_slots, const uint32_t *pre_gpu_slots, uint32_t n_pre_max,
                        const uint32_t *n_pre_dev, cs_stream_t side);
 
+/* The three selections of a step at once: cs_select_victims(tier 0, k_victims), cs_select_victims(tier 1,
+ * k_victims) and cs_select_prefetch(k_prefetch) over the same index and clock, with the same results.  For
+ * index sizes the single-launch select covers (<= 262,144 entries) they run as ONE launch of three
+ * thread-block clusters side by side; otherwise as the three calls in a row.  Arguments as for those calls. */
+int cs_select_step(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, uint32_t k_victims, uint32_t k_prefetch,
+                   uint32_t *gpu_victims, uint32_t *n_gpu_victims, uint32_t *host_victims, uint32_t *n_host_victims,
+                   uint32_t *prefetch_ids, uint32_t *n_prefetch, cs_stream_t stream);
+
 /* ---- one whole step as one call ------------------------------------------------------------------------ */
 
 /* The calls of one scheduler step in their order (Algorithm 1: ObserveTouch for the step's invocations,
  * Evict for both tiers, BetweenStep's prefetch ranking) followed by the transfers that carry the decisions
  * out, with every list and count staying on the device:
  *   main: cs_observe_invocations(chain, agent, evflags, n_events)
- *         cs_select_victims(idx, now, tier 0, k_victims) -> gpu_victims, n_gpu_victims
- *         cs_select_victims(idx, now, tier 1, k_victims) -> host_victims, n_host_victims
- *         cs_select_prefetch(idx, now, k_prefetch)       -> prefetch_ids, n_prefetch
+ *         cs_select_step(idx, now, k_victims, k_prefetch) -> gpu_victims, n_gpu_victims (tier 0),
+ *                                                            host_victims, n_host_victims (tier 1),
+ *                                                            prefetch_ids, n_prefetch
  *         every prefetch candidate whose host slot is one of this step's offload destinations is replaced
  *         by CS_ID_NONE in prefetch_ids (it would be read while it is overwritten); n_prefetch still counts it
  *         cs_compact_blocks(gpu -> stage, gpu_victims -> stage_slots)            (skipped when stage == NULL)

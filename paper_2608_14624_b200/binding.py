@@ -32,7 +32,7 @@ EXPORTS = ("cs_workspace_bytes", "cs_create", "cs_destroy", "cs_observe_invocati
            "cs_select_victims", "cs_select_prefetch", "cs_offload_blocks", "cs_prefetch_blocks",
            "cs_compact_blocks", "cs_get_model", "cs_get_status", "cs_launch_count", "cs_set_mover_ctas",
            "cs_last_cuda_error", "cs_strerror", "cs_version", "cs_select_victims_static", "cs_set_mover_path", "cs_set_select_path",
-           "cs_exact_survival", "cs_use_survival_table", "cs_import_state", "cs_set_select_speculation", "cs_exchange_blocks", "cs_step", "cs_set_survival_sources")
+           "cs_exact_survival", "cs_use_survival_table", "cs_import_state", "cs_set_select_speculation", "cs_exchange_blocks", "cs_step", "cs_set_survival_sources", "cs_select_step")
 
 
 class cs_params(C.Structure):
@@ -99,6 +99,7 @@ def lib():
         L.cs_exchange_blocks.argtypes = [vp, C.POINTER(cs_kv_pool), C.POINTER(cs_kv_pool), vp, vp, u32, vp, vp, vp, u32,
                                          vp, vp]
         L.cs_set_survival_sources.argtypes = [vp, u32, vp]
+        L.cs_select_step.argtypes = [vp, C.POINTER(cs_block_index), u32, u32, u32, vp, vp, vp, vp, vp, vp, vp]
         L.cs_step.argtypes = [vp, C.POINTER(cs_step_io), vp, vp]
         L.cs_get_model.argtypes = [vp] * 10
         L.cs_get_status.argtypes = [vp, C.POINTER(u32), vp]
@@ -210,6 +211,13 @@ CS_SOURCES_LAST_AGENT, CS_SOURCES_ALL_CHAINS = 0, 1
 
 def cs_set_survival_sources(ctx, mode: int, stream=None):
     _chk(lib().cs_set_survival_sources(ctx, mode, _stream(stream)), "cs_set_survival_sources", ctx)
+
+
+def cs_select_step(ctx, idx: cs_block_index, now: int, k_victims: int, k_prefetch: int, gpu_victims, n_gpu_victims,
+                   host_victims, n_host_victims, prefetch_ids, n_prefetch, stream=None):
+    _chk(lib().cs_select_step(ctx, C.byref(idx), now, k_victims, k_prefetch, _ptr(gpu_victims), _ptr(n_gpu_victims),
+                              _ptr(host_victims), _ptr(n_host_victims), _ptr(prefetch_ids), _ptr(n_prefetch),
+                              _stream(stream)), "cs_select_step", ctx)
 
 
 def cs_step(ctx, io: cs_step_io, main=None, side=None):
@@ -389,6 +397,12 @@ class CacheScout:
             n_out = torch.empty(1, dtype=torch.int32, device=self.device)
         cs_select_prefetch(self.ctx, idx.struct(), now, k, ids_out, n_out, stream)
         return ids_out, n_out
+
+    def select_step(self, idx: DeviceIndex, now: int, k_victims: int, k_prefetch: int, gpu_victims, n_gpu_victims,
+                    host_victims, n_host_victims, prefetch_ids, n_prefetch, stream=None):
+        """GPU-tier victims, host-tier victims and prefetch candidates of one step at once."""
+        cs_select_step(self.ctx, idx.struct(), now, k_victims, k_prefetch, gpu_victims, n_gpu_victims, host_victims,
+                       n_host_victims, prefetch_ids, n_prefetch, stream)
 
     def offload_blocks(self, gpu: KVPool, host: KVPool, src_slots, dst_slots, n_max=None, n_dev=None, stream=None):
         cs_offload_blocks(self.ctx, gpu.struct(), host.struct(), src_slots, dst_slots,

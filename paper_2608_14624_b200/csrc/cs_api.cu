@@ -39,7 +39,7 @@ void cs_recency_table_shape(const cs_params *p, uint32_t *gtab_len, uint32_t *ag
     *gtab_len = *age_sat < CS_GTAB_MAX ? *age_sat : CS_GTAB_MAX;
 }
 
-size_t cs_layout_workspace(const cs_params *p, uint32_t gtab_len, void *base, cs_workspace *ws)
+size_t cs_layout_workspace(const cs_params *p, uint32_t gtab_len, void *base, cs_workspace *ws, cs_workspace *ws_job)
 {
     const size_t A = p->n_agents, W = (A + 31) / 32, N = p->max_blocks;
     size_t off = 0;
@@ -74,6 +74,28 @@ size_t cs_layout_workspace(const cs_params *p, uint32_t gtab_len, void *base, cs
     TAKE(spl_id, uint32_t, CS_MAX_SPLITTERS + 1);
     TAKE(bcount, uint32_t, CS_MAX_SPLITTERS + 1);
     TAKE(boff, uint32_t, CS_MAX_SPLITTERS + 2);
+    if (ws) ws->job = ws->sc->sel_job[0];
+    // private candidate / sort regions for the second and third select of a fused launch (cluster path only,
+    // so at most CS_SELECT_CLUSTER_MAX_BLOCKS entries each)
+    const size_t Nc = N < CS_SELECT_CLUSTER_MAX_BLOCKS ? N : CS_SELECT_CLUSTER_MAX_BLOCKS;
+    for (int j = 0; j < 2; ++j) {
+        cs_workspace *const all = ws;
+        cs_workspace *const mine = (all && ws_job) ? &ws_job[j] : nullptr;
+        if (mine) *mine = *all;
+        ws = mine;                             // TAKE fills `mine`, or only advances the offset
+        TAKE(cand_km, unsigned long long, Nc);
+        TAKE(cand_id, uint32_t, Nc);
+        TAKE(cand_bkt, uint32_t, Nc);
+        TAKE(cand_slot, uint32_t, Nc);
+        TAKE(sort_km, unsigned long long, Nc);
+        TAKE(sort_id, uint32_t, Nc);
+        TAKE(spl_km, unsigned long long, CS_MAX_SPLITTERS + 1);
+        TAKE(spl_id, uint32_t, CS_MAX_SPLITTERS + 1);
+        TAKE(bcount, uint32_t, CS_MAX_SPLITTERS + 1);
+        TAKE(boff, uint32_t, CS_MAX_SPLITTERS + 2);
+        if (mine) mine->job = all->sc->sel_job[j + 1];
+        ws = all;
+    }
 #undef TAKE
     return off;
 }
@@ -129,7 +151,7 @@ int cs_workspace_bytes(const cs_params *p, size_t *dev_bytes)
     if (!dev_bytes) return CS_EINVAL;
     uint32_t gl, as;
     cs_recency_table_shape(p, &gl, &as);
-    *dev_bytes = cs_layout_workspace(p, gl, nullptr, nullptr);
+    *dev_bytes = cs_layout_workspace(p, gl, nullptr, nullptr, nullptr);
     return CS_OK;
 }
 
@@ -140,7 +162,7 @@ int cs_create(const cs_params *p, void *dev_workspace, size_t bytes, cs_stream_t
     if (!out || !dev_workspace || (((uintptr_t)dev_workspace) & 255u)) return CS_EINVAL;
     uint32_t gl, as;
     cs_recency_table_shape(p, &gl, &as);
-    size_t need = cs_layout_workspace(p, gl, nullptr, nullptr);
+    size_t need = cs_layout_workspace(p, gl, nullptr, nullptr, nullptr);
     if (bytes < need) return CS_ECAPACITY;
     cs_ctx *ctx = new (std::nothrow) cs_ctx;
     if (!ctx) return CS_ENOMEM;
@@ -149,7 +171,7 @@ int cs_create(const cs_params *p, void *dev_workspace, size_t bytes, cs_stream_t
     ctx->gtab_len = gl;
     ctx->age_sat = as;
     ctx->W = (p->n_agents + 31) / 32;
-    ctx->ws_bytes = cs_layout_workspace(p, gl, dev_workspace, &ctx->ws);
+    ctx->ws_bytes = cs_layout_workspace(p, gl, dev_workspace, &ctx->ws, ctx->ws_job);
     cudaError_t e = cudaGetDevice(&ctx->device);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, ctx->device);
     if (e != cudaSuccess) { delete ctx; return CS_ECUDA; }
@@ -239,6 +261,31 @@ int cs_select_prefetch(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, uin
     return select_common(ctx, idx, now, 1, 1, k, ids_out, n_out, stream);
 }
 
+int cs_select_step(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, uint32_t k_victims, uint32_t k_prefetch,
+                   uint32_t *gpu_victims, uint32_t *n_gpu_victims, uint32_t *host_victims, uint32_t *n_host_victims,
+                   uint32_t *prefetch_ids, uint32_t *n_prefetch, cs_stream_t stream)
+{
+    if (!ctx) return CS_EINVAL;
+    int rc = check_index(ctx, idx);
+    if (rc != CS_OK) return rc;
+    if (k_victims > ctx->p.max_blocks || k_prefetch > ctx->p.max_blocks) return CS_ECAPACITY;
+    uint32_t *const cnt[3] = {n_gpu_victims, n_host_victims, n_prefetch};
+    uint32_t *const ids[3] = {gpu_victims, host_victims, prefetch_ids};
+    for (int q = 0; q < 3; ++q) {
+        if (!cnt[q] || (((uintptr_t)cnt[q]) & 3u)) return CS_EINVAL;
+        if ((q == 2 ? k_prefetch : k_victims) && (!ids[q] || !aligned16(ids[q]))) return CS_EINVAL;
+    }
+    cudaStream_t s = (cudaStream_t)stream;
+    rc = cs_launch_select_step(ctx, idx, now, k_victims, k_prefetch, gpu_victims, n_gpu_victims, host_victims,
+                               n_host_victims, prefetch_ids, n_prefetch, s);
+    if (rc != CS_ENOTIMPL) return rc;
+    // no single-launch form for this index size, path setting or device: three calls
+    rc = cs_launch_select(ctx, idx, now, 0, 0, k_victims, gpu_victims, n_gpu_victims, s);
+    if (rc == CS_OK) rc = cs_launch_select(ctx, idx, now, 0, 1, k_victims, host_victims, n_host_victims, s);
+    if (rc == CS_OK) rc = cs_launch_select(ctx, idx, now, 1, 1, k_prefetch, prefetch_ids, n_prefetch, s);
+    return rc;
+}
+
 static int check_pools(const cs_kv_pool *a, const cs_kv_pool *b)
 {
     if (!a || !b || !a->base || !b->base) return CS_EINVAL;
@@ -314,9 +361,9 @@ int cs_step(cs_ctx *ctx, const cs_step_io *io, cs_stream_t main_, cs_stream_t si
     ctx->step_now_dev = io->now_dev;
     ctx->step_n_events_dev = io->n_events_dev;
     int rc = cs_observe_invocations(ctx, io->chain, io->agent, io->evflags, io->n_events, main_);
-    if (rc == CS_OK) rc = cs_select_victims(ctx, io->idx, io->now, 0, io->k_victims, io->gpu_victims, io->n_gpu_victims, main_);
-    if (rc == CS_OK) rc = cs_select_victims(ctx, io->idx, io->now, 1, io->k_victims, io->host_victims, io->n_host_victims, main_);
-    if (rc == CS_OK) rc = cs_select_prefetch(ctx, io->idx, io->now, io->k_prefetch, io->prefetch_ids, io->n_prefetch, main_);
+    if (rc == CS_OK)
+        rc = cs_select_step(ctx, io->idx, io->now, io->k_victims, io->k_prefetch, io->gpu_victims, io->n_gpu_victims,
+                            io->host_victims, io->n_host_victims, io->prefetch_ids, io->n_prefetch, main_);
     ctx->step_now_dev = nullptr;
     ctx->step_n_events_dev = nullptr;
     if (rc != CS_OK) return rc;

@@ -47,10 +47,11 @@ struct cs_scalars {
                             // threshold (set after a miss: that kind's threshold is moving upwards or jitters)
     uint32_t sel_c_spec;    // candidates appended speculatively by the histogram pass; 0 between calls
     uint32_t sel_spec;      // 1: the speculative candidates cover the k winners, the collect pass is skipped
-    uint32_t sel_cc[2];     // candidate counters of the cluster kernel: a call uses one and clears the other for
-                            // the next call, so that the counter is zero on entry without a barrier
-    uint32_t sel_toggle;    // which of the two the next cluster select uses; flipped by every call on the device, so
-                            // that a captured sequence of calls stays consistent when it is replayed
+    uint32_t sel_job[3][4]; // per concurrent cluster select (the fused launch of a step runs three): two candidate
+                            // counters -- a call uses one and clears the other for the next call, so that the counter is
+                            // zero on entry without a barrier --, which of the two the next call uses (flipped by every
+                            // call on the device, so that a captured sequence stays consistent when replayed), and the
+                            // number of candidates of the last call (inspection only)
     unsigned long long t_phase[8];   // globaltimer stamps of the last cluster select (phase boundaries, ns)
 };
 
@@ -81,11 +82,13 @@ struct cs_workspace {
     uint32_t *spl_id;     // [CS_MAX_SPLITTERS+1]
     uint32_t *bcount;     // [CS_MAX_SPLITTERS+1]
     uint32_t *boff;       // [CS_MAX_SPLITTERS+2]
+    uint32_t *job;        // this call's row of cs_scalars::sel_job
 };
 
 struct cs_ctx {
     cs_params p;
     cs_workspace ws;
+    cs_workspace ws_job[2];        // the same workspace with private candidate / sort regions: jobs 1 and 2 of a fused select
     size_t ws_bytes;
     uint32_t W;            // adjacency words per row
     uint32_t gtab_len;     // ages [0, gtab_len) come from the table
@@ -99,6 +102,7 @@ struct cs_ctx {
     uint32_t source_mode;          // CS_SOURCES_*: where the cached BFS of Eq. 8 starts
     const float *fsurv_override;   // caller's survival table for score / select, NULL = the BFS table of Eq. 8
     int cluster_max_v, cluster_max_pf;   // largest usable cluster of the single-launch select (0 = not probed, -1 = none)
+    int cluster_max_step;                // same for the fused three-select launch
     int bulk_attr_set;     // shared-memory opt-in of the bulk kernel done on this device
     int collect_attr_set;  // same for the collect kernel with age limits
     const uint32_t *step_now_dev;        // set only while cs_step() issues its calls: device-resident clock / event count
@@ -109,7 +113,7 @@ struct cs_ctx {
 };
 
 // ---- workspace layout (host) -------------------------------------------------------------------
-size_t cs_layout_workspace(const cs_params *p, uint32_t gtab_len, void *base, cs_workspace *ws);
+size_t cs_layout_workspace(const cs_params *p, uint32_t gtab_len, void *base, cs_workspace *ws, cs_workspace *ws_job);
 int cs_validate_params(const cs_params *p);
 void cs_recency_table_shape(const cs_params *p, uint32_t *gtab_len, uint32_t *age_sat);
 
@@ -124,6 +128,11 @@ int cs_launch_score(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, const 
                     float *scores_out, cudaStream_t s);
 int cs_launch_select(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, int prefetch, uint32_t tier,
                      uint32_t k, uint32_t *ids_out, uint32_t *n_out, cudaStream_t s);
+int cs_launch_select_step(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, uint32_t k_victims, uint32_t k_prefetch,
+                          uint32_t *gpu_victims, uint32_t *n_gpu, uint32_t *host_victims, uint32_t *n_host,
+                          uint32_t *prefetch_ids, uint32_t *n_prefetch, cudaStream_t s);
+int cs_launch_select_cluster3(cs_ctx *ctx, const void *sel_args3, uint32_t *const ids_out[3], uint32_t *const n_out[3],
+                              cudaStream_t s);
 int cs_launch_select_cluster(cs_ctx *ctx, const void *sel_args, int prefetch, uint32_t *ids_out, uint32_t *n_out,
                              cudaStream_t s);
 int cs_launch_mover(cs_ctx *ctx, const cs_kv_pool *src, const cs_kv_pool *dst, const uint32_t *src_slots,

@@ -148,16 +148,40 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
     }
     return false;
 }
-__device__ __forceinline__ void bulk_load(uint32_t dst_smem, const void *src, uint32_t bytes, uint32_t bar)
+// KV blocks stream through once: both directions of every copy carry an evict-first L2 policy, so the
+// gigabytes a step moves do not push the (L2-resident) block index and tables of the select kernels out.
+#ifndef TM_EVICT_FIRST
+#define TM_EVICT_FIRST 1
+#endif
+__device__ __forceinline__ unsigned long long l2_stream_policy()
 {
+    unsigned long long pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+__device__ __forceinline__ void bulk_load(uint32_t dst_smem, const void *src, uint32_t bytes, uint32_t bar,
+                                          unsigned long long pol)
+{
+#if TM_EVICT_FIRST
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(dst_smem),
+                 "l"(src), "r"(bytes), "r"(bar), "l"(pol)
+                 : "memory");
+#else
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst_smem),
                  "l"(src), "r"(bytes), "r"(bar)
                  : "memory");
+#endif
 }
-__device__ __forceinline__ void bulk_store(void *dst, uint32_t src_smem, uint32_t bytes)
+__device__ __forceinline__ void bulk_store(void *dst, uint32_t src_smem, uint32_t bytes, unsigned long long pol)
 {
+#if TM_EVICT_FIRST
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group.L2::cache_hint [%0], [%1], %2, %3;" ::"l"(dst), "r"(src_smem),
+                 "r"(bytes), "l"(pol)
+                 : "memory");
+#else
     asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src_smem), "r"(bytes)
                  : "memory");
+#endif
 }
 
 // One pipeline per warp, driven by lane 0.  Iteration `it` first stores item it-(STAGES-1)
@@ -169,6 +193,7 @@ __device__ __forceinline__ void bulk_pipeline(unsigned char *my_ring, const uint
                                               unsigned long long n_items, uint32_t *status, Item item)
 {
     constexpr int LAG = TM_STAGES - 1;
+    const unsigned long long pol = l2_stream_policy();
     char *dst_of[TM_STAGES];          // destination of the item loaded into each ring slot
     uint32_t bytes_of[TM_STAGES];
     uint32_t phase_bits = 0;          // parity to wait for, one bit per ring slot
@@ -186,7 +211,7 @@ __device__ __forceinline__ void bulk_pipeline(unsigned char *my_ring, const uint
                 pending &= ~(1u << st);
                 phase_bits ^= 1u << st;
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                bulk_store(dst_of[st], smem_u32(my_ring + (size_t)st * TM_PIECE), bytes_of[st]);
+                bulk_store(dst_of[st], smem_u32(my_ring + (size_t)st * TM_PIECE), bytes_of[st], pol);
             }
             // one group per item, empty for a skipped item, so that group counts match item counts
             asm volatile("cp.async.bulk.commit_group;" ::: "memory");
@@ -204,7 +229,7 @@ __device__ __forceinline__ void bulk_pipeline(unsigned char *my_ring, const uint
                 bytes_of[st] = bytes;
                 pending |= 1u << st;
                 mbar_expect_tx(bar[st], bytes);
-                bulk_load(smem_u32(my_ring + (size_t)st * TM_PIECE), sp, bytes, bar[st]);
+                bulk_load(smem_u32(my_ring + (size_t)st * TM_PIECE), sp, bytes, bar[st], pol);
             }
         }
     }

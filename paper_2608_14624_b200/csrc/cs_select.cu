@@ -611,6 +611,24 @@ int cs_launch_score(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, const 
     return cs_check_launch(ctx);
 }
 
+// The three selects of a step as one launch (cluster path only; CS_ENOTIMPL tells the caller to make three calls).
+int cs_launch_select_step(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, uint32_t k_victims, uint32_t k_prefetch,
+                          uint32_t *gpu_victims, uint32_t *n_gpu, uint32_t *host_victims, uint32_t *n_host,
+                          uint32_t *prefetch_ids, uint32_t *n_prefetch, cudaStream_t s)
+{
+    if (ctx->select_path == CS_SELECT_MULTI || idx->n_blocks > CS_SELECT_CLUSTER_MAX_BLOCKS) return CS_ENOTIMPL;
+    SelArgs a[3];
+    for (int q = 0; q < 3; ++q) {
+        fill_args(ctx, idx, now, ctx->fsurv_override ? ctx->fsurv_override : ctx->ws.fsurv, a[q]);
+        a[q].tier = q == 0 ? 0u : 1u;
+        a[q].k = q == 2 ? k_prefetch : k_victims;
+        a[q].hint_slot = ctx->no_speculation ? 3u : (uint32_t)q;
+    }
+    uint32_t *const ids[3] = {gpu_victims, host_victims, prefetch_ids};
+    uint32_t *const cnt[3] = {n_gpu, n_host, n_prefetch};
+    return cs_launch_select_cluster3(ctx, a, ids, cnt, s);
+}
+
 int cs_launch_select(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, int prefetch, uint32_t tier, uint32_t k,
                      uint32_t *ids_out, uint32_t *n_out, cudaStream_t s)
 {
@@ -768,6 +786,7 @@ extern "C" int cs_select_victims_static(const cs_params *p, const float *fsurv, 
     ws.cand_slot = (uint32_t *)(base + CS_SO_CANDSLOT);
     ws.sort_id = (uint32_t *)(base + CS_SO_SORTID);
     ws.fsurv = const_cast<float *>(fsurv);             // input table, read only
+    ws.job = ws.sc->sel_job[0];
     cudaStream_t s = (cudaStream_t)stream;
     cs_static_prepare_kernel<<<16, 256, 0, s>>>(ws, ctx.gtab_len, p->lambda, p->delta);
     if ((rc = cs_check_launch(&ctx)) != CS_OK) return rc;

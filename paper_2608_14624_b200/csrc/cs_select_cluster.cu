@@ -109,18 +109,19 @@ __device__ __forceinline__ void csel_bitonic(unsigned long long *km, uint32_t *i
 
 __device__ __forceinline__ void csel_stamp(const cs_workspace &ws, uint32_t rank, int slot)
 {
-    if (rank == 0 && threadIdx.x == 0) {
+    if (rank == 0 && threadIdx.x == 0 && ws.job == ws.sc->sel_job[0]) {     // the first (or only) select of a launch
         unsigned long long t;
         asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
         ws.sc->t_phase[slot] = t;
     }
 }
 
+// One whole select by the calling cluster.  `ws` carries this select's private candidate / sort regions
+// and its row of per-call scalars, so several clusters of one launch can run different selects at once.
 template <bool PF>
-__global__ void __launch_bounds__(CSEL_THREADS, 1)
-cs_select_cluster_kernel(SelArgs a, cs_workspace ws, uint32_t *__restrict__ ids_out, uint32_t *__restrict__ n_out_dev)
+__device__ __forceinline__ void csel_body(SelArgs a, const cs_workspace &ws, uint32_t *__restrict__ ids_out,
+                                          uint32_t *__restrict__ n_out_dev, unsigned char *dsm)
 {
-    extern __shared__ __align__(16) unsigned char dsm[];
     resolve_now(a);
     cg::cluster_group cluster = cg::this_cluster();
     const uint32_t CL = cluster.num_blocks(), rank = cluster.block_rank();
@@ -130,9 +131,9 @@ cs_select_cluster_kernel(SelArgs a, cs_workspace ws, uint32_t *__restrict__ ids_
     Tables T;
     load_tables(a, ws, S.tables, T, PF && a.anchor);
     for (uint32_t i = tid; i < CS_HIST_BINS; i += CSEL_THREADS) S.hist[i] = 0;
-    const uint32_t c_slot = *(volatile uint32_t *)&ws.sc->sel_toggle & 1u;   // read here, before any CTA can flip it (first cluster barrier)
-    uint32_t *cand_count = &ws.sc->sel_cc[c_slot];            // zero on entry: the previous call cleared it
-    if (rank == 0 && tid == 0) ws.sc->sel_cc[c_slot ^ 1u] = 0;
+    const uint32_t c_slot = *(volatile uint32_t *)&ws.job[2] & 1u;   // read here, before any CTA can flip it (first cluster barrier)
+    uint32_t *cand_count = &ws.job[c_slot];                   // zero on entry: the previous call cleared it
+    if (rank == 0 && tid == 0) ws.job[c_slot ^ 1u] = 0;
     if (tid == 0) S.misc[1] = 0;
     __syncthreads();
     const bool enabled = !PF || prefetch_enabled(ws, a.A);
@@ -235,7 +236,7 @@ cs_select_cluster_kernel(SelArgs a, cs_workspace ws, uint32_t *__restrict__ ids_
         }
     }
     cluster.sync();
-    if (rank == 0 && tid == 0) ws.sc->sel_toggle = c_slot ^ 1u;      // every CTA has read it: the next call takes the other counter
+    if (rank == 0 && tid == 0) ws.job[2] = c_slot ^ 1u;       // every CTA has read it: the next call takes the other counter
     constexpr uint32_t PER = CS_HIST_BINS / CSEL_THREADS;
     uint32_t loc[PER], sum = 0;
 #pragma unroll
@@ -274,7 +275,7 @@ cs_select_cluster_kernel(SelArgs a, cs_workspace ws, uint32_t *__restrict__ ids_
         cluster.sync();
     }
     const uint32_t c = __ldcg(cand_count);
-    if (rank == 0 && tid == 0) ws.sc->sel_c = c;              // for inspection only
+    if (rank == 0 && tid == 0) ws.job[3] = c;                 // for inspection only
     csel_stamp(ws, rank, 3);
 
     // ---- phase 4, small: CTA 0 sorts everything in shared memory ---------------------------------------------
@@ -385,6 +386,33 @@ cs_select_cluster_kernel(SelArgs a, cs_workspace ws, uint32_t *__restrict__ ids_
     csel_stamp(ws, rank, 7);
 }
 
+template <bool PF>
+__global__ void __launch_bounds__(CSEL_THREADS, 1)
+cs_select_cluster_kernel(SelArgs a, cs_workspace ws, uint32_t *__restrict__ ids_out, uint32_t *__restrict__ n_out_dev)
+{
+    extern __shared__ __align__(16) unsigned char dsm[];
+    csel_body<PF>(a, ws, ids_out, n_out_dev, dsm);
+}
+
+// The three selects of a step in one launch: cluster q of the grid runs select q (GPU-tier victims,
+// host-tier victims, prefetch candidates).  The selects share the index and the tables and nothing else.
+struct SelJob {
+    SelArgs a;
+    cs_workspace ws;
+    uint32_t *ids_out, *n_out;
+    uint32_t prefetch;
+};
+struct SelJobs { SelJob j[3]; };
+
+__global__ void __launch_bounds__(CSEL_THREADS, 1) cs_select_step_kernel(const __grid_constant__ SelJobs jobs)
+{
+    extern __shared__ __align__(16) unsigned char dsm[];
+    const uint32_t q = blockIdx.x / cg::this_cluster().num_blocks();
+    const SelJob &J = jobs.j[q];
+    if (J.prefetch) csel_body<true>(J.a, J.ws, J.ids_out, J.n_out, dsm);
+    else csel_body<false>(J.a, J.ws, J.ids_out, J.n_out, dsm);
+}
+
 // ---------------------------------------------------------------------------------------------
 template <bool PF>
 static int launch_cluster(cs_ctx *ctx, const SelArgs &a, uint32_t *ids_out, uint32_t *n_out, cudaStream_t s)
@@ -424,6 +452,56 @@ static int launch_cluster(cs_ctx *ctx, const SelArgs &a, uint32_t *ids_out, uint
     cfg.gridDim = dim3(cl);
     attr[0].val.clusterDim.x = cl;
     cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, a, ctx->ws, ids_out, n_out);
+    ctx->n_launches++;
+    if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; return CS_ECUDA; }
+    return CS_OK;
+}
+
+int cs_launch_select_cluster3(cs_ctx *ctx, const void *sel_args3, uint32_t *const ids_out[3], uint32_t *const n_out[3],
+                              cudaStream_t s)
+{
+    const SelArgs *a3 = (const SelArgs *)sel_args3;
+    const size_t smem = csel_smem_bytes(a3[0].A, a3[0].gtab_len);
+    int &max_cl = ctx->cluster_max_step;
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.blockDim = dim3(CSEL_THREADS);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (max_cl == 0) {           // first use on this context: shared-memory opt-in, largest cluster of which three fit
+        cudaError_t e = cudaFuncSetAttribute(cs_select_step_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(cs_select_step_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+        if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; (void)cudaGetLastError(); max_cl = -1; return CS_ENOTIMPL; }
+        max_cl = -1;
+        for (int cl = CSEL_MAX_CLUSTER; cl >= 1; cl >>= 1) {
+            cfg.gridDim = dim3(3 * cl);
+            attr[0].val.clusterDim.x = cl;
+            int n_clusters = 0;
+            e = cudaOccupancyMaxActiveClusters(&n_clusters, cs_select_step_kernel, &cfg);
+            if (e == cudaSuccess && n_clusters >= 3) { max_cl = cl; break; }
+            (void)cudaGetLastError();
+        }
+    }
+    if (max_cl < 1) return CS_ENOTIMPL;
+    const uint32_t n_groups = a3[0].n / GRP;
+    int cl = 1;
+    while (cl < max_cl && (uint32_t)cl * CSEL_THREADS < n_groups) cl <<= 1;
+    cfg.gridDim = dim3(3 * cl);
+    attr[0].val.clusterDim.x = cl;
+    SelJobs jobs;
+    for (int q = 0; q < 3; ++q) {
+        jobs.j[q].a = a3[q];
+        jobs.j[q].ws = q == 0 ? ctx->ws : ctx->ws_job[q - 1];
+        jobs.j[q].ids_out = ids_out[q];
+        jobs.j[q].n_out = n_out[q];
+        jobs.j[q].prefetch = q == 2 ? 1u : 0u;
+    }
+    cudaError_t e = cudaLaunchKernelEx(&cfg, cs_select_step_kernel, jobs);
     ctx->n_launches++;
     if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; return CS_ECUDA; }
     return CS_OK;

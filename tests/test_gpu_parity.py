@@ -561,3 +561,34 @@ def test_survival_from_all_chains(name, n_inv):
     o.survival()
     H.compare_model(c, o)
     assert c.get_status() == 0
+
+
+# ---- the three selects of a step in one launch --------------------------------------------------------------
+@pytest.mark.parametrize("name,n,kv,kp", [
+    ("tiny", 2560, 32, 64), ("tiny", 0, 4, 4), ("tiny", 5, 8, 1), ("tiny", 1029, 1029, 700),
+    ("llama8b", 80000, 256, 384), ("llama8b", 80000, 9000, 6000), ("llama70b", 52000 + 5, 128, 192),
+    ("meta1m", 262144, 10000, 2000), ("meta1m", 300000, 500, 500)])
+@pytest.mark.parametrize("path", [cs.CS_SELECT_AUTO, cs.CS_SELECT_MULTI])
+def test_select_step_matches_three_calls_and_oracle(name, n, kv, kp, path):
+    """cs_select_step: one launch of three clusters where the single-launch select applies, three calls
+    elsewhere (300,000 entries, or the multi-launch path forced); lists bit-exact against the oracle, and
+    again on a second and third call with a later clock (remembered thresholds in play)."""
+    cfg = synth.CONFIGS[name]
+    c, o = warm_state(cfg, 800, max(n, 16), r_min=0.02)
+    c.set_select_path(path)
+    idx = synth.make_block_index(cfg, n=n, tier="random" if name == "meta1m" else "range")
+    d = cs.DeviceIndex.from_host(idx, DEV)
+    i32 = lambda m: torch.full((max(m, 4),), 7, dtype=torch.int32, device=DEV)
+    gv, gh, gp, gvn, ghn, gpn = i32(kv), i32(kv), i32(kp), i32(1), i32(1), i32(1)
+    l0 = c.launch_count()
+    for rep, now in enumerate((100_000, 100_001, 100_009)):
+        c.select_step(d, now, kv, kp, gv, gvn, gh, ghn, gp, gpn)
+        s64, s32 = o.scores(idx, now)
+        for got, got_n, k, (o_ids, o_n) in ((gv, gvn, kv, o.select_victims(idx, now, 0, kv, s32)),
+                                            (gh, ghn, kv, o.select_victims(idx, now, 1, kv, s32)),
+                                            (gp, gpn, kp, o.select_prefetch(idx, now, kp, s32))):
+            g = got.cpu().numpy().view(np.uint32)[:k]
+            assert H.assert_list_matches(g, int(got_n[0].item()), o_ids, o_n, s64) == 0, (rep, k)
+    fused = path == cs.CS_SELECT_AUTO and n <= 262144
+    assert c.launch_count() - l0 == (3 if fused else 3 * 3 * 5)
+    assert c.get_status() == 0
