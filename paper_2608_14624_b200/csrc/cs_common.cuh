@@ -153,6 +153,44 @@ static inline int cs_check_launch(cs_ctx *ctx)
 }
 
 #ifdef __CUDACC__
+// Programmatic dependent launch.  The chains of small kernels (observe -> normalise; histogram -> collect ->
+// bucket -> scatter -> rank) are bound by launch latency, so each kernel of a chain is launched with the
+// programmatic-serialisation attribute: its launch overlaps the tail of its predecessor, and its first
+// instruction waits until the predecessor grid has completed and its writes are visible.  A kernel launched
+// without the attribute executes the wait as a no-op.
+#ifndef CS_USE_PDL
+#define CS_USE_PDL 1
+#endif
+__device__ __forceinline__ void cs_wait_for_predecessor()
+{
+#if CS_USE_PDL
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+#endif
+}
+// Lets the successor's launch proceed; called once the calling CTA no longer competes for the SM.
+__device__ __forceinline__ void cs_release_successor()
+{
+#if CS_USE_PDL
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+#endif
+}
+
+template <class... KArgs, class... Args>
+static inline void cs_launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = CS_USE_PDL;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    (void)cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);       // the caller reads the error with cs_check_launch()
+}
+
 // Recency factor of Eq. 9 as every kernel computes it: fp64 exp and add, rounded once to fp32.
 __device__ __forceinline__ float cs_recency(float lambda, float delta, uint32_t age)
 {

@@ -58,6 +58,8 @@ cs_observe_kernel(cs_workspace ws, uint32_t A, uint32_t n_chains, const uint32_t
                   const uint16_t *__restrict__ agent, const uint8_t *__restrict__ evflags, uint32_t n_events,
                   const uint32_t *__restrict__ n_events_dev)
 {
+    cs_wait_for_predecessor();
+    cs_release_successor();
     if (n_events_dev) n_events = min(n_events, *n_events_dev);     // device-resident count (graph replay)
     __shared__ uint32_t s_chain[OBS_THREADS];
     __shared__ uint16_t s_agent[OBS_THREADS];     // CS_AGENT_NONE marks an event that is skipped
@@ -190,6 +192,8 @@ cs_normalise_kernel(cs_workspace ws, uint32_t A, uint32_t W, float eps, float ta
     __shared__ uint32_t s_front[32], s_visit[32], s_next[32];
     __shared__ bool s_is_last;
     const uint32_t tid = threadIdx.x;
+    cs_wait_for_predecessor();
+    cs_release_successor();
 
     // Column sums q_j = sum_i pi_i P_ij of Eq. 2 are accumulated by the row CTAs in 2^-60 fixed
     // point with integer atomics: integer addition commutes, so the sum is bit-identical from run
@@ -453,15 +457,14 @@ int cs_launch_observe(cs_ctx *ctx, const uint32_t *chain, const uint16_t *agent,
 {
     const cs_params &p = ctx->p;
     if (n_events) {
-        cs_observe_kernel<<<1, OBS_THREADS, 0, s>>>(ctx->ws, p.n_agents, p.n_chains, chain, agent, evflags, n_events,
-                                                ctx->step_n_events_dev);
+        cs_launch_chained(cs_observe_kernel, 1, OBS_THREADS, 0, s, ctx->ws, p.n_agents, p.n_chains, chain, agent, evflags,
+                          n_events, ctx->step_n_events_dev);
         int rc = cs_check_launch(ctx);
         if (rc != CS_OK) return rc;
     }
     const uint32_t grid = p.n_agents < 2u * (uint32_t)ctx->sm_count ? p.n_agents : 2u * (uint32_t)ctx->sm_count;
-    cs_normalise_kernel<<<grid, ROW_THREADS, 0, s>>>(ctx->ws, p.n_agents, ctx->W, p.eps, p.tau, p.r_min, p.e_max,
-                                                      p.delta, ctx->source_mode == CS_SOURCES_ALL_CHAINS ? 1u : 0u,
-                                                      p.n_chains);
+    cs_launch_chained(cs_normalise_kernel, grid, ROW_THREADS, 0, s, ctx->ws, p.n_agents, ctx->W, p.eps, p.tau, p.r_min,
+                      p.e_max, p.delta, ctx->source_mode == CS_SOURCES_ALL_CHAINS ? 1u : 0u, p.n_chains);
     return cs_check_launch(ctx);
 }
 

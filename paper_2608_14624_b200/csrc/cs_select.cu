@@ -118,6 +118,8 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_hist_kernel(SelArgs a, cs_
     __shared__ uint32_t s_part[SEL_THREADS];
     __shared__ uint32_t s_b0;
     __shared__ bool s_flag;
+    cs_wait_for_predecessor();
+    cs_release_successor();
     resolve_now(a);
     Tables T;
     load_tables(a, ws, smem, T, PF && a.anchor);
@@ -299,6 +301,8 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_collect_kernel(SelArgs a, 
     __shared__ unsigned long long s_km[CS_SAMPLE];
     __shared__ uint32_t s_id[CS_SAMPLE];
     __shared__ bool s_flag;
+    cs_wait_for_predecessor();
+    cs_release_successor();
     if (ws.sc->sel_spec) return;          // the histogram pass already collected the candidates
     resolve_now(a);
     Tables T;
@@ -411,6 +415,8 @@ __global__ void __launch_bounds__(256) cs_sel_bucket_kernel(cs_workspace ws)
     __shared__ bool s_flag;
     __shared__ uint32_t s_cnt[CS_MAX_SPLITTERS + 1], s_base[CS_MAX_SPLITTERS + 1];
     constexpr int ITEMS = 4;                                  // candidates per thread and reservation round
+    cs_wait_for_predecessor();
+    cs_release_successor();
     const uint32_t c = ws.sc->sel_c, n_spl = ws.sc->sel_n_spl;
     for (uint32_t j = threadIdx.x; j < n_spl; j += blockDim.x) { s_km[j] = ws.spl_km[j]; s_id[j] = ws.spl_id[j]; }
     s_cnt[threadIdx.x] = 0;
@@ -485,6 +491,8 @@ __global__ void __launch_bounds__(256) cs_sel_bucket_kernel(cs_workspace ws)
 __global__ void __launch_bounds__(256) cs_sel_scatter_kernel(cs_workspace ws)
 {
     __shared__ uint32_t s_off[CS_MAX_SPLITTERS + 1];
+    cs_wait_for_predecessor();
+    cs_release_successor();
     const uint32_t c = ws.sc->sel_c, b_last = ws.sc->sel_b_last;
     if (ws.sc->sel_p_end == 0) return;
     s_off[threadIdx.x] = ws.boff[threadIdx.x];
@@ -510,6 +518,8 @@ cs_sel_rank_kernel(cs_workspace ws, uint32_t k, uint32_t *__restrict__ ids_out, 
 {
     __shared__ unsigned long long t_km[RANK_TILE];
     __shared__ uint32_t t_id[RANK_TILE];
+    cs_wait_for_predecessor();
+    cs_release_successor();
     const uint32_t p_end = ws.sc->sel_p_end, n_out = ws.sc->sel_n_out, b_last = ws.sc->sel_b_last;
     const uint32_t gtid = blockIdx.x * blockDim.x + threadIdx.x, nth = gridDim.x * blockDim.x;
     for (uint32_t i = n_out + gtid; i < k; i += nth) ids_out[i] = CS_ID_NONE;
@@ -646,8 +656,8 @@ int cs_launch_select(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, int p
     const size_t sm = table_smem(ctx);
     int rc;
     const uint32_t grid_h = grid;
-    if (prefetch) cs_sel_hist_kernel<true><<<grid_h, SEL_THREADS, sm, s>>>(a, ctx->ws);
-    else cs_sel_hist_kernel<false><<<grid_h, SEL_THREADS, sm, s>>>(a, ctx->ws);
+    if (prefetch) cs_launch_chained(cs_sel_hist_kernel<true>, grid_h, SEL_THREADS, sm, s, a, ctx->ws);
+    else cs_launch_chained(cs_sel_hist_kernel<false>, grid_h, SEL_THREADS, sm, s, a, ctx->ws);
     if ((rc = cs_check_launch(ctx)) != CS_OK) return rc;
     // large indexes: the collect pass prefilters by age limits (one look-up per entry instead of the full key)
     const uint32_t n_cls = idx->n_tokens ? ctx->p.block_tokens : 1u;
@@ -663,14 +673,14 @@ int cs_launch_select(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, int p
             ctx->collect_attr_set = 1;
         }
     }
-    if (prefetch) cs_sel_collect_kernel<true><<<grid, SEL_THREADS, sm_collect, s>>>(a, ctx->ws);
-    else cs_sel_collect_kernel<false><<<grid, SEL_THREADS, sm_collect, s>>>(a, ctx->ws);
+    if (prefetch) cs_launch_chained(cs_sel_collect_kernel<true>, grid, SEL_THREADS, sm_collect, s, a, ctx->ws);
+    else cs_launch_chained(cs_sel_collect_kernel<false>, grid, SEL_THREADS, sm_collect, s, a, ctx->ws);
     if ((rc = cs_check_launch(ctx)) != CS_OK) return rc;
-    cs_sel_bucket_kernel<<<grid_c, 256, 0, s>>>(ctx->ws);
+    cs_launch_chained(cs_sel_bucket_kernel, grid_c, 256, 0, s, ctx->ws);
     if ((rc = cs_check_launch(ctx)) != CS_OK) return rc;
-    cs_sel_scatter_kernel<<<grid_c, 256, 0, s>>>(ctx->ws);
+    cs_launch_chained(cs_sel_scatter_kernel, grid_c, 256, 0, s, ctx->ws);
     if ((rc = cs_check_launch(ctx)) != CS_OK) return rc;
-    cs_sel_rank_kernel<<<CS_MAX_SPLITTERS + 1, 256, 0, s>>>(ctx->ws, k, ids_out, n_out);
+    cs_launch_chained(cs_sel_rank_kernel, CS_MAX_SPLITTERS + 1, 256, 0, s, ctx->ws, k, ids_out, n_out);
     return cs_check_launch(ctx);
 }
 
