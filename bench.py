@@ -943,6 +943,14 @@ def main():
         "roofline": {"kernel": "cs_mover_bulk_kernel (device-to-device compaction of the 256 victims, inside the step, while offload and prefetch run on the side streams)", "bound": "hbm",
                      "achieved": d2d_gbps, "peak": hbm_peak, "unit": "GB/s", "frac": d2d_gbps / hbm_peak, "traffic": traffic,
                      "peak_kind": "of %s" % peak_kind, "algorithmic_bytes_per_launch": 2 * w.k_v * bb, "ms_per_launch": t_c},
+        "roofline_dominant_kernel": {
+            "kernel": ("cs_exchange_bulk_kernel (offload 256 + prefetch 384 blocks in one launch): 98 % of the step's device time; "
+                       "bound by the host link, which is neither HBM nor a tensor pipe, so it is reported beside the HBM roofline above")
+                      if w.fused else "cs_mover_bulk_kernel, offload and prefetch launches",
+            "bound": "host link (PCIe Gen5 x16, both directions)", "achieved": value / world, "unit": "GB/s",
+            "peak": link["bidir_step_mix"], "frac": value / world / link["bidir_step_mix"],
+            "peak_kind": "measured in this run: two concurrent pinned cudaMemcpyAsync copies in the step's 2:3 out:in proportion",
+            "algorithmic_bytes_per_launch": w.bytes_per_step, "ms_per_launch": t_o if w.fused else max(t_o, t_p)},
         "host_link": {"peak_d2h_GBps": link["d2h"], "peak_h2d_GBps": link["h2d"], "peak_bidir_GBps": link["bidir"],
                       "peak_bidir_step_mix_GBps": link["bidir_step_mix"],
                       "how": "pinned cudaMemcpyAsync of 1 GiB, best of 10, same run; step_mix = 2/3 GiB out while 1 GiB comes in, "
