@@ -546,6 +546,13 @@ def mover_sweep(w, hbm_peak, link):
         d_src, d_dst_h = up(src.astype(np.uint32)), up(dst_h.astype(np.uint32))
         d_back = up((G - n + np.arange(n)).astype(np.uint32))              # disjoint from every src
         reps = 5 if n <= 512 else 3
+        # fair comparator for the latency-bound small batches: one contiguous pinned copy of the same size
+        tmp = torch.empty(n * bb, dtype=torch.uint8, device=dev)
+        hview = w.host_buf[:n * bb]
+        with torch.cuda.stream(side):
+            _, cp_o = time_call(torch, side, lambda: hview.copy_(tmp, non_blocking=True), reps)
+            _, cp_p = time_call(torch, side, lambda: tmp.copy_(hview, non_blocking=True), reps)
+        del tmp
         for lay_name, lay in (("layer_major", cs.CS_LAYER_MAJOR), ("block_major", cs.CS_BLOCK_MAJOR)):
             gp = cs.KVPool(w.gpu_buf, G, lay, L)
             med_o, best_o = time_call(torch, side, lambda: c.offload_blocks(gp, w.host_pool, d_src, d_dst_h, stream=side), reps)
@@ -555,6 +562,8 @@ def mover_sweep(w, hbm_peak, link):
             rows.append({"blocks": n, "gpu_layout": lay_name,
                          "offload_GBps": gb / (med_o / 1e3), "offload_frac_of_link": gb / (med_o / 1e3) / link["d2h"],
                          "prefetch_GBps": gb / (med_p / 1e3), "prefetch_frac_of_link": gb / (med_p / 1e3) / link["h2d"],
+                         "memcpy_same_size_d2h_GBps": gb / (cp_o / 1e3), "memcpy_same_size_h2d_GBps": gb / (cp_p / 1e3),
+                         "offload_frac_of_memcpy_same_size": cp_o / med_o, "prefetch_frac_of_memcpy_same_size": cp_p / med_p,
                          "d2d_GBps_rw": 2 * gb / (med_c / 1e3), "d2d_frac_of_hbm": 2 * gb / (med_c / 1e3) / hbm_peak,
                          "offload_ms": med_o, "prefetch_ms": med_p, "d2d_ms": med_c})
     return rows
