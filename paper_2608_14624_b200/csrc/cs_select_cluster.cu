@@ -155,51 +155,34 @@ __device__ __forceinline__ void csel_body(SelArgs a, const cs_workspace &ws, uin
     };
     auto scan = [&](bool do_hist, bool do_collect, uint32_t limit) {
         const uint32_t n_warps = cthreads >> 5;
-        const uint32_t n_iter = (n_tiles + n_warps - 1) / n_warps;       // whole warps stay in the shuffles
+        const uint32_t n_iter = (n_tiles + n_warps - 1) / n_warps;       // whole warps stay in the ballots
+        WarpStage st;
+        stage_init(st, S.km, S.id);                                      // the sort tile is free during the scans
         for (uint32_t it = 0; it < n_iter; ++it) {
             const uint32_t t = it * n_warps + (ctid >> 5);
-            uint32_t mask = 0;
             Group G;
+            uint32_t em = 0;
             if (t < n_tiles) {
                 load_group<PF>(a, t, lane, G);
-                const uint32_t em = group_elig<PF>(a, G);
+                em = group_elig<PF>(a, G);
+            }
+            if (!__any_sync(0xFFFFFFFFu, em != 0)) continue;
 #pragma unroll
-                for (int j = 0; j < GRP; ++j) {
-                    if (!((em >> j) & 1u)) continue;
-                    uint32_t pr, se;
+            for (int j = 0; j < GRP; ++j) {
+                uint32_t pr = 0, se = 0;
+                bool cand = false;
+                if ((em >> j) & 1u) {
                     const uint32_t tok = a.ntok ? grp_u8(G.tk, j) : a.block_tokens;
                     const uint32_t dp = (PF && a.anchor) ? grp_u16(G.dp0, G.dp1, j) : 0u;
                     if (entry_key_rest<PF>(a, T, &ws.sc->status, grp_u16(G.ag0, G.ag1, j), dp, grp_u8(G.fl, j), grp_u32(G, j), tok, pr, se)) {
                         if (do_hist) hist_add(pr);
-                        if (do_collect && (pr >> 20) <= limit) mask |= 1u << j;
+                        cand = (pr >> 20) <= limit;
                     }
                 }
-            }
-            if (!do_collect || !__any_sync(0xFFFFFFFFu, mask != 0)) continue;      // most warps hold no candidate at all
-            const uint32_t cnt = __popc(mask);
-            uint32_t incl = cnt;
-#pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, incl, d);
-                if (lane >= d) incl += v;
-            }
-            uint32_t base = 0;
-            if (lane == 31 && incl) base = atomicAdd(cand_count, incl);
-            base = __shfl_sync(0xFFFFFFFFu, base, 31);
-            uint32_t pos = base + incl - cnt;
-#pragma unroll
-            for (int j = 0; j < GRP; ++j) {
-                if (mask & (1u << j)) {
-                    uint32_t prj, se;
-                    const uint32_t tok = a.ntok ? grp_u8(G.tk, j) : a.block_tokens;
-                    const uint32_t dp = (PF && a.anchor) ? grp_u16(G.dp0, G.dp1, j) : 0u;
-                    entry_key_rest<PF>(a, T, &ws.sc->status, grp_u16(G.ag0, G.ag1, j), dp, grp_u8(G.fl, j), grp_u32(G, j), tok, prj, se);
-                    ws.cand_km[pos] = ((unsigned long long)prj << 32) | se;
-                    ws.cand_id[pos] = grp_id(t, lane, j);
-                    ++pos;
-                }
+                if (do_collect) stage_push(st, cand, pr, se, grp_id(t, lane, j), cand_count, ws.cand_km, ws.cand_id);
             }
         }
+        stage_flush(st, cand_count, ws.cand_km, ws.cand_id);
         if (ctid < a.n - t0) {                                 // ragged tail, one entry per thread
             const uint32_t i = t0 + ctid;
             uint32_t p, se;

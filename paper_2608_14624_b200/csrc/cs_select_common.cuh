@@ -240,6 +240,55 @@ __device__ __forceinline__ void for_each_eligible(const SelArgs &a, const Tables
     }
 }
 
+// Warp-private staging of candidates.  Inside the 16-entry loop of a scan every lane holds at most one
+// candidate per step; a ballot gives each its slot in the warp's shared-memory slice, with no atomic and no
+// second pass over the group.  A slice that is more than half full is appended to the global candidate
+// buffer: one atomic per flush, coalesced writes.  Every call below is made by all 32 lanes of the warp.
+#define STAGE_CAP 64u
+struct WarpStage {
+    unsigned long long *km;      // [STAGE_CAP]
+    uint32_t *id;                // [STAGE_CAP]
+    uint32_t n;                  // staged entries (same value in every lane)
+};
+
+__device__ __forceinline__ void stage_init(WarpStage &st, unsigned long long *km_all, uint32_t *id_all)
+{
+    const uint32_t warp = threadIdx.x >> 5;
+    st.km = km_all + warp * STAGE_CAP;
+    st.id = id_all + warp * STAGE_CAP;
+    st.n = 0;
+}
+
+__device__ __forceinline__ void stage_flush(WarpStage &st, uint32_t *counter, unsigned long long *out_km, uint32_t *out_id)
+{
+    if (st.n == 0) return;
+    const uint32_t lane = threadIdx.x & 31;
+    __syncwarp();
+    uint32_t base = 0;
+    if (lane == 0) base = atomicAdd(counter, st.n);
+    base = __shfl_sync(0xFFFFFFFFu, base, 0);
+    for (uint32_t i = lane; i < st.n; i += 32) {
+        out_km[base + i] = st.km[i];
+        out_id[base + i] = st.id[i];
+    }
+    __syncwarp();
+    st.n = 0;
+}
+
+__device__ __forceinline__ void stage_push(WarpStage &st, bool cand, uint32_t pr, uint32_t se, uint32_t id,
+                                           uint32_t *counter, unsigned long long *out_km, uint32_t *out_id)
+{
+    const uint32_t b = __ballot_sync(0xFFFFFFFFu, cand);
+    if (b == 0) return;
+    if (cand) {
+        const uint32_t pos = st.n + __popc(b & ((1u << (threadIdx.x & 31)) - 1u));
+        st.km[pos] = ((unsigned long long)pr << 32) | se;
+        st.id[pos] = id;
+    }
+    st.n += __popc(b);
+    if (st.n > STAGE_CAP - 32u) stage_flush(st, counter, out_km, out_id);
+}
+
 // The prefetch list is empty unless the gate of Eq. 11 is open and a current agent exists.
 __device__ __forceinline__ bool prefetch_enabled(const cs_workspace &ws, uint32_t A)
 {
