@@ -153,3 +153,65 @@ def test_step_argument_errors():
     with pytest.raises(cs.CacheScoutError) as e:
         cs.cs_step(c.ctx, cs.cs_step_io())                                   # no index, no pools
     assert e.value.code == cs.CS_EINVAL
+
+
+@pytest.mark.parametrize("kv,kp,same_stream,with_stage", [(32, 0, True, False), (0, 16, False, True), (8, 8, True, True)])
+def test_step_variants_one_step(kv, kp, same_stream, with_stage):
+    """One step with an empty list, without a staging pool, and with both transfers on the caller's one stream."""
+    cfg = synth.CONFIGS["tiny"]
+    G, Hs, L, chunk = cfg.gpu_blocks, cfg.host_blocks, cfg.n_layers, cfg.chunk_bytes
+    p = cs.make_params(n_agents=cfg.n_agents, n_chains=cfg.n_chains, max_blocks=cfg.n_index,
+                       block_tokens=cfg.block_tokens, r_min=0.02)
+    c, o = cs.CacheScout(p, DEV), orc.Oracle(H.oracle_params(p))
+    tr = synth.make_trace(cfg)
+    n0 = len(tr.agent) - 4
+    c.observe_invocations(dev(tr.chain[:n0]), dev(tr.agent[:n0]), dev(tr.evflags[:n0]))
+    o.observe(tr.chain[:n0], tr.agent[:n0], tr.evflags[:n0])
+    idx = synth.make_block_index(cfg, now0=1000)
+    free_np = np.arange(G - max(kp, 1), G, dtype=np.uint32)[:kp]
+    idx.flags[free_np.astype(np.int64)] &= np.uint8(~synth.FLAG_VALID & 0xFF)
+    d = cs.DeviceIndex.from_host(idx, DEV)
+    rng = synth.rng_for(cfg, 43)
+    gpu_np = synth.kv_pool_u16(G, L, chunk, rng).view(np.uint8)
+    host_np = synth.kv_pool_u16(Hs, L, chunk, rng).view(np.uint8)
+    gpu = cs.KVPool(dev(gpu_np), G, synth.BLOCK_MAJOR, L)
+    host_t = torch.from_numpy(host_np.copy()).pin_memory()
+    host = cs.KVPool(host_t, Hs, synth.LAYER_MAJOR, L, first_id=G)
+    ks = max(kv, 1)
+    stage = cs.KVPool(torch.zeros(ks * L * 2 * chunk, dtype=torch.uint8, device=DEV), ks, synth.LAYER_MAJOR, L) if with_stage else None
+    packed = torch.arange(ks, dtype=torch.int32, device=DEV)
+    gv, gh, gp, free_d = i32(kv, -1), i32(kv, -1), i32(kp, -1), i32(kp, -1)
+    if kp:
+        free_d[:kp] = dev(free_np.view(np.int32))
+    gvn, ghn, gpn = i32(1), i32(1), i32(1)
+    main = torch.cuda.Stream(device=DEV)
+    side = main if same_stream else torch.cuda.Stream(device=DEV)
+    main.wait_stream(torch.cuda.current_stream())
+    now = 1000 + 7
+    c.step(d, now, dev(tr.chain[n0:].view(np.int32)), dev(tr.agent[n0:].view(np.int16)), dev(tr.evflags[n0:]), 4, kv, kp,
+           gv, gvn, gh, ghn, gp, gpn, gpu, host, free_d, stage=stage, stage_slots=packed if with_stage else None,
+           main=main, side=side, join_main=not same_stream)
+    main.synchronize()
+    o.observe(tr.chain[n0:], tr.agent[n0:], tr.evflags[n0:])
+    H.compare_model(c, o)
+    s64, s32 = o.scores(idx, now)
+    ov, ovn = o.select_victims(idx, now, 0, kv, s32)
+    oh, ohn = o.select_victims(idx, now, 1, kv, s32)
+    op, opn = o.select_prefetch(idx, now, kp, s32)
+    n_off = min(ovn, ohn)
+    op = op.copy()
+    op[:opn][np.isin(op[:opn], oh[:n_off])] = orc.ID_NONE
+    as_u32 = lambda t, n: t.cpu().numpy().view(np.uint32)[:n]
+    assert int(gvn[0].item()) == ovn and np.array_equal(as_u32(gv, ovn), ov[:ovn])
+    assert int(ghn[0].item()) == ohn and np.array_equal(as_u32(gh, ohn), oh[:ohn])
+    assert int(gpn[0].item()) == opn and np.array_equal(as_u32(gp, opn), op[:opn])
+    want_g, want_h = gpu_np.copy(), host_np.copy()
+    orc.move_blocks(gpu_np, synth.BLOCK_MAJOR, G, want_h, synth.LAYER_MAJOR, Hs, L, chunk, ov[:n_off], oh[:n_off] - G)
+    ok = op[:opn] != orc.ID_NONE
+    orc.move_blocks(host_np, synth.LAYER_MAJOR, Hs, want_g, synth.BLOCK_MAJOR, G, L, chunk, op[:opn][ok] - G, free_np[:opn][ok])
+    assert np.array_equal(host_t.numpy(), want_h) and np.array_equal(gpu.buf.cpu().numpy(), want_g)
+    if with_stage and ovn:
+        want_s = np.zeros(ks * L * 2 * chunk, np.uint8)
+        orc.move_blocks(gpu_np, synth.BLOCK_MAJOR, G, want_s, synth.LAYER_MAJOR, ks, L, chunk, ov[:ovn], np.arange(ovn))
+        assert np.array_equal(stage.buf.cpu().numpy(), want_s)
+    assert c.get_status() == 0
