@@ -17,9 +17,9 @@
  *  - Block-index arrays, score / id output arrays and pool bases must be 16-byte aligned (the
  *    kernels use 128-bit accesses); event arrays, slot lists and counts need only their natural
  *    alignment.  A violation is CS_EINVAL before anything is launched.
- *  - All calls on one cs_ctx except the three mover calls share workspace scratch: issue
- *    them on one stream (or order them with events).  The mover calls touch no workspace
- *    scratch besides the status word and may run on a side stream concurrently.
+ *  - All calls on one cs_ctx except the mover calls (offload, prefetch, exchange, compact) share
+ *    workspace scratch: issue them on one stream (or order them with events).  The mover calls
+ *    touch no workspace scratch besides the status word and may run on a side stream concurrently.
  *  - Bad ids inside device arrays (agent >= n_agents, chain >= n_chains, slot >= n_slots)
  *    are detected in the kernels: the entry is skipped and a bit is set in the device
  *    status word (read with cs_get_status()).  Kernels never trap or spin unboundedly.
