@@ -610,6 +610,26 @@ def metadata_scale(torch, cs, synth, dev, hbm_peak, calls=200):
     launches = (c.launch_count() - l0) / (calls + 5)
     ms = np.array([a.elapsed_time(b) for a, b in evs])
     per_call = float(np.median(ms)) * 1e-3
+    # the same two selects issued as ONE call (cs_select_step without the host-tier victims): their kernel chains
+    # run side by side on the context's own streams
+    evs2 = []
+    for call in range(calls + 5, 2 * calls + 10):
+        now = 100_000 + call
+        lo = 64 * (30 + call % (calls + 5))
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        c.observe_invocations(ch[lo:lo + 64], ag[lo:lo + 64], None)
+        c.select_step(d, now, cfg.k_victims, cfg.k_prefetch, v, vn, None, None, pf, pn)
+        e1.record(stream)
+        la[v.long().clamp_(min=0)] = now
+        pi = pf.long().clamp_(min=0)
+        d.flags[pi] &= 0xFB
+        d.flags[fifo[call % 8]] |= 4
+        fifo[call % 8].copy_(pi)
+        if call >= calls + 10:
+            evs2.append((e0, e1))
+    torch.cuda.synchronize(dev)
+    per_call_sbs = float(np.median([a.elapsed_time(b) for a, b in evs2])) * 1e-3
     # the same call captured once into a CUDA graph and replayed (same events and clock every time: timing only)
     cap = torch.cuda.Stream(device=dev)
     cap.wait_stream(stream)
@@ -617,8 +637,7 @@ def metadata_scale(torch, cs, synth, dev, hbm_peak, calls=200):
     lo = 64 * 30
     with torch.cuda.graph(g, stream=cap, capture_error_mode="relaxed"):
         c.observe_invocations(ch[lo:lo + 64], ag[lo:lo + 64], None, stream=cap)
-        c.select_victims(d, 100_000, 0, cfg.k_victims, v, vn, stream=cap)
-        c.select_prefetch(d, 100_000, cfg.k_prefetch, pf, pn, stream=cap)
+        c.select_step(d, 100_000, cfg.k_victims, cfg.k_prefetch, v, vn, None, None, pf, pn, stream=cap)
     gms = []
     with torch.cuda.stream(cap):
         for call in range(calls + 5):
@@ -636,6 +655,7 @@ def metadata_scale(torch, cs, synth, dev, hbm_peak, calls=200):
             "calls_timed": calls, "us_per_call_median": per_call * 1e6, "us_per_call_min": float(ms.min()) * 1e3,
             "blocks_scored_selected_per_s": 2 * N / per_call,
             "algorithmic_GBps": algo_bytes / per_call / 1e9, "frac_of_hbm_peak": algo_bytes / per_call / 1e9 / hbm_peak,
+            "us_per_call_side_by_side": per_call_sbs * 1e6, "blocks_scored_selected_per_s_side_by_side": 2 * N / per_call_sbs,
             "us_per_call_graph_replay": graph_us,
             "kernel_launches_per_call": launches, "n_out": [int(vn[0].item()), int(pn[0].item())]}
 

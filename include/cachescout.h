@@ -224,10 +224,14 @@ int cs_exchange_blocks(cs_ctx *ctx, const cs_kv_pool *gpu, const cs_kv_pool *hos
                        const uint32_t *pre_host_slots, const uint32_t *pre_gpu_slots, uint32_t n_pre_max,
                        const uint32_t *n_pre_dev, cs_stream_t side);
 
-/* The three selections of a step at once: cs_select_victims(tier 0, k_victims), cs_select_victims(tier 1,
- * k_victims) and cs_select_prefetch(k_prefetch) over the same index and clock, with the same results.  For
- * index sizes the single-launch select covers (<= 262,144 entries) they run as ONE launch of three
- * thread-block clusters side by side; otherwise as the three calls in a row.  Arguments as for those calls. */
+/* The selections of a step at once: cs_select_victims(tier 0, k_victims), cs_select_victims(tier 1,
+ * k_victims) and cs_select_prefetch(k_prefetch) over the same index and clock, with the same results, run
+ * side by side.  A selection whose count pointer is NULL is left out.  For index sizes the single-launch
+ * select covers (<= 262,144 entries) they are the thread-block clusters of ONE launch; for larger indexes
+ * each is a chain of grid-wide kernels, the first on `stream` and the others on two streams the context owns,
+ * forked from and joined back into `stream` with events, so that to the caller everything is ordered on
+ * `stream` (beyond 4,194,304 entries the selections run one after the other: private scratch of that size
+ * is not reserved).  Arguments as for the single calls. */
 int cs_select_step(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, uint32_t k_victims, uint32_t k_prefetch,
                    uint32_t *gpu_victims, uint32_t *n_gpu_victims, uint32_t *host_victims, uint32_t *n_host_victims,
                    uint32_t *prefetch_ids, uint32_t *n_prefetch, cs_stream_t stream);

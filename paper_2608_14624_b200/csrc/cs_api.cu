@@ -50,6 +50,7 @@ size_t cs_layout_workspace(const cs_params *p, uint32_t gtab_len, void *base, cs
         off = align_up(off + sizeof(type) * (size_t)(count), 256); \
     } while (0)
     TAKE(sc, cs_scalars, 1);
+    TAKE(sel, cs_sel_state, 1);
     TAKE(C, uint32_t, A * A);
     TAKE(rowsum, uint32_t, A);
     TAKE(cur, uint16_t, p->n_chains);
@@ -74,15 +75,17 @@ size_t cs_layout_workspace(const cs_params *p, uint32_t gtab_len, void *base, cs
     TAKE(spl_id, uint32_t, CS_MAX_SPLITTERS + 1);
     TAKE(bcount, uint32_t, CS_MAX_SPLITTERS + 1);
     TAKE(boff, uint32_t, CS_MAX_SPLITTERS + 2);
-    if (ws) ws->job = ws->sc->sel_job[0];
-    // private candidate / sort regions for the second and third select of a fused launch (cluster path only,
-    // so at most CS_SELECT_CLUSTER_MAX_BLOCKS entries each)
-    const size_t Nc = N < CS_SELECT_CLUSTER_MAX_BLOCKS ? N : CS_SELECT_CLUSTER_MAX_BLOCKS;
+    // Private select state, histogram and candidate / sort regions for the second and third select of a step,
+    // which run beside the first one.  Full size up to CS_CONCURRENT_MAX_BLOCKS entries; beyond that only the
+    // single-launch cluster select (at most CS_SELECT_CLUSTER_MAX_BLOCKS entries) runs selects side by side.
+    const size_t Nc = N <= CS_CONCURRENT_MAX_BLOCKS ? N : CS_SELECT_CLUSTER_MAX_BLOCKS;
     for (int j = 0; j < 2; ++j) {
         cs_workspace *const all = ws;
         cs_workspace *const mine = (all && ws_job) ? &ws_job[j] : nullptr;
         if (mine) *mine = *all;
         ws = mine;                             // TAKE fills `mine`, or only advances the offset
+        TAKE(sel, cs_sel_state, 1);
+        TAKE(hist, uint32_t, CS_HIST_BINS);
         TAKE(cand_km, unsigned long long, Nc);
         TAKE(cand_id, uint32_t, Nc);
         TAKE(cand_bkt, uint32_t, Nc);
@@ -93,7 +96,6 @@ size_t cs_layout_workspace(const cs_params *p, uint32_t gtab_len, void *base, cs
         TAKE(spl_id, uint32_t, CS_MAX_SPLITTERS + 1);
         TAKE(bcount, uint32_t, CS_MAX_SPLITTERS + 1);
         TAKE(boff, uint32_t, CS_MAX_SPLITTERS + 2);
-        if (mine) mine->job = all->sc->sel_job[j + 1];
         ws = all;
     }
 #undef TAKE
@@ -177,10 +179,20 @@ int cs_create(const cs_params *p, void *dev_workspace, size_t bytes, cs_stream_t
     if (e != cudaSuccess) { delete ctx; return CS_ECUDA; }
     ctx->host_link_ctas = 0;
     ctx->d2d_ctas = 0;
-    // fork / join events of cs_step(): host objects, created here so that the call itself creates nothing
+    // fork / join events of cs_step() and the two extra streams (with their events) on which the second and third
+    // select of a step run: host objects, created here so that the calls themselves create nothing
     e = cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_join, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_sel_fork, cudaEventDisableTiming);
+    for (int j = 0; j < 2 && e == cudaSuccess; ++j) {
+        e = cudaStreamCreateWithFlags(&ctx->sel_stream[j], cudaStreamNonBlocking);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_sel_join[j], cudaEventDisableTiming);
+    }
     if (e != cudaSuccess) { cs_destroy(ctx); return CS_ECUDA; }
+    ctx->concurrent_selects = p->max_blocks <= CS_CONCURRENT_MAX_BLOCKS ? 1 : 0;
+    // everything that must start at zero (tickets, counters, histograms of all three select states)
+    e = cudaMemsetAsync(dev_workspace, 0, ctx->ws_bytes, (cudaStream_t)init_stream);
+    if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; cs_destroy(ctx); return CS_ECUDA; }
     rc = cs_launch_init(ctx, (cudaStream_t)init_stream);
     if (rc != CS_OK) { cs_destroy(ctx); return rc; }
     *out = ctx;
@@ -192,6 +204,11 @@ int cs_destroy(cs_ctx *ctx)
     if (!ctx) return CS_EINVAL;
     if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
     if (ctx->ev_join) cudaEventDestroy(ctx->ev_join);
+    if (ctx->ev_sel_fork) cudaEventDestroy(ctx->ev_sel_fork);
+    for (int j = 0; j < 2; ++j) {
+        if (ctx->ev_sel_join[j]) cudaEventDestroy(ctx->ev_sel_join[j]);
+        if (ctx->sel_stream[j]) cudaStreamDestroy(ctx->sel_stream[j]);
+    }
     delete ctx;
     return CS_OK;
 }
@@ -272,18 +289,12 @@ int cs_select_step(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, uint32_
     uint32_t *const cnt[3] = {n_gpu_victims, n_host_victims, n_prefetch};
     uint32_t *const ids[3] = {gpu_victims, host_victims, prefetch_ids};
     for (int q = 0; q < 3; ++q) {
-        if (!cnt[q] || (((uintptr_t)cnt[q]) & 3u)) return CS_EINVAL;
+        if (!cnt[q]) continue;                                   // this select is not wanted
+        if (((uintptr_t)cnt[q]) & 3u) return CS_EINVAL;
         if ((q == 2 ? k_prefetch : k_victims) && (!ids[q] || !aligned16(ids[q]))) return CS_EINVAL;
     }
-    cudaStream_t s = (cudaStream_t)stream;
-    rc = cs_launch_select_step(ctx, idx, now, k_victims, k_prefetch, gpu_victims, n_gpu_victims, host_victims,
-                               n_host_victims, prefetch_ids, n_prefetch, s);
-    if (rc != CS_ENOTIMPL) return rc;
-    // no single-launch form for this index size, path setting or device: three calls
-    rc = cs_launch_select(ctx, idx, now, 0, 0, k_victims, gpu_victims, n_gpu_victims, s);
-    if (rc == CS_OK) rc = cs_launch_select(ctx, idx, now, 0, 1, k_victims, host_victims, n_host_victims, s);
-    if (rc == CS_OK) rc = cs_launch_select(ctx, idx, now, 1, 1, k_prefetch, prefetch_ids, n_prefetch, s);
-    return rc;
+    return cs_launch_select_step(ctx, idx, now, k_victims, k_prefetch, gpu_victims, n_gpu_victims, host_victims,
+                                 n_host_victims, prefetch_ids, n_prefetch, (cudaStream_t)stream);
 }
 
 static int check_pools(const cs_kv_pool *a, const cs_kv_pool *b)
@@ -353,6 +364,7 @@ int cs_exchange_blocks(cs_ctx *ctx, const cs_kv_pool *gpu, const cs_kv_pool *hos
 int cs_step(cs_ctx *ctx, const cs_step_io *io, cs_stream_t main_, cs_stream_t side_)
 {
     if (!ctx || !io || !io->idx || !io->gpu || !io->host) return CS_EINVAL;
+    if (!io->n_gpu_victims || !io->n_host_victims || !io->n_prefetch) return CS_EINVAL;
     if ((io->now_dev && (((uintptr_t)io->now_dev) & 3u)) || (io->n_events_dev && (((uintptr_t)io->n_events_dev) & 3u)))
         return CS_EINVAL;
     if (io->stage && !io->stage_slots) return CS_EINVAL;

@@ -11,6 +11,8 @@
 
 #define CS_SELECT_CLUSTER_MAX_BLOCKS (1u << 18)   // above this the index is scanned by the whole grid instead
 
+#define CS_CONCURRENT_MAX_BLOCKS (1u << 22)        // up to this index size every select of a step has full-size scratch of its own
+
 #define CS_AGE_LIMIT_MIN_BLOCKS (1u << 21)        // index size from which the collect pass builds age limits
 
 #define CS_MOVE_D2D 0
@@ -30,34 +32,40 @@ struct cs_scalars {
     float R;                // Eq. 2
     uint32_t gate;          // Eq. 11: R >= r_min
     uint32_t n_transitions; // sum of all counts
-    uint32_t ticket[6];     // "last CTA done" counters, one per kernel that has an epilogue
-    // select state, rewritten by every select call
-    uint32_t sel_b0;        // threshold bin of the first digit
-    uint32_t sel_n_elig;    // eligible entries
-    uint32_t sel_c;         // candidates collected (first digit <= b0)
-    uint32_t sel_n_spl;     // splitters in use
-    uint32_t sel_b_last;    // last bucket that holds one of the k winners
-    uint32_t sel_p_end;     // end position of that bucket
-    uint32_t sel_n_out;     // min(k, eligible)
+    uint32_t ticket0;       // "last CTA done" counter of the learner refresh
     uint32_t gtab_monotone; // the recency table covers every unsaturated age and never increases with age
     uint32_t sel_hint[4];   // bin up to which the next select of each kind (GPU victims, host victims, prefetch)
                             // collects ahead: the previous threshold bin, plus one while sel_margin > 0; ~0 = none;
                             // slot 3 is never written: calls that must not speculate read it
     uint32_t sel_margin[4]; // per kind: calls left during which the next call collects one bin beyond the remembered
                             // threshold (set after a miss: that kind's threshold is moving upwards or jitters)
-    uint32_t sel_c_spec;    // candidates appended speculatively by the histogram pass; 0 between calls
-    uint32_t sel_spec;      // 1: the speculative candidates cover the k winners, the collect pass is skipped
-    uint32_t sel_job[3][4]; // per concurrent cluster select (the fused launch of a step runs three): two candidate
-                            // counters -- a call uses one and clears the other for the next call, so that the counter is
-                            // zero on entry without a barrier --, which of the two the next call uses (flipped by every
-                            // call on the device, so that a captured sequence stays consistent when replayed), and the
-                            // number of candidates of the last call (inspection only)
+};
+
+// State of one select in flight, rewritten by every call.  The selects of a step that run side by side each
+// have their own (with their own histogram, candidate and sort regions).
+struct cs_sel_state {
+    uint32_t ticket[6];     // "last CTA done" counters, one per kernel that has an epilogue (1..5 in use)
+    uint32_t b0;            // threshold bin of the first digit
+    uint32_t n_elig;        // eligible entries
+    uint32_t c;             // candidates collected (first digit <= b0)
+    uint32_t n_spl;         // splitters in use
+    uint32_t b_last;        // last bucket that holds one of the k winners
+    uint32_t p_end;         // end position of that bucket
+    uint32_t n_out;         // min(k, eligible)
+    uint32_t c_spec;        // candidates appended speculatively by the histogram pass; 0 between calls
+    uint32_t spec;          // 1: the speculative candidates cover the k winners, the collect pass is skipped
+    uint32_t cc[2];         // candidate counters of the cluster kernel: a call uses one and clears the other for the
+                            // next call, so that the counter is zero on entry without a barrier
+    uint32_t toggle;        // which of the two the next call uses; flipped by every call on the device, so that a
+                            // captured sequence of calls stays consistent when it is replayed
+    uint32_t cluster_c;     // candidates of the last cluster select (inspection only)
     unsigned long long t_phase[8];   // globaltimer stamps of the last cluster select (phase boundaries, ns)
 };
 
 // Device pointers into the caller's workspace.
 struct cs_workspace {
     cs_scalars *sc;
+    cs_sel_state *sel;    // this select's state (one per concurrent select)
     uint32_t *C;          // [A*A] transition counts
     uint32_t *rowsum;     // [A]
     uint16_t *cur;        // [n_chains]
@@ -82,7 +90,6 @@ struct cs_workspace {
     uint32_t *spl_id;     // [CS_MAX_SPLITTERS+1]
     uint32_t *bcount;     // [CS_MAX_SPLITTERS+1]
     uint32_t *boff;       // [CS_MAX_SPLITTERS+2]
-    uint32_t *job;        // this call's row of cs_scalars::sel_job
 };
 
 struct cs_ctx {
@@ -107,7 +114,10 @@ struct cs_ctx {
     int collect_attr_set;  // same for the collect kernel with age limits
     const uint32_t *step_now_dev;        // set only while cs_step() issues its calls: device-resident clock / event count
     const uint32_t *step_n_events_dev;
-    cudaEvent_t ev_fork, ev_join;        // cs_step(): main -> side and side -> main, created on first use
+    cudaEvent_t ev_fork, ev_join;        // cs_step(): main -> side and side -> main
+    cudaStream_t sel_stream[2];          // the second and third select of a step run here, beside the first
+    cudaEvent_t ev_sel_fork, ev_sel_join[2];
+    int concurrent_selects;              // the per-select scratch regions are full size
     uint64_t n_launches;
     int last_cuda_error;
 };
@@ -131,10 +141,10 @@ int cs_launch_select(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, int p
 int cs_launch_select_step(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, uint32_t k_victims, uint32_t k_prefetch,
                           uint32_t *gpu_victims, uint32_t *n_gpu, uint32_t *host_victims, uint32_t *n_host,
                           uint32_t *prefetch_ids, uint32_t *n_prefetch, cudaStream_t s);
-int cs_launch_select_cluster3(cs_ctx *ctx, const void *sel_args3, uint32_t *const ids_out[3], uint32_t *const n_out[3],
-                              cudaStream_t s);
-int cs_launch_select_cluster(cs_ctx *ctx, const void *sel_args, int prefetch, uint32_t *ids_out, uint32_t *n_out,
-                             cudaStream_t s);
+int cs_launch_select_clusters(cs_ctx *ctx, int n_jobs, const void *sel_args, const uint32_t *prefetch,
+                              uint32_t *const *ids_out, uint32_t *const *n_out, cudaStream_t s);
+int cs_launch_select_cluster(cs_ctx *ctx, const void *sel_args, const cs_workspace *ws, int prefetch, uint32_t *ids_out,
+                             uint32_t *n_out, cudaStream_t s);
 int cs_launch_mover(cs_ctx *ctx, const cs_kv_pool *src, const cs_kv_pool *dst, const uint32_t *src_slots,
                     const uint32_t *dst_slots, uint32_t n_max, const uint32_t *n_dev, int kind,
                     cudaStream_t s);

@@ -243,7 +243,7 @@ cs_normalise_kernel(cs_workspace ws, uint32_t A, uint32_t W, float eps, float ta
     __threadfence();
     __syncthreads();
     if (tid == 0) {
-        const uint32_t t = atomicAdd(&ws.sc->ticket[0], 1u);
+        const uint32_t t = atomicAdd(&ws.sc->ticket0, 1u);
         s_is_last = (t == gridDim.x - 1);
     }
     __syncthreads();
@@ -270,7 +270,7 @@ cs_normalise_kernel(cs_workspace ws, uint32_t A, uint32_t W, float eps, float ta
         const float Rf = (float)R;
         ws.sc->R = Rf;
         ws.sc->gate = (Rf >= r_min) ? 1u : 0u;
-        ws.sc->ticket[0] = 0;
+        ws.sc->ticket0 = 0;
     }
     if (all_chains) {
         // sources: the current agent of every chain that has one (all live sessions)

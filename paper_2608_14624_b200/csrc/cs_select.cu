@@ -97,7 +97,7 @@ __device__ __forceinline__ void publish_splitters(const cs_workspace &ws, unsign
         }
         ws.bcount[j] = 0;
     }
-    if (threadIdx.x == 0) ws.sc->sel_n_spl = n_spl;
+    if (threadIdx.x == 0) ws.sel->n_spl = n_spl;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -166,7 +166,7 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_hist_kernel(SelArgs a, cs_
                 if (lane >= d) incl += v;
             }
             uint32_t base = 0;
-            if (lane == 31 && incl) base = atomicAdd(&ws.sc->sel_c_spec, incl);
+            if (lane == 31 && incl) base = atomicAdd(&ws.sel->c_spec, incl);
             base = __shfl_sync(0xFFFFFFFFu, base, 31);
             uint32_t pos = base + incl - cnt;
 #pragma unroll
@@ -190,7 +190,7 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_hist_kernel(SelArgs a, cs_
             if (entry_key<PF>(a, T, &ws.sc->status, a.agent[i], a.depth[i], a.ref[i], a.flags[i], a.la[i], tok, pr, se)) {
                 add(pr >> 20);
                 if (hint != 0xFFFFFFFFu && (pr >> 20) <= hint) {
-                    const uint32_t pos = atomicAdd(&ws.sc->sel_c_spec, 1u);
+                    const uint32_t pos = atomicAdd(&ws.sel->c_spec, 1u);
                     ws.cand_km[pos] = ((unsigned long long)pr << 32) | se;
                     ws.cand_id[pos] = i;
                 }
@@ -203,7 +203,7 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_hist_kernel(SelArgs a, cs_
         const uint32_t v = s_hist[i];
         if (v) atomicAdd(&ws.hist[i], v);
     }
-    if (!last_cta_done(&ws.sc->ticket[1], &s_flag)) return;
+    if (!last_cta_done(&ws.sel->ticket[1], &s_flag)) return;
 
     // ---- last CTA: threshold bin = first bin whose inclusive running count reaches k ------------
     constexpr uint32_t PER = CS_HIST_BINS / SEL_THREADS;
@@ -236,18 +236,18 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_hist_kernel(SelArgs a, cs_
     __syncthreads();
     const uint32_t b0 = s_b0;
     const bool spec_ok = hint != 0xFFFFFFFFu && b0 != 0xFFFFFFFFu && b0 <= hint;
-    const uint32_t c_spec = __ldcg(&ws.sc->sel_c_spec);
+    const uint32_t c_spec = __ldcg(&ws.sel->c_spec);
     if (spec_ok)                                             // the shared histogram is free now: it holds the sample
         publish_splitters(ws, (unsigned long long *)s_hist, s_hist + 2 * CS_SAMPLE, c_spec);
     if (threadIdx.x == 0) {
-        ws.sc->sel_b0 = b0;
-        ws.sc->sel_n_elig = total;
-        ws.sc->sel_n_out = total < a.k ? total : a.k;
-        ws.sc->sel_c = spec_ok ? c_spec : 0;
-        ws.sc->sel_c_spec = 0;
-        ws.sc->sel_spec = spec_ok ? 1u : 0u;
+        ws.sel->b0 = b0;
+        ws.sel->n_elig = total;
+        ws.sel->n_out = total < a.k ? total : a.k;
+        ws.sel->c = spec_ok ? c_spec : 0;
+        ws.sel->c_spec = 0;
+        ws.sel->spec = spec_ok ? 1u : 0u;
         remember_threshold(ws.sc, a.hint_slot, a.k && total >= a.k, b0, hint != 0xFFFFFFFFu, spec_ok);
-        ws.sc->ticket[1] = 0;
+        ws.sel->ticket[1] = 0;
     }
 }
 
@@ -303,12 +303,12 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_collect_kernel(SelArgs a, 
     __shared__ bool s_flag;
     cs_wait_for_predecessor();
     cs_release_successor();
-    if (ws.sc->sel_spec) return;          // the histogram pass already collected the candidates
+    if (ws.sel->spec) return;          // the histogram pass already collected the candidates
     resolve_now(a);
     Tables T;
     load_tables(a, ws, smem, T, PF && a.anchor);
     __syncthreads();
-    const uint32_t b0 = ws.sc->sel_b0;
+    const uint32_t b0 = ws.sel->b0;
     const uint32_t lane = threadIdx.x & 31;
     const uint32_t n_cls = a.ntok ? a.block_tokens : 1u;     // size classes: tok = 1 .. block_tokens (or the constant)
     const bool limits = a.use_age_limits && ws.sc->gtab_monotone && b0 != 0xFFFFFFFFu;
@@ -365,7 +365,7 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_collect_kernel(SelArgs a, 
                 if (lane >= d) incl += v;
             }
             uint32_t base = 0;
-            if (lane == 31 && incl) base = atomicAdd(&ws.sc->sel_c, incl);
+            if (lane == 31 && incl) base = atomicAdd(&ws.sel->c, incl);
             base = __shfl_sync(0xFFFFFFFFu, base, 31);
             uint32_t pos = base + incl - cnt;
 #pragma unroll
@@ -391,17 +391,17 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_collect_kernel(SelArgs a, 
             const uint32_t tok = a.ntok ? a.ntok[i] : a.block_tokens;
             if (entry_key<PF>(a, T, &ws.sc->status, a.agent[i], a.depth[i], a.ref[i], a.flags[i], a.la[i], tok, p, se) &&
                 (p >> 20) <= b0) {
-                const uint32_t pos = atomicAdd(&ws.sc->sel_c, 1u);
+                const uint32_t pos = atomicAdd(&ws.sel->c, 1u);
                 ws.cand_km[pos] = ((unsigned long long)p << 32) | se;
                 ws.cand_id[pos] = i;
             }
         }
     }
-    if (!last_cta_done(&ws.sc->ticket[2], &s_flag)) return;
+    if (!last_cta_done(&ws.sel->ticket[2], &s_flag)) return;
 
     // ---- last CTA: sample, sort the sample (bitonic, shared memory), publish splitters -----------
-    publish_splitters(ws, s_km, s_id, __ldcg(&ws.sc->sel_c));
-    if (threadIdx.x == 0) ws.sc->ticket[2] = 0;
+    publish_splitters(ws, s_km, s_id, __ldcg(&ws.sel->c));
+    if (threadIdx.x == 0) ws.sel->ticket[2] = 0;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -417,7 +417,7 @@ __global__ void __launch_bounds__(256) cs_sel_bucket_kernel(cs_workspace ws)
     constexpr int ITEMS = 4;                                  // candidates per thread and reservation round
     cs_wait_for_predecessor();
     cs_release_successor();
-    const uint32_t c = ws.sc->sel_c, n_spl = ws.sc->sel_n_spl;
+    const uint32_t c = ws.sel->c, n_spl = ws.sel->n_spl;
     for (uint32_t j = threadIdx.x; j < n_spl; j += blockDim.x) { s_km[j] = ws.spl_km[j]; s_id[j] = ws.spl_id[j]; }
     s_cnt[threadIdx.x] = 0;
     __syncthreads();
@@ -459,7 +459,7 @@ __global__ void __launch_bounds__(256) cs_sel_bucket_kernel(cs_workspace ws)
         }
         __syncthreads();
     }
-    if (!last_cta_done(&ws.sc->ticket[3], &s_flag)) return;
+    if (!last_cta_done(&ws.sel->ticket[3], &s_flag)) return;
 
     // ---- last CTA: exclusive prefix sum of the bucket sizes; last bucket needed ----------------------
     const uint32_t t = threadIdx.x;                          // blockDim.x == 256 == buckets
@@ -475,14 +475,14 @@ __global__ void __launch_bounds__(256) cs_sel_bucket_kernel(cs_workspace ws)
     const uint32_t excl = s_scan[t] - mine;
     ws.boff[t] = excl;
     if (t == 255) ws.boff[256] = s_scan[255];
-    const uint32_t n_out = ws.sc->sel_n_out;
+    const uint32_t n_out = ws.sel->n_out;
     if (n_out == 0) {
-        if (t == 0) { ws.sc->sel_b_last = 0; ws.sc->sel_p_end = 0; }
+        if (t == 0) { ws.sel->b_last = 0; ws.sel->p_end = 0; }
     } else if (mine && excl <= n_out - 1 && n_out - 1 < excl + mine) {
-        ws.sc->sel_b_last = t;
-        ws.sc->sel_p_end = excl + mine;
+        ws.sel->b_last = t;
+        ws.sel->p_end = excl + mine;
     }
-    if (t == 0) ws.sc->ticket[3] = 0;
+    if (t == 0) ws.sel->ticket[3] = 0;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -493,8 +493,8 @@ __global__ void __launch_bounds__(256) cs_sel_scatter_kernel(cs_workspace ws)
     __shared__ uint32_t s_off[CS_MAX_SPLITTERS + 1];
     cs_wait_for_predecessor();
     cs_release_successor();
-    const uint32_t c = ws.sc->sel_c, b_last = ws.sc->sel_b_last;
-    if (ws.sc->sel_p_end == 0) return;
+    const uint32_t c = ws.sel->c, b_last = ws.sel->b_last;
+    if (ws.sel->p_end == 0) return;
     s_off[threadIdx.x] = ws.boff[threadIdx.x];
     __syncthreads();
     for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < c; i += gridDim.x * blockDim.x) {
@@ -520,7 +520,7 @@ cs_sel_rank_kernel(cs_workspace ws, uint32_t k, uint32_t *__restrict__ ids_out, 
     __shared__ uint32_t t_id[RANK_TILE];
     cs_wait_for_predecessor();
     cs_release_successor();
-    const uint32_t p_end = ws.sc->sel_p_end, n_out = ws.sc->sel_n_out, b_last = ws.sc->sel_b_last;
+    const uint32_t p_end = ws.sel->p_end, n_out = ws.sel->n_out, b_last = ws.sel->b_last;
     const uint32_t gtid = blockIdx.x * blockDim.x + threadIdx.x, nth = gridDim.x * blockDim.x;
     for (uint32_t i = n_out + gtid; i < k; i += nth) ids_out[i] = CS_ID_NONE;
     if (gtid == 0) *n_out_dev = n_out;
@@ -621,43 +621,26 @@ int cs_launch_score(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, const 
     return cs_check_launch(ctx);
 }
 
-// The three selects of a step as one launch (cluster path only; CS_ENOTIMPL tells the caller to make three calls).
-int cs_launch_select_step(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, uint32_t k_victims, uint32_t k_prefetch,
-                          uint32_t *gpu_victims, uint32_t *n_gpu, uint32_t *host_victims, uint32_t *n_host,
-                          uint32_t *prefetch_ids, uint32_t *n_prefetch, cudaStream_t s)
+// One select through the grid-wide kernels (or one single-launch cluster select), on the scratch of `job`.
+static int launch_select_job(cs_ctx *ctx, int job, const cs_block_index *idx, uint32_t now, int prefetch, uint32_t tier,
+                             uint32_t k, uint32_t *ids_out, uint32_t *n_out, cudaStream_t s)
 {
-    if (ctx->select_path == CS_SELECT_MULTI || idx->n_blocks > CS_SELECT_CLUSTER_MAX_BLOCKS) return CS_ENOTIMPL;
-    SelArgs a[3];
-    for (int q = 0; q < 3; ++q) {
-        fill_args(ctx, idx, now, ctx->fsurv_override ? ctx->fsurv_override : ctx->ws.fsurv, a[q]);
-        a[q].tier = q == 0 ? 0u : 1u;
-        a[q].k = q == 2 ? k_prefetch : k_victims;
-        a[q].hint_slot = ctx->no_speculation ? 3u : (uint32_t)q;
-    }
-    uint32_t *const ids[3] = {gpu_victims, host_victims, prefetch_ids};
-    uint32_t *const cnt[3] = {n_gpu, n_host, n_prefetch};
-    return cs_launch_select_cluster3(ctx, a, ids, cnt, s);
-}
-
-int cs_launch_select(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, int prefetch, uint32_t tier, uint32_t k,
-                     uint32_t *ids_out, uint32_t *n_out, cudaStream_t s)
-{
+    const cs_workspace &ws = job == 0 ? ctx->ws : ctx->ws_job[job - 1];
     SelArgs a;
     fill_args(ctx, idx, now, ctx->fsurv_override ? ctx->fsurv_override : ctx->ws.fsurv, a);
     a.tier = tier;
     a.k = k;
     a.hint_slot = ctx->no_speculation ? 3u : (prefetch ? 2u : tier);
     if (ctx->select_path != CS_SELECT_MULTI && idx->n_blocks <= CS_SELECT_CLUSTER_MAX_BLOCKS) {
-        const int rc1 = cs_launch_select_cluster(ctx, &a, prefetch, ids_out, n_out, s);
+        const int rc1 = cs_launch_select_cluster(ctx, &a, &ws, prefetch, ids_out, n_out, s);
         if (rc1 != CS_ENOTIMPL) return rc1;          // no usable cluster on this device: fall through
     }
     const uint32_t grid = scan_grid(ctx, idx->n_blocks, SEL_THREADS * GRP);
     const uint32_t grid_c = scan_grid(ctx, idx->n_blocks, 256);
     const size_t sm = table_smem(ctx);
     int rc;
-    const uint32_t grid_h = grid;
-    if (prefetch) cs_launch_chained(cs_sel_hist_kernel<true>, grid_h, SEL_THREADS, sm, s, a, ctx->ws);
-    else cs_launch_chained(cs_sel_hist_kernel<false>, grid_h, SEL_THREADS, sm, s, a, ctx->ws);
+    if (prefetch) cs_launch_chained(cs_sel_hist_kernel<true>, grid, SEL_THREADS, sm, s, a, ws);
+    else cs_launch_chained(cs_sel_hist_kernel<false>, grid, SEL_THREADS, sm, s, a, ws);
     if ((rc = cs_check_launch(ctx)) != CS_OK) return rc;
     // large indexes: the collect pass prefilters by age limits (one look-up per entry instead of the full key)
     const uint32_t n_cls = idx->n_tokens ? ctx->p.block_tokens : 1u;
@@ -673,15 +656,74 @@ int cs_launch_select(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, int p
             ctx->collect_attr_set = 1;
         }
     }
-    if (prefetch) cs_launch_chained(cs_sel_collect_kernel<true>, grid, SEL_THREADS, sm_collect, s, a, ctx->ws);
-    else cs_launch_chained(cs_sel_collect_kernel<false>, grid, SEL_THREADS, sm_collect, s, a, ctx->ws);
+    if (prefetch) cs_launch_chained(cs_sel_collect_kernel<true>, grid, SEL_THREADS, sm_collect, s, a, ws);
+    else cs_launch_chained(cs_sel_collect_kernel<false>, grid, SEL_THREADS, sm_collect, s, a, ws);
     if ((rc = cs_check_launch(ctx)) != CS_OK) return rc;
-    cs_launch_chained(cs_sel_bucket_kernel, grid_c, 256, 0, s, ctx->ws);
+    cs_launch_chained(cs_sel_bucket_kernel, grid_c, 256, 0, s, ws);
     if ((rc = cs_check_launch(ctx)) != CS_OK) return rc;
-    cs_launch_chained(cs_sel_scatter_kernel, grid_c, 256, 0, s, ctx->ws);
+    cs_launch_chained(cs_sel_scatter_kernel, grid_c, 256, 0, s, ws);
     if ((rc = cs_check_launch(ctx)) != CS_OK) return rc;
-    cs_launch_chained(cs_sel_rank_kernel, CS_MAX_SPLITTERS + 1, 256, 0, s, ctx->ws, k, ids_out, n_out);
+    cs_launch_chained(cs_sel_rank_kernel, CS_MAX_SPLITTERS + 1, 256, 0, s, ws, k, ids_out, n_out);
     return cs_check_launch(ctx);
+}
+
+int cs_launch_select(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, int prefetch, uint32_t tier, uint32_t k,
+                     uint32_t *ids_out, uint32_t *n_out, cudaStream_t s)
+{
+    return launch_select_job(ctx, 0, idx, now, prefetch, tier, k, ids_out, n_out, s);
+}
+
+// The selects of a step side by side.  Select q (0 GPU-tier victims, 1 host-tier victims, 2 prefetch candidates)
+// is skipped when its count pointer is NULL.  Where the single-launch select applies they are the clusters of ONE
+// launch; otherwise every select is a chain of grid-wide kernels, the first on the caller's stream and the others
+// on the context's two extra streams, forked from and joined back into the caller's stream with events (each has
+// its own select state, histogram and candidate / sort regions).  Indexes beyond CS_CONCURRENT_MAX_BLOCKS entries
+// have no private regions of that size: their selects run one after the other.
+int cs_launch_select_step(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, uint32_t k_victims, uint32_t k_prefetch,
+                          uint32_t *gpu_victims, uint32_t *n_gpu, uint32_t *host_victims, uint32_t *n_host,
+                          uint32_t *prefetch_ids, uint32_t *n_prefetch, cudaStream_t s)
+{
+    uint32_t *const ids[3] = {gpu_victims, host_victims, prefetch_ids};
+    uint32_t *const cnt[3] = {n_gpu, n_host, n_prefetch};
+    const uint32_t ks[3] = {k_victims, k_victims, k_prefetch};
+    int jobs[3], n_jobs = 0;
+    for (int q = 0; q < 3; ++q)
+        if (cnt[q]) jobs[n_jobs++] = q;
+    if (n_jobs == 0) return CS_OK;
+    if (ctx->select_path != CS_SELECT_MULTI && idx->n_blocks <= CS_SELECT_CLUSTER_MAX_BLOCKS) {
+        SelArgs a[3];
+        uint32_t *j_ids[3], *j_cnt[3];
+        uint32_t pf[3];
+        for (int i = 0; i < n_jobs; ++i) {
+            const int q = jobs[i];
+            fill_args(ctx, idx, now, ctx->fsurv_override ? ctx->fsurv_override : ctx->ws.fsurv, a[i]);
+            a[i].tier = q == 0 ? 0u : 1u;
+            a[i].k = ks[q];
+            a[i].hint_slot = ctx->no_speculation ? 3u : (uint32_t)q;
+            j_ids[i] = ids[q];
+            j_cnt[i] = cnt[q];
+            pf[i] = q == 2 ? 1u : 0u;
+        }
+        const int rc = cs_launch_select_clusters(ctx, n_jobs, a, pf, j_ids, j_cnt, s);
+        if (rc != CS_ENOTIMPL) return rc;
+    }
+    const bool side_by_side = ctx->concurrent_selects && n_jobs > 1;
+    cudaError_t e = cudaSuccess;
+    if (side_by_side) e = cudaEventRecord(ctx->ev_sel_fork, s);
+    int rc = CS_OK;
+    for (int i = 0; i < n_jobs && rc == CS_OK && e == cudaSuccess; ++i) {
+        const int q = jobs[i];
+        cudaStream_t sq = (side_by_side && i > 0) ? ctx->sel_stream[i - 1] : s;
+        if (side_by_side && i > 0) e = cudaStreamWaitEvent(sq, ctx->ev_sel_fork, 0);
+        if (e != cudaSuccess) break;
+        rc = launch_select_job(ctx, side_by_side ? i : 0, idx, now, q == 2, q == 0 ? 0u : 1u, ks[q], ids[q], cnt[q], sq);
+        if (rc == CS_OK && side_by_side && i > 0) {
+            e = cudaEventRecord(ctx->ev_sel_join[i - 1], sq);
+            if (e == cudaSuccess) e = cudaStreamWaitEvent(s, ctx->ev_sel_join[i - 1], 0);
+        }
+    }
+    if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; return CS_ECUDA; }
+    return rc;
 }
 
 // =============================================================================================
@@ -704,7 +746,8 @@ int cs_launch_select(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, int p
 #define CS_STATIC_ALIGN(x) (((x) + 255u) / 256u * 256u)
 // layout of the static scratch, byte offsets (every region 256-byte aligned)
 #define CS_SO_SC 0u
-#define CS_SO_GTAB (CS_SO_SC + CS_STATIC_ALIGN(sizeof(cs_scalars)))
+#define CS_SO_SEL (CS_SO_SC + CS_STATIC_ALIGN(sizeof(cs_scalars)))
+#define CS_SO_GTAB (CS_SO_SEL + CS_STATIC_ALIGN(sizeof(cs_sel_state)))
 #define CS_SO_HIST (CS_SO_GTAB + CS_GTAB_MAX * 4u)
 #define CS_SO_SPLKM (CS_SO_HIST + CS_HIST_BINS * 4u)
 #define CS_SO_SPLID (CS_SO_SPLKM + CS_STATIC_ALIGN((CS_MAX_SPLITTERS + 1u) * 8u))
@@ -739,6 +782,9 @@ __global__ void cs_static_prepare_kernel(cs_workspace ws, uint32_t gtab_len, flo
         z.last_agent = CS_AGENT_NONE;
         z.sel_hint[0] = z.sel_hint[1] = z.sel_hint[2] = z.sel_hint[3] = 0xFFFFFFFFu;
         *ws.sc = z;
+        cs_sel_state zs;
+        memset(&zs, 0, sizeof(zs));
+        *ws.sel = zs;
     }
 }
 
@@ -783,6 +829,7 @@ extern "C" int cs_select_victims_static(const cs_params *p, const float *fsurv, 
     ctx.cluster_max_v = g_static_cluster[dev];         // probed once per device, not once per call
     cs_workspace &ws = ctx.ws;
     ws.sc = (cs_scalars *)(base + CS_SO_SC);
+    ws.sel = (cs_sel_state *)(base + CS_SO_SEL);
     ws.gtab = (float *)(base + CS_SO_GTAB);
     ws.hist = (uint32_t *)(base + CS_SO_HIST);
     ws.spl_km = (unsigned long long *)(base + CS_SO_SPLKM);
@@ -796,7 +843,6 @@ extern "C" int cs_select_victims_static(const cs_params *p, const float *fsurv, 
     ws.cand_slot = (uint32_t *)(base + CS_SO_CANDSLOT);
     ws.sort_id = (uint32_t *)(base + CS_SO_SORTID);
     ws.fsurv = const_cast<float *>(fsurv);             // input table, read only
-    ws.job = ws.sc->sel_job[0];
     cudaStream_t s = (cudaStream_t)stream;
     cs_static_prepare_kernel<<<16, 256, 0, s>>>(ws, ctx.gtab_len, p->lambda, p->delta);
     if ((rc = cs_check_launch(&ctx)) != CS_OK) return rc;

@@ -109,10 +109,10 @@ __device__ __forceinline__ void csel_bitonic(unsigned long long *km, uint32_t *i
 
 __device__ __forceinline__ void csel_stamp(const cs_workspace &ws, uint32_t rank, int slot)
 {
-    if (rank == 0 && threadIdx.x == 0 && ws.job == ws.sc->sel_job[0]) {     // the first (or only) select of a launch
+    if (rank == 0 && threadIdx.x == 0) {
         unsigned long long t;
         asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-        ws.sc->t_phase[slot] = t;
+        ws.sel->t_phase[slot] = t;
     }
 }
 
@@ -131,9 +131,9 @@ __device__ __forceinline__ void csel_body(SelArgs a, const cs_workspace &ws, uin
     Tables T;
     load_tables(a, ws, S.tables, T, PF && a.anchor);
     for (uint32_t i = tid; i < CS_HIST_BINS; i += CSEL_THREADS) S.hist[i] = 0;
-    const uint32_t c_slot = *(volatile uint32_t *)&ws.job[2] & 1u;   // read here, before any CTA can flip it (first cluster barrier)
-    uint32_t *cand_count = &ws.job[c_slot];                   // zero on entry: the previous call cleared it
-    if (rank == 0 && tid == 0) ws.job[c_slot ^ 1u] = 0;
+    const uint32_t c_slot = *(volatile uint32_t *)&ws.sel->toggle & 1u;   // read here, before any CTA can flip it (first cluster barrier)
+    uint32_t *cand_count = &ws.sel->cc[c_slot];                   // zero on entry: the previous call cleared it
+    if (rank == 0 && tid == 0) ws.sel->cc[c_slot ^ 1u] = 0;
     if (tid == 0) S.misc[1] = 0;
     __syncthreads();
     const bool enabled = !PF || prefetch_enabled(ws, a.A);
@@ -219,7 +219,7 @@ __device__ __forceinline__ void csel_body(SelArgs a, const cs_workspace &ws, uin
         }
     }
     cluster.sync();
-    if (rank == 0 && tid == 0) ws.job[2] = c_slot ^ 1u;       // every CTA has read it: the next call takes the other counter
+    if (rank == 0 && tid == 0) ws.sel->toggle = c_slot ^ 1u;       // every CTA has read it: the next call takes the other counter
     constexpr uint32_t PER = CS_HIST_BINS / CSEL_THREADS;
     uint32_t loc[PER], sum = 0;
 #pragma unroll
@@ -258,7 +258,7 @@ __device__ __forceinline__ void csel_body(SelArgs a, const cs_workspace &ws, uin
         cluster.sync();
     }
     const uint32_t c = __ldcg(cand_count);
-    if (rank == 0 && tid == 0) ws.job[3] = c;                 // for inspection only
+    if (rank == 0 && tid == 0) ws.sel->cluster_c = c;                 // for inspection only
     csel_stamp(ws, rank, 3);
 
     // ---- phase 4, small: CTA 0 sorts everything in shared memory ---------------------------------------------
@@ -385,7 +385,7 @@ struct SelJob {
     uint32_t *ids_out, *n_out;
     uint32_t prefetch;
 };
-struct SelJobs { SelJob j[3]; };
+struct SelJobs { SelJob j[3]; };     // the grid holds one cluster per job in use
 
 __global__ void __launch_bounds__(CSEL_THREADS, 1) cs_select_step_kernel(const __grid_constant__ SelJobs jobs)
 {
@@ -398,7 +398,8 @@ __global__ void __launch_bounds__(CSEL_THREADS, 1) cs_select_step_kernel(const _
 
 // ---------------------------------------------------------------------------------------------
 template <bool PF>
-static int launch_cluster(cs_ctx *ctx, const SelArgs &a, uint32_t *ids_out, uint32_t *n_out, cudaStream_t s)
+static int launch_cluster(cs_ctx *ctx, const SelArgs &a, const cs_workspace &ws, uint32_t *ids_out, uint32_t *n_out,
+                          cudaStream_t s)
 {
     auto kernel = cs_select_cluster_kernel<PF>;
     const size_t smem = csel_smem_bytes(a.A, a.gtab_len);
@@ -434,17 +435,17 @@ static int launch_cluster(cs_ctx *ctx, const SelArgs &a, uint32_t *ids_out, uint
     while (cl < max_cl && (uint32_t)cl * CSEL_THREADS < n_groups) cl <<= 1;
     cfg.gridDim = dim3(cl);
     attr[0].val.clusterDim.x = cl;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, a, ctx->ws, ids_out, n_out);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, a, ws, ids_out, n_out);
     ctx->n_launches++;
     if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; return CS_ECUDA; }
     return CS_OK;
 }
 
-int cs_launch_select_cluster3(cs_ctx *ctx, const void *sel_args3, uint32_t *const ids_out[3], uint32_t *const n_out[3],
-                              cudaStream_t s)
+int cs_launch_select_clusters(cs_ctx *ctx, int n_jobs, const void *sel_args, const uint32_t *prefetch,
+                              uint32_t *const *ids_out, uint32_t *const *n_out, cudaStream_t s)
 {
-    const SelArgs *a3 = (const SelArgs *)sel_args3;
-    const size_t smem = csel_smem_bytes(a3[0].A, a3[0].gtab_len);
+    const SelArgs *aj = (const SelArgs *)sel_args;
+    const size_t smem = csel_smem_bytes(aj[0].A, aj[0].gtab_len);
     int &max_cl = ctx->cluster_max_step;
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[1];
@@ -471,28 +472,29 @@ int cs_launch_select_cluster3(cs_ctx *ctx, const void *sel_args3, uint32_t *cons
         }
     }
     if (max_cl < 1) return CS_ENOTIMPL;
-    const uint32_t n_groups = a3[0].n / GRP;
+    const uint32_t n_groups = aj[0].n / GRP;
     int cl = 1;
     while (cl < max_cl && (uint32_t)cl * CSEL_THREADS < n_groups) cl <<= 1;
-    cfg.gridDim = dim3(3 * cl);
+    cfg.gridDim = dim3(n_jobs * cl);
     attr[0].val.clusterDim.x = cl;
     SelJobs jobs;
-    for (int q = 0; q < 3; ++q) {
-        jobs.j[q].a = a3[q];
+    for (int q = 0; q < n_jobs; ++q) {
+        jobs.j[q].a = aj[q];
         jobs.j[q].ws = q == 0 ? ctx->ws : ctx->ws_job[q - 1];
         jobs.j[q].ids_out = ids_out[q];
         jobs.j[q].n_out = n_out[q];
-        jobs.j[q].prefetch = q == 2 ? 1u : 0u;
+        jobs.j[q].prefetch = prefetch[q];
     }
+    for (int q = n_jobs; q < 3; ++q) jobs.j[q] = jobs.j[0];          // unused slots: defined contents
     cudaError_t e = cudaLaunchKernelEx(&cfg, cs_select_step_kernel, jobs);
     ctx->n_launches++;
     if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; return CS_ECUDA; }
     return CS_OK;
 }
 
-int cs_launch_select_cluster(cs_ctx *ctx, const void *sel_args, int prefetch, uint32_t *ids_out, uint32_t *n_out,
-                             cudaStream_t s)
+int cs_launch_select_cluster(cs_ctx *ctx, const void *sel_args, const cs_workspace *ws, int prefetch, uint32_t *ids_out,
+                             uint32_t *n_out, cudaStream_t s)
 {
     const SelArgs &a = *(const SelArgs *)sel_args;
-    return prefetch ? launch_cluster<true>(ctx, a, ids_out, n_out, s) : launch_cluster<false>(ctx, a, ids_out, n_out, s);
+    return prefetch ? launch_cluster<true>(ctx, a, *ws, ids_out, n_out, s) : launch_cluster<false>(ctx, a, *ws, ids_out, n_out, s);
 }

@@ -591,4 +591,14 @@ def test_select_step_matches_three_calls_and_oracle(name, n, kv, kp, path):
             assert H.assert_list_matches(g, int(got_n[0].item()), o_ids, o_n, s64) == 0, (rep, k)
     fused = path == cs.CS_SELECT_AUTO and n <= 262144
     assert c.launch_count() - l0 == (3 if fused else 3 * 3 * 5)
+    # a select whose count pointer is NULL is left out
+    gh.fill_(7)
+    ghn.fill_(7)
+    now = 100_020
+    c.select_step(d, now, kv, kp, gv, gvn, None, None, gp, gpn)
+    s64, s32 = o.scores(idx, now)
+    for got, got_n, k, (o_ids, o_n) in ((gv, gvn, kv, o.select_victims(idx, now, 0, kv, s32)),
+                                        (gp, gpn, kp, o.select_prefetch(idx, now, kp, s32))):
+        assert H.assert_list_matches(got.cpu().numpy().view(np.uint32)[:k], int(got_n[0].item()), o_ids, o_n, s64) == 0
+    assert bool((gh == 7).all()) and int(ghn[0].item()) == 7
     assert c.get_status() == 0

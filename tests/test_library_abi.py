@@ -37,9 +37,11 @@ def test_workspace_sizing_and_param_validation(lib):
     p = cs.make_params(n_agents=12, n_chains=64, max_blocks=80000)
     small = cs.cs_workspace_bytes(p)
     big = cs.cs_workspace_bytes(cs.make_params(n_agents=256, n_chains=16, max_blocks=1_000_000))
-    # 32 B per entry, plus two private 32 B-per-entry regions for the fused select, capped at 262,144 entries each
+    # 32 B of select scratch per entry for each of the three selects that may run side by side
     assert 80000 * 96 <= small < 80000 * 100 + (1 << 20)
-    assert 32_000_000 + 2 * 32 * 262144 <= big < 40_000_000 + 2 * 32 * 262144
+    assert 96_000_000 <= big < 100_000_000
+    huge = cs.cs_workspace_bytes(cs.make_params(n_agents=256, n_chains=16, max_blocks=64_000_000))
+    assert 64_000_000 * 32 <= huge < 64_000_000 * 33 + (32 << 20)      # beyond 4,194,304 entries: one full-size region only
     for bad in (dict(n_agents=0), dict(n_agents=2000), dict(n_agents=4, eps=0.0), dict(n_agents=4, delta=0.0),
                 dict(n_agents=4, lam=-1.0), dict(n_agents=4, e_max=0), dict(n_agents=4, block_tokens=0),
                 dict(n_agents=4, max_blocks=0), dict(n_agents=4, n_chains=0), dict(n_agents=4, tau=float("nan"))):
