@@ -114,14 +114,19 @@ cs_observe_kernel(cs_workspace ws, uint32_t A, uint32_t n_chains, const uint32_t
 // Level-synchronous: every thread owns a few nodes; a node of the current frontier ORs its
 // adjacency row into the next frontier (shared-memory atomics), so one level costs one round
 // trip to the adjacency matrix whatever the frontier size.  Thread w < W then retires word w.
-// s_front / s_visit / s_next: 32 words each.
+// s_front / s_visit / s_next: 32 words each.  The adjacency matrix is first copied into shared memory when it
+// fits (BFS_SMEM_WORDS; up to 512 agents), so that the levels cost no further trips to global memory.
 // ---------------------------------------------------------------------------------------------
+#define BFS_SMEM_WORDS 8192u
 __device__ void cs_bfs_survival(const uint32_t *__restrict__ adj, uint32_t A, uint32_t W, uint32_t *s_front,
-                                uint32_t *s_visit, uint32_t *s_next, uint16_t *hops, float *fsurv, uint32_t e_max,
-                                float delta)
+                                uint32_t *s_visit, uint32_t *s_next, uint32_t *s_adj, uint16_t *hops, float *fsurv,
+                                uint32_t e_max, float delta)
 {
     // on entry s_front[] holds the source bits (already synchronised by the caller)
     const uint32_t tid = threadIdx.x;
+    const bool in_smem = A * W <= BFS_SMEM_WORDS;
+    if (in_smem)
+        for (uint32_t i = tid; i < A * W; i += blockDim.x) s_adj[i] = __ldcg(&adj[i]);
     for (uint32_t a = tid; a < A; a += blockDim.x)
         hops[a] = ((s_front[a >> 5] >> (a & 31)) & 1u) ? 0 : CS_HOP_NONE;
     if (tid < W) { s_visit[tid] = s_front[tid]; s_next[tid] = 0; }
@@ -130,7 +135,7 @@ __device__ void cs_bfs_survival(const uint32_t *__restrict__ adj, uint32_t A, ui
         for (uint32_t node = tid; node < A; node += blockDim.x) {
             if ((s_front[node >> 5] >> (node & 31)) & 1u) {
                 for (uint32_t w = 0; w < W; ++w) {
-                    const uint32_t v = __ldcg(&adj[node * W + w]);
+                    const uint32_t v = in_smem ? s_adj[node * W + w] : __ldcg(&adj[node * W + w]);
                     if (v) atomicOr(&s_next[w], v);
                 }
             }
@@ -190,6 +195,7 @@ cs_normalise_kernel(cs_workspace ws, uint32_t A, uint32_t W, float eps, float ta
     __shared__ float s_bestv[ROW_THREADS];
     __shared__ uint32_t s_besti[ROW_THREADS];
     __shared__ uint32_t s_front[32], s_visit[32], s_next[32];
+    __shared__ uint32_t s_adj[BFS_SMEM_WORDS];
     __shared__ bool s_is_last;
     const uint32_t tid = threadIdx.x;
     cs_wait_for_predecessor();
@@ -284,7 +290,7 @@ cs_normalise_kernel(cs_workspace ws, uint32_t A, uint32_t W, float eps, float ta
         s_front[tid] = (la < A && (la >> 5) == tid) ? (1u << (la & 31)) : 0u;
     }
     __syncthreads();
-    cs_bfs_survival(ws.adj, A, W, s_front, s_visit, s_next, ws.hops, ws.fsurv, e_max, delta);
+    cs_bfs_survival(ws.adj, A, W, s_front, s_visit, s_next, s_adj, ws.hops, ws.fsurv, e_max, delta);
 }
 
 // BFS + Eq. 8 from explicit sources into the temporary tables (cs_score_blocks with sources).
@@ -293,6 +299,7 @@ cs_survival_kernel(cs_workspace ws, uint32_t A, uint32_t W, const uint16_t *__re
                    uint32_t e_max, float delta)
 {
     __shared__ uint32_t s_front[32], s_visit[32], s_next[32];
+    __shared__ uint32_t s_adj[BFS_SMEM_WORDS];
     const uint32_t tid = threadIdx.x;
     if (tid < 32) s_front[tid] = 0;
     __syncthreads();
@@ -302,7 +309,7 @@ cs_survival_kernel(cs_workspace ws, uint32_t A, uint32_t W, const uint16_t *__re
         else atomicOr(&ws.sc->status, CS_ST_BAD_SOURCE);
     }
     __syncthreads();
-    cs_bfs_survival(ws.adj, A, W, s_front, s_visit, s_next, ws.hops_tmp, ws.fsurv_tmp, e_max, delta);
+    cs_bfs_survival(ws.adj, A, W, s_front, s_visit, s_next, s_adj, ws.hops_tmp, ws.fsurv_tmp, e_max, delta);
 }
 
 // ---------------------------------------------------------------------------------------------
