@@ -969,7 +969,7 @@ def main():
         "blocks_scored_selected_per_s": world * 3 * w.N / (t_s / 1e3),
         "gpu_launches": int(launches),
         "clocks": clocks,
-        "roofline": {"kernel": "cs_mover_bulk_kernel (device-to-device compaction of the 256 victims, inside the step, while offload and prefetch run on the side streams)", "bound": "hbm",
+        "roofline": {"kernel": "cs_mover_bulk_kernel (device-to-device compaction of the 256 victims, inside the step, while the host-link transfers of the previous step run beside it)", "bound": "hbm",
                      "achieved": d2d_gbps, "peak": hbm_peak, "unit": "GB/s", "frac": d2d_gbps / hbm_peak, "traffic": traffic,
                      "peak_kind": "of %s" % peak_kind, "algorithmic_bytes_per_launch": 2 * w.k_v * bb, "ms_per_launch": t_c},
         "roofline_dominant_kernel": {
