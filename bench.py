@@ -349,6 +349,15 @@ class StepWorkload:
         return h2d, d2h
 
 
+def in_flight_factor(alone_ms, both_ms, transfer_ms):
+    """Slowdown of the serving loop during the part of it that overlaps the transfer, when the loop outlasts the
+    transfer: it does transfer_ms / f of its work while the transfer runs and the rest at full speed."""
+    if both_ms <= transfer_ms:
+        return both_ms / alone_ms
+    done_during = alone_ms - (both_ms - transfer_ms)
+    return transfer_ms / done_during if done_during > 0 else float("inf")
+
+
 def fused_step_section(w, steps=10):
     """The whole step as ONE library call (cs_step): issued afresh every step, and captured once into a CUDA
     graph that reads the clock and the event count from device memory and is replayed; then the interference
@@ -435,7 +444,9 @@ def fused_step_section(w, steps=10):
     a = torch.randn(8192, 8192, dtype=torch.bfloat16, device=dev)
     b = torch.randn(8192, 8192, dtype=torch.bfloat16, device=dev)
     o = torch.empty(8192, 8192, dtype=torch.bfloat16, device=dev)
-    loads = {"hbm_copy_8GiB_x16": (lambda: y.copy_(x), 16), "bf16_gemm_8192_x24": (lambda: torch.matmul(a, b, out=o), 24)}
+    small = torch.zeros(1 << 18, dtype=torch.float32, device=dev)          # 1 MiB: a latency-bound kernel per call
+    loads = {"hbm_copy_8GiB_x16": (lambda: y.copy_(x), 16), "bf16_gemm_8192_x24": (lambda: torch.matmul(a, b, out=o), 24),
+             "small_kernel_chain_x4000": (lambda: small.add_(1.0), 4000)}
 
     def transfer():
         c.exchange_blocks(w.gpu_pool, w.host_pool, gv, gh, gp, free_last, n_off_max=kv, n_off_dev=gvn, n_pre_max=kp,
@@ -469,9 +480,68 @@ def fused_step_section(w, steps=10):
         alone, _ = run(load, False)
         both, x_both = run(load, True)
         inter[name] = {"serving_alone_ms": alone, "serving_with_transfer_ms": both, "serving_slowdown": both / alone,
+                       "serving_slowdown_while_transfer_in_flight": in_flight_factor(alone, both, x_both),
                        "transfer_with_serving_ms": x_both, "transfer_slowdown": x_both / x_alone}
+    # the same chain as a CUDA graph (no per-kernel host traffic), disturbed by this library's transfer and by the
+    # same bytes moved by the copy engines (two pinned cudaMemcpyAsync copies, 512 MiB out while 768 MiB come in)
+    cg = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(cg, stream=main, capture_error_mode="relaxed"):
+        for _ in range(1000):
+            small.add_(1.0)
+    side2 = torch.cuda.Stream(device=dev)
+    ce_out_h, ce_in_h = w.host_buf[:512 << 20], w.host_buf[(1 << 30):(1 << 30) + (768 << 20)]
+    ce_out_d = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
+    ce_in_d = torch.empty(768 << 20, dtype=torch.uint8, device=dev)
+
+    def copy_engines():
+        with torch.cuda.stream(side):
+            ce_out_h.copy_(ce_out_d, non_blocking=True)
+        with torch.cuda.stream(side2):
+            ce_in_d.copy_(ce_in_h, non_blocking=True)
+        side.wait_stream(side2)
+
+    def run_graph(disturber):
+        best = None
+        for _ in range(3):
+            torch.cuda.synchronize(dev)
+            m0, m1, s0, s1 = (torch.cuda.Event(enable_timing=True) for _ in range(4))
+            m0.record(main)
+            side.wait_event(m0)
+            side2.wait_event(m0)
+            s0.record(side)
+            if disturber is not None:
+                disturber()
+            s1.record(side)
+            with torch.cuda.stream(main):
+                for _ in range(4):
+                    cg.replay()
+            m1.record(main)
+            torch.cuda.synchronize(dev)
+            t = (m0.elapsed_time(m1), s0.elapsed_time(s1))
+            best = t if best is None or t[0] < best[0] else best
+        return best
+
+    g_alone, _ = run_graph(None)
+    g_ours, g_ours_x = run_graph(transfer)
+    g_ce, g_ce_x = run_graph(copy_engines)
+    inter["graph_chain_4x1000_small_kernels"] = {
+        "alone_ms": g_alone,
+        "with_this_library_transfer_ms": g_ours, "slowdown_while_in_flight": in_flight_factor(g_alone, g_ours, g_ours_x),
+        "with_copy_engine_transfer_ms": g_ce, "copy_engine_transfer_ms": g_ce_x,
+        "slowdown_while_copy_engines_in_flight": in_flight_factor(g_alone, g_ce, g_ce_x)}
+    del ce_out_d, ce_in_d
+    # the knob: a narrower transfer disturbs latency-bound kernels less and moves fewer bytes per second
+    c.set_mover_ctas(8, 0)
+    _, x8 = run(loads["small_kernel_chain_x4000"], True, with_load=False)
+    both8, x8_both = run(loads["small_kernel_chain_x4000"], True)
+    c.set_mover_ctas(0, 0)
+    alone_small = inter["small_kernel_chain_x4000"]["serving_alone_ms"]
+    inter["small_kernel_chain_x4000_transfer_width_8"] = {
+        "transfer_alone_ms": x8, "serving_with_transfer_ms": both8, "serving_slowdown": both8 / alone_small,
+        "serving_slowdown_while_transfer_in_flight": in_flight_factor(alone_small, both8, x8_both),
+        "transfer_with_serving_ms": x8_both, "transfer_slowdown": x8_both / x8}
     out["interference"] = inter
-    del x, y, a, b, o
+    del x, y, a, b, o, small
     return out
 
 
