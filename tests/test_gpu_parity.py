@@ -570,9 +570,9 @@ def test_survival_from_all_chains(name, n_inv):
     ("meta1m", 262144, 10000, 2000), ("meta1m", 300000, 500, 500)])
 @pytest.mark.parametrize("path", [cs.CS_SELECT_AUTO, cs.CS_SELECT_MULTI])
 def test_select_step_matches_three_calls_and_oracle(name, n, kv, kp, path):
-    """cs_select_step: one launch of three clusters where the single-launch select applies, three calls
-    elsewhere (300,000 entries, or the multi-launch path forced); lists bit-exact against the oracle, and
-    again on a second and third call with a later clock (remembered thresholds in play)."""
+    """cs_select_step: one launch of three clusters where the single-launch select applies, three kernel chains
+    side by side elsewhere (300,000 entries, or the multi-launch path forced); lists bit-exact against the oracle,
+    and again on a second and third call with a later clock (remembered thresholds in play)."""
     cfg = synth.CONFIGS[name]
     c, o = warm_state(cfg, 800, max(n, 16), r_min=0.02)
     c.set_select_path(path)
