@@ -199,7 +199,9 @@ int cs_select_victims_static(const cs_params *p, const float *fsurv, const cs_bl
 /* For i < n (n = min(n_max, *n_dev) when n_dev != NULL, else n_max), every layer and both
  * planes: copy the chunk of src slot src_slots[i] to dst slot dst_slots[i].  Entries with
  * CS_ID_NONE on either side are skipped.  src_slots / dst_slots / n_dev: dev.  The two pools
- * must agree in everything but base, n_slots and layout.  Destination slots must be distinct;
+ * must agree in everything but base, n_slots and layout.  A pool base the device cannot address (pageable
+ * host memory that was neither allocated page-locked nor registered) is CS_EINVAL: nothing is launched.
+ * Destination slots must be distinct;
  * when src and dst are the same pool the two slot sets must be disjoint (not checked). */
 int cs_offload_blocks(cs_ctx *ctx, const cs_kv_pool *gpu, const cs_kv_pool *host, const uint32_t *src_slots,
                       const uint32_t *dst_slots, uint32_t n_max, const uint32_t *n_dev, cs_stream_t side);

@@ -297,6 +297,16 @@ int cs_select_step(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, uint32_
                                  n_host_victims, prefetch_ids, n_prefetch, (cudaStream_t)stream);
 }
 
+// A pool the SMs cannot address (pageable host memory that was never registered) would fault the GPU, so the
+// base pointers are looked up before every launch (a host-side query of about a microsecond): device memory,
+// pinned / registered host memory and managed memory pass.
+static bool device_can_address(const void *ptr)
+{
+    cudaPointerAttributes at;
+    if (cudaPointerGetAttributes(&at, ptr) != cudaSuccess) { (void)cudaGetLastError(); return false; }
+    return at.type == cudaMemoryTypeDevice || at.type == cudaMemoryTypeHost || at.type == cudaMemoryTypeManaged;
+}
+
 static int check_pools(const cs_kv_pool *a, const cs_kv_pool *b)
 {
     if (!a || !b || !a->base || !b->base) return CS_EINVAL;
@@ -318,6 +328,7 @@ static int mover_common(cs_ctx *ctx, const cs_kv_pool *src, const cs_kv_pool *ds
     if (!ctx) return CS_EINVAL;
     int rc = check_pools(src, dst);
     if (rc != CS_OK) return rc;
+    if (!device_can_address(src->base) || !device_can_address(dst->base)) return CS_EINVAL;
     if (n_max == 0) return CS_OK;
     if (!src_slots || !dst_slots || (((uintptr_t)src_slots) & 3u) || (((uintptr_t)dst_slots) & 3u)) return CS_EINVAL;
     if (n_dev && (((uintptr_t)n_dev) & 3u)) return CS_EINVAL;
@@ -350,6 +361,7 @@ int cs_exchange_blocks(cs_ctx *ctx, const cs_kv_pool *gpu, const cs_kv_pool *hos
     if (!ctx) return CS_EINVAL;
     int rc = check_pools(gpu, host);
     if (rc != CS_OK) return rc;
+    if (!device_can_address(gpu->base) || !device_can_address(host->base)) return CS_EINVAL;
     if (n_off_max == 0 && n_pre_max == 0) return CS_OK;
     const uint32_t *lists[4] = {off_gpu_slots, off_host_slots, pre_host_slots, pre_gpu_slots};
     for (int i = 0; i < 4; ++i) {

@@ -329,6 +329,17 @@ def test_mover_small_chunks_and_geometry_errors(path):
         cs.cs_compact_blocks(c.ctx, a.struct(), cs.cs_kv_pool(bad.buf.data_ptr(), G, 1, L + 1, heads, hd, tok, 2, 0),
                              dev(s), dev(d), 1)
     assert e.value.code == cs.CS_EINVAL
+    # a pool in pageable host memory is refused on the host: nothing is launched, the device never sees the address
+    pageable = torch.zeros(G * L * 2 * chunk + 64, dtype=torch.uint8)
+    ptr = (pageable.data_ptr() + 15) & ~15
+    l_before = c.launch_count()
+    with pytest.raises(cs.CacheScoutError) as e:
+        cs.cs_offload_blocks(c.ctx, a.struct(), cs.cs_kv_pool(ptr, G, 1, L, heads, hd, tok, 2, 0), dev(s), dev(d), 1)
+    assert e.value.code == cs.CS_EINVAL and c.launch_count() == l_before
+    with pytest.raises(cs.CacheScoutError) as e:
+        cs.cs_exchange_blocks(c.ctx, a.struct(), cs.cs_kv_pool(ptr, G, 1, L, heads, hd, tok, 2, 0), dev(s), dev(d), 1, None,
+                              dev(d), dev(s), 1, None)
+    assert e.value.code == cs.CS_EINVAL and c.launch_count() == l_before
     odd = cs.cs_kv_pool(a.buf.data_ptr(), G, 0, L, 1, 3, 1, 2, 0)          # 6-byte chunks: not 16-byte multiples
     with pytest.raises(cs.CacheScoutError):
         cs.cs_compact_blocks(c.ctx, odd, odd, dev(s), dev(d), 1)
