@@ -222,6 +222,16 @@ int cs_observe_invocations(cs_ctx *ctx, const uint32_t *chain, const uint16_t *a
     return cs_launch_observe(ctx, chain, agent, evflags, n_events, (cudaStream_t)stream);
 }
 
+// Memory the SMs cannot address (pageable host memory that was never registered) would fault the GPU, so pool
+// bases and index arrays are looked up before every launch (a host-side query of about a microsecond): device memory,
+// pinned / registered host memory and managed memory pass.
+static bool device_can_address(const void *ptr)
+{
+    cudaPointerAttributes at;
+    if (cudaPointerGetAttributes(&at, ptr) != cudaSuccess) { (void)cudaGetLastError(); return false; }
+    return at.type == cudaMemoryTypeDevice || at.type == cudaMemoryTypeHost || at.type == cudaMemoryTypeManaged;
+}
+
 static int check_index(const cs_ctx *ctx, const cs_block_index *idx)
 {
     if (!idx) return CS_EINVAL;
@@ -232,6 +242,10 @@ static int check_index(const cs_ctx *ctx, const cs_block_index *idx)
         !aligned16(idx->flags) || !aligned16(idx->last_access) || !aligned16(idx->n_tokens) ||
         !aligned16(idx->anchor_blocks))
         return CS_EINVAL;
+    const void *arrays[7] = {idx->agent, idx->depth, idx->ref_count, idx->flags, idx->last_access, idx->n_tokens,
+                             idx->anchor_blocks};
+    for (int i = 0; i < 7; ++i)
+        if (arrays[i] && !device_can_address(arrays[i])) return CS_EINVAL;     // a host array would fault the kernels
     return CS_OK;
 }
 
@@ -295,16 +309,6 @@ int cs_select_step(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, uint32_
     }
     return cs_launch_select_step(ctx, idx, now, k_victims, k_prefetch, gpu_victims, n_gpu_victims, host_victims,
                                  n_host_victims, prefetch_ids, n_prefetch, (cudaStream_t)stream);
-}
-
-// A pool the SMs cannot address (pageable host memory that was never registered) would fault the GPU, so the
-// base pointers are looked up before every launch (a host-side query of about a microsecond): device memory,
-// pinned / registered host memory and managed memory pass.
-static bool device_can_address(const void *ptr)
-{
-    cudaPointerAttributes at;
-    if (cudaPointerGetAttributes(&at, ptr) != cudaSuccess) { (void)cudaGetLastError(); return false; }
-    return at.type == cudaMemoryTypeDevice || at.type == cudaMemoryTypeHost || at.type == cudaMemoryTypeManaged;
 }
 
 static int check_pools(const cs_kv_pool *a, const cs_kv_pool *b)
