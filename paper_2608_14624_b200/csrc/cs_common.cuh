@@ -22,7 +22,6 @@
 #define CS_HIST_BINS 4096u        // first radix digit of the select: top 12 bits of the primary key
 #define CS_MAX_SPLITTERS 255u     // bucket sort of the candidates: up to 256 buckets
 #define CS_SAMPLE 1024u           // candidates sampled to choose the splitters
-#define CS_SPEC_MARGIN_CALLS 16u    // after a missed speculation: calls that collect one bin beyond the last threshold
 #define CS_GTAB_MAX 4096u          // largest recency table kept in shared memory (ages below saturation)
 
 // Scalars the kernels share, one 256-byte line in the workspace.
@@ -35,10 +34,8 @@ struct cs_scalars {
     uint32_t ticket0;       // "last CTA done" counter of the learner refresh
     uint32_t gtab_monotone; // the recency table covers every unsaturated age and never increases with age
     uint32_t sel_hint[4];   // bin up to which the next select of each kind (GPU victims, host victims, prefetch)
-                            // collects ahead: the previous threshold bin, plus one while sel_margin > 0; ~0 = none;
-                            // slot 3 is never written: calls that must not speculate read it
-    uint32_t sel_margin[4]; // per kind: calls left during which the next call collects one bin beyond the remembered
-                            // threshold (set after a miss: that kind's threshold is moving upwards or jitters)
+                            // collects ahead of its own threshold, chosen from the previous call's histogram;
+                            // ~0 = none; slot 3 is never written: calls that must not speculate read it
 };
 
 // State of one select in flight, rewritten by every call.  The selects of a step that run side by side each

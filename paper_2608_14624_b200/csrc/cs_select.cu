@@ -116,7 +116,7 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_hist_kernel(SelArgs a, cs_
     extern __shared__ float smem[];
     __shared__ __align__(16) uint32_t s_hist[CS_HIST_BINS];
     __shared__ uint32_t s_part[SEL_THREADS];
-    __shared__ uint32_t s_b0;
+    __shared__ uint32_t s_b0, s_ahead;
     __shared__ bool s_flag;
     cs_wait_for_predecessor();
     cs_release_successor();
@@ -236,6 +236,8 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_hist_kernel(SelArgs a, cs_
     __syncthreads();
     const uint32_t b0 = s_b0;
     const bool spec_ok = hint != 0xFFFFFFFFu && b0 != 0xFFFFFFFFu && b0 <= hint;
+    const bool have_b0 = a.k && total >= a.k;
+    const uint32_t ahead = have_b0 ? collect_ahead_limit<PER>(loc, threadIdx.x * PER, before, a.k, b0, &s_ahead) : 0u;
     const uint32_t c_spec = __ldcg(&ws.sel->c_spec);
     if (spec_ok)                                             // the shared histogram is free now: it holds the sample
         publish_splitters(ws, (unsigned long long *)s_hist, s_hist + 2 * CS_SAMPLE, c_spec);
@@ -246,7 +248,7 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_hist_kernel(SelArgs a, cs_
         ws.sel->c = spec_ok ? c_spec : 0;
         ws.sel->c_spec = 0;
         ws.sel->spec = spec_ok ? 1u : 0u;
-        remember_threshold(ws.sc, a.hint_slot, a.k && total >= a.k, b0, hint != 0xFFFFFFFFu, spec_ok);
+        remember_threshold(ws.sc, a.hint_slot, have_b0, ahead);
         ws.sel->ticket[1] = 0;
     }
 }

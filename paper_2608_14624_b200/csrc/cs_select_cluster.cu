@@ -246,7 +246,11 @@ __device__ __forceinline__ void csel_body(SelArgs a, const cs_workspace &ws, uin
     csel_stamp(ws, rank, 2);
     // ---- phase 3: collect the candidates (bin <= b0), unless the first scan already has them ----------------
     const bool spec_ok = hint != 0xFFFFFFFFu && b0 != 0xFFFFFFFFu && b0 <= hint;     // same verdict in every CTA
-    if (rank == 0 && tid == 0) remember_threshold(ws.sc, a.hint_slot, a.k && n_elig >= a.k, b0, hint != 0xFFFFFFFFu, spec_ok);
+    const bool have_b0 = a.k && n_elig >= a.k;
+    if (rank == 0) {                                           // whole CTA 0: same histogram in every CTA
+        const uint32_t ahead = have_b0 ? collect_ahead_limit<PER>(loc, tid * PER, before, a.k, b0, &S.misc[2]) : 0u;
+        if (tid == 0) remember_threshold(ws.sc, a.hint_slot, have_b0, ahead);
+    }
     if (!spec_ok) {
         if (hint != 0xFFFFFFFFu) {                            // drop what the first scan appended
             if (rank == 0 && tid == 0) *cand_count = 0;

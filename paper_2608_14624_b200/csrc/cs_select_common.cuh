@@ -23,20 +23,40 @@ struct SelArgs {
     const uint32_t *now_dev;      // when set, the clock is read from device memory at execution time (graph replay)
 };
 
-// What the next call of this kind may collect ahead of its own threshold.  The threshold bin of
-// consecutive calls moves little; where it moves upwards or jitters (a miss), one extra bin is allowed
-// for the next CS_SPEC_MARGIN_CALLS calls.  Only the amount of work depends on this, never the result.
-__device__ __forceinline__ void remember_threshold(cs_scalars *sc, uint32_t slot, bool valid, uint32_t b0, bool had_hint,
-                                                   bool spec_ok)
+// What the next call of this kind may collect ahead of its own threshold.  The threshold bin of consecutive
+// calls moves little, so the next call's first scan appends every entry up to a remembered bin.  That bin is
+// chosen from this call's exact histogram: the furthest bin whose cumulative population stays within
+// 3 k + 1024 entries, at least the threshold bin itself and at most CS_SPEC_MAX_AHEAD bins beyond it.  Sparse
+// bins (a prefetch list whose best entries leave the tier every call, so its threshold jumps) get several bins
+// of slack for a few thousand extra candidates; dense bins get none.  Only the amount of work depends on this,
+// never the result.  `loc` are the calling thread's bins [first, first + PER), `before` the population below
+// them; every thread of the CTA calls; s_lim is a shared word.
+#define CS_SPEC_MAX_AHEAD 8u
+template <uint32_t PER>
+__device__ __forceinline__ uint32_t collect_ahead_limit(const uint32_t (&loc)[PER], uint32_t first, uint32_t before,
+                                                        uint32_t k, uint32_t b0, uint32_t *s_lim)
 {
-    if (slot >= 3) return;
-    if (!valid) { sc->sel_hint[slot] = 0xFFFFFFFFu; return; }
-    uint32_t m = sc->sel_margin[slot];
-    if (had_hint && !spec_ok) m = CS_SPEC_MARGIN_CALLS;
-    else if (m) --m;
-    sc->sel_margin[slot] = m;
-    const uint32_t lim = b0 + (m ? 1u : 0u);
-    sc->sel_hint[slot] = lim < CS_HIST_BINS ? lim : CS_HIST_BINS - 1;
+    if (threadIdx.x == 0) *s_lim = 0;
+    __syncthreads();
+    const unsigned long long cap = 3ull * k + 1024ull;
+    unsigned long long run = before;
+    uint32_t best = 0xFFFFFFFFu;
+#pragma unroll
+    for (uint32_t q = 0; q < PER; ++q) {
+        run += loc[q];
+        if (run <= cap) best = first + q;
+    }
+    if (best != 0xFFFFFFFFu) atomicMax(s_lim, best);
+    __syncthreads();
+    uint32_t lim = *s_lim;
+    if (lim < b0) lim = b0;
+    if (lim > b0 + CS_SPEC_MAX_AHEAD) lim = b0 + CS_SPEC_MAX_AHEAD;
+    return lim < CS_HIST_BINS ? lim : CS_HIST_BINS - 1;
+}
+
+__device__ __forceinline__ void remember_threshold(cs_scalars *sc, uint32_t slot, bool valid, uint32_t limit)
+{
+    if (slot < 3) sc->sel_hint[slot] = valid ? limit : 0xFFFFFFFFu;
 }
 
 // The clock of a call: by value, or from device memory when the caller asked for that.
