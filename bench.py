@@ -860,7 +860,7 @@ def profile_case(args, torch, device):
     select: metadata-scale index (1,000,000 entries, 256 agents); per step observe 64 events,
             select 10,000 victims and 2,000 prefetch candidates (multi-launch select path).
     select80k: the 80,000-entry index of the Llama-8B configuration, 256 victims / 384 prefetch
-            candidates (single-launch cluster select path)."""
+            candidates (single-launch cluster select path), then the step's three selects as one launch."""
     from paper_2608_14624_b200 import binding as cs
     from paper_2608_14624_b200 import build, synth
     build.build_library()
@@ -899,11 +899,15 @@ def profile_case(args, torch, device):
         v = torch.empty(cfg.k_victims, dtype=torch.int32, device=device)
         pf = torch.empty(cfg.k_prefetch, dtype=torch.int32, device=device)
         vn, pn = torch.zeros(4, dtype=torch.int32, device=device), torch.zeros(4, dtype=torch.int32, device=device)
+        hv = torch.empty(cfg.k_victims, dtype=torch.int32, device=device)
+        hn = torch.zeros(4, dtype=torch.int32, device=device)
         for s in range(max(1, args.steps)):
             lo = 64 * (30 + s)
             c.observe_invocations(ch[lo:lo + 64], ag[lo:lo + 64], None)
             c.select_victims(d, 100_000 + s, 0, cfg.k_victims, v, vn)
             c.select_prefetch(d, 100_000 + s, cfg.k_prefetch, pf, pn)
+            if not big:        # the step's three selects as one launch
+                c.select_step(d, 100_000 + s, cfg.k_victims, cfg.k_prefetch, v, vn, hv, hn, pf, pn)
     torch.cuda.synchronize(device)
     print(json.dumps({"workload": args.workload, "launches": c.launch_count(), "device_status": c.get_status()}))
 
