@@ -613,3 +613,36 @@ def test_select_step_matches_three_calls_and_oracle(name, n, kv, kp, path):
         assert H.assert_list_matches(got.cpu().numpy().view(np.uint32)[:k], int(got_n[0].item()), o_ids, o_n, s64) == 0
     assert bool((gh == 7).all()) and int(ghn[0].item()) == 7
     assert c.get_status() == 0
+
+
+def test_select_step_side_by_side_is_stable_over_many_calls():
+    """The three kernel chains of a step run side by side on three streams with private scratch: over many
+    consecutive calls with a moving clock and a changing index every list must equal the one the same select
+    produces alone (bitwise), and the last call is checked against the oracle."""
+    cfg = synth.CONFIGS["meta1m"]
+    n, kv, kp = 300_000, 3000, 1500
+    c, o = warm_state(cfg, 800, n, r_min=0.02)
+    idx = synth.make_block_index(cfg, n=n, tier="random")
+    d = cs.DeviceIndex.from_host(idx, DEV)
+    i32 = lambda m: torch.full((max(m, 4),), 7, dtype=torch.int32, device=DEV)
+    gv, gh, gp, gvn, ghn, gpn = i32(kv), i32(kv), i32(kp), i32(1), i32(1), i32(1)
+    sv, sh, sp, svn, shn, spn = i32(kv), i32(kv), i32(kp), i32(1), i32(1), i32(1)
+    la = d.last_access.view(torch.int32)
+    bad = torch.zeros(1, dtype=torch.int64, device=DEV)
+    for it in range(120):
+        now = 100_000 + 3 * it
+        if it:
+            la[gv[:kv].long().clamp_(min=0)] = now - 3          # the index changes between calls
+        c.select_step(d, now, kv, kp, gv, gvn, gh, ghn, gp, gpn)
+        c.select_victims(d, now, 0, kv, sv, svn)
+        c.select_victims(d, now, 1, kv, sh, shn)
+        c.select_prefetch(d, now, kp, sp, spn)
+        bad += (gv != sv).sum() + (gh != sh).sum() + (gp != sp).sum() + (gvn != svn).sum() + (ghn != shn).sum() + (gpn != spn).sum()
+    assert int(bad.item()) == 0
+    idx.last_access[:] = d.last_access.cpu().numpy()
+    s64, s32 = o.scores(idx, now)
+    for got, got_n, k, (o_ids, o_n) in ((gv, gvn, kv, o.select_victims(idx, now, 0, kv, s32)),
+                                        (gh, ghn, kv, o.select_victims(idx, now, 1, kv, s32)),
+                                        (gp, gpn, kp, o.select_prefetch(idx, now, kp, s32))):
+        assert H.assert_list_matches(got.cpu().numpy().view(np.uint32)[:k], int(got_n[0].item()), o_ids, o_n, s64) == 0
+    assert c.get_status() == 0
