@@ -265,9 +265,45 @@ __device__ __forceinline__ void csel_body(SelArgs a, const cs_workspace &ws, uin
     if (rank == 0 && tid == 0) ws.sel->cluster_c = c;                 // for inspection only
     csel_stamp(ws, rank, 3);
 
-    // ---- phase 4, small: CTA 0 sorts everything in shared memory ---------------------------------------------
+    // ---- phase 4, small: ordered in shared memory ---------------------------------------------------------------
     if (c <= CSEL_SORT_MAX) {
-        if (rank != 0 || c == 0) return;
+        if (c == 0) return;
+        constexpr uint32_t CH = 2 * CSEL_THREADS;                // keys one CTA orders with the register sort
+        const uint32_t n_chunks = (c + CH - 1) / CH;
+        if (n_chunks > 1 && n_chunks <= CL && n_chunks * n_out <= CH) {
+            // Several CTAs order one chunk each, side by side: the n_out smallest keys of the union lie among the
+            // n_out smallest of every chunk, so CTA 0 only has to order n_chunks * n_out survivors afterwards.
+            if (rank < n_chunks) {
+                const uint32_t beg = rank * CH, m = min(CH, c - beg);
+                for (uint32_t i = tid; i < CH; i += CSEL_THREADS) {
+                    S.km[i] = i < m ? __ldcg(&ws.cand_km[beg + i]) : ~0ull;
+                    S.id[i] = i < m ? __ldcg(&ws.cand_id[beg + i]) : 0xFFFFFFFFu;
+                }
+                __syncthreads();
+                csel_bitonic(S.km, S.id, CH);
+                for (uint32_t i = tid; i < n_out; i += CSEL_THREADS) {
+                    ws.sort_km[rank * n_out + i] = S.km[i];
+                    ws.sort_id[rank * n_out + i] = S.id[i];
+                }
+            }
+            __threadfence();
+            cluster.sync();                                     // every CTA of the cluster gets here
+            if (rank != 0) return;
+            const uint32_t tot = n_chunks * n_out;
+            uint32_t P = 64;
+            while (P < tot) P <<= 1;
+            __syncthreads();
+            for (uint32_t i = tid; i < P; i += CSEL_THREADS) {
+                S.km[i] = i < tot ? __ldcg(&ws.sort_km[i]) : ~0ull;
+                S.id[i] = i < tot ? __ldcg(&ws.sort_id[i]) : 0xFFFFFFFFu;
+            }
+            __syncthreads();
+            csel_bitonic(S.km, S.id, P);
+            for (uint32_t i = tid; i < n_out; i += CSEL_THREADS) ids_out[i] = S.id[i];
+            csel_stamp(ws, rank, 4);
+            return;
+        }
+        if (rank != 0) return;
         uint32_t P = 64;
         while (P < c) P <<= 1;
         for (uint32_t i = tid; i < P; i += CSEL_THREADS) {
