@@ -646,3 +646,47 @@ def test_select_step_side_by_side_is_stable_over_many_calls():
                                         (gp, gpn, kp, o.select_prefetch(idx, now, kp, s32))):
         assert H.assert_list_matches(got.cpu().numpy().view(np.uint32)[:k], int(got_n[0].item()), o_ids, o_n, s64) == 0
     assert c.get_status() == 0
+
+
+# ---- randomised small configurations ------------------------------------------------------------------------
+@pytest.mark.parametrize("case", range(48))
+def test_random_small_configurations(case):
+    """Seeded random draws of everything the paper leaves open (agent count, chains, E_max, tau, lambda, delta,
+    eps, block size, index size, k, with / without token counts and anchors, the copy preference, both BFS source
+    modes): learner state, scores and all three lists on both select paths against the oracle."""
+    rng = np.random.default_rng(7000 + case)
+    A = int(rng.choice([1, 2, 3, 5, 12, 31, 32, 33, 70, 129]))
+    chains = int(rng.choice([1, 3, 17]))
+    base = synth.CONFIGS["tiny"] if A <= 5 else synth.CONFIGS["llama70b"]
+    cfg = synth.shrink(base, n_agents=A, sessions=chains, n_chains=chains, seed=base.seed + 100 + case,
+                       transitions=("dirichlet", float(rng.choice([0.3, 1.0]))) if A < 9 else ("sparse", int(min(4, A - 1))),
+                       block_tokens=int(rng.choice([2, 7, 16, 32])), events_per_step=(1, int(rng.integers(1, 6))))
+    n = int(rng.choice([1, 15, 16, 511, 512, 513, 3000, 9001]))
+    kw = dict(e_max=int(rng.choice([1, 3, 4, 7])), tau=float(rng.choice([0.0, 0.02, 0.2, 1.5])),
+              lam=float(rng.choice([0.0, 0.003, 0.05, 1.0])), delta=float(rng.choice([1e-3, 0.01, 0.5])),
+              eps=float(rng.choice([1e-3, 0.01, 1.0])), r_min=float(rng.choice([0.0, 0.02])),
+              prefer_other_copy=int(rng.integers(0, 2)))
+    tr = synth.make_trace(cfg, n_invocations=int(rng.integers(1, 400)), warmup_frac=float(rng.choice([0.0, 0.2])))
+    c, o = make_ctx(cfg, max(n, 16), **kw)
+    all_chains = bool(rng.integers(0, 2))
+    if all_chains:
+        c.set_survival_sources(cs.CS_SOURCES_ALL_CHAINS)
+    c.observe_invocations(dev(tr.chain), dev(tr.agent), dev(tr.evflags))
+    o.observe(tr.chain, tr.agent, tr.evflags)
+    if all_chains:
+        o.survival(sources=np.unique(o.cur[o.cur != orc.AGENT_NONE]))
+    if abs(o.R - o.p.r_min) < H.R_FRAGILE:
+        pytest.skip("R within the fragile band of r_min for this draw")
+    H.compare_model(c, o)
+    idx = synth.make_block_index(cfg, n=n, tier="random", with_tokens=bool(rng.integers(0, 2)),
+                                 with_anchor=bool(rng.integers(0, 2)))
+    now = 100_000 + int(rng.integers(0, 5000))
+    d = cs.DeviceIndex.from_host(idx, DEV)
+    if n:
+        s64, s32 = o.scores(idx, now)
+        got = c.score_blocks(d, now).cpu().numpy()
+        assert np.all(np.abs(got - s64) <= H.REL_TOL * s64)
+        if kw["lam"] not in (0.003,):                  # (a table that does not cover every age may differ in the last bit)
+            assert np.mean(got == s32) > 0.999
+    ks = sorted({1, int(rng.integers(1, n + 1)), n})
+    assert run_selects(c, o, idx, now, ks) == 0
