@@ -690,3 +690,62 @@ def test_random_small_configurations(case):
             assert np.mean(got == s32) > 0.999
     ks = sorted({1, int(rng.integers(1, n + 1)), n})
     assert run_selects(c, o, idx, now, ks) == 0
+
+
+@pytest.mark.parametrize("case", range(16))
+def test_random_mover_geometries(case):
+    """Seeded random block geometries (layers, heads, head size, tokens, element size), layouts, id offsets, list
+    lengths and sentinels: offload, prefetch, compaction (bulk and load/store paths) and the two-way transfer."""
+    rng = np.random.default_rng(9000 + case)
+    L, heads = int(rng.integers(1, 7)), int(rng.choice([1, 2, 3, 8]))
+    hd, tok, eb = int(rng.choice([8, 40, 64, 128])), int(rng.choice([1, 4, 9, 16])), int(rng.choice([1, 2, 4]))
+    chunk = tok * heads * hd * eb
+    if chunk % 16:
+        hd, chunk = 128, tok * heads * 128 * eb
+    G, Hs = int(rng.integers(20, 60)), int(rng.integers(20, 60))
+    lay_g, lay_h = int(rng.integers(0, 2)), int(rng.integers(0, 2))
+    first_h = int(rng.choice([0, G, 1000]))
+    c = cs.CacheScout(cs.make_params(n_agents=4, max_blocks=64), DEV)
+    c.set_mover_path(cs.CS_MOVER_LDST if case % 4 == 3 else cs.CS_MOVER_BULK)
+    c.set_mover_ctas(int(rng.choice([0, 1, 5, 40])), int(rng.choice([0, 3, 64])))
+    gpu_np = rng.integers(0, 256, G * L * 2 * chunk, dtype=np.uint8)
+    host_np = rng.integers(0, 256, Hs * L * 2 * chunk, dtype=np.uint8)
+    gpu = cs.KVPool(dev(gpu_np), G, lay_g, L, heads, hd, tok, eb)
+    host_t = torch.from_numpy(host_np.copy()).pin_memory()
+    host = cs.KVPool(host_t, Hs, lay_h, L, heads, hd, tok, eb, first_id=first_h)
+    n_off, n_pre = int(rng.integers(0, 12)), int(rng.integers(0, 12))
+    g_perm, h_perm = rng.permutation(G).astype(np.uint32), rng.permutation(Hs).astype(np.uint32)
+    off_src, pre_dst = g_perm[:n_off].copy(), g_perm[n_off:n_off + n_pre].copy()
+    off_dst, pre_src = h_perm[:n_off] + np.uint32(first_h), h_perm[n_off:n_off + n_pre] + np.uint32(first_h)
+    if n_off > 2:
+        off_src[1] = orc.ID_NONE
+    if n_pre > 2:
+        pre_src[0] = orc.ID_NONE
+    opt = lambda a: dev(a) if len(a) else None
+    c.exchange_blocks(gpu, host, opt(off_src), opt(off_dst), opt(pre_src), opt(pre_dst))
+    torch.cuda.synchronize()
+    want_h, want_g = host_np.copy(), gpu_np.copy()
+    unoff = lambda a: np.where(a == orc.ID_NONE, a, a - np.uint32(first_h))
+    orc.move_blocks(gpu_np, lay_g, G, want_h, lay_h, Hs, L, chunk, off_src, unoff(off_dst))
+    orc.move_blocks(host_np, lay_h, Hs, want_g, lay_g, G, L, chunk, unoff(pre_src), pre_dst)
+    assert np.array_equal(host_t.numpy(), want_h) and np.array_equal(gpu.buf.cpu().numpy(), want_g)
+    # the single calls, starting from the state just reached
+    n = int(rng.integers(1, 15))
+    s_g, d_h = rng.permutation(G).astype(np.uint32)[:n], rng.permutation(Hs).astype(np.uint32)[:n] + np.uint32(first_h)
+    c.offload_blocks(gpu, host, dev(s_g), dev(d_h))
+    torch.cuda.synchronize()
+    orc.move_blocks(want_g, lay_g, G, want_h, lay_h, Hs, L, chunk, s_g, unoff(d_h))
+    assert np.array_equal(host_t.numpy(), want_h)
+    back = rng.permutation(G).astype(np.uint32)[:n]
+    c.prefetch_blocks(host, gpu, dev(d_h), dev(back))
+    torch.cuda.synchronize()
+    src_h = want_h.copy()
+    orc.move_blocks(src_h, lay_h, Hs, want_g, lay_g, G, L, chunk, unoff(d_h), back)
+    assert np.array_equal(gpu.buf.cpu().numpy(), want_g)
+    stage = cs.KVPool(torch.zeros(n * L * 2 * chunk, dtype=torch.uint8, device=DEV), n, 1 - lay_g, L, heads, hd, tok, eb)
+    c.compact_blocks(gpu, stage, dev(back), dev(np.arange(n, dtype=np.uint32)))
+    torch.cuda.synchronize()
+    want_s = np.zeros(n * L * 2 * chunk, np.uint8)
+    orc.move_blocks(want_g, lay_g, G, want_s, 1 - lay_g, n, L, chunk, back, np.arange(n))
+    assert np.array_equal(stage.buf.cpu().numpy(), want_s)
+    assert c.get_status() == 0
