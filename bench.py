@@ -214,6 +214,8 @@ class StepWorkload:
         self.fifo = [torch.zeros(self.k_p, dtype=torch.int64, device=device) for _ in range(8)]
         self.fifo_used = 0
         self.bytes_per_step = (self.k_v + self.k_p) * bb
+        # blocks actually moved, counted on the device from the select counts of every step: [offloaded, prefetched]
+        self.moved = torch.zeros(2, dtype=torch.int64, device=device)
         self.timers = {"select": [], "compact": [], "offload": [], "prefetch": [], "observe": []}
         # warm the learner so that the prefetch gate has something to work with
         self.c.observe_invocations(self.d_chain[:2000], self.d_agent[:2000], self.d_flags[:2000])
@@ -258,6 +260,8 @@ class StepWorkload:
             c.select_victims(self.didx, now, 1, self.k_v, self.hv[b], self.hn[b])
             c.select_prefetch(self.didx, now, self.k_p, self.pf[b], self.pn[b])
         rec(t[2], main)
+        self.moved[0] += torch.minimum(self.vn[b][0], self.hn[b][0])       # a victim without a host slot is skipped
+        self.moved[1] += self.pn[b][0]
         c.compact_blocks(self.gpu_pool, self.stage_pool, vict, self.packed, n_max=self.k_v, n_dev=self.vn[b])
         rec(t[3], main)
         ready = torch.cuda.Event()
@@ -341,6 +345,12 @@ class StepWorkload:
             self.timers["offload"].append(t[4].elapsed_time(t[5]))
             self.timers["prefetch"].append(t[6].elapsed_time(t[7]))
         self._pending = []
+
+    def take_moved_bytes(self):
+        """KV bytes the steps since the last call really moved over the link (device-side counts), then reset."""
+        n = int(self.moved.sum().item())
+        self.moved.zero_()
+        return n * self.cfg.block_bytes
 
     def e2e_bytes(self):
         ev = 8 * 7          # <= 8 events x (4 + 2 + 1) bytes
@@ -969,6 +979,7 @@ def main():
     if rank == 0:
         sampler.start()
     l0 = w.c.launch_count()
+    w.take_moved_bytes()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(w.main)
     for s in range(args.steps):
@@ -977,6 +988,7 @@ def main():
     e1.record(w.main)
     barrier()
     clocks = sampler.stop() if rank == 0 else None
+    moved_bytes = w.take_moved_bytes()                 # what the timed steps really moved (this rank)
     launches = w.c.launch_count() - l0
     total_ms = reduce_max_ms(e0.elapsed_time(e1), world, device)
     w.collect_timers()
@@ -988,7 +1000,7 @@ def main():
     if args.skip_aux:
         if rank == 0:
             print(json.dumps({"workload": "step", "ms_per_step": total_ms / args.steps, "gpu_launches": int(launches),
-                              "value": job_value(world, w.bytes_per_step, args.steps, total_ms), "n_out": n_out}))
+                              "value": job_value(world, moved_bytes / args.steps, args.steps, total_ms), "n_out": n_out}))
         if world > 1:
             dist.destroy_process_group()
         return
@@ -999,6 +1011,7 @@ def main():
         w.step(base + s, e2e=True)
     w.drain()
     barrier()
+    w.take_moved_bytes()
     f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     f0.record(w.main)
     for s in range(args.steps):
@@ -1007,14 +1020,15 @@ def main():
     f1.record(w.main)
     barrier()
     e2e_ms = reduce_max_ms(f0.elapsed_time(f1), world, device)
+    e2e_moved = w.take_moved_bytes()
 
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
 
-    value = job_value(world, w.bytes_per_step, args.steps, total_ms)
-    e2e_value = job_value(world, w.bytes_per_step, args.steps, e2e_ms)
+    value = job_value(world, moved_bytes / args.steps, args.steps, total_ms)
+    e2e_value = job_value(world, e2e_moved / args.steps, args.steps, e2e_ms)
     bb = w.cfg.block_bytes
     med = lambda k: float(np.median(w.timers[k])) if w.timers[k] else None
     t_c, t_o, t_p, t_s, t_ob = med("compact"), med("offload"), med("prefetch"), med("select"), med("observe")
@@ -1040,6 +1054,8 @@ def main():
                                    w.cfg.gpu_blocks, w.cfg.host_blocks, w.host_backed, w.N),
                    "l2_policy": "inputs larger than L2: every step moves 1.75 GiB of scattered blocks; index 0.9 MB is L2-resident by design",
                    "replicas": "replicas only (no data-path collective)", "pin_seconds": round(w.t_pin, 2), "quick": bool(args.quick)},
+        "blocks_moved_in_timed_steps": {"counted_on_device": moved_bytes // w.cfg.block_bytes,
+                                        "nominal": args.steps * (w.k_v + w.k_p)},
         "blocks_scored_selected_per_s": world * 3 * w.N / (t_s / 1e3),
         "gpu_launches": int(launches),
         "clocks": clocks,
