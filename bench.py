@@ -389,6 +389,7 @@ def fused_step_section(w, steps=10):
     ev_f = torch.zeros(cap, dtype=w.d_flags.dtype, device=dev)
     fifo = [torch.zeros(kp, dtype=torch.int64, device=dev) for _ in range(8)]
     state = {"s": w.last_s + 1, "n": 0}
+    moved = torch.zeros(1, dtype=torch.int64, device=dev)
 
     def issue(by_value, now=0, n_ev=cap):
         c.step(w.didx, now, ev_c, ev_a, ev_f, n_ev, kv, kp, gv, gvn, gh, ghn, gp, gpn, w.gpu_pool, w.host_pool, free_d,
@@ -407,6 +408,7 @@ def fused_step_section(w, steps=10):
             issue(True, now, n_ev)
         else:
             graph.replay()
+        moved.add_(torch.minimum(gvn[0], ghn[0]) + gpn[0])           # blocks this step really moves
         # engine bookkeeping, as in the main run
         vi = gv[:kv].long().clamp_(min=0)
         w.la_i32[vi] = now
@@ -427,25 +429,27 @@ def fused_step_section(w, steps=10):
             main.synchronize()
             l0 = c.launch_count()
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            moved.zero_()
             e0.record(main)
             for _ in range(k):
                 one_step(graph)
             e1.record(main)
             main.synchronize()
-        return e0.elapsed_time(e1) / k, (c.launch_count() - l0) / k
+        ms = e0.elapsed_time(e1) / k
+        return ms, (c.launch_count() - l0) / k, int(moved.item()) * bb / k / ms / 1e6
 
     w.drain()
     torch.cuda.synchronize(dev)
     with torch.cuda.stream(main):                               # buffers made above belong to this stream from here on
         pass
-    ms_call, launches_call = timed(None, steps)
+    ms_call, launches_call, gbps_call = timed(None, steps)
     g = torch.cuda.CUDAGraph()
     with torch.cuda.graph(g, stream=main, capture_error_mode="relaxed"):
         issue(False)
-    ms_graph, _ = timed(g, steps)
+    ms_graph, _, gbps_graph = timed(g, steps)
     out = {"what": "cs_step: observe + 3 selects + conflict filter + compaction + two-way transfer as one call; steps back to back, no overlap between steps",
-           "ms_per_step_call": ms_call, "GBps_call": w.bytes_per_step / ms_call / 1e6, "kernel_launches_per_step": launches_call,
-           "ms_per_step_graph_replay": ms_graph, "GBps_graph_replay": w.bytes_per_step / ms_graph / 1e6,
+           "ms_per_step_call": ms_call, "GBps_call": gbps_call, "kernel_launches_per_step": launches_call,
+           "ms_per_step_graph_replay": ms_graph, "GBps_graph_replay": gbps_graph,
            "n_out_last_step": [int(gvn[0].item()), int(ghn[0].item()), int(gpn[0].item())], "device_status": c.get_status()}
 
     # ---- interference with synthetic serving kernels ------------------------------------------------------
