@@ -390,6 +390,7 @@ def fused_step_section(w, steps=10):
     fifo = [torch.zeros(kp, dtype=torch.int64, device=dev) for _ in range(8)]
     state = {"s": w.last_s + 1, "n": 0}
     moved = torch.zeros(1, dtype=torch.int64, device=dev)
+    ar_kp = torch.arange(kp, dtype=torch.int32, device=dev)
 
     def issue(by_value, now=0, n_ev=cap):
         c.step(w.didx, now, ev_c, ev_a, ev_f, n_ev, kv, kp, gv, gvn, gh, ghn, gp, gpn, w.gpu_pool, w.host_pool, free_d,
@@ -408,7 +409,8 @@ def fused_step_section(w, steps=10):
             issue(True, now, n_ev)
         else:
             graph.replay()
-        moved.add_(torch.minimum(gvn[0], ghn[0]) + gpn[0])           # blocks this step really moves
+        # blocks this step really moves (prefetch candidates dropped by the conflict rule are sentinels in the list)
+        moved.add_(torch.minimum(gvn[0], ghn[0]) + ((gp[:kp] >= 0) & (ar_kp < gpn[0])).sum())
         # engine bookkeeping, as in the main run
         vi = gv[:kv].long().clamp_(min=0)
         w.la_i32[vi] = now
