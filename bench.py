@@ -260,8 +260,6 @@ class StepWorkload:
             c.select_victims(self.didx, now, 1, self.k_v, self.hv[b], self.hn[b])
             c.select_prefetch(self.didx, now, self.k_p, self.pf[b], self.pn[b])
         rec(t[2], main)
-        self.moved[0] += torch.minimum(self.vn[b][0], self.hn[b][0])       # a victim without a host slot is skipped
-        self.moved[1] += self.pn[b][0]
         c.compact_blocks(self.gpu_pool, self.stage_pool, vict, self.packed, n_max=self.k_v, n_dev=self.vn[b])
         rec(t[3], main)
         ready = torch.cuda.Event()
@@ -308,6 +306,9 @@ class StepWorkload:
             rec(t[7], self.side_p)
             self.done_p[b] = torch.cuda.Event()
             self.done_p[b].record(self.side_p)
+        # accounting, after the transfers have been issued: blocks this step really moves
+        self.moved[0] += torch.minimum(self.vn[b][0], self.hn[b][0])       # a victim without a host slot is skipped
+        self.moved[1] += self.pn[b][0]
         # engine bookkeeping (plumbing, not the method): refilled victim slots are touched now, prefetched
         # host entries now have a GPU copy
         vi = vict.long().clamp_(min=0)
