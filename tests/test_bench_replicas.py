@@ -44,3 +44,17 @@ def test_reference_arm_prints_on_rank_zero_only():
     r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--steps", "1",
                         "--warmup", "0"], capture_output=True, text=True, env=env, timeout=300)
     assert r.returncode == 0 and r.stdout.strip() == ""
+
+
+def test_in_flight_slowdown_factor():
+    """The overlap arithmetic of the interference study: a loop that outlasts the transfer does transfer_ms / f of
+    its work while the transfer runs and the rest at full speed."""
+    import bench
+    # 20 ms of work, transfer 10 ms, everything 2x slower while it runs: 5 ms of work done in 10 ms, 15 ms left
+    assert bench.in_flight_factor(20.0, 25.0, 10.0) == pytest.approx(2.0)
+    # no disturbance at all
+    assert bench.in_flight_factor(20.0, 20.0, 10.0) == pytest.approx(1.0)
+    # the loop ends before the transfer does: plain ratio
+    assert bench.in_flight_factor(5.0, 12.0, 16.0) == pytest.approx(2.4)
+    # nothing got done while the transfer ran
+    assert bench.in_flight_factor(20.0, 30.0, 10.0) == float("inf")
