@@ -72,3 +72,17 @@ def test_product_path_has_no_cpu_fallback():
         pytest.skip("GPU present")
     with pytest.raises(RuntimeError):
         cs.CacheScout(cs.make_params(n_agents=4), "cuda:0")
+
+
+def test_header_is_plain_c_and_cxx():
+    """The boundary header must be usable from C (C99) and from C++ without anything else included."""
+    import shutil
+    import subprocess
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    src = '#include "cachescout.h"\nint use(void) { cs_params p = {0}; cs_step_io io = {0}; return (int)p.n_agents + (int)io.now; }\n'
+    for cc, std, lang in (("gcc", "-std=c99", "c"), ("g++", "-std=c++17", "c++")):
+        if shutil.which(cc) is None:
+            pytest.skip("no %s here" % cc)
+        r = subprocess.run([cc, std, "-Wall", "-Werror", "-pedantic", "-fsyntax-only", "-I", os.path.join(root, "include"),
+                            "-x", lang, "-"], input=src, capture_output=True, text=True)
+        assert r.returncode == 0, r.stderr
