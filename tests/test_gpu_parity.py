@@ -578,7 +578,7 @@ def test_survival_from_all_chains(name, n_inv):
 @pytest.mark.parametrize("name,n,kv,kp", [
     ("tiny", 2560, 32, 64), ("tiny", 0, 4, 4), ("tiny", 5, 8, 1), ("tiny", 1029, 1029, 700),
     ("llama8b", 80000, 256, 384), ("llama8b", 80000, 9000, 6000), ("llama70b", 52000 + 5, 128, 192),
-    ("meta1m", 262144, 10000, 2000), ("meta1m", 300000, 500, 500)])
+    ("meta1m", 262144, 10000, 2000), ("meta1m", 300000, 500, 500), ("meta1m", 1_000_000, 10000, 2000)])
 @pytest.mark.parametrize("path", [cs.CS_SELECT_AUTO, cs.CS_SELECT_MULTI])
 def test_select_step_matches_three_calls_and_oracle(name, n, kv, kp, path):
     """cs_select_step: one launch of three clusters where the single-launch select applies, three kernel chains
