@@ -55,6 +55,8 @@ typedef struct CUstream_st *cs_stream_t;   /* the same type as cudaStream_t */
 #define CS_ST_BAD_SLOT 4u       /* a mover list entry named a slot >= n_slots */
 #define CS_ST_BAD_SOURCE 8u     /* a BFS source >= n_agents */
 #define CS_ST_TIMEOUT 16u       /* a bounded wait inside a kernel ran out; the transfer is incomplete */
+#define CS_ST_LIST_CONFLICT 32u /* cs_validate_*_lists(): a slot is written twice, or written and read, by one transfer */
+#define CS_ST_BAD_SELECTION 64u /* cs_validate_selection(): a list is not the ordered k best eligible entries */
 
 /* ---- sentinels ---------------------------------------------------------------------------- */
 #define CS_AGENT_NONE 0xFFFFu      /* "no current agent yet" (the initial state of Algorithm 1) */
@@ -304,12 +306,67 @@ int cs_get_model(cs_ctx *ctx, uint32_t *C_out, float *P_out, uint16_t *amax_out,
 int cs_import_state(cs_ctx *ctx, const uint32_t *C_in, const uint16_t *cur_in, uint32_t last_agent,
                     cs_stream_t stream);
 
-/* Synchronises `stream`, returns the device status word in *device_status and clears it.
- * Returns CS_EDEVICE_STATUS when it was non-zero. */
+/* Returns the device status word in *device_status and clears it: one small kernel on `stream` swaps the
+ * word with zero atomically, the call then synchronises `stream` and reads the swapped-out value.  Bits
+ * that a kernel on another stream (a transfer on a side stream) sets after the swap stay for the next
+ * call; for an exact report of a finished step, order the side stream before `stream` first.
+ * Returns CS_EDEVICE_STATUS when the word was non-zero. */
 int cs_get_status(cs_ctx *ctx, uint32_t *device_status, cs_stream_t stream);
 
 /* Number of kernels this context has launched so far (host counter). */
 int cs_launch_count(cs_ctx *ctx, uint64_t *n_launches);
+
+/* Work counters kept in the workspace by the kernels themselves (the paper reports only hit rate and
+ * latency, Sec. 5.1; these are this library's metrics).  All cumulative since cs_create() or the last
+ * reset, except `eligible`, which describes the latest select of each kind.  Kinds: 0 GPU-tier victims,
+ * 1 host-tier victims, 2 prefetch candidates; directions: 0 device-to-device, 1 offload, 2 prefetch. */
+typedef struct cs_counters {
+    uint64_t events_seen;           /* events handed to cs_observe_invocations() */
+    uint64_t events_skipped;        /* of those: warmup-flagged, or agent / chain out of range */
+    uint64_t transitions_counted;   /* increments of the transition counts (agent changes) */
+    uint64_t selects[3];            /* selects completed, per kind */
+    uint64_t eligible[3];           /* eligible entries the latest select of the kind saw */
+    uint64_t selected[3];           /* ids emitted, per kind */
+    uint64_t blocks_moved[3];       /* blocks copied, per direction */
+    uint64_t bytes_moved[3];        /* their bytes (block_bytes each) */
+    uint64_t blocks_skipped;        /* mover list entries skipped: CS_ID_NONE or slot out of range */
+} cs_counters;
+
+/* Synchronises `stream` and copies the counters to *out (host memory); reset != 0 clears them afterwards. */
+int cs_get_counters(cs_ctx *ctx, cs_counters *out, uint32_t reset, cs_stream_t stream);
+
+/* ---- checkers (debugging aids; the paper has no counterpart) ------------------------------------------ */
+
+/* Checks a select result on the device, independently of how it was produced: ids_out[0, n) name eligible
+ * entries (same rules as cs_select_victims / cs_select_prefetch with these arguments), their keys are
+ * strictly increasing (so the ids are unique), exactly n eligible entries have a key at or below the last
+ * one, n = min(k, number eligible), and ids_out[n, k) hold CS_ID_NONE.  Any violation sets
+ * CS_ST_BAD_SELECTION in the status word.  One scan of the index; run it on the stream of the select.
+ * prefetch != 0 checks a cs_select_prefetch() list (tier is then ignored). */
+int cs_validate_selection(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, uint32_t prefetch, uint32_t tier,
+                          uint32_t k, const uint32_t *ids_out, const uint32_t *n_out, cs_stream_t stream);
+
+/* Checks the slot lists of a mover call before it is issued (arguments as for cs_compact_blocks /
+ * cs_offload_blocks / cs_prefetch_blocks): two entries with the same destination slot, or -- when src and
+ * dst are the same pool -- a slot that is both read and written, set CS_ST_LIST_CONFLICT.  Entries the
+ * mover would skip (CS_ID_NONE on either side) are ignored.  Cost: n^2 id compares. */
+int cs_validate_move_lists(cs_ctx *ctx, const cs_kv_pool *src, const cs_kv_pool *dst, const uint32_t *src_slots,
+                           const uint32_t *dst_slots, uint32_t n_max, const uint32_t *n_dev, cs_stream_t stream);
+
+/* The same for the two transfers of cs_exchange_blocks() (same arguments): each list on its own, plus
+ * host slots written by the offload and read by the prefetch, and GPU slots read by the offload and written
+ * by the prefetch. */
+int cs_validate_exchange_lists(cs_ctx *ctx, const cs_kv_pool *gpu, const cs_kv_pool *host,
+                               const uint32_t *off_gpu_slots, const uint32_t *off_host_slots, uint32_t n_off_max,
+                               const uint32_t *n_off_dev, const uint32_t *pre_host_slots, const uint32_t *pre_gpu_slots,
+                               uint32_t n_pre_max, const uint32_t *n_pre_dev, cs_stream_t stream);
+
+/* Self-test of the mover's bounded wait (no counterpart in the paper).  Launches one warp that sets up a
+ * transfer barrier, issues NO copy, and waits on the barrier with the mover's own wait routine limited to
+ * `max_polls` polls (1 .. 1,000,000).  Nothing can complete the barrier, so the wait runs out, the kernel
+ * sets CS_ST_TIMEOUT in the status word -- the path a stalled transfer would take -- and returns.  No data
+ * is in flight, so nothing is left behind; the context stays usable. */
+int cs_selftest_bounded_wait(cs_ctx *ctx, uint32_t max_polls, cs_stream_t stream);
 
 /* Width of the mover (0 keeps the default): for transfers that cross the host link and for
  * device-to-device moves.  Unit: warp pipelines on the bulk path (each keeps up to two loads and two

@@ -24,7 +24,7 @@ CS_EV_WARMUP = 1
 CS_LAYER_MAJOR, CS_BLOCK_MAJOR = 0, 1
 CS_STATIC_MAX_BLOCKS = 65536
 CS_MOVER_AUTO, CS_MOVER_LDST, CS_MOVER_BULK = 0, 1, 2
-CS_ST_TIMEOUT = 16
+CS_ST_TIMEOUT, CS_ST_LIST_CONFLICT, CS_ST_BAD_SELECTION = 16, 32, 64
 CS_SELECT_AUTO, CS_SELECT_CLUSTER, CS_SELECT_MULTI = 0, 1, 2
 
 # every symbol include/cachescout.h declares
@@ -32,7 +32,9 @@ EXPORTS = ("cs_workspace_bytes", "cs_create", "cs_destroy", "cs_observe_invocati
            "cs_select_victims", "cs_select_prefetch", "cs_offload_blocks", "cs_prefetch_blocks",
            "cs_compact_blocks", "cs_get_model", "cs_get_status", "cs_launch_count", "cs_set_mover_ctas",
            "cs_last_cuda_error", "cs_strerror", "cs_version", "cs_select_victims_static", "cs_set_mover_path", "cs_set_select_path",
-           "cs_exact_survival", "cs_use_survival_table", "cs_import_state", "cs_set_select_speculation", "cs_exchange_blocks", "cs_step", "cs_set_survival_sources", "cs_select_step")
+           "cs_exact_survival", "cs_use_survival_table", "cs_import_state", "cs_set_select_speculation", "cs_exchange_blocks", "cs_step", "cs_set_survival_sources", "cs_select_step",
+           "cs_get_counters", "cs_validate_selection", "cs_validate_move_lists", "cs_validate_exchange_lists",
+           "cs_selftest_bounded_wait")
 
 
 class cs_params(C.Structure):
@@ -62,6 +64,12 @@ class cs_step_io(C.Structure):
                 ("n_host_victims", C.c_void_p), ("prefetch_ids", C.c_void_p), ("n_prefetch", C.c_void_p),
                 ("gpu", C.POINTER(cs_kv_pool)), ("host", C.POINTER(cs_kv_pool)), ("stage", C.POINTER(cs_kv_pool)),
                 ("stage_slots", C.c_void_p), ("free_gpu_slots", C.c_void_p), ("join_main", C.c_uint32)]
+
+
+class cs_counters(C.Structure):
+    _fields_ = [("events_seen", C.c_uint64), ("events_skipped", C.c_uint64), ("transitions_counted", C.c_uint64),
+                ("selects", C.c_uint64 * 3), ("eligible", C.c_uint64 * 3), ("selected", C.c_uint64 * 3),
+                ("blocks_moved", C.c_uint64 * 3), ("bytes_moved", C.c_uint64 * 3), ("blocks_skipped", C.c_uint64)]
 
 
 class CacheScoutError(RuntimeError):
@@ -112,6 +120,12 @@ def lib():
         L.cs_exact_survival.argtypes = [vp, u32, u32, vp, vp, vp]
         L.cs_use_survival_table.argtypes = [vp, vp]
         L.cs_import_state.argtypes = [vp, vp, vp, u32, vp]
+        L.cs_get_counters.argtypes = [vp, C.POINTER(cs_counters), u32, vp]
+        L.cs_validate_selection.argtypes = [vp, C.POINTER(cs_block_index), u32, u32, u32, u32, vp, vp, vp]
+        L.cs_validate_move_lists.argtypes = [vp, C.POINTER(cs_kv_pool), C.POINTER(cs_kv_pool), vp, vp, u32, vp, vp]
+        L.cs_validate_exchange_lists.argtypes = [vp, C.POINTER(cs_kv_pool), C.POINTER(cs_kv_pool), vp, vp, u32, vp, vp, vp,
+                                                 u32, vp, vp]
+        L.cs_selftest_bounded_wait.argtypes = [vp, u32, vp]
         _lib = L
     return _lib
 
@@ -241,6 +255,35 @@ def cs_get_status(ctx, stream=None, raise_on_set: bool = False) -> int:
     if code not in (CS_OK, CS_EDEVICE_STATUS) or (raise_on_set and code != CS_OK):
         _chk(code, "cs_get_status", ctx)
     return int(st.value)
+
+
+def cs_get_counters(ctx, reset: bool = False, stream=None) -> dict:
+    """Work counters kept by the kernels (synchronises the stream); plain ints and lists of three."""
+    out = cs_counters()
+    _chk(lib().cs_get_counters(ctx, C.byref(out), 1 if reset else 0, _stream(stream)), "cs_get_counters", ctx)
+    return {name: (list(getattr(out, name)) if hasattr(getattr(out, name), "__len__") else int(getattr(out, name)))
+            for name, _ in cs_counters._fields_}
+
+
+def cs_validate_selection(ctx, idx: cs_block_index, now: int, prefetch: bool, tier: int, k: int, ids_out, n_out, stream=None):
+    _chk(lib().cs_validate_selection(ctx, C.byref(idx), now, 1 if prefetch else 0, tier, k, _ptr(ids_out), _ptr(n_out),
+                                     _stream(stream)), "cs_validate_selection", ctx)
+
+
+def cs_validate_move_lists(ctx, src: cs_kv_pool, dst: cs_kv_pool, src_slots, dst_slots, n_max: int, n_dev=None, stream=None):
+    _chk(lib().cs_validate_move_lists(ctx, C.byref(src), C.byref(dst), _ptr(src_slots), _ptr(dst_slots), n_max,
+                                      _ptr(n_dev), _stream(stream)), "cs_validate_move_lists", ctx)
+
+
+def cs_validate_exchange_lists(ctx, gpu: cs_kv_pool, host: cs_kv_pool, off_gpu_slots, off_host_slots, n_off_max: int,
+                               n_off_dev, pre_host_slots, pre_gpu_slots, n_pre_max: int, n_pre_dev, stream=None):
+    _chk(lib().cs_validate_exchange_lists(ctx, C.byref(gpu), C.byref(host), _ptr(off_gpu_slots), _ptr(off_host_slots),
+                                          n_off_max, _ptr(n_off_dev), _ptr(pre_host_slots), _ptr(pre_gpu_slots),
+                                          n_pre_max, _ptr(n_pre_dev), _stream(stream)), "cs_validate_exchange_lists", ctx)
+
+
+def cs_selftest_bounded_wait(ctx, max_polls: int, stream=None):
+    _chk(lib().cs_selftest_bounded_wait(ctx, max_polls, _stream(stream)), "cs_selftest_bounded_wait", ctx)
 
 
 def cs_launch_count(ctx) -> int:
@@ -469,6 +512,28 @@ class CacheScout:
 
     def launch_count(self) -> int:
         return cs_launch_count(self.ctx)
+
+    def counters(self, reset: bool = False, stream=None) -> dict:
+        return cs_get_counters(self.ctx, reset, stream)
+
+    def validate_selection(self, idx: DeviceIndex, now: int, prefetch: bool, tier: int, k: int, ids_out, n_out, stream=None):
+        cs_validate_selection(self.ctx, idx.struct(), now, prefetch, tier, k, ids_out, n_out, stream)
+
+    def validate_move_lists(self, src: KVPool, dst: KVPool, src_slots, dst_slots, n_max=None, n_dev=None, stream=None):
+        cs_validate_move_lists(self.ctx, src.struct(), dst.struct(), src_slots, dst_slots,
+                               int(src_slots.numel()) if n_max is None else n_max, n_dev, stream)
+
+    def validate_exchange_lists(self, gpu: KVPool, host: KVPool, off_gpu_slots, off_host_slots, pre_host_slots,
+                                pre_gpu_slots, n_off_max=None, n_off_dev=None, n_pre_max=None, n_pre_dev=None, stream=None):
+        if n_off_max is None:
+            n_off_max = 0 if off_gpu_slots is None else int(off_gpu_slots.numel())
+        if n_pre_max is None:
+            n_pre_max = 0 if pre_host_slots is None else int(pre_host_slots.numel())
+        cs_validate_exchange_lists(self.ctx, gpu.struct(), host.struct(), off_gpu_slots, off_host_slots, n_off_max,
+                                   n_off_dev, pre_host_slots, pre_gpu_slots, n_pre_max, n_pre_dev, stream)
+
+    def selftest_bounded_wait(self, max_polls: int = 1000, stream=None):
+        cs_selftest_bounded_wait(self.ctx, max_polls, stream)
 
     def exact_survival(self, n_steps: int, a0: int = CS_AGENT_NONE, stream=None):
         """Eq. 6 for every agent: returns (p_surv, p_surv + delta) as device tensors."""

@@ -50,6 +50,7 @@ size_t cs_layout_workspace(const cs_params *p, uint32_t gtab_len, void *base, cs
         off = align_up(off + sizeof(type) * (size_t)(count), 256); \
     } while (0)
     TAKE(sc, cs_scalars, 1);
+    TAKE(cnt, cs_counters, 1);
     TAKE(sel, cs_sel_state, 1);
     TAKE(C, uint32_t, A * A);
     TAKE(rowsum, uint32_t, A);
@@ -128,9 +129,25 @@ cs_step_filter_kernel(uint32_t *__restrict__ prefetch_ids, const uint32_t *__res
     if (hit) prefetch_ids[i] = CS_ID_NONE;
 }
 
+// Memory the SMs cannot address (pageable host memory that was never registered) would fault the GPU, so pool
+// bases and index arrays are looked up before every launch (a host-side query of about a microsecond): device memory,
+// pinned / registered host memory and managed memory pass.
+bool cs_device_can_address(const void *ptr)
+{
+    cudaPointerAttributes at;
+    if (cudaPointerGetAttributes(&at, ptr) != cudaSuccess) { (void)cudaGetLastError(); return false; }
+    return at.type == cudaMemoryTypeDevice || at.type == cudaMemoryTypeHost || at.type == cudaMemoryTypeManaged;
+}
+
+// cs_get_status(): read and clear in one atomic step, so that a bit another stream sets in between is kept.
+__global__ void cs_status_swap_kernel(cs_scalars *sc)
+{
+    sc->status_read = atomicExch(&sc->status, 0u);
+}
+
 extern "C" {
 
-int cs_version(void) { return 100; }
+int cs_version(void) { return 200; }
 
 const char *cs_strerror(int code)
 {
@@ -222,16 +239,6 @@ int cs_observe_invocations(cs_ctx *ctx, const uint32_t *chain, const uint16_t *a
     return cs_launch_observe(ctx, chain, agent, evflags, n_events, (cudaStream_t)stream);
 }
 
-// Memory the SMs cannot address (pageable host memory that was never registered) would fault the GPU, so pool
-// bases and index arrays are looked up before every launch (a host-side query of about a microsecond): device memory,
-// pinned / registered host memory and managed memory pass.
-static bool device_can_address(const void *ptr)
-{
-    cudaPointerAttributes at;
-    if (cudaPointerGetAttributes(&at, ptr) != cudaSuccess) { (void)cudaGetLastError(); return false; }
-    return at.type == cudaMemoryTypeDevice || at.type == cudaMemoryTypeHost || at.type == cudaMemoryTypeManaged;
-}
-
 static int check_index(const cs_ctx *ctx, const cs_block_index *idx)
 {
     if (!idx) return CS_EINVAL;
@@ -245,7 +252,7 @@ static int check_index(const cs_ctx *ctx, const cs_block_index *idx)
     const void *arrays[7] = {idx->agent, idx->depth, idx->ref_count, idx->flags, idx->last_access, idx->n_tokens,
                              idx->anchor_blocks};
     for (int i = 0; i < 7; ++i)
-        if (arrays[i] && !device_can_address(arrays[i])) return CS_EINVAL;     // a host array would fault the kernels
+        if (arrays[i] && !cs_device_can_address(arrays[i])) return CS_EINVAL;     // a host array would fault the kernels
     return CS_OK;
 }
 
@@ -332,7 +339,7 @@ static int mover_common(cs_ctx *ctx, const cs_kv_pool *src, const cs_kv_pool *ds
     if (!ctx) return CS_EINVAL;
     int rc = check_pools(src, dst);
     if (rc != CS_OK) return rc;
-    if (!device_can_address(src->base) || !device_can_address(dst->base)) return CS_EINVAL;
+    if (!cs_device_can_address(src->base) || !cs_device_can_address(dst->base)) return CS_EINVAL;
     if (n_max == 0) return CS_OK;
     if (!src_slots || !dst_slots || (((uintptr_t)src_slots) & 3u) || (((uintptr_t)dst_slots) & 3u)) return CS_EINVAL;
     if (n_dev && (((uintptr_t)n_dev) & 3u)) return CS_EINVAL;
@@ -365,7 +372,7 @@ int cs_exchange_blocks(cs_ctx *ctx, const cs_kv_pool *gpu, const cs_kv_pool *hos
     if (!ctx) return CS_EINVAL;
     int rc = check_pools(gpu, host);
     if (rc != CS_OK) return rc;
-    if (!device_can_address(gpu->base) || !device_can_address(host->base)) return CS_EINVAL;
+    if (!cs_device_can_address(gpu->base) || !cs_device_can_address(host->base)) return CS_EINVAL;
     if (n_off_max == 0 && n_pre_max == 0) return CS_OK;
     const uint32_t *lists[4] = {off_gpu_slots, off_host_slots, pre_host_slots, pre_gpu_slots};
     for (int i = 0; i < 4; ++i) {
@@ -455,13 +462,90 @@ int cs_get_status(cs_ctx *ctx, uint32_t *device_status, cs_stream_t stream)
     if (!ctx || !device_status) return CS_EINVAL;
     cudaStream_t s = (cudaStream_t)stream;
     uint32_t st = 0;
-    cudaError_t e = cudaMemcpyAsync(&st, &ctx->ws.sc->status, sizeof(st), cudaMemcpyDeviceToHost, s);
+    cs_status_swap_kernel<<<1, 1, 0, s>>>(ctx->ws.sc);
+    int rc = cs_check_launch(ctx);
+    if (rc != CS_OK) return rc;
+    cudaError_t e = cudaMemcpyAsync(&st, &ctx->ws.sc->status_read, sizeof(st), cudaMemcpyDeviceToHost, s);
     if (e == cudaSuccess) e = cudaStreamSynchronize(s);
-    if (e == cudaSuccess && st) e = cudaMemsetAsync(&ctx->ws.sc->status, 0, sizeof(st), s);
-    if (e == cudaSuccess && st) e = cudaStreamSynchronize(s);
     if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; return CS_ECUDA; }
     *device_status = st;
     return st ? CS_EDEVICE_STATUS : CS_OK;
+}
+
+int cs_get_counters(cs_ctx *ctx, cs_counters *out, uint32_t reset, cs_stream_t stream)
+{
+    if (!ctx || !out) return CS_EINVAL;
+    cudaStream_t s = (cudaStream_t)stream;
+    cudaError_t e = cudaMemcpyAsync(out, ctx->ws.cnt, sizeof(*out), cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess && reset) e = cudaMemsetAsync(ctx->ws.cnt, 0, sizeof(*out), s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; return CS_ECUDA; }
+    return CS_OK;
+}
+
+int cs_validate_selection(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, uint32_t prefetch, uint32_t tier,
+                          uint32_t k, const uint32_t *ids_out, const uint32_t *n_out, cs_stream_t stream)
+{
+    if (!ctx) return CS_EINVAL;
+    int rc = check_index(ctx, idx);
+    if (rc != CS_OK) return rc;
+    if (!n_out || (((uintptr_t)n_out) & 3u) || (k && !ids_out) || (((uintptr_t)ids_out) & 3u) || tier > 1) return CS_EINVAL;
+    return cs_launch_validate_selection(ctx, idx, now, prefetch ? 1 : 0, prefetch ? 1u : tier, k, ids_out, n_out,
+                                        (cudaStream_t)stream);
+}
+
+static bool list_ok(const uint32_t *p, uint32_t n) { return n == 0 || (p && !(((uintptr_t)p) & 3u)); }
+
+int cs_validate_move_lists(cs_ctx *ctx, const cs_kv_pool *src, const cs_kv_pool *dst, const uint32_t *src_slots,
+                           const uint32_t *dst_slots, uint32_t n_max, const uint32_t *n_dev, cs_stream_t stream)
+{
+    if (!ctx) return CS_EINVAL;
+    int rc = check_pools(src, dst);
+    if (rc != CS_OK) return rc;
+    if (!list_ok(src_slots, n_max) || !list_ok(dst_slots, n_max) || (((uintptr_t)n_dev) & 3u)) return CS_EINVAL;
+    if (n_max == 0) return CS_OK;
+    cudaStream_t s = (cudaStream_t)stream;
+    // two entries with one destination
+    rc = cs_launch_validate_lists(ctx, dst_slots, src_slots, n_max, n_dev, dst_slots, src_slots, n_max, n_dev, 1, s);
+    // one pool: a slot that is read by one entry and written by another
+    if (rc == CS_OK && src->base == dst->base)
+        rc = cs_launch_validate_lists(ctx, dst_slots, src_slots, n_max, n_dev, src_slots, dst_slots, n_max, n_dev, 0, s);
+    return rc;
+}
+
+int cs_validate_exchange_lists(cs_ctx *ctx, const cs_kv_pool *gpu, const cs_kv_pool *host,
+                               const uint32_t *off_gpu_slots, const uint32_t *off_host_slots, uint32_t n_off_max,
+                               const uint32_t *n_off_dev, const uint32_t *pre_host_slots, const uint32_t *pre_gpu_slots,
+                               uint32_t n_pre_max, const uint32_t *n_pre_dev, cs_stream_t stream)
+{
+    if (!ctx) return CS_EINVAL;
+    int rc = check_pools(gpu, host);
+    if (rc != CS_OK) return rc;
+    if (!list_ok(off_gpu_slots, n_off_max) || !list_ok(off_host_slots, n_off_max) || !list_ok(pre_host_slots, n_pre_max) ||
+        !list_ok(pre_gpu_slots, n_pre_max) || (((uintptr_t)n_off_dev) & 3u) || (((uintptr_t)n_pre_dev) & 3u))
+        return CS_EINVAL;
+    cudaStream_t s = (cudaStream_t)stream;
+    if (n_off_max)        // two offloaded blocks into one host slot
+        rc = cs_launch_validate_lists(ctx, off_host_slots, off_gpu_slots, n_off_max, n_off_dev, off_host_slots, off_gpu_slots,
+                                      n_off_max, n_off_dev, 1, s);
+    if (rc == CS_OK && n_pre_max)     // two prefetched blocks into one GPU slot
+        rc = cs_launch_validate_lists(ctx, pre_gpu_slots, pre_host_slots, n_pre_max, n_pre_dev, pre_gpu_slots, pre_host_slots,
+                                      n_pre_max, n_pre_dev, 1, s);
+    if (rc == CS_OK && n_off_max && n_pre_max) {
+        // a host slot the offload writes while the prefetch reads it; a GPU slot the prefetch writes while the offload reads it
+        rc = cs_launch_validate_lists(ctx, off_host_slots, off_gpu_slots, n_off_max, n_off_dev, pre_host_slots, pre_gpu_slots,
+                                      n_pre_max, n_pre_dev, 0, s);
+        if (rc == CS_OK)
+            rc = cs_launch_validate_lists(ctx, pre_gpu_slots, pre_host_slots, n_pre_max, n_pre_dev, off_gpu_slots,
+                                          off_host_slots, n_off_max, n_off_dev, 0, s);
+    }
+    return rc;
+}
+
+int cs_selftest_bounded_wait(cs_ctx *ctx, uint32_t max_polls, cs_stream_t stream)
+{
+    if (!ctx || max_polls < 1 || max_polls > 1000000u) return CS_EINVAL;
+    return cs_launch_bounded_wait_selftest(ctx, max_polls, (cudaStream_t)stream);
 }
 
 int cs_launch_count(cs_ctx *ctx, uint64_t *n)

@@ -33,6 +33,8 @@ struct cs_scalars {
     uint32_t n_transitions; // sum of all counts
     uint32_t ticket0;       // "last CTA done" counter of the learner refresh
     uint32_t gtab_monotone; // the recency table covers every unsaturated age and never increases with age
+    uint32_t status_read;   // cs_get_status(): the value swapped out of `status`
+    uint32_t val_le, val_elig, val_ticket;   // cs_validate_selection(): keys at or below the last one, eligible entries, ticket
     uint32_t sel_hint[4];   // bin up to which the next select of each kind (GPU victims, host victims, prefetch)
                             // collects ahead of its own threshold, chosen from the previous call's histogram;
                             // ~0 = none; slot 3 is never written: calls that must not speculate read it
@@ -55,13 +57,12 @@ struct cs_sel_state {
                             // next call, so that the counter is zero on entry without a barrier
     uint32_t toggle;        // which of the two the next call uses; flipped by every call on the device, so that a
                             // captured sequence of calls stays consistent when it is replayed
-    uint32_t cluster_c;     // candidates of the last cluster select (inspection only)
-    unsigned long long t_phase[8];   // globaltimer stamps of the last cluster select (phase boundaries, ns)
 };
 
 // Device pointers into the caller's workspace.
 struct cs_workspace {
     cs_scalars *sc;
+    cs_counters *cnt;     // work counters (cs_get_counters)
     cs_sel_state *sel;    // this select's state (one per concurrent select)
     uint32_t *C;          // [A*A] transition counts
     uint32_t *rowsum;     // [A]
@@ -105,10 +106,6 @@ struct cs_ctx {
     uint32_t no_speculation;       // 1: the histogram pass never collects ahead of the threshold
     uint32_t source_mode;          // CS_SOURCES_*: where the cached BFS of Eq. 8 starts
     const float *fsurv_override;   // caller's survival table for score / select, NULL = the BFS table of Eq. 8
-    int cluster_max_v, cluster_max_pf;   // largest usable cluster of the single-launch select (0 = not probed, -1 = none)
-    int cluster_max_step;                // same for the fused three-select launch
-    int bulk_attr_set;     // shared-memory opt-in of the bulk kernel done on this device
-    int collect_attr_set;  // same for the collect kernel with age limits
     const uint32_t *step_now_dev;        // set only while cs_step() issues its calls: device-resident clock / event count
     const uint32_t *step_n_events_dev;
     cudaEvent_t ev_fork, ev_join;        // cs_step(): main -> side and side -> main
@@ -145,6 +142,14 @@ int cs_launch_select_cluster(cs_ctx *ctx, const void *sel_args, const cs_workspa
 int cs_launch_mover(cs_ctx *ctx, const cs_kv_pool *src, const cs_kv_pool *dst, const uint32_t *src_slots,
                     const uint32_t *dst_slots, uint32_t n_max, const uint32_t *n_dev, int kind,
                     cudaStream_t s);
+
+int cs_launch_bounded_wait_selftest(cs_ctx *ctx, uint32_t max_polls, cudaStream_t s);
+int cs_launch_validate_selection(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, int prefetch, uint32_t tier,
+                                 uint32_t k, const uint32_t *ids, const uint32_t *n_out, cudaStream_t s);
+int cs_launch_validate_lists(cs_ctx *ctx, const uint32_t *w_list, const uint32_t *w_partner, uint32_t nw_max,
+                             const uint32_t *nw_dev, const uint32_t *x_list, const uint32_t *x_partner, uint32_t nx_max,
+                             const uint32_t *nx_dev, int self, cudaStream_t s);
+bool cs_device_can_address(const void *ptr);
 
 int cs_launch_exchange(cs_ctx *ctx, const cs_kv_pool *gpu, const cs_kv_pool *host, const uint32_t *off_gpu_slots,
                        const uint32_t *off_host_slots, uint32_t n_off_max, const uint32_t *n_off_dev,

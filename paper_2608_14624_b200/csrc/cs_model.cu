@@ -65,6 +65,7 @@ cs_observe_kernel(cs_workspace ws, uint32_t A, uint32_t n_chains, const uint32_t
     __shared__ uint16_t s_agent[OBS_THREADS];     // CS_AGENT_NONE marks an event that is skipped
     __shared__ int s_last;
     const int tid = threadIdx.x;
+    if (tid == 0) atomicAdd((unsigned long long *)&ws.cnt->events_seen, (unsigned long long)n_events);
     for (uint32_t base = 0; base < n_events; base += OBS_THREADS) {
         const uint32_t e = base + tid;
         uint32_t c = 0, a = CS_AGENT_NONE;
@@ -77,7 +78,10 @@ cs_observe_kernel(cs_workspace ws, uint32_t A, uint32_t n_chains, const uint32_t
             if (!warm && a >= A) bad |= CS_ST_BAD_AGENT;
             if (!warm && c >= n_chains) bad |= CS_ST_BAD_CHAIN;
             if (bad) atomicOr(&ws.sc->status, bad);
-            if (warm || bad) a = CS_AGENT_NONE;
+            if (warm || bad) {
+                a = CS_AGENT_NONE;
+                atomicAdd((unsigned long long *)&ws.cnt->events_skipped, 1ull);
+            }
         }
         s_chain[tid] = c;
         s_agent[tid] = (uint16_t)a;
@@ -101,6 +105,7 @@ cs_observe_kernel(cs_workspace ws, uint32_t A, uint32_t n_chains, const uint32_t
                 atomicAdd(&ws.C[prev * A + a], 1u);
                 atomicAdd(&ws.rowsum[prev], 1u);
                 atomicAdd(&ws.sc->n_transitions, 1u);
+                atomicAdd((unsigned long long *)&ws.cnt->transitions_counted, 1ull);
             }
             if (last_of_chain) ws.cur[c] = (uint16_t)a;
             if (s_last == tid) ws.sc->last_agent = a;

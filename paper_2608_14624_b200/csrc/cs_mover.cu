@@ -17,6 +17,8 @@
 //  * load/store path: 4 x 128-bit loads per thread in flight, streaming cache hints.  Used when
 //    asked for (cs_set_mover_path) and as the comparison point in the profiles.
 // No copy is multicast and no kernel waits on another CTA; every mbarrier wait is bounded.
+#include <mutex>
+
 #include "cs_common.cuh"
 
 #define MV_THREADS 256
@@ -44,6 +46,9 @@ struct MoverArgs {
     const uint32_t *src_slots, *dst_slots, *n_dev;
     uint32_t n_max;
     uint32_t *status;
+    cs_counters *cnt;                 // work counters: blocks and bytes per direction, skipped entries
+    uint32_t kind;                    // CS_MOVE_*
+    unsigned long long block_bytes;
 };
 
 __device__ __forceinline__ unsigned long long chunk_offset(uint32_t layout, uint32_t L, uint32_t n_slots, uint32_t l,
@@ -61,12 +66,20 @@ __device__ __forceinline__ bool resolve_piece(const MoverArgs &a, unsigned long 
     const uint32_t r = (uint32_t)(w - (unsigned long long)i * per_block);
     const uint32_t lp = r / a.pieces, piece = r - lp * a.pieces;
     uint32_t s = __ldg(a.src_slots + i), d = __ldg(a.dst_slots + i);
-    if (s == CS_ID_NONE || d == CS_ID_NONE) return false;
+    const bool first = report && r == 0;                // one piece per block does the block's bookkeeping
+    if (s == CS_ID_NONE || d == CS_ID_NONE) {
+        if (first) atomicAdd((unsigned long long *)&a.cnt->blocks_skipped, 1ull);
+        return false;
+    }
     s -= a.src_first;                                   // ids below first_id wrap and fail the range check
     d -= a.dst_first;
     if (s >= a.src_total || d >= a.dst_total) {
-        if (report && r == 0) atomicOr(a.status, CS_ST_BAD_SLOT);
+        if (first) { atomicOr(a.status, CS_ST_BAD_SLOT); atomicAdd((unsigned long long *)&a.cnt->blocks_skipped, 1ull); }
         return false;
+    }
+    if (first) {
+        atomicAdd((unsigned long long *)&a.cnt->blocks_moved[a.kind], 1ull);
+        atomicAdd((unsigned long long *)&a.cnt->bytes_moved[a.kind], a.block_bytes);
     }
     const unsigned long long in_chunk = (unsigned long long)piece * a.piece_bytes;
     sp = a.src + chunk_offset(a.src_layout, a.L, a.src_total, lp >> 1, lp & 1, s, a.chunk) + in_chunk;
@@ -140,9 +153,9 @@ __device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity)
 }
 // Bounded wait: gives up after TM_SPIN_LIMIT polls (each poll may itself block for a short,
 // hardware-bounded time) and reports failure instead of spinning forever.
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, uint32_t limit = TM_SPIN_LIMIT)
 {
-    for (uint32_t spin = 0; spin < TM_SPIN_LIMIT; ++spin) {
+    for (uint32_t spin = 0; spin < limit; ++spin) {
         if (mbar_test(bar, parity)) return true;
         if (spin > 64) __nanosleep(128);
     }
@@ -313,8 +326,10 @@ __global__ void __launch_bounds__(TM_WARPS * 32, 1) cs_exchange_bulk_kernel(Move
 // ---------------------------------------------------------------------------------------------
 static void fill_mover_args(cs_ctx *ctx, MoverArgs &a, const cs_kv_pool *src, const cs_kv_pool *dst,
                             const uint32_t *src_slots, const uint32_t *dst_slots, uint32_t n_max, const uint32_t *n_dev,
-                            uint32_t piece_bytes)
+                            uint32_t piece_bytes, int kind)
 {
+    a.cnt = ctx->ws.cnt;
+    a.kind = (uint32_t)kind;
     a.src = (const char *)src->base;
     a.dst = (char *)dst->base;
     a.src_total = src->n_slots;
@@ -333,16 +348,23 @@ static void fill_mover_args(cs_ctx *ctx, MoverArgs &a, const cs_kv_pool *src, co
     a.n_pipes = 0;
     a.piece_bytes = piece_bytes;
     a.pieces = (uint32_t)((a.chunk + piece_bytes - 1) / piece_bytes);
+    a.block_bytes = 2ull * a.L * a.chunk;
 }
 
+// Shared-memory opt-in of the bulk kernels: an attribute of the function on a device, so it is set once per
+// process and device (always to the same fixed size).
+static std::mutex g_bulk_mu;
+static bool g_bulk_opted[64];
 static int bulk_opt_in(cs_ctx *ctx)
 {
-    if (ctx->bulk_attr_set) return CS_OK;
+    if (ctx->device < 0 || ctx->device >= 64) return CS_EINVAL;
+    std::lock_guard<std::mutex> lock(g_bulk_mu);
+    if (g_bulk_opted[ctx->device]) return CS_OK;
     cudaError_t e = cudaFuncSetAttribute(cs_mover_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TM_SMEM);
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(cs_exchange_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TM_SMEM);
     if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; return CS_ECUDA; }
-    ctx->bulk_attr_set = 1;
+    g_bulk_opted[ctx->device] = true;
     return CS_OK;
 }
 
@@ -351,7 +373,7 @@ int cs_launch_mover(cs_ctx *ctx, const cs_kv_pool *src, const cs_kv_pool *dst, c
 {
     const bool bulk = ctx->mover_path != CS_MOVER_LDST;
     MoverArgs a;
-    fill_mover_args(ctx, a, src, dst, src_slots, dst_slots, n_max, n_dev, bulk ? TM_PIECE : MV_PIECE);
+    fill_mover_args(ctx, a, src, dst, src_slots, dst_slots, n_max, n_dev, bulk ? TM_PIECE : MV_PIECE, kind);
     const unsigned long long total = (unsigned long long)n_max * 2ull * a.L * a.pieces;
     unsigned long long cap;
     if (bulk) {
@@ -383,8 +405,8 @@ int cs_launch_exchange(cs_ctx *ctx, const cs_kv_pool *gpu, const cs_kv_pool *hos
                        const uint32_t *n_pre_dev, cudaStream_t s)
 {
     MoverArgs off, pre;
-    fill_mover_args(ctx, off, gpu, host, off_gpu_slots, off_host_slots, n_off_max, n_off_dev, TM_PIECE);
-    fill_mover_args(ctx, pre, host, gpu, pre_host_slots, pre_gpu_slots, n_pre_max, n_pre_dev, TM_PIECE);
+    fill_mover_args(ctx, off, gpu, host, off_gpu_slots, off_host_slots, n_off_max, n_off_dev, TM_PIECE, CS_MOVE_OFFLOAD);
+    fill_mover_args(ctx, pre, host, gpu, pre_host_slots, pre_gpu_slots, n_pre_max, n_pre_dev, TM_PIECE, CS_MOVE_PREFETCH);
     const unsigned long long total = ((unsigned long long)n_off_max + n_pre_max) * 2ull * off.L * off.pieces;
     const unsigned long long cap = ctx->host_link_ctas ? ctx->host_link_ctas : CS_EXCHANGE_PIPES;
     uint32_t n_pipes = (uint32_t)(total < cap ? total : cap);
@@ -395,5 +417,25 @@ int cs_launch_exchange(cs_ctx *ctx, const cs_kv_pool *gpu, const cs_kv_pool *hos
     const int rc = bulk_opt_in(ctx);
     if (rc != CS_OK) return rc;
     cs_exchange_bulk_kernel<<<grid, wpc * 32, TM_SMEM, s>>>(off, pre);
+    return cs_check_launch(ctx);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Self-test of the bounded wait: one warp, one barrier, no copy.  The wait cannot succeed, so it runs out
+// after `max_polls` polls and the kernel reports exactly as a stalled transfer would.  Nothing is in flight.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(32) cs_bounded_wait_selftest_kernel(uint32_t max_polls, uint32_t *status)
+{
+    __shared__ __align__(8) unsigned long long bar_mem;
+    if (threadIdx.x != 0) return;
+    const uint32_t bar = smem_u32(&bar_mem);
+    mbar_init(bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    if (!mbar_wait_bounded(bar, 0, max_polls)) atomicOr(status, CS_ST_TIMEOUT);
+}
+
+int cs_launch_bounded_wait_selftest(cs_ctx *ctx, uint32_t max_polls, cudaStream_t s)
+{
+    cs_bounded_wait_selftest_kernel<<<1, 32, 0, s>>>(max_polls, &ctx->ws.sc->status);
     return cs_check_launch(ctx);
 }

@@ -245,6 +245,7 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_hist_kernel(SelArgs a, cs_
         ws.sel->b0 = b0;
         ws.sel->n_elig = total;
         ws.sel->n_out = total < a.k ? total : a.k;
+        count_select(ws, a.kind, total, total < a.k ? total : a.k);
         ws.sel->c = spec_ok ? c_spec : 0;
         ws.sel->c_spec = 0;
         ws.sel->spec = spec_ok ? 1u : 0u;
@@ -573,7 +574,7 @@ cs_sel_rank_kernel(cs_workspace ws, uint32_t k, uint32_t *__restrict__ ids_out, 
 }
 
 // ---------------------------------------------------------------------------------------------
-static void fill_args(const cs_ctx *ctx, const cs_block_index *idx, uint32_t now, const float *fsurv, SelArgs &a)
+void cs_fill_sel_args(const cs_ctx *ctx, const cs_block_index *idx, uint32_t now, const float *fsurv, SelArgs &a)
 {
     a.agent = idx->agent;
     a.depth = idx->depth;
@@ -596,10 +597,11 @@ static void fill_args(const cs_ctx *ctx, const cs_block_index *idx, uint32_t now
     a.prefer_copy = ctx->p.prefer_other_copy ? 1u : 0u;
     a.use_age_limits = 0;
     a.hint_slot = 0;
+    a.kind = 0;
     a.now_dev = ctx->step_now_dev;
 }
 
-static uint32_t scan_grid(const cs_ctx *ctx, uint32_t n, uint32_t per_cta, uint32_t ctas_per_sm = 2)
+uint32_t cs_scan_grid(const cs_ctx *ctx, uint32_t n, uint32_t per_cta, uint32_t ctas_per_sm)
 {
     uint32_t g = (n + per_cta - 1) / per_cta;
     const uint32_t cap = ctas_per_sm * (uint32_t)ctx->sm_count;
@@ -607,7 +609,7 @@ static uint32_t scan_grid(const cs_ctx *ctx, uint32_t n, uint32_t per_cta, uint3
     return g ? g : 1u;
 }
 
-static size_t table_smem(const cs_ctx *ctx)
+size_t cs_table_smem(const cs_ctx *ctx)
 {
     return (size_t)(ctx->p.n_agents + ctx->gtab_len) * sizeof(float) + (size_t)ctx->p.n_agents * sizeof(uint16_t) + 16;
 }
@@ -616,11 +618,30 @@ int cs_launch_score(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, const 
                     cudaStream_t s)
 {
     SelArgs a;
-    fill_args(ctx, idx, now, fsurv, a);
+    cs_fill_sel_args(ctx, idx, now, fsurv, a);
     a.anchor = nullptr;
-    const uint32_t grid = scan_grid(ctx, idx->n_blocks, SEL_THREADS * GRP);
-    cs_score_kernel<<<grid, SEL_THREADS, table_smem(ctx), s>>>(a, ctx->ws, scores_out);
+    const uint32_t grid = cs_scan_grid(ctx, idx->n_blocks, SEL_THREADS * GRP);
+    cs_score_kernel<<<grid, SEL_THREADS, cs_table_smem(ctx), s>>>(a, ctx->ws, scores_out);
     return cs_check_launch(ctx);
+}
+
+// Shared-memory opt-in of the scan kernels that keep age limits in shared memory: an attribute of the
+// function on a device, set once per process and device to one fixed size.
+#include <mutex>
+#define SCAN_SMEM_OPT_IN (96 * 1024)
+static std::mutex g_scan_mu;
+static bool g_scan_opted[64];
+static int scan_opt_in(cs_ctx *ctx)
+{
+    if (ctx->device < 0 || ctx->device >= 64) return CS_EINVAL;
+    std::lock_guard<std::mutex> lock(g_scan_mu);
+    if (g_scan_opted[ctx->device]) return CS_OK;
+    cudaError_t e = cudaFuncSetAttribute(cs_sel_collect_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SCAN_SMEM_OPT_IN);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(cs_sel_collect_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SCAN_SMEM_OPT_IN);
+    if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; return CS_ECUDA; }
+    g_scan_opted[ctx->device] = true;
+    return CS_OK;
 }
 
 // One select through the grid-wide kernels (or one single-launch cluster select), on the scratch of `job`.
@@ -629,17 +650,18 @@ static int launch_select_job(cs_ctx *ctx, int job, const cs_block_index *idx, ui
 {
     const cs_workspace &ws = job == 0 ? ctx->ws : ctx->ws_job[job - 1];
     SelArgs a;
-    fill_args(ctx, idx, now, ctx->fsurv_override ? ctx->fsurv_override : ctx->ws.fsurv, a);
+    cs_fill_sel_args(ctx, idx, now, ctx->fsurv_override ? ctx->fsurv_override : ctx->ws.fsurv, a);
     a.tier = tier;
     a.k = k;
     a.hint_slot = ctx->no_speculation ? 3u : (prefetch ? 2u : tier);
+    a.kind = prefetch ? 2u : tier;
     if (ctx->select_path != CS_SELECT_MULTI && idx->n_blocks <= CS_SELECT_CLUSTER_MAX_BLOCKS) {
         const int rc1 = cs_launch_select_cluster(ctx, &a, &ws, prefetch, ids_out, n_out, s);
         if (rc1 != CS_ENOTIMPL) return rc1;          // no usable cluster on this device: fall through
     }
-    const uint32_t grid = scan_grid(ctx, idx->n_blocks, SEL_THREADS * GRP);
-    const uint32_t grid_c = scan_grid(ctx, idx->n_blocks, 256);
-    const size_t sm = table_smem(ctx);
+    const uint32_t grid = cs_scan_grid(ctx, idx->n_blocks, SEL_THREADS * GRP);
+    const uint32_t grid_c = cs_scan_grid(ctx, idx->n_blocks, 256);
+    const size_t sm = cs_table_smem(ctx);
     int rc;
     if (prefetch) cs_launch_chained(cs_sel_hist_kernel<true>, grid, SEL_THREADS, sm, s, a, ws);
     else cs_launch_chained(cs_sel_hist_kernel<false>, grid, SEL_THREADS, sm, s, a, ws);
@@ -650,13 +672,8 @@ static int launch_select_job(cs_ctx *ctx, int job, const cs_block_index *idx, ui
     if (idx->n_blocks >= CS_AGE_LIMIT_MIN_BLOCKS && (size_t)ctx->p.n_agents * n_cls <= AGE_LIM_MAX) {
         a.use_age_limits = 1;
         sm_collect += (size_t)ctx->p.n_agents * n_cls * sizeof(uint32_t);
-        if (!ctx->collect_attr_set) {
-            cudaError_t e = cudaFuncSetAttribute(cs_sel_collect_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
-            if (e == cudaSuccess)
-                e = cudaFuncSetAttribute(cs_sel_collect_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
-            if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; return CS_ECUDA; }
-            ctx->collect_attr_set = 1;
-        }
+        const int rc_opt = scan_opt_in(ctx);
+        if (rc_opt != CS_OK) return rc_opt;
     }
     if (prefetch) cs_launch_chained(cs_sel_collect_kernel<true>, grid, SEL_THREADS, sm_collect, s, a, ws);
     else cs_launch_chained(cs_sel_collect_kernel<false>, grid, SEL_THREADS, sm_collect, s, a, ws);
@@ -698,10 +715,11 @@ int cs_launch_select_step(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, 
         uint32_t pf[3];
         for (int i = 0; i < n_jobs; ++i) {
             const int q = jobs[i];
-            fill_args(ctx, idx, now, ctx->fsurv_override ? ctx->fsurv_override : ctx->ws.fsurv, a[i]);
+            cs_fill_sel_args(ctx, idx, now, ctx->fsurv_override ? ctx->fsurv_override : ctx->ws.fsurv, a[i]);
             a[i].tier = q == 0 ? 0u : 1u;
             a[i].k = ks[q];
             a[i].hint_slot = ctx->no_speculation ? 3u : (uint32_t)q;
+            a[i].kind = (uint32_t)q;
             j_ids[i] = ids[q];
             j_cnt[i] = cnt[q];
             pf[i] = q == 2 ? 1u : 0u;
@@ -742,8 +760,6 @@ int cs_launch_select_step(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, 
 // The array's name is only a host-side handle: the device address is obtained once per device
 // with cudaGetSymbolAddress() and that pointer is what the kernels get.
 // =============================================================================================
-#include <mutex>
-
 #define CS_STATIC_MAX_DEVICES 64
 #define CS_STATIC_ALIGN(x) (((x) + 255u) / 256u * 256u)
 // layout of the static scratch, byte offsets (every region 256-byte aligned)
@@ -761,14 +777,14 @@ int cs_launch_select_step(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, 
 #define CS_SO_CANDBKT (CS_SO_CANDID + CS_STATIC_MAX_BLOCKS * 4u)
 #define CS_SO_CANDSLOT (CS_SO_CANDBKT + CS_STATIC_MAX_BLOCKS * 4u)
 #define CS_SO_SORTID (CS_SO_CANDSLOT + CS_STATIC_MAX_BLOCKS * 4u)
-#define CS_STATIC_BYTES (CS_SO_SORTID + CS_STATIC_MAX_BLOCKS * 4u)
+#define CS_SO_CNT (CS_SO_SORTID + CS_STATIC_MAX_BLOCKS * 4u)
+#define CS_STATIC_BYTES (CS_SO_CNT + CS_STATIC_ALIGN(sizeof(cs_counters)))
 
 static __device__ __align__(256) unsigned char cs_static_scratch[CS_STATIC_BYTES];   // 2 MiB + 40 KiB
 
 static std::mutex g_static_mu;
 static unsigned char *g_static_ptr[CS_STATIC_MAX_DEVICES];     // device address of the array, per device
 static int g_static_sms[CS_STATIC_MAX_DEVICES];
-static int g_static_cluster[CS_STATIC_MAX_DEVICES];   // largest usable select cluster on the device (0 = not probed yet)
 
 // Everything the select kernels expect to find zeroed, and the recency table for this call's
 // lambda / delta.  The array keeps the previous call's contents, so this runs on every call.
@@ -806,8 +822,22 @@ extern "C" int cs_select_victims_static(const cs_params *p, const float *fsurv, 
                               (uintptr_t)idx->flags | (uintptr_t)idx->last_access | (uintptr_t)idx->n_tokens;
         if (any & 15u) return CS_EINVAL;
     }
+    // Memory the SMs cannot address (a pageable host array) would fault the GPU: every pointer the kernels
+    // dereference is looked up first (a host-side query that allocates nothing); nothing is launched on failure.
+    {
+        const void *ptrs[10] = {fsurv, n_out, k ? ids_out : nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
+        if (idx->n_blocks) {
+            ptrs[3] = idx->agent; ptrs[4] = idx->depth; ptrs[5] = idx->ref_count; ptrs[6] = idx->flags;
+            ptrs[7] = idx->last_access; ptrs[8] = idx->n_tokens;
+        }
+        for (int i = 0; i < 10; ++i)
+            if (ptrs[i] && !cs_device_can_address(ptrs[i])) return CS_EINVAL;
+    }
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= CS_STATIC_MAX_DEVICES) return CS_ECUDA;
+    int stream_dev = dev;        // the array of the CURRENT device is used: a stream of another device is refused
+    if (stream && cudaStreamGetDevice((cudaStream_t)stream, &stream_dev) == cudaSuccess && stream_dev != dev) return CS_EINVAL;
+    (void)cudaGetLastError();
     {
         // first call on this device: resolve the device address of the array (once, with the device current)
         std::lock_guard<std::mutex> lock(g_static_mu);
@@ -820,15 +850,20 @@ extern "C" int cs_select_victims_static(const cs_params *p, const float *fsurv, 
             g_static_ptr[dev] = (unsigned char *)ptr;
         }
     }
-    unsigned char *base = g_static_ptr[dev];
+    unsigned char *base;
+    int sms;
+    {
+        std::lock_guard<std::mutex> lock(g_static_mu);
+        base = g_static_ptr[dev];
+        sms = g_static_sms[dev];
+    }
     cs_ctx ctx;                                        // host-side descriptor only; nothing is allocated
     memset(&ctx, 0, sizeof(ctx));
     ctx.p = *p;
     ctx.p.max_blocks = CS_STATIC_MAX_BLOCKS;
     cs_recency_table_shape(p, &ctx.gtab_len, &ctx.age_sat);
     ctx.device = dev;
-    ctx.sm_count = g_static_sms[dev];
-    ctx.cluster_max_v = g_static_cluster[dev];         // probed once per device, not once per call
+    ctx.sm_count = sms;
     cs_workspace &ws = ctx.ws;
     ws.sc = (cs_scalars *)(base + CS_SO_SC);
     ws.sel = (cs_sel_state *)(base + CS_SO_SEL);
@@ -844,11 +879,10 @@ extern "C" int cs_select_victims_static(const cs_params *p, const float *fsurv, 
     ws.cand_bkt = (uint32_t *)(base + CS_SO_CANDBKT);
     ws.cand_slot = (uint32_t *)(base + CS_SO_CANDSLOT);
     ws.sort_id = (uint32_t *)(base + CS_SO_SORTID);
+    ws.cnt = (cs_counters *)(base + CS_SO_CNT);
     ws.fsurv = const_cast<float *>(fsurv);             // input table, read only
     cudaStream_t s = (cudaStream_t)stream;
     cs_static_prepare_kernel<<<16, 256, 0, s>>>(ws, ctx.gtab_len, p->lambda, p->delta);
     if ((rc = cs_check_launch(&ctx)) != CS_OK) return rc;
-    rc = cs_launch_select(&ctx, idx, now, 0, tier, k, ids_out, n_out, s);
-    g_static_cluster[dev] = ctx.cluster_max_v;
-    return rc;
+    return cs_launch_select(&ctx, idx, now, 0, tier, k, ids_out, n_out, s);
 }

@@ -107,15 +107,6 @@ __device__ __forceinline__ void csel_bitonic(unsigned long long *km, uint32_t *i
     }
 }
 
-__device__ __forceinline__ void csel_stamp(const cs_workspace &ws, uint32_t rank, int slot)
-{
-    if (rank == 0 && threadIdx.x == 0) {
-        unsigned long long t;
-        asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-        ws.sel->t_phase[slot] = t;
-    }
-}
-
 // One whole select by the calling cluster.  `ws` carries this select's private candidate / sort regions
 // and its row of per-call scalars, so several clusters of one launch can run different selects at once.
 template <bool PF>
@@ -137,7 +128,6 @@ __device__ __forceinline__ void csel_body(SelArgs a, const cs_workspace &ws, uin
     if (tid == 0) S.misc[1] = 0;
     __syncthreads();
     const bool enabled = !PF || prefetch_enabled(ws, a.A);
-    csel_stamp(ws, rank, 0);
     const uint32_t n_tiles = a.n / TILE;
     const uint32_t cthreads = CL * CSEL_THREADS, ctid = rank * CSEL_THREADS + tid;   // cluster-wide thread id
     const uint32_t t0 = n_tiles * TILE;                                              // start of the ragged tail
@@ -206,7 +196,6 @@ __device__ __forceinline__ void csel_body(SelArgs a, const cs_workspace &ws, uin
     }
     __threadfence();
     cluster.sync();
-    csel_stamp(ws, rank, 1);
 
     // ---- phase 2: reduce the histograms through DSMEM, broadcast, find the threshold bin ---------------
     {
@@ -241,9 +230,8 @@ __device__ __forceinline__ void csel_body(SelArgs a, const cs_workspace &ws, uin
     const uint32_t n_out = n_elig < a.k ? n_elig : a.k;
     // the tail of the list is known now: pad it while the candidates are being collected
     for (uint32_t i = n_out + ctid; i < a.k; i += cthreads) ids_out[i] = CS_ID_NONE;
-    if (ctid == 0) *n_out_dev = n_out;
+    if (ctid == 0) { *n_out_dev = n_out; count_select(ws, a.kind, n_elig, n_out); }
 
-    csel_stamp(ws, rank, 2);
     // ---- phase 3: collect the candidates (bin <= b0), unless the first scan already has them ----------------
     const bool spec_ok = hint != 0xFFFFFFFFu && b0 != 0xFFFFFFFFu && b0 <= hint;     // same verdict in every CTA
     const bool have_b0 = a.k && n_elig >= a.k;
@@ -262,8 +250,6 @@ __device__ __forceinline__ void csel_body(SelArgs a, const cs_workspace &ws, uin
         cluster.sync();
     }
     const uint32_t c = __ldcg(cand_count);
-    if (rank == 0 && tid == 0) ws.sel->cluster_c = c;                 // for inspection only
-    csel_stamp(ws, rank, 3);
 
     // ---- phase 4, small: ordered in shared memory ---------------------------------------------------------------
     if (c <= CSEL_SORT_MAX) {
@@ -300,7 +286,6 @@ __device__ __forceinline__ void csel_body(SelArgs a, const cs_workspace &ws, uin
             __syncthreads();
             csel_bitonic(S.km, S.id, P);
             for (uint32_t i = tid; i < n_out; i += CSEL_THREADS) ids_out[i] = S.id[i];
-            csel_stamp(ws, rank, 4);
             return;
         }
         if (rank != 0) return;
@@ -313,7 +298,6 @@ __device__ __forceinline__ void csel_body(SelArgs a, const cs_workspace &ws, uin
         __syncthreads();
         csel_bitonic(S.km, S.id, P);
         for (uint32_t i = tid; i < n_out; i += CSEL_THREADS) ids_out[i] = S.id[i];
-        csel_stamp(ws, rank, 4);
         return;
     }
 
@@ -337,7 +321,6 @@ __device__ __forceinline__ void csel_body(SelArgs a, const cs_workspace &ws, uin
     }
     __threadfence();
     cluster.sync();
-    csel_stamp(ws, rank, 4);
     // bucket: number of splitters <= key; slot by a global counter per bucket
     unsigned long long *spl_km = S.km;               // shared-memory copy of the splitters
     uint32_t *spl_id = S.id;
@@ -358,7 +341,6 @@ __device__ __forceinline__ void csel_body(SelArgs a, const cs_workspace &ws, uin
     }
     __threadfence();
     cluster.sync();
-    csel_stamp(ws, rank, 5);
     // offsets (every CTA computes the same prefix sum), then scatter the needed buckets into bucket order
     uint32_t *s_off = S.hist;                        // reuse: [CS_MAX_SPLITTERS + 2]
     {
@@ -380,7 +362,6 @@ __device__ __forceinline__ void csel_body(SelArgs a, const cs_workspace &ws, uin
     }
     __threadfence();
     cluster.sync();
-    csel_stamp(ws, rank, 6);
     // rank: buckets round-robin over the CTAs; a bucket is ranked from a shared-memory tile
     for (uint32_t b = rank; b <= b_last; b += CL) {
         const uint32_t beg = s_off[b], end = s_off[b + 1], m = end - beg;
@@ -406,7 +387,6 @@ __device__ __forceinline__ void csel_body(SelArgs a, const cs_workspace &ws, uin
             }
         }
     }
-    csel_stamp(ws, rank, 7);
 }
 
 template <bool PF>
@@ -437,13 +417,29 @@ __global__ void __launch_bounds__(CSEL_THREADS, 1) cs_select_step_kernel(const _
 }
 
 // ---------------------------------------------------------------------------------------------
-template <bool PF>
-static int launch_cluster(cs_ctx *ctx, const SelArgs &a, const cs_workspace &ws, uint32_t *ids_out, uint32_t *n_out,
-                          cudaStream_t s)
+// Per-device set-up of the three cluster kernels, done once per process and device.  The dynamic shared-memory
+// opt-in is an attribute of the FUNCTION (on a device), not of a context, so it is raised once to the fixed
+// maximum any parameter set can ask for (CS_MAX_AGENTS agents, the longest recency table) and never lowered:
+// contexts of different shape and the static-scratch entry point can then share the kernels.  The largest
+// usable cluster is probed with that same maximum, which makes the answer independent of the caller's sizes.
+#include <mutex>
+
+#define CSEL_MAX_DEVICES 64
+struct CselDevice {
+    int ready;                       // 0 = not set up yet
+    int max_v, max_pf, max_step;     // largest usable cluster per kernel (-1 = none)
+};
+static std::mutex g_csel_mu;
+static CselDevice g_csel_dev[CSEL_MAX_DEVICES];
+
+template <class Kernel>
+static int csel_probe(Kernel kernel, size_t smem, int clusters_needed)
 {
-    auto kernel = cs_select_cluster_kernel<PF>;
-    const size_t smem = csel_smem_bytes(a.A, a.gtab_len);
-    int &max_cl = PF ? ctx->cluster_max_pf : ctx->cluster_max_v;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
+        cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return -1;
+    }
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -451,31 +447,65 @@ static int launch_cluster(cs_ctx *ctx, const SelArgs &a, const cs_workspace &ws,
     attr[0].val.clusterDim.z = 1;
     cfg.blockDim = dim3(CSEL_THREADS);
     cfg.dynamicSmemBytes = smem;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    for (int cl = CSEL_MAX_CLUSTER; cl >= 1; cl >>= 1) {
+        cfg.gridDim = dim3(clusters_needed * cl);
+        attr[0].val.clusterDim.x = cl;
+        int n_clusters = 0;
+        const cudaError_t e = cudaOccupancyMaxActiveClusters(&n_clusters, kernel, &cfg);
+        if (e == cudaSuccess && n_clusters >= clusters_needed) return cl;
+        (void)cudaGetLastError();
+    }
+    return -1;
+}
+
+// Returns the device's entry (set up on first use, with `device` current), or nullptr for a device index out of range.
+static const CselDevice *csel_device(int device)
+{
+    if (device < 0 || device >= CSEL_MAX_DEVICES) return nullptr;
+    std::lock_guard<std::mutex> lock(g_csel_mu);
+    CselDevice &d = g_csel_dev[device];
+    if (!d.ready) {
+        const size_t smem_max = csel_smem_bytes(CS_MAX_AGENTS, CS_GTAB_MAX);
+        d.max_v = csel_probe(cs_select_cluster_kernel<false>, smem_max, 1);
+        d.max_pf = csel_probe(cs_select_cluster_kernel<true>, smem_max, 1);
+        d.max_step = csel_probe(cs_select_step_kernel, smem_max, 3);
+        d.ready = 1;
+    }
+    return &d;
+}
+
+// smallest power-of-two cluster that gives every 16-entry group its own thread, at most max_cl
+static int csel_cluster_size(uint32_t n, int max_cl)
+{
+    const uint32_t n_groups = n / GRP;                   // 16 entries per thread and pass
+    int cl = 1;
+    while (cl < max_cl && (uint32_t)cl * CSEL_THREADS < n_groups) cl <<= 1;
+    return cl;
+}
+
+template <bool PF>
+static int launch_cluster(cs_ctx *ctx, const SelArgs &a, const cs_workspace &ws, uint32_t *ids_out, uint32_t *n_out,
+                          cudaStream_t s)
+{
+    const CselDevice *d = csel_device(ctx->device);
+    const int max_cl = d ? (PF ? d->max_pf : d->max_v) : -1;
+    if (max_cl < 1) return CS_ENOTIMPL;
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    const int cl = csel_cluster_size(a.n, max_cl);
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = cl;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.gridDim = dim3(cl);
+    cfg.blockDim = dim3(CSEL_THREADS);
+    cfg.dynamicSmemBytes = csel_smem_bytes(a.A, a.gtab_len);      // <= the opted-in maximum by construction
     cfg.stream = s;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (max_cl == 0) {           // first use on this context: shared-memory opt-in, largest cluster that fits
-        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
-        if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; (void)cudaGetLastError(); max_cl = -1; return CS_ENOTIMPL; }
-        max_cl = -1;
-        for (int cl = CSEL_MAX_CLUSTER; cl >= 1; cl >>= 1) {
-            cfg.gridDim = dim3(cl);
-            attr[0].val.clusterDim.x = cl;
-            int n_clusters = 0;
-            e = cudaOccupancyMaxActiveClusters(&n_clusters, kernel, &cfg);
-            if (e == cudaSuccess && n_clusters >= 1) { max_cl = cl; break; }
-            (void)cudaGetLastError();
-        }
-    }
-    if (max_cl < 1) return CS_ENOTIMPL;
-    // smallest power-of-two cluster that gives every 16-entry group its own thread, at most max_cl
-    const uint32_t n_groups = a.n / GRP;                 // 16 entries per thread and pass
-    int cl = 1;
-    while (cl < max_cl && (uint32_t)cl * CSEL_THREADS < n_groups) cl <<= 1;
-    cfg.gridDim = dim3(cl);
-    attr[0].val.clusterDim.x = cl;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, a, ws, ids_out, n_out);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, cs_select_cluster_kernel<PF>, a, ws, ids_out, n_out);
     ctx->n_launches++;
     if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; return CS_ECUDA; }
     return CS_OK;
@@ -485,38 +515,22 @@ int cs_launch_select_clusters(cs_ctx *ctx, int n_jobs, const void *sel_args, con
                               uint32_t *const *ids_out, uint32_t *const *n_out, cudaStream_t s)
 {
     const SelArgs *aj = (const SelArgs *)sel_args;
-    const size_t smem = csel_smem_bytes(aj[0].A, aj[0].gtab_len);
-    int &max_cl = ctx->cluster_max_step;
+    const CselDevice *d = csel_device(ctx->device);
+    const int max_cl = d ? d->max_step : -1;
+    if (max_cl < 1) return CS_ENOTIMPL;
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[1];
+    const int cl = csel_cluster_size(aj[0].n, max_cl);
     attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = cl;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    cfg.gridDim = dim3(n_jobs * cl);
     cfg.blockDim = dim3(CSEL_THREADS);
-    cfg.dynamicSmemBytes = smem;
+    cfg.dynamicSmemBytes = csel_smem_bytes(aj[0].A, aj[0].gtab_len);
     cfg.stream = s;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (max_cl == 0) {           // first use on this context: shared-memory opt-in, largest cluster of which three fit
-        cudaError_t e = cudaFuncSetAttribute(cs_select_step_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(cs_select_step_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
-        if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; (void)cudaGetLastError(); max_cl = -1; return CS_ENOTIMPL; }
-        max_cl = -1;
-        for (int cl = CSEL_MAX_CLUSTER; cl >= 1; cl >>= 1) {
-            cfg.gridDim = dim3(3 * cl);
-            attr[0].val.clusterDim.x = cl;
-            int n_clusters = 0;
-            e = cudaOccupancyMaxActiveClusters(&n_clusters, cs_select_step_kernel, &cfg);
-            if (e == cudaSuccess && n_clusters >= 3) { max_cl = cl; break; }
-            (void)cudaGetLastError();
-        }
-    }
-    if (max_cl < 1) return CS_ENOTIMPL;
-    const uint32_t n_groups = aj[0].n / GRP;
-    int cl = 1;
-    while (cl < max_cl && (uint32_t)cl * CSEL_THREADS < n_groups) cl <<= 1;
-    cfg.gridDim = dim3(n_jobs * cl);
-    attr[0].val.clusterDim.x = cl;
     SelJobs jobs;
     for (int q = 0; q < n_jobs; ++q) {
         jobs.j[q].a = aj[q];

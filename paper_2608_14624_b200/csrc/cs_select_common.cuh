@@ -20,8 +20,14 @@ struct SelArgs {
     uint32_t tier, k, prefer_copy;
     uint32_t use_age_limits;      // collect pass may prefilter by per-(agent, size) age limits (large indexes)
     uint32_t hint_slot;           // which remembered threshold bin this call may speculate on
+    uint32_t kind;                // 0 GPU-tier victims, 1 host-tier victims, 2 prefetch candidates (work counters)
     const uint32_t *now_dev;      // when set, the clock is read from device memory at execution time (graph replay)
 };
+
+// host helpers defined in cs_select.cu
+void cs_fill_sel_args(const cs_ctx *ctx, const cs_block_index *idx, uint32_t now, const float *fsurv, SelArgs &a);
+uint32_t cs_scan_grid(const cs_ctx *ctx, uint32_t n, uint32_t per_cta, uint32_t ctas_per_sm = 2);
+size_t cs_table_smem(const cs_ctx *ctx);
 
 // What the next call of this kind may collect ahead of its own threshold.  The threshold bin of consecutive
 // calls moves little, so the next call's first scan appends every entry up to a remembered bin.  That bin is
@@ -57,6 +63,15 @@ __device__ __forceinline__ uint32_t collect_ahead_limit(const uint32_t (&loc)[PE
 __device__ __forceinline__ void remember_threshold(cs_scalars *sc, uint32_t slot, bool valid, uint32_t limit)
 {
     if (slot < 3) sc->sel_hint[slot] = valid ? limit : 0xFFFFFFFFu;
+}
+
+// Work counters of one finished select (called by one thread).
+__device__ __forceinline__ void count_select(const cs_workspace &ws, uint32_t kind, uint32_t n_elig, uint32_t n_out)
+{
+    if (kind > 2) return;
+    atomicAdd((unsigned long long *)&ws.cnt->selects[kind], 1ull);
+    atomicAdd((unsigned long long *)&ws.cnt->selected[kind], (unsigned long long)n_out);
+    ws.cnt->eligible[kind] = n_elig;
 }
 
 // The clock of a call: by value, or from device memory when the caller asked for that.

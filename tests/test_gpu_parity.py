@@ -144,12 +144,14 @@ def run_selects(c, o, idx, now, ks, tiers=(0, 1)):
             assert np.array_equal(g_ids, ids2.cpu().numpy().view(np.uint32)[:k]) and g_n == int(n_out2.item())
             o_ids, o_n = o.select_victims(idx, now, tier, k, s32)
             tolerated += H.assert_list_matches(g_ids, g_n, o_ids, o_n, s64)
+            c.validate_selection(d, now, False, tier, k, ids, n_out)        # the device-side checker agrees (status stays 0)
             sel = g_ids[:g_n].astype(np.int64)
             assert not np.any(idx.flags[sel] & synth.FLAG_PINNED) and np.all(idx.ref_count[sel] == 0)
         ids, n_out = c.select_prefetch(d, now, k)
         g_ids, g_n = ids.cpu().numpy().view(np.uint32)[:k], int(n_out.item())
         o_ids, o_n = o.select_prefetch(idx, now, k, s32)
         tolerated += H.assert_list_matches(g_ids, g_n, o_ids, o_n, s64)
+        c.validate_selection(d, now, True, 1, k, ids, n_out)
     assert c.get_status() == 0
     return tolerated
 
@@ -722,6 +724,7 @@ def test_random_mover_geometries(case):
     if n_pre > 2:
         pre_src[0] = orc.ID_NONE
     opt = lambda a: dev(a) if len(a) else None
+    c.validate_exchange_lists(gpu, host, opt(off_src), opt(off_dst), opt(pre_src), opt(pre_dst))     # no slot used twice
     c.exchange_blocks(gpu, host, opt(off_src), opt(off_dst), opt(pre_src), opt(pre_dst))
     torch.cuda.synchronize()
     want_h, want_g = host_np.copy(), gpu_np.copy()
@@ -732,11 +735,13 @@ def test_random_mover_geometries(case):
     # the single calls, starting from the state just reached
     n = int(rng.integers(1, 15))
     s_g, d_h = rng.permutation(G).astype(np.uint32)[:n], rng.permutation(Hs).astype(np.uint32)[:n] + np.uint32(first_h)
+    c.validate_move_lists(gpu, host, dev(s_g), dev(d_h))
     c.offload_blocks(gpu, host, dev(s_g), dev(d_h))
     torch.cuda.synchronize()
     orc.move_blocks(want_g, lay_g, G, want_h, lay_h, Hs, L, chunk, s_g, unoff(d_h))
     assert np.array_equal(host_t.numpy(), want_h)
     back = rng.permutation(G).astype(np.uint32)[:n]
+    c.validate_move_lists(host, gpu, dev(d_h), dev(back))
     c.prefetch_blocks(host, gpu, dev(d_h), dev(back))
     torch.cuda.synchronize()
     src_h = want_h.copy()
