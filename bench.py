@@ -11,7 +11,11 @@ stream (or, with --transfers split, as two launches on two side streams) and ove
 step's selection.  value = KV bytes moved across the host link per second over the K steps.
 
     python bench.py --gpus 1 --steps 20 --warmup 3
+    python bench.py --config llama70b         # the 70B-shaped configuration as the timed workload
     python bench.py --impl reference          # the CPU oracle on the host cores, same metric
+
+The default run times the Llama-3-8B-shaped step (the headline line) and then, as extra keys of the same
+JSON line, the 70B-shaped step, the mover sweep, the metadata-scale calls and the large-index regime.
 """
 from __future__ import annotations
 
@@ -39,7 +43,11 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--host-slots", type=int, default=0, help="host-tier slots backed by pinned memory (0 = auto)")
+    ap.add_argument("--config", default="llama8b", choices=["llama8b", "llama70b"], help="KV shape of the timed step")
+    ap.add_argument("--host-slots", type=int, default=0,
+                    help="host-tier slots backed by pinned memory (0 = as many of the configuration's as --host-frac of the free memory holds)")
+    ap.add_argument("--host-frac", type=float, default=0.40, help="share of the box's available memory the pinned host tier may take")
+    ap.add_argument("--meta-calls", type=int, default=10000, help="score+select calls of the metadata-scale section")
     ap.add_argument("--no-extras", action="store_true", help="skip the mover sweep and the metadata-scale section")
     ap.add_argument("--offload-width", type=int, default=0, help="warp pipelines of the offload mover (0 = library default)")
     ap.add_argument("--prefetch-width", type=int, default=0, help="warp pipelines of the prefetch mover (0 = library default)")
@@ -66,11 +74,52 @@ def measured_peaks():
 
 
 def mem_available_bytes():
+    """Memory this process may still take: MemAvailable, or what its cgroup leaves, whichever is less."""
+    avail = 0
     with open("/proc/meminfo") as f:
         for line in f:
             if line.startswith("MemAvailable:"):
-                return int(line.split()[1]) * 1024
-    return 0
+                avail = int(line.split()[1]) * 1024
+    try:
+        with open("/sys/fs/cgroup/memory.max") as f:
+            lim = f.read().strip()
+        with open("/sys/fs/cgroup/memory.current") as f:
+            cur = int(f.read().strip())
+        if lim != "max":
+            avail = min(avail, max(0, int(lim) - cur))
+    except (OSError, ValueError):
+        pass
+    return avail
+
+
+class PinnedBuffer:
+    """Page-locked host memory of an exact size: a pageable tensor registered with cudaHostRegister (torch's own
+    pinned allocator rounds every request up to a power of two, which would double a 117 GiB tier)."""
+
+    def __init__(self, torch, nbytes):
+        self.torch, self.registered = torch, False
+        t0 = time.time()
+        self.t = torch.empty(nbytes, dtype=torch.uint8)
+        rc = torch.cuda.cudart().cudaHostRegister(self.t.data_ptr(), nbytes, 0)
+        if int(rc) != 0:
+            raise RuntimeError("cudaHostRegister of %d bytes failed (%s)" % (nbytes, rc))
+        self.registered = True
+        self.seconds = time.time() - t0
+
+    def free(self):
+        if self.registered:
+            self.torch.cuda.cudart().cudaHostUnregister(self.t.data_ptr())
+            self.registered = False
+        self.t = None
+
+
+def host_tier_slots(named, block_bytes, asked, frac, n_replicas):
+    """Slots of the host tier that get pinned memory behind them: all the configuration names, unless the box's
+    free memory (times frac, shared by the replicas) is short; then as many as fit (the reduction is reported)."""
+    if asked:
+        return max(1, min(asked, named))
+    budget = int(frac * mem_available_bytes() / max(1, n_replicas))
+    return max(1, min(named, budget // block_bytes))
 
 
 # ---- clocks sampled during the timed region -----------------------------------------------------------
@@ -125,33 +174,30 @@ class ClockSampler:
 
 # ---- the workload ---------------------------------------------------------------------------------------
 class StepWorkload:
-    """Config-1 state on one GPU: pools, index, trace, context, ring of id buffers."""
+    """State of one configuration's scheduler step on one GPU: pools, index, trace, context, ring of id buffers."""
     RING = 3
 
-    def __init__(self, args, device, n_replicas):
+    def __init__(self, args, device, n_replicas, cfg_name="llama8b"):
         import torch
         from paper_2608_14624_b200 import binding as cs
         from paper_2608_14624_b200 import build, synth
         build.build_library()
         self.torch, self.cs, self.synth = torch, cs, synth
         self.dev = device
-        cfg = synth.CONFIGS["llama8b"]
+        cfg = synth.CONFIGS[cfg_name]
+        self.cfg_name = cfg_name
         if args.quick:
             cfg = synth.shrink(cfg, gpu_blocks=2048, host_blocks=6144)
         self.cfg = cfg
         G, Hs, L = cfg.gpu_blocks, cfg.host_blocks, cfg.n_layers
         bb = cfg.block_bytes
-        # host tier: back as many of the 60,000 slots as the box's memory safely allows
-        # (torch's pinned allocator rounds sizes up to a power of two, so only powers of two are asked for)
-        want = args.host_slots or 16384
-        budget = int(0.40 * mem_available_bytes() / max(1, n_replicas))
-        fit = max(1, min(want, Hs, budget // bb))
-        self.host_backed = 1 << (int(fit).bit_length() - 1)
+        # host tier: every slot the configuration names gets pinned memory behind it, unless the box is short of memory
+        self.host_backed = host_tier_slots(Hs, bb, args.host_slots, args.host_frac, n_replicas)
         if args.quick:
             self.host_backed = min(self.host_backed, 1024)
-        t0 = time.time()
-        self.host_buf = torch.empty(self.host_backed * bb, dtype=torch.uint8, pin_memory=True)
-        self.t_pin = time.time() - t0
+        self.pinned = PinnedBuffer(torch, self.host_backed * bb)
+        self.host_buf = self.pinned.t
+        self.t_pin = self.pinned.seconds
         self.gpu_buf = torch.empty(G * bb // 2, dtype=torch.bfloat16, device=device)
         step_elems = 1 << 28
         for lo in range(0, self.gpu_buf.numel(), step_elems):           # N(0,1) bf16 KV values, seeded
@@ -214,8 +260,6 @@ class StepWorkload:
         self.fifo = [torch.zeros(self.k_p, dtype=torch.int64, device=device) for _ in range(8)]
         self.fifo_used = 0
         self.bytes_per_step = (self.k_v + self.k_p) * bb
-        # blocks actually moved, counted on the device from the select counts of every step: [offloaded, prefetched]
-        self.moved = torch.zeros(2, dtype=torch.int64, device=device)
         self.timers = {"select": [], "compact": [], "offload": [], "prefetch": [], "observe": []}
         # warm the learner so that the prefetch gate has something to work with
         self.c.observe_invocations(self.d_chain[:2000], self.d_agent[:2000], self.d_flags[:2000])
@@ -306,9 +350,6 @@ class StepWorkload:
             rec(t[7], self.side_p)
             self.done_p[b] = torch.cuda.Event()
             self.done_p[b].record(self.side_p)
-        # accounting, after the transfers have been issued: blocks this step really moves
-        self.moved[0] += torch.minimum(self.vn[b][0], self.hn[b][0])       # a victim without a host slot is skipped
-        self.moved[1] += self.pn[b][0]
         # engine bookkeeping (plumbing, not the method): refilled victim slots are touched now, prefetched
         # host entries now have a GPU copy
         vi = vict.long().clamp_(min=0)
@@ -348,10 +389,22 @@ class StepWorkload:
         self._pending = []
 
     def take_moved_bytes(self):
-        """KV bytes the steps since the last call really moved over the link (device-side counts), then reset."""
-        n = int(self.moved.sum().item())
-        self.moved.zero_()
-        return n * self.cfg.block_bytes
+        """KV bytes the transfers since the last call really moved over the link: the library's own work counters
+        (kept by the mover kernels, one increment per block copied), read and reset."""
+        self.torch.cuda.synchronize(self.dev)
+        cn = self.c.counters(reset=True)
+        self.last_counters = cn
+        return cn["bytes_moved"][1] + cn["bytes_moved"][2]
+
+    def release(self):
+        """Gives the pools back (the next workload needs the memory)."""
+        self.drain()
+        self.torch.cuda.synchronize(self.dev)
+        self.c.close()
+        self.gpu_buf = self.stage_buf = self.host_buf = None
+        self.gpu_pool = self.host_pool = self.stage_pool = None
+        self.pinned.free()
+        self.torch.cuda.empty_cache()
 
     def e2e_bytes(self):
         ev = 8 * 7          # <= 8 events x (4 + 2 + 1) bytes
@@ -390,8 +443,6 @@ def fused_step_section(w, steps=10):
     ev_f = torch.zeros(cap, dtype=w.d_flags.dtype, device=dev)
     fifo = [torch.zeros(kp, dtype=torch.int64, device=dev) for _ in range(8)]
     state = {"s": w.last_s + 1, "n": 0}
-    moved = torch.zeros(1, dtype=torch.int64, device=dev)
-    ar_kp = torch.arange(kp, dtype=torch.int32, device=dev)
 
     def issue(by_value, now=0, n_ev=cap):
         c.step(w.didx, now, ev_c, ev_a, ev_f, n_ev, kv, kp, gv, gvn, gh, ghn, gp, gpn, w.gpu_pool, w.host_pool, free_d,
@@ -410,8 +461,6 @@ def fused_step_section(w, steps=10):
             issue(True, now, n_ev)
         else:
             graph.replay()
-        # blocks this step really moves (prefetch candidates dropped by the conflict rule are sentinels in the list)
-        moved.add_(torch.minimum(gvn[0], ghn[0]) + ((gp[:kp] >= 0) & (ar_kp < gpn[0])).sum())
         # engine bookkeeping, as in the main run
         vi = gv[:kv].long().clamp_(min=0)
         w.la_i32[vi] = now
@@ -432,14 +481,15 @@ def fused_step_section(w, steps=10):
             main.synchronize()
             l0 = c.launch_count()
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            moved.zero_()
+            c.counters(reset=True)
             e0.record(main)
             for _ in range(k):
                 one_step(graph)
             e1.record(main)
             main.synchronize()
+            cn = c.counters()          # blocks the steps really moved (dropped prefetch candidates are not copied)
         ms = e0.elapsed_time(e1) / k
-        return ms, (c.launch_count() - l0) / k, int(moved.item()) * bb / k / ms / 1e6
+        return ms, (c.launch_count() - l0) / k, (cn["bytes_moved"][1] + cn["bytes_moved"][2]) / k / ms / 1e6
 
     w.drain()
     torch.cuda.synchronize(dev)
@@ -615,23 +665,48 @@ def time_call(torch, stream, fn, reps, warm=1):
     return float(np.median(ts)), float(min(ts))
 
 
+def _block_from_pool(buf_u8, layout, n_slots, L, chunk, slot):
+    """The 2L chunks of one block of a device pool as a flat host array in [layer][plane][byte] order (plain indexing)."""
+    if layout == 0:
+        return buf_u8.view(L, 2, n_slots, chunk)[:, :, slot, :].contiguous().cpu().numpy().reshape(-1)
+    return buf_u8.view(n_slots, L, 2, chunk)[slot].cpu().numpy().reshape(-1)
+
+
+def _check_moved_blocks(orc, get_src, get_dst, src_layout, dst_layout, L, chunk, n, rng, n_samples=32):
+    """After a timed transfer: sampled blocks (every one of their 2L chunks) against the oracle's chunk-by-chunk copy
+    between one-slot stand-in pools.  Returns the number of blocks compared; raises on any differing byte."""
+    picks = rng.choice(n, size=min(n_samples, n), replace=False)
+    for i in picks:
+        stand_src = np.ascontiguousarray(get_src(int(i)))
+        stand_dst = np.zeros_like(stand_src)
+        orc.move_blocks(stand_src, src_layout, 1, stand_dst, dst_layout, 1, L, chunk, [0], [0])
+        if not np.array_equal(get_dst(int(i)), stand_dst):
+            raise RuntimeError("mover sweep: block %d of a %d-block batch differs from the oracle's copy" % (i, n))
+    return len(picks)
+
+
 def mover_sweep(w, hbm_peak, link):
     """Batches of 1..4096 uniformly random scattered blocks: offload, prefetch, device-to-device,
-    GPU pool addressed layer-major and block-major (same memory, two address formulas)."""
+    GPU pool addressed layer-major and block-major (same memory, two address formulas).  After the last
+    repetition of every transfer 32 sampled blocks are compared byte for byte with the oracle's copy."""
+    from oracle import cs_oracle as orc
     torch, cs, synth, c = w.torch, w.cs, w.synth, w.c
     cfg, dev = w.cfg, w.dev
     rng = synth.rng_for(cfg, 11)
-    G, L, bb = cfg.gpu_blocks, cfg.n_layers, cfg.block_bytes
+    G, L, bb, chunk = cfg.gpu_blocks, cfg.n_layers, cfg.block_bytes, cfg.chunk_bytes
     rows = []
     side = w.side_o
+    gpu_u8 = w.gpu_buf.view(torch.uint8)
     up = lambda a: torch.from_numpy(a.view(np.int32)).to(dev)
+    host_block = lambda slot: w.host_buf[slot * bb:(slot + 1) * bb].numpy()
     for n in (1, 8, 64, 512, 4096):
         if n > w.host_backed or 2 * n > G:
             continue
         src, dst_h = synth.mover_batch(n, G - n, w.host_backed, rng)
-        dst_h = dst_h + G                                                   # host pool ids start at G
-        d_src, d_dst_h = up(src.astype(np.uint32)), up(dst_h.astype(np.uint32))
-        d_back = up((G - n + np.arange(n)).astype(np.uint32))              # disjoint from every src
+        back = (G - n + np.arange(n)).astype(np.uint32)                     # disjoint from every src
+        src_rot = np.roll(src, 1)                                           # the compaction moves other blocks than the prefetch did
+        d_src, d_dst_h = up(src.astype(np.uint32)), up((dst_h + G).astype(np.uint32))   # host pool ids start at G
+        d_back, d_src_rot = up(back), up(src_rot.astype(np.uint32))
         reps = 5 if n <= 512 else 3
         # fair comparator for the latency-bound small batches: one contiguous pinned copy of the same size
         tmp = torch.empty(n * bb, dtype=torch.uint8, device=dev)
@@ -642,9 +717,17 @@ def mover_sweep(w, hbm_peak, link):
         del tmp
         for lay_name, lay in (("layer_major", cs.CS_LAYER_MAJOR), ("block_major", cs.CS_BLOCK_MAJOR)):
             gp = cs.KVPool(w.gpu_buf, G, lay, L)
+            pool_block = lambda slot: _block_from_pool(gpu_u8, lay, G, L, chunk, slot)
+            checked = 0
             med_o, best_o = time_call(torch, side, lambda: c.offload_blocks(gp, w.host_pool, d_src, d_dst_h, stream=side), reps)
+            checked += _check_moved_blocks(orc, lambda i: pool_block(int(src[i])), lambda i: host_block(int(dst_h[i])),
+                                           lay, cs.CS_BLOCK_MAJOR, L, chunk, n, rng)
             med_p, best_p = time_call(torch, side, lambda: c.prefetch_blocks(w.host_pool, gp, d_dst_h, d_back, stream=side), reps)
-            med_c, best_c = time_call(torch, side, lambda: c.compact_blocks(gp, gp, d_src, d_back, stream=side), reps)
+            checked += _check_moved_blocks(orc, lambda i: host_block(int(dst_h[i])), lambda i: pool_block(int(back[i])),
+                                           cs.CS_BLOCK_MAJOR, lay, L, chunk, n, rng)
+            med_c, best_c = time_call(torch, side, lambda: c.compact_blocks(gp, gp, d_src_rot, d_back, stream=side), reps)
+            checked += _check_moved_blocks(orc, lambda i: pool_block(int(src_rot[i])), lambda i: pool_block(int(back[i])),
+                                           lay, lay, L, chunk, n, rng)
             gb = n * bb / 1e9
             rows.append({"blocks": n, "gpu_layout": lay_name,
                          "offload_GBps": gb / (med_o / 1e3), "offload_frac_of_link": gb / (med_o / 1e3) / link["d2h"],
@@ -652,7 +735,8 @@ def mover_sweep(w, hbm_peak, link):
                          "memcpy_same_size_d2h_GBps": gb / (cp_o / 1e3), "memcpy_same_size_h2d_GBps": gb / (cp_p / 1e3),
                          "offload_frac_of_memcpy_same_size": cp_o / med_o, "prefetch_frac_of_memcpy_same_size": cp_p / med_p,
                          "d2d_GBps_rw": 2 * gb / (med_c / 1e3), "d2d_frac_of_hbm": 2 * gb / (med_c / 1e3) / hbm_peak,
-                         "offload_ms": med_o, "prefetch_ms": med_p, "d2d_ms": med_c})
+                         "offload_ms": med_o, "prefetch_ms": med_p, "d2d_ms": med_c,
+                         "blocks_byte_checked_against_oracle": checked})
     return rows
 
 
@@ -929,6 +1013,162 @@ def profile_case(args, torch, device):
     print(json.dumps({"workload": args.workload, "launches": c.launch_count(), "device_status": c.get_status()}))
 
 
+WORKLOAD_TEXT = {
+    "llama8b": "llama8b-kv step (BASELINE.json configs[1]): 32 layers x 8 KV heads x 128 bf16, 2 MiB blocks",
+    "llama70b": "llama70b-kv step (BASELINE.json configs[3]): 80 layers x 8 KV heads x 128 bf16, 5 MiB blocks",
+}
+
+
+def oracle_baseline(cfg_name, budget_s):
+    """The oracle as it stands, timed on this machine's host cores for about budget_s seconds of steps."""
+    ow = OracleStep(cfg_name)
+    ow.step(0)
+    t0 = time.perf_counter()
+    n_or = 0
+    while time.perf_counter() - t0 < budget_s and n_or < 40:
+        ow.step(1 + n_or)
+        n_or += 1
+    dt = time.perf_counter() - t0
+    return {"value": ow.bytes_per_step * n_or / dt / 1e9, "unit": "GB/s", "cores": 1, "kind": "oracle",
+            "sample": "%d oracle steps: %s" % (n_or, ow.sample),
+            "blocks_scored_selected_per_s": 3 * ow.idx.n * n_or / dt, "ms_per_step": dt / n_or * 1e3}
+
+
+def measure_step_workload(args, w, ctx):
+    """Warm-up, K timed steps with device-resident inputs (the headline value), K steps end to end, and the
+    per-kernel figures of the step; returns the JSON object of this workload (rank 0's view)."""
+    torch, world, rank, device = ctx["torch"], ctx["world"], ctx["rank"], ctx["device"]
+    barrier, link, hbm_peak, peak_kind = ctx["barrier"], ctx["link"], ctx["hbm_peak"], ctx["peak_kind"]
+    for s in range(args.warmup):
+        w.step(s)
+    w.drain()
+    barrier()
+    sampler = ClockSampler(ctx["local"])
+    if rank == 0:
+        sampler.start()
+    l0 = w.c.launch_count()
+    w.take_moved_bytes()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(w.main)
+    for s in range(args.steps):
+        w.step(args.warmup + s, timed=True)
+    w.drain()
+    e1.record(w.main)
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    launches = w.c.launch_count() - l0
+    moved_bytes = w.take_moved_bytes()                 # what the timed steps really moved (this rank)
+    counters = w.last_counters
+    total_ms = reduce_max_ms(e0.elapsed_time(e1), world, device)
+    w.collect_timers()
+    status = w.c.get_status()
+    last = (args.warmup + args.steps - 1) % w.RING
+    n_out = [int(w.vn[last][0].item()), int(w.hn[last][0].item()), int(w.pn[last][0].item())]
+    if args.skip_aux:
+        return {"workload": "step", "config": w.cfg_name, "ms_per_step": total_ms / args.steps, "gpu_launches": int(launches),
+                "value": job_value(world, moved_bytes / args.steps, args.steps, total_ms), "n_out": n_out}
+
+    # ---- end to end: inputs from pinned host memory, results read back, every step ---------------------------
+    base = args.warmup + args.steps
+    for s in range(2):
+        w.step(base + s, e2e=True)
+    w.drain()
+    barrier()
+    w.take_moved_bytes()
+    f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    f0.record(w.main)
+    for s in range(args.steps):
+        w.step(base + 2 + s, e2e=True)
+    w.drain()
+    f1.record(w.main)
+    barrier()
+    e2e_ms = reduce_max_ms(f0.elapsed_time(f1), world, device)
+    e2e_moved = w.take_moved_bytes()
+    w._pending = []
+    if rank != 0:
+        return {}
+
+    cfg = w.cfg
+    value = job_value(world, moved_bytes / args.steps, args.steps, total_ms)
+    e2e_value = job_value(world, e2e_moved / args.steps, args.steps, e2e_ms)
+    bb = cfg.block_bytes
+    med = lambda k: float(np.median(w.timers[k])) if w.timers[k] else None
+    t_c, t_o, t_p, t_s, t_ob = med("compact"), med("offload"), med("prefetch"), med("select"), med("observe")
+    d2d_gbps = 2 * w.k_v * bb / (t_c / 1e3) / 1e9
+    off_gbps = w.k_v * bb / (t_o / 1e3) / 1e9
+    pre_gbps = w.k_p * bb / (t_p / 1e3) / 1e9
+    sel_bytes = 3 * w.N * 11 + (2 * w.k_v + w.k_p) * 4
+    h2d, d2h = w.e2e_bytes()
+    traffic, traffic_x = None, None
+    tpath = os.path.join(ROOT, "profiles", "ncu_traffic.json")
+    if os.path.exists(tpath) and w.cfg_name == "llama8b":
+        with open(tpath) as f:
+            tj = json.load(f)
+        traffic = tj.get("cs_mover_kernel_d2d_256_blocks_bytes")
+        traffic_x = tj.get("cs_exchange_bulk_kernel_256_out_384_in_dram_bytes")
+    # the two-way transfer: bytes of one launch over its duration on the side stream, against what the link gives two
+    # concurrent pinned cudaMemcpyAsync copies in the same out:in proportion, measured in this run
+    x_ms = t_o if w.fused else max(t_o, t_p)
+    x_gbps = w.bytes_per_step / (x_ms / 1e3) / 1e9
+    # time a perfect duplex link would need for the step's bytes, from the one-direction peaks of this run
+    ideal_ms = max(w.k_v * bb / link["d2h"], w.k_p * bb / link["h2d"]) / 1e6
+    named, backed = cfg.host_blocks, w.host_backed
+    return {
+        "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "u8", "data": "synthetic",
+        "config": {"workload": "%s; GPU pool %d blocks layer-major, host tier %d blocks; %d agents; per step: observe <= 8 invocations, "
+                               "select %d GPU victims + %d host victims + %d prefetch candidates over %d entries, compact %d, "
+                               "offload %d, prefetch %d blocks" % (WORKLOAD_TEXT[w.cfg_name], cfg.gpu_blocks, named, cfg.n_agents,
+                                                                  w.k_v, w.k_v, w.k_p, w.N, w.k_v, w.k_v, w.k_p),
+                   "host_tier": {"named_slots": named, "backed_slots": backed, "reduction": round(1.0 - backed / named, 4),
+                                 "why": "all named slots are pinned" if backed == named else
+                                        "pinned memory limited to %.2f of the box's available memory" % args.host_frac,
+                                 "pinned_GiB": round(backed * bb / GIB, 1), "pin_seconds": round(w.t_pin, 2)},
+                   "l2_policy": "inputs larger than L2: every step moves %.2f GiB of scattered blocks; the %.1f MB index is L2-resident by design"
+                                % ((2 * w.k_v + w.k_p) * bb / GIB, w.N * 11 / 1e6),
+                   "replicas": "replicas only (no data-path collective)", "quick": bool(args.quick)},
+        "blocks_moved_in_timed_steps": {"counted_by_the_mover_kernels": [counters["blocks_moved"][1], counters["blocks_moved"][2]],
+                                        "skipped_list_entries": counters["blocks_skipped"],
+                                        "nominal": args.steps * (w.k_v + w.k_p)},
+        "blocks_scored_selected_per_s": world * 3 * w.N / (t_s / 1e3),
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+        "roofline": {"kernel": ("cs_exchange_bulk_kernel: offload %d + prefetch %d blocks as one launch on the side stream (98 %% of the step's device time)"
+                                % (w.k_v, w.k_p)) if w.fused else "cs_mover_bulk_kernel: offload and prefetch launches on two side streams",
+                     "bound": "host_link", "achieved": x_gbps, "peak": link["bidir_step_mix"], "unit": "GB/s",
+                     "frac": x_gbps / link["bidir_step_mix"], "traffic": traffic_x,
+                     "peak_kind": "measured in this run: two concurrent pinned cudaMemcpyAsync copies of contiguous buffers in the step's "
+                                  "2:3 out:in proportion (PCIe Gen5 x16 is neither HBM nor a tensor pipe)",
+                     "peak_per_direction": {"d2h": link["d2h"], "h2d": link["h2d"], "both_1to1": link["bidir"]},
+                     "ideal_duplex_ms": ideal_ms, "frac_of_ideal_duplex": ideal_ms / x_ms,
+                     "algorithmic_bytes_per_launch": w.bytes_per_step, "ms_per_launch": x_ms,
+                     "traffic_note": "DRAM bytes of one launch (ncu, profiles/): each block crosses HBM once"},
+        "roofline_hbm": {"kernel": "cs_mover_bulk_kernel (device-to-device compaction of the %d victims, inside the step, while the host-link "
+                                   "transfer of the previous step runs beside it)" % w.k_v, "bound": "hbm",
+                         "achieved": d2d_gbps, "peak": hbm_peak, "unit": "GB/s", "frac": d2d_gbps / hbm_peak, "traffic": traffic,
+                         "peak_kind": "of %s" % peak_kind, "algorithmic_bytes_per_launch": 2 * w.k_v * bb, "ms_per_launch": t_c},
+        "host_link": {"peak_d2h_GBps": link["d2h"], "peak_h2d_GBps": link["h2d"], "peak_bidir_GBps": link["bidir"],
+                      "peak_bidir_step_mix_GBps": link["bidir_step_mix"],
+                      "how": "pinned cudaMemcpyAsync of 1 GiB, best of 10, same run; step_mix = 2/3 GiB out while 1 GiB comes in, "
+                             "the proportions of a step, whose inbound direction is the longer one",
+                      "offload_GBps": off_gbps, "offload_frac": off_gbps / link["d2h"], "offload_ms": t_o,
+                      "prefetch_GBps": pre_gbps, "prefetch_frac": pre_gbps / link["h2d"], "prefetch_ms": t_p,
+                      "step_frac_of_bidir": value / world / link["bidir"],
+                      "step_frac_of_bidir_step_mix": value / world / link["bidir_step_mix"],
+                      "transfers": args.transfers,
+                      "note": ("offload and prefetch of a step run as one fused launch (cs_exchange_blocks): both per-direction times "
+                               "are that launch's duration" if w.fused else
+                               "offload and prefetch of a step overlap (full duplex); per-direction times are measured while the other direction is busy")},
+        "select": {"how": "cs_select_step: one launch of three 16-CTA clusters" if w.fused_selects else "three calls", "ms_three_selects": t_s, "ms_observe": t_ob, "algorithmic_bytes": sel_bytes,
+                   "achieved_GBps": sel_bytes / (t_s / 1e3) / 1e9, "frac_of_hbm_peak": sel_bytes / (t_s / 1e3) / 1e9 / hbm_peak,
+                   "n_out_last_step": n_out, "device_status": status},
+        "e2e": {"value": e2e_value, "unit": "GB/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "ms_per_step": e2e_ms / args.steps,
+                "includes": "per step: H2D of the step's events and of the whole index from pinned memory, D2H of the three id lists and counts, host sync on the result"},
+    }
+
+
 def reduce_max_ms(local_ms: float, world: int, device) -> float:
     """Job time = the slowest rank's device time (all-reduce MAX; identity for one rank)."""
     if world <= 1:
@@ -973,150 +1213,38 @@ def main():
     if args.workload != "step":          # one small case of one kernel family, for profiler captures
         profile_case(args, torch, device)
         return
-    w = StepWorkload(args, device, world)
-    cs, synth = w.cs, w.synth
     link = host_link_peak(torch, device) if (rank == 0 and not args.skip_aux) else None
-
-    # ---- device-resident inputs: the headline value ------------------------------------------------------
-    for s in range(args.warmup):
-        w.step(s)
-    w.drain()
-    barrier()
-    sampler = ClockSampler(local)
-    if rank == 0:
-        sampler.start()
-    l0 = w.c.launch_count()
-    w.take_moved_bytes()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(w.main)
-    for s in range(args.steps):
-        w.step(args.warmup + s, timed=True)
-    w.drain()
-    e1.record(w.main)
-    barrier()
-    clocks = sampler.stop() if rank == 0 else None
-    moved_bytes = w.take_moved_bytes()                 # what the timed steps really moved (this rank)
-    launches = w.c.launch_count() - l0
-    total_ms = reduce_max_ms(e0.elapsed_time(e1), world, device)
-    w.collect_timers()
-    status = w.c.get_status()
-    n_out = [int(w.vn[(args.warmup + args.steps - 1) % w.RING][0].item()),
-             int(w.hn[(args.warmup + args.steps - 1) % w.RING][0].item()),
-             int(w.pn[(args.warmup + args.steps - 1) % w.RING][0].item())]
-
+    w = StepWorkload(args, device, world, args.config)
+    cs, synth = w.cs, w.synth
+    ctx = dict(world=world, rank=rank, local=local, device=device, barrier=barrier, link=link, hbm_peak=hbm_peak,
+               peak_kind=peak_kind, torch=torch)
+    out = measure_step_workload(args, w, ctx)
     if args.skip_aux:
         if rank == 0:
-            print(json.dumps({"workload": "step", "ms_per_step": total_ms / args.steps, "gpu_launches": int(launches),
-                              "value": job_value(world, moved_bytes / args.steps, args.steps, total_ms), "n_out": n_out}))
+            print(json.dumps(out))
         if world > 1:
             dist.destroy_process_group()
         return
-
-    # ---- end to end: inputs from pinned host memory, results read back, every step ---------------------------
-    base = args.warmup + args.steps
-    for s in range(2):
-        w.step(base + s, e2e=True)
-    w.drain()
-    barrier()
-    w.take_moved_bytes()
-    f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    f0.record(w.main)
-    for s in range(args.steps):
-        w.step(base + 2 + s, e2e=True)
-    w.drain()
-    f1.record(w.main)
-    barrier()
-    e2e_ms = reduce_max_ms(f0.elapsed_time(f1), world, device)
-    e2e_moved = w.take_moved_bytes()
-
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
-
-    value = job_value(world, moved_bytes / args.steps, args.steps, total_ms)
-    e2e_value = job_value(world, e2e_moved / args.steps, args.steps, e2e_ms)
-    bb = w.cfg.block_bytes
-    med = lambda k: float(np.median(w.timers[k])) if w.timers[k] else None
-    t_c, t_o, t_p, t_s, t_ob = med("compact"), med("offload"), med("prefetch"), med("select"), med("observe")
-    d2d_gbps = 2 * w.k_v * bb / (t_c / 1e3) / 1e9
-    off_gbps = w.k_v * bb / (t_o / 1e3) / 1e9
-    pre_gbps = w.k_p * bb / (t_p / 1e3) / 1e9
-    sel_bytes = 3 * w.N * 11 + (2 * w.k_v + w.k_p) * 4
-    h2d, d2h = w.e2e_bytes()
-    traffic = None
-    tpath = os.path.join(ROOT, "profiles", "ncu_traffic.json")
-    if os.path.exists(tpath):
-        with open(tpath) as f:
-            traffic = json.load(f).get("cs_mover_kernel_d2d_256_blocks_bytes")
-
-    out = {
-        "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "u8", "data": "synthetic",
-        "config": {"workload": "llama8b-kv step (config 1): 32 layers x 8 KV heads x 128 bf16, 2 MiB blocks; GPU pool %d blocks "
-                               "layer-major, host tier %d blocks (%d backed by pinned memory); 12 agents; per step: observe <= 8 "
-                               "invocations, select 256 GPU victims + 256 host victims + 384 prefetch candidates over %d "
-                               "entries, compact 256, offload 256, prefetch 384 blocks" % (
-                                   w.cfg.gpu_blocks, w.cfg.host_blocks, w.host_backed, w.N),
-                   "l2_policy": "inputs larger than L2: every step moves 1.75 GiB of scattered blocks; index 0.9 MB is L2-resident by design",
-                   "replicas": "replicas only (no data-path collective)", "pin_seconds": round(w.t_pin, 2), "quick": bool(args.quick)},
-        "blocks_moved_in_timed_steps": {"counted_on_device": moved_bytes // w.cfg.block_bytes,
-                                        "nominal": args.steps * (w.k_v + w.k_p)},
-        "blocks_scored_selected_per_s": world * 3 * w.N / (t_s / 1e3),
-        "gpu_launches": int(launches),
-        "clocks": clocks,
-        "roofline": {"kernel": "cs_mover_bulk_kernel (device-to-device compaction of the 256 victims, inside the step, while the host-link transfers of the previous step run beside it)", "bound": "hbm",
-                     "achieved": d2d_gbps, "peak": hbm_peak, "unit": "GB/s", "frac": d2d_gbps / hbm_peak, "traffic": traffic,
-                     "peak_kind": "of %s" % peak_kind, "algorithmic_bytes_per_launch": 2 * w.k_v * bb, "ms_per_launch": t_c},
-        "roofline_dominant_kernel": {
-            "kernel": ("cs_exchange_bulk_kernel (offload 256 + prefetch 384 blocks in one launch): 98 % of the step's device time; "
-                       "bound by the host link, which is neither HBM nor a tensor pipe, so it is reported beside the HBM roofline above")
-                      if w.fused else "cs_mover_bulk_kernel, offload and prefetch launches",
-            "bound": "host link (PCIe Gen5 x16, both directions)", "achieved": value / world, "unit": "GB/s",
-            "peak": link["bidir_step_mix"], "frac": value / world / link["bidir_step_mix"],
-            "peak_kind": "measured in this run: two concurrent pinned cudaMemcpyAsync copies in the step's 2:3 out:in proportion",
-            "algorithmic_bytes_per_launch": w.bytes_per_step, "ms_per_launch": t_o if w.fused else max(t_o, t_p)},
-        "host_link": {"peak_d2h_GBps": link["d2h"], "peak_h2d_GBps": link["h2d"], "peak_bidir_GBps": link["bidir"],
-                      "peak_bidir_step_mix_GBps": link["bidir_step_mix"],
-                      "how": "pinned cudaMemcpyAsync of 1 GiB, best of 10, same run; step_mix = 2/3 GiB out while 1 GiB comes in, "
-                             "the proportions of a step, whose inbound direction is the longer one",
-                      "offload_GBps": off_gbps, "offload_frac": off_gbps / link["d2h"], "offload_ms": t_o,
-                      "prefetch_GBps": pre_gbps, "prefetch_frac": pre_gbps / link["h2d"], "prefetch_ms": t_p,
-                      "step_frac_of_bidir": value / world / link["bidir"],
-                      "step_frac_of_bidir_step_mix": value / world / link["bidir_step_mix"],
-                      "transfers": args.transfers,
-                      "note": ("offload and prefetch of a step run as one fused launch (cs_exchange_blocks): both per-direction times "
-                               "are that launch's duration" if w.fused else
-                               "offload and prefetch of a step overlap (full duplex); per-direction times are measured while the other direction is busy")},
-        "select": {"how": "cs_select_step: one launch of three 16-CTA clusters" if w.fused_selects else "three calls", "ms_three_selects": t_s, "ms_observe": t_ob, "algorithmic_bytes": sel_bytes,
-                   "achieved_GBps": sel_bytes / (t_s / 1e3) / 1e9, "frac_of_hbm_peak": sel_bytes / (t_s / 1e3) / 1e9 / hbm_peak,
-                   "n_out_last_step": n_out, "device_status": status},
-        "e2e": {"value": e2e_value, "unit": "GB/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "ms_per_step": e2e_ms / args.steps,
-                "includes": "per step: H2D of the step's events and of the 80,000-entry index from pinned memory, D2H of the three id lists and counts, host sync on the result"},
-    }
     if not args.no_extras and world == 1:
         out["fused_step"] = fused_step_section(w)
         out["mover_sweep"] = mover_sweep(w, hbm_peak, link)
+        w.release()
         del w
-        torch.cuda.empty_cache()
-        out["metadata_scale"] = metadata_scale(torch, cs, synth, device, hbm_peak)
+        other = "llama70b" if args.config == "llama8b" else "llama8b"
+        w2 = StepWorkload(args, device, world, other)
+        sub = measure_step_workload(args, w2, ctx)
+        sub["cpu_baseline"] = oracle_baseline(other, budget_s=8.0)
+        out["second_config"] = sub
+        w2.release()
+        del w2
+        out["metadata_scale"] = metadata_scale(torch, cs, synth, device, hbm_peak, calls=args.meta_calls)
         out["exact_survival"] = exact_survival_section(torch, cs, synth, device)
         out["hbm_regime"] = hbm_regime_section(torch, cs, synth, device, hbm_peak)
-    # the oracle, as it stands, on this machine's host cores
-    ow = OracleStep()
-    ow.step(0)
-    t0 = time.perf_counter()
-    n_or = 0
-    while time.perf_counter() - t0 < 10.0 and n_or < 40:
-        ow.step(1 + n_or)
-        n_or += 1
-    dt = time.perf_counter() - t0
-    out["cpu_baseline"] = {"value": ow.bytes_per_step * n_or / dt / 1e9, "unit": "GB/s", "cores": 1, "kind": "oracle",
-                           "sample": "%d oracle steps: selections over the full 80,000-entry index, mover copies 256+384 blocks of 2 MiB "
-                                     "between two 2,048-slot host stand-in pools (ids modulo 2,048)" % n_or,
-                           "blocks_scored_selected_per_s": 3 * ow.idx.n * n_or / dt, "ms_per_step": dt / n_or * 1e3}
+    out["cpu_baseline"] = oracle_baseline(args.config, budget_s=10.0)     # the oracle, as it stands, on this machine's host cores
     print(json.dumps(out))
     if world > 1:
         dist.destroy_process_group()

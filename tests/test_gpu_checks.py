@@ -154,7 +154,7 @@ def test_counters_agree_with_the_oracle_and_the_lists():
     gv, gh, gp, gvn, ghn, gpn = i32(32), i32(32), i32(64), i32(1), i32(1), i32(1)
     c.select_step(d, now, 32, 64, gv, gvn, gh, ghn, gp, gpn)
     c.set_select_path(cs.CS_SELECT_MULTI)
-    ids, cnt = c.select_victims(d, now, 0, 5000)                    # more than there are eligible entries
+    ids, cnt = c.select_victims(d, now, 0, 2560)                    # more than there are eligible entries
     cn = c.counters()
     assert cn["selects"] == [2, 1, 1]
     assert cn["eligible"][0] == elig(0) and cn["eligible"][1] == elig(1)
