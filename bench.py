@@ -57,7 +57,7 @@ def parse_args():
                     help="the three selects of a step as one launch (cs_select_step) or as three calls")
     ap.add_argument("--exchange-width", type=int, default=0, help="warp pipelines of the fused transfer (0 = library default)")
     ap.add_argument("--quick", action="store_true", help="small pools (debugging only; not a valid bench line)")
-    ap.add_argument("--workload", default="step", choices=["step", "mover", "select", "select80k"],
+    ap.add_argument("--workload", default="step", choices=["step", "mover", "select", "select80k", "select16m", "select64m"],
                     help="'mover'/'select' run one small case of that kernel family only (profiler captures)")
     ap.add_argument("--skip-aux", action="store_true",
                     help="timed steps only: no link-peak probe, end-to-end pass, extras or CPU baseline (profiler launch lists)")
@@ -740,14 +740,17 @@ def mover_sweep(w, hbm_peak, link):
     return rows
 
 
-def metadata_scale(torch, cs, synth, dev, hbm_peak, calls=200):
+def metadata_scale(torch, cs, synth, dev, hbm_peak, calls=10000):
     """1,000,000-entry index, 256 agents: observe 64 events + select 10,000 victims + 2,000 prefetch
-    candidates per call; the first `calls` calls are timed with CUDA events on the stream."""
+    candidates per call, `calls` calls in a row with the index evolving between them; every call is timed
+    with CUDA events on the stream (median and 99th percentile).  Three ways of issuing the same call:
+    the two selects as separate calls, both in one cs_select_step call, and that call replayed from a CUDA graph."""
     cfg = synth.CONFIGS["meta1m"]
     N = 1_000_000
     idx = synth.make_block_index(cfg, n=N, tier="random")
     d = cs.DeviceIndex.from_host(idx, dev)
-    tr = synth.make_trace(cfg, n_invocations=64 * (calls + 40))
+    n_tr = min(calls, 2000)                                    # the event trace is cycled beyond 2,000 calls
+    tr = synth.make_trace(cfg, n_invocations=64 * (n_tr + 40))
     p = cs.make_params(n_agents=cfg.n_agents, n_chains=cfg.n_chains, max_blocks=N, block_tokens=cfg.block_tokens, r_min=0.02)
     c = cs.CacheScout(p, dev)
     ch, ag = torch.from_numpy(tr.chain).to(dev), torch.from_numpy(tr.agent).to(dev)
@@ -758,77 +761,98 @@ def metadata_scale(torch, cs, synth, dev, hbm_peak, calls=200):
     la = d.last_access.view(torch.int32)
     stream = torch.cuda.current_stream(dev)
     fifo = [torch.zeros(cfg.k_prefetch, dtype=torch.int64, device=dev) for _ in range(8)]
-    evs = []
-    l0 = c.launch_count()
-    for call in range(calls + 5):
-        now = 100_000 + call
-        lo = 64 * (30 + call)
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
+    state = {"call": 0}
+
+    def bookkeeping(now):                                      # untimed: victims refilled, prefetched entries leave the
+        la[v.long().clamp_(min=0)] = now                       # host tier and return to it 8 calls later (stationary state)
+        pi = pf.long().clamp_(min=0)
+        d.flags[pi] &= 0xFB
+        if state["call"] >= 8:
+            d.flags[fifo[state["call"] % 8]] |= 4
+        fifo[state["call"] % 8].copy_(pi)
+        state["call"] += 1
+
+    def run(issue, n_calls, warm=5):
+        evs = []
+        l0 = c.launch_count()
+        for k in range(n_calls + warm):
+            call = state["call"]
+            now = 100_000 + call
+            lo = 64 * (30 + call % n_tr)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            issue(now, lo)
+            e1.record(stream)
+            bookkeeping(now)
+            if k >= warm:
+                evs.append((e0, e1))
+        torch.cuda.synchronize(dev)
+        us = np.array([a.elapsed_time(b) for a, b in evs]) * 1e3
+        return {"us_median": float(np.median(us)), "us_p99": float(np.percentile(us, 99)), "us_min": float(us.min()),
+                "us_mean": float(us.mean()), "launches_per_call": (c.launch_count() - l0) / (n_calls + warm)}
+
+    def separate(now, lo):
         c.observe_invocations(ch[lo:lo + 64], ag[lo:lo + 64], None)
         c.select_victims(d, now, 0, cfg.k_victims, v, vn)
         c.select_prefetch(d, now, cfg.k_prefetch, pf, pn)
-        e1.record(stream)
-        la[v.long().clamp_(min=0)] = now                      # untimed bookkeeping: victims refilled
-        pi = pf.long().clamp_(min=0)
-        d.flags[pi] &= 0xFB                                   # prefetched entries leave the host tier ...
-        if call >= 8:
-            d.flags[fifo[call % 8]] |= 4                      # ... and return to it 8 calls later (stationary state)
-        fifo[call % 8].copy_(pi)
-        if call >= 5:
-            evs.append((e0, e1))
-    torch.cuda.synchronize(dev)
-    launches = (c.launch_count() - l0) / (calls + 5)
-    ms = np.array([a.elapsed_time(b) for a, b in evs])
-    per_call = float(np.median(ms)) * 1e-3
-    # the same two selects issued as ONE call (cs_select_step without the host-tier victims): their kernel chains
-    # run side by side on the context's own streams
-    evs2 = []
-    for call in range(calls + 5, 2 * calls + 10):
-        now = 100_000 + call
-        lo = 64 * (30 + call % (calls + 5))
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
+
+    def together(now, lo):
         c.observe_invocations(ch[lo:lo + 64], ag[lo:lo + 64], None)
         c.select_step(d, now, cfg.k_victims, cfg.k_prefetch, v, vn, None, None, pf, pn)
-        e1.record(stream)
-        la[v.long().clamp_(min=0)] = now
-        pi = pf.long().clamp_(min=0)
-        d.flags[pi] &= 0xFB
-        d.flags[fifo[call % 8]] |= 4
-        fifo[call % 8].copy_(pi)
-        if call >= calls + 10:
-            evs2.append((e0, e1))
-    torch.cuda.synchronize(dev)
-    per_call_sbs = float(np.median([a.elapsed_time(b) for a, b in evs2])) * 1e-3
-    # the same call captured once into a CUDA graph and replayed (same events and clock every time: timing only)
+
+    t_wall = time.perf_counter()
+    r_sep = run(separate, calls)
+    r_tog = run(together, calls)
+    # the same call captured once into a CUDA graph that reads the clock from device memory, replayed with fresh events
+    now_d = torch.zeros(4, dtype=torch.int32, device=dev)
+    ev_c, ev_a = torch.zeros(64, dtype=ch.dtype, device=dev), torch.zeros(64, dtype=ag.dtype, device=dev)
     cap = torch.cuda.Stream(device=dev)
     cap.wait_stream(stream)
     g = torch.cuda.CUDAGraph()
-    lo = 64 * 30
     with torch.cuda.graph(g, stream=cap, capture_error_mode="relaxed"):
-        c.observe_invocations(ch[lo:lo + 64], ag[lo:lo + 64], None, stream=cap)
-        c.select_step(d, 100_000, cfg.k_victims, cfg.k_prefetch, v, vn, None, None, pf, pn, stream=cap)
-    gms = []
-    with torch.cuda.stream(cap):
-        for call in range(calls + 5):
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record(cap)
-            g.replay()
-            e1.record(cap)
-            if call >= 5:
-                gms.append((e0, e1))
+        c.observe_invocations(ev_c, ev_a, None, stream=cap)
+        c.set_device_clock(now_d)                  # the captured selects read the clock when they run, not when captured
+        c.select_step(d, 0, cfg.k_victims, cfg.k_prefetch, v, vn, None, None, pf, pn, stream=cap)
+        c.set_device_clock(None)
     cap.synchronize()
-    graph_us = float(np.median([a.elapsed_time(b) for a, b in gms])) * 1e3
+
+    def replay_timed(n_calls, warm=5):
+        evs = []
+        with torch.cuda.stream(cap):
+            for k in range(n_calls + warm):
+                call = state["call"]
+                now = 100_000 + call
+                lo = 64 * (30 + call % n_tr)
+                ev_c.copy_(ch[lo:lo + 64]); ev_a.copy_(ag[lo:lo + 64]); now_d.fill_(now)
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(cap)
+                g.replay()
+                e1.record(cap)
+                bookkeeping(now)
+                if k >= warm:
+                    evs.append((e0, e1))
+        cap.synchronize()
+        us = np.array([a.elapsed_time(b) for a, b in evs]) * 1e3
+        return {"us_median": float(np.median(us)), "us_p99": float(np.percentile(us, 99)), "us_min": float(us.min()),
+                "us_mean": float(us.mean())}
+
+    stream.wait_stream(cap)
+    r_graph = replay_timed(calls)
+    wall = time.perf_counter() - t_wall
+    best = min(r_sep["us_median"], r_tog["us_median"], r_graph["us_median"]) * 1e-6
     algo_bytes = N * (9 + 11) + (cfg.k_victims + cfg.k_prefetch) * 4        # one scan per select when the remembered
     #                                                                        threshold holds: 9 B (victims) + 11 B (prefetch) per entry
-    return {"workload": "metadata-scale: 1,000,000-entry index, 256 agents, k=10000 victims + 2000 prefetch per call",
-            "calls_timed": calls, "us_per_call_median": per_call * 1e6, "us_per_call_min": float(ms.min()) * 1e3,
-            "blocks_scored_selected_per_s": 2 * N / per_call,
-            "algorithmic_GBps": algo_bytes / per_call / 1e9, "frac_of_hbm_peak": algo_bytes / per_call / 1e9 / hbm_peak,
-            "us_per_call_side_by_side": per_call_sbs * 1e6, "blocks_scored_selected_per_s_side_by_side": 2 * N / per_call_sbs,
-            "us_per_call_graph_replay": graph_us,
-            "kernel_launches_per_call": launches, "n_out": [int(vn[0].item()), int(pn[0].item())]}
+    cn = c.counters()
+    return {"workload": "metadata-scale (BASELINE.json configs[4]): 1,000,000-entry index, 256 agents, observe 64 events + k=10000 victims + 2000 prefetch candidates per call",
+            "calls_timed_per_form": calls, "wall_seconds_all_forms": wall,
+            "separate_calls": r_sep, "one_select_step_call": r_tog, "graph_replay": r_graph,
+            "us_per_call_median": best * 1e6, "blocks_scored_selected_per_s": 2 * N / best,
+            "algorithmic_GBps": algo_bytes / best / 1e9, "frac_of_hbm_peak": algo_bytes / best / 1e9 / hbm_peak,
+            "target_frac_of_hbm_peak": 0.60, "target_met": bool(algo_bytes / best / 1e9 / hbm_peak >= 0.60),
+            "note": "11 MB of metadata per call: at 0.60 of the HBM peak a call would last 2.6 us, less than one kernel launch; "
+                    "the call is latency-bound and the fraction is reported as measured",
+            "selects_counted_by_the_kernels": cn["selects"], "n_out": [int(vn[0].item()), int(pn[0].item())],
+            "device_status": c.get_status()}
 
 
 def hbm_regime_section(torch, cs, synth, dev, hbm_peak, n_entries=64_000_000):
@@ -854,7 +878,9 @@ def hbm_regime_section(torch, cs, synth, dev, hbm_peak, n_entries=64_000_000):
     sel_bytes = n_entries * 9 + 4 * k                     # one scan of agent, ref_count, flags, last_access, n_tokens:
     #                                                     the threshold bin remembered from the previous call holds,
     #                                                     so the histogram pass also collects the candidates
-    return {"entries": n_entries, "k": k,
+    cn = c.counters()
+    return {"entries": n_entries, "k": k, "candidates_ordered_per_select": cn["candidates"][0],
+            "selects": cn["selects"][0], "selects_that_read_the_index_once": cn["fast_hits"][0],
             "score_ms": t_score, "score_GBps": score_bytes / t_score / 1e6, "score_frac_of_hbm_peak": score_bytes / t_score / 1e6 / hbm_peak,
             "select_ms": t_sel, "select_GBps": sel_bytes / t_sel / 1e6, "select_frac_of_hbm_peak": sel_bytes / t_sel / 1e6 / hbm_peak,
             "blocks_scored_selected_per_s": n_entries / (t_sel / 1e3), "n_out": int(vn[0].item())}
@@ -890,20 +916,23 @@ def exact_survival_section(torch, cs, synth, dev):
 # ---- the oracle on the host cores (cpu_baseline and --impl reference) ----------------------------------------
 class OracleStep:
     """The same scheduler step computed by the CPU oracle.  Bounded sample: the selections run over
-    the full 80,000-entry index, the mover copies the same 256 + 384 blocks of 2 MiB but between two
-    2,048-slot stand-in pools in host memory (ids taken modulo 2,048), single thread."""
+    the configuration's full index, the mover copies the step's 256 + 384 blocks at their real size but
+    between two stand-in pools of 4 GiB in host memory (ids taken modulo their slot count), single thread."""
 
-    def __init__(self):
+    def __init__(self, cfg_name="llama8b"):
         from oracle import cs_oracle as orc
         from paper_2608_14624_b200 import synth
         self.orc, self.synth = orc, synth
-        cfg = synth.CONFIGS["llama8b"]
+        cfg = synth.CONFIGS[cfg_name]
         self.cfg = cfg
         self.o = orc.Oracle(orc.Params(n_agents=cfg.n_agents, n_chains=cfg.n_chains, block_tokens=cfg.block_tokens, r_min=0.02))
         self.tr = synth.make_trace(cfg)
         self.o.observe(self.tr.chain[:2000], self.tr.agent[:2000], self.tr.evflags[:2000])
         self.idx = synth.make_block_index(cfg)
-        self.S = 2048
+        self.S = (4 * GIB) // cfg.block_bytes            # 2,048 slots of 2 MiB, 819 of 5 MiB
+        self.sample = ("selections over the full %d-entry index; mover copies the step's %d+%d blocks of %.0f MiB between two "
+                       "%d-slot host stand-in pools (ids modulo %d)" % (cfg.n_index, cfg.k_victims, cfg.k_prefetch,
+                                                                        cfg.block_bytes / 2**20, self.S, self.S))
         rng = synth.rng_for(cfg, 21)
         self.a = synth.kv_pool_u16(self.S, cfg.n_layers, cfg.chunk_bytes, rng).view(np.uint8)
         self.b = np.zeros_like(self.a)
@@ -931,7 +960,7 @@ def run_reference(args):
     """--impl reference: the oracle, as it stands, timed on the host cores (rank 0 only)."""
     if int(os.environ.get("RANK", "0")) != 0:
         return
-    ow = OracleStep()
+    ow = OracleStep(args.config)
     for s in range(args.warmup):
         ow.step(s)
     t0 = time.perf_counter()
@@ -939,13 +968,12 @@ def run_reference(args):
         ow.step(args.warmup + s)
     dt = time.perf_counter() - t0
     gbps = ow.bytes_per_step * args.steps / dt / 1e9
-    sample = ("full 80,000-entry index for observe/score/select; mover copies the step's 256+384 blocks of 2 MiB "
-              "between two 2,048-slot host stand-in pools (ids modulo 2,048)")
+    sample = ow.sample
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": gbps, "unit": "GB/s", "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "u8", "data": "synthetic",
-        "config": {"workload": "llama8b-kv step (config 1): observe + 3 selects over 80,000 entries + offload 256 / prefetch 384 blocks of 2 MiB",
+        "config": {"workload": WORKLOAD_TEXT[args.config] + ": observe + 3 selects over the full index + offload 256 / prefetch 384 blocks",
                    "sample": sample},
         "cpu_baseline": {"value": gbps, "unit": "GB/s", "cores": 1, "kind": "oracle", "sample": sample,
                          "blocks_scored_selected_per_s": 3 * ow.idx.n * args.steps / dt},
@@ -965,6 +993,24 @@ def profile_case(args, torch, device):
     from paper_2608_14624_b200 import binding as cs
     from paper_2608_14624_b200 import build, synth
     build.build_library()
+    if args.workload in ("select16m", "select64m"):
+        # one kind of select over an index far larger than L2 (176 MB / 704 MB of metadata): the regime in which the
+        # scans are bound by memory or instruction issue; the first call has no remembered threshold, the rest do
+        cfg = synth.CONFIGS["meta1m"]
+        N = 16_000_000 if args.workload == "select16m" else 64_000_000
+        d = cs.DeviceIndex.from_host(synth.make_block_index(cfg, n=N, tier="random"), device)
+        tr = synth.make_trace(cfg, n_invocations=4000)
+        c = cs.CacheScout(cs.make_params(n_agents=cfg.n_agents, n_chains=cfg.n_chains, max_blocks=N,
+                                         block_tokens=cfg.block_tokens, r_min=0.02), device)
+        c.observe_invocations(torch.from_numpy(tr.chain).to(device), torch.from_numpy(tr.agent).to(device), None)
+        v = torch.empty(cfg.k_victims, dtype=torch.int32, device=device)
+        vn = torch.zeros(4, dtype=torch.int32, device=device)
+        for s in range(max(1, args.steps)):
+            c.select_victims(d, 100_000, 0, cfg.k_victims, v, vn)
+        torch.cuda.synchronize(device)
+        print(json.dumps({"workload": args.workload, "launches": c.launch_count(), "counters": c.counters(),
+                          "device_status": c.get_status()}))
+        return
     if args.workload == "mover":
         cfg = synth.CONFIGS["llama8b"]
         G, Hs, L, bb = 2048, 512, cfg.n_layers, cfg.block_bytes

@@ -231,6 +231,39 @@ int cs_exchange_blocks(cs_ctx *ctx, const cs_kv_pool *gpu, const cs_kv_pool *hos
                        const uint32_t *pre_host_slots, const uint32_t *pre_gpu_slots, uint32_t n_pre_max,
                        const uint32_t *n_pre_dev, cs_stream_t side);
 
+/* ---- the same transfers on the GPU's copy engines --------------------------------------------------------
+ * (No counterpart in the paper, which leaves the transfer to its engine's offload connector, Sec. 4; this is
+ * the alternative to the SM-issued path above for engines whose latency-bound kernels must not share the SMs'
+ * memory system with host-memory traffic.)
+ *
+ * cs_set_mover_staging(): hands the context a caller-owned DEVICE ring (256-byte aligned; at least 4 blocks,
+ * 64-256 MiB is a sensible size) through which staged transfers pass, or takes it away (dev_ring = NULL).
+ * The first call also creates the two streams and the events the staged calls use (host objects, released by
+ * cs_destroy).  The ring must stay alive and unused by others while staged transfers are in flight.
+ *
+ * cs_exchange_blocks_staged(): offload of n_off blocks and prefetch of n_pre blocks.  GPU-side lists
+ * (off_gpu_slots, pre_gpu_slots) are dev arrays exactly as for cs_exchange_blocks().  HOST-side lists
+ * (off_host_ids, pre_host_ids) are arrays in HOST memory, read by this call before it returns: the copy
+ * engines need addresses the host knows.  Each part of the offload list is packed into the ring by the mover
+ * kernel and carried to the host tier by cudaMemcpyAsync, one call per run of consecutive host ids (a list of
+ * consecutive ids becomes a few large copies); the prefetch is the mirror image, ending in a scatter launch.
+ * Kernels run on `stream`, the copies on the context's two streams, ordered by events, so to the caller
+ * everything is ordered on `stream`; the host is never synchronised.
+ * Requirements: the host pool is CS_BLOCK_MAJOR (a block is one run of bytes), both pools agree in geometry.
+ * A host id out of range, CS_ID_NONE included, is CS_EINVAL and nothing is issued (drop such entries and their
+ * GPU-side partners before the call).  CS_ID_NONE or an out-of-range slot in a GPU-side list skips the entry on
+ * the device (status word as usual); for an offload the corresponding host slot then receives unspecified bytes.  Results otherwise equal
+ * cs_exchange_blocks() with the same lists.  The work counters book the blocks as offloaded / prefetched.
+ * cs_offload_blocks_staged() / cs_prefetch_blocks_staged() are the one-directional forms. */
+int cs_set_mover_staging(cs_ctx *ctx, void *dev_ring, size_t bytes);
+int cs_exchange_blocks_staged(cs_ctx *ctx, const cs_kv_pool *gpu, const cs_kv_pool *host, const uint32_t *off_gpu_slots,
+                              const uint32_t *off_host_ids, uint32_t n_off, const uint32_t *pre_host_ids,
+                              const uint32_t *pre_gpu_slots, uint32_t n_pre, cs_stream_t stream);
+int cs_offload_blocks_staged(cs_ctx *ctx, const cs_kv_pool *gpu, const cs_kv_pool *host, const uint32_t *src_slots,
+                             const uint32_t *host_ids, uint32_t n, cs_stream_t stream);
+int cs_prefetch_blocks_staged(cs_ctx *ctx, const cs_kv_pool *host, const cs_kv_pool *gpu, const uint32_t *host_ids,
+                              const uint32_t *dst_slots, uint32_t n, cs_stream_t stream);
+
 /* The selections of a step at once: cs_select_victims(tier 0, k_victims), cs_select_victims(tier 1,
  * k_victims) and cs_select_prefetch(k_prefetch) over the same index and clock, with the same results, run
  * side by side.  A selection whose count pointer is NULL is left out.  For index sizes the single-launch
@@ -327,6 +360,8 @@ typedef struct cs_counters {
     uint64_t selects[3];            /* selects completed, per kind */
     uint64_t eligible[3];           /* eligible entries the latest select of the kind saw */
     uint64_t selected[3];           /* ids emitted, per kind */
+    uint64_t candidates[3];         /* keys the latest select of the kind had to order (k winners + ties of the threshold bin) */
+    uint64_t fast_hits[3];          /* selects whose remembered threshold held: the index was read once, mostly without keys */
     uint64_t blocks_moved[3];       /* blocks copied, per direction */
     uint64_t bytes_moved[3];        /* their bytes (block_bytes each) */
     uint64_t blocks_skipped;        /* mover list entries skipped: CS_ID_NONE or slot out of range */
@@ -422,6 +457,13 @@ int cs_set_select_path(cs_ctx *ctx, uint32_t path);
  * builds its histogram; when the new threshold is not above the remembered one the index is read
  * once instead of twice.  The result never depends on it.  enabled = 0 turns the speculation off. */
 int cs_set_select_speculation(cs_ctx *ctx, uint32_t enabled);
+
+/* Clock source for CUDA-graph replay (the paper's runtime reads now() when a block is touched, Algorithm 1;
+ * a captured call would freeze its `now` argument).  While now_dev (dev, 4-byte aligned) is set, every
+ * cs_score_blocks / cs_select_* call issued on this context reads the clock from that word WHEN ITS KERNELS
+ * RUN and ignores its `now` argument, so one captured sequence serves later steps after the caller has
+ * updated the word.  NULL restores the argument.  Host-side switch, no launch. */
+int cs_set_device_clock(cs_ctx *ctx, const uint32_t *now_dev);
 
 /* cudaError_t of the last failing CUDA call on this context (0 if none). */
 int cs_last_cuda_error(cs_ctx *ctx);

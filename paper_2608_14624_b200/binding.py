@@ -34,7 +34,8 @@ EXPORTS = ("cs_workspace_bytes", "cs_create", "cs_destroy", "cs_observe_invocati
            "cs_last_cuda_error", "cs_strerror", "cs_version", "cs_select_victims_static", "cs_set_mover_path", "cs_set_select_path",
            "cs_exact_survival", "cs_use_survival_table", "cs_import_state", "cs_set_select_speculation", "cs_exchange_blocks", "cs_step", "cs_set_survival_sources", "cs_select_step",
            "cs_get_counters", "cs_validate_selection", "cs_validate_move_lists", "cs_validate_exchange_lists",
-           "cs_selftest_bounded_wait")
+           "cs_selftest_bounded_wait", "cs_set_device_clock", "cs_set_mover_staging", "cs_exchange_blocks_staged",
+           "cs_offload_blocks_staged", "cs_prefetch_blocks_staged")
 
 
 class cs_params(C.Structure):
@@ -69,6 +70,7 @@ class cs_step_io(C.Structure):
 class cs_counters(C.Structure):
     _fields_ = [("events_seen", C.c_uint64), ("events_skipped", C.c_uint64), ("transitions_counted", C.c_uint64),
                 ("selects", C.c_uint64 * 3), ("eligible", C.c_uint64 * 3), ("selected", C.c_uint64 * 3),
+                ("candidates", C.c_uint64 * 3), ("fast_hits", C.c_uint64 * 3),
                 ("blocks_moved", C.c_uint64 * 3), ("bytes_moved", C.c_uint64 * 3), ("blocks_skipped", C.c_uint64)]
 
 
@@ -126,6 +128,11 @@ def lib():
         L.cs_validate_exchange_lists.argtypes = [vp, C.POINTER(cs_kv_pool), C.POINTER(cs_kv_pool), vp, vp, u32, vp, vp, vp,
                                                  u32, vp, vp]
         L.cs_selftest_bounded_wait.argtypes = [vp, u32, vp]
+        L.cs_set_device_clock.argtypes = [vp, vp]
+        L.cs_set_mover_staging.argtypes = [vp, vp, C.c_size_t]
+        L.cs_exchange_blocks_staged.argtypes = [vp, C.POINTER(cs_kv_pool), C.POINTER(cs_kv_pool), vp, vp, u32, vp, vp, u32, vp]
+        L.cs_offload_blocks_staged.argtypes = [vp, C.POINTER(cs_kv_pool), C.POINTER(cs_kv_pool), vp, vp, u32, vp]
+        L.cs_prefetch_blocks_staged.argtypes = [vp, C.POINTER(cs_kv_pool), C.POINTER(cs_kv_pool), vp, vp, u32, vp]
         _lib = L
     return _lib
 
@@ -284,6 +291,46 @@ def cs_validate_exchange_lists(ctx, gpu: cs_kv_pool, host: cs_kv_pool, off_gpu_s
 
 def cs_selftest_bounded_wait(ctx, max_polls: int, stream=None):
     _chk(lib().cs_selftest_bounded_wait(ctx, max_polls, _stream(stream)), "cs_selftest_bounded_wait", ctx)
+
+
+def _host_ids(a):
+    """Host-memory id list for the staged calls: a NumPy uint32 array (or None); returns (keep-alive, address)."""
+    if a is None:
+        return None, None
+    import numpy as np
+    arr = np.ascontiguousarray(a, dtype=np.uint32)
+    return arr, arr.ctypes.data
+
+
+def cs_set_mover_staging(ctx, ring):
+    if ring is None:
+        _chk(lib().cs_set_mover_staging(ctx, None, 0), "cs_set_mover_staging", ctx)
+    else:
+        _chk(lib().cs_set_mover_staging(ctx, _ptr(ring), ring.numel() * ring.element_size()), "cs_set_mover_staging", ctx)
+
+
+def cs_exchange_blocks_staged(ctx, gpu: cs_kv_pool, host: cs_kv_pool, off_gpu_slots, off_host_ids, n_off: int,
+                              pre_host_ids, pre_gpu_slots, n_pre: int, stream=None):
+    ko, po = _host_ids(off_host_ids)
+    kp, pp = _host_ids(pre_host_ids)
+    _chk(lib().cs_exchange_blocks_staged(ctx, C.byref(gpu), C.byref(host), _ptr(off_gpu_slots), po, n_off, pp,
+                                         _ptr(pre_gpu_slots), n_pre, _stream(stream)), "cs_exchange_blocks_staged", ctx)
+
+
+def cs_offload_blocks_staged(ctx, gpu: cs_kv_pool, host: cs_kv_pool, src_slots, host_ids, n: int, stream=None):
+    k, p = _host_ids(host_ids)
+    _chk(lib().cs_offload_blocks_staged(ctx, C.byref(gpu), C.byref(host), _ptr(src_slots), p, n, _stream(stream)),
+         "cs_offload_blocks_staged", ctx)
+
+
+def cs_prefetch_blocks_staged(ctx, host: cs_kv_pool, gpu: cs_kv_pool, host_ids, dst_slots, n: int, stream=None):
+    k, p = _host_ids(host_ids)
+    _chk(lib().cs_prefetch_blocks_staged(ctx, C.byref(host), C.byref(gpu), p, _ptr(dst_slots), n, _stream(stream)),
+         "cs_prefetch_blocks_staged", ctx)
+
+
+def cs_set_device_clock(ctx, now_dev):
+    _chk(lib().cs_set_device_clock(ctx, _ptr(now_dev)), "cs_set_device_clock", ctx)
 
 
 def cs_launch_count(ctx) -> int:
@@ -531,6 +578,24 @@ class CacheScout:
             n_pre_max = 0 if pre_host_slots is None else int(pre_host_slots.numel())
         cs_validate_exchange_lists(self.ctx, gpu.struct(), host.struct(), off_gpu_slots, off_host_slots, n_off_max,
                                    n_off_dev, pre_host_slots, pre_gpu_slots, n_pre_max, n_pre_dev, stream)
+
+    def set_mover_staging(self, ring):
+        """Device ring (a torch uint8 tensor, kept alive here) for the copy-engine transfers; None takes it away."""
+        cs_set_mover_staging(self.ctx, ring)
+        self._ring_keepalive = ring
+
+    def exchange_blocks_staged(self, gpu: KVPool, host: KVPool, off_gpu_slots, off_host_ids, pre_host_ids, pre_gpu_slots,
+                               stream=None):
+        """Offload + prefetch on the copy engines; the host-side id lists are NumPy arrays (host memory)."""
+        n_off = 0 if off_host_ids is None else len(off_host_ids)
+        n_pre = 0 if pre_host_ids is None else len(pre_host_ids)
+        cs_exchange_blocks_staged(self.ctx, gpu.struct(), host.struct(), off_gpu_slots, off_host_ids, n_off, pre_host_ids,
+                                  pre_gpu_slots, n_pre, stream)
+
+    def set_device_clock(self, now_dev):
+        """Selects and scores read the clock from this device word when they run (CUDA-graph replay); None = the argument."""
+        self._clock_keepalive = now_dev
+        cs_set_device_clock(self.ctx, now_dev)
 
     def selftest_bounded_wait(self, max_polls: int = 1000, stream=None):
         cs_selftest_bounded_wait(self.ctx, max_polls, stream)

@@ -226,6 +226,7 @@ int cs_destroy(cs_ctx *ctx)
         if (ctx->ev_sel_join[j]) cudaEventDestroy(ctx->ev_sel_join[j]);
         if (ctx->sel_stream[j]) cudaStreamDestroy(ctx->sel_stream[j]);
     }
+    cs_release_staging(ctx);
     delete ctx;
     return CS_OK;
 }
@@ -591,6 +592,14 @@ int cs_use_survival_table(cs_ctx *ctx, const float *fsurv)
 {
     if (!ctx || (((uintptr_t)fsurv) & 3u)) return CS_EINVAL;
     ctx->fsurv_override = fsurv;
+    return CS_OK;
+}
+
+int cs_set_device_clock(cs_ctx *ctx, const uint32_t *now_dev)
+{
+    if (!ctx || (((uintptr_t)now_dev) & 3u)) return CS_EINVAL;
+    if (now_dev && !cs_device_can_address(now_dev)) return CS_EINVAL;
+    ctx->clock_dev = now_dev;
     return CS_OK;
 }
 

@@ -51,8 +51,9 @@ struct cs_sel_state {
     uint32_t b_last;        // last bucket that holds one of the k winners
     uint32_t p_end;         // end position of that bucket
     uint32_t n_out;         // min(k, eligible)
-    uint32_t c_spec;        // candidates appended speculatively by the histogram pass; 0 between calls
-    uint32_t spec;          // 1: the speculative candidates cover the k winners, the collect pass is skipped
+    uint32_t c_spec;        // candidates appended by the fast pass; 0 between calls
+    uint32_t n_above;       // eligible entries the fast pass found above the remembered bin; 0 between calls
+    uint32_t spec;          // 1: the fast pass's candidates cover the k winners, the histogram and collect passes are skipped
     uint32_t cc[2];         // candidate counters of the cluster kernel: a call uses one and clears the other for the
                             // next call, so that the counter is zero on entry without a barrier
     uint32_t toggle;        // which of the two the next call uses; flipped by every call on the device, so that a
@@ -106,12 +107,21 @@ struct cs_ctx {
     uint32_t no_speculation;       // 1: the histogram pass never collects ahead of the threshold
     uint32_t source_mode;          // CS_SOURCES_*: where the cached BFS of Eq. 8 starts
     const float *fsurv_override;   // caller's survival table for score / select, NULL = the BFS table of Eq. 8
+    const uint32_t *clock_dev;           // cs_set_device_clock(): selects and scores read the clock from here when they run
     const uint32_t *step_now_dev;        // set only while cs_step() issues its calls: device-resident clock / event count
     const uint32_t *step_n_events_dev;
     cudaEvent_t ev_fork, ev_join;        // cs_step(): main -> side and side -> main
     cudaStream_t sel_stream[2];          // the second and third select of a step run here, beside the first
     cudaEvent_t ev_sel_fork, ev_sel_join[2];
     int concurrent_selects;              // the per-select scratch regions are full size
+    // copy-engine path of the mover (cs_set_mover_staging): caller-owned device ring split into four sub-buffers
+    // (two per direction, double-buffered), two streams of the context for the two DMA directions, and the events
+    // that order packing / copying / scattering
+    unsigned char *stage_ring;
+    size_t stage_bytes;
+    cudaStream_t copy_stream[2];         // 0: device -> host, 1: host -> device
+    cudaEvent_t ev_stage_fork, ev_stage_join[2];
+    cudaEvent_t ev_packed[2], ev_copied[2], ev_filled[2], ev_scattered[2];
     uint64_t n_launches;
     int last_cuda_error;
 };
@@ -143,6 +153,9 @@ int cs_launch_mover(cs_ctx *ctx, const cs_kv_pool *src, const cs_kv_pool *dst, c
                     const uint32_t *dst_slots, uint32_t n_max, const uint32_t *n_dev, int kind,
                     cudaStream_t s);
 
+int cs_launch_mover_as(cs_ctx *ctx, const cs_kv_pool *src, const cs_kv_pool *dst, const uint32_t *src_slots,
+                       const uint32_t *dst_slots, uint32_t n_max, const uint32_t *n_dev, int kind, int count_as,
+                       cudaStream_t s);
 int cs_launch_bounded_wait_selftest(cs_ctx *ctx, uint32_t max_polls, cudaStream_t s);
 int cs_launch_validate_selection(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, int prefetch, uint32_t tier,
                                  uint32_t k, const uint32_t *ids, const uint32_t *n_out, cudaStream_t s);
@@ -150,6 +163,7 @@ int cs_launch_validate_lists(cs_ctx *ctx, const uint32_t *w_list, const uint32_t
                              const uint32_t *nw_dev, const uint32_t *x_list, const uint32_t *x_partner, uint32_t nx_max,
                              const uint32_t *nx_dev, int self, cudaStream_t s);
 bool cs_device_can_address(const void *ptr);
+void cs_release_staging(cs_ctx *ctx);
 
 int cs_launch_exchange(cs_ctx *ctx, const cs_kv_pool *gpu, const cs_kv_pool *host, const uint32_t *off_gpu_slots,
                        const uint32_t *off_host_slots, uint32_t n_off_max, const uint32_t *n_off_dev,

@@ -65,7 +65,8 @@ __device__ __forceinline__ bool resolve_piece(const MoverArgs &a, unsigned long 
     const uint32_t i = (uint32_t)(w / per_block);
     const uint32_t r = (uint32_t)(w - (unsigned long long)i * per_block);
     const uint32_t lp = r / a.pieces, piece = r - lp * a.pieces;
-    uint32_t s = __ldg(a.src_slots + i), d = __ldg(a.dst_slots + i);
+    // a missing list means "packed": entry i is slot i (the staging ring of the copy-engine path)
+    uint32_t s = a.src_slots ? __ldg(a.src_slots + i) : i, d = a.dst_slots ? __ldg(a.dst_slots + i) : i;
     const bool first = report && r == 0;                // one piece per block does the block's bookkeeping
     if (s == CS_ID_NONE || d == CS_ID_NONE) {
         if (first) atomicAdd((unsigned long long *)&a.cnt->blocks_skipped, 1ull);
@@ -371,9 +372,19 @@ static int bulk_opt_in(cs_ctx *ctx)
 int cs_launch_mover(cs_ctx *ctx, const cs_kv_pool *src, const cs_kv_pool *dst, const uint32_t *src_slots,
                     const uint32_t *dst_slots, uint32_t n_max, const uint32_t *n_dev, int kind, cudaStream_t s)
 {
+    return cs_launch_mover_as(ctx, src, dst, src_slots, dst_slots, n_max, n_dev, kind, kind, s);
+}
+
+// `kind` decides the width of the launch (which memory the bytes cross), `count_as` the direction the work
+// counters book the blocks under (the pack and scatter launches of the copy-engine path move blocks inside the
+// device on behalf of an offload or a prefetch).
+int cs_launch_mover_as(cs_ctx *ctx, const cs_kv_pool *src, const cs_kv_pool *dst, const uint32_t *src_slots,
+                       const uint32_t *dst_slots, uint32_t n_max, const uint32_t *n_dev, int kind, int count_as,
+                       cudaStream_t s)
+{
     const bool bulk = ctx->mover_path != CS_MOVER_LDST;
     MoverArgs a;
-    fill_mover_args(ctx, a, src, dst, src_slots, dst_slots, n_max, n_dev, bulk ? TM_PIECE : MV_PIECE, kind);
+    fill_mover_args(ctx, a, src, dst, src_slots, dst_slots, n_max, n_dev, bulk ? TM_PIECE : MV_PIECE, count_as);
     const unsigned long long total = (unsigned long long)n_max * 2ull * a.L * a.pieces;
     unsigned long long cap;
     if (bulk) {

@@ -101,43 +101,48 @@ __device__ __forceinline__ void publish_splitters(const cs_workspace &ws, unsign
 }
 
 // ---------------------------------------------------------------------------------------------
-// 1 histogram (+ speculative collect)
+// 0 fast pass (remembered threshold)
 //
-// The threshold bin moves little from one call to the next, so the pass that builds the histogram
-// also appends, speculatively, every entry at or below the bin the previous call of the same kind
-// ended with.  The last CTA finds the true threshold from the exact histogram; if it is not above
-// the remembered one, the candidates are already complete and the collect pass has nothing to do.
-// Otherwise the speculative candidates are dropped and the collect pass runs as usual.  Either
-// way the result is exact: the remembered bin only decides how many times the index is read.
+// The threshold bin moves little from one call to the next, so each kind of call (GPU victims, host
+// victims, prefetch) remembers a bin H at or a little above the one it ended with.  With H known, almost
+// every eligible entry can be dismissed without its key: it lies above H exactly when x = fl(f * g) is on
+// the far side of a per-size threshold (build_x_thresholds), which costs two look-ups, a multiply and a
+// compare.  Those entries are only counted.  The few at or below H get their key, an exact histogram bin
+// and a place in the candidate buffer.  The last CTA then has the exact histogram of bins <= H plus the
+// number of entries above: if the k-th smallest key lies within H the candidates are complete, the
+// sample sort is set up right here and the index has been read ONCE, at a fraction of the instructions of
+// a full-key scan.  Otherwise (the threshold rose above H, or nothing is remembered yet) the pass reports
+// a miss and the full histogram and collect passes below run.  The result never depends on H.
 // ---------------------------------------------------------------------------------------------
 template <bool PF>
-__global__ void __launch_bounds__(SEL_THREADS) cs_sel_hist_kernel(SelArgs a, cs_workspace ws)
+__global__ void __launch_bounds__(SEL_THREADS) cs_sel_fast_kernel(SelArgs a, cs_workspace ws)
 {
     extern __shared__ float smem[];
     __shared__ __align__(16) uint32_t s_hist[CS_HIST_BINS];
+    __shared__ uint32_t s_xt[2 * XT_TOK];
     __shared__ uint32_t s_part[SEL_THREADS];
-    __shared__ uint32_t s_b0, s_ahead;
+    __shared__ uint32_t s_b0, s_ahead, s_above;
     __shared__ bool s_flag;
     cs_wait_for_predecessor();
     cs_release_successor();
+    const uint32_t H = ws.sc->sel_hint[a.hint_slot];        // ~0: nothing remembered
+    if (H == 0xFFFFFFFFu) {                                   // every CTA sees the same word
+        if (blockIdx.x == 0 && threadIdx.x == 0) ws.sel->spec = 0;
+        return;
+    }
     resolve_now(a);
     Tables T;
     load_tables(a, ws, smem, T, PF && a.anchor);
+    build_x_thresholds<PF>(a, H, s_xt);
     for (uint32_t i = threadIdx.x; i < CS_HIST_BINS; i += blockDim.x) s_hist[i] = 0;
+    if (threadIdx.x == 0) s_above = 0;
     __syncthreads();
-    const uint32_t hint = ws.sc->sel_hint[a.hint_slot];     // ~0: nothing remembered, no speculation
     const uint32_t lane = threadIdx.x & 31;
+    uint32_t n_above = 0;
     if (!PF || prefetch_enabled(ws, a.A)) {
         const uint32_t gtid = blockIdx.x * blockDim.x + threadIdx.x, nth = gridDim.x * blockDim.x;
         const uint32_t n_tiles = a.n / TILE, n_warps = nth >> 5;
         const uint32_t n_iter = (n_tiles + n_warps - 1) / n_warps;     // whole warps stay in the shuffles
-        uint32_t run_bin = 0xFFFFFFFFu, run_cnt = 0;                    // adjacent entries often share a bin
-        auto add = [&](uint32_t bin) {
-            if (bin == run_bin) { ++run_cnt; return; }
-            if (run_cnt) atomicAdd(&s_hist[run_bin], run_cnt);
-            run_bin = bin;
-            run_cnt = 1;
-        };
         for (uint32_t it = 0; it < n_iter; ++it) {
             const uint32_t t = it * n_warps + (gtid >> 5);
             uint32_t mask = 0;
@@ -148,16 +153,20 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_hist_kernel(SelArgs a, cs_
 #pragma unroll
                 for (int j = 0; j < GRP; ++j) {
                     if (!((em >> j) & 1u)) continue;
-                    uint32_t pr, se;
+                    const uint32_t ag = grp_u16(G.ag0, G.ag1, j);
+                    if (ag >= a.A) { atomicOr(&ws.sc->status, CS_ST_BAD_AGENT); continue; }
+                    if (PF && a.anchor && !(grp_u16(G.dp0, G.dp1, j) < T.anchor[ag])) continue;
                     const uint32_t tok = a.ntok ? grp_u8(G.tk, j) : a.block_tokens;
-                    const uint32_t dp = (PF && a.anchor) ? grp_u16(G.dp0, G.dp1, j) : 0u;
-                    if (entry_key_rest<PF>(a, T, &ws.sc->status, grp_u16(G.ag0, G.ag1, j), dp, grp_u8(G.fl, j), grp_u32(G, j), tok, pr, se)) {
-                        add(pr >> 20);
-                        if (hint != 0xFFFFFFFFu && (pr >> 20) <= hint) mask |= 1u << j;
-                    }
+                    const uint32_t la = grp_u32(G, j);
+                    const uint32_t age = la <= a.now ? a.now - la : 0u;
+                    const uint32_t xb = __float_as_uint(__fmul_rn(T.fsurv[ag], recency_of_age(a, T, age)));
+                    const uint32_t X = s_xt[((PF && ag != T.a_star) ? XT_TOK : 0u) + tok];
+                    const bool cand = PF ? (xb >= X) : (xb < X);
+                    if (cand) mask |= 1u << j;
+                    else ++n_above;
                 }
             }
-            if (hint == 0xFFFFFFFFu || !__any_sync(0xFFFFFFFFu, mask != 0)) continue;
+            if (!__any_sync(0xFFFFFFFFu, mask != 0)) continue;      // most warps hold no candidate at all
             const uint32_t cnt = __popc(mask);
             uint32_t incl = cnt;
 #pragma unroll
@@ -171,11 +180,12 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_hist_kernel(SelArgs a, cs_
             uint32_t pos = base + incl - cnt;
 #pragma unroll
             for (int j = 0; j < GRP; ++j) {
-                if (mask & (1u << j)) {                       // the key again, for the few that are written
+                if (mask & (1u << j)) {                       // the key, for the few that are kept
                     uint32_t pr, se;
                     const uint32_t tok = a.ntok ? grp_u8(G.tk, j) : a.block_tokens;
                     const uint32_t dp = (PF && a.anchor) ? grp_u16(G.dp0, G.dp1, j) : 0u;
                     entry_key_rest<PF>(a, T, &ws.sc->status, grp_u16(G.ag0, G.ag1, j), dp, grp_u8(G.fl, j), grp_u32(G, j), tok, pr, se);
+                    atomicAdd(&s_hist[pr >> 20], 1u);
                     ws.cand_km[pos] = ((unsigned long long)pr << 32) | se;
                     ws.cand_id[pos] = grp_id(t, lane, j);
                     ++pos;
@@ -183,19 +193,124 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_hist_kernel(SelArgs a, cs_
             }
         }
         const uint32_t t0 = n_tiles * TILE;
-        if (gtid < a.n - t0) {
+        if (gtid < a.n - t0) {                                // ragged tail, one entry per thread, through the key
             const uint32_t i = t0 + gtid;
             uint32_t pr, se;
             const uint32_t tok = a.ntok ? a.ntok[i] : a.block_tokens;
             if (entry_key<PF>(a, T, &ws.sc->status, a.agent[i], a.depth[i], a.ref[i], a.flags[i], a.la[i], tok, pr, se)) {
-                add(pr >> 20);
-                if (hint != 0xFFFFFFFFu && (pr >> 20) <= hint) {
+                if ((pr >> 20) <= H) {
+                    atomicAdd(&s_hist[pr >> 20], 1u);
                     const uint32_t pos = atomicAdd(&ws.sel->c_spec, 1u);
                     ws.cand_km[pos] = ((unsigned long long)pr << 32) | se;
                     ws.cand_id[pos] = i;
+                } else {
+                    ++n_above;
                 }
             }
         }
+    }
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) n_above += __shfl_xor_sync(0xFFFFFFFFu, n_above, d);
+    if (lane == 0 && n_above) atomicAdd(&s_above, n_above);
+    __syncthreads();
+    const uint32_t h_end = H < CS_HIST_BINS ? H + 1u : CS_HIST_BINS;          // bins above H stay empty
+    for (uint32_t i = threadIdx.x; i < h_end; i += blockDim.x) {
+        const uint32_t v = s_hist[i];
+        if (v) atomicAdd(&ws.hist[i], v);
+    }
+    if (threadIdx.x == 0 && s_above) atomicAdd(&ws.sel->n_above, s_above);
+    if (!last_cta_done(&ws.sel->ticket[0], &s_flag)) return;
+
+    // ---- last CTA: is the k-th smallest key within the remembered bin? ---------------------------------
+    constexpr uint32_t PER = CS_HIST_BINS / SEL_THREADS;
+    uint32_t loc[PER], sum = 0;
+#pragma unroll
+    for (uint32_t q = 0; q < PER; ++q) {
+        loc[q] = __ldcg(&ws.hist[threadIdx.x * PER + q]);
+        ws.hist[threadIdx.x * PER + q] = 0;                 // ready for the next pass or call
+        sum += loc[q];
+    }
+    s_part[threadIdx.x] = sum;
+    if (threadIdx.x == 0) s_b0 = 0xFFFFFFFFu;
+    __syncthreads();
+    for (uint32_t d = 1; d < SEL_THREADS; d <<= 1) {         // inclusive scan
+        const uint32_t v = threadIdx.x >= d ? s_part[threadIdx.x - d] : 0;
+        __syncthreads();
+        s_part[threadIdx.x] += v;
+        __syncthreads();
+    }
+    const uint32_t below = s_part[SEL_THREADS - 1];          // eligible entries at or below H
+    const uint32_t total = below + __ldcg(&ws.sel->n_above);
+    const uint32_t before = s_part[threadIdx.x] - sum;
+    if (a.k && below >= a.k && before < a.k && a.k <= before + sum) {
+        uint32_t run = before;
+#pragma unroll
+        for (uint32_t q = 0; q < PER; ++q) {
+            run += loc[q];
+            if (run >= a.k) { s_b0 = threadIdx.x * PER + q; break; }
+        }
+    }
+    __syncthreads();
+    // complete when the k winners lie at or below H, when fewer than k entries are eligible and all of them do, or when k = 0
+    const bool hit = a.k == 0 || below >= a.k || below == total;
+    const uint32_t b0 = a.k == 0 ? 0xFFFFFFFFu : (s_b0 != 0xFFFFFFFFu ? s_b0 : (H < CS_HIST_BINS ? H : CS_HIST_BINS - 1));
+    uint32_t ahead = 0;
+    const bool have_b0 = a.k && below >= a.k;
+    if (hit && have_b0) {
+        ahead = collect_ahead_limit<PER>(loc, threadIdx.x * PER, before, a.k, b0, &s_ahead);
+        if (ahead > H) ahead = H;                             // nothing is known about the bins above H
+    }
+    const uint32_t c_spec = __ldcg(&ws.sel->c_spec);
+    if (hit) publish_splitters(ws, (unsigned long long *)s_hist, s_hist + 2 * CS_SAMPLE, a.k ? c_spec : 0u);
+    if (threadIdx.x == 0) {
+        if (hit) {
+            ws.sel->b0 = b0;
+            ws.sel->n_elig = total;
+            ws.sel->n_out = total < a.k ? total : a.k;
+            ws.sel->c = a.k ? c_spec : 0u;
+            count_select(ws, a.kind, total, total < a.k ? total : a.k);
+            count_candidates(ws, a.kind, a.k ? c_spec : 0u, true);
+            // fewer eligible entries than k: keep H; otherwise tighten it to what the histogram allows
+            if (have_b0) remember_threshold(ws.sc, a.hint_slot, true, ahead);
+        }
+        ws.sel->spec = hit ? 1u : 0u;
+        ws.sel->c_spec = 0;
+        ws.sel->n_above = 0;
+        ws.sel->ticket[0] = 0;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// 1 histogram (runs when the fast pass missed or had nothing to go by)
+//
+// Full keys of all eligible entries into a 4096-bin histogram; the last CTA finds the threshold bin and
+// chooses how far ahead of it the next call of this kind may look.
+// ---------------------------------------------------------------------------------------------
+template <bool PF>
+__global__ void __launch_bounds__(SEL_THREADS) cs_sel_hist_kernel(SelArgs a, cs_workspace ws)
+{
+    extern __shared__ float smem[];
+    __shared__ __align__(16) uint32_t s_hist[CS_HIST_BINS];
+    __shared__ uint32_t s_part[SEL_THREADS];
+    __shared__ uint32_t s_b0, s_ahead;
+    __shared__ bool s_flag;
+    cs_wait_for_predecessor();
+    cs_release_successor();
+    if (ws.sel->spec) return;          // the fast pass already has the candidates
+    resolve_now(a);
+    Tables T;
+    load_tables(a, ws, smem, T, PF && a.anchor);
+    for (uint32_t i = threadIdx.x; i < CS_HIST_BINS; i += blockDim.x) s_hist[i] = 0;
+    __syncthreads();
+    if (!PF || prefetch_enabled(ws, a.A)) {
+        uint32_t run_bin = 0xFFFFFFFFu, run_cnt = 0;                    // adjacent entries often share a bin
+        for_each_eligible<PF>(a, T, &ws.sc->status, [&](uint32_t, uint32_t pr, uint32_t) {
+            const uint32_t bin = pr >> 20;
+            if (bin == run_bin) { ++run_cnt; return; }
+            if (run_cnt) atomicAdd(&s_hist[run_bin], run_cnt);
+            run_bin = bin;
+            run_cnt = 1;
+        });
         if (run_cnt) atomicAdd(&s_hist[run_bin], run_cnt);
     }
     __syncthreads();
@@ -235,20 +350,14 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_hist_kernel(SelArgs a, cs_
     }
     __syncthreads();
     const uint32_t b0 = s_b0;
-    const bool spec_ok = hint != 0xFFFFFFFFu && b0 != 0xFFFFFFFFu && b0 <= hint;
     const bool have_b0 = a.k && total >= a.k;
     const uint32_t ahead = have_b0 ? collect_ahead_limit<PER>(loc, threadIdx.x * PER, before, a.k, b0, &s_ahead) : 0u;
-    const uint32_t c_spec = __ldcg(&ws.sel->c_spec);
-    if (spec_ok)                                             // the shared histogram is free now: it holds the sample
-        publish_splitters(ws, (unsigned long long *)s_hist, s_hist + 2 * CS_SAMPLE, c_spec);
     if (threadIdx.x == 0) {
         ws.sel->b0 = b0;
         ws.sel->n_elig = total;
         ws.sel->n_out = total < a.k ? total : a.k;
         count_select(ws, a.kind, total, total < a.k ? total : a.k);
-        ws.sel->c = spec_ok ? c_spec : 0;
-        ws.sel->c_spec = 0;
-        ws.sel->spec = spec_ok ? 1u : 0u;
+        ws.sel->c = 0;
         remember_threshold(ws.sc, a.hint_slot, have_b0, ahead);
         ws.sel->ticket[1] = 0;
     }
@@ -404,7 +513,7 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_collect_kernel(SelArgs a, 
 
     // ---- last CTA: sample, sort the sample (bitonic, shared memory), publish splitters -----------
     publish_splitters(ws, s_km, s_id, __ldcg(&ws.sel->c));
-    if (threadIdx.x == 0) ws.sel->ticket[2] = 0;
+    if (threadIdx.x == 0) { ws.sel->ticket[2] = 0; count_candidates(ws, a.kind, __ldcg(&ws.sel->c), false); }
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -598,7 +707,7 @@ void cs_fill_sel_args(const cs_ctx *ctx, const cs_block_index *idx, uint32_t now
     a.use_age_limits = 0;
     a.hint_slot = 0;
     a.kind = 0;
-    a.now_dev = ctx->step_now_dev;
+    a.now_dev = ctx->step_now_dev ? ctx->step_now_dev : ctx->clock_dev;
 }
 
 uint32_t cs_scan_grid(const cs_ctx *ctx, uint32_t n, uint32_t per_cta, uint32_t ctas_per_sm)
@@ -663,6 +772,9 @@ static int launch_select_job(cs_ctx *ctx, int job, const cs_block_index *idx, ui
     const uint32_t grid_c = cs_scan_grid(ctx, idx->n_blocks, 256);
     const size_t sm = cs_table_smem(ctx);
     int rc;
+    if (prefetch) cs_launch_chained(cs_sel_fast_kernel<true>, grid, SEL_THREADS, sm, s, a, ws);
+    else cs_launch_chained(cs_sel_fast_kernel<false>, grid, SEL_THREADS, sm, s, a, ws);
+    if ((rc = cs_check_launch(ctx)) != CS_OK) return rc;
     if (prefetch) cs_launch_chained(cs_sel_hist_kernel<true>, grid, SEL_THREADS, sm, s, a, ws);
     else cs_launch_chained(cs_sel_hist_kernel<false>, grid, SEL_THREADS, sm, s, a, ws);
     if ((rc = cs_check_launch(ctx)) != CS_OK) return rc;

@@ -250,6 +250,7 @@ __device__ __forceinline__ void csel_body(SelArgs a, const cs_workspace &ws, uin
         cluster.sync();
     }
     const uint32_t c = __ldcg(cand_count);
+    if (ctid == 0) count_candidates(ws, a.kind, c, spec_ok);
 
     // ---- phase 4, small: ordered in shared memory ---------------------------------------------------------------
     if (c <= CSEL_SORT_MAX) {

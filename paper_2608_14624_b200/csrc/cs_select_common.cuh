@@ -74,6 +74,13 @@ __device__ __forceinline__ void count_select(const cs_workspace &ws, uint32_t ki
     ws.cnt->eligible[kind] = n_elig;
 }
 
+__device__ __forceinline__ void count_candidates(const cs_workspace &ws, uint32_t kind, uint32_t c, bool fast_hit)
+{
+    if (kind > 2) return;
+    ws.cnt->candidates[kind] = c;
+    if (fast_hit) atomicAdd((unsigned long long *)&ws.cnt->fast_hits[kind], 1ull);
+}
+
 // The clock of a call: by value, or from device memory when the caller asked for that.
 __device__ __forceinline__ void resolve_now(SelArgs &a)
 {
@@ -104,14 +111,66 @@ __device__ __forceinline__ void load_tables(const SelArgs &a, const cs_workspace
     T.a_star = (la < a.A) ? ws.amax[la] : 0xFFFFFFFFu;
 }
 
+// Recency factor of Eq. 9 for an age: from the table, the saturated constant, or (a decay so slow that the
+// table does not reach saturation) computed directly.
+__device__ __forceinline__ float recency_of_age(const SelArgs &a, const Tables &T, uint32_t age)
+{
+    if (age < a.gtab_len) return T.gtab[age];
+    if (age >= a.age_sat) return T.g_sat;
+    return cs_recency(a.lambda, a.delta, age);
+}
+
 __device__ __forceinline__ float score_from_age(const SelArgs &a, const Tables &T, uint32_t agent, uint32_t age,
                                                 uint32_t tok)
 {
-    float g;
-    if (age < a.gtab_len) g = T.gtab[age];
-    else if (age >= a.age_sat) g = T.g_sat;
-    else g = cs_recency(a.lambda, a.delta, age);
-    return __fmul_rn(__fmul_rn(T.fsurv[agent], g), (float)tok);      // two roundings, never an FMA
+    return __fmul_rn(__fmul_rn(T.fsurv[agent], recency_of_age(a, T, age)), (float)tok);      // two roundings, never an FMA
+}
+
+// ---------------------------------------------------------------------------------------------
+// Threshold test without the key.  The score is fl(fl(f * g) * |b|) and IEEE multiplication by a positive
+// constant never decreases when its operand grows, so "the first key digit is at most H" is, for a fixed
+// block size, an interval of x = fl(f * g): victims  x < X[|b|],  prefetch candidates  x >= X[class][|b|]
+// (class 0: blocks of a*, class 1: the rest).  X is found once per CTA by binary search over the bit
+// patterns of positive floats; an entry then costs two table look-ups, one multiply and one compare, and only
+// the few entries that pass get a key.  Exact: it is the same product the key is made of.
+// ---------------------------------------------------------------------------------------------
+#define XT_TOK 256u                // |b| is a u8
+#define XT_NONE 0x7F800001u        // above every finite pattern
+
+// smallest bit pattern x in [0, +inf] with bits(fl(x * tok)) >= lim; XT_NONE when there is none
+__device__ __forceinline__ uint32_t first_x_reaching(unsigned long long lim, uint32_t tok)
+{
+    uint32_t lo = 0, hi = 0x7F800001u;
+    const float t = (float)tok;
+    while (lo < hi) {
+        const uint32_t mid = lo + ((hi - lo) >> 1);
+        const unsigned long long bits = __float_as_uint(__fmul_rn(__uint_as_float(mid), t));
+        if (bits >= lim) hi = mid;
+        else lo = mid + 1;
+    }
+    return lo;
+}
+
+// Fills xt[2][XT_TOK] for the remembered bin H (every thread of the CTA calls; synchronise afterwards).
+template <bool PF>
+__device__ __forceinline__ void build_x_thresholds(const SelArgs &a, uint32_t H, uint32_t *xt)
+{
+    for (uint32_t e = threadIdx.x; e < 2 * XT_TOK; e += blockDim.x) {
+        const uint32_t cls = e / XT_TOK, tok = e % XT_TOK;
+        uint32_t x;
+        if (!PF) {
+            // bin = bits >> 20 (bits >> 19 with the copy-preference bit below the score): candidate <=> bits < lim
+            const unsigned long long lim = (unsigned long long)(H + 1u) << (a.prefer_copy ? 19 : 20);
+            x = first_x_reaching(lim, tok);                                  // candidate <=> x bits < this
+        } else if (cls == 0) {
+            // a*: bin = (0x7FFFFFFF - bits) >> 20 <= H  <=>  bits >= 0x80000000 - ((H + 1) << 20)
+            x = H >= 2047u ? 0u : first_x_reaching(0x80000000ull - ((unsigned long long)(H + 1u) << 20), tok);
+        } else {
+            // the rest: bin = 2048 + ((0x7FFFFFFF - bits) >> 20)
+            x = H < 2048u ? XT_NONE : (H >= 4095u ? 0u : first_x_reaching(0x80000000ull - ((unsigned long long)(H - 2047u) << 20), tok));
+        }
+        xt[e] = x;                                                           // prefetch: candidate <=> x bits >= this
+    }
 }
 
 __device__ __forceinline__ float score_of(const SelArgs &a, const Tables &T, uint32_t agent, uint32_t la,

@@ -226,3 +226,32 @@ def test_status_bits_set_between_two_reads_are_not_lost():
         side.synchronize()
         b = c.get_status()
         assert (a | b) == cs.CS_ST_TIMEOUT                            # seen exactly once or twice, never dropped
+
+
+def test_clock_read_from_device_memory_when_the_kernels_run():
+    """cs_set_device_clock: the select takes `now` from a device word at execution time (what a captured
+    CUDA graph needs), on both select paths, and goes back to its argument afterwards."""
+    cfg = synth.CONFIGS["llama8b"]
+    n, k = 40_000 + 3, 300
+    c, o, _ = warm(cfg, 800, n, r_min=0.02)
+    idx = synth.make_block_index(cfg, n=n)
+    d = cs.DeviceIndex.from_host(idx, DEV)
+    clock = torch.zeros(4, dtype=torch.int32, device=DEV)
+    c.set_device_clock(clock)
+    for path in (cs.CS_SELECT_CLUSTER, cs.CS_SELECT_MULTI):
+        c.set_select_path(path)
+        for now in (100_000, 100_777):
+            clock.fill_(now)
+            s64, s32 = o.scores(idx, now)
+            ids, cnt = c.select_victims(d, 5, 0, k)                       # the argument (5) is ignored
+            oi, on = o.select_victims(idx, now, 0, k, s32)
+            assert H.assert_list_matches(ids.cpu().numpy().view(np.uint32)[:k], int(cnt.item()), oi, on, s64) == 0
+            assert np.array_equal(c.score_blocks(d, 5).cpu().numpy(), s32)
+    c.set_device_clock(None)
+    s64, s32 = o.scores(idx, 100_100)
+    ids, cnt = c.select_victims(d, 100_100, 0, k)
+    oi, on = o.select_victims(idx, 100_100, 0, k, s32)
+    assert H.assert_list_matches(ids.cpu().numpy().view(np.uint32)[:k], int(cnt.item()), oi, on, s64) == 0
+    with pytest.raises(cs.CacheScoutError):
+        c.set_device_clock(torch.zeros(4, dtype=torch.int32))                # pageable host memory: refused
+    assert c.get_status() == 0

@@ -31,15 +31,17 @@ def block_bytes_from_pool(buf_u8, layout, n_slots, L, chunk, slot):
     return buf_u8.view(n_slots, L, 2, chunk)[slot].cpu().numpy()
 
 
-@pytest.mark.parametrize("transfers", ["exchange", "split"])
-def test_bench_step_at_full_size_matches_oracle(transfers):
+@pytest.mark.parametrize("cfg_name,transfers", [("llama8b", "exchange"), ("llama8b", "split"), ("llama70b", "exchange")])
+def test_bench_step_at_full_size_matches_oracle(cfg_name, transfers):
+    """The step exactly as bench.py times it (full-size GPU pool and index of the 8B- and the 70B-shaped
+    configuration, the bench's launch configuration), lists against the oracle and sampled blocks byte for byte."""
     import bench
     free = torch.cuda.mem_get_info()[0]
-    if free < 60 * (1 << 30) or bench.mem_available_bytes() < 60 * (1 << 30):
-        pytest.skip("needs 60 GiB of free device and host memory")
-    args = argparse.Namespace(quick=False, host_slots=8192, offload_width=0, prefetch_width=0, transfers=transfers,
-                              exchange_width=0)
-    w = bench.StepWorkload(args, torch.device(DEV), 1)
+    if free < 70 * (1 << 30) or bench.mem_available_bytes() < 60 * (1 << 30):
+        pytest.skip("needs 70 GiB of free device memory and 60 GiB of host memory")
+    args = argparse.Namespace(quick=False, host_slots=8192 if cfg_name == "llama8b" else 4096, host_frac=0.4, offload_width=0,
+                              prefetch_width=0, transfers=transfers, exchange_width=0)
+    w = bench.StepWorkload(args, torch.device(DEV), 1, cfg_name)
     cfg, G, L, chunk = w.cfg, w.cfg.gpu_blocks, w.cfg.n_layers, w.cfg.chunk_bytes
     o = orc.Oracle(H.oracle_params(w.params))
     o.observe(w.tr.chain[:2000], w.tr.agent[:2000], w.tr.evflags[:2000])
@@ -101,6 +103,9 @@ def test_bench_step_at_full_size_matches_oracle(transfers):
         idx.last_access[ov[:ovn].astype(np.int64)] = now
         idx.flags[op[:opn].astype(np.int64)] |= synth.FLAG_OTHER_COPY
     assert w.c.get_status() == 0
+    moved = w.take_moved_bytes()                           # the mover's own counters: every block of both steps
+    assert moved == 2 * (w.k_v + w.k_p) * cfg.block_bytes
+    w.release()
 
 
 def test_mover_70b_block_geometry():

@@ -297,6 +297,21 @@ def test_mover_offload_prefetch_compact(gpu_layout, host_layout, path):
     orc.move_blocks(got, gpu_layout, G, want_s, 1 - gpu_layout, n, L, chunk, s2, d2)
     assert np.array_equal(stage.buf.cpu().numpy(), want_s)
     assert c.get_status() == 0
+    if lay_h == synth.BLOCK_MAJOR:          # the copy-engine path needs contiguous host blocks
+        bb = L * 2 * chunk
+        c.set_mover_staging(torch.empty(4 * int(rng.integers(1, 6)) * bb + 512, dtype=torch.uint8, device=DEV))
+        m = int(rng.integers(1, 12))
+        gp2, hp2 = rng.permutation(G).astype(np.uint32), rng.permutation(Hs).astype(np.uint32)
+        o_src, p_dst = gp2[:m], gp2[m:2 * m]
+        o_dst, p_src = hp2[:m] + np.uint32(first_h), hp2[m:2 * m] + np.uint32(first_h)
+        host_before = host_t.numpy().copy()
+        c.exchange_blocks_staged(gpu, host, dev(o_src), o_dst, p_src, dev(p_dst))
+        torch.cuda.synchronize()
+        orc.move_blocks(want_g, lay_g, G, want_h, lay_h, Hs, L, chunk, o_src, unoff(o_dst))
+        want_g2 = want_g.copy()
+        orc.move_blocks(host_before, lay_h, Hs, want_g2, lay_g, G, L, chunk, unoff(p_src), p_dst)
+        assert np.array_equal(host_t.numpy(), want_h) and np.array_equal(gpu.buf.cpu().numpy(), want_g2)
+        assert c.get_status() == 0
 
     # an out-of-range slot is skipped and reported, nothing else is touched
     bad_src = src.copy()
@@ -387,6 +402,88 @@ def test_exchange_matches_offload_then_prefetch(gpu_layout, host_layout, n_off, 
     assert np.array_equal(host_t.numpy(), want_h)
     assert np.array_equal(gpu.buf.cpu().numpy(), want_g)
     assert c.get_status() == 0
+
+
+@pytest.mark.parametrize("gpu_layout", [0, 1])
+@pytest.mark.parametrize("n_off,n_pre,ring_blocks", [(41, 67, 3), (50, 0, 1), (0, 33, 2), (1, 1, 64), (37, 5, 7), (64, 64, 16)])
+def test_staged_exchange_matches_the_oracle(gpu_layout, n_off, n_pre, ring_blocks):
+    """The copy-engine path (pack -> cudaMemcpyAsync -> host, host -> cudaMemcpyAsync -> scatter) against the
+    oracle's two transfers: rings of 1 to 64 blocks per sub-buffer (many parts, double buffering, a ragged last
+    part), runs of consecutive host ids (merged copies) next to scattered ones, sentinels on either side."""
+    cfg = synth.CONFIGS["tiny"]
+    L, chunk, G, Hs, first_h = cfg.n_layers, cfg.chunk_bytes, 160, 200, 1000
+    bb = cfg.block_bytes
+    rng = synth.rng_for(cfg, 15 + ring_blocks)
+    c, _ = make_ctx(cfg, 64)
+    ring = torch.empty(4 * ring_blocks * bb + 256, dtype=torch.uint8, device=DEV)
+    c.set_mover_staging(ring)
+    gpu_np = synth.kv_pool_u16(G, L, chunk, rng).view(np.uint8)
+    host_np = synth.kv_pool_u16(Hs, L, chunk, rng).view(np.uint8)
+    gpu = cs.KVPool(dev(gpu_np), G, gpu_layout, L)
+    host_t = pinned_zeros(Hs * bb)
+    host_t.numpy()[:] = host_np
+    host = cs.KVPool(host_t, Hs, synth.BLOCK_MAJOR, L, first_id=first_h)
+    g_perm = rng.permutation(G).astype(np.uint32)
+    off_src, pre_dst = g_perm[:n_off].copy(), g_perm[n_off:n_off + n_pre].copy()
+    # host slots: the first half of each list is one run of consecutive slots, the rest scattered
+    h_free = rng.permutation(np.arange(Hs // 2, Hs)).astype(np.uint32)
+    run_o, run_p = n_off // 2, n_pre // 2
+    off_dst = np.concatenate([np.arange(run_o, dtype=np.uint32), h_free[:n_off - run_o]])
+    pre_src = np.concatenate([np.arange(run_o, run_o + run_p, dtype=np.uint32), h_free[n_off - run_o:n_off - run_o + n_pre - run_p]])
+    unspecified = []
+    if n_off > 8:
+        unspecified.append(int(off_dst[6]))
+        off_src[6] = orc.ID_NONE                                # skipped on the device: that host slot gets unspecified bytes
+    if n_pre > 8:
+        pre_dst[2] = orc.ID_NONE                                # skipped on the device
+    side = torch.cuda.Stream(device=DEV)
+    side.wait_stream(torch.cuda.current_stream())
+    ids = lambda a: np.where(a == orc.ID_NONE, a, a + np.uint32(first_h))
+    c.exchange_blocks_staged(gpu, host, dev(off_src) if n_off else None, ids(off_dst) if n_off else None,
+                             ids(pre_src) if n_pre else None, dev(pre_dst) if n_pre else None, stream=side)
+    side.synchronize()
+    want_h, want_g = host_np.copy(), gpu_np.copy()
+    orc.move_blocks(gpu_np, gpu_layout, G, want_h, synth.BLOCK_MAJOR, Hs, L, chunk, off_src, off_dst)
+    orc.move_blocks(host_np, synth.BLOCK_MAJOR, Hs, want_g, gpu_layout, G, L, chunk, pre_src, pre_dst)
+    got_h = host_t.numpy().copy()
+    for slot in unspecified:
+        got_h[slot * bb:(slot + 1) * bb] = want_h[slot * bb:(slot + 1) * bb]
+    assert np.array_equal(got_h, want_h)
+    assert np.array_equal(gpu.buf.cpu().numpy(), want_g)
+    cn = c.counters()
+    assert cn["blocks_moved"][1] == np.count_nonzero(off_src != orc.ID_NONE)
+    assert cn["blocks_moved"][2] == np.count_nonzero(pre_dst != orc.ID_NONE)
+    assert c.get_status() == 0
+    # a second transfer right behind the first on the same stream reuses the ring safely: move everything back
+    if n_off and n_pre == 0:
+        keep = np.ones(n_off, bool)
+        back = off_src
+        cs.cs_prefetch_blocks_staged(c.ctx, host.struct(), gpu.struct(), ids(off_dst[keep]), dev(back[keep]),
+                                     int(keep.sum()), stream=side)
+        side.synchronize()
+        ok = keep & (off_src != orc.ID_NONE)
+        assert np.array_equal(H.pool_view(gpu.buf.cpu().numpy(), gpu_layout, G, L, chunk)[off_src[ok]],
+                              H.pool_view(gpu_np, gpu_layout, G, L, chunk)[off_src[ok]])
+    # errors: no ring, host ids out of range, a layer-major host pool
+    with pytest.raises(cs.CacheScoutError) as e:
+        c.exchange_blocks_staged(gpu, host, dev(g_perm[:1]), np.array([first_h + Hs], np.uint32), None, None)
+    assert e.value.code == cs.CS_EINVAL
+    with pytest.raises(cs.CacheScoutError) as e:             # a sentinel in a host list: the device could not know of the skip
+        c.exchange_blocks_staged(gpu, host, dev(g_perm[:1]), np.array([orc.ID_NONE], np.uint32), None, None)
+    assert e.value.code == cs.CS_EINVAL
+    bad_host = cs.KVPool(host_t, Hs, synth.LAYER_MAJOR, L, first_id=first_h)
+    with pytest.raises(cs.CacheScoutError) as e:
+        c.exchange_blocks_staged(gpu, bad_host, dev(g_perm[:1]), np.array([first_h], np.uint32), None, None)
+    assert e.value.code == cs.CS_EINVAL
+    c.set_mover_staging(None)
+    with pytest.raises(cs.CacheScoutError) as e:
+        c.exchange_blocks_staged(gpu, host, dev(g_perm[:1]), np.array([first_h], np.uint32), None, None)
+    assert e.value.code == cs.CS_EINVAL
+    tiny_ring = torch.empty(2 * bb, dtype=torch.uint8, device=DEV)          # less than four blocks
+    c.set_mover_staging(tiny_ring)
+    with pytest.raises(cs.CacheScoutError) as e:
+        c.exchange_blocks_staged(gpu, host, dev(g_perm[:1]), np.array([first_h], np.uint32), None, None)
+    assert e.value.code == cs.CS_ECAPACITY
 
 
 def test_offload_straight_from_select_output():
@@ -603,7 +700,7 @@ def test_select_step_matches_three_calls_and_oracle(name, n, kv, kp, path):
             g = got.cpu().numpy().view(np.uint32)[:k]
             assert H.assert_list_matches(g, int(got_n[0].item()), o_ids, o_n, s64) == 0, (rep, k)
     fused = path == cs.CS_SELECT_AUTO and n <= 262144
-    assert c.launch_count() - l0 == (3 if fused else 3 * 3 * 5)
+    assert c.launch_count() - l0 == (3 if fused else 3 * 3 * 6)
     # a select whose count pointer is NULL is left out
     gh.fill_(7)
     ghn.fill_(7)
@@ -754,3 +851,18 @@ def test_random_mover_geometries(case):
     orc.move_blocks(want_g, lay_g, G, want_s, 1 - lay_g, n, L, chunk, back, np.arange(n))
     assert np.array_equal(stage.buf.cpu().numpy(), want_s)
     assert c.get_status() == 0
+    if lay_h == synth.BLOCK_MAJOR:          # the copy-engine path needs contiguous host blocks
+        bb = L * 2 * chunk
+        c.set_mover_staging(torch.empty(4 * int(rng.integers(1, 6)) * bb + 512, dtype=torch.uint8, device=DEV))
+        m = int(rng.integers(1, 12))
+        gp2, hp2 = rng.permutation(G).astype(np.uint32), rng.permutation(Hs).astype(np.uint32)
+        o_src, p_dst = gp2[:m], gp2[m:2 * m]
+        o_dst, p_src = hp2[:m] + np.uint32(first_h), hp2[m:2 * m] + np.uint32(first_h)
+        host_before = host_t.numpy().copy()
+        c.exchange_blocks_staged(gpu, host, dev(o_src), o_dst, p_src, dev(p_dst))
+        torch.cuda.synchronize()
+        orc.move_blocks(want_g, lay_g, G, want_h, lay_h, Hs, L, chunk, o_src, unoff(o_dst))
+        want_g2 = want_g.copy()
+        orc.move_blocks(host_before, lay_h, Hs, want_g2, lay_g, G, L, chunk, unoff(p_src), p_dst)
+        assert np.array_equal(host_t.numpy(), want_h) and np.array_equal(gpu.buf.cpu().numpy(), want_g2)
+        assert c.get_status() == 0
