@@ -51,8 +51,10 @@ def parse_args():
     ap.add_argument("--no-extras", action="store_true", help="skip the mover sweep and the metadata-scale section")
     ap.add_argument("--offload-width", type=int, default=0, help="warp pipelines of the offload mover (0 = library default)")
     ap.add_argument("--prefetch-width", type=int, default=0, help="warp pipelines of the prefetch mover (0 = library default)")
-    ap.add_argument("--transfers", default="exchange", choices=["exchange", "split"],
-                    help="offload and prefetch of a step as one fused launch (exchange) or as two launches on two streams (split)")
+    ap.add_argument("--transfers", default="exchange", choices=["exchange", "split", "staged"],
+                    help="offload and prefetch of a step as one fused SM-issued launch (exchange), as two launches on two streams "
+                         "(split), or on the copy engines through a device ring after reading the id lists back (staged)")
+    ap.add_argument("--ring-mib", type=int, default=256, help="device ring of the staged transfers, MiB")
     ap.add_argument("--selects", default="fused", choices=["fused", "separate"],
                     help="the three selects of a step as one launch (cs_select_step) or as three calls")
     ap.add_argument("--exchange-width", type=int, default=0, help="warp pipelines of the fused transfer (0 = library default)")
@@ -255,7 +257,12 @@ class StepWorkload:
         self.done_p = [None] * self.RING
         self.now0 = 100_000
         self.w_off, self.w_pre = args.offload_width, args.prefetch_width
-        self.fused, self.w_ex = args.transfers == "exchange", args.exchange_width
+        self.fused, self.w_ex = args.transfers in ("exchange", "staged"), args.exchange_width
+        self.staged = args.transfers == "staged"
+        if self.staged:
+            self.ring = torch.empty(max(getattr(args, "ring_mib", 256), 4 * bb >> 20) << 20, dtype=torch.uint8, device=device)
+            self.c.set_mover_staging(self.ring)
+            self.dst_host = [free0.cpu().numpy().view(np.uint32).copy() for _ in range(self.RING)]
         self.fused_selects = getattr(args, "selects", "fused") == "fused"
         self.fifo = [torch.zeros(self.k_p, dtype=torch.int64, device=device) for _ in range(8)]
         self.fifo_used = 0
@@ -308,7 +315,36 @@ class StepWorkload:
         rec(t[3], main)
         ready = torch.cuda.Event()
         ready.record(main)
-        if self.fused:
+        if self.staged:
+            # copy-engine path: the host must know the host-tier slots, so the three lists and counts are read back
+            # (a few KB and one host synchronisation per step), conflicts are dropped on the host (a candidate whose
+            # host slot receives an offloaded block in this step), and the transfers are issued with host id lists
+            r, kv, kp = self.res_pin, self.k_v, self.k_p
+            r[:kv].copy_(vict, non_blocking=True)
+            r[kv:2 * kv].copy_(self.hv[b][:kv], non_blocking=True)
+            r[2 * kv:2 * kv + kp].copy_(self.pf[b][:kp], non_blocking=True)
+            r[-16:-15].copy_(self.vn[b][:1], non_blocking=True)
+            r[-15:-14].copy_(self.hn[b][:1], non_blocking=True)
+            r[-14:-13].copy_(self.pn[b][:1], non_blocking=True)
+            main.synchronize()
+            rv = r.numpy().view(np.uint32)
+            n_off, n_pre = int(min(rv[-16], rv[-15])), int(rv[-14])
+            off_host, pre_host = rv[kv:kv + n_off].copy(), rv[2 * kv:2 * kv + n_pre].copy()
+            keep = ~np.isin(pre_host, off_host)
+            pre_gpu = self.dst[prev]
+            if not keep.all():
+                pre_host = pre_host[keep]
+                pre_gpu = torch.from_numpy(self.dst_host[prev][:n_pre][keep].view(np.int32)).to(self.dev)
+            self.dst_host[b][:kv] = rv[:kv]
+            self.side_o.wait_event(ready)
+            rec(t[4], self.side_o)
+            c.exchange_blocks_staged(self.gpu_pool, self.host_pool, vict[:n_off], off_host, pre_host, pre_gpu, stream=self.side_o)
+            rec(t[5], self.side_o)
+            self.done_o[b] = torch.cuda.Event()
+            self.done_o[b].record(self.side_o)
+            self.done_p[b] = self.done_o[b]
+            t[6], t[7] = t[4], t[5]
+        elif self.fused:
             # one launch on side stream 1: GPU victims -> the slots of the host-tier victims, and the prefetch
             # candidates -> the slots freed one step earlier (their offload ran in the previous launch of this stream)
             self.side_o.wait_event(ready)
@@ -607,8 +643,68 @@ def fused_step_section(w, steps=10):
         "transfer_alone_ms": x8, "serving_with_transfer_ms": both8, "serving_slowdown": both8 / alone_small,
         "serving_slowdown_while_transfer_in_flight": in_flight_factor(alone_small, both8, x8_both),
         "transfer_with_serving_ms": x8_both, "transfer_slowdown": x8_both / x8}
+    # ---- the same 256 out + 384 in through three forms of transfer: what each gives the link and what it costs the
+    #      kernels running beside it (a graph-replayed chain of small kernels, this library's own fused select, and the
+    #      in-step compaction) ------------------------------------------------------------------------------------
+    r_np = lambda t, n: t[:n].cpu().numpy().view(np.uint32).copy()
+    n_off, n_pre = int(min(gvn[0].item(), ghn[0].item())), int(gpn[0].item())
+    off_host, pre_host = r_np(gh, n_off), r_np(gp, n_pre)
+    keep = (pre_host != 0xFFFFFFFF) & ~np.isin(pre_host, off_host)
+    pre_host_k = pre_host[keep]
+    pre_gpu_k = torch.from_numpy(r_np(free_last, n_pre)[keep].view(np.int32)).to(dev)
+    ring = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    c.set_mover_staging(ring)
+    sv, sh, sp, svn, shn, spn = i32(kv), i32(kv), i32(kp), i32(1), i32(1), i32(1)
+    now_sel = w.now0 + state["s"]
+
+    def staged():
+        c.exchange_blocks_staged(w.gpu_pool, w.host_pool, gv[:n_off], off_host, pre_host_k, pre_gpu_k, stream=side)
+
+    def beside(op, reps, disturber):
+        """Per-call time of `reps` back-to-back calls of op on the main stream while the disturber runs on the side stream."""
+        best, x_ms = None, 0.0
+        for _ in range(3):
+            torch.cuda.synchronize(dev)
+            m0, e0, e1, s0, s1 = (torch.cuda.Event(enable_timing=True) for _ in range(5))
+            m0.record(main)
+            side.wait_event(m0)
+            s0.record(side)
+            if disturber is not None:
+                disturber()
+            s1.record(side)
+            with torch.cuda.stream(main):
+                e0.record(main)
+                for _ in range(reps):
+                    op()
+                e1.record(main)
+            torch.cuda.synchronize(dev)
+            t = e0.elapsed_time(e1) / reps
+            if best is None or t < best:
+                best, x_ms = t, s0.elapsed_time(s1)
+        return best, x_ms
+
+    sel_op = lambda: c.select_step(w.didx, now_sel, kv, kp, sv, svn, sh, shn, sp, spn, stream=main)
+    cmp_op = lambda: c.compact_blocks(w.gpu_pool, w.stage_pool, gv, w.packed, n_max=kv, n_dev=gvn, stream=main)
+    sel_alone, _ = beside(sel_op, 20, None)
+    cmp_alone, _ = beside(cmp_op, 10, None)
+    variants = []
+    for name, width, fn in (("sm_direct_width_32", 0, transfer), ("sm_direct_width_8", 8, transfer), ("staged_copy_engines", 0, staged)):
+        c.set_mover_ctas(width, 0)
+        _, x_alone_ms = beside(lambda: None, 1, fn)
+        g_ms, g_x = run_graph(fn)
+        sel_ms, _ = beside(sel_op, 20, fn)
+        cmp_ms, _ = beside(cmp_op, 10, fn)
+        moved = (n_off + (len(pre_host_k) if fn is staged else n_pre)) * bb
+        variants.append({"transfer": name, "transfer_alone_ms": x_alone_ms, "link_GBps": moved / x_alone_ms / 1e6,
+                         "graph_chain_slowdown_while_in_flight": in_flight_factor(g_alone, g_ms, g_x),
+                         "fused_select_ms_alone": sel_alone, "fused_select_ms_beside": sel_ms, "fused_select_slowdown": sel_ms / sel_alone,
+                         "compaction_ms_alone": cmp_alone, "compaction_ms_beside": cmp_ms,
+                         "compaction_GBps_beside": 2 * kv * bb / cmp_ms / 1e6, "compaction_slowdown": cmp_ms / cmp_alone})
+    c.set_mover_ctas(0, 0)
+    c.set_mover_staging(None)
+    inter["transfer_variants"] = variants
     out["interference"] = inter
-    del x, y, a, b, o, small
+    del x, y, a, b, o, small, ring
     return out
 
 
