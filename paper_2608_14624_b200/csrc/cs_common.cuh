@@ -18,6 +18,7 @@
 #define CS_MOVE_D2D 0
 #define CS_MOVE_OFFLOAD 1
 #define CS_MOVE_PREFETCH 2
+#define CS_MOVE_STAGE 3            // pack / scatter launch of the copy-engine path: inside the device, deliberately narrow
 
 #define CS_HIST_BINS 4096u        // first radix digit of the select: top 12 bits of the primary key
 #define CS_MAX_SPLITTERS 255u     // bucket sort of the candidates: up to 256 buckets
@@ -120,6 +121,7 @@ struct cs_ctx {
     unsigned char *stage_ring;
     size_t stage_bytes;
     cudaStream_t copy_stream[2];         // 0: device -> host, 1: host -> device
+    cudaStream_t scatter_stream;         // scatter launches of staged prefetches
     cudaEvent_t ev_stage_fork, ev_stage_join[2];
     cudaEvent_t ev_packed[2], ev_copied[2], ev_filled[2], ev_scattered[2];
     uint64_t n_launches;

@@ -352,6 +352,15 @@ static void fill_mover_args(cs_ctx *ctx, MoverArgs &a, const cs_kv_pool *src, co
     a.block_bytes = 2ull * a.L * a.chunk;
 }
 
+// Shape of a bulk launch.  Narrow transfers (every host-link transfer: at most a few dozen pipelines) run one
+// pipeline per CTA with a 48 KiB ring, which fits the SMs' default shared-memory split; only wide device-to-device
+// moves pack four pipelines (192 KiB) into a CTA.  A launch that needs the large split costs ~8 us more before
+// its first copy is issued, which is most of what a one-block transfer loses against a plain memcpy.
+static uint32_t bulk_warps_per_cta(uint32_t n_pipes)
+{
+    return n_pipes <= 64u ? 1u : TM_WARPS;
+}
+
 // Shared-memory opt-in of the bulk kernels: an attribute of the function on a device, so it is set once per
 // process and device (always to the same fixed size).
 static std::mutex g_bulk_mu;
@@ -389,19 +398,23 @@ int cs_launch_mover_as(cs_ctx *ctx, const cs_kv_pool *src, const cs_kv_pool *dst
     unsigned long long cap;
     if (bulk) {
         // width in warp pipelines (each keeps <= 2 loads and 2 stores of 16 KiB in flight)
-        const uint32_t dflt = kind == CS_MOVE_D2D ? 2u * (uint32_t)ctx->sm_count : (kind == CS_MOVE_OFFLOAD ? 8u : 24u);
-        const uint32_t asked = kind == CS_MOVE_D2D ? ctx->d2d_ctas : ctx->host_link_ctas;
+        // (a pack / scatter launch of the copy-engine path only has to keep ahead of the host link: 64 pipelines move
+        //  about 1.5 TB/s and leave most SMs to the kernels running beside it)
+        const uint32_t dflt = kind == CS_MOVE_D2D ? 2u * (uint32_t)ctx->sm_count
+                            : (kind == CS_MOVE_STAGE ? 64u : (kind == CS_MOVE_OFFLOAD ? 8u : 24u));
+        const uint32_t asked = kind == CS_MOVE_D2D ? ctx->d2d_ctas : (kind == CS_MOVE_STAGE ? 0u : ctx->host_link_ctas);
         cap = asked ? asked : dflt;
         a.n_pipes = (uint32_t)(total < cap ? total : cap);
         if (a.n_pipes == 0) a.n_pipes = 1;
-        const uint32_t wpc = a.n_pipes < TM_WARPS ? a.n_pipes : TM_WARPS;
+        const uint32_t wpc = bulk_warps_per_cta(a.n_pipes);
         const uint32_t grid = (a.n_pipes + wpc - 1) / wpc;
         const int rc = bulk_opt_in(ctx);
         if (rc != CS_OK) return rc;
-        cs_mover_bulk_kernel<<<grid, wpc * 32, TM_SMEM, s>>>(a);
+        cs_mover_bulk_kernel<<<grid, wpc * 32, (size_t)wpc * TM_STAGES * TM_PIECE, s>>>(a);
     } else {
-        const uint32_t dflt = kind == CS_MOVE_D2D ? 8u * (uint32_t)ctx->sm_count : (kind == CS_MOVE_OFFLOAD ? 8u : 12u);
-        const uint32_t asked = kind == CS_MOVE_D2D ? ctx->d2d_ctas : ctx->host_link_ctas;
+        const uint32_t dflt = kind == CS_MOVE_D2D ? 8u * (uint32_t)ctx->sm_count
+                            : (kind == CS_MOVE_STAGE ? 64u : (kind == CS_MOVE_OFFLOAD ? 8u : 12u));
+        const uint32_t asked = kind == CS_MOVE_D2D ? ctx->d2d_ctas : (kind == CS_MOVE_STAGE ? 0u : ctx->host_link_ctas);
         cap = asked ? asked : dflt;
         const uint32_t grid = (uint32_t)(total < cap ? total : cap);
         cs_mover_kernel<<<grid ? grid : 1u, MV_THREADS, 0, s>>>(a);
@@ -423,11 +436,11 @@ int cs_launch_exchange(cs_ctx *ctx, const cs_kv_pool *gpu, const cs_kv_pool *hos
     uint32_t n_pipes = (uint32_t)(total < cap ? total : cap);
     if (n_pipes == 0) n_pipes = 1;
     off.n_pipes = pre.n_pipes = n_pipes;
-    const uint32_t wpc = n_pipes < TM_WARPS ? n_pipes : TM_WARPS;
+    const uint32_t wpc = bulk_warps_per_cta(n_pipes);
     const uint32_t grid = (n_pipes + wpc - 1) / wpc;
     const int rc = bulk_opt_in(ctx);
     if (rc != CS_OK) return rc;
-    cs_exchange_bulk_kernel<<<grid, wpc * 32, TM_SMEM, s>>>(off, pre);
+    cs_exchange_bulk_kernel<<<grid, wpc * 32, (size_t)wpc * TM_STAGES * TM_PIECE, s>>>(off, pre);
     return cs_check_launch(ctx);
 }
 

@@ -105,23 +105,43 @@ __device__ __forceinline__ void publish_splitters(const cs_workspace &ws, unsign
 //
 // The threshold bin moves little from one call to the next, so each kind of call (GPU victims, host
 // victims, prefetch) remembers a bin H at or a little above the one it ended with.  With H known, almost
-// every eligible entry can be dismissed without its key: it lies above H exactly when x = fl(f * g) is on
-// the far side of a per-size threshold (build_x_thresholds), which costs two look-ups, a multiply and a
-// compare.  Those entries are only counted.  The few at or below H get their key, an exact histogram bin
-// and a place in the candidate buffer.  The last CTA then has the exact histogram of bins <= H plus the
-// number of entries above: if the k-th smallest key lies within H the candidates are complete, the
-// sample sort is set up right here and the index has been read ONCE, at a fraction of the instructions of
-// a full-key scan.  Otherwise (the threshold rose above H, or nothing is remembered yet) the pass reports
-// a miss and the full histogram and collect passes below run.  The result never depends on H.
+// every eligible entry can be dismissed without its key, in two steps:
+//   a  by age alone.  For victims (low scores = old blocks) an entry younger than a cut A_c cannot reach
+//      H whatever its agent and size: fl(f_min * g(age)) is already on the far side of the largest per-size
+//      threshold X (build_x_thresholds), g never increases with age, and IEEE products are monotone.  That is
+//      ONE integer compare on last_access per entry.  For prefetch candidates (high scores = young blocks)
+//      the same holds with the roles swapped, for entries of agents other than a*.
+//   b  what is left (a few per cent) is queued per warp as entry ids and worked off with all 32 lanes
+//      busy: two table look-ups, one multiply and one compare against X decide exactly whether the entry's
+//      first key digit is <= H; only then is the key built, binned and appended to the candidate buffer.
+// Dismissed entries are only counted.  The last CTA has the exact histogram of bins <= H plus the number
+// of entries above: if the k-th smallest key lies within H the candidates are complete, the sample sort is
+// set up right here, and the index has been read ONCE at a fraction of the instructions of a full-key
+// scan.  Otherwise (the threshold rose above H, or nothing is remembered yet) the pass reports a miss and
+// the full histogram and collect passes below run.  The result never depends on H.
 // ---------------------------------------------------------------------------------------------
+#define FQ_CAP 544u                 // per-warp queue: at most 31 left over + the 512 entries of one warp tile
+
+__device__ __forceinline__ uint32_t nibble_of_byte_flags(uint32_t ok)      // 0xFF / 0x00 per byte -> 4 bits
+{
+    return (((((ok >> 7) & 0x01010101u) * 0x01020408u) >> 24) & 0xFu);
+}
+
+// Largest value of every 16-bit half over eight packed words.
+__device__ __forceinline__ uint32_t max_halves(const uint4 &a, const uint4 &b)
+{
+    const uint32_t m0 = __vmaxu2(__vmaxu2(a.x, a.y), __vmaxu2(a.z, a.w)), m1 = __vmaxu2(__vmaxu2(b.x, b.y), __vmaxu2(b.z, b.w));
+    const uint32_t m = __vmaxu2(m0, m1);
+    return max(m & 0xFFFFu, m >> 16);
+}
+
 template <bool PF>
 __global__ void __launch_bounds__(SEL_THREADS) cs_sel_fast_kernel(SelArgs a, cs_workspace ws)
 {
-    extern __shared__ float smem[];
-    __shared__ __align__(16) uint32_t s_hist[CS_HIST_BINS];
+    extern __shared__ float smem[];                 // tables, then the per-warp queues (reused by the epilogue)
     __shared__ uint32_t s_xt[2 * XT_TOK];
     __shared__ uint32_t s_part[SEL_THREADS];
-    __shared__ uint32_t s_b0, s_ahead, s_above;
+    __shared__ uint32_t s_b0, s_ahead, s_above, s_fbits, s_xext;
     __shared__ bool s_flag;
     cs_wait_for_predecessor();
     cs_release_successor();
@@ -133,65 +153,184 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_fast_kernel(SelArgs a, cs_
     resolve_now(a);
     Tables T;
     load_tables(a, ws, smem, T, PF && a.anchor);
+    const size_t table_words = ((size_t)(a.A + a.gtab_len) * 4 + (size_t)a.A * 2 + 15) / 16 * 4;
+    uint32_t *queues = (uint32_t *)smem + table_words;
     build_x_thresholds<PF>(a, H, s_xt);
-    for (uint32_t i = threadIdx.x; i < CS_HIST_BINS; i += blockDim.x) s_hist[i] = 0;
-    if (threadIdx.x == 0) s_above = 0;
+    if (threadIdx.x == 0) { s_above = 0; s_fbits = PF ? 0u : 0x7F800000u; s_xext = PF ? 0xFFFFFFFFu : 0u; }
     __syncthreads();
-    const uint32_t lane = threadIdx.x & 31;
+    // ---- the age cut -------------------------------------------------------------------------------------
+    // victims: f_min over the agents and the largest X over the sizes in range; prefetch: f_max and the smallest X
+    // of the agents other than a*.  (fsurv is positive, so floats order like their bit patterns.)
+    const uint32_t tok_lo = a.ntok ? 1u : a.block_tokens, tok_hi = a.block_tokens;
+    {
+        uint32_t fb = PF ? 0u : 0x7F800000u, xe = PF ? 0xFFFFFFFFu : 0u;
+        for (uint32_t i = threadIdx.x; i < a.A; i += blockDim.x) {
+            const uint32_t b = __float_as_uint(T.fsurv[i]);
+            fb = PF ? max(fb, b) : min(fb, b);
+        }
+        for (uint32_t t = tok_lo + threadIdx.x; t <= tok_hi; t += blockDim.x) {
+            const uint32_t x = s_xt[(PF ? XT_TOK : 0u) + t];
+            xe = PF ? min(xe, x) : max(xe, x);
+        }
+        if (PF) { atomicMax(&s_fbits, fb); atomicMin(&s_xext, xe); }
+        else { atomicMin(&s_fbits, fb); atomicMax(&s_xext, xe); }
+    }
+    __syncthreads();
+    bool have_cut = false;
+    uint32_t la_cut = 0;
+    if (ws.sc->gtab_monotone && a.gtab_len == a.age_sat) {
+        const float f_ext = __uint_as_float(s_fbits);
+        const uint32_t x_ext = s_xext;
+        // dismissed(age): victims  fl(f_min g) >= X_max (true for young ages);  prefetch  fl(f_max g) < X_min (true for old ages)
+        auto dismissed = [&](uint32_t age) {
+            const uint32_t xb = __float_as_uint(__fmul_rn(f_ext, recency_of_age(a, T, age)));
+            return PF ? (xb < x_ext) : (xb >= x_ext);
+        };
+        if (!PF) {
+            if (x_ext != XT_NONE && dismissed(0)) {                 // largest age that is still dismissed
+                uint32_t lo = 0, hi = a.age_sat;
+                while (lo < hi) {
+                    const uint32_t mid = lo + ((hi - lo + 1) >> 1);
+                    if (dismissed(mid)) lo = mid;
+                    else hi = mid - 1;
+                }
+                have_cut = true;                                    // young <=> age <= lo <=> last_access >= now - lo
+                la_cut = (lo >= a.age_sat || lo >= a.now) ? 0u : a.now - lo;
+            }
+        } else {
+            if (x_ext == XT_NONE) { have_cut = true; la_cut = 0xFFFFFFFFu; }      // no entry of another agent can qualify
+            else if (dismissed(a.age_sat)) {                        // smallest age that is dismissed
+                uint32_t lo = 0, hi = a.age_sat;
+                while (lo < hi) {
+                    const uint32_t mid = lo + ((hi - lo) >> 1);
+                    if (dismissed(mid)) hi = mid;
+                    else lo = mid + 1;
+                }
+                if (lo == 0) { have_cut = true; la_cut = 0xFFFFFFFFu; }
+                else if (lo <= a.now) { have_cut = true; la_cut = a.now - lo; }   // old <=> age >= lo <=> last_access <= now - lo
+            }
+        }
+    }
+    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint32_t *q = queues + warp * FQ_CAP;
+    uint32_t qn = 0;                                           // queued ids of this warp (same value in every lane)
     uint32_t n_above = 0;
-    if (!PF || prefetch_enabled(ws, a.A)) {
-        const uint32_t gtid = blockIdx.x * blockDim.x + threadIdx.x, nth = gridDim.x * blockDim.x;
-        const uint32_t n_tiles = a.n / TILE, n_warps = nth >> 5;
-        const uint32_t n_iter = (n_tiles + n_warps - 1) / n_warps;     // whole warps stay in the shuffles
-        for (uint32_t it = 0; it < n_iter; ++it) {
-            const uint32_t t = it * n_warps + (gtid >> 5);
-            uint32_t mask = 0;
-            Group G;
-            if (t < n_tiles) {
-                load_group<PF>(a, t, lane, G);
-                const uint32_t em = group_elig<PF>(a, G);
-#pragma unroll
-                for (int j = 0; j < GRP; ++j) {
-                    if (!((em >> j) & 1u)) continue;
-                    const uint32_t ag = grp_u16(G.ag0, G.ag1, j);
-                    if (ag >= a.A) { atomicOr(&ws.sc->status, CS_ST_BAD_AGENT); continue; }
-                    if (PF && a.anchor && !(grp_u16(G.dp0, G.dp1, j) < T.anchor[ag])) continue;
-                    const uint32_t tok = a.ntok ? grp_u8(G.tk, j) : a.block_tokens;
-                    const uint32_t la = grp_u32(G, j);
+    const bool enabled = !PF || prefetch_enabled(ws, a.A);
+
+    // Works off whole rounds of 32 queued entries (all of them when `all`), every lane busy.
+    auto drain = [&](bool all) {
+        const uint32_t rounds = all ? (qn + 31u) / 32u : qn / 32u;
+        for (uint32_t r = 0; r < rounds; ++r) {
+            const uint32_t i = r * 32u + lane;
+            bool cand = false;
+            uint32_t id = 0, ag = 0, la = 0, tok = a.block_tokens, dp = 0;
+            if (i < qn) {
+                id = q[i];
+                ag = __ldg(a.agent + id);
+                la = __ldg(a.la + id);
+                if (a.ntok) tok = __ldg(a.ntok + id);
+                if (PF && a.anchor) dp = __ldg(a.depth + id);
+                bool elig = true;
+                if (ag >= a.A) { atomicOr(&ws.sc->status, CS_ST_BAD_AGENT); elig = false; }
+                else if (PF && a.anchor && !(dp < T.anchor[ag])) elig = false;
+                if (elig) {
                     const uint32_t age = la <= a.now ? a.now - la : 0u;
                     const uint32_t xb = __float_as_uint(__fmul_rn(T.fsurv[ag], recency_of_age(a, T, age)));
                     const uint32_t X = s_xt[((PF && ag != T.a_star) ? XT_TOK : 0u) + tok];
-                    const bool cand = PF ? (xb >= X) : (xb < X);
-                    if (cand) mask |= 1u << j;
-                    else ++n_above;
+                    cand = PF ? (xb >= X) : (xb < X);
+                    if (!cand) ++n_above;
                 }
             }
-            if (!__any_sync(0xFFFFFFFFu, mask != 0)) continue;      // most warps hold no candidate at all
-            const uint32_t cnt = __popc(mask);
+            const uint32_t bal = __ballot_sync(0xFFFFFFFFu, cand);
+            if (bal == 0) continue;
+            uint32_t base = 0;
+            if (lane == 0) base = atomicAdd(&ws.sel->c_spec, (uint32_t)__popc(bal));
+            base = __shfl_sync(0xFFFFFFFFu, base, 0);
+            if (cand) {
+                uint32_t pr, se;
+                entry_key_rest<PF>(a, T, &ws.sc->status, ag, dp, __ldg(a.flags + id), la, tok, pr, se);
+                atomicAdd(&ws.hist[pr >> 20], 1u);                  // few entries get here: straight into the global histogram
+                const uint32_t pos = base + __popc(bal & ((1u << lane) - 1u));
+                ws.cand_km[pos] = ((unsigned long long)pr << 32) | se;
+                ws.cand_id[pos] = id;
+            }
+        }
+        if (!all) {
+            const uint32_t done = rounds * 32u, left = qn - done;        // < 32
+            __syncwarp();
+            const uint32_t v = lane < left ? q[done + lane] : 0u;
+            __syncwarp();
+            if (lane < left) q[lane] = v;
+            __syncwarp();
+            qn = left;
+        } else {
+            qn = 0;
+        }
+    };
+
+    if (enabled) {
+        const uint32_t gtid = blockIdx.x * blockDim.x + threadIdx.x, nth = gridDim.x * blockDim.x;
+        const uint32_t n_tiles = a.n / TILE, n_warps = nth >> 5;
+        const uint32_t n_iter = (n_tiles + n_warps - 1) / n_warps;     // whole warps stay in the shuffles
+        const uint32_t tok_span = tok_hi - tok_lo + 1u;
+        for (uint32_t it = 0; it < n_iter; ++it) {
+            const uint32_t t = it * n_warps + (gtid >> 5);
+            uint32_t rem = 0;                                          // entries that need the exact test
+            if (t < n_tiles) {
+                Group G;
+                load_group<PF>(a, t, lane, G);
+                const uint32_t em = group_elig<PF>(a, G);
+                if (!PF) {
+                    uint32_t dm = 0;                                   // dismissed by age (and safe to dismiss)
+                    if (have_cut && max_halves(G.ag0, G.ag1) < a.A) {
+#pragma unroll
+                        for (int j = 0; j < GRP; ++j) dm |= (grp_u32(G, j) >= la_cut ? 1u : 0u) << j;
+                        if (a.ntok) {                                  // sizes outside [1, block_tokens] take the exact test
+                            uint32_t in = 0;
+#pragma unroll
+                            for (int w = 0; w < 4; ++w) {
+                                const uint32_t x = __vsub4(u4_word(G.tk, w), 0x01010101u * tok_lo);
+                                in |= nibble_of_byte_flags(__vcmpltu4(x, 0x01010101u * tok_span)) << (4 * w);
+                            }
+                            dm &= in;
+                        }
+                    }
+                    n_above += __popc(em & dm);
+                    rem = em & ~dm;
+                } else {
+#pragma unroll
+                    for (int j = 0; j < GRP; ++j) {
+                        if (!((em >> j) & 1u)) continue;
+                        const uint32_t ag = grp_u16(G.ag0, G.ag1, j);
+                        const uint32_t tok = a.ntok ? grp_u8(G.tk, j) : a.block_tokens;
+                        if (!have_cut || ag >= a.A || ag == T.a_star || tok - tok_lo >= tok_span) { rem |= 1u << j; continue; }
+                        if (a.anchor && !(grp_u16(G.dp0, G.dp1, j) < T.anchor[ag])) continue;      // not eligible
+                        if (grp_u32(G, j) <= la_cut) ++n_above;
+                        else rem |= 1u << j;
+                    }
+                }
+            }
+            // queue the remaining entries of the warp (ids only), then work off whole rounds
+            const uint32_t cnt = __popc(rem);
             uint32_t incl = cnt;
 #pragma unroll
             for (int d = 1; d < 32; d <<= 1) {
                 const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, incl, d);
                 if (lane >= d) incl += v;
             }
-            uint32_t base = 0;
-            if (lane == 31 && incl) base = atomicAdd(&ws.sel->c_spec, incl);
-            base = __shfl_sync(0xFFFFFFFFu, base, 31);
-            uint32_t pos = base + incl - cnt;
-#pragma unroll
-            for (int j = 0; j < GRP; ++j) {
-                if (mask & (1u << j)) {                       // the key, for the few that are kept
-                    uint32_t pr, se;
-                    const uint32_t tok = a.ntok ? grp_u8(G.tk, j) : a.block_tokens;
-                    const uint32_t dp = (PF && a.anchor) ? grp_u16(G.dp0, G.dp1, j) : 0u;
-                    entry_key_rest<PF>(a, T, &ws.sc->status, grp_u16(G.ag0, G.ag1, j), dp, grp_u8(G.fl, j), grp_u32(G, j), tok, pr, se);
-                    atomicAdd(&s_hist[pr >> 20], 1u);
-                    ws.cand_km[pos] = ((unsigned long long)pr << 32) | se;
-                    ws.cand_id[pos] = grp_id(t, lane, j);
-                    ++pos;
-                }
+            const uint32_t total = __shfl_sync(0xFFFFFFFFu, incl, 31);
+            if (total == 0) continue;
+            uint32_t pos = qn + incl - cnt;
+            while (rem) {
+                const int j = __ffs(rem) - 1;
+                rem &= rem - 1;
+                q[pos++] = grp_id(t, lane, j);
             }
+            qn += total;
+            __syncwarp();
+            if (qn >= 32u) drain(false);
         }
+        drain(true);
         const uint32_t t0 = n_tiles * TILE;
         if (gtid < a.n - t0) {                                // ragged tail, one entry per thread, through the key
             const uint32_t i = t0 + gtid;
@@ -199,7 +338,7 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_fast_kernel(SelArgs a, cs_
             const uint32_t tok = a.ntok ? a.ntok[i] : a.block_tokens;
             if (entry_key<PF>(a, T, &ws.sc->status, a.agent[i], a.depth[i], a.ref[i], a.flags[i], a.la[i], tok, pr, se)) {
                 if ((pr >> 20) <= H) {
-                    atomicAdd(&s_hist[pr >> 20], 1u);
+                    atomicAdd(&ws.hist[pr >> 20], 1u);
                     const uint32_t pos = atomicAdd(&ws.sel->c_spec, 1u);
                     ws.cand_km[pos] = ((unsigned long long)pr << 32) | se;
                     ws.cand_id[pos] = i;
@@ -213,11 +352,6 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_fast_kernel(SelArgs a, cs_
     for (int d = 16; d > 0; d >>= 1) n_above += __shfl_xor_sync(0xFFFFFFFFu, n_above, d);
     if (lane == 0 && n_above) atomicAdd(&s_above, n_above);
     __syncthreads();
-    const uint32_t h_end = H < CS_HIST_BINS ? H + 1u : CS_HIST_BINS;          // bins above H stay empty
-    for (uint32_t i = threadIdx.x; i < h_end; i += blockDim.x) {
-        const uint32_t v = s_hist[i];
-        if (v) atomicAdd(&ws.hist[i], v);
-    }
     if (threadIdx.x == 0 && s_above) atomicAdd(&ws.sel->n_above, s_above);
     if (!last_cta_done(&ws.sel->ticket[0], &s_flag)) return;
 
@@ -225,10 +359,10 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_fast_kernel(SelArgs a, cs_
     constexpr uint32_t PER = CS_HIST_BINS / SEL_THREADS;
     uint32_t loc[PER], sum = 0;
 #pragma unroll
-    for (uint32_t q = 0; q < PER; ++q) {
-        loc[q] = __ldcg(&ws.hist[threadIdx.x * PER + q]);
-        ws.hist[threadIdx.x * PER + q] = 0;                 // ready for the next pass or call
-        sum += loc[q];
+    for (uint32_t qq = 0; qq < PER; ++qq) {
+        loc[qq] = __ldcg(&ws.hist[threadIdx.x * PER + qq]);
+        ws.hist[threadIdx.x * PER + qq] = 0;                 // ready for the next pass or call
+        sum += loc[qq];
     }
     s_part[threadIdx.x] = sum;
     if (threadIdx.x == 0) s_b0 = 0xFFFFFFFFu;
@@ -245,9 +379,9 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_fast_kernel(SelArgs a, cs_
     if (a.k && below >= a.k && before < a.k && a.k <= before + sum) {
         uint32_t run = before;
 #pragma unroll
-        for (uint32_t q = 0; q < PER; ++q) {
-            run += loc[q];
-            if (run >= a.k) { s_b0 = threadIdx.x * PER + q; break; }
+        for (uint32_t qq = 0; qq < PER; ++qq) {
+            run += loc[qq];
+            if (run >= a.k) { s_b0 = threadIdx.x * PER + qq; break; }
         }
     }
     __syncthreads();
@@ -261,7 +395,10 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_fast_kernel(SelArgs a, cs_
         if (ahead > H) ahead = H;                             // nothing is known about the bins above H
     }
     const uint32_t c_spec = __ldcg(&ws.sel->c_spec);
-    if (hit) publish_splitters(ws, (unsigned long long *)s_hist, s_hist + 2 * CS_SAMPLE, a.k ? c_spec : 0u);
+    if (hit) {                                                // the queues are idle now: they hold the sample
+        unsigned long long *s_km = (unsigned long long *)(((uintptr_t)queues + 7) & ~(uintptr_t)7);
+        publish_splitters(ws, s_km, (uint32_t *)(s_km + CS_SAMPLE), a.k ? c_spec : 0u);
+    }
     if (threadIdx.x == 0) {
         if (hit) {
             ws.sel->b0 = b0;
@@ -748,6 +885,10 @@ static int scan_opt_in(cs_ctx *ctx)
     cudaError_t e = cudaFuncSetAttribute(cs_sel_collect_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SCAN_SMEM_OPT_IN);
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(cs_sel_collect_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SCAN_SMEM_OPT_IN);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(cs_sel_fast_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SCAN_SMEM_OPT_IN);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(cs_sel_fast_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SCAN_SMEM_OPT_IN);
     if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; return CS_ECUDA; }
     g_scan_opted[ctx->device] = true;
     return CS_OK;
@@ -772,8 +913,10 @@ static int launch_select_job(cs_ctx *ctx, int job, const cs_block_index *idx, ui
     const uint32_t grid_c = cs_scan_grid(ctx, idx->n_blocks, 256);
     const size_t sm = cs_table_smem(ctx);
     int rc;
-    if (prefetch) cs_launch_chained(cs_sel_fast_kernel<true>, grid, SEL_THREADS, sm, s, a, ws);
-    else cs_launch_chained(cs_sel_fast_kernel<false>, grid, SEL_THREADS, sm, s, a, ws);
+    const size_t sm_fast = (sm + 15) / 16 * 16 + (size_t)(SEL_THREADS / 32) * FQ_CAP * sizeof(uint32_t) + 16;   // tables + per-warp queues
+    if ((rc = scan_opt_in(ctx)) != CS_OK) return rc;
+    if (prefetch) cs_launch_chained(cs_sel_fast_kernel<true>, grid, SEL_THREADS, sm_fast, s, a, ws);
+    else cs_launch_chained(cs_sel_fast_kernel<false>, grid, SEL_THREADS, sm_fast, s, a, ws);
     if ((rc = cs_check_launch(ctx)) != CS_OK) return rc;
     if (prefetch) cs_launch_chained(cs_sel_hist_kernel<true>, grid, SEL_THREADS, sm, s, a, ws);
     else cs_launch_chained(cs_sel_hist_kernel<false>, grid, SEL_THREADS, sm, s, a, ws);

@@ -10,12 +10,14 @@
 //
 // Ring: caller-owned device memory (cs_set_mover_staging), split into four sub-buffers, two per direction,
 // so that packing / scattering one part overlaps the copies of the other.  All ordering is by events between
-// the caller's stream (kernels) and two streams of the context (one per DMA direction); nothing synchronises
-// with the host.
+// the caller's stream (pack launches) and three streams of the context (one per DMA direction, one for the
+// scatter launches); nothing synchronises with the host.
 #include "cs_common.cuh"
 
 void cs_release_staging(cs_ctx *ctx)
 {
+    if (ctx->scatter_stream) cudaStreamDestroy(ctx->scatter_stream);
+    ctx->scatter_stream = nullptr;
     for (int j = 0; j < 2; ++j) {
         if (ctx->copy_stream[j]) cudaStreamDestroy(ctx->copy_stream[j]);
         if (ctx->ev_stage_join[j]) cudaEventDestroy(ctx->ev_stage_join[j]);
@@ -46,6 +48,7 @@ extern "C" int cs_set_mover_staging(cs_ctx *ctx, void *dev_ring, size_t bytes)
     }
     if (!ctx->copy_stream[0]) {                             // host objects, made once
         cudaError_t e = make_event(&ctx->ev_stage_fork);
+        if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&ctx->scatter_stream, cudaStreamNonBlocking);
         for (int j = 0; j < 2 && e == cudaSuccess; ++j) {
             e = cudaStreamCreateWithFlags(&ctx->copy_stream[j], cudaStreamNonBlocking);
             if (e == cudaSuccess) e = make_event(&ctx->ev_stage_join[j]);
@@ -134,49 +137,49 @@ extern "C" int cs_exchange_blocks_staged(cs_ctx *ctx, const cs_kv_pool *gpu, con
     if (rc != CS_OK) return rc;
     if (!host_ids_ok(host, off_host_ids, n_off) || !host_ids_ok(host, pre_host_ids, n_pre)) return CS_EINVAL;
     if (n_off == 0 && n_pre == 0) return CS_OK;
-    cudaStream_t S = (cudaStream_t)stream, CO = ctx->copy_stream[0], CP = ctx->copy_stream[1];
+    // The two directions are independent pipelines: pack launches on the caller's stream feed the device-to-host
+    // copies, host-to-device copies feed scatter launches on a stream of the context; neither waits for the other.
+    cudaStream_t S = (cudaStream_t)stream, CO = ctx->copy_stream[0], CP = ctx->copy_stream[1], KP = ctx->scatter_stream;
     const uint32_t cap = P.cap;
     const uint32_t nco = (n_off + cap - 1) / cap, ncp = (n_pre + cap - 1) / cap;
     cudaError_t e = cudaSuccess;
-    // both DMA streams start after everything already on the caller's stream (the previous user of the ring included)
+    // everything starts after what is already on the caller's stream (the previous user of the ring included)
     CK(cudaEventRecord(ctx->ev_stage_fork, S));
     CK(cudaStreamWaitEvent(CO, ctx->ev_stage_fork, 0));
     CK(cudaStreamWaitEvent(CP, ctx->ev_stage_fork, 0));
+    CK(cudaStreamWaitEvent(KP, ctx->ev_stage_fork, 0));
     for (uint32_t c = 0; c < (nco > ncp ? nco : ncp) && e == cudaSuccess && rc == CS_OK; ++c) {
         const int b = (int)(c & 1u);
         const uint32_t lo = c * cap;
-        if (c < ncp) {                                       // prefetch part c: host -> ring on the copy engine
+        if (c < ncp) {                                       // prefetch part c: host -> ring on the copy engine, then scatter
             const uint32_t hi = lo + cap < n_pre ? lo + cap : n_pre;
             if (c >= 2) CK(cudaStreamWaitEvent(CP, ctx->ev_scattered[b], 0));      // the ring buffer is free again
             CK(copy_runs(host, pre_host_ids, lo, hi, (unsigned char *)P.ring[1][b].base, P.block_bytes, false, CP));
             CK(cudaEventRecord(ctx->ev_filled[b], CP));
+            CK(cudaStreamWaitEvent(KP, ctx->ev_filled[b], 0));
+            if (e == cudaSuccess)
+                rc = cs_launch_mover_as(ctx, &P.ring[1][b], gpu, nullptr, pre_gpu_slots + lo, hi - lo, nullptr, CS_MOVE_STAGE,
+                                        CS_MOVE_PREFETCH, KP);
+            CK(cudaEventRecord(ctx->ev_scattered[b], KP));
         }
-        if (c < nco) {                                       // offload part c: pack on the SMs, ring -> host on the copy engine
+        if (c < nco && rc == CS_OK) {                        // offload part c: pack on the SMs, ring -> host on the copy engine
             const uint32_t hi = lo + cap < n_off ? lo + cap : n_off;
             if (c >= 2) CK(cudaStreamWaitEvent(S, ctx->ev_copied[b], 0));
             if (e == cudaSuccess)
-                rc = cs_launch_mover_as(ctx, gpu, &P.ring[0][b], off_gpu_slots + lo, nullptr, hi - lo, nullptr, CS_MOVE_D2D,
+                rc = cs_launch_mover_as(ctx, gpu, &P.ring[0][b], off_gpu_slots + lo, nullptr, hi - lo, nullptr, CS_MOVE_STAGE,
                                         CS_MOVE_OFFLOAD, S);
             CK(cudaEventRecord(ctx->ev_packed[b], S));
             CK(cudaStreamWaitEvent(CO, ctx->ev_packed[b], 0));
             CK(copy_runs(host, off_host_ids, lo, hi, (unsigned char *)P.ring[0][b].base, P.block_bytes, true, CO));
             CK(cudaEventRecord(ctx->ev_copied[b], CO));
         }
-        if (c < ncp && rc == CS_OK) {                        // scatter part c from the ring into the GPU pool
-            const uint32_t hi = lo + cap < n_pre ? lo + cap : n_pre;
-            CK(cudaStreamWaitEvent(S, ctx->ev_filled[b], 0));
-            if (e == cudaSuccess)
-                rc = cs_launch_mover_as(ctx, &P.ring[1][b], gpu, nullptr, pre_gpu_slots + lo, hi - lo, nullptr, CS_MOVE_D2D,
-                                        CS_MOVE_PREFETCH, S);
-            CK(cudaEventRecord(ctx->ev_scattered[b], S));
-        }
     }
-    // the caller's stream ends after the last copies to the host (the scatters are already on it)
+    // the caller's stream ends after the last copies to the host and the last scatter
     if (nco) {
         CK(cudaEventRecord(ctx->ev_stage_join[0], CO));
         CK(cudaStreamWaitEvent(S, ctx->ev_stage_join[0], 0));
     }
-    CK(cudaEventRecord(ctx->ev_stage_join[1], CP));
+    CK(cudaEventRecord(ctx->ev_stage_join[1], KP));
     CK(cudaStreamWaitEvent(S, ctx->ev_stage_join[1], 0));
     if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; return CS_ECUDA; }
     return rc;
