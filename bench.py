@@ -61,6 +61,8 @@ def parse_args():
     ap.add_argument("--quick", action="store_true", help="small pools (debugging only; not a valid bench line)")
     ap.add_argument("--workload", default="step", choices=["step", "mover", "select", "select80k", "select16m", "select64m"],
                     help="'mover'/'select' run one small case of that kernel family only (profiler captures)")
+    ap.add_argument("--kineto", action="store_true",
+                    help="with --workload select / select80k: warm per-kernel device times from the CUDA profiler API (torch.profiler)")
     ap.add_argument("--skip-aux", action="store_true",
                     help="timed steps only: no link-peak probe, end-to-end pass, extras or CPU baseline (profiler launch lists)")
     return ap.parse_args()
@@ -660,6 +662,15 @@ def fused_step_section(w, steps=10):
     def staged():
         c.exchange_blocks_staged(w.gpu_pool, w.host_pool, gv[:n_off], off_host, pre_host_k, pre_gpu_k, stream=side)
 
+    # the same transfer when the engine numbers the host tier itself, as consecutive runs (a log-structured host tier:
+    # the i-th offloaded block of a step goes to slot first + i): a step's transfer is a handful of large copies
+    G0 = w.cfg.gpu_blocks
+    run_off = (G0 + np.arange(n_off)).astype(np.uint32)
+    run_pre = (G0 + n_off + np.arange(len(pre_host_k))).astype(np.uint32)
+
+    def staged_runs():
+        c.exchange_blocks_staged(w.gpu_pool, w.host_pool, gv[:n_off], run_off, run_pre, pre_gpu_k, stream=side)
+
     def beside(op, reps, disturber):
         """Per-call time of `reps` back-to-back calls of op on the main stream while the disturber runs on the side stream."""
         best, x_ms = None, 0.0
@@ -688,13 +699,15 @@ def fused_step_section(w, steps=10):
     sel_alone, _ = beside(sel_op, 20, None)
     cmp_alone, _ = beside(cmp_op, 10, None)
     variants = []
-    for name, width, fn in (("sm_direct_width_32", 0, transfer), ("sm_direct_width_8", 8, transfer), ("staged_copy_engines", 0, staged)):
+    for name, width, fn in (("sm_direct_width_32", 0, transfer), ("sm_direct_width_8", 8, transfer),
+                            ("staged_copy_engines_scattered_host_slots", 0, staged),
+                            ("staged_copy_engines_consecutive_host_slots", 0, staged_runs)):
         c.set_mover_ctas(width, 0)
         _, x_alone_ms = beside(lambda: None, 1, fn)
         g_ms, g_x = run_graph(fn)
         sel_ms, _ = beside(sel_op, 20, fn)
         cmp_ms, _ = beside(cmp_op, 10, fn)
-        moved = (n_off + (len(pre_host_k) if fn is staged else n_pre)) * bb
+        moved = (n_off + (n_pre if fn is transfer else len(pre_host_k))) * bb
         variants.append({"transfer": name, "transfer_alone_ms": x_alone_ms, "link_GBps": moved / x_alone_ms / 1e6,
                          "graph_chain_slowdown_while_in_flight": in_flight_factor(g_alone, g_ms, g_x),
                          "fused_select_ms_alone": sel_alone, "fused_select_ms_beside": sel_ms, "fused_select_slowdown": sel_ms / sel_alone,
@@ -746,13 +759,20 @@ def host_link_peak(torch, device, n_bytes=GIB, reps=10):
     return out
 
 
-def time_call(torch, stream, fn, reps, warm=1):
+def time_call(torch, stream, fn, reps, warm=1, hide_host=True):
+    """Median and best device time of fn's work on `stream` (CUDA events).  With hide_host the stream is first given
+    ~150 us of busy-waiting, during which the host enqueues the first event, fn's launches and the second event:
+    the measured span is then the device's time for the work itself, not the host's time to issue it (what a
+    pipelined caller sees; it matters for transfers of a few tens of microseconds)."""
     for _ in range(warm):
         fn()
     stream.synchronize()
     ts = []
     for _ in range(reps):
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        if hide_host:
+            with torch.cuda.stream(stream):
+                torch.cuda._sleep(300_000)
         e0.record(stream)
         fn()
         e1.record(stream)
@@ -1144,13 +1164,34 @@ def profile_case(args, torch, device):
         vn, pn = torch.zeros(4, dtype=torch.int32, device=device), torch.zeros(4, dtype=torch.int32, device=device)
         hv = torch.empty(cfg.k_victims, dtype=torch.int32, device=device)
         hn = torch.zeros(4, dtype=torch.int32, device=device)
-        for s in range(max(1, args.steps)):
+        def one(s):
             lo = 64 * (30 + s)
             c.observe_invocations(ch[lo:lo + 64], ag[lo:lo + 64], None)
             c.select_victims(d, 100_000 + s, 0, cfg.k_victims, v, vn)
             c.select_prefetch(d, 100_000 + s, cfg.k_prefetch, pf, pn)
             if not big:        # the step's three selects as one launch
                 c.select_step(d, 100_000 + s, cfg.k_victims, cfg.k_prefetch, v, vn, hv, hn, pf, pn)
+
+        n_steps = max(1, args.steps)
+        if args.kineto:        # warm device times per kernel (L2-resident index, no serialisation), first 5 steps untimed
+            from torch.profiler import ProfilerActivity, profile
+            for s in range(min(5, n_steps)):
+                one(s)
+            torch.cuda.synchronize(device)
+            with profile(activities=[ProfilerActivity.CUDA]) as prof:
+                for s in range(min(5, n_steps), n_steps):
+                    one(s)
+                torch.cuda.synchronize(device)
+            per = {}
+            for e in prof.events():
+                if e.device_type == torch.autograd.DeviceType.CUDA and "cs_" in e.name:
+                    per.setdefault(e.name.split("(")[0], []).append(e.device_time)
+            print(json.dumps({"kernel_us_median_warm": {k: round(float(np.median(x)), 2) for k, x in per.items()},
+                              "launches_per_kernel": {k: len(x) for k, x in per.items()},
+                              "note": "durations of kernels launched with programmatic dependent launch include the wait for their predecessor"}))
+        else:
+            for s in range(n_steps):
+                one(s)
     torch.cuda.synchronize(device)
     print(json.dumps({"workload": args.workload, "launches": c.launch_count(), "device_status": c.get_status()}))
 

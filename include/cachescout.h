@@ -238,7 +238,7 @@ int cs_exchange_blocks(cs_ctx *ctx, const cs_kv_pool *gpu, const cs_kv_pool *hos
  *
  * cs_set_mover_staging(): hands the context a caller-owned DEVICE ring (256-byte aligned; at least 4 blocks,
  * 64-256 MiB is a sensible size) through which staged transfers pass, or takes it away (dev_ring = NULL).
- * The first call also creates the three streams and the events the staged calls use (host objects, released by
+ * The first call also creates the five streams and the events the staged calls use (host objects, released by
  * cs_destroy).  The ring must stay alive and unused by others while staged transfers are in flight.
  *
  * cs_exchange_blocks_staged(): offload of n_off blocks and prefetch of n_pre blocks.  GPU-side lists
@@ -247,7 +247,7 @@ int cs_exchange_blocks(cs_ctx *ctx, const cs_kv_pool *gpu, const cs_kv_pool *hos
  * engines need addresses the host knows.  Each part of the offload list is packed into the ring by the mover
  * kernel and carried to the host tier by cudaMemcpyAsync, one call per run of consecutive host ids (a list of
  * consecutive ids becomes a few large copies); the prefetch is the mirror image, ending in a scatter launch.
- * The two directions are independent pipelines (pack launches on `stream`; copies and scatter launches on three
+ * The two directions are independent pipelines (pack launches on `stream`; copies and scatter launches on five
  * streams of the context), forked from and joined back into `stream` by events, so to the caller everything
  * is ordered on `stream`; the host is never synchronised.
  * Requirements: the host pool is CS_BLOCK_MAJOR (a block is one run of bytes), both pools agree in geometry.

@@ -429,9 +429,14 @@ class KVPool:
         return self.n_layers * 2 * self.chunk_bytes
 
     def struct(self) -> cs_kv_pool:
-        assert self.buf.numel() * self.buf.element_size() >= self.n_slots * self.block_bytes
-        return cs_kv_pool(_ptr(self.buf), self.n_slots, self.layout, self.n_layers, self.n_kv_heads, self.head_dim,
-                          self.block_tokens, self.elem_bytes, self.first_id)
+        """The C struct (built once: the fields of a pool are not meant to change after construction)."""
+        s = self.__dict__.get("_struct")
+        if s is None:
+            assert self.buf.numel() * self.buf.element_size() >= self.n_slots * self.block_bytes
+            s = cs_kv_pool(_ptr(self.buf), self.n_slots, self.layout, self.n_layers, self.n_kv_heads, self.head_dim,
+                           self.block_tokens, self.elem_bytes, self.first_id)
+            self.__dict__["_struct"] = s
+        return s
 
 
 class CacheScout:

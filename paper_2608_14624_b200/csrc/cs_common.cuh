@@ -120,10 +120,10 @@ struct cs_ctx {
     // that order packing / copying / scattering
     unsigned char *stage_ring;
     size_t stage_bytes;
-    cudaStream_t copy_stream[2];         // 0: device -> host, 1: host -> device
+    cudaStream_t copy_stream[4];         // 0, 1: device -> host; 2, 3: host -> device
     cudaStream_t scatter_stream;         // scatter launches of staged prefetches
     cudaEvent_t ev_stage_fork, ev_stage_join[2];
-    cudaEvent_t ev_packed[2], ev_copied[2], ev_filled[2], ev_scattered[2];
+    cudaEvent_t ev_packed[2], ev_copied[4], ev_filled[4], ev_scattered[2];   // [ring buffer] or [2 * ring buffer + copy stream]
     uint64_t n_launches;
     int last_cuda_error;
 };

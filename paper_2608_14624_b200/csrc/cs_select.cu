@@ -122,11 +122,6 @@ __device__ __forceinline__ void publish_splitters(const cs_workspace &ws, unsign
 // ---------------------------------------------------------------------------------------------
 #define FQ_CAP 544u                 // per-warp queue: at most 31 left over + the 512 entries of one warp tile
 
-__device__ __forceinline__ uint32_t nibble_of_byte_flags(uint32_t ok)      // 0xFF / 0x00 per byte -> 4 bits
-{
-    return (((((ok >> 7) & 0x01010101u) * 0x01020408u) >> 24) & 0xFu);
-}
-
 // Largest value of every 16-bit half over eight packed words.
 __device__ __forceinline__ uint32_t max_halves(const uint4 &a, const uint4 &b)
 {
@@ -139,9 +134,11 @@ template <bool PF>
 __global__ void __launch_bounds__(SEL_THREADS) cs_sel_fast_kernel(SelArgs a, cs_workspace ws)
 {
     extern __shared__ float smem[];                 // tables, then the per-warp queues (reused by the epilogue)
+    __shared__ __align__(16) uint32_t s_hist[CS_HIST_BINS];   // bins of the candidates (the threshold bin is dense: global
+                                                              // atomics on one address per candidate would serialise)
     __shared__ uint32_t s_xt[2 * XT_TOK];
     __shared__ uint32_t s_part[SEL_THREADS];
-    __shared__ uint32_t s_b0, s_ahead, s_above, s_fbits, s_xext;
+    __shared__ uint32_t s_b0, s_ahead, s_above;
     __shared__ bool s_flag;
     cs_wait_for_predecessor();
     cs_release_successor();
@@ -155,65 +152,67 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_fast_kernel(SelArgs a, cs_
     load_tables(a, ws, smem, T, PF && a.anchor);
     const size_t table_words = ((size_t)(a.A + a.gtab_len) * 4 + (size_t)a.A * 2 + 15) / 16 * 4;
     uint32_t *queues = (uint32_t *)smem + table_words;
+    const size_t cut_off_words = table_words + (size_t)(SEL_THREADS / 32) * (FQ_CAP + STAGE_CAP * 3) + 4;     // after queues and staging
     build_x_thresholds<PF>(a, H, s_xt);
-    if (threadIdx.x == 0) { s_above = 0; s_fbits = PF ? 0u : 0x7F800000u; s_xext = PF ? 0xFFFFFFFFu : 0u; }
+    for (uint32_t i = threadIdx.x; i < CS_HIST_BINS; i += blockDim.x) s_hist[i] = 0;
+    if (threadIdx.x == 0) s_above = 0;
     __syncthreads();
-    // ---- the age cut -------------------------------------------------------------------------------------
-    // victims: f_min over the agents and the largest X over the sizes in range; prefetch: f_max and the smallest X
-    // of the agents other than a*.  (fsurv is positive, so floats order like their bit patterns.)
-    const uint32_t tok_lo = a.ntok ? 1u : a.block_tokens, tok_hi = a.block_tokens;
+    // ---- the age cuts, one per agent, for blocks of the common size ----------------------------------------
+    // victims: s_cut[agent] = number of ages (0, 1, ..) that are dismissed, i.e. for which fl(f g(age)) >= X;
+    // prefetch: s_cut[agent] = first age that is dismissed, i.e. fl(f g(age)) < X of the agents other than a*.
+    // Both rely on g never increasing with age (checked when the table was built) and on the table covering every
+    // unsaturated age; otherwise nothing is dismissed by age and every eligible entry takes the exact test.
+    const uint32_t Tb = a.block_tokens;
+    uint32_t *s_cut = (uint32_t *)smem + cut_off_words;
     {
-        uint32_t fb = PF ? 0u : 0x7F800000u, xe = PF ? 0xFFFFFFFFu : 0u;
-        for (uint32_t i = threadIdx.x; i < a.A; i += blockDim.x) {
-            const uint32_t b = __float_as_uint(T.fsurv[i]);
-            fb = PF ? max(fb, b) : min(fb, b);
+        const bool usable = ws.sc->gtab_monotone && a.gtab_len == a.age_sat;
+        const uint32_t X = s_xt[(PF ? XT_TOK : 0u) + Tb];
+        for (uint32_t e = threadIdx.x; e < a.A; e += blockDim.x) {
+            const float f = T.fsurv[e];
+            auto dismissed = [&](uint32_t age) {
+                const uint32_t xb = __float_as_uint(__fmul_rn(f, recency_of_age(a, T, age)));
+                return PF ? (xb < X) : (xb >= X);
+            };
+            uint32_t cut;
+            if (!PF) {
+                cut = 0;                                            // none
+                if (usable && X != XT_NONE && dismissed(0)) {
+                    if (dismissed(a.age_sat)) cut = 0xFFFFFFFFu;    // every age
+                    else {
+                        uint32_t lo = 0, hi = a.age_sat;            // largest dismissed age
+                        while (lo < hi) {
+                            const uint32_t mid = lo + ((hi - lo + 1) >> 1);
+                            if (dismissed(mid)) lo = mid;
+                            else hi = mid - 1;
+                        }
+                        cut = lo + 1;
+                    }
+                }
+            } else {
+                cut = 0xFFFFFFFFu;                                  // none
+                if (usable && (X == XT_NONE || dismissed(0))) cut = 0;          // every age
+                else if (usable && dismissed(a.age_sat)) {
+                    uint32_t lo = 0, hi = a.age_sat;                // smallest dismissed age
+                    while (lo < hi) {
+                        const uint32_t mid = lo + ((hi - lo) >> 1);
+                        if (dismissed(mid)) hi = mid;
+                        else lo = mid + 1;
+                    }
+                    cut = lo;
+                }
+            }
+            s_cut[e] = cut;
         }
-        for (uint32_t t = tok_lo + threadIdx.x; t <= tok_hi; t += blockDim.x) {
-            const uint32_t x = s_xt[(PF ? XT_TOK : 0u) + t];
-            xe = PF ? min(xe, x) : max(xe, x);
-        }
-        if (PF) { atomicMax(&s_fbits, fb); atomicMin(&s_xext, xe); }
-        else { atomicMin(&s_fbits, fb); atomicMax(&s_xext, xe); }
     }
     __syncthreads();
-    bool have_cut = false;
-    uint32_t la_cut = 0;
-    if (ws.sc->gtab_monotone && a.gtab_len == a.age_sat) {
-        const float f_ext = __uint_as_float(s_fbits);
-        const uint32_t x_ext = s_xext;
-        // dismissed(age): victims  fl(f_min g) >= X_max (true for young ages);  prefetch  fl(f_max g) < X_min (true for old ages)
-        auto dismissed = [&](uint32_t age) {
-            const uint32_t xb = __float_as_uint(__fmul_rn(f_ext, recency_of_age(a, T, age)));
-            return PF ? (xb < x_ext) : (xb >= x_ext);
-        };
-        if (!PF) {
-            if (x_ext != XT_NONE && dismissed(0)) {                 // largest age that is still dismissed
-                uint32_t lo = 0, hi = a.age_sat;
-                while (lo < hi) {
-                    const uint32_t mid = lo + ((hi - lo + 1) >> 1);
-                    if (dismissed(mid)) lo = mid;
-                    else hi = mid - 1;
-                }
-                have_cut = true;                                    // young <=> age <= lo <=> last_access >= now - lo
-                la_cut = (lo >= a.age_sat || lo >= a.now) ? 0u : a.now - lo;
-            }
-        } else {
-            if (x_ext == XT_NONE) { have_cut = true; la_cut = 0xFFFFFFFFu; }      // no entry of another agent can qualify
-            else if (dismissed(a.age_sat)) {                        // smallest age that is dismissed
-                uint32_t lo = 0, hi = a.age_sat;
-                while (lo < hi) {
-                    const uint32_t mid = lo + ((hi - lo) >> 1);
-                    if (dismissed(mid)) hi = mid;
-                    else lo = mid + 1;
-                }
-                if (lo == 0) { have_cut = true; la_cut = 0xFFFFFFFFu; }
-                else if (lo <= a.now) { have_cut = true; la_cut = a.now - lo; }   // old <=> age >= lo <=> last_access <= now - lo
-            }
-        }
-    }
     const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     uint32_t *q = queues + warp * FQ_CAP;
     uint32_t qn = 0;                                           // queued ids of this warp (same value in every lane)
+    WarpStage st;
+    {
+        unsigned long long *stage_km = (unsigned long long *)(((uintptr_t)(queues + (SEL_THREADS / 32) * FQ_CAP) + 7) & ~(uintptr_t)7);
+        stage_init(st, stage_km, (uint32_t *)(stage_km + (SEL_THREADS / 32) * STAGE_CAP));
+    }
     uint32_t n_above = 0;
     const bool enabled = !PF || prefetch_enabled(ws, a.A);
 
@@ -241,19 +240,13 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_fast_kernel(SelArgs a, cs_
                     if (!cand) ++n_above;
                 }
             }
-            const uint32_t bal = __ballot_sync(0xFFFFFFFFu, cand);
-            if (bal == 0) continue;
-            uint32_t base = 0;
-            if (lane == 0) base = atomicAdd(&ws.sel->c_spec, (uint32_t)__popc(bal));
-            base = __shfl_sync(0xFFFFFFFFu, base, 0);
+            uint32_t pr = 0, se = 0;
             if (cand) {
-                uint32_t pr, se;
                 entry_key_rest<PF>(a, T, &ws.sc->status, ag, dp, __ldg(a.flags + id), la, tok, pr, se);
-                atomicAdd(&ws.hist[pr >> 20], 1u);                  // few entries get here: straight into the global histogram
-                const uint32_t pos = base + __popc(bal & ((1u << lane) - 1u));
-                ws.cand_km[pos] = ((unsigned long long)pr << 32) | se;
-                ws.cand_id[pos] = id;
+                atomicAdd(&s_hist[pr >> 20], 1u);
             }
+            // candidates gather in the warp's slice of shared memory and leave it 32 or more at a time
+            stage_push(st, cand, pr, se, id, &ws.sel->c_spec, ws.cand_km, ws.cand_id);
         }
         if (!all) {
             const uint32_t done = rounds * 32u, left = qn - done;        // < 32
@@ -272,7 +265,6 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_fast_kernel(SelArgs a, cs_
         const uint32_t gtid = blockIdx.x * blockDim.x + threadIdx.x, nth = gridDim.x * blockDim.x;
         const uint32_t n_tiles = a.n / TILE, n_warps = nth >> 5;
         const uint32_t n_iter = (n_tiles + n_warps - 1) / n_warps;     // whole warps stay in the shuffles
-        const uint32_t tok_span = tok_hi - tok_lo + 1u;
         for (uint32_t it = 0; it < n_iter; ++it) {
             const uint32_t t = it * n_warps + (gtid >> 5);
             uint32_t rem = 0;                                          // entries that need the exact test
@@ -281,18 +273,19 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_fast_kernel(SelArgs a, cs_
                 load_group<PF>(a, t, lane, G);
                 const uint32_t em = group_elig<PF>(a, G);
                 if (!PF) {
-                    uint32_t dm = 0;                                   // dismissed by age (and safe to dismiss)
-                    if (have_cut && max_halves(G.ag0, G.ag1) < a.A) {
+                    uint32_t dm = 0;                                   // dismissed by age: young, of the common size
+                    if (max_halves(G.ag0, G.ag1) < a.A) {              // (a bad agent id anywhere: everything takes the exact test)
 #pragma unroll
-                        for (int j = 0; j < GRP; ++j) dm |= (grp_u32(G, j) >= la_cut ? 1u : 0u) << j;
-                        if (a.ntok) {                                  // sizes outside [1, block_tokens] take the exact test
-                            uint32_t in = 0;
+                        for (int j = 0; j < GRP; ++j) {
+                            const uint32_t la = grp_u32(G, j), age = max(a.now, la) - la;
+                            dm |= (age < s_cut[grp_u16(G.ag0, G.ag1, j)] ? 1u : 0u) << j;
+                        }
+                        if (a.ntok) {
+                            uint32_t same = 0;
 #pragma unroll
-                            for (int w = 0; w < 4; ++w) {
-                                const uint32_t x = __vsub4(u4_word(G.tk, w), 0x01010101u * tok_lo);
-                                in |= nibble_of_byte_flags(__vcmpltu4(x, 0x01010101u * tok_span)) << (4 * w);
-                            }
-                            dm &= in;
+                            for (int w = 0; w < 4; ++w)
+                                same |= nibble_of_flags(zero_bytes(u4_word(G.tk, w) ^ (0x01010101u * Tb))) << (4 * w);
+                            dm &= same;
                         }
                     }
                     n_above += __popc(em & dm);
@@ -302,10 +295,11 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_fast_kernel(SelArgs a, cs_
                     for (int j = 0; j < GRP; ++j) {
                         if (!((em >> j) & 1u)) continue;
                         const uint32_t ag = grp_u16(G.ag0, G.ag1, j);
-                        const uint32_t tok = a.ntok ? grp_u8(G.tk, j) : a.block_tokens;
-                        if (!have_cut || ag >= a.A || ag == T.a_star || tok - tok_lo >= tok_span) { rem |= 1u << j; continue; }
+                        const uint32_t tok = a.ntok ? grp_u8(G.tk, j) : Tb;
+                        if (ag >= a.A || ag == T.a_star || tok != Tb) { rem |= 1u << j; continue; }
                         if (a.anchor && !(grp_u16(G.dp0, G.dp1, j) < T.anchor[ag])) continue;      // not eligible
-                        if (grp_u32(G, j) <= la_cut) ++n_above;
+                        const uint32_t la = grp_u32(G, j), age = max(a.now, la) - la;
+                        if (age >= s_cut[ag]) ++n_above;
                         else rem |= 1u << j;
                     }
                 }
@@ -331,6 +325,7 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_fast_kernel(SelArgs a, cs_
             if (qn >= 32u) drain(false);
         }
         drain(true);
+        stage_flush(st, &ws.sel->c_spec, ws.cand_km, ws.cand_id);
         const uint32_t t0 = n_tiles * TILE;
         if (gtid < a.n - t0) {                                // ragged tail, one entry per thread, through the key
             const uint32_t i = t0 + gtid;
@@ -338,7 +333,7 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_fast_kernel(SelArgs a, cs_
             const uint32_t tok = a.ntok ? a.ntok[i] : a.block_tokens;
             if (entry_key<PF>(a, T, &ws.sc->status, a.agent[i], a.depth[i], a.ref[i], a.flags[i], a.la[i], tok, pr, se)) {
                 if ((pr >> 20) <= H) {
-                    atomicAdd(&ws.hist[pr >> 20], 1u);
+                    atomicAdd(&s_hist[pr >> 20], 1u);
                     const uint32_t pos = atomicAdd(&ws.sel->c_spec, 1u);
                     ws.cand_km[pos] = ((unsigned long long)pr << 32) | se;
                     ws.cand_id[pos] = i;
@@ -352,6 +347,13 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_fast_kernel(SelArgs a, cs_
     for (int d = 16; d > 0; d >>= 1) n_above += __shfl_xor_sync(0xFFFFFFFFu, n_above, d);
     if (lane == 0 && n_above) atomicAdd(&s_above, n_above);
     __syncthreads();
+    {
+        const uint32_t h_end = H < CS_HIST_BINS ? H + 1u : CS_HIST_BINS;          // bins above H stay empty
+        for (uint32_t i = threadIdx.x; i < h_end; i += blockDim.x) {
+            const uint32_t v = s_hist[i];
+            if (v) atomicAdd(&ws.hist[i], v);
+        }
+    }
     if (threadIdx.x == 0 && s_above) atomicAdd(&ws.sel->n_above, s_above);
     if (!last_cta_done(&ws.sel->ticket[0], &s_flag)) return;
 
@@ -913,7 +915,8 @@ static int launch_select_job(cs_ctx *ctx, int job, const cs_block_index *idx, ui
     const uint32_t grid_c = cs_scan_grid(ctx, idx->n_blocks, 256);
     const size_t sm = cs_table_smem(ctx);
     int rc;
-    const size_t sm_fast = (sm + 15) / 16 * 16 + (size_t)(SEL_THREADS / 32) * FQ_CAP * sizeof(uint32_t) + 16;   // tables + per-warp queues
+    const size_t sm_fast = (sm + 15) / 16 * 16 + (size_t)(SEL_THREADS / 32) * (FQ_CAP * sizeof(uint32_t) + STAGE_CAP * 12) + 32 +
+                           (size_t)ctx->p.n_agents * sizeof(uint32_t);   // tables, per-warp queues, per-warp candidate staging, age cuts
     if ((rc = scan_opt_in(ctx)) != CS_OK) return rc;
     if (prefetch) cs_launch_chained(cs_sel_fast_kernel<true>, grid, SEL_THREADS, sm_fast, s, a, ws);
     else cs_launch_chained(cs_sel_fast_kernel<false>, grid, SEL_THREADS, sm_fast, s, a, ws);

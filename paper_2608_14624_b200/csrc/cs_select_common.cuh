@@ -288,6 +288,17 @@ __device__ __forceinline__ uint32_t grp_u32(const Group &G, int j)
 // Flag / ref_count rules for the 16 entries of a group at once, four entries per 32-bit word
 // (byte-wise SIMD compares): bit j of the result is set when entry j is VALID, not PINNED, on the
 // requested tier (prefetch: on the host tier without a GPU copy) and unreferenced.
+// 0x80 in every byte of x that is zero (exact for all four bytes at once, plain integer operations).
+__device__ __forceinline__ uint32_t zero_bytes(uint32_t x)
+{
+    return ~(((x & 0x7F7F7F7Fu) + 0x7F7F7F7Fu) | x | 0x7F7F7F7Fu);
+}
+// The four 0x80 flags of a word gathered into a nibble (bit i = byte i).
+__device__ __forceinline__ uint32_t nibble_of_flags(uint32_t t)
+{
+    return (((t >> 7) * 0x01020408u) >> 24) & 0xFu;
+}
+
 template <bool PF>
 __device__ __forceinline__ uint32_t group_elig(const SelArgs &a, const Group &G)
 {
@@ -296,9 +307,9 @@ __device__ __forceinline__ uint32_t group_elig(const SelArgs &a, const Group &G)
     uint32_t out = 0;
 #pragma unroll
     for (int w = 0; w < 4; ++w) {
-        const uint32_t ok = __vcmpeq4(u4_word(G.fl, w) & fmask, fpat) & __vcmpeq4(u4_word(G.rf, w), 0u);
-        const uint32_t t = (ok >> 7) & 0x01010101u;                    // one bit per byte
-        out |= (((t * 0x01020408u) >> 24) & 0xFu) << (4 * w);           // gather bytes' bits into a nibble
+        // a byte of x is zero exactly when the entry's flags match the pattern and its ref_count is 0
+        const uint32_t x = ((u4_word(G.fl, w) & fmask) ^ fpat) | u4_word(G.rf, w);
+        out |= nibble_of_flags(zero_bytes(x)) << (4 * w);
     }
     return out;
 }

@@ -10,7 +10,7 @@
 //
 // Ring: caller-owned device memory (cs_set_mover_staging), split into four sub-buffers, two per direction,
 // so that packing / scattering one part overlaps the copies of the other.  All ordering is by events between
-// the caller's stream (pack launches) and three streams of the context (one per DMA direction, one for the
+// the caller's stream (pack launches) and five streams of the context (two per DMA direction, one for the
 // scatter launches); nothing synchronises with the host.
 #include "cs_common.cuh"
 
@@ -18,15 +18,18 @@ void cs_release_staging(cs_ctx *ctx)
 {
     if (ctx->scatter_stream) cudaStreamDestroy(ctx->scatter_stream);
     ctx->scatter_stream = nullptr;
-    for (int j = 0; j < 2; ++j) {
+    for (int j = 0; j < 4; ++j) {
         if (ctx->copy_stream[j]) cudaStreamDestroy(ctx->copy_stream[j]);
-        if (ctx->ev_stage_join[j]) cudaEventDestroy(ctx->ev_stage_join[j]);
-        if (ctx->ev_packed[j]) cudaEventDestroy(ctx->ev_packed[j]);
         if (ctx->ev_copied[j]) cudaEventDestroy(ctx->ev_copied[j]);
         if (ctx->ev_filled[j]) cudaEventDestroy(ctx->ev_filled[j]);
-        if (ctx->ev_scattered[j]) cudaEventDestroy(ctx->ev_scattered[j]);
         ctx->copy_stream[j] = nullptr;
-        ctx->ev_stage_join[j] = ctx->ev_packed[j] = ctx->ev_copied[j] = ctx->ev_filled[j] = ctx->ev_scattered[j] = nullptr;
+        ctx->ev_copied[j] = ctx->ev_filled[j] = nullptr;
+    }
+    for (int j = 0; j < 2; ++j) {
+        if (ctx->ev_stage_join[j]) cudaEventDestroy(ctx->ev_stage_join[j]);
+        if (ctx->ev_packed[j]) cudaEventDestroy(ctx->ev_packed[j]);
+        if (ctx->ev_scattered[j]) cudaEventDestroy(ctx->ev_scattered[j]);
+        ctx->ev_stage_join[j] = ctx->ev_packed[j] = ctx->ev_scattered[j] = nullptr;
     }
     if (ctx->ev_stage_fork) cudaEventDestroy(ctx->ev_stage_fork);
     ctx->ev_stage_fork = nullptr;
@@ -49,12 +52,14 @@ extern "C" int cs_set_mover_staging(cs_ctx *ctx, void *dev_ring, size_t bytes)
     if (!ctx->copy_stream[0]) {                             // host objects, made once
         cudaError_t e = make_event(&ctx->ev_stage_fork);
         if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&ctx->scatter_stream, cudaStreamNonBlocking);
-        for (int j = 0; j < 2 && e == cudaSuccess; ++j) {
+        for (int j = 0; j < 4 && e == cudaSuccess; ++j) {
             e = cudaStreamCreateWithFlags(&ctx->copy_stream[j], cudaStreamNonBlocking);
-            if (e == cudaSuccess) e = make_event(&ctx->ev_stage_join[j]);
-            if (e == cudaSuccess) e = make_event(&ctx->ev_packed[j]);
             if (e == cudaSuccess) e = make_event(&ctx->ev_copied[j]);
             if (e == cudaSuccess) e = make_event(&ctx->ev_filled[j]);
+        }
+        for (int j = 0; j < 2 && e == cudaSuccess; ++j) {
+            e = make_event(&ctx->ev_stage_join[j]);
+            if (e == cudaSuccess) e = make_event(&ctx->ev_packed[j]);
             if (e == cudaSuccess) e = make_event(&ctx->ev_scattered[j]);
         }
         if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; cs_release_staging(ctx); return CS_ECUDA; }
@@ -100,13 +105,16 @@ static bool host_ids_ok(const cs_kv_pool *host, const uint32_t *ids, uint32_t n)
     return true;
 }
 
-// One cudaMemcpyAsync per run of consecutive host slots within ring positions [lo, hi) of a sub-buffer.
+// One cudaMemcpyAsync per run of consecutive host slots within ring positions [lo, hi) of a sub-buffer, the runs
+// dealt alternately to two streams so that two copies of a direction are in flight (a copy of a single 2 MiB block
+// carries a few microseconds of fixed cost on its engine, which a second engine hides).
 static cudaError_t copy_runs(const cs_kv_pool *host, const uint32_t *ids, uint32_t lo, uint32_t hi, unsigned char *ring,
-                             size_t bb, bool to_host, cudaStream_t s)
+                             size_t bb, bool to_host, cudaStream_t s0, cudaStream_t s1)
 {
     cudaError_t e = cudaSuccess;
-    uint32_t i = lo;
+    uint32_t i = lo, turn = 0;
     while (i < hi && e == cudaSuccess) {
+        cudaStream_t s = (turn++ & 1u) ? s1 : s0;
         uint32_t j = i + 1;
         while (j < hi && ids[j] == ids[j - 1] + 1) ++j;
         unsigned char *h = (unsigned char *)host->base + (size_t)(ids[i] - host->first_id) * bb;
@@ -139,45 +147,51 @@ extern "C" int cs_exchange_blocks_staged(cs_ctx *ctx, const cs_kv_pool *gpu, con
     if (n_off == 0 && n_pre == 0) return CS_OK;
     // The two directions are independent pipelines: pack launches on the caller's stream feed the device-to-host
     // copies, host-to-device copies feed scatter launches on a stream of the context; neither waits for the other.
-    cudaStream_t S = (cudaStream_t)stream, CO = ctx->copy_stream[0], CP = ctx->copy_stream[1], KP = ctx->scatter_stream;
+    cudaStream_t S = (cudaStream_t)stream, KP = ctx->scatter_stream;
+    cudaStream_t *CO = &ctx->copy_stream[0], *CP = &ctx->copy_stream[2];          // two streams per DMA direction
     const uint32_t cap = P.cap;
     const uint32_t nco = (n_off + cap - 1) / cap, ncp = (n_pre + cap - 1) / cap;
     cudaError_t e = cudaSuccess;
     // everything starts after what is already on the caller's stream (the previous user of the ring included)
     CK(cudaEventRecord(ctx->ev_stage_fork, S));
-    CK(cudaStreamWaitEvent(CO, ctx->ev_stage_fork, 0));
-    CK(cudaStreamWaitEvent(CP, ctx->ev_stage_fork, 0));
+    for (int j = 0; j < 4; ++j) CK(cudaStreamWaitEvent(ctx->copy_stream[j], ctx->ev_stage_fork, 0));
     CK(cudaStreamWaitEvent(KP, ctx->ev_stage_fork, 0));
     for (uint32_t c = 0; c < (nco > ncp ? nco : ncp) && e == cudaSuccess && rc == CS_OK; ++c) {
         const int b = (int)(c & 1u);
         const uint32_t lo = c * cap;
-        if (c < ncp) {                                       // prefetch part c: host -> ring on the copy engine, then scatter
+        if (c < ncp) {                                       // prefetch part c: host -> ring on the copy engines, then scatter
             const uint32_t hi = lo + cap < n_pre ? lo + cap : n_pre;
-            if (c >= 2) CK(cudaStreamWaitEvent(CP, ctx->ev_scattered[b], 0));      // the ring buffer is free again
-            CK(copy_runs(host, pre_host_ids, lo, hi, (unsigned char *)P.ring[1][b].base, P.block_bytes, false, CP));
-            CK(cudaEventRecord(ctx->ev_filled[b], CP));
-            CK(cudaStreamWaitEvent(KP, ctx->ev_filled[b], 0));
+            for (int j = 0; j < 2; ++j) {
+                if (c >= 2) CK(cudaStreamWaitEvent(CP[j], ctx->ev_scattered[b], 0));      // the ring buffer is free again
+            }
+            CK(copy_runs(host, pre_host_ids, lo, hi, (unsigned char *)P.ring[1][b].base, P.block_bytes, false, CP[0], CP[1]));
+            for (int j = 0; j < 2; ++j) {
+                CK(cudaEventRecord(ctx->ev_filled[2 * b + j], CP[j]));
+                CK(cudaStreamWaitEvent(KP, ctx->ev_filled[2 * b + j], 0));
+            }
             if (e == cudaSuccess)
                 rc = cs_launch_mover_as(ctx, &P.ring[1][b], gpu, nullptr, pre_gpu_slots + lo, hi - lo, nullptr, CS_MOVE_STAGE,
                                         CS_MOVE_PREFETCH, KP);
             CK(cudaEventRecord(ctx->ev_scattered[b], KP));
         }
-        if (c < nco && rc == CS_OK) {                        // offload part c: pack on the SMs, ring -> host on the copy engine
+        if (c < nco && rc == CS_OK) {                        // offload part c: pack on the SMs, ring -> host on the copy engines
             const uint32_t hi = lo + cap < n_off ? lo + cap : n_off;
-            if (c >= 2) CK(cudaStreamWaitEvent(S, ctx->ev_copied[b], 0));
+            if (c >= 2) {
+                CK(cudaStreamWaitEvent(S, ctx->ev_copied[2 * b], 0));
+                CK(cudaStreamWaitEvent(S, ctx->ev_copied[2 * b + 1], 0));
+            }
             if (e == cudaSuccess)
                 rc = cs_launch_mover_as(ctx, gpu, &P.ring[0][b], off_gpu_slots + lo, nullptr, hi - lo, nullptr, CS_MOVE_STAGE,
                                         CS_MOVE_OFFLOAD, S);
             CK(cudaEventRecord(ctx->ev_packed[b], S));
-            CK(cudaStreamWaitEvent(CO, ctx->ev_packed[b], 0));
-            CK(copy_runs(host, off_host_ids, lo, hi, (unsigned char *)P.ring[0][b].base, P.block_bytes, true, CO));
-            CK(cudaEventRecord(ctx->ev_copied[b], CO));
+            for (int j = 0; j < 2; ++j) CK(cudaStreamWaitEvent(CO[j], ctx->ev_packed[b], 0));
+            CK(copy_runs(host, off_host_ids, lo, hi, (unsigned char *)P.ring[0][b].base, P.block_bytes, true, CO[0], CO[1]));
+            for (int j = 0; j < 2; ++j) CK(cudaEventRecord(ctx->ev_copied[2 * b + j], CO[j]));
         }
     }
     // the caller's stream ends after the last copies to the host and the last scatter
     if (nco) {
-        CK(cudaEventRecord(ctx->ev_stage_join[0], CO));
-        CK(cudaStreamWaitEvent(S, ctx->ev_stage_join[0], 0));
+        for (int j = 0; j < 4; ++j) CK(cudaStreamWaitEvent(S, ctx->ev_copied[j], 0));   // (an event never recorded counts as done)
     }
     CK(cudaEventRecord(ctx->ev_stage_join[1], KP));
     CK(cudaStreamWaitEvent(S, ctx->ev_stage_join[1], 0));
