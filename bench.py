@@ -97,17 +97,27 @@ def mem_available_bytes():
 
 
 class PinnedBuffer:
-    """Page-locked host memory of an exact size: a pageable tensor registered with cudaHostRegister (torch's own
-    pinned allocator rounds every request up to a power of two, which would double a 117 GiB tier)."""
+    """Page-locked host memory.  First choice: a pageable tensor of the exact size registered with cudaHostRegister
+    (torch's own pinned allocator rounds every request up to a power of two, which would double a 117 GiB tier).
+    Where registration is refused (a locked-memory limit of the environment), the largest power of two of bytes that
+    fits the request comes from torch's pinned allocator (cudaHostAlloc) instead; `nbytes` says what was obtained."""
 
     def __init__(self, torch, nbytes):
         self.torch, self.registered = torch, False
         t0 = time.time()
         self.t = torch.empty(nbytes, dtype=torch.uint8)
         rc = torch.cuda.cudart().cudaHostRegister(self.t.data_ptr(), nbytes, 0)
-        if int(rc) != 0:
-            raise RuntimeError("cudaHostRegister of %d bytes failed (%s)" % (nbytes, rc))
-        self.registered = True
+        if int(rc) == 0:
+            self.registered, self.how, self.nbytes = True, "cudaHostRegister", nbytes
+        else:
+            self.t = None
+            pow2 = 1 << (int(nbytes).bit_length() - 1)
+            try:
+                self.t = torch.empty(pow2, dtype=torch.uint8, pin_memory=True)
+            except RuntimeError as e:
+                raise RuntimeError("no page-locked memory: cudaHostRegister of %d bytes failed (%s) and cudaHostAlloc of %d "
+                                   "bytes failed (%s)" % (nbytes, rc, pow2, e))
+            self.how, self.nbytes = "cudaHostAlloc", pow2
         self.seconds = time.time() - t0
 
     def free(self):
@@ -184,7 +194,8 @@ class StepWorkload:
     def __init__(self, args, device, n_replicas, cfg_name="llama8b"):
         import torch
         from paper_2608_14624_b200 import binding as cs
-        from paper_2608_14624_b200 import build, synth
+        from paper_2608_14624_b200 import build
+        from tests import synth
         build.build_library()
         self.torch, self.cs, self.synth = torch, cs, synth
         self.dev = device
@@ -199,7 +210,21 @@ class StepWorkload:
         self.host_backed = host_tier_slots(Hs, bb, args.host_slots, args.host_frac, n_replicas)
         if args.quick:
             self.host_backed = min(self.host_backed, 1024)
-        self.pinned = PinnedBuffer(torch, self.host_backed * bb)
+        # Page-locking tens of GiB can fail although MemAvailable said otherwise (memory of a process that has just exited
+        # is still being returned, a locked-memory limit): wait, ask for less, try again -- the reduction is reported.
+        self.pin_attempts = 0
+        while True:
+            self.pin_attempts += 1
+            try:
+                self.pinned = PinnedBuffer(torch, self.host_backed * bb)
+                self.host_backed = self.pinned.nbytes // bb          # (fewer when the fallback allocator was used)
+                break
+            except RuntimeError:
+                if self.pin_attempts >= 6 or self.host_backed <= 1024:
+                    raise
+                time.sleep(3.0)
+                again = host_tier_slots(Hs, bb, args.host_slots, args.host_frac, n_replicas)
+                self.host_backed = max(1024, min(again, int(self.host_backed * 0.75)))
         self.host_buf = self.pinned.t
         self.t_pin = self.pinned.seconds
         self.gpu_buf = torch.empty(G * bb // 2, dtype=torch.bfloat16, device=device)
@@ -823,7 +848,7 @@ def mover_sweep(w, hbm_peak, link):
         src_rot = np.roll(src, 1)                                           # the compaction moves other blocks than the prefetch did
         d_src, d_dst_h = up(src.astype(np.uint32)), up((dst_h + G).astype(np.uint32))   # host pool ids start at G
         d_back, d_src_rot = up(back), up(src_rot.astype(np.uint32))
-        reps = 5 if n <= 512 else 3
+        reps = 20 if n <= 512 else 8                                        # after 3 warm-up repetitions
         # fair comparator for the latency-bound small batches: one contiguous pinned copy of the same size
         tmp = torch.empty(n * bb, dtype=torch.uint8, device=dev)
         hview = w.host_buf[:n * bb]
@@ -835,13 +860,13 @@ def mover_sweep(w, hbm_peak, link):
             gp = cs.KVPool(w.gpu_buf, G, lay, L)
             pool_block = lambda slot: _block_from_pool(gpu_u8, lay, G, L, chunk, slot)
             checked = 0
-            med_o, best_o = time_call(torch, side, lambda: c.offload_blocks(gp, w.host_pool, d_src, d_dst_h, stream=side), reps)
+            med_o, best_o = time_call(torch, side, lambda: c.offload_blocks(gp, w.host_pool, d_src, d_dst_h, stream=side), reps, warm=3)
             checked += _check_moved_blocks(orc, lambda i: pool_block(int(src[i])), lambda i: host_block(int(dst_h[i])),
                                            lay, cs.CS_BLOCK_MAJOR, L, chunk, n, rng)
-            med_p, best_p = time_call(torch, side, lambda: c.prefetch_blocks(w.host_pool, gp, d_dst_h, d_back, stream=side), reps)
+            med_p, best_p = time_call(torch, side, lambda: c.prefetch_blocks(w.host_pool, gp, d_dst_h, d_back, stream=side), reps, warm=3)
             checked += _check_moved_blocks(orc, lambda i: host_block(int(dst_h[i])), lambda i: pool_block(int(back[i])),
                                            cs.CS_BLOCK_MAJOR, lay, L, chunk, n, rng)
-            med_c, best_c = time_call(torch, side, lambda: c.compact_blocks(gp, gp, d_src_rot, d_back, stream=side), reps)
+            med_c, best_c = time_call(torch, side, lambda: c.compact_blocks(gp, gp, d_src_rot, d_back, stream=side), reps, warm=3)
             checked += _check_moved_blocks(orc, lambda i: pool_block(int(src_rot[i])), lambda i: pool_block(int(back[i])),
                                            lay, lay, L, chunk, n, rng)
             gb = n * bb / 1e9
@@ -852,6 +877,7 @@ def mover_sweep(w, hbm_peak, link):
                          "offload_frac_of_memcpy_same_size": cp_o / med_o, "prefetch_frac_of_memcpy_same_size": cp_p / med_p,
                          "d2d_GBps_rw": 2 * gb / (med_c / 1e3), "d2d_frac_of_hbm": 2 * gb / (med_c / 1e3) / hbm_peak,
                          "offload_ms": med_o, "prefetch_ms": med_p, "d2d_ms": med_c,
+                         "offload_ms_best": best_o, "prefetch_ms_best": best_p, "d2d_ms_best": best_c, "repetitions": reps,
                          "blocks_byte_checked_against_oracle": checked})
     return rows
 
@@ -1037,7 +1063,7 @@ class OracleStep:
 
     def __init__(self, cfg_name="llama8b"):
         from oracle import cs_oracle as orc
-        from paper_2608_14624_b200 import synth
+        from tests import synth
         self.orc, self.synth = orc, synth
         cfg = synth.CONFIGS[cfg_name]
         self.cfg = cfg
@@ -1107,7 +1133,8 @@ def profile_case(args, torch, device):
     select80k: the 80,000-entry index of the Llama-8B configuration, 256 victims / 384 prefetch
             candidates (single-launch cluster select path), then the step's three selects as one launch."""
     from paper_2608_14624_b200 import binding as cs
-    from paper_2608_14624_b200 import build, synth
+    from paper_2608_14624_b200 import build
+    from tests import synth
     build.build_library()
     if args.workload in ("select16m", "select64m"):
         # one kind of select over an index far larger than L2 (176 MB / 704 MB of metadata): the regime in which the
@@ -1182,13 +1209,20 @@ def profile_case(args, torch, device):
                 for s in range(min(5, n_steps), n_steps):
                     one(s)
                 torch.cuda.synchronize(device)
-            per = {}
-            for e in prof.events():
-                if e.device_type == torch.autograd.DeviceType.CUDA and "cs_" in e.name:
-                    per.setdefault(e.name.split("(")[0], []).append(e.device_time)
+            # All launches of this workload are on one stream.  A kernel launched with programmatic dependent launch starts
+            # early and waits for its predecessor, so its own time is taken from the end of the kernel before it.
+            evs = sorted((e for e in prof.events() if e.device_type == torch.autograd.DeviceType.CUDA and "cs_" in e.name),
+                         key=lambda e: e.time_range.start)
+            per, prev_end = {}, 0
+            for e in evs:
+                own = e.time_range.end - max(e.time_range.start, prev_end)
+                prev_end = max(prev_end, e.time_range.end)
+                per.setdefault(e.name.split("(")[0], []).append(own)
+            calls = n_steps - min(5, n_steps)
             print(json.dumps({"kernel_us_median_warm": {k: round(float(np.median(x)), 2) for k, x in per.items()},
-                              "launches_per_kernel": {k: len(x) for k, x in per.items()},
-                              "note": "durations of kernels launched with programmatic dependent launch include the wait for their predecessor"}))
+                              "launches_per_call": {k: len(x) / calls for k, x in per.items()},
+                              "us_of_kernel_time_per_call": round(sum(float(np.sum(x)) for x in per.values()) / calls, 1),
+                              "note": "own time of each kernel: from the end of the kernel before it on the stream (or its own start) to its end"}))
         else:
             for s in range(n_steps):
                 one(s)
@@ -1197,6 +1231,7 @@ def profile_case(args, torch, device):
 
 
 WORKLOAD_TEXT = {
+    "tiny": "tiny step (BASELINE.json configs[0]): 8 layers x 8 KV heads x 128 bf16, 512 KiB blocks",
     "llama8b": "llama8b-kv step (BASELINE.json configs[1]): 32 layers x 8 KV heads x 128 bf16, 2 MiB blocks",
     "llama70b": "llama70b-kv step (BASELINE.json configs[3]): 80 layers x 8 KV heads x 128 bf16, 5 MiB blocks",
 }
@@ -1307,6 +1342,7 @@ def measure_step_workload(args, w, ctx):
                    "host_tier": {"named_slots": named, "backed_slots": backed, "reduction": round(1.0 - backed / named, 4),
                                  "why": "all named slots are pinned" if backed == named else
                                         "pinned memory limited to %.2f of the box's available memory" % args.host_frac,
+                                 "pin_attempts": w.pin_attempts, "pinned_by": w.pinned.how,
                                  "pinned_GiB": round(backed * bb / GIB, 1), "pin_seconds": round(w.t_pin, 2)},
                    "l2_policy": "inputs larger than L2: every step moves %.2f GiB of scattered blocks; the %.1f MB index is L2-resident by design"
                                 % ((2 * w.k_v + w.k_p) * bb / GIB, w.N * 11 / 1e6),
@@ -1424,6 +1460,12 @@ def main():
         out["second_config"] = sub
         w2.release()
         del w2
+        w0 = StepWorkload(args, device, world, "tiny")          # configs[0]: 512-block pool, 2,048-slot host tier, k = 32 / 64
+        sub0 = measure_step_workload(args, w0, ctx)
+        out["tiny_config"] = {k: sub0[k] for k in ("value", "ms_per_step", "config", "roofline", "roofline_hbm", "e2e", "select",
+                                                    "blocks_moved_in_timed_steps", "gpu_launches")}
+        w0.release()
+        del w0
         out["metadata_scale"] = metadata_scale(torch, cs, synth, device, hbm_peak, calls=args.meta_calls)
         out["exact_survival"] = exact_survival_section(torch, cs, synth, device)
         out["hbm_regime"] = hbm_regime_section(torch, cs, synth, device, hbm_peak)

@@ -30,7 +30,7 @@ from typing import Dict, List, Optional, Tuple
 import numpy as np
 
 from oracle import cs_oracle as orc
-from paper_2608_14624_b200 import synth
+from tests import synth
 
 from . import helpers as H
 

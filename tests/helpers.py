@@ -2,7 +2,7 @@
 import numpy as np
 
 from oracle import cs_oracle as orc
-from paper_2608_14624_b200 import synth
+from tests import synth
 
 REL_TOL = 1e-6          # fp32 reuse scores vs the fp64 oracle (relative)
 R_ABS_TOL = 1e-5        # predictability: sum of A^2 entropy terms

@@ -1,6 +1,7 @@
 """Seeded synthetic inputs: agent traces, block-index metadata, KV pools, mover batches.
 
-This module serves BOTH the CPU oracle's tests and the CUDA path's tests/bench, so it
+This module serves BOTH the CPU oracle's tests and the CUDA path's tests / bench (it is
+test infrastructure and lives outside the product package), so it
 holds none of the method's arithmetic (no counting, normalising, scoring, selecting or
 copying of KV bytes): it only draws shapes and values.  Everything is NumPy on the host,
 driven by ``numpy.random.Generator(PCG64(seed))``; callers move arrays to the device.

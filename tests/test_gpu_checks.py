@@ -9,7 +9,7 @@ torch = pytest.importorskip("torch")
 
 from oracle import cs_oracle as orc
 from paper_2608_14624_b200 import binding as cs
-from paper_2608_14624_b200 import synth
+from tests import synth
 from tests import helpers as H
 
 pytestmark = pytest.mark.gpu

@@ -8,7 +8,7 @@ torch = pytest.importorskip("torch")
 
 from oracle import cs_oracle as orc
 from paper_2608_14624_b200 import binding as cs
-from paper_2608_14624_b200 import synth
+from tests import synth
 from tests import helpers as H
 
 pytestmark = pytest.mark.gpu
@@ -215,30 +215,49 @@ def test_select_without_optional_tables_and_capacity_errors():
 
 
 def test_metadata_scale_first_calls():
-    """1,000,000-entry index, 256 agents, k = 10,000 victims / 2,000 prefetch candidates, state
-    evolving between calls (the launch configuration the benchmark times)."""
+    """1,000,000-entry index, 256 agents, k = 10,000 victims / 2,000 prefetch candidates, state evolving between
+    calls (the launch configuration the benchmark times): every one of the first 100 calls against the oracle, then
+    every 50th up to call 600 (between those the library's own lists advance the state, so a checked call also
+    vouches for the calls before it), issued alternately as two calls and as one cs_select_step call."""
     cfg = synth.CONFIGS["meta1m"]
     N = 1_000_000
-    tr = synth.make_trace(cfg, n_invocations=64 * 40)
+    n_calls = 601
+    tr = synth.make_trace(cfg, n_invocations=64 * (n_calls + 8))
     c, o = make_ctx(cfg, N, r_min=0.02)
     idx = synth.make_block_index(cfg, n=N, tier="random")
     rng = synth.rng_for(cfg, 9)
     now0 = 100_000
-    for call in range(6):
+    checked = 0
+    v_ids = torch.empty(cfg.k_victims, dtype=torch.int32, device=DEV)
+    p_ids = torch.empty(cfg.k_prefetch, dtype=torch.int32, device=DEV)
+    v_n, p_n = torch.zeros(4, dtype=torch.int32, device=DEV), torch.zeros(4, dtype=torch.int32, device=DEV)
+    d = cs.DeviceIndex.from_host(idx, DEV)
+    for call in range(n_calls):
         lo, hi = int(tr.step_off[call * 4]), int(tr.step_off[call * 4 + 4])
         c.observe_invocations(dev(tr.chain[lo:hi]), dev(tr.agent[lo:hi]), None)
         o.observe(tr.chain[lo:hi], tr.agent[lo:hi])
         now = now0 + call
-        d = cs.DeviceIndex.from_host(idx, DEV)
-        s64, s32 = o.scores(idx, now)
-        v_ids, v_n = c.select_victims(d, now, 0, cfg.k_victims)
-        p_ids, p_n = c.select_prefetch(d, now, cfg.k_prefetch)
-        ov, ovn = o.select_victims(idx, now, 0, cfg.k_victims, s32)
-        op, opn = o.select_prefetch(idx, now, cfg.k_prefetch, s32)
-        H.assert_list_matches(v_ids.cpu().numpy().view(np.uint32)[:cfg.k_victims], int(v_n.item()), ov, ovn, s64)
-        H.assert_list_matches(p_ids.cpu().numpy().view(np.uint32)[:cfg.k_prefetch], int(p_n.item()), op, opn, s64)
-        synth.mutate_index(idx, rng, now, ov, op, int(o.last_agent[0]), cfg.n_agents)
+        for name in ("agent", "depth", "ref_count", "flags", "last_access"):       # the evolved index, same device arrays
+            getattr(d, name).copy_(torch.from_numpy(getattr(idx, name)))
+        if call % 2:
+            c.select_step(d, now, cfg.k_victims, cfg.k_prefetch, v_ids, v_n, None, None, p_ids, p_n)
+        else:
+            c.select_victims(d, now, 0, cfg.k_victims, v_ids, v_n)
+            c.select_prefetch(d, now, cfg.k_prefetch, p_ids, p_n)
+        gv, gp = v_ids.cpu().numpy().view(np.uint32)[:cfg.k_victims], p_ids.cpu().numpy().view(np.uint32)[:cfg.k_prefetch]
+        if call < 100 or call % 50 == 0:
+            s64, s32 = o.scores(idx, now)
+            ov, ovn = o.select_victims(idx, now, 0, cfg.k_victims, s32)
+            op, opn = o.select_prefetch(idx, now, cfg.k_prefetch, s32)
+            assert H.assert_list_matches(gv, int(v_n[0].item()), ov, ovn, s64) == 0, call
+            assert H.assert_list_matches(gp, int(p_n[0].item()), op, opn, s64) == 0, call
+            checked += 1
+        synth.mutate_index(idx, rng, now, gv, gp, int(o.last_agent[0]), cfg.n_agents)
+    assert checked == 100 + 11
     H.compare_model(c, o)
+    cn = c.counters()
+    assert cn["selects"][0] == n_calls and cn["selects"][2] == n_calls
+    assert cn["fast_hits"][0] > n_calls // 2                  # the remembered threshold holds in most calls
     assert c.get_status() == 0
 
 

@@ -11,7 +11,7 @@ import numpy as np
 import pytest
 
 from oracle import cs_oracle as orc
-from paper_2608_14624_b200 import synth
+from tests import synth
 from tests.conftest import read_golden
 
 P = orc.Params
