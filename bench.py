@@ -1327,7 +1327,8 @@ def measure_step_workload(args, w, ctx):
     # the two-way transfer: bytes of one launch over its duration on the side stream, against what the link gives two
     # concurrent pinned cudaMemcpyAsync copies in the same out:in proportion, measured in this run
     x_ms = t_o if w.fused else max(t_o, t_p)
-    x_gbps = w.bytes_per_step / (x_ms / 1e3) / 1e9
+    x_bytes = moved_bytes / args.steps                   # what a launch really moved (the nominal 256 + 384 blocks at full size)
+    x_gbps = x_bytes / (x_ms / 1e3) / 1e9
     # time a perfect duplex link would need for the step's bytes, from the one-direction peaks of this run
     ideal_ms = max(w.k_v * bb / link["d2h"], w.k_p * bb / link["h2d"]) / 1e6
     named, backed = cfg.host_blocks, w.host_backed
@@ -1361,7 +1362,7 @@ def measure_step_workload(args, w, ctx):
                                   "2:3 out:in proportion (PCIe Gen5 x16 is neither HBM nor a tensor pipe)",
                      "peak_per_direction": {"d2h": link["d2h"], "h2d": link["h2d"], "both_1to1": link["bidir"]},
                      "ideal_duplex_ms": ideal_ms, "frac_of_ideal_duplex": ideal_ms / x_ms,
-                     "algorithmic_bytes_per_launch": w.bytes_per_step, "ms_per_launch": x_ms,
+                     "algorithmic_bytes_per_launch": x_bytes, "ms_per_launch": x_ms,
                      "traffic_note": "DRAM bytes of one launch (ncu, profiles/): each block crosses HBM once"},
         "roofline_hbm": {"kernel": "cs_mover_bulk_kernel (device-to-device compaction of the %d victims, inside the step, while the host-link "
                                    "transfer of the previous step runs beside it)" % w.k_v, "bound": "hbm",
