@@ -234,6 +234,7 @@ int cs_destroy(cs_ctx *ctx)
 int cs_observe_invocations(cs_ctx *ctx, const uint32_t *chain, const uint16_t *agent, const uint8_t *evflags,
                            uint32_t n_events, cs_stream_t stream)
 {
+    CS_RANGE("cs_observe_invocations");
     if (!ctx) return CS_EINVAL;
     if (n_events && (!chain || !agent)) return CS_EINVAL;
     if ((((uintptr_t)chain) & 3u) || (((uintptr_t)agent) & 1u)) return CS_EINVAL;   // scalar loads: natural alignment
@@ -260,6 +261,7 @@ static int check_index(const cs_ctx *ctx, const cs_block_index *idx)
 int cs_score_blocks(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, const uint16_t *sources,
                     uint32_t n_sources, float *scores_out, cs_stream_t stream)
 {
+    CS_RANGE("cs_score_blocks");
     if (!ctx) return CS_EINVAL;
     int rc = check_index(ctx, idx);
     if (rc != CS_OK) return rc;
@@ -291,12 +293,14 @@ static int select_common(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, i
 int cs_select_victims(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, uint32_t tier, uint32_t k,
                       uint32_t *ids_out, uint32_t *n_out, cs_stream_t stream)
 {
+    CS_RANGE("cs_select_victims");
     return select_common(ctx, idx, now, 0, tier, k, ids_out, n_out, stream);
 }
 
 int cs_select_prefetch(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, uint32_t k, uint32_t *ids_out,
                        uint32_t *n_out, cs_stream_t stream)
 {
+    CS_RANGE("cs_select_prefetch");
     return select_common(ctx, idx, now, 1, 1, k, ids_out, n_out, stream);
 }
 
@@ -304,6 +308,7 @@ int cs_select_step(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, uint32_
                    uint32_t *gpu_victims, uint32_t *n_gpu_victims, uint32_t *host_victims, uint32_t *n_host_victims,
                    uint32_t *prefetch_ids, uint32_t *n_prefetch, cs_stream_t stream)
 {
+    CS_RANGE("cs_select_step");
     if (!ctx) return CS_EINVAL;
     int rc = check_index(ctx, idx);
     if (rc != CS_OK) return rc;
@@ -350,18 +355,21 @@ static int mover_common(cs_ctx *ctx, const cs_kv_pool *src, const cs_kv_pool *ds
 int cs_offload_blocks(cs_ctx *ctx, const cs_kv_pool *gpu, const cs_kv_pool *host, const uint32_t *src_slots,
                       const uint32_t *dst_slots, uint32_t n_max, const uint32_t *n_dev, cs_stream_t side)
 {
+    CS_RANGE("cs_offload_blocks");
     return mover_common(ctx, gpu, host, src_slots, dst_slots, n_max, n_dev, CS_MOVE_OFFLOAD, side);
 }
 
 int cs_prefetch_blocks(cs_ctx *ctx, const cs_kv_pool *host, const cs_kv_pool *gpu, const uint32_t *src_slots,
                        const uint32_t *dst_slots, uint32_t n_max, const uint32_t *n_dev, cs_stream_t side)
 {
+    CS_RANGE("cs_prefetch_blocks");
     return mover_common(ctx, host, gpu, src_slots, dst_slots, n_max, n_dev, CS_MOVE_PREFETCH, side);
 }
 
 int cs_compact_blocks(cs_ctx *ctx, const cs_kv_pool *src, const cs_kv_pool *dst, const uint32_t *src_slots,
                       const uint32_t *dst_slots, uint32_t n_max, const uint32_t *n_dev, cs_stream_t stream)
 {
+    CS_RANGE("cs_compact_blocks");
     return mover_common(ctx, src, dst, src_slots, dst_slots, n_max, n_dev, CS_MOVE_D2D, stream);
 }
 
@@ -370,6 +378,7 @@ int cs_exchange_blocks(cs_ctx *ctx, const cs_kv_pool *gpu, const cs_kv_pool *hos
                        const uint32_t *pre_host_slots, const uint32_t *pre_gpu_slots, uint32_t n_pre_max,
                        const uint32_t *n_pre_dev, cs_stream_t side)
 {
+    CS_RANGE("cs_exchange_blocks");
     if (!ctx) return CS_EINVAL;
     int rc = check_pools(gpu, host);
     if (rc != CS_OK) return rc;
@@ -387,6 +396,7 @@ int cs_exchange_blocks(cs_ctx *ctx, const cs_kv_pool *gpu, const cs_kv_pool *hos
 
 int cs_step(cs_ctx *ctx, const cs_step_io *io, cs_stream_t main_, cs_stream_t side_)
 {
+    CS_RANGE("cs_step");
     if (!ctx || !io || !io->idx || !io->gpu || !io->host) return CS_EINVAL;
     if (!io->n_gpu_victims || !io->n_host_victims || !io->n_prefetch) return CS_EINVAL;
     if ((io->now_dev && (((uintptr_t)io->now_dev) & 3u)) || (io->n_events_dev && (((uintptr_t)io->n_events_dev) & 3u)))
@@ -454,6 +464,7 @@ int cs_get_model(cs_ctx *ctx, uint32_t *C_out, float *P_out, uint16_t *amax_out,
 
 int cs_import_state(cs_ctx *ctx, const uint32_t *C_in, const uint16_t *cur_in, uint32_t last_agent, cs_stream_t stream)
 {
+    CS_RANGE("cs_import_state");
     if (!ctx || !C_in || (((uintptr_t)C_in) & 3u) || (((uintptr_t)cur_in) & 1u)) return CS_EINVAL;
     return cs_launch_import(ctx, C_in, cur_in, last_agent, (cudaStream_t)stream);
 }
@@ -487,6 +498,7 @@ int cs_get_counters(cs_ctx *ctx, cs_counters *out, uint32_t reset, cs_stream_t s
 int cs_validate_selection(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, uint32_t prefetch, uint32_t tier,
                           uint32_t k, const uint32_t *ids_out, const uint32_t *n_out, cs_stream_t stream)
 {
+    CS_RANGE("cs_validate_selection");
     if (!ctx) return CS_EINVAL;
     int rc = check_index(ctx, idx);
     if (rc != CS_OK) return rc;
@@ -500,6 +512,7 @@ static bool list_ok(const uint32_t *p, uint32_t n) { return n == 0 || (p && !(((
 int cs_validate_move_lists(cs_ctx *ctx, const cs_kv_pool *src, const cs_kv_pool *dst, const uint32_t *src_slots,
                            const uint32_t *dst_slots, uint32_t n_max, const uint32_t *n_dev, cs_stream_t stream)
 {
+    CS_RANGE("cs_validate_move_lists");
     if (!ctx) return CS_EINVAL;
     int rc = check_pools(src, dst);
     if (rc != CS_OK) return rc;
@@ -519,6 +532,7 @@ int cs_validate_exchange_lists(cs_ctx *ctx, const cs_kv_pool *gpu, const cs_kv_p
                                const uint32_t *n_off_dev, const uint32_t *pre_host_slots, const uint32_t *pre_gpu_slots,
                                uint32_t n_pre_max, const uint32_t *n_pre_dev, cs_stream_t stream)
 {
+    CS_RANGE("cs_validate_exchange_lists");
     if (!ctx) return CS_EINVAL;
     int rc = check_pools(gpu, host);
     if (rc != CS_OK) return rc;
@@ -580,6 +594,7 @@ int cs_set_mover_path(cs_ctx *ctx, uint32_t path)
 
 int cs_exact_survival(cs_ctx *ctx, uint32_t a0, uint32_t n_steps, float *psurv_out, float *fsurv_out, cs_stream_t stream)
 {
+    CS_RANGE("cs_exact_survival");
     if (!ctx) return CS_EINVAL;
     if (a0 != CS_AGENT_NONE && a0 >= ctx->p.n_agents) return CS_EINVAL;
     if (n_steps > 4096) return CS_EINVAL;

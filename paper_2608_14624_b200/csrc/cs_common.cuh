@@ -5,6 +5,20 @@
 
 #include "cachescout.h"
 
+// NVTX ranges around the entry points that enqueue work: a timeline tool shows which library call a kernel belongs
+// to.  Header-only (NVTX 3 loads the tool's injection library on first use; without a tool a range costs a few
+// nanoseconds).  -DCS_NO_NVTX compiles the ranges out.
+#ifndef CS_NO_NVTX
+#include <nvtx3/nvToolsExt.h>
+struct cs_nvtx_range {
+    explicit cs_nvtx_range(const char *name) { nvtxRangePushA(name); }
+    ~cs_nvtx_range() { nvtxRangePop(); }
+};
+#define CS_RANGE(name) cs_nvtx_range cs_range_guard_(name)
+#else
+#define CS_RANGE(name) do { } while (0)
+#endif
+
 #if defined(__CUDA_ARCH__) && (__CUDA_ARCH__ < 1000)
 #error "libcachescout is written for sm_100a (B200) only"
 #endif

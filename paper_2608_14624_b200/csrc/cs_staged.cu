@@ -133,6 +133,7 @@ extern "C" int cs_exchange_blocks_staged(cs_ctx *ctx, const cs_kv_pool *gpu, con
                                          const uint32_t *pre_host_ids, const uint32_t *pre_gpu_slots, uint32_t n_pre,
                                          cs_stream_t stream)
 {
+    CS_RANGE("cs_exchange_blocks_staged");
     if (!ctx || !gpu || !host || !gpu->base || !host->base) return CS_EINVAL;
     if (gpu->n_layers != host->n_layers || gpu->n_kv_heads != host->n_kv_heads || gpu->head_dim != host->head_dim ||
         gpu->block_tokens != host->block_tokens || gpu->elem_bytes != host->elem_bytes || gpu->layout > 1)
