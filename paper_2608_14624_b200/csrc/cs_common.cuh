@@ -43,6 +43,7 @@ struct cs_nvtx_range {
 struct cs_scalars {
     uint32_t status;        // CS_ST_* bits
     uint32_t last_agent;    // agent of the last non-warmup event, CS_AGENT_NONE initially
+    uint32_t a_star;        // arg-max successor of last_agent (Eq. 10), ~0 while there is no current agent; kept by the refresh
     float R;                // Eq. 2
     uint32_t gate;          // Eq. 11: R >= r_min
     uint32_t n_transitions; // sum of all counts

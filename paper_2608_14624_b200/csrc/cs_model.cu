@@ -25,6 +25,7 @@ __global__ void cs_init_kernel(cs_workspace ws, uint32_t A, uint32_t n_chains, u
         cs_scalars z;
         memset(&z, 0, sizeof(z));
         z.last_agent = CS_AGENT_NONE;
+        z.a_star = 0xFFFFFFFFu;
         z.sel_hint[0] = z.sel_hint[1] = z.sel_hint[2] = z.sel_hint[3] = 0xFFFFFFFFu;
         *ws.sc = z;
     }
@@ -281,6 +282,7 @@ cs_normalise_kernel(cs_workspace ws, uint32_t A, uint32_t W, float eps, float ta
         const float Rf = (float)R;
         ws.sc->R = Rf;
         ws.sc->gate = (Rf >= r_min) ? 1u : 0u;
+        ws.sc->a_star = la < A ? (uint32_t)__ldcg(&ws.amax[la]) : 0xFFFFFFFFu;      // Eq. 10, for the prefetch ranking
         ws.sc->ticket0 = 0;
     }
     if (all_chains) {

@@ -140,22 +140,27 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_fast_kernel(SelArgs a, cs_
     __shared__ uint32_t s_part[SEL_THREADS];
     __shared__ uint32_t s_b0, s_ahead, s_above;
     __shared__ bool s_flag;
-    cs_wait_for_predecessor();
     cs_release_successor();
+    // Before waiting for the predecessor grid: everything that depends only on the context's constants and on the
+    // remembered bin (a stale bin would cost time, never correctness: the result does not depend on H).
     const uint32_t H = ws.sc->sel_hint[a.hint_slot];        // ~0: nothing remembered
+    Tables T;
+    const size_t table_words = ((size_t)(a.A + a.gtab_len) * 4 + (size_t)a.A * 2 + 15) / 16 * 4;
+    uint32_t *queues = (uint32_t *)smem + table_words;
+    const size_t cut_off_words = table_words + (size_t)(SEL_THREADS / 32) * (FQ_CAP + STAGE_CAP * 3) + 4;     // after queues and staging
+    if (H != 0xFFFFFFFFu) {
+        load_tables_static(a, ws, smem, T);
+        build_x_thresholds<PF>(a, H, s_xt);
+        for (uint32_t i = threadIdx.x; i < CS_HIST_BINS; i += blockDim.x) s_hist[i] = 0;
+        if (threadIdx.x == 0) s_above = 0;
+    }
+    cs_wait_for_predecessor();
     if (H == 0xFFFFFFFFu) {                                   // every CTA sees the same word
         if (blockIdx.x == 0 && threadIdx.x == 0) ws.sel->spec = 0;
         return;
     }
     resolve_now(a);
-    Tables T;
-    load_tables(a, ws, smem, T, PF && a.anchor);
-    const size_t table_words = ((size_t)(a.A + a.gtab_len) * 4 + (size_t)a.A * 2 + 15) / 16 * 4;
-    uint32_t *queues = (uint32_t *)smem + table_words;
-    const size_t cut_off_words = table_words + (size_t)(SEL_THREADS / 32) * (FQ_CAP + STAGE_CAP * 3) + 4;     // after queues and staging
-    build_x_thresholds<PF>(a, H, s_xt);
-    for (uint32_t i = threadIdx.x; i < CS_HIST_BINS; i += blockDim.x) s_hist[i] = 0;
-    if (threadIdx.x == 0) s_above = 0;
+    load_tables_dynamic(a, ws, T, PF && a.anchor);
     __syncthreads();
     // ---- the age cuts, one per agent, for blocks of the common size ----------------------------------------
     // victims: s_cut[agent] = number of ages (0, 1, ..) that are dismissed, i.e. for which fl(f g(age)) >= X;
@@ -222,11 +227,12 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_fast_kernel(SelArgs a, cs_
         for (uint32_t r = 0; r < rounds; ++r) {
             const uint32_t i = r * 32u + lane;
             bool cand = false;
-            uint32_t id = 0, ag = 0, la = 0, tok = a.block_tokens, dp = 0;
+            uint32_t id = 0, ag = 0, la = 0, tok = a.block_tokens, dp = 0, fl = 0;
             if (i < qn) {
                 id = q[i];
                 ag = __ldg(a.agent + id);
                 la = __ldg(a.la + id);
+                fl = __ldg(a.flags + id);                        // (needed by the key of a candidate: one round trip, not two)
                 if (a.ntok) tok = __ldg(a.ntok + id);
                 if (PF && a.anchor) dp = __ldg(a.depth + id);
                 bool elig = true;
@@ -242,7 +248,7 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_fast_kernel(SelArgs a, cs_
             }
             uint32_t pr = 0, se = 0;
             if (cand) {
-                entry_key_rest<PF>(a, T, &ws.sc->status, ag, dp, __ldg(a.flags + id), la, tok, pr, se);
+                entry_key_rest<PF>(a, T, &ws.sc->status, ag, dp, fl, la, tok, pr, se);
                 atomicAdd(&s_hist[pr >> 20], 1u);
             }
             // candidates gather in the warp's slice of shared memory and leave it 32 or more at a time
@@ -366,18 +372,10 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_fast_kernel(SelArgs a, cs_
         ws.hist[threadIdx.x * PER + qq] = 0;                 // ready for the next pass or call
         sum += loc[qq];
     }
-    s_part[threadIdx.x] = sum;
     if (threadIdx.x == 0) s_b0 = 0xFFFFFFFFu;
-    __syncthreads();
-    for (uint32_t d = 1; d < SEL_THREADS; d <<= 1) {         // inclusive scan
-        const uint32_t v = threadIdx.x >= d ? s_part[threadIdx.x - d] : 0;
-        __syncthreads();
-        s_part[threadIdx.x] += v;
-        __syncthreads();
-    }
-    const uint32_t below = s_part[SEL_THREADS - 1];          // eligible entries at or below H
+    uint32_t below;                                          // eligible entries at or below H
+    const uint32_t before = sel_block_scan(sum, s_part, below);
     const uint32_t total = below + __ldcg(&ws.sel->n_above);
-    const uint32_t before = s_part[threadIdx.x] - sum;
     if (a.k && below >= a.k && before < a.k && a.k <= before + sum) {
         uint32_t run = before;
 #pragma unroll
@@ -1056,6 +1054,7 @@ __global__ void cs_static_prepare_kernel(cs_workspace ws, uint32_t gtab_len, flo
         cs_scalars z;
         memset(&z, 0, sizeof(z));
         z.last_agent = CS_AGENT_NONE;
+        z.a_star = 0xFFFFFFFFu;
         z.sel_hint[0] = z.sel_hint[1] = z.sel_hint[2] = z.sel_hint[3] = 0xFFFFFFFFu;
         *ws.sc = z;
         cs_sel_state zs;

@@ -96,19 +96,30 @@ struct Tables {
     uint32_t a_star;
 };
 
-__device__ __forceinline__ void load_tables(const SelArgs &a, const cs_workspace &ws, float *smem, Tables &T,
-                                            bool want_anchor)
+// The recency table depends only on the context's constants (written when the context was created), so a kernel
+// launched with programmatic dependent launch may copy it before it waits for its predecessor ...
+__device__ __forceinline__ void load_tables_static(const SelArgs &a, const cs_workspace &ws, float *smem, Tables &T)
 {
     T.fsurv = smem;
     T.gtab = smem + a.A;
     T.anchor = (uint16_t *)(smem + a.A + a.gtab_len);
-    for (uint32_t i = threadIdx.x; i < a.A; i += blockDim.x) T.fsurv[i] = a.fsurv[i];
     for (uint32_t i = threadIdx.x; i < a.gtab_len; i += blockDim.x) T.gtab[i] = ws.gtab[i];
+    T.g_sat = cs_recency(a.lambda, a.delta, a.age_sat);
+}
+// ... while the survival table, the anchor lengths and a* may have been written by that predecessor.
+__device__ __forceinline__ void load_tables_dynamic(const SelArgs &a, const cs_workspace &ws, Tables &T, bool want_anchor)
+{
+    for (uint32_t i = threadIdx.x; i < a.A; i += blockDim.x) T.fsurv[i] = a.fsurv[i];
     if (want_anchor)
         for (uint32_t i = threadIdx.x; i < a.A; i += blockDim.x) T.anchor[i] = a.anchor[i];
-    T.g_sat = cs_recency(a.lambda, a.delta, a.age_sat);
-    const uint32_t la = ws.sc->last_agent;
-    T.a_star = (la < a.A) ? ws.amax[la] : 0xFFFFFFFFu;
+    T.a_star = ws.sc->a_star;           // arg-max successor of the current agent, kept by the learner refresh
+}
+
+__device__ __forceinline__ void load_tables(const SelArgs &a, const cs_workspace &ws, float *smem, Tables &T,
+                                            bool want_anchor)
+{
+    load_tables_static(a, ws, smem, T);
+    load_tables_dynamic(a, ws, T, want_anchor);
 }
 
 // Recency factor of Eq. 9 for an age: from the table, the saturated constant, or (a decay so slow that the
@@ -409,6 +420,35 @@ __device__ __forceinline__ bool last_cta_done(uint32_t *ticket, bool *s_flag)
     const bool last = *s_flag;
     if (last) __threadfence();
     return last;
+}
+
+// Exclusive prefix sum of one value per thread over a CTA of SEL_THREADS threads (warp shuffles, three barriers);
+// also returns the total.  s_part: at least 64 words.
+__device__ __forceinline__ uint32_t sel_block_scan(uint32_t v, uint32_t *s_part, uint32_t &total)
+{
+    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint32_t incl = v;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+        if (lane >= d) incl += t;
+    }
+    __syncthreads();
+    if (lane == 31) s_part[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+        uint32_t w = lane < (SEL_THREADS / 32) ? s_part[lane] : 0;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, w, d);
+            if (lane >= d) w += t;
+        }
+        s_part[32 + lane] = w;                         // inclusive warp totals
+    }
+    __syncthreads();
+    total = s_part[32 + SEL_THREADS / 32 - 1];
+    const uint32_t before = warp ? s_part[32 + warp - 1] : 0;
+    return before + incl - v;
 }
 
 __device__ __forceinline__ bool key_less(unsigned long long km_a, uint32_t id_a, unsigned long long km_b,
