@@ -15,8 +15,10 @@
  *    library never allocates or frees device or pinned memory; it owns only the small
  *    host-side cs_ctx, with a few CUDA events and two streams of its own (made by cs_create,
  *    released by cs_destroy; cs_step and cs_select_step fork onto them and join back, so callers
- *    see everything ordered on the streams they pass).  All scratch lives in the workspace the
- *    caller hands to cs_create().
+ *    see everything ordered on the streams they pass), plus five more streams and their events
+ *    once cs_set_mover_staging() has been called.  All scratch lives in the workspace the
+ *    caller hands to cs_create() (and, for the copy-engine transfers, in the ring handed to
+ *    cs_set_mover_staging()).
  *  - Block-index arrays, score / id output arrays and pool bases must be 16-byte aligned (the
  *    kernels use 128-bit accesses); event arrays, slot lists and counts need only their natural
  *    alignment.  A violation is CS_EINVAL before anything is launched.
