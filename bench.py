@@ -1331,6 +1331,7 @@ def measure_step_workload(args, w, ctx):
     x_gbps = x_bytes / (x_ms / 1e3) / 1e9
     # time a perfect duplex link would need for the step's bytes, from the one-direction peaks of this run
     ideal_ms = max(w.k_v * bb / link["d2h"], w.k_p * bb / link["h2d"]) / 1e6
+    ideal_ms *= x_bytes / float((w.k_v + w.k_p) * bb)    # a launch that found fewer eligible blocks moved fewer bytes
     named, backed = cfg.host_blocks, w.host_backed
     return {
         "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
