@@ -60,6 +60,7 @@ size_t cs_layout_workspace(const cs_params *p, uint32_t gtab_len, void *base, cs
     TAKE(rowH, double, A);
     TAKE(qfix, unsigned long long, A);
     TAKE(adj, uint32_t, A * W);
+    TAKE(adjT, uint32_t, 2 * A * W);
     TAKE(hops, uint16_t, A);
     TAKE(fsurv, float, A);
     TAKE(hops_tmp, uint16_t, A);

@@ -51,6 +51,7 @@ struct cs_scalars {
     uint32_t gtab_monotone; // the recency table covers every unsaturated age and never increases with age
     uint32_t status_read;   // cs_get_status(): the value swapped out of `status`
     uint32_t val_le, val_elig, val_ticket;   // cs_validate_selection(): keys at or below the last one, eligible entries, ticket
+    uint32_t adjT_cur;      // which copy of the transposed adjacency the last refresh filled
     uint32_t sel_hint[4];   // bin up to which the next select of each kind (GPU victims, host victims, prefetch)
                             // collects ahead of its own threshold, chosen from the previous call's histogram;
                             // ~0 = none; slot 3 is never written: calls that must not speculate read it
@@ -70,6 +71,9 @@ struct cs_sel_state {
     uint32_t c_spec;        // candidates appended by the fast pass; 0 between calls
     uint32_t n_above;       // eligible entries the fast pass found above the remembered bin; 0 between calls
     uint32_t spec;          // 1: the fast pass's candidates cover the k winners, the histogram and collect passes are skipped
+    uint32_t placed;        // 1: every bucket has a fixed region of `cap` keys in the sort arrays, filled by the bucket launch
+    uint32_t cap;           // keys per bucket region
+    uint32_t overflow;      // 1: a bucket outgrew its region; the scatter launch groups the buckets instead
     uint32_t cc[2];         // candidate counters of the cluster kernel: a call uses one and clears the other for the
                             // next call, so that the counter is zero on entry without a barrier
     uint32_t toggle;        // which of the two the next call uses; flipped by every call on the device, so that a
@@ -89,6 +93,8 @@ struct cs_workspace {
     double *rowH;         // [A] sum_j P_ij ln P_ij
     unsigned long long *qfix;   // [A] column sums of Eq. 2 in 2^-60 fixed point, zero between refreshes
     uint32_t *adj;        // [A*W] Eq. 7 adjacency, one bit per edge, W = ceil(A/32)
+    uint32_t *adjT;       // [2][A*W] its transpose (row v = the predecessors of v), two copies used in turn: a refresh
+                          // fills one with atomics and clears the other for the refresh after it
     uint16_t *hops;       // [A]
     float *fsurv;         // [A] p~ + delta for the cached source
     uint16_t *hops_tmp;   // [A] same, for cs_score_blocks() with explicit sources
@@ -204,6 +210,29 @@ static inline int cs_check_launch(cs_ctx *ctx)
 #ifndef CS_USE_PDL
 #define CS_USE_PDL 1
 #endif
+// Loads that stay where they are written.  The compiler is free to sink an ordinary load to its first use, which
+// turns "fetch sixteen words, then work on them" into sixteen round trips to L2, one after the other (measured:
+// 950 cycles each).  These can neither be sunk nor reordered against each other or against other memory
+// operations, so a run of them is in flight together and costs one round trip.
+__device__ __forceinline__ uint32_t cs_ld_cg_pinned(const uint32_t *p)
+{
+    uint32_t v;
+    asm volatile("ld.global.cg.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ uint2 cs_ld_cg_pinned(const uint2 *p)
+{
+    uint2 v;
+    asm volatile("ld.global.cg.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ ulonglong2 cs_ld_cg_pinned(const ulonglong2 *p)
+{
+    ulonglong2 v;
+    asm volatile("ld.global.cg.v2.u64 {%0, %1}, [%2];" : "=l"(v.x), "=l"(v.y) : "l"(p) : "memory");
+    return v;
+}
+
 __device__ __forceinline__ void cs_wait_for_predecessor()
 {
 #if CS_USE_PDL

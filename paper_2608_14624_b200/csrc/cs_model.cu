@@ -117,75 +117,134 @@ cs_observe_kernel(cs_workspace ws, uint32_t A, uint32_t n_chains, const uint32_t
 
 // ---------------------------------------------------------------------------------------------
 // BFS over the bit-matrix graph from a set of source bits, then Eq. 8.  Runs inside one CTA.
-// Level-synchronous: every thread owns a few nodes; a node of the current frontier ORs its
-// adjacency row into the next frontier (shared-memory atomics), so one level costs one round
-// trip to the adjacency matrix whatever the frontier size.  Thread w < W then retires word w.
-// s_front / s_visit / s_next: 32 words each.  The adjacency matrix is first copied into shared memory when it
-// fits (BFS_SMEM_WORDS; up to 512 agents), so that the levels cost no further trips to global memory.
+// s_front: 64 words (two frontiers, used in turn), s_visit / s_next: 32 words each, s_hops: one entry per agent.
+//
+// Up to one agent per thread the search PULLS: thread v holds row v of the TRANSPOSED adjacency matrix (the
+// predecessors of v; kept up to date in global memory by the refresh, fetched ahead of time into registers) and at
+// every level ANDs it with the frontier.  A level is then W broadcast loads and ANDs per node, all nodes in
+// parallel, one ballot per warp for the next frontier and ONE barrier -- whatever the frontier size, with no
+// atomics and no divergent loops.  (A push over the frontier's nodes by one warp was tried: lanes that walk
+// different frontier words run one after the other, 80 cycles per node.  So was a transpose built in shared memory
+// by this CTA: 3 us of shared-memory atomics.)
+// More agents take the level-synchronous push from global memory: a node of the current frontier ORs its adjacency
+// row into the next frontier (shared-memory atomics), two barriers per level.
 // ---------------------------------------------------------------------------------------------
-#define BFS_SMEM_WORDS 8192u
-__device__ void cs_bfs_survival(const uint32_t *__restrict__ adj, uint32_t A, uint32_t W, uint32_t *s_front,
-                                uint32_t *s_visit, uint32_t *s_next, uint32_t *s_adj, uint16_t *hops, float *fsurv,
-                                uint32_t e_max, float delta)
+#define BFS_ROW_WORDS 8u                   // words of a row when the search pulls (one agent per thread: 256 agents)
+struct BfsRow { uint32_t w[BFS_ROW_WORDS]; };
+__device__ __forceinline__ bool cs_bfs_pulls(uint32_t A) { return A <= ROW_THREADS; }
+
+// Row threadIdx.x of the transposed adjacency matrix, fetched so that the trip to global memory overlaps whatever
+// the caller does in between (zero where the search will not pull, or for a thread without a node).
+__device__ __forceinline__ void cs_bfs_load_row(const uint32_t *adjT, uint32_t A, uint32_t W, BfsRow &row)
 {
-    // on entry s_front[] holds the source bits (already synchronised by the caller)
+    if (!cs_bfs_pulls(A)) {
+#pragma unroll
+        for (uint32_t w = 0; w < BFS_ROW_WORDS; ++w) row.w[w] = 0u;
+        return;
+    }
+    const bool mine = threadIdx.x < A;
+    const uint32_t *r = adjT + (mine ? threadIdx.x * W : 0u);          // (always a valid address; unused words are masked)
+#pragma unroll
+    for (uint32_t w = 0; w < BFS_ROW_WORDS; ++w) row.w[w] = cs_ld_cg_pinned(r + (w < W ? w : 0u));
+#pragma unroll
+    for (uint32_t w = 0; w < BFS_ROW_WORDS; ++w)
+        if (!mine || w >= W) row.w[w] = 0u;
+}
+
+__device__ __forceinline__ void cs_bfs_survival(const uint32_t *__restrict__ adj, uint32_t A, uint32_t W, const BfsRow &rowT,
+                                                uint32_t *s_front, uint32_t *s_visit, uint32_t *s_next, uint16_t *s_hops,
+                                                uint16_t *hops, float *fsurv, uint32_t e_max, float delta)
+{
+    // on entry s_front[0 .. 32) holds the source bits and s_front[32 .. 64) zeroes (synchronised by the caller)
     const uint32_t tid = threadIdx.x;
-    const bool in_smem = A * W <= BFS_SMEM_WORDS;
-    if (in_smem)
-        for (uint32_t i = tid; i < A * W; i += blockDim.x) s_adj[i] = __ldcg(&adj[i]);
-    for (uint32_t a = tid; a < A; a += blockDim.x)
-        hops[a] = ((s_front[a >> 5] >> (a & 31)) & 1u) ? 0 : CS_HOP_NONE;
-    if (tid < W) { s_visit[tid] = s_front[tid]; s_next[tid] = 0; }
-    __syncthreads();
-    for (uint32_t level = 1; level <= A; ++level) {
-        for (uint32_t node = tid; node < A; node += blockDim.x) {
-            if ((s_front[node >> 5] >> (node & 31)) & 1u) {
-                for (uint32_t w = 0; w < W; ++w) {
-                    const uint32_t v = in_smem ? s_adj[node * W + w] : __ldcg(&adj[node * W + w]);
-                    if (v) atomicOr(&s_next[w], v);
+    if (cs_bfs_pulls(A)) {
+        const uint32_t v = tid;                                       // blockDim.x >= A
+        bool seen = v >= A || ((s_front[v >> 5] >> (v & 31)) & 1u);
+        uint32_t my_hops = (v < A && seen) ? 0u : CS_HOP_NONE;
+        for (uint32_t level = 1; level <= A; ++level) {
+            const uint32_t *cur = s_front + ((level & 1u) ? 0u : 32u);
+            uint32_t *nxt = s_front + ((level & 1u) ? 32u : 0u);
+            uint32_t hit = 0;
+#pragma unroll
+            for (uint32_t w = 0; w < BFS_ROW_WORDS; ++w) hit |= rowT.w[w] & cur[w];
+            const bool fresh = hit != 0u && !seen;
+            const uint32_t word = __ballot_sync(0xFFFFFFFFu, fresh);
+            if ((tid & 31u) == 0) nxt[tid >> 5] = word;
+            if (fresh) { seen = true; my_hops = level; }
+            if (!__syncthreads_or(fresh)) break;
+        }
+        if (v < A) s_hops[v] = (uint16_t)my_hops;
+    } else {
+        for (uint32_t a = tid; a < A; a += blockDim.x)
+            s_hops[a] = ((s_front[a >> 5] >> (a & 31)) & 1u) ? 0 : CS_HOP_NONE;
+        if (tid < W) { s_visit[tid] = s_front[tid]; s_next[tid] = 0; }
+        __syncthreads();
+        for (uint32_t level = 1; level <= A; ++level) {
+            for (uint32_t node = tid; node < A; node += blockDim.x) {
+                if ((s_front[node >> 5] >> (node & 31)) & 1u) {
+                    for (uint32_t w = 0; w < W; ++w) {
+                        const uint32_t v = __ldcg(&adj[node * W + w]);
+                        if (v) atomicOr(&s_next[w], v);
+                    }
                 }
             }
-        }
-        __syncthreads();
-        uint32_t acc = 0;
-        if (tid < W) {
-            acc = s_next[tid] & ~s_visit[tid];
-            s_next[tid] = 0;
-            s_front[tid] = acc;
-            s_visit[tid] |= acc;
-            uint32_t bits = acc;
-            while (bits) {
-                const uint32_t b2 = tid * 32 + (__ffs(bits) - 1);
-                bits &= bits - 1;
-                if (b2 < A) hops[b2] = (uint16_t)level;
+            __syncthreads();
+            uint32_t acc = 0;
+            if (tid < W) {
+                acc = s_next[tid] & ~s_visit[tid];
+                s_next[tid] = 0;
+                s_front[tid] = acc;
+                s_visit[tid] |= acc;
+                uint32_t bits = acc;
+                while (bits) {
+                    const uint32_t b2 = tid * 32 + (__ffs(bits) - 1);
+                    bits &= bits - 1;
+                    if (b2 < A) s_hops[b2] = (uint16_t)level;
+                }
             }
+            if (!__syncthreads_or(acc != 0)) break;
         }
-        if (!__syncthreads_or(acc != 0)) break;
     }
     __syncthreads();
     for (uint32_t a = tid; a < A; a += blockDim.x) {
-        const uint32_t h = hops[a];
+        const uint32_t h = s_hops[a];
         const uint32_t m = h < e_max ? h : e_max;          // CS_HOP_NONE > e_max by construction
         const double ptilde = 1.0 - (double)m / (double)e_max;
+        hops[a] = (uint16_t)h;
         fsurv[a] = (float)(ptilde + (double)delta);
     }
 }
 
-// Deterministic block reductions (fixed tree, so results do not depend on scheduling).
+// Deterministic block reductions: a fixed butterfly inside each warp, then the warp sums added in warp order, so the
+// result does not depend on scheduling.  s_red: one entry per warp (two for the pair form).
 template <typename T>
 __device__ T cs_block_sum(T v, T *s_red)
 {
-    const uint32_t tid = threadIdx.x;
+    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, d);
+    __syncthreads();                                       // an earlier result may still be being read
+    if (lane == 0) s_red[warp] = v;
     __syncthreads();
-    s_red[tid] = v;
-    __syncthreads();
-    for (uint32_t s = blockDim.x >> 1; s > 0; s >>= 1) {
-        if (tid < s) s_red[tid] += s_red[tid + s];
-        __syncthreads();
-    }
     T r = s_red[0];
-    __syncthreads();
+    for (uint32_t w = 1; w < n_warps; ++w) r += s_red[w];
     return r;
+}
+
+__device__ void cs_block_sum2(double &a, double &b, double *s_red)
+{
+    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) {
+        a += __shfl_xor_sync(0xFFFFFFFFu, a, d);
+        b += __shfl_xor_sync(0xFFFFFFFFu, b, d);
+    }
+    __syncthreads();
+    if (lane == 0) { s_red[warp] = a; s_red[32 + warp] = b; }
+    __syncthreads();
+    a = s_red[0];
+    b = s_red[32];
+    for (uint32_t w = 1; w < n_warps; ++w) { a += s_red[w]; b += s_red[32 + w]; }
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -197,11 +256,11 @@ __global__ void __launch_bounds__(ROW_THREADS)
 cs_normalise_kernel(cs_workspace ws, uint32_t A, uint32_t W, float eps, float tau, float r_min, uint32_t e_max,
                     float delta, uint32_t all_chains, uint32_t n_chains)
 {
-    __shared__ double s_red[ROW_THREADS];
-    __shared__ float s_bestv[ROW_THREADS];
-    __shared__ uint32_t s_besti[ROW_THREADS];
-    __shared__ uint32_t s_front[32], s_visit[32], s_next[32];
-    __shared__ uint32_t s_adj[BFS_SMEM_WORDS];
+    __shared__ double s_red[64];
+    __shared__ float s_bestv[ROW_THREADS / 32];
+    __shared__ uint32_t s_besti[ROW_THREADS / 32];
+    __shared__ uint32_t s_front[64], s_visit[32], s_next[32];
+    __shared__ uint16_t s_hops[CS_MAX_AGENTS];
     __shared__ bool s_is_last;
     const uint32_t tid = threadIdx.x;
     cs_wait_for_predecessor();
@@ -211,6 +270,8 @@ cs_normalise_kernel(cs_workspace ws, uint32_t A, uint32_t W, float eps, float ta
     // point with integer atomics: integer addition commutes, so the sum is bit-identical from run
     // to run whatever order the CTAs finish in (a float atomic would not be).
     const uint32_t n_total = ws.sc->n_transitions;
+    const uint32_t fill = ws.sc->adjT_cur ^ 1u;              // every CTA reads this before the last one flips it
+    uint32_t *adjT_fill = ws.adjT + (size_t)fill * A * W, *adjT_clear = ws.adjT + (size_t)(fill ^ 1u) * A * W;
     const double inv_total = n_total ? 1.0 / (double)n_total : 0.0;
     for (uint32_t i = blockIdx.x; i < A; i += gridDim.x) {
         const uint32_t n_i = ws.rowsum[i];
@@ -233,22 +294,33 @@ cs_normalise_kernel(cs_workspace ws, uint32_t A, uint32_t W, float eps, float ta
             }
             const uint32_t bits = __ballot_sync(0xFFFFFFFFu, edge);
             if ((tid & 31) == 0 && (j >> 5) < W) ws.adj[i * W + (j >> 5)] = bits;
+            if (edge) atomicOr(&adjT_fill[j * W + (i >> 5)], 1u << (i & 31));      // the transpose: i precedes j
         }
-        // arg-max: max value, then min index
-        s_bestv[tid] = bestv;
-        s_besti[tid] = besti;
+        for (uint32_t w = tid; w < W; w += ROW_THREADS) adjT_clear[i * W + w] = 0;  // for the refresh after this one
+        // arg-max (max value, then min index) and the entropy term: a butterfly inside each warp, then the warp results
+        // combined in warp order by thread 0
+        const uint32_t lane = tid & 31, warp = tid >> 5;
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) {
+            const float v = __shfl_xor_sync(0xFFFFFFFFu, bestv, d);
+            const uint32_t x = __shfl_xor_sync(0xFFFFFFFFu, besti, d);
+            if (v > bestv || (v == bestv && x < besti)) { bestv = v; besti = x; }
+            h += __shfl_xor_sync(0xFFFFFFFFu, h, d);
+        }
+        __syncthreads();                                         // the partials of the row before have been read
+        if (lane == 0) { s_bestv[warp] = bestv; s_besti[warp] = besti; s_red[warp] = h; }
         __syncthreads();
-        for (uint32_t s = ROW_THREADS >> 1; s > 0; s >>= 1) {
-            if (tid < s) {
-                const float v = s_bestv[tid + s];
-                const uint32_t x = s_besti[tid + s];
-                if (v > s_bestv[tid] || (v == s_bestv[tid] && x < s_besti[tid])) { s_bestv[tid] = v; s_besti[tid] = x; }
+        if (tid == 0) {
+            float bv = s_bestv[0];
+            uint32_t bi = s_besti[0];
+            double hs = s_red[0];
+            for (uint32_t w = 1; w < ROW_THREADS / 32; ++w) {
+                if (s_bestv[w] > bv || (s_bestv[w] == bv && s_besti[w] < bi)) { bv = s_bestv[w]; bi = s_besti[w]; }
+                hs += s_red[w];
             }
-            __syncthreads();
+            ws.amax[i] = (uint16_t)bi;
+            ws.rowH[i] = hs;
         }
-        if (tid == 0) ws.amax[i] = (uint16_t)s_besti[0];
-        const double hsum = cs_block_sum<double>(h, s_red);
-        if (tid == 0) ws.rowH[i] = hsum;
     }
 
     // ---- last CTA done: global quantities ---------------------------------------------------------
@@ -262,6 +334,10 @@ cs_normalise_kernel(cs_workspace ws, uint32_t A, uint32_t W, float eps, float ta
     if (!s_is_last) return;
     __threadfence();
 
+    BfsRow rowT;                                                         // in flight during the sums
+    cs_bfs_load_row(adjT_fill, A, W, rowT);
+    const uint32_t la = __ldcg(&ws.sc->last_agent);
+    if (tid < 64) s_front[tid] = (tid < 32 && !all_chains && la < A && (la >> 5) == tid) ? (1u << (la & 31)) : 0u;
     const uint32_t N = __ldcg(&ws.sc->n_transitions);
     double Hc = 0.0, Hm = 0.0;
     if (N > 0) {
@@ -273,9 +349,7 @@ cs_normalise_kernel(cs_workspace ws, uint32_t A, uint32_t W, float eps, float ta
         }
     }
     for (uint32_t j = tid; j < A; j += ROW_THREADS) ws.qfix[j] = 0;      // ready for the next refresh
-    Hc = cs_block_sum<double>(Hc, s_red);
-    Hm = cs_block_sum<double>(Hm, s_red);
-    const uint32_t la = __ldcg(&ws.sc->last_agent);
+    cs_block_sum2(Hc, Hm, s_red);                                        // (its barriers also order s_front's zeroes)
     if (tid == 0) {
         double R = 0.0;
         if (N > 0 && Hm > 0.0) R = 1.0 - Hc / Hm;
@@ -283,21 +357,18 @@ cs_normalise_kernel(cs_workspace ws, uint32_t A, uint32_t W, float eps, float ta
         ws.sc->R = Rf;
         ws.sc->gate = (Rf >= r_min) ? 1u : 0u;
         ws.sc->a_star = la < A ? (uint32_t)__ldcg(&ws.amax[la]) : 0xFFFFFFFFu;      // Eq. 10, for the prefetch ranking
+        ws.sc->adjT_cur = fill;
         ws.sc->ticket0 = 0;
     }
     if (all_chains) {
         // sources: the current agent of every chain that has one (all live sessions)
-        if (tid < 32) s_front[tid] = 0;
-        __syncthreads();
         for (uint32_t ch = tid; ch < n_chains; ch += ROW_THREADS) {
             const uint32_t a = __ldcg(&ws.cur[ch]);
             if (a < A) atomicOr(&s_front[a >> 5], 1u << (a & 31));
         }
-    } else if (tid < 32) {
-        s_front[tid] = (la < A && (la >> 5) == tid) ? (1u << (la & 31)) : 0u;
     }
     __syncthreads();
-    cs_bfs_survival(ws.adj, A, W, s_front, s_visit, s_next, s_adj, ws.hops, ws.fsurv, e_max, delta);
+    cs_bfs_survival(ws.adj, A, W, rowT, s_front, s_visit, s_next, s_hops, ws.hops, ws.fsurv, e_max, delta);
 }
 
 // BFS + Eq. 8 from explicit sources into the temporary tables (cs_score_blocks with sources).
@@ -305,10 +376,12 @@ __global__ void __launch_bounds__(ROW_THREADS)
 cs_survival_kernel(cs_workspace ws, uint32_t A, uint32_t W, const uint16_t *__restrict__ sources, uint32_t n_sources,
                    uint32_t e_max, float delta)
 {
-    __shared__ uint32_t s_front[32], s_visit[32], s_next[32];
-    __shared__ uint32_t s_adj[BFS_SMEM_WORDS];
+    __shared__ uint32_t s_front[64], s_visit[32], s_next[32];
+    __shared__ uint16_t s_hops[CS_MAX_AGENTS];
     const uint32_t tid = threadIdx.x;
-    if (tid < 32) s_front[tid] = 0;
+    BfsRow rowT;
+    cs_bfs_load_row(ws.adjT + (size_t)ws.sc->adjT_cur * A * W, A, W, rowT);
+    if (tid < 64) s_front[tid] = 0;
     __syncthreads();
     for (uint32_t s = tid; s < n_sources; s += ROW_THREADS) {
         const uint32_t a = sources[s];
@@ -316,7 +389,7 @@ cs_survival_kernel(cs_workspace ws, uint32_t A, uint32_t W, const uint16_t *__re
         else atomicOr(&ws.sc->status, CS_ST_BAD_SOURCE);
     }
     __syncthreads();
-    cs_bfs_survival(ws.adj, A, W, s_front, s_visit, s_next, s_adj, ws.hops_tmp, ws.fsurv_tmp, e_max, delta);
+    cs_bfs_survival(ws.adj, A, W, rowT, s_front, s_visit, s_next, s_hops, ws.hops_tmp, ws.fsurv_tmp, e_max, delta);
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -68,28 +68,41 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_score_kernel(SelArgs a, cs_wor
 }
 
 // ---------------------------------------------------------------------------------------------
-// Sample sort set-up, run by one CTA once every candidate is in the buffer: sort <= 1024 sampled
-// keys in shared memory, publish <= 255 splitters, clear the bucket counters.
+// Sample sort set-up, run by one CTA (or half of one) once every candidate is in the buffer: sort P <= 1024 sampled
+// keys in shared memory, publish <= 255 splitters, clear the bucket counters, and decide where the buckets will
+// live.  When the candidates are few for the size of the sort region (8 c <= its capacity), every bucket gets a
+// fixed region of `cap` keys -- at least eight times the mean bucket -- that the bucket launch fills directly.
+// P: power of two, 64 <= P <= min(CS_SAMPLE, 2 * threads of the group).
 // ---------------------------------------------------------------------------------------------
+#define RANK_TILE 2048u                 // keys of the shared-memory tile a bucket is sorted in
+#define CS_SPLIT_SAMPLE_MAX 32768u      // up to this many candidates half a CTA sorts a 512-key sample (fast pass)
 __device__ __forceinline__ void publish_splitters(const cs_workspace &ws, unsigned long long *s_km, uint32_t *s_id,
-                                                  uint32_t c)
+                                                  uint32_t c, uint32_t sort_cap, uint32_t P, const CtaPart &cp)
 {
-    const uint32_t n_samp = c < CS_SAMPLE ? c : CS_SAMPLE;
-    for (uint32_t i = threadIdx.x; i < CS_SAMPLE; i += blockDim.x) {
-        if (i < n_samp) {
-            const uint32_t pos = (uint32_t)(((unsigned long long)i * c) / n_samp);
-            s_km[i] = __ldcg(&ws.cand_km[pos]);
-            s_id[i] = __ldcg(&ws.cand_id[pos]);
-        } else {
-            s_km[i] = ~0ull;
-            s_id[i] = 0xFFFFFFFFu;
+    const uint32_t n_samp = c < P ? c : P;
+    {
+        // a group sorts two keys per thread: both are fetched before either is stored
+        const uint32_t i0 = cp.t, i1 = cp.t + cp.n;
+        unsigned long long k0 = ~0ull, k1 = ~0ull;
+        uint32_t d0 = 0xFFFFFFFFu, d1 = 0xFFFFFFFFu;
+        if (i0 < n_samp) {
+            const uint32_t pos = (uint32_t)(((unsigned long long)i0 * c) / n_samp);
+            k0 = __ldcg(&ws.cand_km[pos]);
+            d0 = __ldcg(&ws.cand_id[pos]);
         }
+        if (i1 < n_samp) {
+            const uint32_t pos = (uint32_t)(((unsigned long long)i1 * c) / n_samp);
+            k1 = __ldcg(&ws.cand_km[pos]);
+            d1 = __ldcg(&ws.cand_id[pos]);
+        }
+        if (i0 < P) { s_km[i0] = k0; s_id[i0] = d0; }
+        if (i1 < P) { s_km[i1] = k1; s_id[i1] = d1; }
     }
-    __syncthreads();
-    bitonic_sort_fast(s_km, s_id, CS_SAMPLE);            // 512 threads, two keys each
+    part_sync(cp);
+    bitonic_sort_fast(s_km, s_id, P, cp);
     uint32_t n_spl = c / 64;
     if (n_spl > CS_MAX_SPLITTERS) n_spl = CS_MAX_SPLITTERS;
-    for (uint32_t j = threadIdx.x; j <= CS_MAX_SPLITTERS; j += blockDim.x) {
+    for (uint32_t j = cp.t; j <= CS_MAX_SPLITTERS; j += cp.n) {
         if (j < n_spl) {
             const uint32_t q = (uint32_t)(((unsigned long long)(j + 1) * n_samp) / (n_spl + 1));
             ws.spl_km[j] = s_km[q];
@@ -97,7 +110,14 @@ __device__ __forceinline__ void publish_splitters(const cs_workspace &ws, unsign
         }
         ws.bcount[j] = 0;
     }
-    if (threadIdx.x == 0) ws.sel->n_spl = n_spl;
+    if (cp.t == 0) {
+        uint32_t cap = sort_cap / (n_spl + 1u);
+        if (cap > RANK_TILE) cap = RANK_TILE;
+        ws.sel->n_spl = n_spl;
+        ws.sel->placed = (c && 8ull * c <= sort_cap) ? 1u : 0u;
+        ws.sel->cap = cap;
+        ws.sel->overflow = 0;
+    }
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -363,53 +383,73 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_fast_kernel(SelArgs a, cs_
     if (threadIdx.x == 0 && s_above) atomicAdd(&ws.sel->n_above, s_above);
     if (!last_cta_done(&ws.sel->ticket[0], &s_flag)) return;
 
-    // ---- last CTA: is the k-th smallest key within the remembered bin? ---------------------------------
-    constexpr uint32_t PER = CS_HIST_BINS / SEL_THREADS;
-    uint32_t loc[PER], sum = 0;
+    // ---- last CTA -----------------------------------------------------------------------------------------
+    // Two things are left and neither needs the other: whether the k-th smallest key lies within the remembered
+    // bin (a scan of the histogram), and the splitters for ordering the candidates (a sort of a sample of them).
+    // With few candidates half of the CTA is enough for the sample, so the two halves do one each, side by side;
+    // the sample sort is then wasted on a miss, which costs nothing on the critical path.
+    constexpr uint32_t HALF = SEL_THREADS / 2;
+    const uint32_t c_spec = __ldcg(&ws.sel->c_spec);
+    const uint32_t c_use = a.k ? c_spec : 0u;
+    const bool small = c_use <= CS_SPLIT_SAMPLE_MAX;
+    unsigned long long *s_km = (unsigned long long *)(((uintptr_t)queues + 7) & ~(uintptr_t)7);   // the queues are idle now
+    uint32_t *s_id = (uint32_t *)(s_km + CS_SAMPLE);
+    if (threadIdx.x >= HALF) {
+        if (small) publish_splitters(ws, s_km, s_id, c_use, a.sort_cap, CS_SAMPLE / 2, CtaPart{threadIdx.x - HALF, HALF, 2u});
+    } else {
+        const CtaPart cp{threadIdx.x, HALF, 1u};
+        constexpr uint32_t PER = CS_HIST_BINS / HALF;
+        uint32_t loc[PER], sum = 0;
+        {
+            uint4 *h4 = (uint4 *)(ws.hist + threadIdx.x * PER);
 #pragma unroll
-    for (uint32_t qq = 0; qq < PER; ++qq) {
-        loc[qq] = __ldcg(&ws.hist[threadIdx.x * PER + qq]);
-        ws.hist[threadIdx.x * PER + qq] = 0;                 // ready for the next pass or call
-        sum += loc[qq];
-    }
-    if (threadIdx.x == 0) s_b0 = 0xFFFFFFFFu;
-    uint32_t below;                                          // eligible entries at or below H
-    const uint32_t before = sel_block_scan(sum, s_part, below);
-    const uint32_t total = below + __ldcg(&ws.sel->n_above);
-    if (a.k && below >= a.k && before < a.k && a.k <= before + sum) {
-        uint32_t run = before;
+            for (uint32_t qq = 0; qq < PER / 4; ++qq) {
+                const uint4 v = __ldcg(h4 + qq);
+                h4[qq] = make_uint4(0u, 0u, 0u, 0u);             // ready for the next pass or call
+                loc[4 * qq] = v.x; loc[4 * qq + 1] = v.y; loc[4 * qq + 2] = v.z; loc[4 * qq + 3] = v.w;
+                sum += v.x + v.y + v.z + v.w;
+            }
+        }
+        if (threadIdx.x == 0) s_b0 = 0xFFFFFFFFu;
+        uint32_t below;                                          // eligible entries at or below H
+        const uint32_t before = sel_block_scan(sum, s_part, below, cp);
+        const uint32_t total = below + __ldcg(&ws.sel->n_above);
+        if (a.k && below >= a.k && before < a.k && a.k <= before + sum) {
+            uint32_t run = before;
 #pragma unroll
-        for (uint32_t qq = 0; qq < PER; ++qq) {
-            run += loc[qq];
-            if (run >= a.k) { s_b0 = threadIdx.x * PER + qq; break; }
+            for (uint32_t qq = 0; qq < PER; ++qq) {
+                run += loc[qq];
+                if (run >= a.k) { s_b0 = threadIdx.x * PER + qq; break; }
+            }
+        }
+        part_sync(cp);
+        // complete when the k winners lie at or below H, when fewer than k entries are eligible and all of them do, or when k = 0
+        const bool hit = a.k == 0 || below >= a.k || below == total;
+        const uint32_t b0 = a.k == 0 ? 0xFFFFFFFFu : (s_b0 != 0xFFFFFFFFu ? s_b0 : (H < CS_HIST_BINS ? H : CS_HIST_BINS - 1));
+        uint32_t ahead = 0;
+        const bool have_b0 = a.k && below >= a.k;
+        if (hit && have_b0) {
+            ahead = collect_ahead_limit<PER>(loc, threadIdx.x * PER, before, a.k, b0, &s_ahead, cp);
+            if (ahead > H) ahead = H;                             // nothing is known about the bins above H
+        }
+        if (threadIdx.x == 0) {
+            s_flag = hit;
+            if (hit) {
+                ws.sel->b0 = b0;
+                ws.sel->n_elig = total;
+                ws.sel->n_out = total < a.k ? total : a.k;
+                ws.sel->c = c_use;
+                count_select(ws, a.kind, total, total < a.k ? total : a.k);
+                count_candidates(ws, a.kind, c_use, true);
+                // fewer eligible entries than k: keep H; otherwise tighten it to what the histogram allows
+                if (have_b0) remember_threshold(ws.sc, a.hint_slot, true, ahead);
+            }
         }
     }
     __syncthreads();
-    // complete when the k winners lie at or below H, when fewer than k entries are eligible and all of them do, or when k = 0
-    const bool hit = a.k == 0 || below >= a.k || below == total;
-    const uint32_t b0 = a.k == 0 ? 0xFFFFFFFFu : (s_b0 != 0xFFFFFFFFu ? s_b0 : (H < CS_HIST_BINS ? H : CS_HIST_BINS - 1));
-    uint32_t ahead = 0;
-    const bool have_b0 = a.k && below >= a.k;
-    if (hit && have_b0) {
-        ahead = collect_ahead_limit<PER>(loc, threadIdx.x * PER, before, a.k, b0, &s_ahead);
-        if (ahead > H) ahead = H;                             // nothing is known about the bins above H
-    }
-    const uint32_t c_spec = __ldcg(&ws.sel->c_spec);
-    if (hit) {                                                // the queues are idle now: they hold the sample
-        unsigned long long *s_km = (unsigned long long *)(((uintptr_t)queues + 7) & ~(uintptr_t)7);
-        publish_splitters(ws, s_km, (uint32_t *)(s_km + CS_SAMPLE), a.k ? c_spec : 0u);
-    }
+    const bool hit = s_flag;
+    if (hit && !small) publish_splitters(ws, s_km, s_id, c_use, a.sort_cap, CS_SAMPLE, whole_cta());
     if (threadIdx.x == 0) {
-        if (hit) {
-            ws.sel->b0 = b0;
-            ws.sel->n_elig = total;
-            ws.sel->n_out = total < a.k ? total : a.k;
-            ws.sel->c = a.k ? c_spec : 0u;
-            count_select(ws, a.kind, total, total < a.k ? total : a.k);
-            count_candidates(ws, a.kind, a.k ? c_spec : 0u, true);
-            // fewer eligible entries than k: keep H; otherwise tighten it to what the histogram allows
-            if (have_b0) remember_threshold(ws.sc, a.hint_slot, true, ahead);
-        }
         ws.sel->spec = hit ? 1u : 0u;
         ws.sel->c_spec = 0;
         ws.sel->n_above = 0;
@@ -488,7 +528,7 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_hist_kernel(SelArgs a, cs_
     __syncthreads();
     const uint32_t b0 = s_b0;
     const bool have_b0 = a.k && total >= a.k;
-    const uint32_t ahead = have_b0 ? collect_ahead_limit<PER>(loc, threadIdx.x * PER, before, a.k, b0, &s_ahead) : 0u;
+    const uint32_t ahead = have_b0 ? collect_ahead_limit<PER>(loc, threadIdx.x * PER, before, a.k, b0, &s_ahead, whole_cta()) : 0u;
     if (threadIdx.x == 0) {
         ws.sel->b0 = b0;
         ws.sel->n_elig = total;
@@ -649,47 +689,138 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_collect_kernel(SelArgs a, 
     if (!last_cta_done(&ws.sel->ticket[2], &s_flag)) return;
 
     // ---- last CTA: sample, sort the sample (bitonic, shared memory), publish splitters -----------
-    publish_splitters(ws, s_km, s_id, __ldcg(&ws.sel->c));
+    publish_splitters(ws, s_km, s_id, __ldcg(&ws.sel->c), a.sort_cap, CS_SAMPLE, whole_cta());
     if (threadIdx.x == 0) { ws.sel->ticket[2] = 0; count_candidates(ws, a.kind, __ldcg(&ws.sel->c), false); }
 }
 
 // ---------------------------------------------------------------------------------------------
-// 3 bucket (+ offsets)
+// Sorts the first m <= RANK_TILE keys of a shared-memory tile ascending (bitonic; m is padded to a power of two
+// with keys that sort last).  Whole CTA.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void sort_tile(unsigned long long *t_km, uint32_t *t_id, uint32_t m)
+{
+    uint32_t P = 64;
+    while (P < m) P <<= 1;
+    for (uint32_t i = m + threadIdx.x; i < P; i += blockDim.x) { t_km[i] = ~0ull; t_id[i] = 0xFFFFFFFFu; }
+    __syncthreads();
+    if (P <= 2 * blockDim.x) {
+        bitonic_sort_fast(t_km, t_id, P, whole_cta());
+        return;
+    }
+    for (uint32_t size = 2; size <= P; size <<= 1) {
+        for (uint32_t stride = size >> 1; stride > 0; stride >>= 1) {
+            for (uint32_t t = threadIdx.x; t < P / 2; t += blockDim.x) {
+                const uint32_t lo = 2 * t - (t & (stride - 1));
+                const uint32_t hi = lo + stride;
+                const bool up = (lo & size) == 0;
+                const unsigned long long ka = t_km[lo], kb = t_km[hi];
+                const uint32_t ia = t_id[lo], ib = t_id[hi];
+                if (key_less(kb, ib, ka, ia) == up) {
+                    t_km[lo] = kb; t_id[lo] = ib;
+                    t_km[hi] = ka; t_id[hi] = ia;
+                }
+            }
+            __syncthreads();
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Exclusive prefix sum of the bucket sizes, computed by every CTA that needs it (256 counters, L2-resident):
+// s_off[b] = first output position of bucket b, s_off[256] = candidates in all buckets.  Also returns the last
+// bucket that holds one of the n_out winners (0 when n_out = 0).  Whole CTA of 256 threads.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t bucket_offsets(const cs_workspace &ws, uint32_t n_spl, uint32_t n_out, uint32_t *s_off,
+                                                   uint32_t *s_tmp)
+{
+    const uint32_t t = threadIdx.x, lane = t & 31, warp = t >> 5;
+    const uint32_t mine = t <= n_spl ? __ldcg(&ws.bcount[t]) : 0u;
+    uint32_t incl = mine;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+        if (lane >= d) incl += v;
+    }
+    if (t == 0) s_tmp[8] = 0;
+    if (lane == 31) s_tmp[warp] = incl;
+    __syncthreads();
+    uint32_t before = 0;
+#pragma unroll
+    for (uint32_t w = 0; w < 8; ++w) before += w < warp ? s_tmp[w] : 0u;
+    const uint32_t excl = before + incl - mine;
+    s_off[t] = excl;
+    if (t == 255) s_off[256] = excl + mine;
+    if (n_out && mine && excl <= n_out - 1 && n_out - 1 < excl + mine) s_tmp[8] = t;
+    __syncthreads();
+    return s_tmp[8];
+}
+
+// ---------------------------------------------------------------------------------------------
+// 3 bucket
+//
+// Each candidate finds its bucket by binary search over the splitters and takes a slot in it.
+// Roomy case (few candidates for the size of the sort region): the slot comes straight from one atomic on the
+// bucket's counter and the key is written to slot `slot` of the bucket's own fixed-size region, so that the
+// buckets are ready for the rank launch and the scatter launch has nothing to do.  A bucket that outgrows its
+// region sets `overflow`: bucket and slot of every candidate are recorded as well, and the scatter and rank
+// launches then take the general route.
+// General case: per round a CTA takes 1024 candidates, counts them per bucket in shared memory and reserves the
+// CTA's range in each non-empty bucket with one global atomic; bucket and slot are recorded for the scatter launch.
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) cs_sel_bucket_kernel(cs_workspace ws)
 {
     __shared__ unsigned long long s_km[CS_MAX_SPLITTERS + 1];
     __shared__ uint32_t s_id[CS_MAX_SPLITTERS + 1];
-    __shared__ uint32_t s_scan[CS_MAX_SPLITTERS + 1];
-    __shared__ bool s_flag;
     __shared__ uint32_t s_cnt[CS_MAX_SPLITTERS + 1], s_base[CS_MAX_SPLITTERS + 1];
-    constexpr int ITEMS = 4;                                  // candidates per thread and reservation round
+    constexpr int ITEMS = 4;                                  // candidates per thread and round
     cs_wait_for_predecessor();
     cs_release_successor();
-    const uint32_t c = ws.sel->c, n_spl = ws.sel->n_spl;
+    const uint32_t c = ws.sel->c, n_spl = ws.sel->n_spl, placed = ws.sel->placed, cap = ws.sel->cap;
     for (uint32_t j = threadIdx.x; j < n_spl; j += blockDim.x) { s_km[j] = ws.spl_km[j]; s_id[j] = ws.spl_id[j]; }
     s_cnt[threadIdx.x] = 0;
     __syncthreads();
-    // Per round a CTA takes 1024 candidates: each finds its bucket and a CTA-local slot (shared-memory
-    // atomics), then one global atomic per non-empty bucket reserves the CTA's range in that bucket.
     for (uint32_t base = blockIdx.x * (256 * ITEMS); base < c; base += gridDim.x * (256 * ITEMS)) {
-        uint32_t bkt[ITEMS], loc[ITEMS];
+        unsigned long long km[ITEMS];
+        uint32_t id[ITEMS], bkt[ITEMS], loc[ITEMS];
+#pragma unroll
+        for (int u = 0; u < ITEMS; ++u) {                     // all of the round's keys are fetched before any is used
+            const uint32_t i = base + u * 256 + threadIdx.x;
+            km[u] = i < c ? __ldcg(&ws.cand_km[i]) : 0ull;
+            id[u] = i < c ? __ldcg(&ws.cand_id[i]) : 0u;
+        }
 #pragma unroll
         for (int u = 0; u < ITEMS; ++u) {
             const uint32_t i = base + u * 256 + threadIdx.x;
             bkt[u] = 0xFFFFFFFFu;
             if (i < c) {
-                const unsigned long long km = ws.cand_km[i];
-                const uint32_t id = ws.cand_id[i];
                 uint32_t lo = 0, hi = n_spl;                 // bucket = number of splitters <= key
                 while (lo < hi) {
                     const uint32_t mid = (lo + hi) >> 1;
-                    if (key_less(km, id, s_km[mid], s_id[mid])) hi = mid;
+                    if (key_less(km[u], id[u], s_km[mid], s_id[mid])) hi = mid;
                     else lo = mid + 1;
                 }
                 bkt[u] = lo;
-                loc[u] = atomicAdd(&s_cnt[lo], 1u);
+                if (!placed) loc[u] = atomicAdd(&s_cnt[lo], 1u);
             }
+        }
+        if (placed) {
+#pragma unroll
+            for (int u = 0; u < ITEMS; ++u)                   // the round's atomics are in flight together
+                if (bkt[u] != 0xFFFFFFFFu) loc[u] = atomicAdd(&ws.bcount[bkt[u]], 1u);
+#pragma unroll
+            for (int u = 0; u < ITEMS; ++u) {
+                const uint32_t i = base + u * 256 + threadIdx.x;
+                if (bkt[u] == 0xFFFFFFFFu) continue;
+                ws.cand_bkt[i] = bkt[u];
+                ws.cand_slot[i] = loc[u];
+                if (loc[u] < cap) {
+                    ws.sort_km[(size_t)bkt[u] * cap + loc[u]] = km[u];
+                    ws.sort_id[(size_t)bkt[u] * cap + loc[u]] = id[u];
+                } else {
+                    ws.sel->overflow = 1;
+                }
+            }
+            continue;
         }
         __syncthreads();
         {
@@ -708,44 +839,21 @@ __global__ void __launch_bounds__(256) cs_sel_bucket_kernel(cs_workspace ws)
         }
         __syncthreads();
     }
-    if (!last_cta_done(&ws.sel->ticket[3], &s_flag)) return;
-
-    // ---- last CTA: exclusive prefix sum of the bucket sizes; last bucket needed ----------------------
-    const uint32_t t = threadIdx.x;                          // blockDim.x == 256 == buckets
-    const uint32_t mine = (t <= n_spl) ? __ldcg(&ws.bcount[t]) : 0u;
-    s_scan[t] = mine;
-    __syncthreads();
-    for (uint32_t d = 1; d < 256; d <<= 1) {
-        const uint32_t v = t >= d ? s_scan[t - d] : 0;
-        __syncthreads();
-        s_scan[t] += v;
-        __syncthreads();
-    }
-    const uint32_t excl = s_scan[t] - mine;
-    ws.boff[t] = excl;
-    if (t == 255) ws.boff[256] = s_scan[255];
-    const uint32_t n_out = ws.sel->n_out;
-    if (n_out == 0) {
-        if (t == 0) { ws.sel->b_last = 0; ws.sel->p_end = 0; }
-    } else if (mine && excl <= n_out - 1 && n_out - 1 < excl + mine) {
-        ws.sel->b_last = t;
-        ws.sel->p_end = excl + mine;
-    }
-    if (t == 0) ws.sel->ticket[3] = 0;
 }
 
 // ---------------------------------------------------------------------------------------------
-// 4 scatter
+// 4 scatter (general case only: candidates of the needed buckets are grouped by bucket)
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) cs_sel_scatter_kernel(cs_workspace ws)
 {
-    __shared__ uint32_t s_off[CS_MAX_SPLITTERS + 1];
+    __shared__ uint32_t s_off[CS_MAX_SPLITTERS + 2];
+    __shared__ uint32_t s_tmp[16];
     cs_wait_for_predecessor();
     cs_release_successor();
-    const uint32_t c = ws.sel->c, b_last = ws.sel->b_last;
-    if (ws.sel->p_end == 0) return;
-    s_off[threadIdx.x] = ws.boff[threadIdx.x];
-    __syncthreads();
+    if (ws.sel->placed && !ws.sel->overflow) return;         // the buckets are in their regions already
+    const uint32_t c = ws.sel->c, n_out = ws.sel->n_out;
+    if (n_out == 0) return;
+    const uint32_t b_last = bucket_offsets(ws, ws.sel->n_spl, n_out, s_off, s_tmp);
     for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < c; i += gridDim.x * blockDim.x) {
         const uint32_t b = ws.cand_bkt[i];
         if (b > b_last) continue;
@@ -758,7 +866,6 @@ __global__ void __launch_bounds__(256) cs_sel_scatter_kernel(cs_workspace ws)
 // ---------------------------------------------------------------------------------------------
 // 5 rank and emit
 // ---------------------------------------------------------------------------------------------
-#define RANK_TILE 2048u
 // Each needed bucket is ordered by one CTA: a bitonic sort of the bucket in a shared-memory tile
 // (O(m log^2 m), so an unlucky large bucket costs little more than an average one), after which
 // position i of the bucket is position offset + i of the output list.
@@ -767,52 +874,35 @@ cs_sel_rank_kernel(cs_workspace ws, uint32_t k, uint32_t *__restrict__ ids_out, 
 {
     __shared__ unsigned long long t_km[RANK_TILE];
     __shared__ uint32_t t_id[RANK_TILE];
+    __shared__ uint32_t s_off[CS_MAX_SPLITTERS + 2];
+    __shared__ uint32_t s_tmp[16];
     cs_wait_for_predecessor();
     cs_release_successor();
-    const uint32_t p_end = ws.sel->p_end, n_out = ws.sel->n_out, b_last = ws.sel->b_last;
+    const uint32_t n_out = ws.sel->n_out, cap = ws.sel->cap;
+    const bool in_regions = ws.sel->placed && !ws.sel->overflow;
     const uint32_t gtid = blockIdx.x * blockDim.x + threadIdx.x, nth = gridDim.x * blockDim.x;
     for (uint32_t i = n_out + gtid; i < k; i += nth) ids_out[i] = CS_ID_NONE;
     if (gtid == 0) *n_out_dev = n_out;
-    if (p_end == 0) return;
+    if (n_out == 0) return;
+    const uint32_t b_last = bucket_offsets(ws, ws.sel->n_spl, n_out, s_off, s_tmp);
     for (uint32_t b = blockIdx.x; b <= b_last; b += gridDim.x) {
-        const uint32_t beg = ws.boff[b], end = ws.boff[b + 1], m = end - beg;
+        const uint32_t beg = s_off[b], end = s_off[b + 1], m = end - beg;
+        const size_t src = in_regions ? (size_t)b * cap : (size_t)beg;      // where the bucket's keys are
         __syncthreads();
         if (m <= RANK_TILE) {
-            uint32_t P = 64;
-            while (P < m) P <<= 1;
-            for (uint32_t i = threadIdx.x; i < P; i += blockDim.x) {
-                t_km[i] = i < m ? ws.sort_km[beg + i] : ~0ull;
-                t_id[i] = i < m ? ws.sort_id[beg + i] : 0xFFFFFFFFu;
+            for (uint32_t i = threadIdx.x; i < m; i += blockDim.x) {
+                t_km[i] = ws.sort_km[src + i];
+                t_id[i] = ws.sort_id[src + i];
             }
-            __syncthreads();
-            if (P <= 2 * blockDim.x) {
-                bitonic_sort_fast(t_km, t_id, P);
-            } else {
-                for (uint32_t size = 2; size <= P; size <<= 1) {
-                    for (uint32_t stride = size >> 1; stride > 0; stride >>= 1) {
-                        for (uint32_t t = threadIdx.x; t < P / 2; t += blockDim.x) {
-                            const uint32_t lo = 2 * t - (t & (stride - 1));
-                            const uint32_t hi = lo + stride;
-                            const bool up = (lo & size) == 0;
-                            const unsigned long long ka = t_km[lo], kb = t_km[hi];
-                            const uint32_t ia = t_id[lo], ib = t_id[hi];
-                            if (key_less(kb, ib, ka, ia) == up) {
-                                t_km[lo] = kb; t_id[lo] = ib;
-                                t_km[hi] = ka; t_id[hi] = ia;
-                            }
-                        }
-                        __syncthreads();
-                    }
-                }
-            }
+            sort_tile(t_km, t_id, m);
             for (uint32_t i = threadIdx.x; i < m; i += blockDim.x)
                 if (beg + i < n_out) ids_out[beg + i] = t_id[i];
         } else {                                              // larger than the tile: rank straight from global memory
             for (uint32_t i = threadIdx.x; i < m; i += blockDim.x) {
-                const unsigned long long km = ws.sort_km[beg + i];
-                const uint32_t id = ws.sort_id[beg + i];
+                const unsigned long long km = ws.sort_km[src + i];
+                const uint32_t id = ws.sort_id[src + i];
                 uint32_t rank = 0;
-                for (uint32_t q = beg; q < end; ++q) rank += key_less(ws.sort_km[q], ws.sort_id[q], km, id) ? 1u : 0u;
+                for (uint32_t q = 0; q < m; ++q) rank += key_less(ws.sort_km[src + q], ws.sort_id[src + q], km, id) ? 1u : 0u;
                 if (beg + rank < n_out) ids_out[beg + rank] = id;
             }
         }
@@ -845,6 +935,7 @@ void cs_fill_sel_args(const cs_ctx *ctx, const cs_block_index *idx, uint32_t now
     a.hint_slot = 0;
     a.kind = 0;
     a.now_dev = ctx->step_now_dev ? ctx->step_now_dev : ctx->clock_dev;
+    a.sort_cap = 0;
 }
 
 uint32_t cs_scan_grid(const cs_ctx *ctx, uint32_t n, uint32_t per_cta, uint32_t ctas_per_sm)
@@ -905,6 +996,7 @@ static int launch_select_job(cs_ctx *ctx, int job, const cs_block_index *idx, ui
     a.k = k;
     a.hint_slot = ctx->no_speculation ? 3u : (prefetch ? 2u : tier);
     a.kind = prefetch ? 2u : tier;
+    a.sort_cap = ctx->p.max_blocks;          // keys the sort region of this select holds
     if (ctx->select_path != CS_SELECT_MULTI && idx->n_blocks <= CS_SELECT_CLUSTER_MAX_BLOCKS) {
         const int rc1 = cs_launch_select_cluster(ctx, &a, &ws, prefetch, ids_out, n_out, s);
         if (rc1 != CS_ENOTIMPL) return rc1;          // no usable cluster on this device: fall through

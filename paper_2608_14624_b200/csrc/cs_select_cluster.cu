@@ -88,7 +88,7 @@ __device__ __forceinline__ uint32_t csel_block_scan(uint32_t v, uint32_t *s_part
 // In-place bitonic sort of P (power of two) keys in shared memory, ascending by (km, id).
 __device__ __forceinline__ void csel_bitonic(unsigned long long *km, uint32_t *id, uint32_t P)
 {
-    if (P >= 64 && P <= 2 * CSEL_THREADS) { bitonic_sort_fast(km, id, P); return; }
+    if (P >= 64 && P <= 2 * CSEL_THREADS) { bitonic_sort_fast(km, id, P, whole_cta()); return; }
     for (uint32_t size = 2; size <= P; size <<= 1) {
         for (uint32_t stride = size >> 1; stride > 0; stride >>= 1) {
             for (uint32_t t = threadIdx.x; t < P / 2; t += blockDim.x) {
@@ -236,7 +236,7 @@ __device__ __forceinline__ void csel_body(SelArgs a, const cs_workspace &ws, uin
     const bool spec_ok = hint != 0xFFFFFFFFu && b0 != 0xFFFFFFFFu && b0 <= hint;     // same verdict in every CTA
     const bool have_b0 = a.k && n_elig >= a.k;
     if (rank == 0) {                                           // whole CTA 0: same histogram in every CTA
-        const uint32_t ahead = have_b0 ? collect_ahead_limit<PER>(loc, tid * PER, before, a.k, b0, &S.misc[2]) : 0u;
+        const uint32_t ahead = have_b0 ? collect_ahead_limit<PER>(loc, tid * PER, before, a.k, b0, &S.misc[2], whole_cta()) : 0u;
         if (tid == 0) remember_threshold(ws.sc, a.hint_slot, have_b0, ahead);
     }
     if (!spec_ok) {

@@ -22,12 +22,23 @@ struct SelArgs {
     uint32_t hint_slot;           // which remembered threshold bin this call may speculate on
     uint32_t kind;                // 0 GPU-tier victims, 1 host-tier victims, 2 prefetch candidates (work counters)
     const uint32_t *now_dev;      // when set, the clock is read from device memory at execution time (graph replay)
+    uint32_t sort_cap;            // keys the sort region holds (0: buckets never get fixed regions)
 };
 
 // host helpers defined in cs_select.cu
 void cs_fill_sel_args(const cs_ctx *ctx, const cs_block_index *idx, uint32_t now, const float *fsurv, SelArgs &a);
 uint32_t cs_scan_grid(const cs_ctx *ctx, uint32_t n, uint32_t per_cta, uint32_t ctas_per_sm = 2);
 size_t cs_table_smem(const cs_ctx *ctx);
+
+// A group of whole warps of a CTA that synchronises on a barrier of its own, so that two halves of a CTA can work on
+// different things at the same time: t = index of the calling thread within the group, n = its threads,
+// bar = hardware barrier (0 = the one of __syncthreads(), for the whole CTA).
+struct CtaPart { uint32_t t, n, bar; };
+__device__ __forceinline__ CtaPart whole_cta() { return CtaPart{threadIdx.x, blockDim.x, 0u}; }
+__device__ __forceinline__ void part_sync(const CtaPart &p)
+{
+    asm volatile("bar.sync %0, %1;" ::"r"(p.bar), "r"(p.n) : "memory");
+}
 
 // What the next call of this kind may collect ahead of its own threshold.  The threshold bin of consecutive
 // calls moves little, so the next call's first scan appends every entry up to a remembered bin.  That bin is
@@ -36,14 +47,14 @@ size_t cs_table_smem(const cs_ctx *ctx);
 // bins (a prefetch list whose best entries leave the tier every call, so its threshold jumps) get several bins
 // of slack for a few thousand extra candidates; dense bins get none.  Only the amount of work depends on this,
 // never the result.  `loc` are the calling thread's bins [first, first + PER), `before` the population below
-// them; every thread of the CTA calls; s_lim is a shared word.
+// them; every thread of the group calls; s_lim is a shared word.
 #define CS_SPEC_MAX_AHEAD 8u
 template <uint32_t PER>
 __device__ __forceinline__ uint32_t collect_ahead_limit(const uint32_t (&loc)[PER], uint32_t first, uint32_t before,
-                                                        uint32_t k, uint32_t b0, uint32_t *s_lim)
+                                                        uint32_t k, uint32_t b0, uint32_t *s_lim, const CtaPart &cp)
 {
-    if (threadIdx.x == 0) *s_lim = 0;
-    __syncthreads();
+    if (cp.t == 0) *s_lim = 0;
+    part_sync(cp);
     const unsigned long long cap = 3ull * k + 1024ull;
     unsigned long long run = before;
     uint32_t best = 0xFFFFFFFFu;
@@ -53,7 +64,7 @@ __device__ __forceinline__ uint32_t collect_ahead_limit(const uint32_t (&loc)[PE
         if (run <= cap) best = first + q;
     }
     if (best != 0xFFFFFFFFu) atomicMax(s_lim, best);
-    __syncthreads();
+    part_sync(cp);
     uint32_t lim = *s_lim;
     if (lim < b0) lim = b0;
     if (lim > b0 + CS_SPEC_MAX_AHEAD) lim = b0 + CS_SPEC_MAX_AHEAD;
@@ -422,22 +433,22 @@ __device__ __forceinline__ bool last_cta_done(uint32_t *ticket, bool *s_flag)
     return last;
 }
 
-// Exclusive prefix sum of one value per thread over a CTA of SEL_THREADS threads (warp shuffles, three barriers);
-// also returns the total.  s_part: at least 64 words.
-__device__ __forceinline__ uint32_t sel_block_scan(uint32_t v, uint32_t *s_part, uint32_t &total)
+// Exclusive prefix sum of one value per thread over a group of warps (warp shuffles, three barriers); also returns
+// the total.  s_part: at least 64 words.
+__device__ __forceinline__ uint32_t sel_block_scan(uint32_t v, uint32_t *s_part, uint32_t &total, const CtaPart &cp)
 {
-    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t lane = cp.t & 31, warp = cp.t >> 5, n_warps = cp.n >> 5;
     uint32_t incl = v;
 #pragma unroll
     for (int d = 1; d < 32; d <<= 1) {
         const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, incl, d);
         if (lane >= d) incl += t;
     }
-    __syncthreads();
+    part_sync(cp);
     if (lane == 31) s_part[warp] = incl;
-    __syncthreads();
+    part_sync(cp);
     if (warp == 0) {
-        uint32_t w = lane < (SEL_THREADS / 32) ? s_part[lane] : 0;
+        uint32_t w = lane < n_warps ? s_part[lane] : 0;
 #pragma unroll
         for (int d = 1; d < 32; d <<= 1) {
             const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, w, d);
@@ -445,8 +456,8 @@ __device__ __forceinline__ uint32_t sel_block_scan(uint32_t v, uint32_t *s_part,
         }
         s_part[32 + lane] = w;                         // inclusive warp totals
     }
-    __syncthreads();
-    total = s_part[32 + SEL_THREADS / 32 - 1];
+    part_sync(cp);
+    total = s_part[32 + n_warps - 1];
     const uint32_t before = warp ? s_part[32 + warp - 1] : 0;
     return before + incl - v;
 }
@@ -460,10 +471,10 @@ __device__ __forceinline__ bool key_less(unsigned long long km_a, uint32_t id_a,
 
 
 // ---------------------------------------------------------------------------------------------
-// Bitonic sort of P keys (power of two, 64 <= P <= 2 * blockDim.x) held in shared memory,
+// Bitonic sort of P keys (power of two, 64 <= P <= 2 * threads of the group) held in shared memory,
 // ascending by (km, id).  Each thread keeps two neighbouring elements in registers; compare-
 // exchange steps whose partner lies in the same warp (element distance <= 32) use shuffles and
-// no barrier, only the longer distances go through shared memory.  Called by the whole CTA.
+// no barrier, only the longer distances go through shared memory.  Called by every thread of the group.
 // ---------------------------------------------------------------------------------------------
 __device__ __forceinline__ void cx_keep(unsigned long long &k, uint32_t &i, unsigned long long pk, uint32_t pi,
                                         bool keep_min)
@@ -472,9 +483,9 @@ __device__ __forceinline__ void cx_keep(unsigned long long &k, uint32_t &i, unsi
     if (partner_less == keep_min) { k = pk; i = pi; }
 }
 
-__device__ __forceinline__ void bitonic_sort_fast(unsigned long long *km, uint32_t *id, uint32_t P)
+__device__ __forceinline__ void bitonic_sort_fast(unsigned long long *km, uint32_t *id, uint32_t P, const CtaPart &cp)
 {
-    const uint32_t t = threadIdx.x;
+    const uint32_t t = cp.t;
     const bool act = t < P / 2;                           // whole warps, because P >= 64
     unsigned long long k0 = 0, k1 = 0;
     uint32_t i0 = 0, i1 = 0;
@@ -484,7 +495,7 @@ __device__ __forceinline__ void bitonic_sort_fast(unsigned long long *km, uint32
         uint32_t stride = size >> 1;
         if (stride >= 64) {                               // partners in other warps: through shared memory
             if (act) { km[2 * t] = k0; km[2 * t + 1] = k1; id[2 * t] = i0; id[2 * t + 1] = i1; }
-            __syncthreads();
+            part_sync(cp);
             for (; stride >= 64; stride >>= 1) {
                 if (act) {
                     const uint32_t lo = 2 * t - (t & (stride - 1)), hi = lo + stride;
@@ -493,7 +504,7 @@ __device__ __forceinline__ void bitonic_sort_fast(unsigned long long *km, uint32
                     const uint32_t ia = id[lo], ib = id[hi];
                     if (key_less(kb, ib, ka, ia) == up2) { km[lo] = kb; id[lo] = ib; km[hi] = ka; id[hi] = ia; }
                 }
-                __syncthreads();
+                part_sync(cp);
             }
             if (act) { k0 = km[2 * t]; k1 = km[2 * t + 1]; i0 = id[2 * t]; i1 = id[2 * t + 1]; }
         }
@@ -512,7 +523,7 @@ __device__ __forceinline__ void bitonic_sort_fast(unsigned long long *km, uint32
             }
         }
     }
-    __syncthreads();
+    part_sync(cp);
     if (act) { km[2 * t] = k0; km[2 * t + 1] = k1; id[2 * t] = i0; id[2 * t + 1] = i1; }
-    __syncthreads();
+    part_sync(cp);
 }

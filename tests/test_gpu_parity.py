@@ -595,6 +595,24 @@ def test_maximum_agent_count():
     assert np.all(np.abs(ps.cpu().numpy() - want) <= H.REL_TOL * np.maximum(want, 1e-3))
 
 
+@pytest.mark.parametrize("A,stride", [(40, 1), (300, 1), (300, 7), (512, 1), (512, 33), (544, 1), (96, 5)])
+def test_bfs_on_deep_path_graphs(A, stride):
+    """A workflow that is one long path (agent i is followed by agent i + stride mod A, over and over): the BFS from
+    the current agent is as deep as the graph allows, the adjacency rows have 2 .. 17 words, and every hop count up
+    to the depth appears once in the exported table."""
+    cfg = synth.shrink(synth.CONFIGS["meta1m"], n_agents=A, sessions=2, n_chains=2, events_per_step=(8, 8))
+    order = (np.arange(3 * A + 11, dtype=np.int64) * stride) % A
+    chain = np.zeros(len(order), dtype=np.uint32)
+    agent = order.astype(np.uint16)
+    c, o = make_ctx(cfg, 64, tau=0.3, e_max=50, r_min=0.0)
+    for lo in range(0, len(order), 97):                     # ragged batches, so predecessors are carried between calls
+        c.observe_invocations(dev(chain[lo:lo + 97]), dev(agent[lo:lo + 97]), None)
+        o.observe(chain[lo:lo + 97], agent[lo:lo + 97])
+    m = H.compare_model(c, o)
+    reach = m["hops"][m["hops"] != 0xFFFF]
+    assert int(reach.max()) == A // int(np.gcd(A, stride)) - 1      # the path was walked to its end
+
+
 def test_checkpoint_and_resume_of_the_learner():
     cfg = synth.CONFIGS["llama70b"]
     tr = synth.make_trace(cfg, n_invocations=4000, warmup_frac=0.05)
