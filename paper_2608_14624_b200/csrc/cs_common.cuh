@@ -60,20 +60,19 @@ struct cs_scalars {
 // State of one select in flight, rewritten by every call.  The selects of a step that run side by side each
 // have their own (with their own histogram, candidate and sort regions).
 struct cs_sel_state {
-    uint32_t ticket[6];     // "last CTA done" counters, one per kernel that has an epilogue (1..5 in use)
-    uint32_t b0;            // threshold bin of the first digit
-    uint32_t n_elig;        // eligible entries
+    // what the bucket launch reads first, as one 16-byte word
     uint32_t c;             // candidates collected (first digit <= b0)
     uint32_t n_spl;         // splitters in use
-    uint32_t b_last;        // last bucket that holds one of the k winners
-    uint32_t p_end;         // end position of that bucket
+    uint32_t placed;        // 1: every bucket has a fixed region of `cap` keys in the sort arrays, filled by the bucket launch
+    uint32_t cap;           // keys per bucket region
     uint32_t n_out;         // min(k, eligible)
+    uint32_t overflow;      // 1: a bucket outgrew its region; the scatter launch groups the buckets instead
+    uint32_t b0;            // threshold bin of the first digit
+    uint32_t n_elig;        // eligible entries
+    uint32_t ticket[6];     // "last CTA done" counters, one per kernel that has an epilogue
     uint32_t c_spec;        // candidates appended by the fast pass; 0 between calls
     uint32_t n_above;       // eligible entries the fast pass found above the remembered bin; 0 between calls
     uint32_t spec;          // 1: the fast pass's candidates cover the k winners, the histogram and collect passes are skipped
-    uint32_t placed;        // 1: every bucket has a fixed region of `cap` keys in the sort arrays, filled by the bucket launch
-    uint32_t cap;           // keys per bucket region
-    uint32_t overflow;      // 1: a bucket outgrew its region; the scatter launch groups the buckets instead
     uint32_t cc[2];         // candidate counters of the cluster kernel: a call uses one and clears the other for the
                             // next call, so that the counter is zero on entry without a barrier
     uint32_t toggle;        // which of the two the next call uses; flipped by every call on the device, so that a
@@ -224,6 +223,18 @@ __device__ __forceinline__ uint2 cs_ld_cg_pinned(const uint2 *p)
 {
     uint2 v;
     asm volatile("ld.global.cg.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ unsigned long long cs_ld_cg_pinned(const unsigned long long *p)
+{
+    unsigned long long v;
+    asm volatile("ld.global.cg.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ uint4 cs_ld_cg_pinned(const uint4 *p)
+{
+    uint4 v;
+    asm volatile("ld.global.cg.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
     return v;
 }
 __device__ __forceinline__ ulonglong2 cs_ld_cg_pinned(const ulonglong2 *p)

@@ -7,6 +7,7 @@
 
 #define OBS_THREADS 1024
 #define ROW_THREADS 256
+#define OBS_FUSED_MAX 256u     // events up to which a batch is applied inside the refresh launch (one per thread)
 
 // ---------------------------------------------------------------------------------------------
 // Initial state of Algorithm 1: zero counts, no current agent; plus the recency table.
@@ -254,8 +255,15 @@ __device__ void cs_block_sum2(double &a, double &b, double *s_red)
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(ROW_THREADS)
 cs_normalise_kernel(cs_workspace ws, uint32_t A, uint32_t W, float eps, float tau, float r_min, uint32_t e_max,
-                    float delta, uint32_t all_chains, uint32_t n_chains)
+                    float delta, uint32_t all_chains, uint32_t n_chains, const uint32_t *__restrict__ ev_chain,
+                    const uint16_t *__restrict__ ev_agent, const uint8_t *__restrict__ ev_flags, uint32_t n_events,
+                    const uint32_t *__restrict__ n_events_dev)
 {
+    __shared__ uint32_t s_evc[OBS_FUSED_MAX];        // the batch: chain of event e,
+    __shared__ uint16_t s_eva[OBS_FUSED_MAX];        // its agent (CS_AGENT_NONE: skipped),
+    __shared__ uint16_t s_evp[OBS_FUSED_MAX];        // and the agent it follows when that is a counted transition
+    __shared__ uint32_t s_add[CS_MAX_AGENTS];        // what the batch adds to the row being worked on
+    __shared__ int s_last_live;
     __shared__ double s_red[64];
     __shared__ float s_bestv[ROW_THREADS / 32];
     __shared__ uint32_t s_besti[ROW_THREADS / 32];
@@ -269,12 +277,59 @@ cs_normalise_kernel(cs_workspace ws, uint32_t A, uint32_t W, float eps, float ta
     // Column sums q_j = sum_i pi_i P_ij of Eq. 2 are accumulated by the row CTAs in 2^-60 fixed
     // point with integer atomics: integer addition commutes, so the sum is bit-identical from run
     // to run whatever order the CTAs finish in (a float atomic would not be).
-    const uint32_t n_total = ws.sc->n_transitions;
+    // ---- a small batch of events is applied here, by every CTA to the rows it owns, instead of by a launch of its
+    // own: each CTA stages the batch, finds every event's predecessor (in the batch, else the chain's current agent)
+    // exactly as cs_observe_kernel does, and adds the transitions that start at row i to row i.  What is shared --
+    // cur[], the last agent, the totals and the counters -- is written by the last CTA, after every CTA has read it.
+    if (n_events_dev) n_events = min(n_events, *n_events_dev);
+    uint32_t n_new = 0, n_skipped = 0;
+    if (n_events) {
+        uint32_t c = 0, a = CS_AGENT_NONE;
+        if (tid == 0) s_last_live = -1;
+        if (tid < n_events) {
+            c = ev_chain[tid];
+            a = ev_agent[tid];
+            const bool warm = ev_flags && (ev_flags[tid] & CS_EV_WARMUP);
+            uint32_t bad = 0;
+            if (!warm && a >= A) bad |= CS_ST_BAD_AGENT;
+            if (!warm && c >= n_chains) bad |= CS_ST_BAD_CHAIN;
+            if (bad && blockIdx.x == 0) atomicOr(&ws.sc->status, bad);
+            if (warm || bad) a = CS_AGENT_NONE;
+        }
+        s_evc[tid] = c;
+        s_eva[tid] = (uint16_t)a;
+        __syncthreads();
+        const bool live = tid < n_events && a != CS_AGENT_NONE;
+        uint32_t prev = CS_AGENT_NONE;
+        if (live) {
+            int j = (int)tid - 1;
+            for (; j >= 0; --j)
+                if (s_evc[j] == c && s_eva[j] != CS_AGENT_NONE) { prev = s_eva[j]; break; }
+            if (j < 0) prev = ws.cur[c];
+            atomicMax(&s_last_live, (int)tid);
+        }
+        const bool counted = live && prev != CS_AGENT_NONE && prev != a;
+        s_evp[tid] = (uint16_t)(counted ? prev : CS_AGENT_NONE);
+        n_new = (uint32_t)__syncthreads_count(counted);
+        n_skipped = (uint32_t)__syncthreads_count(tid < n_events && a == CS_AGENT_NONE);
+    }
+    const uint32_t n_total = ws.sc->n_transitions + n_new;
     const uint32_t fill = ws.sc->adjT_cur ^ 1u;              // every CTA reads this before the last one flips it
     uint32_t *adjT_fill = ws.adjT + (size_t)fill * A * W, *adjT_clear = ws.adjT + (size_t)(fill ^ 1u) * A * W;
     const double inv_total = n_total ? 1.0 / (double)n_total : 0.0;
     for (uint32_t i = blockIdx.x; i < A; i += gridDim.x) {
-        const uint32_t n_i = ws.rowsum[i];
+        uint32_t n_i = ws.rowsum[i];
+        // transitions of the batch that start at agent i
+        const bool mine = n_events && tid < n_events && s_evp[tid] == i;
+        const uint32_t row_new = n_events ? (uint32_t)__syncthreads_count(mine) : 0u;
+        if (row_new) {
+            for (uint32_t j = tid; j < A; j += ROW_THREADS) s_add[j] = 0;
+            __syncthreads();
+            if (mine) atomicAdd(&s_add[s_eva[tid]], 1u);
+            __syncthreads();
+            n_i += row_new;
+            if (tid == 0) ws.rowsum[i] = n_i;
+        }
         const double pi_fix = (double)n_i * inv_total * 1152921504606846976.0;      // pi_i * 2^60
         const float den = __fadd_rn((float)n_i, __fmul_rn((float)A, eps));
         float bestv = -1.0f;
@@ -284,7 +339,9 @@ cs_normalise_kernel(cs_workspace ws, uint32_t A, uint32_t W, float eps, float ta
             const uint32_t j = j0 + tid;
             bool edge = false;
             if (j < A) {
-                const float p = __fdiv_rn(__fadd_rn((float)ws.C[i * A + j], eps), den);
+                uint32_t cij = ws.C[i * A + j];
+                if (row_new && s_add[j]) { cij += s_add[j]; ws.C[i * A + j] = cij; }
+                const float p = __fdiv_rn(__fadd_rn((float)cij, eps), den);
                 ws.P[i * A + j] = p;
                 if (p > bestv) { bestv = p; besti = j; }         // strict: the lowest j among equals stays
                 const double pd = (double)p;
@@ -336,9 +393,29 @@ cs_normalise_kernel(cs_workspace ws, uint32_t A, uint32_t W, float eps, float ta
 
     BfsRow rowT;                                                         // in flight during the sums
     cs_bfs_load_row(adjT_fill, A, W, rowT);
-    const uint32_t la = __ldcg(&ws.sc->last_agent);
+    uint32_t la = __ldcg(&ws.sc->last_agent);
+    if (n_events) {
+        // the batch's effect on what all CTAs share (every other CTA is done reading it)
+        const uint32_t a = tid < n_events ? s_eva[tid] : CS_AGENT_NONE;
+        if (a != CS_AGENT_NONE) {
+            const uint32_t c = s_evc[tid];
+            bool last_of_chain = true;
+            for (uint32_t q = tid + 1; q < n_events; ++q)
+                if (s_evc[q] == c && s_eva[q] != CS_AGENT_NONE) { last_of_chain = false; break; }
+            if (last_of_chain) ws.cur[c] = (uint16_t)a;
+        }
+        __threadfence();                                      // (cur[] is read back below when every chain is a source)
+        if (s_last_live >= 0) la = s_eva[s_last_live];
+        if (tid == 0) {
+            ws.sc->last_agent = la;
+            ws.sc->n_transitions = n_total;
+            atomicAdd((unsigned long long *)&ws.cnt->events_seen, (unsigned long long)n_events);
+            if (n_skipped) atomicAdd((unsigned long long *)&ws.cnt->events_skipped, (unsigned long long)n_skipped);
+            if (n_new) atomicAdd((unsigned long long *)&ws.cnt->transitions_counted, (unsigned long long)n_new);
+        }
+    }
     if (tid < 64) s_front[tid] = (tid < 32 && !all_chains && la < A && (la >> 5) == tid) ? (1u << (la & 31)) : 0u;
-    const uint32_t N = __ldcg(&ws.sc->n_transitions);
+    const uint32_t N = n_total;
     double Hc = 0.0, Hm = 0.0;
     if (N > 0) {
         const double invN = 1.0 / (double)N;
@@ -543,7 +620,8 @@ int cs_launch_observe(cs_ctx *ctx, const uint32_t *chain, const uint16_t *agent,
                       uint32_t n_events, cudaStream_t s)
 {
     const cs_params &p = ctx->p;
-    if (n_events) {
+    const bool fused = n_events <= OBS_FUSED_MAX;             // small batches ride along with the refresh
+    if (n_events && !fused) {
         cs_launch_chained(cs_observe_kernel, 1, OBS_THREADS, 0, s, ctx->ws, p.n_agents, p.n_chains, chain, agent, evflags,
                           n_events, ctx->step_n_events_dev);
         int rc = cs_check_launch(ctx);
@@ -551,7 +629,10 @@ int cs_launch_observe(cs_ctx *ctx, const uint32_t *chain, const uint16_t *agent,
     }
     const uint32_t grid = p.n_agents < 2u * (uint32_t)ctx->sm_count ? p.n_agents : 2u * (uint32_t)ctx->sm_count;
     cs_launch_chained(cs_normalise_kernel, grid, ROW_THREADS, 0, s, ctx->ws, p.n_agents, ctx->W, p.eps, p.tau, p.r_min,
-                      p.e_max, p.delta, ctx->source_mode == CS_SOURCES_ALL_CHAINS ? 1u : 0u, p.n_chains);
+                      p.e_max, p.delta, ctx->source_mode == CS_SOURCES_ALL_CHAINS ? 1u : 0u, p.n_chains,
+                      fused ? chain : (const uint32_t *)nullptr, fused ? agent : (const uint16_t *)nullptr,
+                      fused ? evflags : (const uint8_t *)nullptr, fused ? n_events : 0u,
+                      fused ? (const uint32_t *)ctx->step_n_events_dev : (const uint32_t *)nullptr);
     return cs_check_launch(ctx);
 }
 

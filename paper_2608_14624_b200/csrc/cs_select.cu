@@ -767,7 +767,7 @@ __device__ __forceinline__ uint32_t bucket_offsets(const cs_workspace &ws, uint3
 // General case: per round a CTA takes 1024 candidates, counts them per bucket in shared memory and reserves the
 // CTA's range in each non-empty bucket with one global atomic; bucket and slot are recorded for the scatter launch.
 // ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) cs_sel_bucket_kernel(cs_workspace ws)
+__global__ void __launch_bounds__(256) cs_sel_bucket_kernel(cs_workspace ws, uint32_t sort_cap)
 {
     __shared__ unsigned long long s_km[CS_MAX_SPLITTERS + 1];
     __shared__ uint32_t s_id[CS_MAX_SPLITTERS + 1];
@@ -775,32 +775,56 @@ __global__ void __launch_bounds__(256) cs_sel_bucket_kernel(cs_workspace ws)
     constexpr int ITEMS = 4;                                  // candidates per thread and round
     cs_wait_for_predecessor();
     cs_release_successor();
-    const uint32_t c = ws.sel->c, n_spl = ws.sel->n_spl, placed = ws.sel->placed, cap = ws.sel->cap;
-    for (uint32_t j = threadIdx.x; j < n_spl; j += blockDim.x) { s_km[j] = ws.spl_km[j]; s_id[j] = ws.spl_id[j]; }
+    // Everything the first round needs is asked for at once -- the select's state, the splitters and the round's keys
+    // (addresses bounded by the capacity of the buffers; what lies beyond the live counts is ignored below) -- so that
+    // the launch starts with one trip to L2 instead of three.
+    unsigned long long km[ITEMS];
+    uint32_t id[ITEMS], bkt[ITEMS], loc[ITEMS];
+    const uint32_t base0 = blockIdx.x * (256 * ITEMS);
+    const uint4 st = cs_ld_cg_pinned((const uint4 *)&ws.sel->c);          // c, n_spl, placed, cap
+#pragma unroll
+    for (int u = 0; u < ITEMS; ++u) {
+        const uint32_t i = base0 + u * 256 + threadIdx.x, ii = i < sort_cap ? i : 0u;
+        km[u] = cs_ld_cg_pinned(ws.cand_km + ii);
+        id[u] = cs_ld_cg_pinned(ws.cand_id + ii);
+    }
+    const unsigned long long my_spl_km = cs_ld_cg_pinned(ws.spl_km + threadIdx.x);
+    const uint32_t my_spl_id = cs_ld_cg_pinned(ws.spl_id + threadIdx.x);
+    const uint32_t c = st.x, n_spl = st.y, placed = st.z, cap = st.w;
+    // splitters past the last one sort behind every key, so that the search below always takes eight steps
+    s_km[threadIdx.x] = threadIdx.x < n_spl ? my_spl_km : ~0ull;
+    s_id[threadIdx.x] = threadIdx.x < n_spl ? my_spl_id : 0xFFFFFFFFu;
     s_cnt[threadIdx.x] = 0;
     __syncthreads();
-    for (uint32_t base = blockIdx.x * (256 * ITEMS); base < c; base += gridDim.x * (256 * ITEMS)) {
-        unsigned long long km[ITEMS];
-        uint32_t id[ITEMS], bkt[ITEMS], loc[ITEMS];
+    for (uint32_t base = base0; base < c; base += gridDim.x * (256 * ITEMS)) {
+        if (base != base0) {
 #pragma unroll
-        for (int u = 0; u < ITEMS; ++u) {                     // all of the round's keys are fetched before any is used
-            const uint32_t i = base + u * 256 + threadIdx.x;
-            km[u] = i < c ? __ldcg(&ws.cand_km[i]) : 0ull;
-            id[u] = i < c ? __ldcg(&ws.cand_id[i]) : 0u;
+            for (int u = 0; u < ITEMS; ++u) {                 // all of the round's keys are fetched before any is used
+                const uint32_t i = base + u * 256 + threadIdx.x, ii = i < c ? i : 0u;
+                km[u] = cs_ld_cg_pinned(ws.cand_km + ii);
+                id[u] = cs_ld_cg_pinned(ws.cand_id + ii);
+            }
+        }
+        // bucket = number of splitters <= key: a branch-free descent over the 255 (padded) splitters, the round's four
+        // keys side by side
+        uint32_t pos[ITEMS];
+#pragma unroll
+        for (int u = 0; u < ITEMS; ++u) pos[u] = 0;
+#pragma unroll 1
+        for (uint32_t step = 128; step > 0; step >>= 1) {
+#pragma unroll
+            for (int u = 0; u < ITEMS; ++u) {
+                const uint32_t probe = pos[u] + step - 1u;
+                if (!key_less(km[u], id[u], s_km[probe], s_id[probe])) pos[u] += step;
+            }
         }
 #pragma unroll
         for (int u = 0; u < ITEMS; ++u) {
             const uint32_t i = base + u * 256 + threadIdx.x;
             bkt[u] = 0xFFFFFFFFu;
             if (i < c) {
-                uint32_t lo = 0, hi = n_spl;                 // bucket = number of splitters <= key
-                while (lo < hi) {
-                    const uint32_t mid = (lo + hi) >> 1;
-                    if (key_less(km[u], id[u], s_km[mid], s_id[mid])) hi = mid;
-                    else lo = mid + 1;
-                }
-                bkt[u] = lo;
-                if (!placed) loc[u] = atomicAdd(&s_cnt[lo], 1u);
+                bkt[u] = pos[u] < n_spl ? pos[u] : n_spl;    // (a key equal to the padding stays in the last bucket)
+                if (!placed) loc[u] = atomicAdd(&s_cnt[bkt[u]], 1u);
             }
         }
         if (placed) {
@@ -1026,7 +1050,7 @@ static int launch_select_job(cs_ctx *ctx, int job, const cs_block_index *idx, ui
     if (prefetch) cs_launch_chained(cs_sel_collect_kernel<true>, grid, SEL_THREADS, sm_collect, s, a, ws);
     else cs_launch_chained(cs_sel_collect_kernel<false>, grid, SEL_THREADS, sm_collect, s, a, ws);
     if ((rc = cs_check_launch(ctx)) != CS_OK) return rc;
-    cs_launch_chained(cs_sel_bucket_kernel, grid_c, 256, 0, s, ws);
+    cs_launch_chained(cs_sel_bucket_kernel, grid_c, 256, 0, s, ws, (uint32_t)ctx->p.max_blocks);
     if ((rc = cs_check_launch(ctx)) != CS_OK) return rc;
     cs_launch_chained(cs_sel_scatter_kernel, grid_c, 256, 0, s, ws);
     if ((rc = cs_check_launch(ctx)) != CS_OK) return rc;

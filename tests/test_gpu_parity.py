@@ -595,6 +595,44 @@ def test_maximum_agent_count():
     assert np.all(np.abs(ps.cpu().numpy() - want) <= H.REL_TOL * np.maximum(want, 1e-3))
 
 
+@pytest.mark.parametrize("A,chains,all_sources", [(4, 3, False), (256, 40, False), (256, 40, True), (1024, 9, False), (70, 1, True)])
+def test_small_batches_ride_with_the_refresh(A, chains, all_sources):
+    """Batches of up to 256 events are applied inside the refresh launch (every row CTA adds the batch's transitions
+    to its own rows, the last CTA writes the shared state); larger ones take the launch of their own.  Sizes on both
+    sides of that limit, chains that repeat inside a batch, warm-up events, bad agent and chain ids, one and all
+    chains as BFS sources: the learner state after every batch, the status bits and the event counters."""
+    base = synth.CONFIGS["tiny"] if A <= 5 else synth.CONFIGS["meta1m"]
+    cfg = synth.shrink(base, n_agents=A, sessions=chains, n_chains=chains, events_per_step=(4, 4))
+    tr = synth.make_trace(cfg, n_invocations=3000, warmup_frac=0.15)
+    agent, chain, evflags = tr.agent.copy(), tr.chain.copy(), tr.evflags.copy()
+    bad_at = [70, 700, 1400, 1500]                   # 70, 1400, 1500 fall into batches of <= 256 events, 700 into one of 257
+    evflags[bad_at] = 0
+    agent[70] = A + 1
+    chain[700] = chains
+    chain[1400] = chains + 5
+    agent[1500] = 0xFFFE
+    c, o = make_ctx(cfg, 64, r_min=0.0)
+    if all_sources:
+        c.set_survival_sources(cs.CS_SOURCES_ALL_CHAINS)
+    l0 = c.launch_count()
+    lo = 0
+    for size in (1, 2, 64, 255, 256, 257, 256, 300, 5, 256, 1024, 130):
+        hi = lo + size
+        c.observe_invocations(dev(chain[lo:hi]), dev(agent[lo:hi]), dev(evflags[lo:hi]))
+        o.observe(chain[lo:hi], agent[lo:hi], evflags[lo:hi])
+        if all_sources:
+            o.survival(sources=np.unique(o.cur[o.cur != orc.AGENT_NONE]))
+        H.compare_model(c, o)
+        lo = hi
+    assert c.launch_count() - l0 == 12 + 3           # one launch per batch, one more for the three batches above 256 events
+    assert c.get_status() == (cs.CS_ST_BAD_AGENT | cs.CS_ST_BAD_CHAIN)
+    cn = c.counters()
+    live = (evflags[:lo] & cs.CS_EV_WARMUP) == 0
+    bad = np.zeros(lo, bool); bad[bad_at] = True
+    assert cn["events_seen"] == lo and cn["events_skipped"] == int(np.sum(~live | bad))
+    assert cn["transitions_counted"] == int(o.C.sum())
+
+
 @pytest.mark.parametrize("A,stride", [(40, 1), (300, 1), (300, 7), (512, 1), (512, 33), (544, 1), (96, 5)])
 def test_bfs_on_deep_path_graphs(A, stride):
     """A workflow that is one long path (agent i is followed by agent i + stride mod A, over and over): the BFS from
