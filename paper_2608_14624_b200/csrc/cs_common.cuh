@@ -109,7 +109,6 @@ struct cs_workspace {
     unsigned long long *spl_km;     // [CS_MAX_SPLITTERS+1]
     uint32_t *spl_id;     // [CS_MAX_SPLITTERS+1]
     uint32_t *bcount;     // [CS_MAX_SPLITTERS+1]
-    uint32_t *boff;       // [CS_MAX_SPLITTERS+2]
 };
 
 struct cs_ctx {

@@ -404,7 +404,7 @@ cs_normalise_kernel(cs_workspace ws, uint32_t A, uint32_t W, float eps, float ta
                 if (s_evc[q] == c && s_eva[q] != CS_AGENT_NONE) { last_of_chain = false; break; }
             if (last_of_chain) ws.cur[c] = (uint16_t)a;
         }
-        __threadfence();                                      // (cur[] is read back below when every chain is a source)
+        if (all_chains) __threadfence();                      // (cur[] is read back below when every chain is a source)
         if (s_last_live >= 0) la = s_eva[s_last_live];
         if (tid == 0) {
             ws.sc->last_agent = la;

@@ -11,17 +11,20 @@
 //   prefetch: primary = (not a*)<<31 | ~score bits[30:0], secondary = ~last_access
 //
 // This file holds the multi-launch path, used for indexes above 262,144 entries (smaller ones take
-// the single-launch cluster kernel of cs_select_cluster.cu).  Five launches, none of which waits
+// the single-launch cluster kernel of cs_select_cluster.cu).  Six launches, none of which waits
 // on another CTA:
+//   0 fast pass : one scan against the threshold bin remembered from the last call of this kind; when the k
+//                 winners lie within it (the usual case) the candidates are complete and launches 1 and 2
+//                 return at once.  Its last CTA searches the threshold and sorts the splitter sample side by side.
 //   1 histogram : 4096-bin histogram of the top 12 primary bits; the last CTA to finish finds
 //                 the threshold bin b0 (first bin whose running count reaches k).
 //   2 collect   : every eligible entry whose bin <= b0 is appended to the candidate buffer
 //                 (c >= min(k, eligible) keys); the last CTA samples <= 1024 candidates,
 //                 sorts them in shared memory and publishes <= 255 splitters.
-//   3 bucket    : each candidate finds its bucket by binary search over the splitters and
-//                 takes a slot in it; the last CTA prefix-sums the bucket sizes and finds the
-//                 last bucket that can hold one of the k winners.
-//   4 scatter   : candidates of the needed buckets are grouped by bucket.
+//   3 bucket    : each candidate finds its bucket by a search over the splitters and takes a slot in it; with few
+//                 candidates the key goes straight into the bucket's own fixed-size region.
+//   4 scatter   : otherwise the candidates of the needed buckets are grouped by bucket (every CTA derives the
+//                 bucket offsets from the 256 counters itself).
 //   5 rank      : every needed bucket is sorted by one CTA in a shared-memory tile; bucket offset
 //                 + position in the bucket is the position in the output list.
 // Keys are unique (the id is part of the key), so the order is total and the output does not
@@ -1142,8 +1145,7 @@ int cs_launch_select_step(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, 
 #define CS_SO_SPLKM (CS_SO_HIST + CS_HIST_BINS * 4u)
 #define CS_SO_SPLID (CS_SO_SPLKM + CS_STATIC_ALIGN((CS_MAX_SPLITTERS + 1u) * 8u))
 #define CS_SO_BCOUNT (CS_SO_SPLID + CS_STATIC_ALIGN((CS_MAX_SPLITTERS + 1u) * 4u))
-#define CS_SO_BOFF (CS_SO_BCOUNT + CS_STATIC_ALIGN((CS_MAX_SPLITTERS + 1u) * 4u))
-#define CS_SO_CANDKM (CS_SO_BOFF + CS_STATIC_ALIGN((CS_MAX_SPLITTERS + 2u) * 4u))
+#define CS_SO_CANDKM (CS_SO_BCOUNT + CS_STATIC_ALIGN((CS_MAX_SPLITTERS + 1u) * 4u))
 #define CS_SO_SORTKM (CS_SO_CANDKM + CS_STATIC_MAX_BLOCKS * 8u)
 #define CS_SO_CANDID (CS_SO_SORTKM + CS_STATIC_MAX_BLOCKS * 8u)
 #define CS_SO_CANDBKT (CS_SO_CANDID + CS_STATIC_MAX_BLOCKS * 4u)
@@ -1245,7 +1247,6 @@ extern "C" int cs_select_victims_static(const cs_params *p, const float *fsurv, 
     ws.spl_km = (unsigned long long *)(base + CS_SO_SPLKM);
     ws.spl_id = (uint32_t *)(base + CS_SO_SPLID);
     ws.bcount = (uint32_t *)(base + CS_SO_BCOUNT);
-    ws.boff = (uint32_t *)(base + CS_SO_BOFF);
     ws.cand_km = (unsigned long long *)(base + CS_SO_CANDKM);
     ws.sort_km = (unsigned long long *)(base + CS_SO_SORTKM);
     ws.cand_id = (uint32_t *)(base + CS_SO_CANDID);
