@@ -262,6 +262,7 @@ cs_normalise_kernel(cs_workspace ws, uint32_t A, uint32_t W, float eps, float ta
     __shared__ uint32_t s_evc[OBS_FUSED_MAX];        // the batch: chain of event e,
     __shared__ uint16_t s_eva[OBS_FUSED_MAX];        // its agent (CS_AGENT_NONE: skipped),
     __shared__ uint16_t s_evp[OBS_FUSED_MAX];        // and the agent it follows when that is a counted transition
+    __shared__ uint8_t s_succ[OBS_FUSED_MAX];        // 1: a later live event of the batch has the same chain
     __shared__ uint32_t s_add[CS_MAX_AGENTS];        // what the batch adds to the row being worked on
     __shared__ int s_last_live;
     __shared__ double s_red[64];
@@ -298,6 +299,7 @@ cs_normalise_kernel(cs_workspace ws, uint32_t A, uint32_t W, float eps, float ta
         }
         s_evc[tid] = c;
         s_eva[tid] = (uint16_t)a;
+        s_succ[tid] = 0;
         __syncthreads();
         const bool live = tid < n_events && a != CS_AGENT_NONE;
         uint32_t prev = CS_AGENT_NONE;
@@ -306,6 +308,7 @@ cs_normalise_kernel(cs_workspace ws, uint32_t A, uint32_t W, float eps, float ta
             for (; j >= 0; --j)
                 if (s_evc[j] == c && s_eva[j] != CS_AGENT_NONE) { prev = s_eva[j]; break; }
             if (j < 0) prev = ws.cur[c];
+            else s_succ[j] = 1;                                // event j is not the last of its chain in this batch
             atomicMax(&s_last_live, (int)tid);
         }
         const bool counted = live && prev != CS_AGENT_NONE && prev != a;
@@ -398,11 +401,7 @@ cs_normalise_kernel(cs_workspace ws, uint32_t A, uint32_t W, float eps, float ta
         // the batch's effect on what all CTAs share (every other CTA is done reading it)
         const uint32_t a = tid < n_events ? s_eva[tid] : CS_AGENT_NONE;
         if (a != CS_AGENT_NONE) {
-            const uint32_t c = s_evc[tid];
-            bool last_of_chain = true;
-            for (uint32_t q = tid + 1; q < n_events; ++q)
-                if (s_evc[q] == c && s_eva[q] != CS_AGENT_NONE) { last_of_chain = false; break; }
-            if (last_of_chain) ws.cur[c] = (uint16_t)a;
+            if (!s_succ[tid]) ws.cur[s_evc[tid]] = (uint16_t)a;       // the chain's last live event of the batch
         }
         if (all_chains) __threadfence();                      // (cur[] is read back below when every chain is a source)
         if (s_last_live >= 0) la = s_eva[s_last_live];

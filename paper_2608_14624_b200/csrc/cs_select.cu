@@ -398,7 +398,11 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_fast_kernel(SelArgs a, cs_
     unsigned long long *s_km = (unsigned long long *)(((uintptr_t)queues + 7) & ~(uintptr_t)7);   // the queues are idle now
     uint32_t *s_id = (uint32_t *)(s_km + CS_SAMPLE);
     if (threadIdx.x >= HALF) {
-        if (small) publish_splitters(ws, s_km, s_id, c_use, a.sort_cap, CS_SAMPLE / 2, CtaPart{threadIdx.x - HALF, HALF, 2u});
+        if (small) {
+            // a sample of at least twice the splitters (c / 64 of them): 128, 256 or 512 keys
+            const uint32_t P = c_use <= 4096u ? 128u : (c_use <= 8192u ? 256u : CS_SAMPLE / 2);
+            publish_splitters(ws, s_km, s_id, c_use, a.sort_cap, P, CtaPart{threadIdx.x - HALF, HALF, 2u});
+        }
     } else {
         const CtaPart cp{threadIdx.x, HALF, 1u};
         constexpr uint32_t PER = CS_HIST_BINS / HALF;
