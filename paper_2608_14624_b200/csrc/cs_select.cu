@@ -819,10 +819,18 @@ __global__ void __launch_bounds__(256) cs_sel_bucket_kernel(cs_workspace ws, uin
         for (int u = 0; u < ITEMS; ++u) pos[u] = 0;
 #pragma unroll 1
         for (uint32_t step = 128; step > 0; step >>= 1) {
+            unsigned long long sk[ITEMS];
+            uint32_t si[ITEMS];
 #pragma unroll
-            for (int u = 0; u < ITEMS; ++u) {
+            for (int u = 0; u < ITEMS; ++u) {                 // the step's eight loads first, ...
                 const uint32_t probe = pos[u] + step - 1u;
-                if (!key_less(km[u], id[u], s_km[probe], s_id[probe])) pos[u] += step;
+                sk[u] = s_km[probe];
+                si[u] = s_id[probe];
+            }
+#pragma unroll
+            for (int u = 0; u < ITEMS; ++u) {                 // ... then the compares, with no short-circuit branch
+                const bool lt = (km[u] < sk[u]) | ((km[u] == sk[u]) & (id[u] < si[u]));
+                pos[u] += lt ? 0u : step;
             }
         }
 #pragma unroll
