@@ -993,7 +993,9 @@ def metadata_scale(torch, cs, synth, dev, hbm_peak, calls=10000):
             "target_frac_of_hbm_peak": 0.60, "target_met": bool(algo_bytes / best / 1e9 / hbm_peak >= 0.60),
             "note": "11 MB of metadata per call: at 0.60 of the HBM peak a call would last 2.6 us, less than one kernel launch; "
                     "the call is latency-bound and the fraction is reported as measured",
-            "selects_counted_by_the_kernels": cn["selects"], "n_out": [int(vn[0].item()), int(pn[0].item())],
+            "selects_counted_by_the_kernels": cn["selects"], "selects_whose_threshold_held": cn["fast_hits"],
+            "selects_with_buckets_filled_in_place": cn["region_selects"], "of_those_regrouped": cn["region_overflows"],
+            "n_out": [int(vn[0].item()), int(pn[0].item())],
             "device_status": c.get_status()}
 
 

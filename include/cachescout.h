@@ -368,6 +368,8 @@ typedef struct cs_counters {
     uint64_t blocks_moved[3];       /* blocks copied, per direction */
     uint64_t bytes_moved[3];        /* their bytes (block_bytes each) */
     uint64_t blocks_skipped;        /* mover list entries skipped: CS_ID_NONE or slot out of range */
+    uint64_t region_selects[3];     /* multi-launch selects whose sample-sort buckets were filled in place (cs_set_select_bucket_regions) */
+    uint64_t region_overflows[3];   /* of those: a bucket outgrew its region and the buckets were grouped by a launch of their own */
 } cs_counters;
 
 /* Synchronises `stream` and copies the counters to *out (host memory); reset != 0 clears them afterwards. */
@@ -460,6 +462,15 @@ int cs_set_select_path(cs_ctx *ctx, uint32_t path);
  * builds its histogram; when the new threshold is not above the remembered one the index is read
  * once instead of twice.  The result never depends on it.  enabled = 0 turns the speculation off. */
 int cs_set_select_speculation(cs_ctx *ctx, uint32_t enabled);
+
+/* The multi-launch select orders its candidates by a sample sort into <= 256 buckets.  When the candidates are few
+ * for the size of the workspace (8 c <= max_blocks) every bucket owns a fixed region of the sort arrays --
+ * max_blocks / (buckets) keys, at most 2048 -- which the bucket launch fills directly; a bucket that outgrows its
+ * region makes the call fall back to grouping the buckets in a launch of its own.  max_keys caps that region
+ * (0 = no cap, the default; 1 = every bucket with two keys or more takes the fallback).  The result never depends
+ * on it: the setting exists so that both routes can be exercised and compared.  Host-side, takes effect from the
+ * next select call. */
+int cs_set_select_bucket_regions(cs_ctx *ctx, uint32_t max_keys);
 
 /* Clock source for CUDA-graph replay (the paper's runtime reads now() when a block is touched, Algorithm 1;
  * a captured call would freeze its `now` argument).  While now_dev (dev, 4-byte aligned) is set, every

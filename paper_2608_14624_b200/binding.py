@@ -35,7 +35,7 @@ EXPORTS = ("cs_workspace_bytes", "cs_create", "cs_destroy", "cs_observe_invocati
            "cs_exact_survival", "cs_use_survival_table", "cs_import_state", "cs_set_select_speculation", "cs_exchange_blocks", "cs_step", "cs_set_survival_sources", "cs_select_step",
            "cs_get_counters", "cs_validate_selection", "cs_validate_move_lists", "cs_validate_exchange_lists",
            "cs_selftest_bounded_wait", "cs_set_device_clock", "cs_set_mover_staging", "cs_exchange_blocks_staged",
-           "cs_offload_blocks_staged", "cs_prefetch_blocks_staged")
+           "cs_offload_blocks_staged", "cs_prefetch_blocks_staged", "cs_set_select_bucket_regions")
 
 
 class cs_params(C.Structure):
@@ -71,7 +71,8 @@ class cs_counters(C.Structure):
     _fields_ = [("events_seen", C.c_uint64), ("events_skipped", C.c_uint64), ("transitions_counted", C.c_uint64),
                 ("selects", C.c_uint64 * 3), ("eligible", C.c_uint64 * 3), ("selected", C.c_uint64 * 3),
                 ("candidates", C.c_uint64 * 3), ("fast_hits", C.c_uint64 * 3),
-                ("blocks_moved", C.c_uint64 * 3), ("bytes_moved", C.c_uint64 * 3), ("blocks_skipped", C.c_uint64)]
+                ("blocks_moved", C.c_uint64 * 3), ("bytes_moved", C.c_uint64 * 3), ("blocks_skipped", C.c_uint64),
+                ("region_selects", C.c_uint64 * 3), ("region_overflows", C.c_uint64 * 3)]
 
 
 class CacheScoutError(RuntimeError):
@@ -119,6 +120,7 @@ def lib():
         L.cs_set_mover_path.argtypes = [vp, u32]
         L.cs_set_select_path.argtypes = [vp, u32]
         L.cs_set_select_speculation.argtypes = [vp, u32]
+        L.cs_set_select_bucket_regions.argtypes = [vp, u32]
         L.cs_exact_survival.argtypes = [vp, u32, u32, vp, vp, vp]
         L.cs_use_survival_table.argtypes = [vp, vp]
         L.cs_import_state.argtypes = [vp, vp, vp, u32, vp]
@@ -362,6 +364,10 @@ def cs_use_survival_table(ctx, fsurv):
 
 def cs_set_select_speculation(ctx, enabled: bool):
     _chk(lib().cs_set_select_speculation(ctx, 1 if enabled else 0), "cs_set_select_speculation")
+
+
+def cs_set_select_bucket_regions(ctx, max_keys: int):
+    _chk(lib().cs_set_select_bucket_regions(ctx, int(max_keys)), "cs_set_select_bucket_regions")
 
 
 def cs_set_select_path(ctx, path: int):
@@ -627,6 +633,9 @@ class CacheScout:
 
     def set_select_speculation(self, enabled: bool):
         cs_set_select_speculation(self.ctx, enabled)
+
+    def set_select_bucket_regions(self, max_keys: int):
+        cs_set_select_bucket_regions(self.ctx, max_keys)
 
     def set_select_path(self, path: int):
         cs_set_select_path(self.ctx, path)

@@ -146,7 +146,7 @@ __global__ void cs_status_swap_kernel(cs_scalars *sc)
 
 extern "C" {
 
-int cs_version(void) { return 200; }
+int cs_version(void) { return 201; }
 
 const char *cs_strerror(int code)
 {
@@ -628,6 +628,13 @@ int cs_set_select_speculation(cs_ctx *ctx, uint32_t enabled)
 {
     if (!ctx) return CS_EINVAL;
     ctx->no_speculation = enabled ? 0u : 1u;
+    return CS_OK;
+}
+
+int cs_set_select_bucket_regions(cs_ctx *ctx, uint32_t max_keys)
+{
+    if (!ctx) return CS_EINVAL;
+    ctx->region_cap_max = max_keys;
     return CS_OK;
 }
 

@@ -125,6 +125,7 @@ struct cs_ctx {
     uint32_t mover_path;   // CS_MOVER_*
     uint32_t select_path;  // CS_SELECT_*
     uint32_t no_speculation;       // 1: the histogram pass never collects ahead of the threshold
+    uint32_t region_cap_max;       // cap on the keys of a bucket's own region in the sort arrays (0: none)
     uint32_t source_mode;          // CS_SOURCES_*: where the cached BFS of Eq. 8 starts
     const float *fsurv_override;   // caller's survival table for score / select, NULL = the BFS table of Eq. 8
     const uint32_t *clock_dev;           // cs_set_device_clock(): selects and scores read the clock from here when they run

@@ -80,7 +80,8 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_score_kernel(SelArgs a, cs_wor
 #define RANK_TILE 2048u                 // keys of the shared-memory tile a bucket is sorted in
 #define CS_SPLIT_SAMPLE_MAX 32768u      // up to this many candidates half a CTA sorts a 512-key sample (fast pass)
 __device__ __forceinline__ void publish_splitters(const cs_workspace &ws, unsigned long long *s_km, uint32_t *s_id,
-                                                  uint32_t c, uint32_t sort_cap, uint32_t P, const CtaPart &cp)
+                                                  uint32_t c, uint32_t sort_cap, uint32_t region_cap_max, uint32_t P,
+                                                  const CtaPart &cp)
 {
     const uint32_t n_samp = c < P ? c : P;
     {
@@ -116,6 +117,7 @@ __device__ __forceinline__ void publish_splitters(const cs_workspace &ws, unsign
     if (cp.t == 0) {
         uint32_t cap = sort_cap / (n_spl + 1u);
         if (cap > RANK_TILE) cap = RANK_TILE;
+        if (region_cap_max && cap > region_cap_max) cap = region_cap_max;
         ws.sel->n_spl = n_spl;
         ws.sel->placed = (c && 8ull * c <= sort_cap) ? 1u : 0u;
         ws.sel->cap = cap;
@@ -401,7 +403,7 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_fast_kernel(SelArgs a, cs_
         if (small) {
             // a sample of at least twice the splitters (c / 64 of them): 128, 256 or 512 keys
             const uint32_t P = c_use <= 4096u ? 128u : (c_use <= 8192u ? 256u : CS_SAMPLE / 2);
-            publish_splitters(ws, s_km, s_id, c_use, a.sort_cap, P, CtaPart{threadIdx.x - HALF, HALF, 2u});
+            publish_splitters(ws, s_km, s_id, c_use, a.sort_cap, a.region_cap_max, P, CtaPart{threadIdx.x - HALF, HALF, 2u});
         }
     } else {
         const CtaPart cp{threadIdx.x, HALF, 1u};
@@ -455,7 +457,7 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_fast_kernel(SelArgs a, cs_
     }
     __syncthreads();
     const bool hit = s_flag;
-    if (hit && !small) publish_splitters(ws, s_km, s_id, c_use, a.sort_cap, CS_SAMPLE, whole_cta());
+    if (hit && !small) publish_splitters(ws, s_km, s_id, c_use, a.sort_cap, a.region_cap_max, CS_SAMPLE, whole_cta());
     if (threadIdx.x == 0) {
         ws.sel->spec = hit ? 1u : 0u;
         ws.sel->c_spec = 0;
@@ -696,7 +698,7 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_collect_kernel(SelArgs a, 
     if (!last_cta_done(&ws.sel->ticket[2], &s_flag)) return;
 
     // ---- last CTA: sample, sort the sample (bitonic, shared memory), publish splitters -----------
-    publish_splitters(ws, s_km, s_id, __ldcg(&ws.sel->c), a.sort_cap, CS_SAMPLE, whole_cta());
+    publish_splitters(ws, s_km, s_id, __ldcg(&ws.sel->c), a.sort_cap, a.region_cap_max, CS_SAMPLE, whole_cta());
     if (threadIdx.x == 0) { ws.sel->ticket[2] = 0; count_candidates(ws, a.kind, __ldcg(&ws.sel->c), false); }
 }
 
@@ -909,7 +911,7 @@ __global__ void __launch_bounds__(256) cs_sel_scatter_kernel(cs_workspace ws)
 // (O(m log^2 m), so an unlucky large bucket costs little more than an average one), after which
 // position i of the bucket is position offset + i of the output list.
 __global__ void __launch_bounds__(256)
-cs_sel_rank_kernel(cs_workspace ws, uint32_t k, uint32_t *__restrict__ ids_out, uint32_t *__restrict__ n_out_dev)
+cs_sel_rank_kernel(cs_workspace ws, uint32_t k, uint32_t kind, uint32_t *__restrict__ ids_out, uint32_t *__restrict__ n_out_dev)
 {
     __shared__ unsigned long long t_km[RANK_TILE];
     __shared__ uint32_t t_id[RANK_TILE];
@@ -921,7 +923,13 @@ cs_sel_rank_kernel(cs_workspace ws, uint32_t k, uint32_t *__restrict__ ids_out, 
     const bool in_regions = ws.sel->placed && !ws.sel->overflow;
     const uint32_t gtid = blockIdx.x * blockDim.x + threadIdx.x, nth = gridDim.x * blockDim.x;
     for (uint32_t i = n_out + gtid; i < k; i += nth) ids_out[i] = CS_ID_NONE;
-    if (gtid == 0) *n_out_dev = n_out;
+    if (gtid == 0) {
+        *n_out_dev = n_out;
+        if (ws.sel->placed && kind < 3) {                     // work counters: how the buckets got to their places
+            atomicAdd((unsigned long long *)&ws.cnt->region_selects[kind], 1ull);
+            if (ws.sel->overflow) atomicAdd((unsigned long long *)&ws.cnt->region_overflows[kind], 1ull);
+        }
+    }
     if (n_out == 0) return;
     const uint32_t b_last = bucket_offsets(ws, ws.sel->n_spl, n_out, s_off, s_tmp);
     for (uint32_t b = blockIdx.x; b <= b_last; b += gridDim.x) {
@@ -975,6 +983,7 @@ void cs_fill_sel_args(const cs_ctx *ctx, const cs_block_index *idx, uint32_t now
     a.kind = 0;
     a.now_dev = ctx->step_now_dev ? ctx->step_now_dev : ctx->clock_dev;
     a.sort_cap = 0;
+    a.region_cap_max = ctx->region_cap_max;
 }
 
 uint32_t cs_scan_grid(const cs_ctx *ctx, uint32_t n, uint32_t per_cta, uint32_t ctas_per_sm)
@@ -1069,7 +1078,7 @@ static int launch_select_job(cs_ctx *ctx, int job, const cs_block_index *idx, ui
     if ((rc = cs_check_launch(ctx)) != CS_OK) return rc;
     cs_launch_chained(cs_sel_scatter_kernel, grid_c, 256, 0, s, ws);
     if ((rc = cs_check_launch(ctx)) != CS_OK) return rc;
-    cs_launch_chained(cs_sel_rank_kernel, CS_MAX_SPLITTERS + 1, 256, 0, s, ws, k, ids_out, n_out);
+    cs_launch_chained(cs_sel_rank_kernel, CS_MAX_SPLITTERS + 1, 256, 0, s, ws, k, a.kind, ids_out, n_out);
     return cs_check_launch(ctx);
 }
 

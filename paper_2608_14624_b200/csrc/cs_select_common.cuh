@@ -23,6 +23,7 @@ struct SelArgs {
     uint32_t kind;                // 0 GPU-tier victims, 1 host-tier victims, 2 prefetch candidates (work counters)
     const uint32_t *now_dev;      // when set, the clock is read from device memory at execution time (graph replay)
     uint32_t sort_cap;            // keys the sort region holds (0: buckets never get fixed regions)
+    uint32_t region_cap_max;      // cap on a bucket's own region (0: none)
 };
 
 // host helpers defined in cs_select.cu

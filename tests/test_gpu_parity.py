@@ -695,6 +695,28 @@ def test_select_large_index_uses_age_limits(with_tokens, prefer):
     assert c.get_status() == 0
 
 
+@pytest.mark.parametrize("max_keys", [0, 1, 40, 100_000])
+def test_bucket_regions_and_their_fallback(max_keys):
+    """With few candidates the sample sort's buckets live in fixed regions of the sort arrays that the bucket launch
+    fills directly; a bucket that outgrows its region sends the call down the general route (buckets grouped by a
+    launch of its own).  Capping the region (1 and 40 keys against buckets of ~64) forces that route on every call;
+    the lists must not change.  Three clocks in a row, so that both the first call (full histogram and collect passes)
+    and the calls that reuse the remembered threshold are covered; the cluster path is unaffected by the setting."""
+    cfg = synth.CONFIGS["meta1m"]
+    n = 400_000
+    c, o = warm_state(cfg, 3000, n, r_min=0.02)
+    c.set_select_bucket_regions(max_keys)
+    idx = synth.make_block_index(cfg, n=n, tier="random")
+    for now in (100_000, 100_001, 100_007):
+        assert run_selects(c, o, idx, now, (9_000, 700)) == 0
+    cn = c.counters()
+    assert all(x > 0 for x in cn["region_selects"])          # 8 c <= 400,000 for k = 700, and mostly for k = 9,000
+    if max_keys in (1, 40):
+        assert all(x > 0 for x in cn["region_overflows"])
+    else:
+        assert cn["region_overflows"] == [0, 0, 0]
+
+
 # ---- hop table from every live session's current agent ----------------------------------------------------
 @pytest.mark.parametrize("name,n_inv", [("tiny", 60), ("llama8b", 400), ("meta1m", 3000)])
 def test_survival_from_all_chains(name, n_inv):
