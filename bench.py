@@ -63,6 +63,9 @@ def parse_args():
                     help="'mover'/'select' run one small case of that kernel family only (profiler captures)")
     ap.add_argument("--kineto", action="store_true",
                     help="with --workload select / select80k: warm per-kernel device times from the CUDA profiler API (torch.profiler)")
+    ap.add_argument("--phase-stamps", action="store_true",
+                    help="with --workload select: build the profiling variant of the library (kernels store the GPU's global "
+                         "timer at phase boundaries) and print where the time of a graph-replayed metadata-scale call goes")
     ap.add_argument("--skip-aux", action="store_true",
                     help="timed steps only: no link-peak probe, end-to-end pass, extras or CPU baseline (profiler launch lists)")
     return ap.parse_args()
@@ -1125,6 +1128,81 @@ def run_reference(args):
     }))
 
 
+PHASE_NAMES = {0: "refresh: entry", 1: "refresh: dependency wait over", 2: "refresh: rows of CTA 0 done (events applied, Eq. 3, arg-max, adjacency)",
+               3: "refresh: last CTA starts", 4: "refresh: cur[] / last agent written, Eq. 2 done", 5: "refresh: BFS and Eq. 8 done",
+               8: "scan: entry", 9: "scan: tables, thresholds, histogram set up", 10: "scan: dependency wait over",
+               11: "scan: index read, queues worked off (CTA 0)", 12: "scan: candidates and histogram flushed (CTA 0)",
+               13: "scan: last CTA starts", 14: "scan: threshold found, splitters published",
+               24: "bucket: dependency wait over (histogram and collect launches returned)", 25: "bucket: CTA 0 done",
+               26: "scatter: dependency wait over", 27: "rank: dependency wait over", 28: "rank: CTA 0 done"}
+
+
+def phase_timeline(args, torch, device):
+    """Where the time of one metadata-scale call goes (1,000,000 entries, 256 agents: observe 64 events, 10,000 victims,
+    2,000 prefetch candidates as one cs_select_step, replayed from a CUDA graph).  Needs the profiling build of the
+    library: every kernel stores the GPU's global nanosecond timer at its phase boundaries, read back after each call.
+    Prints medians over the calls after a warm-up, in microseconds from the first stamp of the call."""
+    from paper_2608_14624_b200 import binding as cs
+    from paper_2608_14624_b200 import build
+    from tests import synth
+    assert cs._lib is None, "the library is loaded already"
+    cs.LIB_PATH = build.build_stamped_library()                           # the binding loads it on first use
+    cfg = synth.CONFIGS["meta1m"]
+    N, calls, warm = 1_000_000, max(20, args.steps), 20
+    d = cs.DeviceIndex.from_host(synth.make_block_index(cfg, n=N, tier="random"), device)
+    tr = synth.make_trace(cfg, n_invocations=64 * (calls + warm + 40))
+    c = cs.CacheScout(cs.make_params(n_agents=cfg.n_agents, n_chains=cfg.n_chains, max_blocks=N, block_tokens=cfg.block_tokens,
+                                     r_min=0.02), device)
+    ch, ag = torch.from_numpy(tr.chain).to(device), torch.from_numpy(tr.agent).to(device)
+    c.observe_invocations(ch[:64 * 30], ag[:64 * 30], None)
+    v = torch.empty(cfg.k_victims, dtype=torch.int32, device=device)
+    pf = torch.empty(cfg.k_prefetch, dtype=torch.int32, device=device)
+    vn, pn = torch.zeros(4, dtype=torch.int32, device=device), torch.zeros(4, dtype=torch.int32, device=device)
+    la = d.last_access.view(torch.int32)
+    fifo = [torch.zeros(cfg.k_prefetch, dtype=torch.int64, device=device) for _ in range(8)]
+    now_d = torch.zeros(4, dtype=torch.int32, device=device)
+    ev_c, ev_a = torch.zeros(64, dtype=ch.dtype, device=device), torch.zeros(64, dtype=ag.dtype, device=device)
+    cap = torch.cuda.Stream(device=device)
+    cap.wait_stream(torch.cuda.current_stream())
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=cap, capture_error_mode="relaxed"):
+        c.observe_invocations(ev_c, ev_a, None, stream=cap)
+        c.set_device_clock(now_d)
+        c.select_step(d, 0, cfg.k_victims, cfg.k_prefetch, v, vn, None, None, pf, pn, stream=cap)
+        c.set_device_clock(None)
+    cap.synchronize()
+    rows, timed = [], []
+    with torch.cuda.stream(cap):
+        for i in range(calls + warm):
+            now, lo = 100_000 + i, 64 * (30 + i)
+            ev_c.copy_(ch[lo:lo + 64]); ev_a.copy_(ag[lo:lo + 64]); now_d.fill_(now)
+            torch.cuda._sleep(400_000)                                     # the host gets ahead: nothing below waits for it
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(cap); g.replay(); e1.record(cap)
+            cap.synchronize()
+            if i >= warm:
+                timed.append(e0.elapsed_time(e1) * 1e3)
+                rows.append(np.array(c.phase_stamps(), dtype=np.int64))
+            la[v.long().clamp_(min=0)] = now                              # the index evolves as in metadata_scale
+            pi = pf.long().clamp_(min=0); d.flags[pi] &= 0xFB
+            if i >= 8:
+                d.flags[fifo[i % 8]] |= 4
+            fifo[i % 8].copy_(pi)
+            cap.synchronize()
+    R = np.stack(rows)
+    rel = (R - R[:, 0:1]) / 1000.0
+    line = {"workload": "phase stamps: metadata-scale call replayed from a CUDA graph", "calls": calls,
+            "event_timed_us_median": float(np.median(timed)), "fast_hits": c.counters()["fast_hits"], "phases_us_median": []}
+    for base, who in ((0, ""), (8, " [victims]"), (16, " [prefetch]"), (24, " [victims]"), (32, " [prefetch]")):
+        for k in range(8):
+            name = PHASE_NAMES.get((base if base < 16 else base - (8 if base in (16, 32) else 0)) + k)
+            if name is None or R[0, base + k] == 0:
+                continue
+            line["phases_us_median"].append([round(float(np.median(rel[:, base + k])), 2), name + who])
+    line["phases_us_median"].sort()
+    print(json.dumps(line))
+
+
 def profile_case(args, torch, device):
     """Small cases for profiler captures (a few GB on the device, inputs larger than L2).
     mover : 2,048-block GPU pool (4 GiB), 512-slot pinned host tier (1 GiB); per step one
@@ -1137,6 +1215,8 @@ def profile_case(args, torch, device):
     from paper_2608_14624_b200 import binding as cs
     from paper_2608_14624_b200 import build
     from tests import synth
+    if args.phase_stamps:
+        return phase_timeline(args, torch, device)
     build.build_library()
     if args.workload in ("select16m", "select64m"):
         # one kind of select over an index far larger than L2 (176 MB / 704 MB of metadata): the regime in which the

@@ -408,6 +408,15 @@ int cs_validate_exchange_lists(cs_ctx *ctx, const cs_kv_pool *gpu, const cs_kv_p
  * is in flight, so nothing is left behind; the context stays usable. */
 int cs_selftest_bounded_wait(cs_ctx *ctx, uint32_t max_polls, cs_stream_t stream);
 
+/* Phase stamps of the latest calls (profiling builds only: a library compiled with -DCS_PHASE_STAMPS makes its kernels
+ * store the GPU's global nanosecond timer at phase boundaries -- refresh: entry, dependency wait over, rows done, last
+ * CTA starts, sums done, end; scans: entry, set-up done, wait over, index read, flushed, last CTA starts, tail done;
+ * ordering: bucket wait over / done, scatter wait over, rank wait over / done -- slots as in the CS_PS_* list of
+ * csrc/cs_common.cuh, the prefetch select's eight slots above the victims').  Synchronises the device and copies the
+ * CS_PHASE_STAMP_SLOTS stamps to `out` (host).  An ordinary build returns CS_ENOTIMPL and stores nothing. */
+#define CS_PHASE_STAMP_SLOTS 64
+int cs_debug_phase_stamps(cs_ctx *ctx, uint64_t *out);
+
 /* Width of the mover (0 keeps the default): for transfers that cross the host link and for
  * device-to-device moves.  Unit: warp pipelines on the bulk path (each keeps up to two loads and two
  * stores of 16 KiB in flight; defaults 8 offload / 24 prefetch / 2 per SM device-to-device), CTAs of

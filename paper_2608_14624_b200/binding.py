@@ -35,7 +35,7 @@ EXPORTS = ("cs_workspace_bytes", "cs_create", "cs_destroy", "cs_observe_invocati
            "cs_exact_survival", "cs_use_survival_table", "cs_import_state", "cs_set_select_speculation", "cs_exchange_blocks", "cs_step", "cs_set_survival_sources", "cs_select_step",
            "cs_get_counters", "cs_validate_selection", "cs_validate_move_lists", "cs_validate_exchange_lists",
            "cs_selftest_bounded_wait", "cs_set_device_clock", "cs_set_mover_staging", "cs_exchange_blocks_staged",
-           "cs_offload_blocks_staged", "cs_prefetch_blocks_staged", "cs_set_select_bucket_regions")
+           "cs_offload_blocks_staged", "cs_prefetch_blocks_staged", "cs_set_select_bucket_regions", "cs_debug_phase_stamps")
 
 
 class cs_params(C.Structure):
@@ -121,6 +121,7 @@ def lib():
         L.cs_set_select_path.argtypes = [vp, u32]
         L.cs_set_select_speculation.argtypes = [vp, u32]
         L.cs_set_select_bucket_regions.argtypes = [vp, u32]
+        L.cs_debug_phase_stamps.argtypes = [vp, vp]
         L.cs_exact_survival.argtypes = [vp, u32, u32, vp, vp, vp]
         L.cs_use_survival_table.argtypes = [vp, vp]
         L.cs_import_state.argtypes = [vp, vp, vp, u32, vp]
@@ -366,8 +367,16 @@ def cs_set_select_speculation(ctx, enabled: bool):
     _chk(lib().cs_set_select_speculation(ctx, 1 if enabled else 0), "cs_set_select_speculation")
 
 
+def cs_debug_phase_stamps(ctx):
+    """Phase stamps (ns of the GPU's global timer) of the latest calls as a list; a library built without
+    -DCS_PHASE_STAMPS raises CS_ENOTIMPL."""
+    out = (C.c_uint64 * 64)()
+    _chk(lib().cs_debug_phase_stamps(ctx, C.cast(out, C.c_void_p)), "cs_debug_phase_stamps")
+    return list(out)
+
+
 def cs_set_select_bucket_regions(ctx, max_keys: int):
-    _chk(lib().cs_set_select_bucket_regions(ctx, int(max_keys)), "cs_set_select_bucket_regions")
+    _chk(lib().cs_set_select_bucket_regions(ctx, int(max_keys)), "cs_set_select_bucket_regions", "cs_debug_phase_stamps")
 
 
 def cs_set_select_path(ctx, path: int):
@@ -636,6 +645,9 @@ class CacheScout:
 
     def set_select_bucket_regions(self, max_keys: int):
         cs_set_select_bucket_regions(self.ctx, max_keys)
+
+    def phase_stamps(self):
+        return cs_debug_phase_stamps(self.ctx)
 
     def set_select_path(self, path: int):
         cs_set_select_path(self.ctx, path)

@@ -31,6 +31,21 @@ def _stale() -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
+LIB_STAMPS = os.path.join(HERE, "libcachescout_stamps.so")     # the same sources with -DCS_PHASE_STAMPS (profiling)
+
+
+def build_stamped_library() -> str:
+    """The profiling build: kernels store the global timer at phase boundaries (cs_debug_phase_stamps)."""
+    nvcc = os.environ.get("NVCC", "nvcc")
+    cmd = [nvcc] + [f for f in NVCC_FLAGS if f not in ("-Xptxas", "-v")] + ["-DCS_PHASE_STAMPS", "-I", os.path.join(ROOT, "include"),
+                                                                          "-I", CSRC, "-o", LIB_STAMPS] + sources()
+    res = subprocess.run(cmd, capture_output=True, text=True)
+    if res.returncode != 0:
+        sys.stderr.write(res.stdout + res.stderr)
+        raise RuntimeError("nvcc failed building libcachescout_stamps.so")
+    return LIB_STAMPS
+
+
 def build_library(force: bool = False, verbose: bool = False) -> str:
     """Compile every .cu under csrc/ into one shared library; returns its path."""
     if not force and not _stale():

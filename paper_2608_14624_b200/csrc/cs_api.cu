@@ -638,6 +638,20 @@ int cs_set_select_bucket_regions(cs_ctx *ctx, uint32_t max_keys)
     return CS_OK;
 }
 
+int cs_debug_phase_stamps(cs_ctx *ctx, uint64_t *out)
+{
+    if (!ctx || !out) return CS_EINVAL;
+#ifdef CS_PHASE_STAMPS
+    static_assert(CS_PHASE_STAMP_SLOTS == CS_N_PHASE_STAMPS, "header and kernels disagree on the number of stamps");
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e == cudaSuccess) e = cudaMemcpy(out, ctx->ws.sc->stamps, sizeof(uint64_t) * CS_N_PHASE_STAMPS, cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; return CS_ECUDA; }
+    return CS_OK;
+#else
+    return CS_ENOTIMPL;
+#endif
+}
+
 int cs_last_cuda_error(cs_ctx *ctx) { return ctx ? ctx->last_cuda_error : 0; }
 
 } // extern "C"

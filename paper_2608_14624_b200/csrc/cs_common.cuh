@@ -40,6 +40,32 @@ struct cs_nvtx_range {
 #define CS_GTAB_MAX 4096u          // largest recency table kept in shared memory (ages below saturation)
 
 // Scalars the kernels share, one 256-byte line in the workspace.
+// Phase stamps (builds with -DCS_PHASE_STAMPS only; cs_debug_phase_stamps() reads them).  A call's kernels are chains
+// of dependent steps whose cost is latency, not work, so "where does the time go" is answered by the GPU's global
+// nanosecond timer read at the boundaries: CS_STAMP(ws, slot, cond) stores it into slot `slot` when `cond` holds
+// (one thread of one CTA).  In ordinary builds the macro is empty and the slots do not exist.
+#define CS_N_PHASE_STAMPS 64
+enum {
+    CS_PS_REFRESH_ENTRY = 0, CS_PS_REFRESH_WAITED, CS_PS_REFRESH_ROWS_DONE, CS_PS_REFRESH_LAST_CTA, CS_PS_REFRESH_SUMS_DONE,
+    CS_PS_REFRESH_END,
+    CS_PS_SCAN_ENTRY = 8,       // + 8 for the prefetch select: entry, set-up done, waited, index read, flushed, last CTA, tail done
+    CS_PS_SCAN_SETUP, CS_PS_SCAN_WAITED, CS_PS_SCAN_READ, CS_PS_SCAN_FLUSHED, CS_PS_SCAN_LAST_CTA, CS_PS_SCAN_TAIL_DONE,
+    CS_PS_BUCKET_WAITED = 24,   // + 8 for the prefetch select: bucket waited / done, scatter waited, rank waited / done
+    CS_PS_BUCKET_DONE, CS_PS_SCATTER_WAITED, CS_PS_RANK_WAITED, CS_PS_RANK_DONE
+};
+#ifdef CS_PHASE_STAMPS
+#define CS_STAMP(ws, slot, cond)                                                         \
+    do {                                                                                 \
+        if (cond) {                                                                      \
+            unsigned long long cs_t_;                                                    \
+            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(cs_t_)::"memory");          \
+            (ws).sc->stamps[slot] = cs_t_;                                               \
+        }                                                                                \
+    } while (0)
+#else
+#define CS_STAMP(ws, slot, cond) do { } while (0)
+#endif
+
 struct cs_scalars {
     uint32_t status;        // CS_ST_* bits
     uint32_t last_agent;    // agent of the last non-warmup event, CS_AGENT_NONE initially
@@ -55,6 +81,9 @@ struct cs_scalars {
     uint32_t sel_hint[4];   // bin up to which the next select of each kind (GPU victims, host victims, prefetch)
                             // collects ahead of its own threshold, chosen from the previous call's histogram;
                             // ~0 = none; slot 3 is never written: calls that must not speculate read it
+#ifdef CS_PHASE_STAMPS
+    unsigned long long stamps[CS_N_PHASE_STAMPS];   // %globaltimer at phase boundaries of the latest call (profiling builds)
+#endif
 };
 
 // State of one select in flight, rewritten by every call.  The selects of a step that run side by side each

@@ -272,12 +272,11 @@ cs_normalise_kernel(cs_workspace ws, uint32_t A, uint32_t W, float eps, float ta
     __shared__ uint16_t s_hops[CS_MAX_AGENTS];
     __shared__ bool s_is_last;
     const uint32_t tid = threadIdx.x;
+    CS_STAMP(ws, CS_PS_REFRESH_ENTRY, blockIdx.x == 0 && tid == 0);
     cs_wait_for_predecessor();
+    CS_STAMP(ws, CS_PS_REFRESH_WAITED, blockIdx.x == 0 && tid == 0);
     cs_release_successor();
 
-    // Column sums q_j = sum_i pi_i P_ij of Eq. 2 are accumulated by the row CTAs in 2^-60 fixed
-    // point with integer atomics: integer addition commutes, so the sum is bit-identical from run
-    // to run whatever order the CTAs finish in (a float atomic would not be).
     // ---- a small batch of events is applied here, by every CTA to the rows it owns, instead of by a launch of its
     // own: each CTA stages the batch, finds every event's predecessor (in the batch, else the chain's current agent)
     // exactly as cs_observe_kernel does, and adds the transitions that start at row i to row i.  What is shared --
@@ -316,6 +315,9 @@ cs_normalise_kernel(cs_workspace ws, uint32_t A, uint32_t W, float eps, float ta
         n_new = (uint32_t)__syncthreads_count(counted);
         n_skipped = (uint32_t)__syncthreads_count(tid < n_events && a == CS_AGENT_NONE);
     }
+    // Column sums q_j = sum_i pi_i P_ij of Eq. 2 are accumulated by the row CTAs in 2^-60 fixed
+    // point with integer atomics: integer addition commutes, so the sum is bit-identical from run
+    // to run whatever order the CTAs finish in (a float atomic would not be).
     const uint32_t n_total = ws.sc->n_transitions + n_new;
     const uint32_t fill = ws.sc->adjT_cur ^ 1u;              // every CTA reads this before the last one flips it
     uint32_t *adjT_fill = ws.adjT + (size_t)fill * A * W, *adjT_clear = ws.adjT + (size_t)(fill ^ 1u) * A * W;
@@ -383,6 +385,7 @@ cs_normalise_kernel(cs_workspace ws, uint32_t A, uint32_t W, float eps, float ta
         }
     }
 
+    CS_STAMP(ws, CS_PS_REFRESH_ROWS_DONE, blockIdx.x == 0 && tid == 0);
     // ---- last CTA done: global quantities ---------------------------------------------------------
     __threadfence();
     __syncthreads();
@@ -393,6 +396,7 @@ cs_normalise_kernel(cs_workspace ws, uint32_t A, uint32_t W, float eps, float ta
     __syncthreads();
     if (!s_is_last) return;
     __threadfence();
+    CS_STAMP(ws, CS_PS_REFRESH_LAST_CTA, tid == 0);
 
     BfsRow rowT;                                                         // in flight during the sums
     cs_bfs_load_row(adjT_fill, A, W, rowT);
@@ -425,7 +429,8 @@ cs_normalise_kernel(cs_workspace ws, uint32_t A, uint32_t W, float eps, float ta
         }
     }
     for (uint32_t j = tid; j < A; j += ROW_THREADS) ws.qfix[j] = 0;      // ready for the next refresh
-    cs_block_sum2(Hc, Hm, s_red);                                        // (its barriers also order s_front's zeroes)
+    cs_block_sum2(Hc, Hm, s_red);
+    CS_STAMP(ws, CS_PS_REFRESH_SUMS_DONE, tid == 0);                                        // (its barriers also order s_front's zeroes)
     if (tid == 0) {
         double R = 0.0;
         if (N > 0 && Hm > 0.0) R = 1.0 - Hc / Hm;
@@ -445,6 +450,7 @@ cs_normalise_kernel(cs_workspace ws, uint32_t A, uint32_t W, float eps, float ta
     }
     __syncthreads();
     cs_bfs_survival(ws.adj, A, W, rowT, s_front, s_visit, s_next, s_hops, ws.hops, ws.fsurv, e_max, delta);
+    CS_STAMP(ws, CS_PS_REFRESH_END, tid == 0);
 }
 
 // BFS + Eq. 8 from explicit sources into the temporary tables (cs_score_blocks with sources).

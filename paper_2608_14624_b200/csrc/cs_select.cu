@@ -165,6 +165,8 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_fast_kernel(SelArgs a, cs_
     __shared__ uint32_t s_part[SEL_THREADS];
     __shared__ uint32_t s_b0, s_ahead, s_above;
     __shared__ bool s_flag;
+    constexpr int PS = PF ? 8 : 0;                  // phase-stamp slots of this kind of scan (profiling builds)
+    CS_STAMP(ws, CS_PS_SCAN_ENTRY + PS, blockIdx.x == 0 && threadIdx.x == 0);
     cs_release_successor();
     // Before waiting for the predecessor grid: everything that depends only on the context's constants and on the
     // remembered bin (a stale bin would cost time, never correctness: the result does not depend on H).
@@ -179,7 +181,9 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_fast_kernel(SelArgs a, cs_
         for (uint32_t i = threadIdx.x; i < CS_HIST_BINS; i += blockDim.x) s_hist[i] = 0;
         if (threadIdx.x == 0) s_above = 0;
     }
+    CS_STAMP(ws, CS_PS_SCAN_SETUP + PS, blockIdx.x == 0 && threadIdx.x == 0);
     cs_wait_for_predecessor();
+    CS_STAMP(ws, CS_PS_SCAN_WAITED + PS, blockIdx.x == 0 && threadIdx.x == 0);
     if (H == 0xFFFFFFFFu) {                                   // every CTA sees the same word
         if (blockIdx.x == 0 && threadIdx.x == 0) ws.sel->spec = 0;
         return;
@@ -357,6 +361,7 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_fast_kernel(SelArgs a, cs_
         }
         drain(true);
         stage_flush(st, &ws.sel->c_spec, ws.cand_km, ws.cand_id);
+        CS_STAMP(ws, CS_PS_SCAN_READ + PS, blockIdx.x == 0 && threadIdx.x == 0);
         const uint32_t t0 = n_tiles * TILE;
         if (gtid < a.n - t0) {                                // ragged tail, one entry per thread, through the key
             const uint32_t i = t0 + gtid;
@@ -386,7 +391,9 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_fast_kernel(SelArgs a, cs_
         }
     }
     if (threadIdx.x == 0 && s_above) atomicAdd(&ws.sel->n_above, s_above);
+    CS_STAMP(ws, CS_PS_SCAN_FLUSHED + PS, blockIdx.x == 0 && threadIdx.x == 0);
     if (!last_cta_done(&ws.sel->ticket[0], &s_flag)) return;
+    CS_STAMP(ws, CS_PS_SCAN_LAST_CTA + PS, threadIdx.x == 0);
 
     // ---- last CTA -----------------------------------------------------------------------------------------
     // Two things are left and neither needs the other: whether the k-th smallest key lies within the remembered
@@ -464,6 +471,7 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_fast_kernel(SelArgs a, cs_
         ws.sel->n_above = 0;
         ws.sel->ticket[0] = 0;
     }
+    CS_STAMP(ws, CS_PS_SCAN_TAIL_DONE + PS, threadIdx.x == 0);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -776,24 +784,28 @@ __device__ __forceinline__ uint32_t bucket_offsets(const cs_workspace &ws, uint3
 // General case: per round a CTA takes 1024 candidates, counts them per bucket in shared memory and reserves the
 // CTA's range in each non-empty bucket with one global atomic; bucket and slot are recorded for the scatter launch.
 // ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) cs_sel_bucket_kernel(cs_workspace ws, uint32_t sort_cap)
+__global__ void __launch_bounds__(256) cs_sel_bucket_kernel(cs_workspace ws, uint32_t sort_cap, uint32_t kind)
 {
     __shared__ unsigned long long s_km[CS_MAX_SPLITTERS + 1];
     __shared__ uint32_t s_id[CS_MAX_SPLITTERS + 1];
     __shared__ uint32_t s_cnt[CS_MAX_SPLITTERS + 1], s_base[CS_MAX_SPLITTERS + 1];
     constexpr int ITEMS = 4;                                  // candidates per thread and round
+    const int PS = kind == 2 ? 8 : 0;                         // phase-stamp slots (profiling builds)
     cs_wait_for_predecessor();
+    CS_STAMP(ws, CS_PS_BUCKET_WAITED + PS, blockIdx.x == 0 && threadIdx.x == 0);
     cs_release_successor();
     // Everything the first round needs is asked for at once -- the select's state, the splitters and the round's keys
     // (addresses bounded by the capacity of the buffers; what lies beyond the live counts is ignored below) -- so that
     // the launch starts with one trip to L2 instead of three.
     unsigned long long km[ITEMS];
     uint32_t id[ITEMS], bkt[ITEMS], loc[ITEMS];
-    const uint32_t base0 = blockIdx.x * (256 * ITEMS);
+    // Item u of a round lies one grid-wide sweep (sweep = 256 keys per CTA) after item u - 1, so that few candidates
+    // spread over all CTAs with one live key per thread instead of filling a few CTAs with four.
+    const uint32_t sweep = gridDim.x * 256u, lane0 = blockIdx.x * 256u + threadIdx.x;
     const uint4 st = cs_ld_cg_pinned((const uint4 *)&ws.sel->c);          // c, n_spl, placed, cap
 #pragma unroll
     for (int u = 0; u < ITEMS; ++u) {
-        const uint32_t i = base0 + u * 256 + threadIdx.x, ii = i < sort_cap ? i : 0u;
+        const uint32_t i = u * sweep + lane0, ii = i < sort_cap ? i : 0u;
         km[u] = cs_ld_cg_pinned(ws.cand_km + ii);
         id[u] = cs_ld_cg_pinned(ws.cand_id + ii);
     }
@@ -805,11 +817,11 @@ __global__ void __launch_bounds__(256) cs_sel_bucket_kernel(cs_workspace ws, uin
     s_id[threadIdx.x] = threadIdx.x < n_spl ? my_spl_id : 0xFFFFFFFFu;
     s_cnt[threadIdx.x] = 0;
     __syncthreads();
-    for (uint32_t base = base0; base < c; base += gridDim.x * (256 * ITEMS)) {
-        if (base != base0) {
+    for (uint32_t base = 0; base < c; base += sweep * ITEMS) {
+        if (base != 0) {
 #pragma unroll
             for (int u = 0; u < ITEMS; ++u) {                 // all of the round's keys are fetched before any is used
-                const uint32_t i = base + u * 256 + threadIdx.x, ii = i < c ? i : 0u;
+                const uint32_t i = base + u * sweep + lane0, ii = i < c ? i : 0u;
                 km[u] = cs_ld_cg_pinned(ws.cand_km + ii);
                 id[u] = cs_ld_cg_pinned(ws.cand_id + ii);
             }
@@ -837,7 +849,7 @@ __global__ void __launch_bounds__(256) cs_sel_bucket_kernel(cs_workspace ws, uin
         }
 #pragma unroll
         for (int u = 0; u < ITEMS; ++u) {
-            const uint32_t i = base + u * 256 + threadIdx.x;
+            const uint32_t i = base + u * sweep + lane0;
             bkt[u] = 0xFFFFFFFFu;
             if (i < c) {
                 bkt[u] = pos[u] < n_spl ? pos[u] : n_spl;    // (a key equal to the padding stays in the last bucket)
@@ -850,7 +862,7 @@ __global__ void __launch_bounds__(256) cs_sel_bucket_kernel(cs_workspace ws, uin
                 if (bkt[u] != 0xFFFFFFFFu) loc[u] = atomicAdd(&ws.bcount[bkt[u]], 1u);
 #pragma unroll
             for (int u = 0; u < ITEMS; ++u) {
-                const uint32_t i = base + u * 256 + threadIdx.x;
+                const uint32_t i = base + u * sweep + lane0;
                 if (bkt[u] == 0xFFFFFFFFu) continue;
                 ws.cand_bkt[i] = bkt[u];
                 ws.cand_slot[i] = loc[u];
@@ -872,7 +884,7 @@ __global__ void __launch_bounds__(256) cs_sel_bucket_kernel(cs_workspace ws, uin
         __syncthreads();
 #pragma unroll
         for (int u = 0; u < ITEMS; ++u) {
-            const uint32_t i = base + u * 256 + threadIdx.x;
+            const uint32_t i = base + u * sweep + lane0;
             if (bkt[u] != 0xFFFFFFFFu) {
                 ws.cand_bkt[i] = bkt[u];
                 ws.cand_slot[i] = s_base[bkt[u]] + loc[u];
@@ -880,16 +892,20 @@ __global__ void __launch_bounds__(256) cs_sel_bucket_kernel(cs_workspace ws, uin
         }
         __syncthreads();
     }
+    CS_STAMP(ws, CS_PS_BUCKET_DONE + PS, blockIdx.x == 0 && threadIdx.x == 0);
+    (void)PS;
 }
 
 // ---------------------------------------------------------------------------------------------
 // 4 scatter (general case only: candidates of the needed buckets are grouped by bucket)
 // ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) cs_sel_scatter_kernel(cs_workspace ws)
+__global__ void __launch_bounds__(256) cs_sel_scatter_kernel(cs_workspace ws, uint32_t kind)
 {
     __shared__ uint32_t s_off[CS_MAX_SPLITTERS + 2];
     __shared__ uint32_t s_tmp[16];
     cs_wait_for_predecessor();
+    CS_STAMP(ws, CS_PS_SCATTER_WAITED + (kind == 2 ? 8 : 0), blockIdx.x == 0 && threadIdx.x == 0);
+    (void)kind;
     cs_release_successor();
     if (ws.sel->placed && !ws.sel->overflow) return;         // the buckets are in their regions already
     const uint32_t c = ws.sel->c, n_out = ws.sel->n_out;
@@ -918,6 +934,7 @@ cs_sel_rank_kernel(cs_workspace ws, uint32_t k, uint32_t kind, uint32_t *__restr
     __shared__ uint32_t s_off[CS_MAX_SPLITTERS + 2];
     __shared__ uint32_t s_tmp[16];
     cs_wait_for_predecessor();
+    CS_STAMP(ws, CS_PS_RANK_WAITED + (kind == 2 ? 8 : 0), blockIdx.x == 0 && threadIdx.x == 0);
     cs_release_successor();
     const uint32_t n_out = ws.sel->n_out, cap = ws.sel->cap;
     const bool in_regions = ws.sel->placed && !ws.sel->overflow;
@@ -954,6 +971,7 @@ cs_sel_rank_kernel(cs_workspace ws, uint32_t k, uint32_t kind, uint32_t *__restr
             }
         }
     }
+    CS_STAMP(ws, CS_PS_RANK_DONE + (kind == 2 ? 8 : 0), blockIdx.x == 0 && threadIdx.x == 0);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -1074,9 +1092,9 @@ static int launch_select_job(cs_ctx *ctx, int job, const cs_block_index *idx, ui
     if (prefetch) cs_launch_chained(cs_sel_collect_kernel<true>, grid, SEL_THREADS, sm_collect, s, a, ws);
     else cs_launch_chained(cs_sel_collect_kernel<false>, grid, SEL_THREADS, sm_collect, s, a, ws);
     if ((rc = cs_check_launch(ctx)) != CS_OK) return rc;
-    cs_launch_chained(cs_sel_bucket_kernel, grid_c, 256, 0, s, ws, (uint32_t)ctx->p.max_blocks);
+    cs_launch_chained(cs_sel_bucket_kernel, grid_c, 256, 0, s, ws, (uint32_t)ctx->p.max_blocks, a.kind);
     if ((rc = cs_check_launch(ctx)) != CS_OK) return rc;
-    cs_launch_chained(cs_sel_scatter_kernel, grid_c, 256, 0, s, ws);
+    cs_launch_chained(cs_sel_scatter_kernel, grid_c, 256, 0, s, ws, a.kind);
     if ((rc = cs_check_launch(ctx)) != CS_OK) return rc;
     cs_launch_chained(cs_sel_rank_kernel, CS_MAX_SPLITTERS + 1, 256, 0, s, ws, k, a.kind, ids_out, n_out);
     return cs_check_launch(ctx);
