@@ -1134,7 +1134,9 @@ PHASE_NAMES = {0: "refresh: entry", 1: "refresh: dependency wait over", 2: "refr
                11: "scan: index read, queues worked off (CTA 0)", 12: "scan: candidates and histogram flushed (CTA 0)",
                13: "scan: last CTA starts", 14: "scan: threshold found, splitters published",
                24: "bucket: dependency wait over (histogram and collect launches returned)", 25: "bucket: CTA 0 done",
-               26: "scatter: dependency wait over", 27: "rank: dependency wait over", 28: "rank: CTA 0 done"}
+               26: "scatter: dependency wait over", 27: "rank: dependency wait over", 28: "rank: CTA 0 done",
+               29: "bucket: state, splitters and keys arrived (CTA 0)", 30: "bucket: buckets found (CTA 0)",
+               31: "bucket: slots taken (CTA 0)"}
 
 
 def phase_timeline(args, torch, device):

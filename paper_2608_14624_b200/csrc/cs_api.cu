@@ -75,7 +75,7 @@ size_t cs_layout_workspace(const cs_params *p, uint32_t gtab_len, void *base, cs
     TAKE(sort_id, uint32_t, N);
     TAKE(spl_km, unsigned long long, CS_MAX_SPLITTERS + 1);
     TAKE(spl_id, uint32_t, CS_MAX_SPLITTERS + 1);
-    TAKE(bcount, uint32_t, CS_MAX_SPLITTERS + 1);
+    TAKE(bcount, uint32_t, (CS_MAX_SPLITTERS + 1) * CS_BCOUNT_STRIDE);
     // Private select state, histogram and candidate / sort regions for the second and third select of a step,
     // which run beside the first one.  Full size up to CS_CONCURRENT_MAX_BLOCKS entries; beyond that only the
     // single-launch cluster select (at most CS_SELECT_CLUSTER_MAX_BLOCKS entries) runs selects side by side.
@@ -95,7 +95,7 @@ size_t cs_layout_workspace(const cs_params *p, uint32_t gtab_len, void *base, cs
         TAKE(sort_id, uint32_t, Nc);
         TAKE(spl_km, unsigned long long, CS_MAX_SPLITTERS + 1);
         TAKE(spl_id, uint32_t, CS_MAX_SPLITTERS + 1);
-        TAKE(bcount, uint32_t, CS_MAX_SPLITTERS + 1);
+        TAKE(bcount, uint32_t, (CS_MAX_SPLITTERS + 1) * CS_BCOUNT_STRIDE);
             ws = all;
     }
 #undef TAKE

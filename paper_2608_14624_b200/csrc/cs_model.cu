@@ -20,7 +20,7 @@ __global__ void cs_init_kernel(cs_workspace ws, uint32_t A, uint32_t n_chains, u
     for (uint32_t i = tid; i < A; i += nth) { ws.rowsum[i] = 0; ws.qfix[i] = 0; }
     for (uint32_t i = tid; i < n_chains; i += nth) ws.cur[i] = CS_AGENT_NONE;
     for (uint32_t i = tid; i < CS_HIST_BINS; i += nth) ws.hist[i] = 0;
-    for (uint32_t i = tid; i <= CS_MAX_SPLITTERS; i += nth) ws.bcount[i] = 0;
+    for (uint32_t i = tid; i <= CS_MAX_SPLITTERS; i += nth) CS_BCOUNT(ws, i) = 0;
     for (uint32_t i = tid; i < gtab_len; i += nth) ws.gtab[i] = cs_recency(lambda, delta, i);
     if (tid == 0) {
         cs_scalars z;

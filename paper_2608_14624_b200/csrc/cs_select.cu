@@ -112,7 +112,7 @@ __device__ __forceinline__ void publish_splitters(const cs_workspace &ws, unsign
             ws.spl_km[j] = s_km[q];
             ws.spl_id[j] = s_id[q];
         }
-        ws.bcount[j] = 0;
+        CS_BCOUNT(ws, j) = 0;
     }
     if (cp.t == 0) {
         uint32_t cap = sort_cap / (n_spl + 1u);
@@ -751,7 +751,7 @@ __device__ __forceinline__ uint32_t bucket_offsets(const cs_workspace &ws, uint3
                                                    uint32_t *s_tmp)
 {
     const uint32_t t = threadIdx.x, lane = t & 31, warp = t >> 5;
-    const uint32_t mine = t <= n_spl ? __ldcg(&ws.bcount[t]) : 0u;
+    const uint32_t mine = t <= n_spl ? __ldcg(&CS_BCOUNT(ws, t)) : 0u;
     uint32_t incl = mine;
 #pragma unroll
     for (int d = 1; d < 32; d <<= 1) {
@@ -817,6 +817,7 @@ __global__ void __launch_bounds__(256) cs_sel_bucket_kernel(cs_workspace ws, uin
     s_id[threadIdx.x] = threadIdx.x < n_spl ? my_spl_id : 0xFFFFFFFFu;
     s_cnt[threadIdx.x] = 0;
     __syncthreads();
+    CS_STAMP(ws, CS_PS_BUCKET_STAGED + PS, blockIdx.x == 0 && threadIdx.x == 0);
     for (uint32_t base = 0; base < c; base += sweep * ITEMS) {
         if (base != 0) {
 #pragma unroll
@@ -856,10 +857,12 @@ __global__ void __launch_bounds__(256) cs_sel_bucket_kernel(cs_workspace ws, uin
                 if (!placed) loc[u] = atomicAdd(&s_cnt[bkt[u]], 1u);
             }
         }
+        CS_STAMP(ws, CS_PS_BUCKET_SEARCHED + PS, blockIdx.x == 0 && threadIdx.x == 0 && base == 0);
         if (placed) {
 #pragma unroll
             for (int u = 0; u < ITEMS; ++u)                   // the round's atomics are in flight together
-                if (bkt[u] != 0xFFFFFFFFu) loc[u] = atomicAdd(&ws.bcount[bkt[u]], 1u);
+                if (bkt[u] != 0xFFFFFFFFu) loc[u] = atomicAdd(&CS_BCOUNT(ws, bkt[u]), 1u);
+            CS_STAMP(ws, CS_PS_BUCKET_SLOTS + PS, blockIdx.x == 0 && threadIdx.x == 0 && base == 0 && loc[0] != 0xFFFFFFF1u);
 #pragma unroll
             for (int u = 0; u < ITEMS; ++u) {
                 const uint32_t i = base + u * sweep + lane0;
@@ -878,7 +881,7 @@ __global__ void __launch_bounds__(256) cs_sel_bucket_kernel(cs_workspace ws, uin
         __syncthreads();
         {
             const uint32_t n_b = s_cnt[threadIdx.x];
-            if (n_b) s_base[threadIdx.x] = atomicAdd(&ws.bcount[threadIdx.x], n_b);
+            if (n_b) s_base[threadIdx.x] = atomicAdd(&CS_BCOUNT(ws, threadIdx.x), n_b);
             s_cnt[threadIdx.x] = 0;
         }
         __syncthreads();
@@ -1184,7 +1187,7 @@ int cs_launch_select_step(cs_ctx *ctx, const cs_block_index *idx, uint32_t now, 
 #define CS_SO_SPLKM (CS_SO_HIST + CS_HIST_BINS * 4u)
 #define CS_SO_SPLID (CS_SO_SPLKM + CS_STATIC_ALIGN((CS_MAX_SPLITTERS + 1u) * 8u))
 #define CS_SO_BCOUNT (CS_SO_SPLID + CS_STATIC_ALIGN((CS_MAX_SPLITTERS + 1u) * 4u))
-#define CS_SO_CANDKM (CS_SO_BCOUNT + CS_STATIC_ALIGN((CS_MAX_SPLITTERS + 1u) * 4u))
+#define CS_SO_CANDKM (CS_SO_BCOUNT + CS_STATIC_ALIGN((CS_MAX_SPLITTERS + 1u) * CS_BCOUNT_STRIDE * 4u))
 #define CS_SO_SORTKM (CS_SO_CANDKM + CS_STATIC_MAX_BLOCKS * 8u)
 #define CS_SO_CANDID (CS_SO_SORTKM + CS_STATIC_MAX_BLOCKS * 8u)
 #define CS_SO_CANDBKT (CS_SO_CANDID + CS_STATIC_MAX_BLOCKS * 4u)
@@ -1205,7 +1208,7 @@ __global__ void cs_static_prepare_kernel(cs_workspace ws, uint32_t gtab_len, flo
 {
     const uint32_t tid = blockIdx.x * blockDim.x + threadIdx.x, nth = gridDim.x * blockDim.x;
     for (uint32_t i = tid; i < CS_HIST_BINS; i += nth) ws.hist[i] = 0;
-    for (uint32_t i = tid; i <= CS_MAX_SPLITTERS; i += nth) ws.bcount[i] = 0;
+    for (uint32_t i = tid; i <= CS_MAX_SPLITTERS; i += nth) CS_BCOUNT(ws, i) = 0;
     for (uint32_t i = tid; i < gtab_len; i += nth) ws.gtab[i] = cs_recency(lambda, delta, i);
     if (tid == 0) {
         cs_scalars z;

@@ -317,7 +317,7 @@ __device__ __forceinline__ void csel_body(SelArgs a, const cs_workspace &ws, uin
                 ws.spl_km[j] = S.km[q];
                 ws.spl_id[j] = S.id[q];
             }
-            ws.bcount[j] = 0;
+            CS_BCOUNT(ws, j) = 0;
         }
     }
     __threadfence();
@@ -338,14 +338,14 @@ __device__ __forceinline__ void csel_body(SelArgs a, const cs_workspace &ws, uin
             else lo = mid + 1;
         }
         ws.cand_bkt[i] = lo;
-        ws.cand_slot[i] = atomicAdd(&ws.bcount[lo], 1u);
+        ws.cand_slot[i] = atomicAdd(&CS_BCOUNT(ws, lo), 1u);
     }
     __threadfence();
     cluster.sync();
     // offsets (every CTA computes the same prefix sum), then scatter the needed buckets into bucket order
     uint32_t *s_off = S.hist;                        // reuse: [CS_MAX_SPLITTERS + 2]
     {
-        const uint32_t mine = tid <= CS_MAX_SPLITTERS ? __ldcg(&ws.bcount[tid]) : 0u;
+        const uint32_t mine = tid <= CS_MAX_SPLITTERS ? __ldcg(&CS_BCOUNT(ws, tid)) : 0u;
         uint32_t total;
         const uint32_t excl = csel_block_scan(mine, S.part, total);
         if (tid <= CS_MAX_SPLITTERS) s_off[tid] = excl;
