@@ -459,7 +459,7 @@ int cs_use_survival_table(cs_ctx *ctx, const float *fsurv);
 
 /* Implementation of the two select calls: CS_SELECT_AUTO (= the single-launch cluster kernel up
  * to 262,144 index entries, the multi-launch path above), CS_SELECT_CLUSTER, CS_SELECT_MULTI
- * (histogram / collect / bucket / scatter / rank as five grid-wide launches).  Both give the
+ * (fast pass / histogram / collect / bucket / scatter / rank as six grid-wide launches).  Both give the
  * same lists. */
 #define CS_SELECT_AUTO 0u
 #define CS_SELECT_CLUSTER 1u

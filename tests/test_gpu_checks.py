@@ -255,3 +255,12 @@ def test_clock_read_from_device_memory_when_the_kernels_run():
     with pytest.raises(cs.CacheScoutError):
         c.set_device_clock(torch.zeros(4, dtype=torch.int32))                # pageable host memory: refused
     assert c.get_status() == 0
+
+
+def test_phase_stamps_need_the_profiling_build():
+    """cs_debug_phase_stamps() belongs to builds with -DCS_PHASE_STAMPS; the ordinary library says so and stores nothing."""
+    cfg = synth.CONFIGS["tiny"]
+    c = cs.CacheScout(cs.make_params(n_agents=cfg.n_agents, n_chains=cfg.n_chains, max_blocks=64, block_tokens=cfg.block_tokens), DEV)
+    with pytest.raises(cs.CacheScoutError) as e:
+        c.phase_stamps()
+    assert e.value.code == cs.CS_ENOTIMPL
