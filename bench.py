@@ -1136,7 +1136,8 @@ PHASE_NAMES = {0: "refresh: entry", 1: "refresh: dependency wait over", 2: "refr
                24: "bucket: dependency wait over (histogram and collect launches returned)", 25: "bucket: CTA 0 done",
                26: "scatter: dependency wait over", 27: "rank: dependency wait over", 28: "rank: CTA 0 done",
                29: "bucket: state, splitters and keys arrived (CTA 0)", 30: "bucket: buckets found (CTA 0)",
-               31: "bucket: slots taken (CTA 0)"}
+               31: "bucket: slots taken (CTA 0)",
+               40: "rank: bucket offsets known (CTA 0)", 41: "rank: bucket 0 in the tile", 42: "rank: bucket 0 sorted"}
 
 
 def phase_timeline(args, torch, device):
@@ -1195,9 +1196,10 @@ def phase_timeline(args, torch, device):
     rel = (R - R[:, 0:1]) / 1000.0
     line = {"workload": "phase stamps: metadata-scale call replayed from a CUDA graph", "calls": calls,
             "event_timed_us_median": float(np.median(timed)), "fast_hits": c.counters()["fast_hits"], "phases_us_median": []}
-    for base, who in ((0, ""), (8, " [victims]"), (16, " [prefetch]"), (24, " [victims]"), (32, " [prefetch]")):
+    for base, who in ((0, ""), (8, " [victims]"), (16, " [prefetch]"), (24, " [victims]"), (32, " [prefetch]"), (40, " [victims]"),
+                      (48, " [prefetch]")):
         for k in range(8):
-            name = PHASE_NAMES.get((base if base < 16 else base - (8 if base in (16, 32) else 0)) + k)
+            name = PHASE_NAMES.get((base - 8 if base in (16, 32, 48) else base) + k)
             if name is None or R[0, base + k] == 0:
                 continue
             line["phases_us_median"].append([round(float(np.median(rel[:, base + k])), 2), name + who])

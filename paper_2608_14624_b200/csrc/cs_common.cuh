@@ -54,7 +54,9 @@ enum {
     CS_PS_SCAN_SETUP, CS_PS_SCAN_WAITED, CS_PS_SCAN_READ, CS_PS_SCAN_FLUSHED, CS_PS_SCAN_LAST_CTA, CS_PS_SCAN_TAIL_DONE,
     CS_PS_BUCKET_WAITED = 24,   // + 8 for the prefetch select: bucket waited / done, scatter waited, rank waited / done
     CS_PS_BUCKET_DONE, CS_PS_SCATTER_WAITED, CS_PS_RANK_WAITED, CS_PS_RANK_DONE, CS_PS_BUCKET_STAGED, CS_PS_BUCKET_SEARCHED,
-    CS_PS_BUCKET_SLOTS
+    CS_PS_BUCKET_SLOTS,
+    CS_PS_RANK_OFFSETS = 40,    // + 8 for the prefetch select: bucket offsets known, bucket in the tile, tile sorted (CTA 0)
+    CS_PS_RANK_LOADED, CS_PS_RANK_SORTED
 };
 #ifdef CS_PHASE_STAMPS
 #define CS_STAMP(ws, slot, cond)                                                         \

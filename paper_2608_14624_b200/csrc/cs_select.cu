@@ -952,6 +952,7 @@ cs_sel_rank_kernel(cs_workspace ws, uint32_t k, uint32_t kind, uint32_t *__restr
     }
     if (n_out == 0) return;
     const uint32_t b_last = bucket_offsets(ws, ws.sel->n_spl, n_out, s_off, s_tmp);
+    CS_STAMP(ws, CS_PS_RANK_OFFSETS + (kind == 2 ? 8 : 0), blockIdx.x == 0 && threadIdx.x == 0);
     for (uint32_t b = blockIdx.x; b <= b_last; b += gridDim.x) {
         const uint32_t beg = s_off[b], end = s_off[b + 1], m = end - beg;
         const size_t src = in_regions ? (size_t)b * cap : (size_t)beg;      // where the bucket's keys are
@@ -961,7 +962,9 @@ cs_sel_rank_kernel(cs_workspace ws, uint32_t k, uint32_t kind, uint32_t *__restr
                 t_km[i] = ws.sort_km[src + i];
                 t_id[i] = ws.sort_id[src + i];
             }
+            CS_STAMP(ws, CS_PS_RANK_LOADED + (kind == 2 ? 8 : 0), blockIdx.x == 0 && threadIdx.x == 0 && t_km[0] != 1ull);
             sort_tile(t_km, t_id, m);
+            CS_STAMP(ws, CS_PS_RANK_SORTED + (kind == 2 ? 8 : 0), blockIdx.x == 0 && threadIdx.x == 0);
             for (uint32_t i = threadIdx.x; i < m; i += blockDim.x)
                 if (beg + i < n_out) ids_out[beg + i] = t_id[i];
         } else {                                              // larger than the tile: rank straight from global memory
