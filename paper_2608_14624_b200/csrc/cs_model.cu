@@ -8,6 +8,7 @@
 #define OBS_THREADS 1024
 #define ROW_THREADS 256
 #define OBS_FUSED_MAX 256u     // events up to which a batch is applied inside the refresh launch (one per thread)
+static_assert(OBS_FUSED_MAX == ROW_THREADS, "the refresh kernel stages one event per thread");
 
 // ---------------------------------------------------------------------------------------------
 // Initial state of Algorithm 1: zero counts, no current agent; plus the recency table.
