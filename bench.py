@@ -99,6 +99,22 @@ def mem_available_bytes():
     return avail
 
 
+def clear_cuda_last_error(torch):
+    """A runtime call that fails (here: cudaHostRegister refused for lack of lockable memory) leaves its code behind as the
+    thread's "last error", and torch reads that after its next kernel launch.  cudaGetLastError() of the runtime torch
+    uses returns and clears it; where that library cannot be reached by name, one throw-away launch takes the blame."""
+    try:
+        import ctypes
+        ctypes.CDLL("libcudart.so.12").cudaGetLastError()
+    except OSError:
+        pass
+    try:
+        torch.empty(1, device="cuda").fill_(0)
+        torch.cuda.synchronize()
+    except RuntimeError:
+        pass
+
+
 class PinnedBuffer:
     """Page-locked host memory.  First choice: a pageable tensor of the exact size registered with cudaHostRegister
     (torch's own pinned allocator rounds every request up to a power of two, which would double a 117 GiB tier).
@@ -114,6 +130,7 @@ class PinnedBuffer:
             self.registered, self.how, self.nbytes = True, "cudaHostRegister", nbytes
         else:
             self.t = None
+            clear_cuda_last_error(torch)             # or the next kernel launch reports the refused registration as its own
             pow2 = 1 << (int(nbytes).bit_length() - 1)
             try:
                 self.t = torch.empty(pow2, dtype=torch.uint8, pin_memory=True)
