@@ -86,6 +86,7 @@ struct cs_scalars {
     uint32_t sel_hint[4];   // bin up to which the next select of each kind (GPU victims, host victims, prefetch)
                             // collects ahead of its own threshold, chosen from the previous call's histogram;
                             // ~0 = none; slot 3 is never written: calls that must not speculate read it
+    unsigned long long qbase;   // Eq. 2 column sums: what every column gets from the rows' zero-count entries (see qfix)
 #ifdef CS_PHASE_STAMPS
     unsigned long long stamps[CS_N_PHASE_STAMPS];   // %globaltimer at phase boundaries of the latest call (profiling builds)
 #endif
@@ -124,7 +125,8 @@ struct cs_workspace {
     float *P;             // [A*A] Eq. 3
     uint16_t *amax;       // [A]
     double *rowH;         // [A] sum_j P_ij ln P_ij
-    unsigned long long *qfix;   // [A] column sums of Eq. 2 in 2^-60 fixed point, zero between refreshes
+    unsigned long long *qfix;   // [A] column sums of Eq. 2 in 2^-60 fixed point, WITHOUT the part that is the same for every
+                                // column (sc->qbase); zero between refreshes
     uint32_t *adj;        // [A*W] Eq. 7 adjacency, one bit per edge, W = ceil(A/32)
     uint32_t *adjT;       // [2][A*W] its transpose (row v = the predecessors of v), two copies used in turn: a refresh
                           // fills one with atomics and clears the other for the refresh after it

@@ -338,6 +338,11 @@ cs_normalise_kernel(cs_workspace ws, uint32_t A, uint32_t W, float eps, float ta
         }
         const double pi_fix = (double)n_i * inv_total * 1152921504606846976.0;      // pi_i * 2^60
         const float den = __fadd_rn((float)n_i, __fmul_rn((float)A, eps));
+        // Most entries of a row have a zero count and therefore the same P = eps / den: their contribution to the
+        // column sums is one number per row, added once to a scalar instead of A times to A columns; a column with a
+        // count gets the difference on top.  Integer arithmetic, so the sums are bit for bit what A atomics per row gave.
+        const long long base_fix = __double2ll_rn(pi_fix * (double)__fdiv_rn(__fadd_rn(0.0f, eps), den));
+        if (tid == 0 && n_i) atomicAdd(&ws.sc->qbase, (unsigned long long)base_fix);
         float bestv = -1.0f;
         uint32_t besti = 0xFFFFFFFFu;
         double h = 0.0;
@@ -353,7 +358,7 @@ cs_normalise_kernel(cs_workspace ws, uint32_t A, uint32_t W, float eps, float ta
                 const double pd = (double)p;
                 h += pd * log(pd);
                 edge = p >= tau;
-                if (n_i) atomicAdd(&ws.qfix[j], (unsigned long long)__double2ll_rn(pi_fix * pd));
+                if (n_i && cij) atomicAdd(&ws.qfix[j], (unsigned long long)(__double2ll_rn(pi_fix * pd) - base_fix));
             }
             const uint32_t bits = __ballot_sync(0xFFFFFFFFu, edge);
             if ((tid & 31) == 0 && (j >> 5) < W) ws.adj[i * W + (j >> 5)] = bits;
@@ -420,16 +425,19 @@ cs_normalise_kernel(cs_workspace ws, uint32_t A, uint32_t W, float eps, float ta
     }
     if (tid < 64) s_front[tid] = (tid < 32 && !all_chains && la < A && (la >> 5) == tid) ? (1u << (la & 31)) : 0u;
     const uint32_t N = n_total;
+    const unsigned long long qbase = __ldcg(&ws.sc->qbase);
     double Hc = 0.0, Hm = 0.0;
     if (N > 0) {
         const double invN = 1.0 / (double)N;
         for (uint32_t i = tid; i < A; i += ROW_THREADS) Hc -= ((double)__ldcg(&ws.rowsum[i]) * invN) * __ldcg(&ws.rowH[i]);
         for (uint32_t j = tid; j < A; j += ROW_THREADS) {
-            const double q = (double)__ldcg(&ws.qfix[j]) * (1.0 / 1152921504606846976.0);
+            const double q = (double)(__ldcg(&ws.qfix[j]) + qbase) * (1.0 / 1152921504606846976.0);
             if (q > 0.0) Hm -= q * log(q);
         }
     }
     for (uint32_t j = tid; j < A; j += ROW_THREADS) ws.qfix[j] = 0;      // ready for the next refresh
+    __syncthreads();                                                     // (every thread has read qbase)
+    if (tid == 0) ws.sc->qbase = 0;
     cs_block_sum2(Hc, Hm, s_red);
     CS_STAMP(ws, CS_PS_REFRESH_SUMS_DONE, tid == 0);                                        // (its barriers also order s_front's zeroes)
     if (tid == 0) {
