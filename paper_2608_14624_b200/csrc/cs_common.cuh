@@ -263,6 +263,12 @@ __device__ __forceinline__ uint2 cs_ld_cg_pinned(const uint2 *p)
     asm volatile("ld.global.cg.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p) : "memory");
     return v;
 }
+__device__ __forceinline__ uint16_t cs_ld_cg_pinned(const uint16_t *p)
+{
+    uint16_t v;
+    asm volatile("ld.global.cg.u16 %0, [%1];" : "=h"(v) : "l"(p) : "memory");
+    return v;
+}
 __device__ __forceinline__ unsigned long long cs_ld_cg_pinned(const unsigned long long *p)
 {
     unsigned long long v;

@@ -406,7 +406,14 @@ cs_normalise_kernel(cs_workspace ws, uint32_t A, uint32_t W, float eps, float ta
 
     BfsRow rowT;                                                         // in flight during the sums
     cs_bfs_load_row(adjT_fill, A, W, rowT);
-    uint32_t la = __ldcg(&ws.sc->last_agent);
+    // the operands of Eq. 2 (the first ROW_THREADS of each array) travel with it, so that the sums below start on data
+    // that has arrived instead of on a trip of their own
+    const uint32_t t0_ = tid < A ? tid : 0u;
+    const uint32_t pre_rowsum = cs_ld_cg_pinned(ws.rowsum + t0_);
+    const unsigned long long pre_rowH = cs_ld_cg_pinned((const unsigned long long *)ws.rowH + t0_);
+    const unsigned long long pre_qfix = cs_ld_cg_pinned(ws.qfix + t0_);
+    const unsigned long long qbase = cs_ld_cg_pinned(&ws.sc->qbase);
+    uint32_t la = cs_ld_cg_pinned(&ws.sc->last_agent);
     if (n_events) {
         // the batch's effect on what all CTAs share (every other CTA is done reading it)
         const uint32_t a = tid < n_events ? s_eva[tid] : CS_AGENT_NONE;
@@ -424,14 +431,20 @@ cs_normalise_kernel(cs_workspace ws, uint32_t A, uint32_t W, float eps, float ta
         }
     }
     if (tid < 64) s_front[tid] = (tid < 32 && !all_chains && la < A && (la >> 5) == tid) ? (1u << (la & 31)) : 0u;
+    // Eq. 10's arg-max successor of the (now final) last agent: asked for here, used by thread 0 after the sums
+    const uint32_t a_star_pre = (tid == 0 && la < A) ? (uint32_t)cs_ld_cg_pinned(ws.amax + la) : 0xFFFFFFFFu;
     const uint32_t N = n_total;
-    const unsigned long long qbase = __ldcg(&ws.sc->qbase);
     double Hc = 0.0, Hm = 0.0;
     if (N > 0) {
         const double invN = 1.0 / (double)N;
-        for (uint32_t i = tid; i < A; i += ROW_THREADS) Hc -= ((double)__ldcg(&ws.rowsum[i]) * invN) * __ldcg(&ws.rowH[i]);
+        for (uint32_t i = tid; i < A; i += ROW_THREADS) {
+            const uint32_t rs = i == tid ? pre_rowsum : __ldcg(&ws.rowsum[i]);
+            const double rh = i == tid ? __longlong_as_double((long long)pre_rowH) : __ldcg(&ws.rowH[i]);
+            Hc -= ((double)rs * invN) * rh;
+        }
         for (uint32_t j = tid; j < A; j += ROW_THREADS) {
-            const double q = (double)(__ldcg(&ws.qfix[j]) + qbase) * (1.0 / 1152921504606846976.0);
+            const unsigned long long qf = j == tid ? pre_qfix : __ldcg(&ws.qfix[j]);
+            const double q = (double)(qf + qbase) * (1.0 / 1152921504606846976.0);
             if (q > 0.0) Hm -= q * log(q);
         }
     }
@@ -446,7 +459,7 @@ cs_normalise_kernel(cs_workspace ws, uint32_t A, uint32_t W, float eps, float ta
         const float Rf = (float)R;
         ws.sc->R = Rf;
         ws.sc->gate = (Rf >= r_min) ? 1u : 0u;
-        ws.sc->a_star = la < A ? (uint32_t)__ldcg(&ws.amax[la]) : 0xFFFFFFFFu;      // Eq. 10, for the prefetch ranking
+        ws.sc->a_star = a_star_pre;                           // Eq. 10, for the prefetch ranking
         ws.sc->adjT_cur = fill;
         ws.sc->ticket0 = 0;
     }
