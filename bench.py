@@ -1154,7 +1154,11 @@ PHASE_NAMES = {0: "refresh: entry", 1: "refresh: dependency wait over", 2: "refr
                26: "scatter: dependency wait over", 27: "rank: dependency wait over", 28: "rank: CTA 0 done",
                29: "bucket: state, splitters and keys arrived (CTA 0)", 30: "bucket: buckets found (CTA 0)",
                31: "bucket: slots taken (CTA 0)",
-               40: "rank: bucket offsets known (CTA 0)", 41: "rank: bucket 0 in the tile", 42: "rank: bucket 0 sorted"}
+               40: "rank: bucket offsets known (CTA 0)", 41: "rank: bucket 0 in the tile", 42: "rank: bucket 0 sorted",
+               56: "scan: per-call tables loaded [victims]", 57: "scan: age cuts built [victims]",
+               58: "scan: index tiles walked, whole rounds of the queue worked off (CTA 0) [victims]",
+               60: "scan: per-call tables loaded [prefetch]", 61: "scan: age cuts built [prefetch]",
+               62: "scan: index tiles walked, whole rounds of the queue worked off (CTA 0) [prefetch]"}
 
 
 def phase_timeline(args, torch, device):
@@ -1214,7 +1218,7 @@ def phase_timeline(args, torch, device):
     line = {"workload": "phase stamps: metadata-scale call replayed from a CUDA graph", "calls": calls,
             "event_timed_us_median": float(np.median(timed)), "fast_hits": c.counters()["fast_hits"], "phases_us_median": []}
     for base, who in ((0, ""), (8, " [victims]"), (16, " [prefetch]"), (24, " [victims]"), (32, " [prefetch]"), (40, " [victims]"),
-                      (48, " [prefetch]")):
+                      (48, " [prefetch]"), (56, "")):
         for k in range(8):
             name = PHASE_NAMES.get((base - 8 if base in (16, 32, 48) else base) + k)
             if name is None or R[0, base + k] == 0:

@@ -56,7 +56,9 @@ enum {
     CS_PS_BUCKET_DONE, CS_PS_SCATTER_WAITED, CS_PS_RANK_WAITED, CS_PS_RANK_DONE, CS_PS_BUCKET_STAGED, CS_PS_BUCKET_SEARCHED,
     CS_PS_BUCKET_SLOTS,
     CS_PS_RANK_OFFSETS = 40,    // + 8 for the prefetch select: bucket offsets known, bucket in the tile, tile sorted (CTA 0)
-    CS_PS_RANK_LOADED, CS_PS_RANK_SORTED
+    CS_PS_RANK_LOADED, CS_PS_RANK_SORTED,
+    CS_PS_SCAN_TABLES = 56,     // + 4 for the prefetch select: per-call tables loaded, age cuts built, index tiles walked (CTA 0)
+    CS_PS_SCAN_CUTS, CS_PS_SCAN_WALKED
 };
 #ifdef CS_PHASE_STAMPS
 #define CS_STAMP(ws, slot, cond)                                                         \

@@ -191,6 +191,7 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_fast_kernel(SelArgs a, cs_
     resolve_now(a);
     load_tables_dynamic(a, ws, T, PF && a.anchor);
     __syncthreads();
+    CS_STAMP(ws, CS_PS_SCAN_TABLES + PS / 2, blockIdx.x == 0 && threadIdx.x == 0);
     // ---- the age cuts, one per agent, for blocks of the common size ----------------------------------------
     // victims: s_cut[agent] = number of ages (0, 1, ..) that are dismissed, i.e. for which fl(f g(age)) >= X;
     // prefetch: s_cut[agent] = first age that is dismissed, i.e. fl(f g(age)) < X of the agents other than a*.
@@ -239,6 +240,7 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_fast_kernel(SelArgs a, cs_
         }
     }
     __syncthreads();
+    CS_STAMP(ws, CS_PS_SCAN_CUTS + PS / 2, blockIdx.x == 0 && threadIdx.x == 0);
     const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     uint32_t *q = queues + warp * FQ_CAP;
     uint32_t qn = 0;                                           // queued ids of this warp (same value in every lane)
@@ -359,6 +361,7 @@ __global__ void __launch_bounds__(SEL_THREADS) cs_sel_fast_kernel(SelArgs a, cs_
             __syncwarp();
             if (qn >= 32u) drain(false);
         }
+        CS_STAMP(ws, CS_PS_SCAN_WALKED + PS / 2, blockIdx.x == 0 && threadIdx.x == 0);
         drain(true);
         stage_flush(st, &ws.sel->c_spec, ws.cand_km, ws.cand_id);
         CS_STAMP(ws, CS_PS_SCAN_READ + PS, blockIdx.x == 0 && threadIdx.x == 0);
